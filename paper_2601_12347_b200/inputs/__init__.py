@@ -1,0 +1,398 @@
+"""Seeded synthetic inputs: graphs, features, weights and update streams.
+
+This module serves both the CUDA path and the CPU oracle and therefore holds none of the
+method's arithmetic: it only draws graphs, feature rows, weight matrices and batches of updates.
+Everything is a pure function of the seeds given, so both sides see identical inputs.
+
+The graphs stand in for the public datasets the paper measures on (Table 2): "sparse" has the
+vertex / edge / feature / class counts of the citation graph, "dense" those of the product graph.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+
+OP_ADD_EDGE = 0
+OP_DEL_EDGE = 1
+OP_SET_FEATURE = 2
+
+# one update record: for edge ops (u, v) = (source, sink); for a feature update u is the vertex
+# and v the index of its row in the batch's feature payload
+UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
+
+KIND_SAGE = 0      # h = act(W_self h_v + W_neigh agg_v + b)
+KIND_GRAPHCONV = 1  # h = act(W agg_v + b)            (no self term)
+KIND_GIN = 2       # h = act(W2 relu(W1 ((1+eps) h_v + agg_v) + b1) + b2)
+
+AGG_SUM = 0
+AGG_MEAN = 1
+AGG_WSUM_GCN = 2   # coefficient 1/sqrt(deg_out(u) * deg_in(v))
+
+ACT_IDENTITY = 0
+ACT_RELU = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SUBSTREAM = {"graph": 1, "features": 2, "weights": 3, "updates": 4, "warmup": 5, "perm": 6,
+              "drop": 7, "order": 8}
+
+
+def _rng(seed: int, stream: str) -> np.random.Generator:
+    return np.random.Generator(np.random.PCG64([int(seed), _SUBSTREAM[stream]]))
+
+
+# --------------------------------------------------------------------------------------------
+# native helper (R-MAT pair draws)
+# --------------------------------------------------------------------------------------------
+_lib = None
+
+
+def build_native(force: bool = False) -> str:
+    """Compile the R-MAT pair generator with gcc; returns the path of the shared object."""
+    src = os.path.join(_HERE, "rmat_gen.c")
+    out = os.path.join(_HERE, "_rmat_gen.so")
+    if force or not os.path.exists(out) or os.path.getmtime(out) < os.path.getmtime(src):
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", out, src])
+    return out
+
+
+def _native():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build_native())
+        lib.rmat_pairs.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int64, ctypes.c_int,
+                                   ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                   ctypes.c_void_p, ctypes.c_void_p]
+        lib.rmat_pairs.restype = None
+        _lib = lib
+    return _lib
+
+
+# --------------------------------------------------------------------------------------------
+# graphs
+# --------------------------------------------------------------------------------------------
+def _sorted_unique(k: np.ndarray) -> np.ndarray:
+    """Sorted distinct values (in-place sort + neighbour compare)."""
+    k.sort()
+    if k.size == 0:
+        return k
+    keep = np.empty(k.size, dtype=bool)
+    keep[0] = True
+    np.not_equal(k[1:], k[:-1], out=keep[1:])
+    return k[keep]
+
+
+def er_graph(n: int, m: int, seed: int) -> Tuple[np.ndarray, np.ndarray]:
+    """Directed G(n, M): exactly m distinct ordered pairs, no self-loops."""
+    rng = _rng(seed, "graph")
+    keys = np.empty(0, dtype=np.int64)
+    while keys.size < m:
+        need = m - keys.size
+        u = rng.integers(0, n, size=need + need // 8 + 16, dtype=np.int64)
+        v = rng.integers(0, n, size=u.size, dtype=np.int64)
+        k = (u * n + v)[u != v]
+        k = k[~np.isin(k, keys)]
+        _, first = np.unique(k, return_index=True)
+        k = k[np.sort(first)][:need]
+        keys = np.concatenate([keys, k])
+    return (keys // n).astype(np.int32), (keys % n).astype(np.int32)
+
+
+def rmat_graph(n: int, m: int, seed: int, a: float = 0.57, b: float = 0.19, c: float = 0.19
+               ) -> Tuple[np.ndarray, np.ndarray]:
+    """R-MAT graph with exactly m distinct directed edges on n vertices, no self-loops.
+
+    scale = ceil(log2 n); pairs with an endpoint >= n, self-loops and duplicates are rejected.
+    Candidates are drawn in rounds; if a round overshoots, a seeded uniformly random subset of
+    the distinct pairs is dropped.  Vertex ids are then relabelled by one seeded permutation and
+    the edge order is shuffled.
+    """
+    lib = _native()
+    scale = max(1, int(np.ceil(np.log2(n))))
+    keys = np.empty(0, dtype=np.int64)
+    drawn = 0
+    while keys.size < m:
+        need = m - keys.size
+        cnt = int(need * (1.35 if keys.size == 0 else 2.0)) + 1024
+        u = np.empty(cnt, dtype=np.int32)
+        v = np.empty(cnt, dtype=np.int32)
+        lib.rmat_pairs(ctypes.c_uint64(seed), ctypes.c_uint64(drawn), cnt, scale, a, b, c,
+                       u.ctypes.data, v.ctypes.data)
+        drawn += cnt
+        ok = (u < n) & (v < n) & (u != v)
+        k = u[ok].astype(np.int64) * n + v[ok]
+        del u, v, ok
+        k = _sorted_unique(k)
+        if keys.size:
+            k = k[~np.isin(k, keys, assume_unique=True)]
+            keys = np.union1d(keys, k)
+        else:
+            keys = k
+    if keys.size > m:
+        drop = _rng(seed, "drop").choice(keys.size, size=keys.size - m, replace=False)
+        mask = np.ones(keys.size, dtype=bool)
+        mask[drop] = False
+        keys = keys[mask]
+    perm = _rng(seed, "perm").permutation(n).astype(np.int32)
+    order = _rng(seed, "order").permutation(m)
+    src = perm[keys // n][order]
+    dst = perm[keys % n][order]
+    return np.ascontiguousarray(src, dtype=np.int32), np.ascontiguousarray(dst, dtype=np.int32)
+
+
+def features(n: int, d: int, seed: int, stream: str = "features") -> np.ndarray:
+    """n x d fp32 rows ~ N(0, 1)."""
+    return _rng(seed, stream).standard_normal((n, d), dtype=np.float32)
+
+
+# --------------------------------------------------------------------------------------------
+# models
+# --------------------------------------------------------------------------------------------
+@dataclass
+class LayerSpec:
+    kind: int
+    d_in: int
+    d_out: int
+    act: int
+    d_hidden: int = 0          # GIN only: width of the MLP's hidden layer
+    eps: float = 0.0           # GIN only
+
+
+@dataclass
+class ModelSpec:
+    agg: int
+    layers: List[LayerSpec]
+
+    @property
+    def dims(self) -> List[int]:
+        return [self.layers[0].d_in] + [l.d_out for l in self.layers]
+
+    @property
+    def self_term(self) -> bool:
+        return self.layers[0].kind != KIND_GRAPHCONV
+
+    @property
+    def src_norm(self) -> bool:
+        return self.agg == AGG_WSUM_GCN
+
+
+def sage_model(dims: List[int], agg: int = AGG_MEAN, last_act: int = ACT_IDENTITY) -> ModelSpec:
+    L = len(dims) - 1
+    return ModelSpec(agg, [LayerSpec(KIND_SAGE, dims[i], dims[i + 1],
+                                     ACT_RELU if i < L - 1 else last_act) for i in range(L)])
+
+
+def graphconv_model(dims: List[int], agg: int, last_act: int = ACT_IDENTITY) -> ModelSpec:
+    L = len(dims) - 1
+    return ModelSpec(agg, [LayerSpec(KIND_GRAPHCONV, dims[i], dims[i + 1],
+                                     ACT_RELU if i < L - 1 else last_act) for i in range(L)])
+
+
+def gin_model(d0: int, hidden: int, n_layers: int, eps: float = 0.0,
+              last_act: int = ACT_IDENTITY) -> ModelSpec:
+    dims = [d0] + [hidden] * n_layers
+    return ModelSpec(AGG_SUM, [LayerSpec(KIND_GIN, dims[i], dims[i + 1],
+                                         ACT_RELU if i < n_layers - 1 else last_act,
+                                         d_hidden=hidden, eps=eps) for i in range(n_layers)])
+
+
+def _glorot(rng: np.random.Generator, fan_in: int, fan_out: int) -> np.ndarray:
+    a = np.sqrt(6.0 / (fan_in + fan_out))
+    return rng.uniform(-a, a, size=(fan_in, fan_out)).astype(np.float32)
+
+
+def make_weights(model: ModelSpec, seed: int, zero_bias: bool = True) -> List[Dict[str, np.ndarray]]:
+    """Glorot-uniform matrices (input-major: fan_in x fan_out, row-major), one dict per layer.
+
+    SAGE: Wa = W_self, Wb = W_neigh, ba.   GraphConv: Wa, ba.   GIN: Wa (d_in x hid), ba,
+    Wb (hid x d_out), bb.  Biases are zero unless zero_bias is False (then small uniform).
+    """
+    rng = _rng(seed, "weights")
+    out = []
+    for l in model.layers:
+        def bias(n):
+            if zero_bias:
+                return np.zeros(n, dtype=np.float32)
+            return rng.uniform(-0.1, 0.1, size=n).astype(np.float32)
+        if l.kind == KIND_SAGE:
+            w = {"Wa": _glorot(rng, l.d_in, l.d_out), "Wb": _glorot(rng, l.d_in, l.d_out),
+                 "ba": bias(l.d_out)}
+        elif l.kind == KIND_GRAPHCONV:
+            w = {"Wa": _glorot(rng, l.d_in, l.d_out), "ba": bias(l.d_out)}
+        else:
+            w = {"Wa": _glorot(rng, l.d_in, l.d_hidden), "ba": bias(l.d_hidden),
+                 "Wb": _glorot(rng, l.d_hidden, l.d_out), "bb": bias(l.d_out)}
+        out.append(w)
+    return out
+
+
+# --------------------------------------------------------------------------------------------
+# update streams
+# --------------------------------------------------------------------------------------------
+class UpdateStream:
+    """Batches of edge additions, edge deletions and feature replacements.
+
+    Each update's type is drawn i.i.d. from (p_add, p_del, p_feat).  An addition is a uniform
+    ordered pair u != v that is not an edge of the current graph; a deletion is uniform over the
+    current edges; a feature update names a uniform vertex and carries a fresh N(0,1) row.  No
+    pair and no feature vertex appears twice within one batch.  The stream keeps its own record
+    of which edges exist, so it needs no feedback from whoever applies the batches.
+
+    With `hubs` given (an array of vertex ids), endpoints are restricted to hubs: additions join
+    two hubs, a deletion removes a uniform current out-edge of a uniformly drawn hub, feature
+    updates name hubs.
+    """
+
+    def __init__(self, n: int, src: np.ndarray, dst: np.ndarray, d0: int, seed: int,
+                 stream: str = "updates", mix: Tuple[float, float, float] = (0.4, 0.4, 0.2),
+                 hubs: Optional[np.ndarray] = None):
+        self.n = int(n)
+        self.d0 = int(d0)
+        self.rng = _rng(seed, stream)
+        self.mix = np.asarray(mix, dtype=np.float64)
+        self.init_keys = np.sort(src.astype(np.int64) * self.n + dst.astype(np.int64))
+        self.e0 = self.init_keys.size
+        self.touched: Dict[int, bool] = {}       # pair key -> currently an edge?
+        self.added: List[int] = []               # live edges that are not initial edges
+        self.added_pos: Dict[int, int] = {}
+        self.hubs = None if hubs is None else np.asarray(hubs, dtype=np.int64)
+        self.n_edges = self.e0
+
+    # -- membership ---------------------------------------------------------------------
+    def _in_init(self, key: int) -> bool:
+        i = int(np.searchsorted(self.init_keys, key))
+        return i < self.e0 and int(self.init_keys[i]) == key
+
+    def _present(self, key: int) -> bool:
+        t = self.touched.get(key)
+        return self._in_init(key) if t is None else t
+
+    def _set(self, key: int, present: bool) -> None:
+        was_init = self._in_init(key)
+        self.touched[key] = present
+        if not was_init:
+            if present:
+                self.added_pos[key] = len(self.added)
+                self.added.append(key)
+            else:
+                i = self.added_pos.pop(key)
+                last = self.added.pop()
+                if last != key:
+                    self.added[i] = last
+                    self.added_pos[last] = i
+        self.n_edges += 1 if present else -1
+
+    # -- draws --------------------------------------------------------------------------
+    def _draw_vertex(self) -> int:
+        if self.hubs is not None:
+            return int(self.hubs[self.rng.integers(0, self.hubs.size)])
+        return int(self.rng.integers(0, self.n))
+
+    def _draw_add(self, in_batch) -> int:
+        while True:
+            u, v = self._draw_vertex(), self._draw_vertex()
+            key = u * self.n + v
+            if u != v and key not in in_batch and not self._present(key):
+                return key
+
+    def _draw_del(self, in_batch) -> Optional[int]:
+        if self.n_edges - len(in_batch) <= 0:
+            return None
+        for _ in range(100000):
+            if self.hubs is not None:
+                u = self._draw_vertex()
+                lo = int(np.searchsorted(self.init_keys, u * self.n))
+                hi = int(np.searchsorted(self.init_keys, (u + 1) * self.n))
+                if hi == lo:
+                    continue
+                key = int(self.init_keys[self.rng.integers(lo, hi)])
+            else:
+                r = int(self.rng.integers(0, self.e0 + len(self.added)))
+                key = int(self.init_keys[r]) if r < self.e0 else self.added[r - self.e0]
+            if key not in in_batch and self._present(key):
+                return key
+        return None
+
+    def next_batch(self, b: int) -> Tuple[np.ndarray, np.ndarray]:
+        """Returns (updates[b] of UPDATE_DTYPE, feature_rows[n_feat, d0] fp32)."""
+        kinds = self.rng.choice(3, size=b, p=self.mix)
+        ups = np.zeros(b, dtype=UPDATE_DTYPE)
+        rows: List[np.ndarray] = []
+        in_batch = set()
+        feat_seen = set()
+        for i, k in enumerate(kinds):
+            if k == OP_DEL_EDGE:
+                key = self._draw_del(in_batch)
+                if key is None:
+                    k = OP_ADD_EDGE
+            if k == OP_ADD_EDGE:
+                key = self._draw_add(in_batch)
+            if k == OP_SET_FEATURE:
+                while True:
+                    v = self._draw_vertex()
+                    if v not in feat_seen:
+                        break
+                feat_seen.add(v)
+                ups[i] = (OP_SET_FEATURE, v, len(rows))
+                rows.append(self.rng.standard_normal(self.d0, dtype=np.float32))
+            else:
+                in_batch.add(key)
+                ups[i] = (k, key // self.n, key % self.n)
+        for rec in ups:
+            if rec["op"] != OP_SET_FEATURE:
+                self._set(int(rec["u"]) * self.n + int(rec["v"]), rec["op"] == OP_ADD_EDGE)
+        feat = np.stack(rows) if rows else np.zeros((0, self.d0), dtype=np.float32)
+        return ups, np.ascontiguousarray(feat, dtype=np.float32)
+
+
+def top_out_degree(n: int, src: np.ndarray, frac: float = 0.01) -> np.ndarray:
+    """Ids of the ceil(frac * n) vertices of largest out-degree (ties broken by lower id)."""
+    deg = np.bincount(src, minlength=n)
+    k = int(np.ceil(frac * n))
+    order = np.lexsort((np.arange(n), -deg))
+    return np.sort(order[:k]).astype(np.int32)
+
+
+# --------------------------------------------------------------------------------------------
+# named workloads
+# --------------------------------------------------------------------------------------------
+@dataclass
+class Workload:
+    name: str
+    n: int
+    e: int
+    graph: str                 # "er" | "rmat"
+    model: ModelSpec
+    seed: int = 0
+    batch_sizes: Tuple[int, ...] = (100,)
+    n_batches: int = 100
+    extra: dict = field(default_factory=dict)
+
+
+def workloads() -> Dict[str, Workload]:
+    n_s, e_s = 169_343, 1_166_243
+    n_d, e_d = 2_449_029, 123_718_280
+    return {
+        "tiny": Workload("tiny", 2000, 20000, "er", sage_model([32, 32, 16]), 0, (100,), 10),
+        "sparse": Workload("sparse", n_s, e_s, "rmat", sage_model([128, 256, 40]), 0,
+                           (1, 10, 100, 1000), 100),
+        "sparse-deep-gin": Workload("sparse-deep-gin", n_s, e_s, "rmat", gin_model(128, 256, 3), 0,
+                                    (100, 1000), 100),
+        "sparse-deep-gcn": Workload("sparse-deep-gcn", n_s, e_s, "rmat",
+                                    graphconv_model([128, 256, 256, 40], AGG_WSUM_GCN), 0,
+                                    (100, 1000), 100),
+        "dense-2l": Workload("dense-2l", n_d, e_d, "rmat", sage_model([100, 256, 47]), 0,
+                             (10, 100, 1000, 10000), 100),
+        "dense-3l": Workload("dense-3l", n_d, e_d, "rmat", sage_model([100, 256, 256, 47]), 0,
+                             (10, 100, 1000, 10000), 100),
+    }
+
+
+def make_graph(w: Workload) -> Tuple[np.ndarray, np.ndarray]:
+    if w.graph == "er":
+        return er_graph(w.n, w.e, w.seed)
+    return rmat_graph(w.n, w.e, w.seed)

@@ -1,0 +1,80 @@
+"""The seeded input generators: reproducible, and with the structure the workloads call for."""
+import importlib.util
+import json
+import os
+
+import numpy as np
+
+from paper_2601_12347_b200 import inputs as I
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def test_generators_match_recorded_checksums():
+    spec = importlib.util.spec_from_file_location(
+        "write_generator_checksums", os.path.join(GOLD, "write_generator_checksums.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    want = json.load(open(os.path.join(GOLD, "generator_checksums.json")))
+    assert mod.checksums() == want
+
+
+def test_graphs_are_simple_and_exact_size():
+    for name in ("tiny", "sparse"):
+        w = I.workloads()[name]
+        src, dst = I.make_graph(w)
+        assert src.size == dst.size == w.e
+        assert src.min() >= 0 and src.max() < w.n and dst.min() >= 0 and dst.max() < w.n
+        assert np.all(src != dst)
+        keys = src.astype(np.int64) * w.n + dst
+        assert np.unique(keys).size == w.e
+    # the R-MAT stand-in is skewed: many vertices without out-edges, a few very large hubs
+    deg = np.bincount(src, minlength=w.n)
+    assert (deg == 0).mean() > 0.3 and deg.max() > 1000
+
+
+def test_update_stream_mix_and_consistency():
+    w = I.workloads()["tiny"]
+    src, dst = I.make_graph(w)
+    st = I.UpdateStream(w.n, src, dst, 32, 0)
+    edges = set(zip(src.tolist(), dst.tolist()))
+    counts = np.zeros(3, dtype=np.int64)
+    for _ in range(20):
+        ups, rows = st.next_batch(100)
+        assert ups.size == 100 and rows.shape == (int((ups["op"] == I.OP_SET_FEATURE).sum()), 32)
+        seen = set()
+        for r in ups:
+            counts[r["op"]] += 1
+            if r["op"] == I.OP_SET_FEATURE:
+                assert 0 <= r["v"] < rows.shape[0]
+                continue
+            p = (int(r["u"]), int(r["v"]))
+            assert p not in seen
+            seen.add(p)
+            if r["op"] == I.OP_ADD_EDGE:
+                assert p not in edges and p[0] != p[1]
+            else:
+                assert p in edges
+        for r in ups:
+            p = (int(r["u"]), int(r["v"]))
+            if r["op"] == I.OP_ADD_EDGE:
+                edges.add(p)
+            elif r["op"] == I.OP_DEL_EDGE:
+                edges.discard(p)
+        assert len(edges) == st.n_edges
+    frac = counts / counts.sum()
+    assert abs(frac[0] - 0.4) < 0.05 and abs(frac[1] - 0.4) < 0.05 and abs(frac[2] - 0.2) < 0.05
+
+
+def test_hub_stream_only_touches_hubs():
+    w = I.workloads()["sparse"]
+    src, dst = I.make_graph(w)
+    hubs = I.top_out_degree(w.n, src)
+    assert hubs.size == int(np.ceil(0.01 * w.n))
+    st = I.UpdateStream(w.n, src, dst, 8, 0, mix=(0.1, 0.8, 0.1), hubs=hubs)
+    ups, rows = st.next_batch(200)
+    hs = set(hubs.tolist())
+    for r in ups:
+        assert int(r["u"]) in hs
+        if r["op"] == I.OP_ADD_EDGE:
+            assert int(r["v"]) in hs
