@@ -1,0 +1,191 @@
+/* ripple.h -- C ABI of the B200-native incremental GNN inference library.
+ *
+ * The library keeps, resident on one GPU, a dynamic directed graph, the vertex features H^0 and
+ * the cached per-layer embeddings H^1..H^L of an L-layer GNN with a linear aggregator, and
+ * brings them up to date after each batch of updates by incremental propagation: only the
+ * vertices of the L-hop propagation tree of the batch are touched, and the result equals full
+ * layer-wise inference on the updated graph (RIPPLE++, Sec. 3.1 and Sec. 3.3).
+ *
+ * Conventions
+ *   - Edge (u, v): u is the source, v the sink; v aggregates over its in-neighbours (Eq. 1).
+ *   - The vertex set {0..N-1} is fixed at creation.  The graph is simple and directed; a
+ *     self-loop is an ordinary edge.
+ *   - All matrices are fp32, row-major.  Device matrices returned by the library have a leading
+ *     dimension `ld` >= width (a multiple of 4 floats); columns beyond the width hold zeros.
+ *   - Pointers marked HOST must be dereferenceable by the CPU, DEVICE by the GPU the context
+ *     lives on; pointers marked HOST|DEVICE are accompanied by a `ripple_mem` flag.
+ *   - The caller owns every buffer it passes in; the library copies what it keeps.  Pointers
+ *     handed out by the library are borrowed and stay valid until the next ripple_apply_batch,
+ *     ripple_recompute_full or ripple_destroy on the same context.
+ *   - Every call returns a ripple_status; nothing aborts or traps.  After a non-zero status,
+ *     ripple_last_error() describes it.  A batch that is rejected leaves graph, features and
+ *     embeddings exactly as they were.
+ *   - A context is not thread-safe; all of its work runs on the stream given at creation and
+ *     each call returns after that stream has finished the call's work.
+ */
+#ifndef RIPPLE_H
+#define RIPPLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RIPPLE_MAX_LAYERS 8
+
+typedef struct ripple_ctx ripple_ctx;
+
+typedef enum {
+    RIPPLE_OK = 0,
+    RIPPLE_ERR_INVALID_ARG = 1,  /* null pointer, bad enum, bad dimension, unknown op code       */
+    RIPPLE_ERR_VERTEX_RANGE = 2, /* a vertex id outside [0, N) or a payload row outside range    */
+    RIPPLE_ERR_CAPACITY = 3,     /* batch larger than max_batch, or overflow edge pool exhausted  */
+    RIPPLE_ERR_OOM = 4,          /* device allocation failed                                     */
+    RIPPLE_ERR_CUDA = 5,         /* a CUDA runtime call failed                                   */
+    RIPPLE_ERR_TIMEOUT = 6       /* a bounded device-side wait gave up                           */
+} ripple_status;
+
+typedef enum { RIPPLE_MEM_HOST = 0, RIPPLE_MEM_DEVICE = 1 } ripple_mem;
+
+/* Aggregators of Table 1.  WSUM_GCN is the weighted sum with alpha_uv = 1/sqrt(deg_out(u) deg_in(v))
+ * taken from the current graph and recomputed whenever a degree changes. */
+typedef enum { RIPPLE_AGG_SUM = 0, RIPPLE_AGG_MEAN = 1, RIPPLE_AGG_WSUM_GCN = 2 } ripple_agg;
+
+/* Update functions (Eq. 2) of the model families of Sec. 6.1.1, x_v = normalised aggregate:
+ *   SAGE       h = act(Wa^T h_v + Wb^T x_v + ba)                         (self term)
+ *   GRAPHCONV  h = act(Wa^T x_v + ba)                                    (no self term)
+ *   GIN        h = act(Wb^T relu(Wa^T ((1 + eps) h_v + x_v) + ba) + bb)  (self term) */
+typedef enum { RIPPLE_LAYER_SAGE = 0, RIPPLE_LAYER_GRAPHCONV = 1, RIPPLE_LAYER_GIN = 2 } ripple_layer_kind;
+
+typedef enum { RIPPLE_ACT_IDENTITY = 0, RIPPLE_ACT_RELU = 1 } ripple_act;
+
+/* The three update types on this path (of the five of Sec. 3.1). */
+typedef enum { RIPPLE_OP_ADD_EDGE = 0, RIPPLE_OP_DEL_EDGE = 1, RIPPLE_OP_SET_FEATURE = 2 } ripple_op;
+
+/* One update.  ADD_EDGE / DEL_EDGE: edge (u, v).  SET_FEATURE: vertex u takes row `v` of the
+ * batch's feature payload. */
+typedef struct {
+    int32_t op;
+    int32_t u;
+    int32_t v;
+} ripple_update;
+
+/* Initial graph in coordinate form: num_edges distinct pairs (src[i], dst[i]), any order.
+ * src / dst: HOST|DEVICE per `mem`.  Duplicate pairs are not allowed (not checked). */
+typedef struct {
+    int64_t num_vertices;
+    int64_t num_edges;
+    const int32_t* src;
+    const int32_t* dst;
+    int32_t mem; /* ripple_mem */
+} ripple_graph;
+
+/* One layer.  Matrices are input-major: Wa[k * cols + j] multiplies input k into output j.
+ *   SAGE:      Wa = W_self (d_in x d_out), Wb = W_neigh (d_in x d_out), ba (d_out)
+ *   GRAPHCONV: Wa (d_in x d_out), ba (d_out)
+ *   GIN:       Wa (d_in x d_hidden), ba (d_hidden), Wb (d_hidden x d_out), bb (d_out)
+ * All HOST pointers; biases may be NULL (zero).  d_in of layer l must equal d_out of layer l-1. */
+typedef struct {
+    int32_t kind; /* ripple_layer_kind */
+    int32_t d_in;
+    int32_t d_hidden;
+    int32_t d_out;
+    int32_t act; /* ripple_act */
+    float eps;
+    const float* Wa;
+    const float* Wb;
+    const float* ba;
+    const float* bb;
+} ripple_layer;
+
+typedef enum { RIPPLE_SCATTER_AUTO = 0, RIPPLE_SCATTER_PUSH = 1, RIPPLE_SCATTER_PULL = 2 } ripple_scatter_mode;
+typedef enum { RIPPLE_GEMM_AUTO = 0, RIPPLE_GEMM_FP32 = 1, RIPPLE_GEMM_TF32 = 2 } ripple_gemm_mode;
+
+/* Zero-initialise for defaults. */
+typedef struct {
+    double slack;         /* spare adjacency capacity per vertex as a fraction of its degree (default 0.25) */
+    int64_t pool_edges;   /* overflow pool size per direction, in edges (default max(E/4, 1<<20))           */
+    int64_t max_batch;    /* largest n accepted by ripple_apply_batch (default 16384)                       */
+    int32_t scatter_mode; /* ripple_scatter_mode: how delta messages reach the aggregates                   */
+    int32_t gemm_mode;    /* ripple_gemm_mode: arithmetic of the affected-row layer update                  */
+    int32_t timing;       /* non-zero: record per-stage CUDA-event times into ripple_stats                  */
+    int32_t device;       /* CUDA device ordinal, or -1 for the current device                              */
+    void* stream;         /* cudaStream_t to run on (NULL: the library creates its own)                     */
+} ripple_options;
+
+typedef struct {
+    int32_t num_layers;
+    int64_t num_edges;                            /* after the last batch                                 */
+    int64_t n_ops, n_added, n_deleted;            /* last batch: ops given, net edges added / deleted     */
+    int64_t n_noop_add, n_noop_del, n_superseded; /* add-existing, delete-missing, shadowed by a later op */
+    int64_t n_feature;                            /* distinct vertices with a feature update              */
+    int64_t affected[RIPPLE_MAX_LAYERS + 1];      /* |A_l|, l = 0..L                                      */
+    int64_t senders[RIPPLE_MAX_LAYERS + 1];       /* |C_l|: vertices whose outgoing message changed       */
+    int64_t active_edges[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: edges carrying a message at hop l          */
+    int32_t scatter_pull[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: 1 if hop l gathered over in-edges          */
+    int64_t pool_used, pool_size;                 /* overflow pool, edges, out-direction                  */
+    /* CUDA-event times of the last batch in milliseconds (zero unless options.timing) */
+    float ms_total, ms_graph;
+    float ms_frontier[RIPPLE_MAX_LAYERS + 1];
+    float ms_scatter[RIPPLE_MAX_LAYERS + 1];
+    float ms_update[RIPPLE_MAX_LAYERS + 1];
+    float ms_bootstrap;                           /* last ripple_create / ripple_recompute_full           */
+    int64_t gpu_launches;                         /* kernels launched by the last call                    */
+} ripple_stats;
+
+/* Sec. 3.1 (preliminaries): the bootstrap embeddings exist before updates arrive.  Builds the
+ * device graph store from `g`, copies `features` (N x d0, HOST|DEVICE per feat_mem, row-major,
+ * leading dimension d0) and the L layers, runs full layer-wise inference (Eq. 1-2) to fill
+ * H^1..H^L and the cached aggregates, and returns the context in *out.  On failure *out = NULL;
+ * for statuses other than INVALID_ARG the text is available from ripple_last_error(NULL). */
+ripple_status ripple_create(const ripple_graph* g, const float* features, int32_t feat_mem,
+                            const ripple_layer* layers, int32_t L, int32_t agg,
+                            const ripple_options* opt, ripple_ctx** out);
+
+/* Sec. 3.1 (batched updates) and Sec. 3.3 (apply, then propagate hop by hop).  Applies ups[0..n)
+ * in order (the last operation on a pair, and the last payload of a vertex, win; adding an
+ * existing edge or deleting a missing one is counted and ignored), then propagates the changes
+ * through all L layers.  ups and feat_rows (n_rows x d0, leading dimension d0) are HOST|DEVICE
+ * per `mem`.  Returns after the embeddings are up to date.  n = 0 is valid. */
+ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update* ups, int64_t n,
+                                 const float* feat_rows, int64_t n_rows, int32_t mem);
+
+/* Sec. 3.1: updated predictions are available right after the batch.  *dev_ptr: DEVICE pointer
+ * to H^layer (N x *ld), layer in 0..L. */
+ripple_status ripple_get_embeddings(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld);
+
+/* The cached un-normalised aggregate S^layer (the persistent inbox of Sec. 3.3.2):
+ * S_v = sum over in-neighbours u of c_u h^{layer-1}_u.  DEVICE, N x *ld, layer in 1..L. */
+ripple_status ripple_get_aggregate(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld);
+
+/* Trigger-based inference (Sec. 2.2): the vertices whose H^layer the last batch recomputed --
+ * hop `layer` of the propagation tree (Sec. 3.3) -- as ascending ids.  DEVICE, layer in 0..L. */
+ripple_status ripple_get_affected(ripple_ctx* ctx, int32_t layer, const int32_t** dev_ids, int64_t* count);
+
+/* Current graph in canonical CSR over out-edges: rowptr (HOST, N + 1 entries), col (HOST,
+ * col_capacity >= number of edges, ascending within each row).  For parity checks. */
+ripple_status ripple_export_graph(ripple_ctx* ctx, int64_t* rowptr, int32_t* col, int64_t col_capacity);
+
+/* Degree arrays of the current graph: DEVICE, N entries each. */
+ripple_status ripple_get_degrees(ripple_ctx* ctx, const int32_t** deg_out, const int32_t** deg_in);
+
+/* Full layer-wise inference (Eq. 1-2) over the current graph, overwriting all cached state: the
+ * recompute-everything alternative that incremental propagation is compared against. */
+ripple_status ripple_recompute_full(ripple_ctx* ctx);
+
+/* Counters and timings of the last batch (HOST struct, filled by the call). */
+ripple_status ripple_get_stats(ripple_ctx* ctx, ripple_stats* out);
+
+/* Text of the last error on ctx (or of the last failed ripple_create if ctx is NULL). */
+const char* ripple_last_error(ripple_ctx* ctx);
+
+void ripple_destroy(ripple_ctx* ctx);
+
+/* Library version string. */
+const char* ripple_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RIPPLE_H */

@@ -1,0 +1,244 @@
+// Per-layer affected sets (the hops of the propagation tree, Sec. 3.3) and sender lists.
+//
+//   A_l = sinks(dE) U Out_new(C_{l-1}) U (self term ? A_{l-1} : {})        l = 1..L,  A_0 = F
+//   C_l = A_l U (source coefficients depend on out-degree ? sources(dE) : {})
+//
+// Membership is collected in an N-bit bitmap (duplicates vanish in the OR) and turned into an
+// ascending id list by a popcount scan; the bitmap is cleared by the same pass.  Out-lists are
+// walked edge-balanced: the concatenated out-edges of the sender list are cut into equal chunks
+// and each warp finds its rows by binary search in the degree prefix, so a hub costs what its
+// edges cost, not one long warp.
+#include "device_utils.cuh"
+#include "ripple_internal.cuh"
+
+#include <algorithm>
+
+namespace rp {
+
+constexpr int SCAN_T = 256;
+constexpr int SCAN_ITEMS = 4;
+constexpr int SCAN_TILE = SCAN_T * SCAN_ITEMS;
+
+// ---------------------------------------------------------------------------------------------
+// exclusive prefix sum of deg[list[i]] (or deg[i]) over i < n, n known only on the device
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int scan_count(const int* n_dev, int n_host) { return n_dev ? *n_dev : n_host; }
+
+__global__ void k_scan_tiles(const int32_t* __restrict__ list, const int* n_dev, int n_host,
+                             const int32_t* __restrict__ deg, int64_t* tile_sums) {
+    __shared__ int64_t scratch[33];
+    int n = scan_count(n_dev, n_host);
+    int n_tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        int64_t s = 0;
+#pragma unroll
+        for (int k = 0; k < SCAN_ITEMS; ++k) {
+            int i = t * SCAN_TILE + k * SCAN_T + threadIdx.x;
+            if (i < n) s += deg[list ? list[i] : i];
+        }
+        int64_t total;
+        block_exclusive_scan<int64_t>(s, scratch, total);
+        if (threadIdx.x == 0) tile_sums[t] = total;
+        __syncthreads();
+    }
+}
+
+__global__ void k_scan_tile_sums(const int* n_dev, int n_host, int64_t* tile_sums, int64_t* out,
+                                 unsigned long long* total_dev) {
+    __shared__ int64_t scratch[33];
+    int n = scan_count(n_dev, n_host);
+    int n_tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
+    int64_t carry = 0;
+    for (int t0 = 0; t0 < n_tiles; t0 += blockDim.x) {
+        int t = t0 + threadIdx.x;
+        int64_t x = t < n_tiles ? tile_sums[t] : 0, total;
+        int64_t ex = block_exclusive_scan<int64_t>(x, scratch, total);
+        if (t < n_tiles) tile_sums[t] = carry + ex;
+        carry += total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        out[n] = carry;
+        if (total_dev) *total_dev = (unsigned long long)carry;
+    }
+}
+
+__global__ void k_scan_write(const int32_t* __restrict__ list, const int* n_dev, int n_host,
+                             const int32_t* __restrict__ deg, const int64_t* __restrict__ tile_sums,
+                             int64_t* out) {
+    __shared__ int64_t scratch[33];
+    int n = scan_count(n_dev, n_host);
+    int n_tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        // thread owns SCAN_ITEMS consecutive items so the block scan yields their base directly
+        int i0 = t * SCAN_TILE + threadIdx.x * SCAN_ITEMS;
+        int64_t x[SCAN_ITEMS], s = 0;
+#pragma unroll
+        for (int k = 0; k < SCAN_ITEMS; ++k) {
+            int i = i0 + k;
+            x[k] = i < n ? deg[list ? list[i] : i] : 0;
+            s += x[k];
+        }
+        int64_t total;
+        int64_t base = tile_sums[t] + block_exclusive_scan<int64_t>(s, scratch, total);
+#pragma unroll
+        for (int k = 0; k < SCAN_ITEMS; ++k) {
+            int i = i0 + k;
+            if (i < n) out[i] = base;
+            base += x[k];
+        }
+        __syncthreads();
+    }
+}
+
+void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, const int32_t* deg,
+                  int64_t* out, unsigned long long* total_dev) {
+    int max_tiles = std::max(1, div_up(c->N, SCAN_TILE));
+    int grid = std::min(max_tiles, c->n_sm * 8);
+    RP_LAUNCH(c, k_scan_tiles, grid, SCAN_T, 0, list, n_dev, n_host, deg, c->tile_sums);
+    RP_LAUNCH(c, k_scan_tile_sums, 1, 1024, 0, n_dev, n_host, c->tile_sums, out, total_dev);
+    RP_LAUNCH(c, k_scan_write, grid, SCAN_T, 0, list, n_dev, n_host, deg, c->tile_sums, out);
+}
+
+// ---------------------------------------------------------------------------------------------
+// bitmap -> ascending id list (clears the bitmap)
+// ---------------------------------------------------------------------------------------------
+constexpr int CMP_T = 256;  // one word per thread
+
+__global__ void k_bitmap_tile_counts(const uint32_t* __restrict__ bitmap, int n_words, int* tile_cnt) {
+    __shared__ int scratch[33];
+    int w = blockIdx.x * CMP_T + threadIdx.x;
+    int pc = w < n_words ? __popc(bitmap[w]) : 0;
+    int total;
+    block_exclusive_scan<int>(pc, scratch, total);
+    if (threadIdx.x == 0) tile_cnt[blockIdx.x] = total;
+}
+
+__global__ void k_bitmap_compact(uint32_t* bitmap, int n_words, const int* __restrict__ tile_cnt,
+                                 int32_t* list, int* count_out, const int32_t* __restrict__ deg_in,
+                                 unsigned long long* pull_work) {
+    __shared__ int scratch[33];
+    __shared__ int tile_base;
+    __shared__ unsigned long long work;
+    // base of this tile: sum of the counts of the tiles before it
+    int part = 0;
+    for (int t = threadIdx.x; t < (int)blockIdx.x; t += CMP_T) part += tile_cnt[t];
+    int total;
+    block_exclusive_scan<int>(part, scratch, total);
+    if (threadIdx.x == 0) { tile_base = total; work = 0ull; }
+    __syncthreads();
+    int w = blockIdx.x * CMP_T + threadIdx.x;
+    uint32_t bits = w < n_words ? bitmap[w] : 0u;
+    if (bits) bitmap[w] = 0u;
+    int pc = __popc(bits);
+    int off = tile_base + block_exclusive_scan<int>(pc, scratch, total);
+    unsigned long long my_work = 0;
+    while (bits) {
+        int b = __ffs(bits) - 1;
+        bits &= bits - 1;
+        int v = (w << 5) + b;
+        list[off++] = v;
+        if (deg_in) my_work += (unsigned long long)deg_in[v];
+    }
+    if (pull_work) {
+        my_work = warp_sum(my_work);
+        if (lane_id() == 0 && my_work) atomicAdd(&work, my_work);
+        __syncthreads();
+        if (threadIdx.x == 0 && work) atomicAdd(pull_work, work);
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) *count_out = tile_base + total;
+}
+
+static void bitmap_to_list(Ctx* c, int32_t* list, int* count_dev, unsigned long long* pull_work) {
+    int tiles = div_up(c->n_words, CMP_T);
+    int* tile_cnt = reinterpret_cast<int*>(c->tile_sums);  // scan scratch is free here
+    RP_LAUNCH(c, k_bitmap_tile_counts, tiles, CMP_T, 0, c->bitmap, c->n_words, tile_cnt);
+    RP_LAUNCH(c, k_bitmap_compact, tiles, CMP_T, 0, c->bitmap, c->n_words, tile_cnt, list, count_dev,
+              pull_work ? c->side[1].deg : nullptr, pull_work);
+}
+
+// ---------------------------------------------------------------------------------------------
+// marking
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void set_bit(uint32_t* bitmap, int v) {
+    uint32_t m = 1u << (v & 31);
+    if (!(bitmap[v >> 5] & m)) atomicOr(&bitmap[v >> 5], m);
+}
+
+constexpr int WALK_CHUNK = 256;  // edges per warp work item
+
+__global__ void k_mark_frontier(Ctl* ctl, int l, int self_term, const int32_t* __restrict__ senders,
+                                const int64_t* __restrict__ coff, Side out, const Rec* __restrict__ rec,
+                                const int32_t* __restrict__ A_prev, uint32_t* bitmap) {
+    if (ctl->abort) return;
+    const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gsize = gridDim.x * blockDim.x;
+    // sinks of net edge changes are affected at every hop
+    for (int i = gtid; i < ctl->n_rec; i += gsize) set_bit(bitmap, rec[i].v);
+    if (self_term)
+        for (int i = gtid; i < ctl->nA[l - 1]; i += gsize) set_bit(bitmap, A_prev[i]);
+    // out-neighbours of the senders of the previous hop
+    const int nC = ctl->nC[l - 1];
+    if (nC == 0) return;
+    const int64_t E = coff[nC];
+    const int warp = gtid >> 5, nwarps = gsize >> 5, lane = lane_id();
+    for (int64_t e0 = (int64_t)warp * WALK_CHUNK; e0 < E; e0 += (int64_t)nwarps * WALK_CHUNK) {
+        int64_t e1 = min(e0 + WALK_CHUNK, E);
+        int i = upper_row(coff, nC, e0);
+        int64_t e = e0;
+        while (e < e1) {
+            int64_t row_end = coff[i + 1];
+            if (row_end <= e) { ++i; continue; }
+            int64_t seg_end = min(e1, row_end);
+            int64_t base = out.start[senders[i]] + (e - coff[i]);
+            for (int64_t j = lane; j < seg_end - e; j += 32) set_bit(bitmap, out.col[base + j]);
+            e = seg_end;
+            ++i;
+        }
+    }
+}
+
+void frontier_seed_features(Ctx* c, int n) {
+    (void)n;
+    bitmap_to_list(c, c->A[0], &c->ctl->nA[0], nullptr);
+}
+
+void frontier_build(Ctx* c, int l, int n) {
+    (void)n;
+    RP_LAUNCH(c, k_mark_frontier, c->n_sm * 8, 256, 0, c->ctl, l, (int)c->self_term, c->Clist[(l - 1) & 1],
+              c->coff, c->side[0], c->rec, c->A[l - 1], c->bitmap);
+    bitmap_to_list(c, c->A[l], &c->ctl->nA[l], &c->ctl->pull_work[l]);
+}
+
+// ---------------------------------------------------------------------------------------------
+// sender lists
+// ---------------------------------------------------------------------------------------------
+__global__ void k_senders_from_affected(Ctl* ctl, int l, const int32_t* __restrict__ A, int32_t* senders,
+                                        int32_t* posmap) {
+    if (ctl->abort) return;
+    int n = ctl->nA[l];
+    if (blockIdx.x == 0 && threadIdx.x == 0) ctl->nC[l] = n;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        int v = A[i];
+        senders[i] = v;
+        posmap[v] = i;
+    }
+}
+
+__global__ void k_senders_release(Ctl* ctl, int l, const int32_t* __restrict__ senders, int32_t* posmap) {
+    int n = ctl->nC[l];
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
+        posmap[senders[i]] = -1;
+}
+
+void senders_build(Ctx* c, int l, int n) {
+    int32_t* senders = c->Clist[l & 1];
+    RP_LAUNCH(c, k_senders_from_affected, c->n_sm * 4, 256, 0, c->ctl, l, c->A[l], senders, c->posmap);
+    if (c->src_norm && n > 0) extra_sender_rows(c, l, n);
+    scan_degrees(c, senders, &c->ctl->nC[l], 0, c->side[0].deg, c->coff, &c->ctl->E[l + 1]);
+}
+
+void senders_release(Ctx* c, int l) {
+    RP_LAUNCH(c, k_senders_release, c->n_sm * 4, 256, 0, c->ctl, l, c->Clist[l & 1], c->posmap);
+}
+
+}  // namespace rp

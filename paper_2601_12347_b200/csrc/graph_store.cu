@@ -1,0 +1,453 @@
+// GPU-resident dynamic graph store: both directions of the adjacency as CSR with per-vertex
+// slack, backed by an overflow pool, and the batched insert/delete kernels.
+//
+// A batch is normalised on the device ("Apply" step of Sec. 3.3): the last operation on a pair
+// wins (pair hash table + atomicMax of the op index), the winner is compared with the stored
+// row (warp-cooperative search) and becomes a net change record or a counted no-op.  Records
+// are then applied without any per-row lock and without scanning rows again:
+//   deletions  tombstone their slot; the row's last n_del slots ("tail") are read, the live
+//              ones among them are packed to the front of the tail and handed out, by ticket,
+//              to the holes in front of the tail (a many-at-once swap-with-last);
+//   additions  take slot new_deg + rank, rank from an atomic per-row counter; a row that would
+//              overflow its capacity first moves into the overflow pool with doubled capacity.
+// Nothing is mutated until the whole batch has been validated and the pool demand is known to
+// fit, so a rejected batch leaves the store untouched.
+#include "device_utils.cuh"
+#include "ripple_internal.cuh"
+
+#include <algorithm>
+#include <vector>
+
+namespace rp {
+
+// ---------------------------------------------------------------------------------------------
+// build from COO
+// ---------------------------------------------------------------------------------------------
+__global__ void k_count_degrees(const int32_t* __restrict__ src, const int32_t* __restrict__ dst,
+                                int64_t E, int N, int32_t* deg_out, int32_t* deg_in, Ctl* ctl) {
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < E;
+         e += (int64_t)gridDim.x * blockDim.x) {
+        int u = src[e], v = dst[e];
+        if ((unsigned)u >= (unsigned)N || (unsigned)v >= (unsigned)N) {
+            atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_VERTEX_RANGE);
+            continue;
+        }
+        atomicAdd(&deg_out[u], 1);
+        atomicAdd(&deg_in[v], 1);
+    }
+}
+
+__global__ void k_capacities(int N, const int32_t* __restrict__ deg, int32_t* cap, float slack) {
+    int v = blockIdx.x * blockDim.x + threadIdx.x;
+    if (v >= N) return;
+    int d = deg[v];
+    int extra = (int)ceilf((float)d * slack) + 4;
+    cap[v] = (d + extra + 3) & ~3;
+}
+
+__global__ void k_fill_rows(const int32_t* __restrict__ src, const int32_t* __restrict__ dst,
+                            int64_t E, int N, Side out, Side in) {
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < E;
+         e += (int64_t)gridDim.x * blockDim.x) {
+        int u = src[e], v = dst[e];
+        if ((unsigned)u >= (unsigned)N || (unsigned)v >= (unsigned)N) continue;
+        int p = atomicAdd(&out.cnt_add[u], 1);
+        out.col[out.start[u] + p] = v;
+        int q = atomicAdd(&in.cnt_add[v], 1);
+        in.col[in.start[v] + q] = u;
+    }
+}
+
+static cudaError_t alloc_side(Side& s, int N) {
+    cudaError_t e;
+    size_t nb = sizeof(int32_t) * (size_t)N;
+    if ((e = cudaMalloc(&s.start, sizeof(int64_t) * ((size_t)N + 1)))) return e;
+    int32_t** arrs[] = {&s.cap, &s.deg, &s.cnt_del, &s.cnt_add, &s.tick_a, &s.tick_b, &s.touch};
+    for (auto a : arrs) {
+        if ((e = cudaMalloc(a, nb))) return e;
+        if ((e = cudaMemset(*a, 0, nb))) return e;
+    }
+    return cudaSuccess;
+}
+
+cudaError_t graph_build(Ctx* c, const int32_t* src, const int32_t* dst, int64_t E, double slack,
+                        int64_t pool_edges) {
+    cudaError_t e;
+    const int N = c->N;
+    for (int s = 0; s < 2; ++s)
+        if ((e = alloc_side(c->side[s], N))) return e;
+    Side& out = c->side[0];
+    Side& in = c->side[1];
+    const int T = 256;
+    int grid_e = (int)std::min<int64_t>(std::max<int64_t>(div_up(E, T), 1), (int64_t)c->n_sm * 16);
+    if (E > 0) RP_LAUNCH(c, k_count_degrees, grid_e, T, 0, src, dst, E, N, out.deg, in.deg, c->ctl);
+    for (int s = 0; s < 2; ++s) {
+        RP_LAUNCH(c, k_capacities, div_up(N, T), T, 0, N, c->side[s].deg, c->side[s].cap, (float)slack);
+        scan_degrees(c, nullptr, nullptr, N, c->side[s].cap, c->side[s].start, &c->ctl->pool_next[s]);
+    }
+    if ((e = cudaMemcpyAsync(c->ctl_host, c->ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, c->stream))) return e;
+    if ((e = cudaStreamSynchronize(c->stream))) return e;
+    if (c->ctl_host->err) return cudaSuccess;  // caller inspects ctl_host->err
+    for (int s = 0; s < 2; ++s) {
+        Side& sd = c->side[s];
+        sd.base_end = (int64_t)c->ctl_host->pool_next[s];
+        sd.col_size = sd.base_end + pool_edges;
+        if ((e = cudaMalloc(&sd.col, sizeof(int32_t) * (size_t)std::max<int64_t>(sd.col_size, 4)))) return e;
+    }
+    if (E > 0) RP_LAUNCH(c, k_fill_rows, grid_e, T, 0, src, dst, E, N, out, in);
+    for (int s = 0; s < 2; ++s)
+        if ((e = cudaMemsetAsync(c->side[s].cnt_add, 0, sizeof(int32_t) * (size_t)N, c->stream))) return e;
+    return cudaStreamSynchronize(c->stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// batch normalisation
+// ---------------------------------------------------------------------------------------------
+__global__ void k_classify(const ripple_update* __restrict__ ups, int n, int n_rows, int N, Ctl* ctl,
+                           unsigned long long* hkeys, int32_t* hseq, int hmask, int32_t* op_slot,
+                           int32_t* feat_last) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    ripple_update op = ups[i];
+    op_slot[i] = -1;
+    if (op.op < 0 || op.op > 2) {
+        atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_INVALID_ARG);
+        ctl->abort = 1;
+        return;
+    }
+    bool bad = (unsigned)op.u >= (unsigned)N;
+    if (op.op == RIPPLE_OP_SET_FEATURE) bad |= (unsigned)op.v >= (unsigned)n_rows;
+    else bad |= (unsigned)op.v >= (unsigned)N;
+    if (bad) {
+        atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_VERTEX_RANGE);
+        ctl->abort = 1;
+        return;
+    }
+    if (op.op == RIPPLE_OP_SET_FEATURE) {
+        atomicMax(&feat_last[op.u], i);
+        return;
+    }
+    unsigned long long key = (unsigned long long)op.u * (unsigned long long)N + (unsigned long long)op.v + 1ull;
+    int h = (int)(mix64(key) & (unsigned long long)hmask);
+    for (int probe = 0; probe <= hmask; ++probe) {
+        unsigned long long prev = atomicCAS(&hkeys[h], 0ull, key);
+        if (prev == 0ull || prev == key) {
+            atomicMax(&hseq[h], i);
+            op_slot[i] = h;
+            return;
+        }
+        h = (h + 1) & hmask;
+    }
+    atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_CAPACITY);  // table full: cannot happen with hsize >= 2 max_batch
+    ctl->abort = 1;
+}
+
+// position of x in row [base, base + deg), or -1; the whole warp calls this
+__device__ __forceinline__ int warp_find(const int32_t* __restrict__ col, int64_t base, int deg, int x) {
+    int found = -1;
+    for (int j0 = 0; j0 < deg; j0 += 32) {
+        int j = j0 + lane_id();
+        bool hit = j < deg && col[base + j] == x;
+        unsigned m = __ballot_sync(FULL, hit);
+        if (m) { found = j0 + __ffs(m) - 1; break; }
+    }
+    return found;
+}
+
+// One warp per op: winners are compared with the stored graph and become records or no-ops.
+__global__ void k_resolve(const ripple_update* __restrict__ ups, int n, Ctl* ctl,
+                          const int32_t* __restrict__ hseq, const int32_t* __restrict__ op_slot,
+                          const int32_t* __restrict__ feat_last, Side out, Side in, Rec* rec,
+                          uint32_t* bitmap) {
+    if (ctl->abort) return;
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (int i = warp; i < n; i += nwarps) {
+        ripple_update op = ups[i];
+        if (op.op == RIPPLE_OP_SET_FEATURE) {
+            if (lane_id() == 0 && feat_last[op.u] == i) {
+                atomicAdd(&ctl->n_feat, 1);
+                atomicOr(&bitmap[op.u >> 5], 1u << (op.u & 31));
+            }
+            continue;
+        }
+        if (hseq[op_slot[i]] != i) {
+            if (lane_id() == 0) atomicAdd(&ctl->n_superseded, 1);
+            continue;
+        }
+        int j_out = warp_find(out.col, out.start[op.u], out.deg[op.u], op.v);
+        bool is_add = op.op == RIPPLE_OP_ADD_EDGE;
+        if (is_add == (j_out >= 0)) {
+            if (lane_id() == 0) atomicAdd(is_add ? &ctl->n_noop_add : &ctl->n_noop_del, 1);
+            continue;
+        }
+        int j_in = -1;
+        if (!is_add) j_in = warp_find(in.col, in.start[op.v], in.deg[op.v], op.u);
+        if (lane_id() == 0) {
+            int r = atomicAdd(&ctl->n_rec, 1);
+            atomicAdd(is_add ? &ctl->n_add : &ctl->n_del, 1);
+            Rec x;
+            x.u = op.u; x.v = op.v; x.sign = is_add ? 1 : -1;
+            x.pos[0] = j_out; x.pos[1] = j_in;
+            x.tail_val[0] = x.tail_val[1] = RP_TOMB;
+            x.deg_out_old = out.deg[op.u];
+            x.rep[0] = atomicAdd(&out.touch[op.u], 1) == 0;
+            x.rep[1] = atomicAdd(&in.touch[op.v], 1) == 0;
+            x.rank[0] = atomicAdd(is_add ? &out.cnt_add[op.u] : &out.cnt_del[op.u], 1);
+            x.rank[1] = atomicAdd(is_add ? &in.cnt_add[op.v] : &in.cnt_del[op.v], 1);
+            rec[r] = x;
+        }
+    }
+}
+
+__device__ __forceinline__ int grown_capacity(int cap, int need) {
+    int want = max(2 * cap, need + (need >> 2) + 4);
+    return (want + 3) & ~3;
+}
+
+// Rows whose additions do not fit: list them and add up the pool entries they will take.
+__global__ void k_plan_growth(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
+                              int32_t* grow_out, int32_t* grow_in) {
+    if (ctl->abort) return;
+    int n = ctl->n_rec;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * n; i += gridDim.x * blockDim.x) {
+        int s = i & 1;
+        const Rec& x = rec[i >> 1];
+        if (x.sign < 0 || x.rank[s] != 0) continue;
+        const Side& sd = s ? in : out;
+        int row = s ? x.v : x.u;
+        int need = sd.deg[row] - sd.cnt_del[row] + sd.cnt_add[row];
+        if (need > sd.cap[row]) {
+            int g = atomicAdd(&ctl->n_grow[s], 1);
+            (s ? grow_in : grow_out)[g] = row;
+            atomicAdd(&ctl->pool_need[s], (unsigned long long)grown_capacity(sd.cap[row], need));
+        }
+    }
+}
+
+__global__ void k_plan_check(Ctl* ctl, long long col_size_out, long long col_size_in) {
+    if (ctl->abort) return;
+    if (ctl->pool_next[0] + ctl->pool_need[0] > (unsigned long long)col_size_out ||
+        ctl->pool_next[1] + ctl->pool_need[1] > (unsigned long long)col_size_in) {
+        ctl->err = (int)RIPPLE_ERR_CAPACITY;
+        ctl->abort = 1;
+    }
+}
+
+void graph_batch_classify(Ctx* c, int n, int n_rows) {
+    if (n <= 0) return;
+    const int T = 256;
+    RP_LAUNCH(c, k_classify, div_up(n, T), T, 0, c->ups_dev, n, n_rows, c->N, c->ctl, c->hkeys, c->hseq,
+              c->hsize - 1, c->op_slot, c->feat_last);
+    int warps_per_block = T / 32;
+    int grid = std::min(div_up(n, warps_per_block), c->n_sm * 8);
+    RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, n, c->ctl, c->hseq, c->op_slot, c->feat_last,
+              c->side[0], c->side[1], c->rec, c->bitmap);
+    RP_LAUNCH(c, k_plan_growth, std::min(div_up(2 * n, T), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[0],
+              c->side[1], c->grow_list[0], c->grow_list[1]);
+    RP_LAUNCH(c, k_plan_check, 1, 1, 0, c->ctl, (long long)c->side[0].col_size, (long long)c->side[1].col_size);
+}
+
+// ---------------------------------------------------------------------------------------------
+// mutation
+// ---------------------------------------------------------------------------------------------
+#define FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row)                                                  \
+    int n_ = (ctl)->n_rec;                                                                        \
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * n_; i += gridDim.x * blockDim.x)
+
+__global__ void k_del_mark(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
+    if (ctl->abort) return;
+    FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
+        int s = i & 1;
+        const Rec& x = rec[i >> 1];
+        if (x.sign > 0) continue;
+        const Side& sd = s ? in : out;
+        int row = s ? x.v : x.u;
+        sd.col[sd.start[row] + x.pos[s]] = RP_TOMB;
+    }
+}
+
+__global__ void k_del_tail_read(Ctl* ctl, Rec* rec, Side out, Side in) {
+    if (ctl->abort) return;
+    FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
+        int s = i & 1;
+        Rec& x = rec[i >> 1];
+        if (x.sign > 0) continue;
+        const Side& sd = s ? in : out;
+        int row = s ? x.v : x.u;
+        int new_deg = sd.deg[row] - sd.cnt_del[row];
+        x.tail_val[s] = sd.col[sd.start[row] + new_deg + x.rank[s]];
+    }
+}
+
+__global__ void k_del_tail_pack(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
+    if (ctl->abort) return;
+    FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
+        int s = i & 1;
+        const Rec& x = rec[i >> 1];
+        if (x.sign > 0 || x.tail_val[s] == RP_TOMB) continue;
+        const Side& sd = s ? in : out;
+        int row = s ? x.v : x.u;
+        int new_deg = sd.deg[row] - sd.cnt_del[row];
+        int t = atomicAdd(&sd.tick_a[row], 1);
+        sd.col[sd.start[row] + new_deg + t] = x.tail_val[s];
+    }
+}
+
+__global__ void k_del_fill(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
+    if (ctl->abort) return;
+    FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
+        int s = i & 1;
+        const Rec& x = rec[i >> 1];
+        if (x.sign > 0) continue;
+        const Side& sd = s ? in : out;
+        int row = s ? x.v : x.u;
+        int new_deg = sd.deg[row] - sd.cnt_del[row];
+        if (x.pos[s] >= new_deg) continue;
+        int t = atomicAdd(&sd.tick_b[row], 1);
+        sd.col[sd.start[row] + x.pos[s]] = sd.col[sd.start[row] + new_deg + t];
+    }
+}
+
+// One warp per growing row: take a block from the pool, move the row, double its capacity.
+__global__ void k_grow_rows(Ctl* ctl, Side out, Side in, const int32_t* __restrict__ grow_out,
+                            const int32_t* __restrict__ grow_in) {
+    if (ctl->abort) return;
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int nwarps = (gridDim.x * blockDim.x) >> 5;
+    int n0 = ctl->n_grow[0], n1 = ctl->n_grow[1];
+    for (int g = warp; g < n0 + n1; g += nwarps) {
+        int s = g >= n0;
+        Side& sd = s ? in : out;
+        int row = s ? grow_in[g - n0] : grow_out[g];
+        int live = sd.deg[row] - sd.cnt_del[row];
+        int need = live + sd.cnt_add[row];
+        int ncap = grown_capacity(sd.cap[row], need);
+        unsigned long long off = 0;
+        if (lane_id() == 0) off = atomicAdd(&ctl->pool_next[s], (unsigned long long)ncap);
+        off = __shfl_sync(FULL, off, 0);
+        int64_t old = sd.start[row];
+        for (int j = lane_id(); j < live; j += 32) sd.col[off + j] = sd.col[old + j];
+        __syncwarp();
+        if (lane_id() == 0) { sd.start[row] = (int64_t)off; sd.cap[row] = ncap; }
+    }
+}
+
+__global__ void k_add_write(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
+    if (ctl->abort) return;
+    FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
+        int s = i & 1;
+        const Rec& x = rec[i >> 1];
+        if (x.sign < 0) continue;
+        const Side& sd = s ? in : out;
+        int row = s ? x.v : x.u;
+        int live = sd.deg[row] - sd.cnt_del[row];
+        sd.col[sd.start[row] + live + x.rank[s]] = s ? x.u : x.v;
+    }
+}
+
+__global__ void k_commit_degrees(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
+                                 int32_t* deg_out_old) {
+    if (ctl->abort) return;
+    FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
+        int s = i & 1;
+        const Rec& x = rec[i >> 1];
+        if (!x.rep[s]) continue;
+        const Side& sd = s ? in : out;
+        int row = s ? x.v : x.u;
+        sd.deg[row] = sd.deg[row] - sd.cnt_del[row] + sd.cnt_add[row];
+        if (s == 0) deg_out_old[row] = x.deg_out_old;
+    }
+}
+
+void graph_batch_mutate(Ctx* c, int n) {
+    if (n <= 0) return;
+    const int T = 256;
+    int grid = std::min(div_up(2 * n, T), c->n_sm * 8);
+    Side& o = c->side[0];
+    Side& i = c->side[1];
+    RP_LAUNCH(c, k_del_mark, grid, T, 0, c->ctl, c->rec, o, i);
+    RP_LAUNCH(c, k_del_tail_read, grid, T, 0, c->ctl, c->rec, o, i);
+    RP_LAUNCH(c, k_del_tail_pack, grid, T, 0, c->ctl, c->rec, o, i);
+    RP_LAUNCH(c, k_del_fill, grid, T, 0, c->ctl, c->rec, o, i);
+    RP_LAUNCH(c, k_grow_rows, std::min(div_up(2 * n, T / 32), c->n_sm * 8), T, 0, c->ctl, o, i,
+              c->grow_list[0], c->grow_list[1]);
+    RP_LAUNCH(c, k_add_write, grid, T, 0, c->ctl, c->rec, o, i);
+    RP_LAUNCH(c, k_commit_degrees, grid, T, 0, c->ctl, c->rec, o, i, c->deg_out_old);
+}
+
+// ---------------------------------------------------------------------------------------------
+// per-batch scratch back to its resting state (runs for rejected batches too)
+// ---------------------------------------------------------------------------------------------
+__global__ void k_cleanup(const ripple_update* __restrict__ ups, int n, int N, Ctl* ctl,
+                          const Rec* __restrict__ rec, Side out, Side in, unsigned long long* hkeys,
+                          int32_t* hseq, const int32_t* __restrict__ op_slot, int32_t* feat_last,
+                          int32_t* deg_out_old, uint32_t* bitmap) {
+    int n_rec = ctl->n_rec;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        ripple_update op = ups[i];
+        int slot = op_slot[i];
+        if (slot >= 0) { hkeys[slot] = 0ull; hseq[slot] = -1; }
+        if (op.op == RIPPLE_OP_SET_FEATURE && (unsigned)op.u < (unsigned)N) {
+            feat_last[op.u] = -1;
+            if (ctl->abort) atomicAnd(&bitmap[op.u >> 5], ~(1u << (op.u & 31)));
+        }
+        if (i < n_rec) {
+            const Rec& x = rec[i];
+            out.cnt_del[x.u] = 0; out.cnt_add[x.u] = 0; out.tick_a[x.u] = 0; out.tick_b[x.u] = 0; out.touch[x.u] = 0;
+            in.cnt_del[x.v] = 0; in.cnt_add[x.v] = 0; in.tick_a[x.v] = 0; in.tick_b[x.v] = 0; in.touch[x.v] = 0;
+            deg_out_old[x.u] = -1;
+        }
+    }
+}
+
+void graph_batch_cleanup(Ctx* c, int n) {
+    if (n <= 0) return;
+    const int T = 256;
+    RP_LAUNCH(c, k_cleanup, std::min(div_up(n, T), c->n_sm * 8), T, 0, c->ups_dev, n, c->N, c->ctl, c->rec,
+              c->side[0], c->side[1], c->hkeys, c->hseq, c->op_slot, c->feat_last, c->deg_out_old, c->bitmap);
+}
+
+// ---------------------------------------------------------------------------------------------
+// canonical export (parity checks)
+// ---------------------------------------------------------------------------------------------
+__global__ void k_export_rows(int N, Side out, const int64_t* __restrict__ rowptr, int32_t* col) {
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (int v = warp; v < N; v += nwarps) {
+        int64_t base = out.start[v], dst = rowptr[v];
+        int deg = out.deg[v];
+        for (int j = lane_id(); j < deg; j += 32) col[dst + j] = out.col[base + j];
+    }
+}
+
+cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, int64_t col_capacity, int64_t* n_edges) {
+    cudaError_t e;
+    const int N = c->N;
+    std::vector<int32_t> deg((size_t)N);
+    if ((e = cudaMemcpyAsync(deg.data(), c->side[0].deg, sizeof(int32_t) * (size_t)N, cudaMemcpyDeviceToHost, c->stream))) return e;
+    if ((e = cudaStreamSynchronize(c->stream))) return e;
+    rowptr[0] = 0;
+    for (int v = 0; v < N; ++v) rowptr[v + 1] = rowptr[v] + deg[v];
+    *n_edges = rowptr[N];
+    if (rowptr[N] > col_capacity) return cudaErrorInvalidValue;
+    if (rowptr[N] == 0) return cudaSuccess;
+    int64_t* rp_dev = nullptr;
+    int32_t* col_dev = nullptr;
+    if ((e = cudaMalloc(&rp_dev, sizeof(int64_t) * ((size_t)N + 1)))) return e;
+    if ((e = cudaMalloc(&col_dev, sizeof(int32_t) * (size_t)rowptr[N]))) { cudaFree(rp_dev); return e; }
+    e = cudaMemcpyAsync(rp_dev, rowptr, sizeof(int64_t) * ((size_t)N + 1), cudaMemcpyHostToDevice, c->stream);
+    if (!e) {
+        RP_LAUNCH(c, k_export_rows, c->n_sm * 8, 256, 0, N, c->side[0], rp_dev, col_dev);
+        e = cudaMemcpyAsync(col, col_dev, sizeof(int32_t) * (size_t)rowptr[N], cudaMemcpyDeviceToHost, c->stream);
+    }
+    if (!e) e = cudaStreamSynchronize(c->stream);
+    cudaFree(rp_dev);
+    cudaFree(col_dev);
+    if (e) return e;
+#pragma omp parallel for schedule(dynamic, 1024)
+    for (int v = 0; v < N; ++v) std::sort(col + rowptr[v], col + rowptr[v + 1]);
+    return cudaSuccess;
+}
+
+}  // namespace rp

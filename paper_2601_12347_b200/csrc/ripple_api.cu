@@ -1,0 +1,435 @@
+// C ABI of the ripple library: argument checks, device state set-up, and the per-batch launch
+// chain.  See include/ripple.h for the contract of every entry point.
+#include "ripple_internal.cuh"
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace rp;
+
+static thread_local char g_create_err[512] = "";
+
+static void set_err(Ctx* c, const char* fmt, ...) {
+    char* dst = c ? c->err : g_create_err;
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(dst, 512, fmt, ap);
+    va_end(ap);
+}
+
+#define CK(call)                                                                              \
+    do {                                                                                      \
+        cudaError_t e_ = (call);                                                              \
+        if (e_ != cudaSuccess) {                                                              \
+            set_err(c, "%s failed: %s", #call, cudaGetErrorString(e_));                       \
+            st = e_ == cudaErrorMemoryAllocation ? RIPPLE_ERR_OOM : RIPPLE_ERR_CUDA;          \
+            goto fail;                                                                        \
+        }                                                                                     \
+    } while (0)
+
+template <typename T>
+static cudaError_t dev_alloc(T** p, size_t count, int fill_byte = -2) {
+    cudaError_t e = cudaMalloc(p, sizeof(T) * std::max<size_t>(count, 1));
+    if (e) return e;
+    if (fill_byte != -2) e = cudaMemset(*p, fill_byte, sizeof(T) * std::max<size_t>(count, 1));
+    return e;
+}
+
+__global__ void k_ctl_reset(Ctl* ctl, int n_ops) {
+    unsigned long long keep0 = ctl->pool_next[0], keep1 = ctl->pool_next[1];
+    Ctl z;
+    memset(&z, 0, sizeof(Ctl));
+    z.pool_next[0] = keep0;
+    z.pool_next[1] = keep1;
+    z.n_ops = n_ops;
+    *ctl = z;
+}
+
+static void destroy_ctx(Ctx* c) {
+    if (!c) return;
+    cudaSetDevice(c->device);
+    if (c->stream) cudaStreamSynchronize(c->stream);
+    for (int s = 0; s < 2; ++s) {
+        Side& sd = c->side[s];
+        cudaFree(sd.col); cudaFree(sd.start); cudaFree(sd.cap); cudaFree(sd.deg);
+        cudaFree(sd.cnt_del); cudaFree(sd.cnt_add); cudaFree(sd.tick_a); cudaFree(sd.tick_b); cudaFree(sd.touch);
+        cudaFree(c->grow_list[s]); cudaFree(c->D[s]); cudaFree(c->Clist[s]);
+    }
+    for (int l = 0; l <= RP_MAXL; ++l) {
+        cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->A[l]);
+        cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
+    }
+    cudaFree(c->T); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->posmap); cudaFree(c->deg_out_old);
+    cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hseq);
+    cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
+    if (c->ctl_host) cudaFreeHost(c->ctl_host);
+    for (auto& e : c->ev) if (e) cudaEventDestroy(e);
+    if (c->own_stream && c->stream) cudaStreamDestroy(c->stream);
+    delete c;
+}
+
+static ripple_status sync_and_fetch_ctl(Ctx* c) {
+    cudaError_t e = cudaMemcpyAsync(c->ctl_host, c->ctl, sizeof(Ctl), cudaMemcpyDeviceToHost, c->stream);
+    if (!e) e = cudaStreamSynchronize(c->stream);
+    if (!e) e = cudaGetLastError();
+    if (e) {
+        set_err(c, "CUDA error while running the batch: %s", cudaGetErrorString(e));
+        return RIPPLE_ERR_CUDA;
+    }
+    return RIPPLE_OK;
+}
+
+// full layer-wise inference over the current graph (Eq. 1-2): bootstrap and recompute-all
+static ripple_status run_full(Ctx* c) {
+    c->launches = 0;
+    RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, 0);
+    if (c->timing) cudaEventRecord(c->ev[0], c->stream);
+    for (int l = 1; l <= c->L; ++l) {
+        spmm_full(c, l);
+        update_rows(c, l, true);
+    }
+    if (c->timing) cudaEventRecord(c->ev[1], c->stream);
+    ripple_status st = sync_and_fetch_ctl(c);
+    if (st) return st;
+    if (c->timing) cudaEventElapsedTime(&c->stats.ms_bootstrap, c->ev[0], c->ev[1]);
+    c->stats.gpu_launches = c->launches;
+    return RIPPLE_OK;
+}
+
+static std::vector<float> padded_matrix(const float* src, int rows, int cols, int rows_p, int cols_p) {
+    std::vector<float> m((size_t)rows_p * cols_p, 0.f);
+    if (src)
+        for (int r = 0; r < rows; ++r) memcpy(&m[(size_t)r * cols_p], src + (size_t)r * cols, sizeof(float) * cols);
+    return m;
+}
+
+extern "C" ripple_status ripple_create(const ripple_graph* g, const float* features, int32_t feat_mem,
+                                       const ripple_layer* layers, int32_t L, int32_t agg,
+                                       const ripple_options* opt, ripple_ctx** out) {
+    Ctx* c = nullptr;
+    ripple_status st = RIPPLE_ERR_INVALID_ARG;
+    if (out) *out = nullptr;
+    g_create_err[0] = 0;
+    if (!g || !features || !layers || !out) { set_err(nullptr, "null argument"); return st; }
+    if (L < 1 || L > RP_MAXL) { set_err(nullptr, "L must be in 1..%d", RP_MAXL); return st; }
+    if (agg < 0 || agg > 2) { set_err(nullptr, "unknown aggregator %d", agg); return st; }
+    if (g->num_vertices < 1 || g->num_vertices > 0x7fffffff - 64 || g->num_edges < 0 ||
+        (g->num_edges > 0 && (!g->src || !g->dst))) {
+        set_err(nullptr, "bad graph description");
+        return st;
+    }
+    for (int l = 0; l < L; ++l) {
+        const ripple_layer& y = layers[l];
+        bool ok = y.kind >= 0 && y.kind <= 2 && y.d_in >= 1 && y.d_out >= 1 && y.d_in <= 1024 && y.d_out <= 1024 &&
+                  (y.act == 0 || y.act == 1) && y.Wa && y.kind == layers[0].kind;
+        if (y.kind == RIPPLE_LAYER_SAGE) ok = ok && y.Wb;
+        if (y.kind == RIPPLE_LAYER_GIN) ok = ok && y.Wb && y.d_hidden >= 1 && y.d_hidden <= 1024;
+        if (l > 0) ok = ok && y.d_in == layers[l - 1].d_out;
+        if (!ok) { set_err(nullptr, "bad description of layer %d", l + 1); return st; }
+    }
+    {
+        ripple_options o{};
+        if (opt) o = *opt;
+        if (o.slack <= 0) o.slack = 0.25;
+        if (o.max_batch <= 0) o.max_batch = 16384;
+        if (o.pool_edges <= 0) o.pool_edges = std::max<int64_t>(g->num_edges / 4, 1 << 20);
+        o.pool_edges = std::max<int64_t>(o.pool_edges, 4);
+        c = new (std::nothrow) Ctx();
+        if (!c) { set_err(nullptr, "host allocation failed"); return RIPPLE_ERR_OOM; }
+        memset(static_cast<void*>(c), 0, sizeof(Ctx));
+        int32_t *src_dev = nullptr, *dst_dev = nullptr;
+        bool own_coo = false;
+        const int N = (int)g->num_vertices;
+        const int64_t E = g->num_edges;
+        int max_ld = 0, max_hid = 0;
+
+        if (o.device >= 0) CK(cudaSetDevice(o.device));
+        CK(cudaGetDevice(&c->device));
+        CK(cudaDeviceGetAttribute(&c->n_sm, cudaDevAttrMultiProcessorCount, c->device));
+        if (o.stream) c->stream = (cudaStream_t)o.stream;
+        else { CK(cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking)); c->own_stream = true; }
+        c->N = N; c->L = L; c->agg = agg; c->E0 = E;
+        c->max_batch = o.max_batch;
+        c->scatter_mode = o.scatter_mode; c->gemm_mode = o.gemm_mode; c->timing = o.timing;
+        c->self_term = layers[0].kind != RIPPLE_LAYER_GRAPHCONV;
+        c->src_norm = agg == RIPPLE_AGG_WSUM_GCN;
+        CK(dev_alloc(&c->ctl, 1, 0));
+        CK(cudaMallocHost(&c->ctl_host, sizeof(Ctl)));
+        memset(c->ctl_host, 0, sizeof(Ctl));
+        c->n_words = (N + 31) / 32;
+        c->n_tile_sums = std::max(div_up(N, 1024) + 2, div_up(c->n_words, 256) + 2);
+        CK(dev_alloc(&c->tile_sums, (size_t)c->n_tile_sums, 0));
+        for (auto& e : c->ev) CK(cudaEventCreate(&e));
+
+        // graph
+        if (E > 0 && g->mem == RIPPLE_MEM_HOST) {
+            own_coo = true;
+            CK(dev_alloc(&src_dev, (size_t)E));
+            CK(dev_alloc(&dst_dev, (size_t)E));
+            CK(cudaMemcpyAsync(src_dev, g->src, sizeof(int32_t) * (size_t)E, cudaMemcpyHostToDevice, c->stream));
+            CK(cudaMemcpyAsync(dst_dev, g->dst, sizeof(int32_t) * (size_t)E, cudaMemcpyHostToDevice, c->stream));
+        } else {
+            src_dev = const_cast<int32_t*>(g->src);
+            dst_dev = const_cast<int32_t*>(g->dst);
+        }
+        {
+            cudaError_t e = graph_build(c, src_dev, dst_dev, E, o.slack, o.pool_edges);
+            if (own_coo) { cudaFree(src_dev); cudaFree(dst_dev); }
+            CK(e);
+            if (c->ctl_host->err) {
+                set_err(nullptr, "an edge endpoint is outside [0, N)");
+                st = RIPPLE_ERR_VERTEX_RANGE;
+                goto fail;
+            }
+        }
+
+        // model and cached state
+        c->d[0] = layers[0].d_in; c->ld[0] = pad4(c->d[0]);
+        for (int l = 1; l <= L; ++l) {
+            const ripple_layer& y = layers[l - 1];
+            LayerDev& ly = c->layer[l];
+            c->d[l] = y.d_out; c->ld[l] = pad4(y.d_out);
+            ly.kind = y.kind; ly.d_in = y.d_in; ly.d_hid = y.d_hidden; ly.d_out = y.d_out; ly.act = y.act; ly.eps = y.eps;
+            ly.ld_in = pad4(y.d_in); ly.ld_hid = pad4(y.d_hidden); ly.ld_out = pad4(y.d_out);
+            std::vector<float> w1, b1, w2, b2;
+            if (y.kind == RIPPLE_LAYER_SAGE) {
+                w1 = padded_matrix(y.Wa, y.d_in, y.d_out, ly.ld_in, ly.ld_out);
+                std::vector<float> wn = padded_matrix(y.Wb, y.d_in, y.d_out, ly.ld_in, ly.ld_out);
+                w1.insert(w1.end(), wn.begin(), wn.end());
+                b1 = padded_matrix(y.ba, 1, y.d_out, 1, ly.ld_out);
+            } else if (y.kind == RIPPLE_LAYER_GRAPHCONV) {
+                w1 = padded_matrix(y.Wa, y.d_in, y.d_out, ly.ld_in, ly.ld_out);
+                b1 = padded_matrix(y.ba, 1, y.d_out, 1, ly.ld_out);
+            } else {
+                w1 = padded_matrix(y.Wa, y.d_in, y.d_hidden, ly.ld_in, ly.ld_hid);
+                b1 = padded_matrix(y.ba, 1, y.d_hidden, 1, ly.ld_hid);
+                w2 = padded_matrix(y.Wb, y.d_hidden, y.d_out, ly.ld_hid, ly.ld_out);
+                b2 = padded_matrix(y.bb, 1, y.d_out, 1, ly.ld_out);
+                max_hid = std::max(max_hid, ly.ld_hid);
+            }
+            CK(dev_alloc(&ly.W1, w1.size()));
+            CK(cudaMemcpy(ly.W1, w1.data(), sizeof(float) * w1.size(), cudaMemcpyHostToDevice));
+            CK(dev_alloc(&ly.b1, b1.size()));
+            CK(cudaMemcpy(ly.b1, b1.data(), sizeof(float) * b1.size(), cudaMemcpyHostToDevice));
+            if (!w2.empty()) {
+                CK(dev_alloc(&ly.W2, w2.size()));
+                CK(cudaMemcpy(ly.W2, w2.data(), sizeof(float) * w2.size(), cudaMemcpyHostToDevice));
+                CK(dev_alloc(&ly.b2, b2.size()));
+                CK(cudaMemcpy(ly.b2, b2.data(), sizeof(float) * b2.size(), cudaMemcpyHostToDevice));
+            }
+        }
+        for (int l = 0; l <= L; ++l) {
+            max_ld = std::max(max_ld, c->ld[l]);
+            CK(dev_alloc(&c->H[l], (size_t)N * c->ld[l], 0));
+            if (l > 0) CK(dev_alloc(&c->S[l], (size_t)N * c->ld[l - 1], 0));
+            CK(dev_alloc(&c->A[l], (size_t)N + 32));
+        }
+        CK(cudaMemcpy2D(c->H[0], sizeof(float) * c->ld[0], features, sizeof(float) * c->d[0],
+                        sizeof(float) * c->d[0], (size_t)N,
+                        feat_mem == RIPPLE_MEM_DEVICE ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice));
+        if (max_hid) CK(dev_alloc(&c->T, (size_t)N * max_hid));
+        for (int s = 0; s < 2; ++s) {
+            CK(dev_alloc(&c->D[s], (size_t)N * max_ld));
+            CK(dev_alloc(&c->Clist[s], (size_t)N + 32));
+            CK(dev_alloc(&c->grow_list[s], (size_t)o.max_batch));
+        }
+        CK(dev_alloc(&c->coff, (size_t)N + 2, 0));
+        CK(dev_alloc(&c->bitmap, (size_t)c->n_words + 256, 0));
+        CK(dev_alloc(&c->posmap, (size_t)N, 0xFF));
+        CK(dev_alloc(&c->deg_out_old, (size_t)N, 0xFF));
+        CK(dev_alloc(&c->feat_last, (size_t)N, 0xFF));
+        // batch staging
+        CK(dev_alloc(&c->ups_dev, (size_t)o.max_batch));
+        CK(dev_alloc(&c->feat_dev, (size_t)o.max_batch * c->d[0]));
+        c->hsize = 1024;
+        while (c->hsize < 4 * o.max_batch) c->hsize <<= 1;
+        CK(dev_alloc(&c->hkeys, (size_t)c->hsize, 0));
+        CK(dev_alloc(&c->hseq, (size_t)c->hsize, 0xFF));
+        CK(dev_alloc(&c->op_slot, (size_t)o.max_batch));
+        CK(dev_alloc(&c->rec, (size_t)o.max_batch));
+        CK(cudaDeviceSynchronize());
+
+        st = run_full(c);
+        if (st) { memcpy(g_create_err, c->err, sizeof(g_create_err)); goto fail_keep_msg; }
+        c->stats.num_layers = L;
+        c->stats.num_edges = E;
+        *out = reinterpret_cast<ripple_ctx*>(c);
+        return RIPPLE_OK;
+    }
+fail:
+    if (c && c->err[0]) memcpy(g_create_err, c->err, sizeof(g_create_err));
+fail_keep_msg:
+    destroy_ctx(c);
+    return st;
+}
+
+extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update* ups, int64_t n,
+                                            const float* feat_rows, int64_t n_rows, int32_t mem) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c) return RIPPLE_ERR_INVALID_ARG;
+    ripple_status st = RIPPLE_OK;
+    if (n < 0 || n_rows < 0 || (n > 0 && !ups) || (n_rows > 0 && !feat_rows) || (mem != 0 && mem != 1)) {
+        set_err(c, "bad arguments to ripple_apply_batch");
+        return RIPPLE_ERR_INVALID_ARG;
+    }
+    if (n > c->max_batch || n_rows > c->max_batch) {
+        set_err(c, "batch of %lld updates exceeds max_batch = %lld", (long long)n, (long long)c->max_batch);
+        return RIPPLE_ERR_CAPACITY;
+    }
+    cudaSetDevice(c->device);
+    const int nb = (int)n, nr = (int)n_rows, L = c->L;
+    ripple_update* own_ups = c->ups_dev;
+    float* own_feat = c->feat_dev;
+    c->launches = 0;
+    int evi = 0;
+#define STAMP() do { if (c->timing) cudaEventRecord(c->ev[evi], c->stream); ++evi; } while (0)
+    if (mem == RIPPLE_MEM_HOST) {
+        if (nb) CK(cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, cudaMemcpyHostToDevice, c->stream));
+        if (nr) CK(cudaMemcpyAsync(c->feat_dev, feat_rows, sizeof(float) * (size_t)nr * c->d[0], cudaMemcpyHostToDevice, c->stream));
+    } else {
+        // device inputs are used in place
+        c->ups_dev = const_cast<ripple_update*>(ups);
+        c->feat_dev = const_cast<float*>(feat_rows);
+    }
+    RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, nb);
+    STAMP();  // 0
+    // Apply (Sec. 3.3): normalise the batch, mutate both adjacency directions, replace features
+    graph_batch_classify(c, nb, nr);
+    graph_batch_mutate(c, nb);
+    frontier_seed_features(c, nb);
+    feature_rows(c, nb);
+    senders_build(c, 0, nb);
+    STAMP();  // 1
+    // one superstep per hop (Sec. 3.3.1): frontier, send + aggregate, compute + prepare
+    for (int l = 1; l <= L; ++l) {
+        frontier_build(c, l, nb);
+        STAMP();
+        scatter_layer(c, l, nb);
+        senders_release(c, l - 1);
+        STAMP();
+        update_rows(c, l, false);
+        if (l < L) senders_build(c, l, nb);
+        STAMP();
+    }
+    graph_batch_cleanup(c, nb);
+    STAMP();
+#undef STAMP
+    c->ups_dev = own_ups;
+    c->feat_dev = own_feat;
+    st = sync_and_fetch_ctl(c);
+    if (st) return st;
+    {
+        const Ctl& h = *c->ctl_host;
+        ripple_stats& s = c->stats;
+        s.gpu_launches = c->launches;
+        s.n_ops = nb;
+        if (h.err) {
+            st = (ripple_status)h.err;
+            set_err(c, st == RIPPLE_ERR_VERTEX_RANGE ? "batch rejected: vertex id or payload row out of range"
+                       : st == RIPPLE_ERR_CAPACITY   ? "batch rejected: overflow edge pool exhausted"
+                                                     : "batch rejected: unknown op code");
+            s.n_added = s.n_deleted = s.n_noop_add = s.n_noop_del = s.n_superseded = s.n_feature = 0;
+            for (int l = 0; l <= L; ++l) s.affected[l] = s.senders[l] = s.active_edges[l] = 0;
+            return st;
+        }
+        s.n_added = h.n_add; s.n_deleted = h.n_del; s.n_noop_add = h.n_noop_add; s.n_noop_del = h.n_noop_del;
+        s.n_superseded = h.n_superseded; s.n_feature = h.n_feat;
+        s.num_edges += h.n_add - h.n_del;
+        for (int l = 0; l <= L; ++l) {
+            s.affected[l] = h.nA[l];
+            s.senders[l] = h.nC[l];
+            s.active_edges[l] = l ? (int64_t)h.E[l] + h.n_rec : 0;
+            s.scatter_pull[l] = h.pull[l];
+        }
+        s.pool_used = (int64_t)h.pool_next[0] - c->side[0].base_end;
+        s.pool_size = c->side[0].col_size - c->side[0].base_end;
+        if (c->timing) {
+            cudaEventElapsedTime(&s.ms_total, c->ev[0], c->ev[evi - 1]);
+            cudaEventElapsedTime(&s.ms_graph, c->ev[0], c->ev[1]);
+            for (int l = 1; l <= L; ++l) {
+                int b = 1 + 3 * (l - 1);
+                cudaEventElapsedTime(&s.ms_frontier[l], c->ev[b], c->ev[b + 1]);
+                cudaEventElapsedTime(&s.ms_scatter[l], c->ev[b + 1], c->ev[b + 2]);
+                cudaEventElapsedTime(&s.ms_update[l], c->ev[b + 2], c->ev[b + 3]);
+            }
+        }
+    }
+    return RIPPLE_OK;
+fail:
+    c->ups_dev = own_ups;
+    c->feat_dev = own_feat;
+    return st;
+}
+
+extern "C" ripple_status ripple_get_embeddings(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !dev_ptr || !ld || layer < 0 || layer > c->L) return RIPPLE_ERR_INVALID_ARG;
+    *dev_ptr = c->H[layer];
+    *ld = c->ld[layer];
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_get_aggregate(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !dev_ptr || !ld || layer < 1 || layer > c->L) return RIPPLE_ERR_INVALID_ARG;
+    *dev_ptr = c->S[layer];
+    *ld = c->ld[layer - 1];
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_get_affected(ripple_ctx* ctx, int32_t layer, const int32_t** dev_ids, int64_t* count) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !dev_ids || !count || layer < 0 || layer > c->L) return RIPPLE_ERR_INVALID_ARG;
+    *dev_ids = c->A[layer];
+    *count = c->stats.affected[layer];
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_export_graph(ripple_ctx* ctx, int64_t* rowptr, int32_t* col, int64_t col_capacity) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !rowptr || (!col && col_capacity > 0)) return RIPPLE_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    int64_t ne = 0;
+    cudaError_t e = graph_export(c, rowptr, col, col_capacity, &ne);
+    if (e == cudaErrorInvalidValue) {
+        set_err(c, "col_capacity %lld is smaller than the edge count %lld", (long long)col_capacity, (long long)ne);
+        return RIPPLE_ERR_INVALID_ARG;
+    }
+    if (e) { set_err(c, "export failed: %s", cudaGetErrorString(e)); return RIPPLE_ERR_CUDA; }
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_get_degrees(ripple_ctx* ctx, const int32_t** deg_out, const int32_t** deg_in) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !deg_out || !deg_in) return RIPPLE_ERR_INVALID_ARG;
+    *deg_out = c->side[0].deg;
+    *deg_in = c->side[1].deg;
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_recompute_full(ripple_ctx* ctx) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c) return RIPPLE_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    return run_full(c);
+}
+
+extern "C" ripple_status ripple_get_stats(ripple_ctx* ctx, ripple_stats* out) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !out) return RIPPLE_ERR_INVALID_ARG;
+    *out = c->stats;
+    return RIPPLE_OK;
+}
+
+extern "C" const char* ripple_last_error(ripple_ctx* ctx) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    return c ? c->err : g_create_err;
+}
+
+extern "C" void ripple_destroy(ripple_ctx* ctx) { destroy_ctx(reinterpret_cast<Ctx*>(ctx)); }
+
+extern "C" const char* ripple_version(void) { return "ripple-b200 0.1 (sm_100a)"; }

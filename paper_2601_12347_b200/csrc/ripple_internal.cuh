@@ -1,0 +1,159 @@
+// Internal declarations shared by the CUDA translation units of the ripple library.
+//
+// Control flow: the host never learns a frontier size in the middle of a batch.  Every kernel
+// reads its work size from a control block in device memory (Ctl) and runs as a grid-stride loop
+// over a fixed grid, so a batch is one uninterrupted chain of launches on one stream; the control
+// block is copied to pinned host memory once, at the end.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ripple.h"
+
+#define RP_MAXL RIPPLE_MAX_LAYERS
+#define RP_TOMB (-1)
+
+namespace rp {
+
+// ---- device-resident control block -----------------------------------------------------------
+struct Ctl {
+    int abort;   // set by validation / planning: the batch is rejected, mutate nothing
+    int err;     // ripple_status recorded on the device
+    int err_info;
+    int n_ops;
+    int n_rec;   // net edge changes of the batch (|dE+| + |dE-|)
+    int n_add, n_del, n_noop_add, n_noop_del, n_superseded, n_feat;
+    int n_grow[2];
+    unsigned long long pool_need[2];
+    unsigned long long pool_next[2];  // next free entry of each side's adjacency array
+    int nA[RP_MAXL + 1];              // |A_l|
+    int nC[RP_MAXL + 1];              // |C_l| (A_l plus sources of edge changes when coefficients depend on them)
+    unsigned long long E[RP_MAXL + 1];          // out-edges of C_{l-1} (+ edge records): message count of hop l
+    unsigned long long pull_work[RP_MAXL + 1];  // in-edges of A_l
+    int pull[RP_MAXL + 1];
+    int work_counter[8];              // dynamic work distribution tickets (reset by the consumer)
+};
+
+// One direction of the adjacency: row r holds col[start[r] .. start[r] + deg[r]), capacity cap[r].
+// Rows start in the base region; a row that outgrows its slack moves into the overflow pool
+// (the tail of the same array) with doubled capacity.
+struct Side {
+    int32_t* col;
+    int64_t* start;
+    int32_t* cap;
+    int32_t* deg;
+    int64_t col_size;  // base region + pool, entries
+    int64_t base_end;  // first pool entry
+    // per-row scratch of the batched update (all zero between batches)
+    int32_t* cnt_del;
+    int32_t* cnt_add;
+    int32_t* tick_a;
+    int32_t* tick_b;
+    int32_t* touch;
+};
+
+// One net edge change.  side 0 = out-list of u (stores v), side 1 = in-list of v (stores u).
+struct Rec {
+    int32_t u, v;
+    int32_t sign;        // +1 added, -1 deleted
+    int32_t pos[2];      // deleted: slot of the entry inside its row
+    int32_t rank[2];     // rank among the row's additions (resp. deletions) of this batch
+    int32_t tail_val[2]; // deleted: entry found at tail slot new_deg + rank
+    int32_t rep[2];      // 1 for the first record that touched the row
+    int32_t deg_out_old; // out-degree of u before the batch
+};
+
+struct LayerDev {
+    int kind, d_in, d_hid, d_out, act;
+    float eps;
+    int ld_in, ld_hid, ld_out;  // padded widths (multiples of 4)
+    float* W1;   // SAGE: [W_self; W_neigh] (2 d_in x ld_out); GRAPHCONV: d_in x ld_out; GIN: d_in x ld_hid
+    float* b1;   // ld_out (SAGE, GRAPHCONV) or ld_hid (GIN)
+    float* W2;   // GIN: d_hid x ld_out
+    float* b2;   // GIN: ld_out
+};
+
+struct Ctx {
+    int device;
+    cudaStream_t stream;
+    bool own_stream;
+    int N, L, agg;
+    bool self_term, src_norm;
+    int64_t E0;
+    int64_t max_batch;
+    int scatter_mode, gemm_mode, timing;
+    int n_sm;
+    LayerDev layer[RP_MAXL + 1];
+    int d[RP_MAXL + 1], ld[RP_MAXL + 1];
+    Side side[2];
+    float* H[RP_MAXL + 1];
+    float* S[RP_MAXL + 1];
+    float* T;          // GIN hidden rows (compact, N x ld_hid)
+    float* D[2];       // delta rows, ping-pong (compact, N x max ld)
+    int32_t* A[RP_MAXL + 1];   // affected lists
+    int32_t* Clist[2];         // sender list, ping-pong (A_l followed by extra sources)
+    int64_t* coff;             // exclusive prefix of out-degrees over the sender list (+1)
+    uint32_t* bitmap;          // N bits
+    int n_words;
+    int32_t* posmap;           // vertex -> index in the current sender list, or -1
+    int32_t* deg_out_old;      // vertex -> out-degree before the batch, or -1
+    int32_t* feat_last;        // vertex -> index of its last SET_FEATURE op in the batch, or -1
+    // batch staging
+    ripple_update* ups_dev;
+    float* feat_dev;
+    ripple_update* ups_pin;
+    float* feat_pin;
+    unsigned long long* hkeys; // pair hash table
+    int32_t* hseq;
+    int32_t* op_slot;
+    int hsize;
+    Rec* rec;
+    int32_t* grow_list[2];
+    // scan scratch
+    int64_t* tile_sums;
+    int n_tile_sums;
+    Ctl* ctl;        // device
+    Ctl* ctl_host;   // pinned
+    ripple_stats stats;
+    cudaEvent_t ev[4 + 3 * (RP_MAXL + 1) + 2];
+    int64_t launches;
+    char err[512];
+};
+
+// ---- helpers -----------------------------------------------------------------------------------
+inline int div_up(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+inline int pad4(int x) { return (x + 3) & ~3; }
+
+#define RP_LAUNCH(ctx, kernel, grid, block, smem, ...)                         \
+    do {                                                                        \
+        kernel<<<(grid), (block), (smem), (ctx)->stream>>>(__VA_ARGS__);        \
+        (ctx)->launches++;                                                      \
+    } while (0)
+
+// graph_store.cu
+cudaError_t graph_build(Ctx* c, const int32_t* src_dev, const int32_t* dst_dev, int64_t E,
+                        double slack, int64_t pool_edges);
+void graph_batch_classify(Ctx* c, int n, int n_rows);   // validate, dedupe, find net changes, plan
+void graph_batch_mutate(Ctx* c, int n);                 // apply the net changes to both directions
+void graph_batch_cleanup(Ctx* c, int n);                // reset per-batch scratch
+cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, int64_t col_capacity, int64_t* n_edges);
+
+// frontier.cu
+void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, const int32_t* deg,
+                  int64_t* out, unsigned long long* total_dev);
+void frontier_seed_features(Ctx* c, int n);             // A_0 from the batch's feature updates
+void frontier_build(Ctx* c, int l, int n);              // A_l from C_{l-1}, edge records, A_{l-1}
+void senders_build(Ctx* c, int l, int n);               // C_l, posmap, coff, E_{l+1}
+void senders_release(Ctx* c, int l);                    // clear posmap entries of C_l
+
+// scatter.cu
+void spmm_full(Ctx* c, int l);                          // S^l for every vertex (bootstrap)
+void scatter_layer(Ctx* c, int l, int n);               // delta messages of hop l into S^l
+
+// layer_update.cu
+void update_rows(Ctx* c, int l, bool full);             // re-apply Update^l + activation, emit deltas
+void feature_rows(Ctx* c, int n);                       // hop 0: overwrite feature rows, emit deltas
+void extra_sender_rows(Ctx* c, int l, int n);           // deltas of senders whose row did not change
+
+}  // namespace rp
