@@ -1,0 +1,345 @@
+#!/usr/bin/env python
+"""Benchmark of the incremental-propagation hot path.
+
+A step is one pass of the whole path over one batch of B synthetic updates: normalise the batch,
+update the graph store, build the per-layer frontiers, scatter the delta messages, re-apply the
+layer update to the affected rows.  Default workload: the dense graph (2 449 029 vertices,
+123 718 280 edges, 100 features), 2-layer GraphSAGE-mean 100-256-47, B = 1000.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--batch B]
+    python bench.py --impl reference ...     # the CPU oracle on the same workload (host cores)
+
+Prints one JSON line (rank 0).  With N > 1 (under torchrun) every rank runs an independent replica
+of the workload on its own GPU with its own update stream; there is no data-path collective.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2601_12347_b200 import inputs as I  # noqa: E402
+
+METRIC = "updates_per_sec"
+UNIT = "updates/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def pct(xs, p):
+    xs = sorted(xs)
+    if not xs:
+        return None
+    k = max(0, min(len(xs) - 1, int(np.ceil(p / 100.0 * len(xs))) - 1))
+    return xs[k]
+
+
+def scatter_bytes(stats, l, ld):
+    """Algorithmic bytes of hop l's scatter in the form that ran (fp32, row width ld floats).
+    push: each sender row read once, its out-list read once, one read + one write of an aggregate
+    row per message.  pull: in-lists of the affected sinks, one delta row per message, one read +
+    one write of each affected aggregate row."""
+    e = stats["active_edges"][l] - (stats["n_added"] + stats["n_deleted"])
+    if stats["scatter_pull"][l]:
+        # in-list entry + position-map entry per in-edge of an affected sink; every sender's delta
+        # row once (it is re-read from L2 after that); read + write of each affected aggregate row
+        return stats["in_edges"][l] * 8 + stats["senders"][l - 1] * 4 * ld + stats["affected"][l] * 8 * ld
+    return stats["senders"][l - 1] * (4 * ld + 8) + 4 * e + e * 8 * ld
+
+
+def make_workload(name, seed):
+    w = I.workloads()[name]
+    w.seed = seed
+    src, dst = I.make_graph(w)
+    X = I.features(w.n, w.model.dims[0], w.seed)
+    W = I.make_weights(w.model, w.seed)
+    return w, src, dst, X, W
+
+
+def run_reference(args, rank, world):
+    """The CPU oracle (incremental route) on the same workload; one step = one batch."""
+    if rank != 0:
+        return
+    from oracle import oracle as O
+    O.build()
+    w, src, dst, X, W = make_workload(args.workload, args.seed)
+    orc = O.Oracle(w.n, src, dst, X, w.model, W)
+    stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], w.seed)
+    lat = []
+    for s in range(args.warmup + args.steps):
+        ups, rows = stream.next_batch(args.batch)
+        t0 = time.perf_counter()
+        assert orc.apply_incremental(ups, rows) == 0
+        if s >= args.warmup:
+            lat.append(time.perf_counter() - t0)
+    total = sum(lat)
+    value = args.batch * len(lat) / total
+    cores = O.num_threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(lat),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": f"{args.workload}, batch {args.batch}", "batch": args.batch,
+                   "vertices": w.n, "edges": w.e, "dims": w.model.dims},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{len(lat)} batches of {args.batch} updates, incremental route; "
+                                   "message scatter single-threaded, compute step on all cores"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "latency_ms": {"p50": 1e3 * pct(lat, 50), "p99": 1e3 * pct(lat, 99)},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def cpu_baseline(args, w, src, dst, X, W, budget_s=20.0):
+    """The oracle as it stands, timed on the host cores on a bounded sample of the workload."""
+    from oracle import oracle as O
+    O.build()
+    t0 = time.perf_counter()
+    orc = O.Oracle(w.n, src, dst, X, w.model, W)
+    setup = time.perf_counter() - t0
+    stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], w.seed)
+    spent, nb = 0.0, 0
+    while spent < budget_s and nb < 50:
+        ups, rows = stream.next_batch(args.batch)
+        t0 = time.perf_counter()
+        assert orc.apply_incremental(ups, rows) == 0
+        spent += time.perf_counter() - t0
+        nb += 1
+    orc.close()
+    return {"value": args.batch * nb / spent, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"first {nb} batches of {args.batch} updates of the same stream "
+                      f"({spent:.1f} s; oracle set-up incl. its own bootstrap {setup:.0f} s, untimed)"}
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2601_12347_b200 import build as B
+    from paper_2601_12347_b200 import ripple
+    B.build_library()
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    seed = args.seed + rank
+    w, src, dst, X, W = make_workload(args.workload, seed)
+    L = len(w.model.layers)
+    rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=max(args.batch, 16),
+                       scatter_mode=args.scatter)
+    bootstrap_ms = rp.stats()["ms_bootstrap"]
+    stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], seed)
+    K, Wm = args.steps, args.warmup
+    batches = [stream.next_batch(args.batch) for _ in range(Wm + 2 * K)]
+
+    def to_dev(ups, rows):
+        u = torch.from_numpy(np.stack([ups["op"], ups["u"], ups["v"]], axis=1).astype(np.int32)).cuda()
+        return u, torch.from_numpy(rows).cuda()
+
+    def to_pinned(ups, rows):
+        u = torch.from_numpy(np.stack([ups["op"], ups["u"], ups["v"]], axis=1).astype(np.int32)).pin_memory()
+        return u, torch.from_numpy(rows).pin_memory()
+
+    dev_batches = [to_dev(*b) for b in batches[: Wm + K]]
+    pin_batches = [to_pinned(*b) for b in batches[Wm + K:]]
+    st = rp.stream
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(Wm):
+        rp.apply_batch(*dev_batches[i])
+
+    # ---- device-resident timing -------------------------------------------------------------
+    sampler = ClockSampler(local_rank)
+    launches = 0
+    sc_ms, sc_bytes, stage = 0.0, 0, {"graph": 0.0, "frontier": 0.0, "scatter": 0.0, "update": 0.0}
+    sizes = {"affected": np.zeros(L + 1), "active_edges": np.zeros(L + 1)}
+    ld_last = (w.model.dims[L - 1] + 3) // 4 * 4
+    pulls = 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    ev0.record(st)
+    for i in range(Wm, Wm + K):
+        rp.apply_batch(*dev_batches[i])
+        s = rp.stats()
+        launches += s["gpu_launches"]
+        stage["graph"] += s["ms_graph"]
+        for l in range(1, L + 1):
+            stage["frontier"] += s["ms_frontier"][l]
+            stage["scatter"] += s["ms_scatter"][l]
+            stage["update"] += s["ms_update"][l]
+        pulls += s["scatter_pull"][L]
+        sc_ms += s["ms_scatter_kernel"][L]
+        sc_bytes += scatter_bytes(s, L, ld_last)
+        sizes["affected"] += np.array(s["affected"][: L + 1])
+        sizes["active_edges"] += np.array(s["active_edges"][: L + 1])
+    ev1.record(st)
+    barrier()
+    clocks = sampler.stop()
+    dev_ms = ev0.elapsed_time(ev1)
+
+    # ---- end to end: pinned host inputs, H2D inside, result ids read back ----------------------
+    lat = []
+    h2d = d2h = 0
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st)
+    for u, r in pin_batches:
+        t0 = time.perf_counter()
+        rp.apply_batch(u, r)
+        ids = rp.affected(L).cpu()        # trigger-style read-out: who changed at the last layer
+        lat.append(time.perf_counter() - t0)
+        h2d += u.numel() * 4 + r.numel() * 4
+        d2h += ids.numel() * 4
+    e1.record(st)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    if world > 1:
+        t = torch.tensor([dev_ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dev_ms, e2e_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        rp.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = load_peaks()
+    achieved = (sc_bytes / 1e9) / (sc_ms / 1e3) if sc_ms > 0 else None
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": (achieved / peak) if achieved else None, "traffic": None,
+                "kernel": f"{'k_scatter_pull' if pulls * 2 > K else 'k_scatter_push'} (hop {L}, row width {ld_last} floats)",
+                "pull_steps": int(pulls),
+                "peak_source": f"of {peak_kind}",
+                "ms_per_launch": sc_ms / K,
+                "algorithmic_bytes_per_launch": sc_bytes / K}
+    line = {
+        "metric": METRIC, "value": world * args.batch * K / (dev_ms / 1e3), "unit": UNIT,
+        "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": dev_ms / K,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": f"{args.workload}, batch {args.batch}", "batch": args.batch,
+                   "vertices": w.n, "edges": w.e, "dims": w.model.dims,
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                   "l2": "working set (aggregate and embedding rows, GBs) far larger than L2; no flush needed"},
+        "clocks": clocks,
+        "e2e": {"value": world * args.batch * K / (e2e_ms / 1e3), "unit": UNIT,
+                "h2d_bytes_per_step": h2d // K, "d2h_bytes_per_step": d2h // K},
+        "gpu_launches": int(launches),
+        "latency_ms": {"p50": 1e3 * pct(lat, 50), "p99": 1e3 * pct(lat, 99), "mean": 1e3 * float(np.mean(lat)),
+                       "note": "host wall clock around the C-ABI call with pinned host inputs"},
+        "roofline": roofline,
+        "stage_ms_per_step": {k: v / K for k, v in stage.items()},
+        "per_layer": {"affected": (sizes["affected"] / K).tolist(),
+                      "active_edges": (sizes["active_edges"] / K).tolist()},
+        "bootstrap_ms": bootstrap_ms,
+    }
+    rp.close()
+    del rp
+    torch.cuda.empty_cache()
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(args, w, src, dst, X, W)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="dense-2l")
+    ap.add_argument("--batch", type=int, default=1000)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--scatter", type=int, default=0, help="0 auto, 1 push, 2 pull")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        if world > 1 and rank != 0:
+            args.no_cpu_baseline = True
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -124,12 +124,14 @@ typedef struct {
     int64_t senders[RIPPLE_MAX_LAYERS + 1];       /* |C_l|: vertices whose outgoing message changed       */
     int64_t active_edges[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: edges carrying a message at hop l          */
     int32_t scatter_pull[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: 1 if hop l gathered over in-edges          */
+    int64_t in_edges[RIPPLE_MAX_LAYERS + 1];      /* l = 1..L: in-edges of A_l (what a gather walks)      */
     int64_t pool_used, pool_size;                 /* overflow pool, edges, out-direction                  */
     /* CUDA-event times of the last batch in milliseconds (zero unless options.timing) */
     float ms_total, ms_graph;
     float ms_frontier[RIPPLE_MAX_LAYERS + 1];
     float ms_scatter[RIPPLE_MAX_LAYERS + 1];
     float ms_update[RIPPLE_MAX_LAYERS + 1];
+    float ms_scatter_kernel[RIPPLE_MAX_LAYERS + 1]; /* the push or pull kernel alone, l = 1..L               */
     float ms_bootstrap;                           /* last ripple_create / ripple_recompute_full           */
     int64_t gpu_launches;                         /* kernels launched by the last call                    */
 } ripple_stats;

@@ -23,7 +23,7 @@ def build(force: bool = False) -> str:
     src = os.path.join(_HERE, "ripple_oracle.c")
     out = os.path.join(_HERE, "_ripple_oracle.so")
     if force or not os.path.exists(out) or os.path.getmtime(out) < os.path.getmtime(src):
-        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", out, src, "-lm"])
+        subprocess.check_call(["gcc", "-O3", "-fopenmp", "-shared", "-fPIC", "-o", out, src, "-lm"])
     return out
 
 
@@ -62,8 +62,14 @@ def _load():
     lib.orc_export_csr.restype = None
     lib.orc_row_from_prev.argtypes = [vp, i32, i32, vp, i64, vp, vp]
     lib.orc_row_from_prev.restype = None
+    lib.orc_num_threads.argtypes = []
+    lib.orc_num_threads.restype = i32
     _lib = lib
     return lib
+
+
+def num_threads() -> int:
+    return int(_load().orc_num_threads())
 
 
 class Oracle:

@@ -30,6 +30,9 @@
  * Edge (u, v): u is the source, v the sink; v aggregates over its in-neighbours.
  */
 #include <math.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
@@ -519,6 +522,7 @@ int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const flo
 
         /* Compute: re-apply Update and the activation to the hop-l vertices, keeping old rows */
         double *oldAn = (double *)malloc(sizeof(double) * ((size_t)nAn * (size_t)J + 1));
+#pragma omp parallel for schedule(dynamic, 64)
         for (int i = 0; i < nAn; ++i) {
             int v = An[i];
             double *row = o->H[l] + (size_t)v * J;
@@ -597,6 +601,18 @@ void orc_row_from_prev(const oracle_t *o, int l, int v, const float *Hprev, int6
 }
 
 /* ------------------------------------------------------------------------------------------ */
+/* threads the parallel loops (full inference, the compute step) run on */
+int orc_num_threads(void) {
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp single
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}
 double *orc_H(oracle_t *o, int l) { return o->H[l]; }
 double *orc_S(oracle_t *o, int l) { return o->S[l]; }
 double *orc_full_H(oracle_t *o, int l) { return l == 0 ? o->H[0] : o->FH[l]; }

@@ -68,6 +68,7 @@ static void destroy_ctx(Ctx* c) {
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
     for (auto& e : c->ev) if (e) cudaEventDestroy(e);
+    for (auto& e : c->ev_sc) if (e) cudaEventDestroy(e);
     if (c->own_stream && c->stream) cudaStreamDestroy(c->stream);
     delete c;
 }
@@ -164,6 +165,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         c->n_tile_sums = std::max(div_up(N, 1024) + 2, div_up(c->n_words, 256) + 2);
         CK(dev_alloc(&c->tile_sums, (size_t)c->n_tile_sums, 0));
         for (auto& e : c->ev) CK(cudaEventCreate(&e));
+        for (auto& e : c->ev_sc) CK(cudaEventCreate(&e));
 
         // graph
         if (E > 0 && g->mem == RIPPLE_MEM_HOST) {
@@ -344,6 +346,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
             s.senders[l] = h.nC[l];
             s.active_edges[l] = l ? (int64_t)h.E[l] + h.n_rec : 0;
             s.scatter_pull[l] = h.pull[l];
+            s.in_edges[l] = (int64_t)h.pull_work[l];
         }
         s.pool_used = (int64_t)h.pool_next[0] - c->side[0].base_end;
         s.pool_size = c->side[0].col_size - c->side[0].base_end;
@@ -355,6 +358,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
                 cudaEventElapsedTime(&s.ms_frontier[l], c->ev[b], c->ev[b + 1]);
                 cudaEventElapsedTime(&s.ms_scatter[l], c->ev[b + 1], c->ev[b + 2]);
                 cudaEventElapsedTime(&s.ms_update[l], c->ev[b + 2], c->ev[b + 3]);
+                cudaEventElapsedTime(&s.ms_scatter_kernel[l], c->ev_sc[2 * l], c->ev_sc[2 * l + 1]);
             }
         }
     }

@@ -117,6 +117,7 @@ struct Ctx {
     Ctl* ctl_host;   // pinned
     ripple_stats stats;
     cudaEvent_t ev[4 + 3 * (RP_MAXL + 1) + 2];
+    cudaEvent_t ev_sc[2 * (RP_MAXL + 1)];  // tight brackets around each hop's main scatter kernel
     int64_t launches;
     char err[512];
 };

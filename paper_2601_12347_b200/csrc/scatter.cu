@@ -226,6 +226,7 @@ void scatter_layer(Ctx* c, int l, int n) {
     RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode, ld);
     const int T = 256;
     const int grid = c->n_sm * 8;
+    if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
 #define PUSH(NV) RP_LAUNCH(c, k_scatter_push<NV>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], D, ld, c->S[l])
 #define PULL(NV) RP_LAUNCH(c, k_scatter_pull<NV>, grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->posmap, D, ld, c->S[l])
     if (c->scatter_mode != RIPPLE_SCATTER_PULL) {
@@ -236,6 +237,7 @@ void scatter_layer(Ctx* c, int l, int n) {
     }
 #undef PUSH
 #undef PULL
+    if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
     if (n > 0)
         RP_LAUNCH(c, k_scatter_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, c->rec,
                   (int)c->src_norm, c->side[0].deg, c->posmap, c->H[l - 1], D, ld, c->S[l]);

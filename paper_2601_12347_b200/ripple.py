@@ -68,10 +68,11 @@ class _Stats(ctypes.Structure):
                 ("n_noop_add", ctypes.c_int64), ("n_noop_del", ctypes.c_int64),
                 ("n_superseded", ctypes.c_int64), ("n_feature", ctypes.c_int64),
                 ("affected", _A), ("senders", _A), ("active_edges", _A), ("scatter_pull", _I),
+                ("in_edges", _A),
                 ("pool_used", ctypes.c_int64), ("pool_size", ctypes.c_int64),
                 ("ms_total", ctypes.c_float), ("ms_graph", ctypes.c_float),
                 ("ms_frontier", _F), ("ms_scatter", _F), ("ms_update", _F),
-                ("ms_bootstrap", ctypes.c_float), ("gpu_launches", ctypes.c_int64)]
+                ("ms_scatter_kernel", _F), ("ms_bootstrap", ctypes.c_float), ("gpu_launches", ctypes.c_int64)]
 
 
 _lib = None
@@ -280,8 +281,8 @@ class Ripple:
                                           "n_noop_add", "n_noop_del", "n_superseded", "n_feature",
                                           "pool_used", "pool_size", "ms_total", "ms_graph",
                                           "ms_bootstrap", "gpu_launches")}
-        for k in ("affected", "senders", "active_edges", "scatter_pull", "ms_frontier", "ms_scatter",
-                  "ms_update"):
+        for k in ("affected", "senders", "active_edges", "scatter_pull", "in_edges", "ms_frontier", "ms_scatter",
+                  "ms_update", "ms_scatter_kernel"):
             out[k] = list(getattr(s, k))[: L + 1]
         return out
 

@@ -1,0 +1,418 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, on the same seeded inputs.
+
+Bit-exact: graph state (canonical CSR), per-layer affected sets, update counters.
+Within max |delta| <= 1e-4 (1 + |ref|): embeddings and cached aggregates (fp32 arithmetic).
+"""
+import numpy as np
+import pytest
+
+from paper_2601_12347_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2601_12347_b200 import build as B
+    B.build_library()
+    from paper_2601_12347_b200 import ripple
+    from oracle.oracle import Oracle
+    torch.cuda.set_device(0)
+    return ripple, Oracle
+
+
+# Extra slack for the unnormalised-sum GIN stack, as a fraction of the largest |ref| in the row.
+# On the skewed R-MAT graph its rows grow to 1e4 (layer 2) and 1e6 (layer 3), so an element that
+# cancels to O(1) carries the rounding of O(1e6) partial sums: fp32 unit roundoff 6e-8 times the
+# sqrt(K) growth of a K = 256 dot product is about 1e-6 of the row's scale, and no fp32 path can
+# meet 1e-4 (1 + |ref|) on such elements.  Measured: 2e-6 of the row maximum; bound: 1e-5.
+GIN_ROW_SLACK = 1e-5
+
+
+def max_err(got, ref, row_slack=0.0):
+    got = np.asarray(got, dtype=np.float64)
+    if not ref.size:
+        return 0.0
+    den = 1.0 + np.abs(ref)
+    if row_slack:
+        den = den + (row_slack / TOL) * np.max(np.abs(ref), axis=1, keepdims=True)
+    return float(np.max(np.abs(got - ref) / den))
+
+
+def check_graph(rp, orc):
+    rowptr, col = rp.export_graph()
+    orp, ocol = orc.export_csr()
+    assert np.array_equal(rowptr, orp), "row pointers differ"
+    assert np.array_equal(col, ocol), "column indices differ"
+    do, di = rp.degrees()
+    odo, odi = orc.degrees()
+    assert np.array_equal(do.cpu().numpy(), odo) and np.array_equal(di.cpu().numpy(), odi)
+
+
+def check_frontiers(rp, orc, L):
+    st = rp.stats()
+    for l in range(L + 1):
+        a = rp.affected(l).cpu().numpy()
+        assert np.array_equal(a, orc.affected(l)), f"affected set of layer {l} differs"
+        assert st["affected"][l] == a.size
+    c = orc.counts()
+    assert (st["n_added"], st["n_deleted"], st["n_noop_add"], st["n_noop_del"], st["n_superseded"]) == \
+        (c["added"], c["deleted"], c["noop_add"], c["noop_del"], c["superseded"])
+    for l in range(1, L + 1):
+        assert st["active_edges"][l] == orc.active_edges(l)
+
+
+def check_values(rp, refH, L, refS=None, tol=TOL, row_slack=0.0):
+    """Embeddings within tol (1 + |ref|).  The cached aggregate S_v is an fp32 sum of deg_in(v)
+    terms, so its rounding error grows like sqrt(deg_in): its bound is scaled by that factor (a
+    lost or doubled message is an O(1) error and still fails)."""
+    worst = 0.0
+    for l in range(L + 1):
+        e = max_err(rp.embeddings(l).cpu().numpy(), refH[l], row_slack)
+        assert e <= tol, f"H^{l}: max err {e}"
+        worst = max(worst, e)
+    if refS is not None:
+        deg_in = rp.degrees()[1].cpu().numpy().astype(np.float64)
+        scale = np.sqrt(np.maximum(deg_in, 1.0))[:, None]
+        for l in range(1, L + 1):
+            got = rp.aggregate(l).cpu().numpy().astype(np.float64)
+            den = 1.0 + np.abs(refS[l])
+            if row_slack:
+                den = den + (row_slack / TOL) * np.max(np.abs(refS[l]), axis=1, keepdims=True)
+            e = float(np.max(np.abs(got - refS[l]) / (den * scale)))
+            assert e <= tol, f"S^{l}: max scaled err {e}"
+    return worst
+
+
+def small_models():
+    return {
+        "sage_mean": I.sage_model([18, 36, 10], I.AGG_MEAN),
+        "sage_sum_3l": I.sage_model([18, 36, 20, 10], I.AGG_SUM),
+        "gc_sum": I.graphconv_model([18, 36, 10], I.AGG_SUM),
+        "gc_mean_3l": I.graphconv_model([18, 36, 20, 10], I.AGG_MEAN),
+        "gcn_wsum_3l": I.graphconv_model([18, 36, 20, 10], I.AGG_WSUM_GCN),
+        "gin_3l": I.gin_model(18, 24, 3, eps=0.25),
+    }
+
+
+def ups_array(recs):
+    a = np.zeros(len(recs), dtype=I.UPDATE_DTYPE)
+    for i, r in enumerate(recs):
+        a[i] = r
+    return a
+
+
+# ---------------------------------------------------------------------------------------------
+def test_tiny_config_every_batch_against_full_recompute(env):
+    ripple, Oracle = env
+    w = I.workloads()["tiny"]
+    src, dst = I.make_graph(w)
+    X = I.features(w.n, w.model.dims[0], w.seed)
+    W = I.make_weights(w.model, w.seed)
+    L = len(w.model.layers)
+    rp = ripple.Ripple(w.n, src, dst, X, w.model, W)
+    orc = Oracle(w.n, src, dst, X, w.model, W)
+    check_graph(rp, orc)
+    check_values(rp, [orc.H(l) for l in range(L + 1)], L, [None] + [orc.S(l) for l in range(1, L + 1)])
+    stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], w.seed)
+    for b in range(w.n_batches):
+        ups, rows = stream.next_batch(100)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, L)
+        check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+    rp.close()
+
+
+@pytest.mark.parametrize("name", list(small_models().keys()))
+@pytest.mark.parametrize("mode", ["auto", "push", "pull"])
+def test_every_model_kind_and_scatter_direction(env, name, mode):
+    ripple, Oracle = env
+    model = small_models()[name]
+    L = len(model.layers)
+    n, m = 700, 6000
+    src, dst = I.er_graph(n, m, 3)
+    # a hub so that one row is much longer than the rest, and a self-loop
+    hub_dst = np.arange(1, 400, dtype=np.int32)
+    have = set(zip(src.tolist(), dst.tolist()))
+    extra = [(0, int(v)) for v in hub_dst if (0, int(v)) not in have] + [(5, 5)]
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    X = I.features(n, model.dims[0], 3)
+    W = I.make_weights(model, 3, zero_bias=False)
+    sm = {"auto": ripple.SCATTER_AUTO, "push": ripple.SCATTER_PUSH, "pull": ripple.SCATTER_PULL}[mode]
+    rp = ripple.Ripple(n, src, dst, X, model, W, scatter_mode=sm)
+    orc = Oracle(n, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 3)
+    sizes = [1, 1, 2, 7, 33, 100, 1, 250, 64, 5] * 3
+    for b, bs in enumerate(sizes):
+        ups, rows = stream.next_batch(bs)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, L)
+        if b % 5 == 4 or b == len(sizes) - 1:
+            check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+    st = rp.stats()
+    if mode == "pull":
+        assert all(st["scatter_pull"][l] == 1 for l in range(1, L + 1))
+    if mode == "push":
+        assert all(st["scatter_pull"][l] == 0 for l in range(1, L + 1))
+    rp.close()
+
+
+def test_device_resident_inputs_give_the_same_result(env):
+    import torch
+    ripple, Oracle = env
+    model = small_models()["sage_mean"]
+    n, m = 500, 4000
+    src, dst = I.er_graph(n, m, 9)
+    X = I.features(n, model.dims[0], 9)
+    W = I.make_weights(model, 9)
+    rp = ripple.Ripple(n, torch.from_numpy(src).cuda(), torch.from_numpy(dst).cuda(),
+                       torch.from_numpy(X).cuda(), model, W)
+    orc = Oracle(n, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 9)
+    for _ in range(5):
+        ups, rows = stream.next_batch(50)
+        dev_ups = torch.from_numpy(np.stack([ups["op"], ups["u"], ups["v"]], axis=1).astype(np.int32)).cuda()
+        rp.apply_batch(dev_ups, torch.from_numpy(rows).cuda())
+        assert orc.apply_incremental(ups, rows) == 0
+    check_graph(rp, orc)
+    check_frontiers(rp, orc, 2)
+    check_values(rp, orc.full(), 2)
+    rp.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# batch semantics, degenerate and error cases
+# ---------------------------------------------------------------------------------------------
+def _small(seed=41, name="sage_mean"):
+    model = small_models()[name]
+    n, m = 300, 2000
+    src, dst = I.er_graph(n, m, seed)
+    X = I.features(n, model.dims[0], seed)
+    W = I.make_weights(model, seed, zero_bias=False)
+    return n, src, dst, X, model, W
+
+
+def test_repeated_items_empty_batches_and_noops(env):
+    ripple, Oracle = env
+    n, src, dst, X, model, W = _small()
+    present = set(zip(src.tolist(), dst.tolist()))
+    missing = [(a, b) for a in range(20) for b in range(20) if a != b and (a, b) not in present]
+    (u, v), (mu, mv) = missing[0], missing[5]
+    eu, ev = int(src[0]), int(dst[0])
+    rows = I.features(3, model.dims[0], 77)
+    recs = [
+        (I.OP_ADD_EDGE, u, v), (I.OP_DEL_EDGE, u, v),
+        (I.OP_DEL_EDGE, eu, ev), (I.OP_ADD_EDGE, eu, ev), (I.OP_ADD_EDGE, eu, ev),
+        (I.OP_SET_FEATURE, 4, 0), (I.OP_SET_FEATURE, 4, 2),
+        (I.OP_DEL_EDGE, int(src[1]), int(dst[1])),
+        (I.OP_ADD_EDGE, int(src[2]), int(dst[2])),
+        (I.OP_DEL_EDGE, mu, mv),
+        (I.OP_ADD_EDGE, 6, 6),
+    ]
+    rp = ripple.Ripple(n, src, dst, X, model, W)
+    orc = Oracle(n, src, dst, X, model, W)
+    before = [rp.embeddings(l).clone() for l in range(3)]
+    rp.apply_batch(ups_array([]))
+    assert orc.apply_incremental(ups_array([])) == 0
+    check_frontiers(rp, orc, 2)
+    for l in range(3):
+        assert bool((rp.embeddings(l) == before[l]).all())
+    rp.apply_batch(ups_array(recs), rows)
+    assert orc.apply_incremental(ups_array(recs), rows) == 0
+    check_graph(rp, orc)
+    check_frontiers(rp, orc, 2)
+    check_values(rp, orc.full(), 2)
+    # rows outside the affected sets are bit-identical to what they were
+    for l in range(3):
+        mask = np.ones(n, dtype=bool)
+        mask[orc.affected(l)] = False
+        assert np.array_equal(rp.embeddings(l).cpu().numpy()[mask], before[l].cpu().numpy()[mask])
+    # a feature update that repeats the stored values: affected structurally, values bit-identical
+    cur = [rp.embeddings(l).clone() for l in range(3)]
+    same = rp.embeddings(0)[[11]].cpu().numpy().copy()
+    rp.apply_batch(ups_array([(I.OP_SET_FEATURE, 11, 0)]), same)
+    assert orc.apply_incremental(ups_array([(I.OP_SET_FEATURE, 11, 0)]), same) == 0
+    check_frontiers(rp, orc, 2)
+    assert rp.stats()["affected"][0] == 1
+    for l in range(3):
+        assert np.allclose(rp.embeddings(l).cpu().numpy(), cur[l].cpu().numpy(), rtol=0, atol=1e-6)
+    rp.close()
+
+
+def test_invalid_batches_are_rejected_and_leave_state_untouched(env):
+    ripple, Oracle = env
+    n, src, dst, X, model, W = _small()
+    rp = ripple.Ripple(n, src, dst, X, model, W, max_batch=64)
+    orc = Oracle(n, src, dst, X, model, W)
+    before = [rp.embeddings(l).clone() for l in range(3)]
+    good = (I.OP_DEL_EDGE, int(src[0]), int(dst[0]))
+    rows = I.features(1, model.dims[0], 1)
+    bad_batches = [
+        (ups_array([good, (I.OP_ADD_EDGE, 0, n)]), None, ripple.ERR_VERTEX_RANGE),
+        (ups_array([good, (I.OP_ADD_EDGE, -1, 2)]), None, ripple.ERR_VERTEX_RANGE),
+        (ups_array([good, (7, 1, 2)]), None, ripple.ERR_INVALID_ARG),
+        (ups_array([good, (I.OP_SET_FEATURE, 1, 1)]), rows, ripple.ERR_VERTEX_RANGE),
+        (ups_array([good] * 65), None, ripple.ERR_CAPACITY),
+    ]
+    for ups, r, want in bad_batches:
+        with pytest.raises(ripple.RippleError) as ei:
+            rp.apply_batch(ups, r)
+        assert ei.value.status == want
+        check_graph(rp, orc)
+        for l in range(3):
+            assert bool((rp.embeddings(l) == before[l]).all())
+    # and the context keeps working
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 2)
+    ups, r = stream.next_batch(40)
+    rp.apply_batch(ups, r)
+    assert orc.apply_incremental(ups, r) == 0
+    check_graph(rp, orc)
+    check_frontiers(rp, orc, 2)
+    check_values(rp, orc.full(), 2)
+    rp.close()
+
+
+def test_rows_outgrow_their_slack_and_the_pool_can_run_out(env):
+    ripple, Oracle = env
+    n, src, dst, X, model, W = _small(seed=43, name="gcn_wsum_3l")
+    rp = ripple.Ripple(n, src, dst, X, model, W, slack=0.01, pool_edges=4096)
+    orc = Oracle(n, src, dst, X, model, W)
+    present = set(zip(src.tolist(), dst.tolist()))
+    # vertex 7 gains an out-edge to (almost) everyone, vertex 9 an in-edge from everyone
+    todo = [(7, v) for v in range(n) if v != 7 and (7, v) not in present]
+    todo += [(u, 9) for u in range(n) if u != 9 and (u, 9) not in present and u != 7]
+    for i in range(0, len(todo), 90):
+        ups = ups_array([(I.OP_ADD_EDGE, a, b) for a, b in todo[i:i + 90]])
+        rp.apply_batch(ups)
+        assert orc.apply_incremental(ups) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, 3)
+    check_values(rp, orc.full(), 3)
+    assert rp.stats()["pool_used"] > 0
+    # now shrink them again, many deletions in the same row in one batch
+    for i in range(0, len(todo), 200):
+        ups = ups_array([(I.OP_DEL_EDGE, a, b) for a, b in todo[i:i + 200]])
+        rp.apply_batch(ups)
+        assert orc.apply_incremental(ups) == 0
+        check_graph(rp, orc)
+    check_values(rp, orc.full(), 3)
+    rp.close()
+    # a pool that is too small: the batch that would overflow it is rejected as a whole
+    rp = ripple.Ripple(n, src, dst, X, model, W, slack=0.01, pool_edges=64)
+    orc = Oracle(n, src, dst, X, model, W)
+    before = [rp.embeddings(l).clone() for l in range(4)]
+    ups = ups_array([(I.OP_ADD_EDGE, a, b) for a, b in todo[:250]])
+    with pytest.raises(ripple.RippleError) as ei:
+        rp.apply_batch(ups)
+    assert ei.value.status == ripple.ERR_CAPACITY
+    check_graph(rp, orc)
+    for l in range(4):
+        assert bool((rp.embeddings(l) == before[l]).all())
+    small = ups_array([(I.OP_ADD_EDGE, a, b) for a, b in todo[:3]])
+    rp.apply_batch(small)
+    assert orc.apply_incremental(small) == 0
+    check_graph(rp, orc)
+    check_values(rp, orc.full(), 3)
+    rp.close()
+
+
+def test_star_graph_mass_deletion_and_isolated_vertices(env):
+    """Degenerate structure: one hub pointing at everyone, most vertices without out-edges;
+    deleting most of the hub's edges in one batch exercises the tail logic of the row update."""
+    ripple, Oracle = env
+    n = 600
+    src = np.zeros(n - 1, dtype=np.int32)
+    dst = np.arange(1, n, dtype=np.int32)
+    model = I.sage_model([8, 12, 4], I.AGG_MEAN)
+    X = I.features(n, 8, 5)
+    W = I.make_weights(model, 5)
+    rp = ripple.Ripple(n, src, dst, X, model, W)
+    orc = Oracle(n, src, dst, X, model, W)
+    rng = np.random.default_rng(0)
+    victims = rng.permutation(np.arange(1, n))[:500]
+    ups = ups_array([(I.OP_DEL_EDGE, 0, int(v)) for v in victims] + [(I.OP_SET_FEATURE, 0, 0)])
+    rows = I.features(1, 8, 6)
+    rp.apply_batch(ups, rows)
+    assert orc.apply_incremental(ups, rows) == 0
+    check_graph(rp, orc)
+    check_frontiers(rp, orc, 2)
+    check_values(rp, orc.full(), 2)
+    # delete the rest: the graph becomes empty
+    rest = [int(v) for v in range(1, n) if v not in set(victims.tolist())]
+    ups = ups_array([(I.OP_DEL_EDGE, 0, v) for v in rest])
+    rp.apply_batch(ups)
+    assert orc.apply_incremental(ups) == 0
+    check_graph(rp, orc)
+    assert rp.stats()["num_edges"] == 0
+    check_values(rp, orc.full(), 2)
+    rp.recompute_full()
+    check_values(rp, orc.full(), 2)
+    rp.close()
+
+
+def test_recompute_full_matches_incremental_state(env):
+    ripple, Oracle = env
+    n, src, dst, X, model, W = _small(seed=47, name="gin_3l")
+    rp = ripple.Ripple(n, src, dst, X, model, W)
+    orc = Oracle(n, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 47)
+    for _ in range(10):
+        ups, rows = stream.next_batch(30)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+    inc = [rp.embeddings(l).clone() for l in range(4)]
+    rp.recompute_full()
+    ref = orc.full()
+    for l in range(4):
+        assert max_err(rp.embeddings(l).cpu().numpy(), ref[l]) <= TOL
+        assert max_err(inc[l].cpu().numpy(), ref[l]) <= TOL
+    rp.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# the named workloads
+# ---------------------------------------------------------------------------------------------
+def _run_workload(env, wname, batch, n_batches, check_every, scatter_mode=0, row_slack=0.0):
+    ripple, Oracle = env
+    w = I.workloads()[wname]
+    src, dst = I.make_graph(w)
+    X = I.features(w.n, w.model.dims[0], w.seed)
+    W = I.make_weights(w.model, w.seed)
+    L = len(w.model.layers)
+    rp = ripple.Ripple(w.n, src, dst, X, w.model, W, scatter_mode=scatter_mode)
+    orc = Oracle(w.n, src, dst, X, w.model, W)
+    stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], w.seed)
+    for b in range(n_batches):
+        ups, rows = stream.next_batch(batch)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        check_frontiers(rp, orc, L)
+        if b % check_every == check_every - 1:
+            check_graph(rp, orc)
+            check_values(rp, [orc.H(l) for l in range(L + 1)], L, row_slack=row_slack)
+    check_graph(rp, orc)
+    worst = check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)],
+                         row_slack=row_slack)
+    rp.close()
+    return worst
+
+
+@pytest.mark.parametrize("batch", [1, 10, 100, 1000])
+def test_sparse_config_100_consecutive_batches(env, batch):
+    _run_workload(env, "sparse", batch, 100, 25)
+
+
+@pytest.mark.parametrize("wname", ["sparse-deep-gin", "sparse-deep-gcn"])
+@pytest.mark.parametrize("batch", [100, 1000])
+def test_sparse_deep_configs_100_consecutive_batches(env, wname, batch):
+    _run_workload(env, wname, batch, 100, 50, row_slack=GIN_ROW_SLACK if "gin" in wname else 0.0)
