@@ -242,6 +242,7 @@ def run_ours(args, rank, world, local_rank):
             stage["update"] += s["ms_update"][l]
         pulls += s["scatter_pull"][L]
         sc_ms += s["ms_scatter_kernel"][L]
+        ld_last = s["message_width"][L]
         sc_bytes += scatter_bytes(s, L, ld_last)
         sizes["affected"] += np.array(s["affected"][: L + 1])
         sizes["active_edges"] += np.array(s["active_edges"][: L + 1])

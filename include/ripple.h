@@ -110,6 +110,9 @@ typedef struct {
     int32_t scatter_mode; /* ripple_scatter_mode: how delta messages reach the aggregates                   */
     int32_t gemm_mode;    /* ripple_gemm_mode: arithmetic of the affected-row layer update                  */
     int32_t timing;       /* non-zero: record per-stage CUDA-event times into ripple_stats                  */
+    int32_t pre_transform;/* 0: a layer narrower than its input applies its neighbour matrix to the sender
+                             rows before the scatter (messages and the cached aggregate then have the
+                             layer's output width); 1: never, aggregates always hold input-width rows    */
     int32_t device;       /* CUDA device ordinal, or -1 for the current device                              */
     void* stream;         /* cudaStream_t to run on (NULL: the library creates its own)                     */
 } ripple_options;
@@ -125,6 +128,7 @@ typedef struct {
     int64_t active_edges[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: edges carrying a message at hop l          */
     int32_t scatter_pull[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: 1 if hop l gathered over in-edges          */
     int64_t in_edges[RIPPLE_MAX_LAYERS + 1];      /* l = 1..L: in-edges of A_l (what a gather walks)      */
+    int32_t message_width[RIPPLE_MAX_LAYERS + 1]; /* l = 1..L: floats per message / aggregate row (padded) */
     int64_t pool_used, pool_size;                 /* overflow pool, edges, out-direction                  */
     /* CUDA-event times of the last batch in milliseconds (zero unless options.timing) */
     float ms_total, ms_graph;
@@ -158,8 +162,12 @@ ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update* ups, int6
 ripple_status ripple_get_embeddings(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld);
 
 /* The cached un-normalised aggregate S^layer (the persistent inbox of Sec. 3.3.2):
- * S_v = sum over in-neighbours u of c_u h^{layer-1}_u.  DEVICE, N x *ld, layer in 1..L. */
-ripple_status ripple_get_aggregate(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld);
+ * S_v = sum over in-neighbours u of c_u h^{layer-1}_u, or, if *transformed is set, of
+ * c_u W_n^T h^{layer-1}_u with W_n the layer's neighbour matrix (Wb for SAGE, Wa otherwise); see
+ * ripple_options.pre_transform.  DEVICE, N x *ld with *width meaningful columns, layer in 1..L.
+ * width and transformed may be NULL. */
+ripple_status ripple_get_aggregate(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld,
+                                   int32_t* width, int32_t* transformed);
 
 /* Trigger-based inference (Sec. 2.2): the vertices whose H^layer the last batch recomputed --
  * hop `layer` of the propagation tree (Sec. 3.3) -- as ascending ids.  DEVICE, layer in 0..L. */

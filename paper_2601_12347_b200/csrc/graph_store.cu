@@ -142,48 +142,61 @@ __global__ void k_classify(const ripple_update* __restrict__ ups, int n, int n_r
     ctl->abort = 1;
 }
 
-// position of x in row [base, base + deg), or -1; the whole warp calls this
-__device__ __forceinline__ int warp_find(const int32_t* __restrict__ col, int64_t base, int deg, int x) {
-    int found = -1;
-    for (int j0 = 0; j0 < deg; j0 += 32) {
-        int j = j0 + lane_id();
-        bool hit = j < deg && col[base + j] == x;
-        unsigned m = __ballot_sync(FULL, hit);
-        if (m) { found = j0 + __ffs(m) - 1; break; }
+// Position of x in row [base, base + deg), or -1; the whole block calls this.  Rows start on
+// 16-byte boundaries, so every thread compares four entries per load; a hub row of 150 K entries
+// costs a block of 256 threads about 150 iterations.
+__device__ __forceinline__ int block_find(const int32_t* __restrict__ col, int64_t base, int deg, int x,
+                                          volatile int* s_found) {
+    __syncthreads();
+    if (threadIdx.x == 0) *s_found = -1;
+    __syncthreads();
+    const int4* row4 = reinterpret_cast<const int4*>(col + base);
+    const int n4 = deg >> 2;
+    for (int q0 = 0; q0 < n4; q0 += blockDim.x) {
+        int q = q0 + threadIdx.x;
+        if (q < n4) {
+            int4 e = __ldg(row4 + q);
+            int hit = e.x == x ? 0 : e.y == x ? 1 : e.z == x ? 2 : e.w == x ? 3 : -1;
+            if (hit >= 0) *s_found = 4 * q + hit;
+        }
+        if ((q0 & (4 * blockDim.x - 1)) == 0 && *s_found >= 0) break;  // peek now and then
     }
-    return found;
+    int j = 4 * n4 + threadIdx.x;
+    if (j < deg && col[base + j] == x) *s_found = j;
+    __syncthreads();
+    return *s_found;
 }
 
-// One warp per op: winners are compared with the stored graph and become records or no-ops.
-__global__ void k_resolve(const ripple_update* __restrict__ ups, int n, Ctl* ctl,
-                          const int32_t* __restrict__ hseq, const int32_t* __restrict__ op_slot,
-                          const int32_t* __restrict__ feat_last, Side out, Side in, Rec* rec,
-                          uint32_t* bitmap) {
+// One block per op: winners are compared with the stored graph and become records or no-ops.
+__global__ void __launch_bounds__(256)
+k_resolve(const ripple_update* __restrict__ ups, int n, Ctl* ctl,
+          const int32_t* __restrict__ hseq, const int32_t* __restrict__ op_slot,
+          const int32_t* __restrict__ feat_last, Side out, Side in, Rec* rec,
+          uint32_t* bitmap) {
+    __shared__ int s_found;
     if (ctl->abort) return;
-    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    int nwarps = (gridDim.x * blockDim.x) >> 5;
-    for (int i = warp; i < n; i += nwarps) {
+    for (int i = blockIdx.x; i < n; i += gridDim.x) {
         ripple_update op = ups[i];
         if (op.op == RIPPLE_OP_SET_FEATURE) {
-            if (lane_id() == 0 && feat_last[op.u] == i) {
+            if (threadIdx.x == 0 && feat_last[op.u] == i) {
                 atomicAdd(&ctl->n_feat, 1);
                 atomicOr(&bitmap[op.u >> 5], 1u << (op.u & 31));
             }
             continue;
         }
         if (hseq[op_slot[i]] != i) {
-            if (lane_id() == 0) atomicAdd(&ctl->n_superseded, 1);
+            if (threadIdx.x == 0) atomicAdd(&ctl->n_superseded, 1);
             continue;
         }
-        int j_out = warp_find(out.col, out.start[op.u], out.deg[op.u], op.v);
+        int j_out = block_find(out.col, out.start[op.u], out.deg[op.u], op.v, &s_found);
         bool is_add = op.op == RIPPLE_OP_ADD_EDGE;
         if (is_add == (j_out >= 0)) {
-            if (lane_id() == 0) atomicAdd(is_add ? &ctl->n_noop_add : &ctl->n_noop_del, 1);
+            if (threadIdx.x == 0) atomicAdd(is_add ? &ctl->n_noop_add : &ctl->n_noop_del, 1);
             continue;
         }
         int j_in = -1;
-        if (!is_add) j_in = warp_find(in.col, in.start[op.v], in.deg[op.v], op.u);
-        if (lane_id() == 0) {
+        if (!is_add) j_in = block_find(in.col, in.start[op.v], in.deg[op.v], op.u, &s_found);
+        if (threadIdx.x == 0) {
             int r = atomicAdd(&ctl->n_rec, 1);
             atomicAdd(is_add ? &ctl->n_add : &ctl->n_del, 1);
             Rec x;
@@ -239,8 +252,7 @@ void graph_batch_classify(Ctx* c, int n, int n_rows) {
     const int T = 256;
     RP_LAUNCH(c, k_classify, div_up(n, T), T, 0, c->ups_dev, n, n_rows, c->N, c->ctl, c->hkeys, c->hseq,
               c->hsize - 1, c->op_slot, c->feat_last);
-    int warps_per_block = T / 32;
-    int grid = std::min(div_up(n, warps_per_block), c->n_sm * 8);
+    int grid = std::min(n, c->n_sm * 8);
     RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, n, c->ctl, c->hseq, c->op_slot, c->feat_last,
               c->side[0], c->side[1], c->rec, c->bitmap);
     RP_LAUNCH(c, k_plan_growth, std::min(div_up(2 * n, T), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[0],

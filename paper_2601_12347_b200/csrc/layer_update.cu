@@ -11,7 +11,7 @@ namespace rp {
 
 __device__ __forceinline__ float coef_deg(int deg) { return deg > 0 ? 1.0f / sqrtf((float)deg) : 0.0f; }
 
-enum { A_CONCAT = 0, A_SUM = 1, A_AGG = 2, A_DENSE = 3 };
+enum { A_CONCAT = 0, A_SUM = 1, A_AGG = 2, A_DENSE = 3, A_SELF = 4 };
 enum { EPI_COMMIT = 0, EPI_TEMP = 1 };
 
 struct UpdParams {
@@ -34,6 +34,7 @@ struct UpdParams {
     // epilogue
     float* Hout; int ld_o;          // COMMIT: rows by id; TEMP: compact rows
     float* Dout;                    // COMMIT: compact delta rows (may be null)
+    const float* addend; int ld_add; // rows by id added as row_scale * addend before bias (may be null)
     int src_norm;
     const int32_t* deg_out;
     const int32_t* deg_out_old;
@@ -85,6 +86,9 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
                 if (v >= 0 && k < p.K) {
                     if (p.a_mode == A_DENSE) {
                         a = *reinterpret_cast<const float4*>(p.Hprev + (size_t)(r0 + ar) * p.ld_h + k);
+                    } else if (p.a_mode == A_SELF) {
+                        float4 h = __ldg(reinterpret_cast<const float4*>(p.Hprev + (size_t)v * p.ld_h + k));
+                        a = make_float4(p.alpha * h.x, p.alpha * h.y, p.alpha * h.z, p.alpha * h.w);
                     } else if (p.a_mode == A_CONCAT) {
                         if (k < p.ld_h) a = __ldg(reinterpret_cast<const float4*>(p.Hprev + (size_t)v * p.ld_h + k));
                         else {
@@ -131,6 +135,11 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
                 const int lr = ty * TM + a2, v = row_id[lr];
                 if (v < 0) continue;
                 float4 h = make_float4(acc[a2][0] + bias.x, acc[a2][1] + bias.y, acc[a2][2] + bias.z, acc[a2][3] + bias.w);
+                if (p.addend) {
+                    float4 s = *reinterpret_cast<const float4*>(p.addend + (size_t)v * p.ld_add + col);
+                    float sc = row_scale[lr];
+                    h.x += sc * s.x; h.y += sc * s.y; h.z += sc * s.z; h.w += sc * s.w;
+                }
                 if (p.act == RIPPLE_ACT_RELU) { h.x = fmaxf(h.x, 0.f); h.y = fmaxf(h.y, 0.f); h.z = fmaxf(h.z, 0.f); h.w = fmaxf(h.w, 0.f); }
                 if (p.epi_mode == EPI_TEMP) {
                     *reinterpret_cast<float4*>(p.Hout + (size_t)(r0 + lr) * p.ld_o + col) = h;
@@ -154,38 +163,62 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
     }
 }
 
+// rows_out[i] = rows_in[i] * W_n for i < n: the neighbour part of layer l applied to compact rows
+// (sender deltas, record rows, or every embedding row at bootstrap)
+void neighbour_transform(Ctx* c, int l, const float* rows_in, int ld_rows, const int* n_dev, int n_host,
+                         float* rows_out) {
+    const LayerDev& ly = c->layer[l];
+    UpdParams p{};
+    p.list = nullptr; p.n_dev = n_dev; p.n_host = n_host;
+    p.a_mode = A_DENSE; p.epi_mode = EPI_TEMP;
+    p.Hprev = rows_in; p.ld_h = ld_rows;
+    p.K = ly.ld_in;
+    p.W = ly.kind == RIPPLE_LAYER_SAGE ? ly.W1 + (size_t)ly.ld_in * ly.ld_out : ly.W1;
+    p.ldw = c->ws[l]; p.bias = nullptr; p.n_cols = c->ws[l];
+    p.act = RIPPLE_ACT_IDENTITY; p.Hout = rows_out; p.ld_o = c->ws[l];
+    RP_LAUNCH(c, k_update_rows, c->n_sm * 4, 256, 0, c->ctl, p);
+}
+
 void update_rows(Ctx* c, int l, bool full) {
     const LayerDev& ly = c->layer[l];
+    const bool pre = c->pre[l];
     UpdParams p{};
     p.list = full ? nullptr : c->A[l];
     p.n_dev = full ? nullptr : &c->ctl->nA[l];
     p.n_host = c->N;
     p.Hprev = c->H[l - 1]; p.ld_h = c->ld[l - 1];
-    p.S = c->S[l]; p.ld_s = c->ld[l - 1];
+    p.S = c->S[l]; p.ld_s = c->ws[l];
+    p.alpha = 1.0f;
     p.agg = c->agg;
     p.deg_in = c->side[1].deg;
     p.src_norm = c->src_norm;
     p.deg_out = c->side[0].deg;
     p.deg_out_old = c->deg_out_old;
+    if (pre) { p.addend = c->S[l]; p.ld_add = c->ws[l]; }
     const int grid = c->n_sm * 4;
     if (ly.kind == RIPPLE_LAYER_GIN) {
         // hidden = relu(W1^T ((1 + eps) h + x) + b1), kept as compact rows
-        p.a_mode = A_SUM; p.epi_mode = EPI_TEMP; p.alpha = 1.0f + ly.eps;
+        p.a_mode = pre ? A_SELF : A_SUM; p.epi_mode = EPI_TEMP; p.alpha = 1.0f + ly.eps;
         p.K = ly.ld_in; p.W = ly.W1; p.ldw = ly.ld_hid; p.bias = ly.b1; p.n_cols = ly.ld_hid;
         p.act = RIPPLE_ACT_RELU; p.Hout = c->T; p.ld_o = ly.ld_hid; p.Dout = nullptr;
         RP_LAUNCH(c, k_update_rows, grid, 256, 0, c->ctl, p);
-        p.a_mode = A_DENSE; p.epi_mode = EPI_COMMIT;
+        p.a_mode = A_DENSE; p.epi_mode = EPI_COMMIT; p.addend = nullptr;
         p.Hprev = c->T; p.ld_h = ly.ld_hid;
         p.K = ly.ld_hid; p.W = ly.W2; p.ldw = ly.ld_out; p.bias = ly.b2; p.n_cols = ly.ld_out;
-        p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = full ? nullptr : c->D[l & 1];
+        p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = (full || l == c->L) ? nullptr : c->D[l & 1];  // the last hop sends nothing
         RP_LAUNCH(c, k_update_rows, grid, 256, 0, c->ctl, p);
         return;
     }
-    p.a_mode = ly.kind == RIPPLE_LAYER_SAGE ? A_CONCAT : A_AGG;
     p.epi_mode = EPI_COMMIT;
-    p.K = ly.kind == RIPPLE_LAYER_SAGE ? 2 * ly.ld_in : ly.ld_in;
+    if (ly.kind == RIPPLE_LAYER_SAGE) {
+        p.a_mode = pre ? A_SELF : A_CONCAT;
+        p.K = pre ? ly.ld_in : 2 * ly.ld_in;
+    } else {
+        p.a_mode = A_AGG;
+        p.K = pre ? 0 : ly.ld_in;   // transformed inbox: nothing left to multiply
+    }
     p.W = ly.W1; p.ldw = ly.ld_out; p.bias = ly.b1; p.n_cols = ly.ld_out;
-    p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = full ? nullptr : c->D[l & 1];
+    p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = (full || l == c->L) ? nullptr : c->D[l & 1];  // the last hop sends nothing
     RP_LAUNCH(c, k_update_rows, grid, 256, 0, c->ctl, p);
 }
 

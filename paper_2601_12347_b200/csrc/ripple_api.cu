@@ -63,7 +63,7 @@ static void destroy_ctx(Ctx* c) {
         cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->A[l]);
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
     }
-    cudaFree(c->T); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->posmap); cudaFree(c->deg_out_old);
+    cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hseq);
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
@@ -224,16 +224,26 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                 CK(cudaMemcpy(ly.b2, b2.data(), sizeof(float) * b2.size(), cudaMemcpyHostToDevice));
             }
         }
+        for (int l = 1; l <= L; ++l) {
+            // a layer narrower than its input transforms the few sender rows before the scatter
+            const LayerDev& ly = c->layer[l];
+            const int target = ly.kind == RIPPLE_LAYER_GIN ? ly.ld_hid : ly.ld_out;
+            c->pre[l] = o.pre_transform == 0 && target < ly.ld_in;
+            c->ws[l] = c->pre[l] ? target : ly.ld_in;
+        }
         for (int l = 0; l <= L; ++l) {
             max_ld = std::max(max_ld, c->ld[l]);
             CK(dev_alloc(&c->H[l], (size_t)N * c->ld[l], 0));
-            if (l > 0) CK(dev_alloc(&c->S[l], (size_t)N * c->ld[l - 1], 0));
+            if (l > 0) CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0));
             CK(dev_alloc(&c->A[l], (size_t)N + 32));
         }
         CK(cudaMemcpy2D(c->H[0], sizeof(float) * c->ld[0], features, sizeof(float) * c->d[0],
                         sizeof(float) * c->d[0], (size_t)N,
                         feat_mem == RIPPLE_MEM_DEVICE ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice));
         if (max_hid) CK(dev_alloc(&c->T, (size_t)N * max_hid));
+        CK(dev_alloc(&c->Dt, (size_t)N * max_ld));
+        CK(dev_alloc(&c->M, (size_t)o.max_batch * max_ld));
+        CK(dev_alloc(&c->Mt, (size_t)o.max_batch * max_ld));
         for (int s = 0; s < 2; ++s) {
             CK(dev_alloc(&c->D[s], (size_t)N * max_ld));
             CK(dev_alloc(&c->Clist[s], (size_t)N + 32));
@@ -347,6 +357,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
             s.active_edges[l] = l ? (int64_t)h.E[l] + h.n_rec : 0;
             s.scatter_pull[l] = h.pull[l];
             s.in_edges[l] = (int64_t)h.pull_work[l];
+            s.message_width[l] = l ? c->ws[l] : 0;
         }
         s.pool_used = (int64_t)h.pool_next[0] - c->side[0].base_end;
         s.pool_size = c->side[0].col_size - c->side[0].base_end;
@@ -377,11 +388,15 @@ extern "C" ripple_status ripple_get_embeddings(ripple_ctx* ctx, int32_t layer, c
     return RIPPLE_OK;
 }
 
-extern "C" ripple_status ripple_get_aggregate(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld) {
+extern "C" ripple_status ripple_get_aggregate(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld,
+                                              int32_t* width, int32_t* transformed) {
     Ctx* c = reinterpret_cast<Ctx*>(ctx);
     if (!c || !dev_ptr || !ld || layer < 1 || layer > c->L) return RIPPLE_ERR_INVALID_ARG;
     *dev_ptr = c->S[layer];
-    *ld = c->ld[layer - 1];
+    *ld = c->ws[layer];
+    const LayerDev& ly = c->layer[layer];
+    if (width) *width = c->pre[layer] ? (ly.kind == RIPPLE_LAYER_GIN ? ly.d_hid : ly.d_out) : ly.d_in;
+    if (transformed) *transformed = c->pre[layer] ? 1 : 0;
     return RIPPLE_OK;
 }
 

@@ -91,6 +91,11 @@ struct Ctx {
     float* S[RP_MAXL + 1];
     float* T;          // GIN hidden rows (compact, N x ld_hid)
     float* D[2];       // delta rows, ping-pong (compact, N x max ld)
+    float* Dt;         // delta rows after the neighbour transform (compact, N x max inbox width)
+    float* M;          // edge-record rows (compact, max_batch x max ld) and their transform
+    float* Mt;
+    bool pre[RP_MAXL + 1];   // layer applies its neighbour transform before the scatter
+    int ws[RP_MAXL + 1];     // row width (floats, padded) of S^l and of hop-l messages
     int32_t* A[RP_MAXL + 1];   // affected lists
     int32_t* Clist[2];         // sender list, ping-pong (A_l followed by extra sources)
     int64_t* coff;             // exclusive prefix of out-degrees over the sender list (+1)
@@ -154,6 +159,8 @@ void scatter_layer(Ctx* c, int l, int n);               // delta messages of hop
 
 // layer_update.cu
 void update_rows(Ctx* c, int l, bool full);             // re-apply Update^l + activation, emit deltas
+void neighbour_transform(Ctx* c, int l, const float* rows_in, int ld_rows, const int* n_dev, int n_host,
+                         float* rows_out);              // compact rows times the layer's neighbour matrix
 void feature_rows(Ctx* c, int n);                       // hop 0: overwrite feature rows, emit deltas
 void extra_sender_rows(Ctx* c, int l, int n);           // deltas of senders whose row did not change
 

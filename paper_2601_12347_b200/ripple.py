@@ -56,7 +56,7 @@ class _Options(ctypes.Structure):
     _fields_ = [("slack", ctypes.c_double), ("pool_edges", ctypes.c_int64),
                 ("max_batch", ctypes.c_int64), ("scatter_mode", ctypes.c_int32),
                 ("gemm_mode", ctypes.c_int32), ("timing", ctypes.c_int32),
-                ("device", ctypes.c_int32), ("stream", ctypes.c_void_p)]
+                ("pre_transform", ctypes.c_int32), ("device", ctypes.c_int32), ("stream", ctypes.c_void_p)]
 
 
 class _Stats(ctypes.Structure):
@@ -68,7 +68,7 @@ class _Stats(ctypes.Structure):
                 ("n_noop_add", ctypes.c_int64), ("n_noop_del", ctypes.c_int64),
                 ("n_superseded", ctypes.c_int64), ("n_feature", ctypes.c_int64),
                 ("affected", _A), ("senders", _A), ("active_edges", _A), ("scatter_pull", _I),
-                ("in_edges", _A),
+                ("in_edges", _A), ("message_width", _I),
                 ("pool_used", ctypes.c_int64), ("pool_size", ctypes.c_int64),
                 ("ms_total", ctypes.c_float), ("ms_graph", ctypes.c_float),
                 ("ms_frontier", _F), ("ms_scatter", _F), ("ms_update", _F),
@@ -94,7 +94,7 @@ def load_library(path: Optional[str] = None):
     lib.ripple_create.argtypes = [P(_Graph), vp, i32, P(_Layer), i32, i32, P(_Options), P(vp)]
     lib.ripple_apply_batch.argtypes = [vp, vp, i64, vp, i64, i32]
     lib.ripple_get_embeddings.argtypes = [vp, i32, P(vp), P(i64)]
-    lib.ripple_get_aggregate.argtypes = [vp, i32, P(vp), P(i64)]
+    lib.ripple_get_aggregate.argtypes = [vp, i32, P(vp), P(i64), P(i32), P(i32)]
     lib.ripple_get_affected.argtypes = [vp, i32, P(vp), P(i64)]
     lib.ripple_export_graph.argtypes = [vp, vp, vp, i64]
     lib.ripple_get_degrees.argtypes = [vp, P(vp), P(vp)]
@@ -136,11 +136,12 @@ class Ripple:
     def __init__(self, n: int, src, dst, features, model, weights: Sequence[Dict[str, np.ndarray]],
                  slack: float = 0.0, pool_edges: int = 0, max_batch: int = 0,
                  scatter_mode: int = SCATTER_AUTO, gemm_mode: int = GEMM_AUTO, timing: bool = False,
-                 stream=None):
+                 pre_transform: bool = True, stream=None):
         import torch
         self._torch = torch
         self.lib = load_library()
         self.n = int(n)
+        self.model, self.weights = model, weights
         self.L = len(model.layers)
         self.dims = [model.layers[0].d_in] + [l.d_out for l in model.layers]
         self.h = ctypes.c_void_p(None)
@@ -177,6 +178,7 @@ class Ripple:
         opt = _Options()
         opt.slack, opt.pool_edges, opt.max_batch = float(slack), int(pool_edges), int(max_batch)
         opt.scatter_mode, opt.gemm_mode, opt.timing = int(scatter_mode), int(gemm_mode), int(bool(timing))
+        opt.pre_transform = 0 if pre_transform else 1
         opt.device = torch.cuda.current_device()
         self._stream = stream if stream is not None else torch.cuda.Stream()
         opt.stream = self._stream.cuda_stream
@@ -250,7 +252,14 @@ class Ripple:
         return self._matrix(self.lib.ripple_get_embeddings, layer, self.dims[layer])
 
     def aggregate(self, layer: int):
-        return self._matrix(self.lib.ripple_get_aggregate, layer, self.dims[layer - 1])
+        """(tensor view N x width, transformed): the cached aggregate of `layer`; if transformed,
+        its rows are sums of W_n^T h_u instead of h_u."""
+        ptr, ld = ctypes.c_void_p(), ctypes.c_int64()
+        width, tr = ctypes.c_int32(), ctypes.c_int32()
+        self._check(self.lib.ripple_get_aggregate(self.h, layer, ctypes.byref(ptr), ctypes.byref(ld),
+                                                  ctypes.byref(width), ctypes.byref(tr)))
+        arr = _DevArray(ptr.value, (self.n, width.value), "<f4", strides=(4 * ld.value, 4), owner=self)
+        return self._torch.as_tensor(arr, device="cuda"), bool(tr.value)
 
     def affected(self, layer: int):
         ptr, cnt = ctypes.c_void_p(), ctypes.c_int64()
@@ -281,7 +290,7 @@ class Ripple:
                                           "n_noop_add", "n_noop_del", "n_superseded", "n_feature",
                                           "pool_used", "pool_size", "ms_total", "ms_graph",
                                           "ms_bootstrap", "gpu_launches")}
-        for k in ("affected", "senders", "active_edges", "scatter_pull", "in_edges", "ms_frontier", "ms_scatter",
+        for k in ("affected", "senders", "active_edges", "scatter_pull", "in_edges", "message_width", "ms_frontier", "ms_scatter",
                   "ms_update", "ms_scatter_kernel"):
             out[k] = list(getattr(s, k))[: L + 1]
         return out

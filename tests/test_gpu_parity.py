@@ -80,11 +80,16 @@ def check_values(rp, refH, L, refS=None, tol=TOL, row_slack=0.0):
         deg_in = rp.degrees()[1].cpu().numpy().astype(np.float64)
         scale = np.sqrt(np.maximum(deg_in, 1.0))[:, None]
         for l in range(1, L + 1):
-            got = rp.aggregate(l).cpu().numpy().astype(np.float64)
-            den = 1.0 + np.abs(refS[l])
+            view, transformed = rp.aggregate(l)
+            got = view.cpu().numpy().astype(np.float64)
+            want = refS[l]
+            if transformed:   # the library caches sum_u c_u W_n^T h_u for this layer
+                wl = rp.weights[l - 1]
+                want = want @ (wl["Wb"] if rp.model.layers[l - 1].kind == I.KIND_SAGE else wl["Wa"]).astype(np.float64)
+            den = 1.0 + np.abs(want)
             if row_slack:
-                den = den + (row_slack / TOL) * np.max(np.abs(refS[l]), axis=1, keepdims=True)
-            e = float(np.max(np.abs(got - refS[l]) / (den * scale)))
+                den = den + (row_slack / TOL) * np.max(np.abs(want), axis=1, keepdims=True)
+            e = float(np.max(np.abs(got - want) / (den * scale)))
             assert e <= tol, f"S^{l}: max scaled err {e}"
     return worst
 
@@ -97,6 +102,7 @@ def small_models():
         "gc_mean_3l": I.graphconv_model([18, 36, 20, 10], I.AGG_MEAN),
         "gcn_wsum_3l": I.graphconv_model([18, 36, 20, 10], I.AGG_WSUM_GCN),
         "gin_3l": I.gin_model(18, 24, 3, eps=0.25),
+        "gin_narrow_2l": I.gin_model(40, 16, 2, eps=0.1),
     }
 
 
@@ -131,7 +137,7 @@ def test_tiny_config_every_batch_against_full_recompute(env):
 
 
 @pytest.mark.parametrize("name", list(small_models().keys()))
-@pytest.mark.parametrize("mode", ["auto", "push", "pull"])
+@pytest.mark.parametrize("mode", ["auto", "push", "pull", "push-notransform"])
 def test_every_model_kind_and_scatter_direction(env, name, mode):
     ripple, Oracle = env
     model = small_models()[name]
@@ -146,8 +152,11 @@ def test_every_model_kind_and_scatter_direction(env, name, mode):
     dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
     X = I.features(n, model.dims[0], 3)
     W = I.make_weights(model, 3, zero_bias=False)
-    sm = {"auto": ripple.SCATTER_AUTO, "push": ripple.SCATTER_PUSH, "pull": ripple.SCATTER_PULL}[mode]
-    rp = ripple.Ripple(n, src, dst, X, model, W, scatter_mode=sm)
+    sm = {"auto": ripple.SCATTER_AUTO, "push": ripple.SCATTER_PUSH, "pull": ripple.SCATTER_PULL,
+          "push-notransform": ripple.SCATTER_PUSH}[mode]
+    rp = ripple.Ripple(n, src, dst, X, model, W, scatter_mode=sm, pre_transform=mode != "push-notransform")
+    narrowing = any((ly.d_hidden or ly.d_out) + 3 < ly.d_in for ly in model.layers)
+    assert any(rp.aggregate(l)[1] for l in range(1, L + 1)) == (narrowing and mode != "push-notransform")
     orc = Oracle(n, src, dst, X, model, W)
     stream = I.UpdateStream(n, src, dst, model.dims[0], 3)
     sizes = [1, 1, 2, 7, 33, 100, 1, 250, 64, 5] * 3
@@ -162,7 +171,7 @@ def test_every_model_kind_and_scatter_direction(env, name, mode):
     st = rp.stats()
     if mode == "pull":
         assert all(st["scatter_pull"][l] == 1 for l in range(1, L + 1))
-    if mode == "push":
+    if mode.startswith("push"):
         assert all(st["scatter_pull"][l] == 0 for l in range(1, L + 1))
     rp.close()
 
