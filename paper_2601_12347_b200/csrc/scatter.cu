@@ -266,14 +266,14 @@ __global__ void k_scatter_records(Ctl* ctl, const Rec* __restrict__ rec, const f
     }
 }
 
-// Direction of hop l, decided on the device.  Measured on the dense R-MAT graph (123.7 M edges,
-// rows of 256 floats): pushing 22 M messages takes 5.4 ms, gathering them over the 1.15 M
-// affected sinks' in-lists 6.0 ms, so pushing wins until the messages cover most of the in-edges
-// that a gather would walk anyway.
+// Direction of hop l, decided on the device.  Measured on the dense R-MAT graph (123.7 M edges):
+// pushing 22 M messages of 256 floats takes 5.4 ms where gathering them over the in-lists of the
+// 1.15 M affected sinks takes 6.0 ms, and on a saturated hop (122 M messages of 48 floats over
+// 123.7 M in-edges) pushing is several times faster than the gather, whose per-edge position
+// lookup and dependent row loads leave it latency-bound.  So the automatic choice is to push;
+// the gather stays selectable for comparison.
 __global__ void k_choose_direction(Ctl* ctl, int l, int mode) {
-    if (mode == RIPPLE_SCATTER_PULL) { ctl->pull[l] = 1; return; }
-    if (mode == RIPPLE_SCATTER_PUSH) { ctl->pull[l] = 0; return; }
-    ctl->pull[l] = ctl->E[l] > 0 && (double)ctl->E[l] > 0.6 * (double)ctl->pull_work[l];
+    ctl->pull[l] = mode == RIPPLE_SCATTER_PULL;
 }
 
 void scatter_layer(Ctx* c, int l, int n) {
@@ -302,7 +302,7 @@ void scatter_layer(Ctx* c, int l, int n) {
 #define PUSH(NV, LPR) RP_LAUNCH(c, (k_scatter_push<NV, LPR>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, ld, c->S[l])
 #define PULL(NV, LPR) RP_LAUNCH(c, (k_scatter_pull<NV, 32>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->posmap, Dm, ld, c->S[l])
     if (c->scatter_mode != RIPPLE_SCATTER_PULL) RP_WIDTH_DISPATCH(ld, PUSH);
-    if (c->scatter_mode != RIPPLE_SCATTER_PUSH) RP_WIDTH_DISPATCH(ld, PULL);
+    if (c->scatter_mode == RIPPLE_SCATTER_PULL) RP_WIDTH_DISPATCH(ld, PULL);
 #undef PUSH
 #undef PULL
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
