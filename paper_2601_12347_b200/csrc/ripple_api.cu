@@ -60,7 +60,7 @@ static void destroy_ctx(Ctx* c) {
         cudaFree(c->grow_list[s]); cudaFree(c->D[s]); cudaFree(c->Clist[s]);
     }
     for (int l = 0; l <= RP_MAXL; ++l) {
-        cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->A[l]);
+        cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->A[l]);
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
     }
     cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->posmap); cudaFree(c->deg_out_old);
@@ -234,7 +234,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         for (int l = 0; l <= L; ++l) {
             max_ld = std::max(max_ld, c->ld[l]);
             CK(dev_alloc(&c->H[l], (size_t)N * c->ld[l], 0));
-            if (l > 0) CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0));
+            if (l > 0) { CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0)); CK(dev_alloc(&c->dS[l], (size_t)N * c->ws[l], 0)); }
             CK(dev_alloc(&c->A[l], (size_t)N + 32));
         }
         CK(cudaMemcpy2D(c->H[0], sizeof(float) * c->ld[0], features, sizeof(float) * c->d[0],
@@ -322,6 +322,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
         STAMP();
         scatter_layer(c, l, nb);
         senders_release(c, l - 1);
+        fold_deltas(c, l);
         STAMP();
         update_rows(c, l, false);
         if (l < L) senders_build(c, l, nb);

