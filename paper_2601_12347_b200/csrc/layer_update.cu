@@ -1,44 +1,16 @@
 // Affected-row layer update (Compute + Prepare of Sec. 3.3.1): gather [h^{l-1}_v || x_v] for the
 // rows of A_l, multiply by the layer weights, add bias, apply the activation, write h^l_v in
 // place and emit the delta row D_v = c_new h_new - c_old h_old for the next hop (Sec. 3.3.3).
-// fp32 SIMT path: register-tiled GEMM whose A operand is gathered by row id.
-#include "device_utils.cuh"
-#include "ripple_internal.cuh"
+//
+// Two forms of the same contraction, chosen on the device from the row count:
+//   SIMT fp32    register-tiled GEMM whose A operand is gathered by row id (this file); used
+//                while the affected set is too small to be a real dense contraction;
+//   tensor core  tcgen05 TF32 with a 3-term split that keeps fp32 accuracy (layer_update_tc.cu).
+#include "layer_update.cuh"
 
 #include <algorithm>
 
 namespace rp {
-
-__device__ __forceinline__ float coef_deg(int deg) { return deg > 0 ? 1.0f / sqrtf((float)deg) : 0.0f; }
-
-enum { A_CONCAT = 0, A_SUM = 1, A_AGG = 2, A_DENSE = 3, A_SELF = 4 };
-enum { EPI_COMMIT = 0, EPI_TEMP = 1 };
-
-struct UpdParams {
-    const int32_t* list;  // row ids (null: identity)
-    const int* n_dev;     // row count on the device (null: n_host)
-    int n_host;
-    int a_mode, epi_mode;
-    // A operand
-    const float* Hprev; int ld_h;   // previous-layer rows (CONCAT, SUM) or dense rows (DENSE)
-    const float* S; int ld_s;       // aggregate rows
-    float alpha;                    // SUM: (1 + eps)
-    int agg;                        // sink-side normalisation
-    const int32_t* deg_in;
-    int K;                          // reduction length (CONCAT: 2 * ld_h)
-    // B operand
-    const float* W; int ldw;        // K x ldw
-    const float* bias;
-    int n_cols;                     // ldw (padded output width)
-    int act;
-    // epilogue
-    float* Hout; int ld_o;          // COMMIT: rows by id; TEMP: compact rows
-    float* Dout;                    // COMMIT: compact delta rows (may be null)
-    const float* addend; int ld_add; // rows by id added as row_scale * addend before bias (may be null)
-    int src_norm;
-    const int32_t* deg_out;
-    const int32_t* deg_out_old;
-};
 
 constexpr int BM = 64, BN = 64, BK = 16, TM = 4, TN = 4;
 
@@ -49,7 +21,8 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
     __shared__ __align__(16) float Bs[BK][BN];
     __shared__ int row_id[BM];
     __shared__ float row_scale[BM];
-    const int n = p.n_dev ? *p.n_dev : p.n_host;
+    const int n = upd_rows(p);
+    if (upd_use_tc(p, n)) return;
     const int row_tiles = (n + BM - 1) / BM, col_tiles = (p.n_cols + BN - 1) / BN;
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     for (int tile = blockIdx.x; tile < row_tiles * col_tiles; tile += gridDim.x) {
@@ -61,11 +34,7 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
             float sc = 0.f;
             if (i < n) {
                 v = p.list ? p.list[i] : i;
-                if (p.a_mode != A_DENSE) {
-                    sc = 1.0f;
-                    if (p.agg == RIPPLE_AGG_MEAN) { int d = p.deg_in[v]; sc = d > 0 ? 1.0f / (float)d : 0.f; }
-                    else if (p.agg == RIPPLE_AGG_WSUM_GCN) sc = coef_deg(p.deg_in[v]);
-                }
+                sc = upd_row_scale(p, v);
             }
             row_id[tid] = v;
             row_scale[tid] = sc;
@@ -83,29 +52,7 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
             float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
             {
                 const int v = row_id[ar], k = k0 + ak;
-                if (v >= 0 && k < p.K) {
-                    if (p.a_mode == A_DENSE) {
-                        a = *reinterpret_cast<const float4*>(p.Hprev + (size_t)(r0 + ar) * p.ld_h + k);
-                    } else if (p.a_mode == A_SELF) {
-                        float4 h = __ldg(reinterpret_cast<const float4*>(p.Hprev + (size_t)v * p.ld_h + k));
-                        a = make_float4(p.alpha * h.x, p.alpha * h.y, p.alpha * h.z, p.alpha * h.w);
-                    } else if (p.a_mode == A_CONCAT) {
-                        if (k < p.ld_h) a = __ldg(reinterpret_cast<const float4*>(p.Hprev + (size_t)v * p.ld_h + k));
-                        else {
-                            float4 s = *reinterpret_cast<const float4*>(p.S + (size_t)v * p.ld_s + (k - p.ld_h));
-                            float sc = row_scale[ar];
-                            a = make_float4(sc * s.x, sc * s.y, sc * s.z, sc * s.w);
-                        }
-                    } else {
-                        float4 s = *reinterpret_cast<const float4*>(p.S + (size_t)v * p.ld_s + k);
-                        float sc = row_scale[ar];
-                        a = make_float4(sc * s.x, sc * s.y, sc * s.z, sc * s.w);
-                        if (p.a_mode == A_SUM) {
-                            float4 h = __ldg(reinterpret_cast<const float4*>(p.Hprev + (size_t)v * p.ld_h + k));
-                            a.x += p.alpha * h.x; a.y += p.alpha * h.y; a.z += p.alpha * h.z; a.w += p.alpha * h.w;
-                        }
-                    }
-                }
+                if (v >= 0 && k < p.K) a = upd_load_a(p, v, r0 + ar, k, row_scale[ar]);
             }
             float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
             if (k0 + bk < p.K && c0 + bn < p.n_cols)
@@ -126,41 +73,31 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
                     for (int b2 = 0; b2 < TN; ++b2) acc[a2][b2] = fmaf(ar4[a2], br4[b2], acc[a2][b2]);
             }
         }
-        // epilogue
         const int col = c0 + tx * TN;
         if (col < p.n_cols) {
-            float4 bias = p.bias ? __ldg(reinterpret_cast<const float4*>(p.bias + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int a2 = 0; a2 < TM; ++a2) {
                 const int lr = ty * TM + a2, v = row_id[lr];
                 if (v < 0) continue;
-                float4 h = make_float4(acc[a2][0] + bias.x, acc[a2][1] + bias.y, acc[a2][2] + bias.z, acc[a2][3] + bias.w);
-                if (p.addend) {
-                    float4 s = *reinterpret_cast<const float4*>(p.addend + (size_t)v * p.ld_add + col);
-                    float sc = row_scale[lr];
-                    h.x += sc * s.x; h.y += sc * s.y; h.z += sc * s.z; h.w += sc * s.w;
-                }
-                if (p.act == RIPPLE_ACT_RELU) { h.x = fmaxf(h.x, 0.f); h.y = fmaxf(h.y, 0.f); h.z = fmaxf(h.z, 0.f); h.w = fmaxf(h.w, 0.f); }
-                if (p.epi_mode == EPI_TEMP) {
-                    *reinterpret_cast<float4*>(p.Hout + (size_t)(r0 + lr) * p.ld_o + col) = h;
-                } else {
-                    float4* dst = reinterpret_cast<float4*>(p.Hout + (size_t)v * p.ld_o + col);
-                    if (p.Dout) {
-                        float4 o = *dst;
-                        float cn = 1.f, co = 1.f;
-                        if (p.src_norm) {
-                            int dn = p.deg_out[v], dold = p.deg_out_old[v];
-                            cn = coef_deg(dn);
-                            co = dold >= 0 ? coef_deg(dold) : cn;
-                        }
-                        float4 d = make_float4(cn * h.x - co * o.x, cn * h.y - co * o.y, cn * h.z - co * o.z, cn * h.w - co * o.w);
-                        *reinterpret_cast<float4*>(p.Dout + (size_t)(r0 + lr) * p.ld_o + col) = d;
-                    }
-                    *dst = h;
-                }
+                upd_epilogue4(p, v, r0 + lr, col, make_float4(acc[a2][0], acc[a2][1], acc[a2][2], acc[a2][3]),
+                              row_scale[lr]);
             }
         }
     }
+}
+
+// launches both forms; exactly one of them does the work (decided on the device)
+static void launch_update(Ctx* c, UpdParams& p, const TcW& tw) {
+    p.tc_mode = TC_OFF;
+    // measured on the dense graph: the tensor-core form wins for wide outputs (256 columns: 5.5 ms
+    // against 9.8 ms SIMT) and loses for narrow ones, where staging latency dominates
+    if (tw.hi && c->gemm_mode != RIPPLE_GEMM_FP32 && p.K > 0 && tw.n_pad >= 128) {
+        p.tc_mode = c->gemm_mode == RIPPLE_GEMM_TF32 ? TC_TF32 : TC_TF32X3;
+        p.tc_min_rows = 1024;
+        p.Wt_hi = tw.hi; p.Wt_lo = tw.lo; p.k_pad = tw.k_pad; p.n_pad = tw.n_pad;
+    }
+    RP_LAUNCH(c, k_update_rows, c->n_sm * 4, 256, 0, c->ctl, p);
+    if (p.tc_mode != TC_OFF) launch_update_tc(c, p);
 }
 
 // rows_out[i] = rows_in[i] * W_n for i < n: the neighbour part of layer l applied to compact rows
@@ -176,7 +113,25 @@ void neighbour_transform(Ctx* c, int l, const float* rows_in, int ld_rows, const
     p.W = ly.kind == RIPPLE_LAYER_SAGE ? ly.W1 + (size_t)ly.ld_in * ly.ld_out : ly.W1;
     p.ldw = c->ws[l]; p.bias = nullptr; p.n_cols = c->ws[l];
     p.act = RIPPLE_ACT_IDENTITY; p.Hout = rows_out; p.ld_o = c->ws[l];
-    RP_LAUNCH(c, k_update_rows, c->n_sm * 4, 256, 0, c->ctl, p);
+    launch_update(c, p, ly.tc_nbr);
+}
+
+// Z^l_v = W_self^T h^{l-1}_v for the rows whose h^{l-1} changed (all rows at bootstrap).  A SAGE
+// layer that is narrower than its input keeps this self projection cached next to the transformed
+// aggregate, so that its affected-row update needs no contraction at all: the projection is
+// recomputed where the layer's input changed (A_{l-1}), not where its output is needed (A_l).
+void self_project(Ctx* c, int l, bool full) {
+    if (!c->Z[l]) return;
+    const LayerDev& ly = c->layer[l];
+    UpdParams p{};
+    p.list = full ? nullptr : c->A[l - 1];
+    p.n_dev = full ? nullptr : &c->ctl->nA[l - 1];
+    p.n_host = c->N;
+    p.a_mode = A_SELF; p.epi_mode = EPI_COMMIT; p.alpha = 1.0f;
+    p.Hprev = c->H[l - 1]; p.ld_h = c->ld[l - 1];
+    p.K = ly.ld_in; p.W = ly.W1; p.ldw = ly.ld_out; p.n_cols = ly.ld_out;
+    p.act = RIPPLE_ACT_IDENTITY; p.Hout = c->Z[l]; p.ld_o = ly.ld_out;
+    launch_update(c, p, ly.tc_main);
 }
 
 void update_rows(Ctx* c, int l, bool full) {
@@ -195,31 +150,32 @@ void update_rows(Ctx* c, int l, bool full) {
     p.deg_out = c->side[0].deg;
     p.deg_out_old = c->deg_out_old;
     if (pre) { p.addend = c->S[l]; p.ld_add = c->ws[l]; }
-    const int grid = c->n_sm * 4;
+    float* dout = (full || l == c->L) ? nullptr : c->D[l & 1];  // the last hop sends nothing
     if (ly.kind == RIPPLE_LAYER_GIN) {
         // hidden = relu(W1^T ((1 + eps) h + x) + b1), kept as compact rows
         p.a_mode = pre ? A_SELF : A_SUM; p.epi_mode = EPI_TEMP; p.alpha = 1.0f + ly.eps;
         p.K = ly.ld_in; p.W = ly.W1; p.ldw = ly.ld_hid; p.bias = ly.b1; p.n_cols = ly.ld_hid;
         p.act = RIPPLE_ACT_RELU; p.Hout = c->T; p.ld_o = ly.ld_hid; p.Dout = nullptr;
-        RP_LAUNCH(c, k_update_rows, grid, 256, 0, c->ctl, p);
+        launch_update(c, p, ly.tc_main);
         p.a_mode = A_DENSE; p.epi_mode = EPI_COMMIT; p.addend = nullptr;
         p.Hprev = c->T; p.ld_h = ly.ld_hid;
         p.K = ly.ld_hid; p.W = ly.W2; p.ldw = ly.ld_out; p.bias = ly.b2; p.n_cols = ly.ld_out;
-        p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = (full || l == c->L) ? nullptr : c->D[l & 1];  // the last hop sends nothing
-        RP_LAUNCH(c, k_update_rows, grid, 256, 0, c->ctl, p);
+        p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = dout;
+        launch_update(c, p, ly.tc_2);
         return;
     }
     p.epi_mode = EPI_COMMIT;
     if (ly.kind == RIPPLE_LAYER_SAGE) {
         p.a_mode = pre ? A_SELF : A_CONCAT;
-        p.K = pre ? ly.ld_in : 2 * ly.ld_in;
+        p.K = pre ? 0 : 2 * ly.ld_in;   // narrow layer: self projection and aggregate are both cached
+        if (pre) p.addend2 = c->Z[l];
     } else {
         p.a_mode = A_AGG;
         p.K = pre ? 0 : ly.ld_in;   // transformed inbox: nothing left to multiply
     }
     p.W = ly.W1; p.ldw = ly.ld_out; p.bias = ly.b1; p.n_cols = ly.ld_out;
-    p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = (full || l == c->L) ? nullptr : c->D[l & 1];  // the last hop sends nothing
-    RP_LAUNCH(c, k_update_rows, grid, 256, 0, c->ctl, p);
+    p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = dout;
+    launch_update(c, p, ly.tc_main);
 }
 
 // ---------------------------------------------------------------------------------------------

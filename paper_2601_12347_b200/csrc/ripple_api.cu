@@ -60,8 +60,9 @@ static void destroy_ctx(Ctx* c) {
         cudaFree(c->grow_list[s]); cudaFree(c->D[s]); cudaFree(c->Clist[s]);
     }
     for (int l = 0; l <= RP_MAXL; ++l) {
-        cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->A[l]);
+        cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->Z[l]); cudaFree(c->A[l]);
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
+        for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
     cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hseq);
@@ -91,6 +92,7 @@ static ripple_status run_full(Ctx* c) {
     if (c->timing) cudaEventRecord(c->ev[0], c->stream);
     for (int l = 1; l <= c->L; ++l) {
         spmm_full(c, l);
+        self_project(c, l, true);
         update_rows(c, l, true);
     }
     if (c->timing) cudaEventRecord(c->ev[1], c->stream);
@@ -213,6 +215,23 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                 b2 = padded_matrix(y.bb, 1, y.d_out, 1, ly.ld_out);
                 max_hid = std::max(max_hid, ly.ld_hid);
             }
+            {
+                // a layer narrower than its input transforms the few sender rows before the scatter
+                const int target = y.kind == RIPPLE_LAYER_GIN ? ly.ld_hid : ly.ld_out;
+                c->pre[l] = o.pre_transform == 0 && target < ly.ld_in;
+                c->ws[l] = c->pre[l] ? target : ly.ld_in;
+                if (o.gemm_mode != RIPPLE_GEMM_FP32) {   // transposed, tf32-split copies for the tensor-core form
+                    const float* wn = y.kind == RIPPLE_LAYER_SAGE ? w1.data() + (size_t)ly.ld_in * ly.ld_out : w1.data();
+                    if (y.kind == RIPPLE_LAYER_SAGE)
+                        CK(tc_weights_build(&ly.tc_main, w1.data(), c->pre[l] ? ly.ld_in : 2 * ly.ld_in, ly.ld_out));
+                    else if (y.kind == RIPPLE_LAYER_GIN)
+                        CK(tc_weights_build(&ly.tc_main, w1.data(), ly.ld_in, ly.ld_hid));
+                    else if (!c->pre[l])
+                        CK(tc_weights_build(&ly.tc_main, w1.data(), ly.ld_in, ly.ld_out));
+                    if (c->pre[l]) CK(tc_weights_build(&ly.tc_nbr, wn, ly.ld_in, c->ws[l]));
+                    if (y.kind == RIPPLE_LAYER_GIN) CK(tc_weights_build(&ly.tc_2, w2.data(), ly.ld_hid, ly.ld_out));
+                }
+            }
             CK(dev_alloc(&ly.W1, w1.size()));
             CK(cudaMemcpy(ly.W1, w1.data(), sizeof(float) * w1.size(), cudaMemcpyHostToDevice));
             CK(dev_alloc(&ly.b1, b1.size()));
@@ -224,17 +243,11 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                 CK(cudaMemcpy(ly.b2, b2.data(), sizeof(float) * b2.size(), cudaMemcpyHostToDevice));
             }
         }
-        for (int l = 1; l <= L; ++l) {
-            // a layer narrower than its input transforms the few sender rows before the scatter
-            const LayerDev& ly = c->layer[l];
-            const int target = ly.kind == RIPPLE_LAYER_GIN ? ly.ld_hid : ly.ld_out;
-            c->pre[l] = o.pre_transform == 0 && target < ly.ld_in;
-            c->ws[l] = c->pre[l] ? target : ly.ld_in;
-        }
         for (int l = 0; l <= L; ++l) {
             max_ld = std::max(max_ld, c->ld[l]);
             CK(dev_alloc(&c->H[l], (size_t)N * c->ld[l], 0));
-            if (l > 0) { CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0)); CK(dev_alloc(&c->dS[l], (size_t)N * c->ws[l], 0)); }
+            if (l > 0) { CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0)); CK(dev_alloc(&c->dS[l], (size_t)N * c->ws[l], 0));
+                         if (c->pre[l] && c->layer[l].kind == RIPPLE_LAYER_SAGE) CK(dev_alloc(&c->Z[l], (size_t)N * c->ws[l], 0)); }
             CK(dev_alloc(&c->A[l], (size_t)N + 32));
         }
         CK(cudaMemcpy2D(c->H[0], sizeof(float) * c->ld[0], features, sizeof(float) * c->d[0],
@@ -324,6 +337,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
         senders_release(c, l - 1);
         fold_deltas(c, l);
         STAMP();
+        self_project(c, l, false);
         update_rows(c, l, false);
         if (l < L) senders_build(c, l, nb);
         STAMP();

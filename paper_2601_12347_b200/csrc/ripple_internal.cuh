@@ -64,6 +64,13 @@ struct Rec {
     int32_t deg_out_old; // out-degree of u before the batch
 };
 
+// transposed (K contiguous), tf32-split copy of a weight block for the tensor-core layer update
+struct TcW {
+    float* hi;
+    float* lo;
+    int k_pad, n_pad;
+};
+
 struct LayerDev {
     int kind, d_in, d_hid, d_out, act;
     float eps;
@@ -72,6 +79,9 @@ struct LayerDev {
     float* b1;   // ld_out (SAGE, GRAPHCONV) or ld_hid (GIN)
     float* W2;   // GIN: d_hid x ld_out
     float* b2;   // GIN: ld_out
+    TcW tc_main; // weights of the affected-row GEMM (GIN: first matrix)
+    TcW tc_nbr;  // neighbour matrix, for layers that transform before the scatter
+    TcW tc_2;    // GIN: second matrix
 };
 
 struct Ctx {
@@ -89,6 +99,7 @@ struct Ctx {
     Side side[2];
     float* H[RP_MAXL + 1];
     float* S[RP_MAXL + 1];
+    float* Z[RP_MAXL + 1];    // cached self projection W_self^T h^{l-1} of narrow SAGE layers (N x ws), else null
     float* dS[RP_MAXL + 1];   // per-batch message accumulator, zero outside a batch (same shape as S)
     float* T;          // GIN hidden rows (compact, N x ld_hid)
     float* D[2];       // delta rows, ping-pong (compact, N x max ld)
@@ -161,9 +172,13 @@ void fold_deltas(Ctx* c, int l);                        // S^l += dS^l, dS^l = 0
 
 // layer_update.cu
 void update_rows(Ctx* c, int l, bool full);             // re-apply Update^l + activation, emit deltas
+void self_project(Ctx* c, int l, bool full);            // refresh the cached self projection of a narrow SAGE layer
 void neighbour_transform(Ctx* c, int l, const float* rows_in, int ld_rows, const int* n_dev, int n_host,
                          float* rows_out);              // compact rows times the layer's neighbour matrix
 void feature_rows(Ctx* c, int n);                       // hop 0: overwrite feature rows, emit deltas
 void extra_sender_rows(Ctx* c, int l, int n);           // deltas of senders whose row did not change
+
+// layer_update_tc.cu
+cudaError_t tc_weights_build(TcW* out, const float* W_host, int K, int ldw);
 
 }  // namespace rp
