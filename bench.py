@@ -318,8 +318,85 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_table(args):
+    """One JSON line per (workload, batch size): latency percentiles over 100 consecutive batches
+    through the C ABI from pinned host buffers, stage times, frontier sizes, the last hop's scatter
+    rate, and the oracle on a bounded sample of the same stream.  Feeds the table in the benchmark spec."""
+    import torch
+    from paper_2601_12347_b200 import build as B
+    from paper_2601_12347_b200 import ripple
+    B.build_library()
+    torch.cuda.set_device(0)
+    peak, peak_kind = load_peaks()
+    for name in args.table.split(","):
+        w, src, dst, X, W = make_workload(name, args.seed)
+        L = len(w.model.layers)
+        rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=16384, scatter_mode=args.scatter)
+        boot = rp.stats()["ms_bootstrap"]
+        stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], args.seed)
+        orc = ostream = None
+        if not args.no_cpu_baseline:
+            from oracle import oracle as O
+            O.build()
+            orc = O.Oracle(w.n, src, dst, X, w.model, W)
+            ostream = I.UpdateStream(w.n, src, dst, w.model.dims[0], args.seed)
+        for bsz in w.batch_sizes:
+            nb = args.table_batches
+            batches = [stream.next_batch(bsz) for _ in range(5 + nb)]
+            pinned = []
+            for ups, rows in batches:
+                u = torch.from_numpy(np.stack([ups["op"], ups["u"], ups["v"]], axis=1).astype(np.int32)).pin_memory()
+                pinned.append((u, torch.from_numpy(rows).pin_memory()))
+            lat, sc_ms, sc_bytes = [], 0.0, 0
+            stage = {"graph": 0.0, "frontier": 0.0, "scatter": 0.0, "update": 0.0}
+            aff, act = np.zeros(L + 1), np.zeros(L + 1)
+            for i, (u, r) in enumerate(pinned):
+                t0 = time.perf_counter()
+                rp.apply_batch(u, r)
+                dt = time.perf_counter() - t0
+                if i < 5:
+                    continue
+                lat.append(dt)
+                s = rp.stats()
+                stage["graph"] += s["ms_graph"]
+                for l in range(1, L + 1):
+                    stage["frontier"] += s["ms_frontier"][l]
+                    stage["scatter"] += s["ms_scatter"][l]
+                    stage["update"] += s["ms_update"][l]
+                sc_ms += s["ms_scatter_kernel"][L]
+                sc_bytes += scatter_bytes(s, L, s["message_width"][L])
+                aff += np.array(s["affected"][: L + 1])
+                act += np.array(s["active_edges"][: L + 1])
+            line = {"workload": name, "batch": bsz, "batches": nb,
+                    "updates_per_sec": bsz * nb / sum(lat),
+                    "latency_ms": {"mean": 1e3 * float(np.mean(lat)), "p50": 1e3 * pct(lat, 50), "p99": 1e3 * pct(lat, 99)},
+                    "stage_ms": {k: v / nb for k, v in stage.items()},
+                    "affected": (aff / nb).round(1).tolist(), "active_edges": (act / nb).round(1).tolist(),
+                    "last_hop_scatter": {"ms": sc_ms / nb, "algorithmic_GBps": (sc_bytes / 1e9) / (sc_ms / 1e3) if sc_ms else None,
+                                         "frac_of_" + peak_kind: ((sc_bytes / 1e9) / (sc_ms / 1e3) / peak) if sc_ms else None},
+                    "bootstrap_ms": boot}
+            if orc is not None:
+                spent, done = 0.0, 0
+                while spent < args.oracle_seconds and done < nb:
+                    ups, rows = ostream.next_batch(bsz)
+                    t0 = time.perf_counter()
+                    assert orc.apply_incremental(ups, rows) == 0
+                    spent += time.perf_counter() - t0
+                    done += 1
+                line["oracle"] = {"updates_per_sec": bsz * done / spent, "batches": done, "cores": O.num_threads()}
+            print(json.dumps(line), flush=True)
+        rp.close()
+        del rp
+        if orc is not None:
+            orc.close()
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--table", default="", help="comma-separated workloads: print one line per batch size")
+    ap.add_argument("--table-batches", type=int, default=100)
+    ap.add_argument("--oracle-seconds", type=float, default=10.0)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
@@ -334,7 +411,10 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.impl == "reference":
+    if args.table:
+        if rank == 0:
+            run_table(args)
+    elif args.impl == "reference":
         run_reference(args, rank, world)
     else:
         if world > 1 and rank != 0:

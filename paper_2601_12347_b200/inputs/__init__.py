@@ -387,6 +387,10 @@ def workloads() -> Dict[str, Workload]:
                                     (100, 1000), 100),
         "dense-2l": Workload("dense-2l", n_d, e_d, "rmat", sage_model([100, 256, 47]), 0,
                              (10, 100, 1000, 10000), 100),
+        # a smaller graph of the same kind and the same model as dense-2l: larger than L2, small
+        # enough to profile (a few GB on the device)
+        "mid-2l": Workload("mid-2l", 1_000_000, 30_000_000, "rmat", sage_model([100, 256, 47]), 0,
+                           (1000,), 20),
         "dense-3l": Workload("dense-3l", n_d, e_d, "rmat", sage_model([100, 256, 256, 47]), 0,
                              (10, 100, 1000, 10000), 100),
     }

@@ -39,11 +39,20 @@ def gin_row_slack(n_batches):
     return 3e-5 * float(np.sqrt(1.0 + n_batches))
 
 
-def max_err(got, ref, row_slack=0.0):
+# A second effect of the same stack: when an edge from a hub is deleted, its contribution (1e4 at
+# layer 2) is subtracted from the sink's cached aggregate; what remains of a now small row carries
+# the fp32 rounding of the removed term, eps32 * 1e4 = 1e-3 absolute, whatever the row's present
+# size (measured: 1.3e-3 on a layer-3 row whose largest entry is 0.36).  This is a property of
+# incremental subtraction in fp32, not of a kernel.  Bound: 16 * 2^-24 * max |H^{l-1}|, absolute.
+def gin_abs_slack(ref_prev):
+    return 16.0 * 2.0 ** -24 * float(np.max(np.abs(ref_prev)))
+
+
+def max_err(got, ref, row_slack=0.0, abs_slack=0.0):
     got = np.asarray(got, dtype=np.float64)
     if not ref.size:
         return 0.0
-    den = 1.0 + np.abs(ref)
+    den = 1.0 + np.abs(ref) + abs_slack / TOL
     if row_slack:
         den = den + (row_slack / TOL) * np.max(np.abs(ref), axis=1, keepdims=True)
     return float(np.max(np.abs(got - ref) / den))
@@ -78,7 +87,8 @@ def check_values(rp, refH, L, refS=None, tol=TOL, row_slack=0.0):
     lost or doubled message is an O(1) error and still fails)."""
     worst = 0.0
     for l in range(L + 1):
-        e = max_err(rp.embeddings(l).cpu().numpy(), refH[l], row_slack)
+        e = max_err(rp.embeddings(l).cpu().numpy(), refH[l], row_slack,
+                    gin_abs_slack(refH[l - 1]) if (row_slack and l > 0) else 0.0)
         assert e <= tol, f"H^{l}: max err {e}"
         worst = max(worst, e)
     if refS is not None:
@@ -94,6 +104,7 @@ def check_values(rp, refH, L, refS=None, tol=TOL, row_slack=0.0):
             den = 1.0 + np.abs(want)
             if row_slack:
                 den = den + (row_slack / TOL) * np.max(np.abs(want), axis=1, keepdims=True)
+                den = den + gin_abs_slack(refH[l - 1]) / TOL
             e = float(np.max(np.abs(got - want) / (den * scale)))
             assert e <= tol, f"S^{l}: max scaled err {e}"
     return worst
