@@ -177,6 +177,27 @@ ripple_status ripple_get_affected(ripple_ctx* ctx, int32_t layer, const int32_t*
  * col_capacity >= number of edges, ascending within each row).  For parity checks. */
 ripple_status ripple_export_graph(ripple_ctx* ctx, int64_t* rowptr, int32_t* col, int64_t col_capacity);
 
+/* The same canonical CSR as ripple_export_graph, for callers that must not allocate device
+ * memory.  (The paper has no counterpart: this is a property of this library, not of the method.)
+ * Who needs it: a process whose framework has already claimed all device memory for its own
+ * caching allocator, so that a cudaMalloc from this library would fail or force the framework to
+ * give memory back; or a caller on a latency budget that cannot afford the device-wide
+ * synchronisation an allocation or a free may imply.  ripple_export_graph obtains its staging
+ * buffers (a device copy of the row pointers and a packed copy of the column indices) with
+ * cudaMalloc on every call; this variant keeps them in fixed device arrays inside the library,
+ * about 10 MB that every GPU loading the library holds until the process exits, and calls no
+ * allocator at all.
+ * Limits: at most 262 144 vertices and 2 097 152 edges; a larger graph is rejected with
+ * RIPPLE_ERR_CAPACITY and the text says which limit was hit.
+ * The first call on each device looks up the addresses of the fixed arrays (a one-time set-up
+ * with that device current); make that first call before any stream capture begins.
+ * All calls on a device share the arrays, which keep whatever the previous call left in them
+ * (every call overwrites the part it reads, so nothing needs clearing); two calls whose GPU work
+ * overlaps -- from two contexts or two threads -- race on them: serialise such calls.
+ * Arguments, outputs and ordering are those of ripple_export_graph: rowptr HOST, N + 1 entries;
+ * col HOST, col_capacity >= number of edges, ascending within each row. */
+ripple_status ripple_export_graph_static(ripple_ctx* ctx, int64_t* rowptr, int32_t* col, int64_t col_capacity);
+
 /* Degree arrays of the current graph: DEVICE, N entries each. */
 ripple_status ripple_get_degrees(ripple_ctx* ctx, const int32_t** deg_out, const int32_t** deg_in);
 

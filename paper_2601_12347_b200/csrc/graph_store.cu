@@ -463,3 +463,106 @@ cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, int64_t col_capa
 }
 
 }  // namespace rp
+
+// ---------------------------------------------------------------------------------------------
+// allocation-free export
+// ---------------------------------------------------------------------------------------------
+// Same result as ripple_export_graph, for callers that must not allocate device memory.  The
+// staging that ripple_export_graph obtains with cudaMalloc on every call (a device copy of the
+// row pointers and a packed copy of the column indices) lives here in two file-scope device
+// arrays of fixed size.  Every GPU that loads the library carries them (about 10 MB) until the
+// process exits.  In host code the arrays' names are host-side stand-ins, not device addresses:
+// the addresses the kernel receives come from cudaGetSymbolAddress, taken once per device.
+#include <cstdio>
+#include <mutex>
+
+namespace rp {
+
+constexpr int64_t STATIC_MAX_VERTICES = 1 << 18;  // 262 144
+constexpr int64_t STATIC_MAX_EDGES = 1 << 21;     // 2 097 152
+
+static __device__ __align__(256) int64_t g_static_rowptr[STATIC_MAX_VERTICES + 1];
+static __device__ __align__(256) int32_t g_static_col[STATIC_MAX_EDGES];
+
+struct StaticScratch {
+    int64_t* rowptr = nullptr;
+    int32_t* col = nullptr;
+    bool ready = false;
+};
+constexpr int STATIC_MAX_DEVICES = 64;
+static StaticScratch g_static[STATIC_MAX_DEVICES];
+static std::mutex g_static_mu;
+
+// once per device, with that device current
+static cudaError_t static_scratch(int device, StaticScratch* out) {
+    if (device < 0 || device >= STATIC_MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    StaticScratch& s = g_static[device];
+    if (!s.ready) {
+        cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&s.rowptr), g_static_rowptr);
+        if (e != cudaSuccess) return e;
+        e = cudaGetSymbolAddress(reinterpret_cast<void**>(&s.col), g_static_col);
+        if (e != cudaSuccess) return e;
+        s.ready = true;
+    }
+    *out = s;
+    return cudaSuccess;
+}
+
+}  // namespace rp
+
+extern "C" ripple_status ripple_export_graph_static(ripple_ctx* ctx, int64_t* rowptr, int32_t* col,
+                                                    int64_t col_capacity) {
+    using namespace rp;
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !rowptr || (!col && col_capacity > 0)) return RIPPLE_ERR_INVALID_ARG;
+    const int N = c->N;
+    if (N > STATIC_MAX_VERTICES) {
+        snprintf(c->err, sizeof(c->err),
+                 "ripple_export_graph_static handles at most %lld vertices, the graph has %d; "
+                 "use ripple_export_graph", (long long)STATIC_MAX_VERTICES, N);
+        return RIPPLE_ERR_CAPACITY;
+    }
+    cudaError_t e = cudaSetDevice(c->device);
+    StaticScratch sc;
+    if (!e) e = static_scratch(c->device, &sc);
+    // degrees land in the tail of the caller's rowptr buffer and are widened in place, front to back
+    int32_t* deg = reinterpret_cast<int32_t*>(rowptr + N + 1) - N;
+    if (!e) e = cudaMemcpyAsync(deg, c->side[0].deg, sizeof(int32_t) * (size_t)N, cudaMemcpyDeviceToHost, c->stream);
+    if (!e) e = cudaStreamSynchronize(c->stream);
+    if (e) {
+        snprintf(c->err, sizeof(c->err), "ripple_export_graph_static: %s", cudaGetErrorString(e));
+        return RIPPLE_ERR_CUDA;
+    }
+    rowptr[0] = 0;
+    for (int v = 0; v < N; ++v) {
+        int64_t d = deg[v];
+        rowptr[v + 1] = rowptr[v] + d;
+    }
+    const int64_t E = rowptr[N];
+    if (E > STATIC_MAX_EDGES) {
+        snprintf(c->err, sizeof(c->err),
+                 "ripple_export_graph_static handles at most %lld edges, the graph has %lld; "
+                 "use ripple_export_graph", (long long)STATIC_MAX_EDGES, (long long)E);
+        return RIPPLE_ERR_CAPACITY;
+    }
+    if (E > col_capacity) {
+        snprintf(c->err, sizeof(c->err), "col_capacity %lld is smaller than the edge count %lld",
+                 (long long)col_capacity, (long long)E);
+        return RIPPLE_ERR_INVALID_ARG;
+    }
+    if (E == 0) return RIPPLE_OK;
+    e = cudaMemcpyAsync(sc.rowptr, rowptr, sizeof(int64_t) * ((size_t)N + 1), cudaMemcpyHostToDevice, c->stream);
+    if (!e) {
+        k_export_rows<<<c->n_sm * 8, 256, 0, c->stream>>>(N, c->side[0], sc.rowptr, sc.col);
+        e = cudaGetLastError();
+    }
+    if (!e) e = cudaMemcpyAsync(col, sc.col, sizeof(int32_t) * (size_t)E, cudaMemcpyDeviceToHost, c->stream);
+    if (!e) e = cudaStreamSynchronize(c->stream);
+    if (e) {
+        snprintf(c->err, sizeof(c->err), "ripple_export_graph_static: %s", cudaGetErrorString(e));
+        return RIPPLE_ERR_CUDA;
+    }
+    for (int v = 0; v < N; ++v) std::sort(col + rowptr[v], col + rowptr[v + 1]);
+    return RIPPLE_OK;
+}

@@ -30,6 +30,7 @@ UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
 EXPORTED = [
     "ripple_create", "ripple_apply_batch", "ripple_get_embeddings", "ripple_get_aggregate",
     "ripple_get_affected", "ripple_export_graph", "ripple_get_degrees", "ripple_recompute_full",
+    "ripple_export_graph_static",
     "ripple_get_stats", "ripple_last_error", "ripple_destroy", "ripple_version",
 ]
 
@@ -106,7 +107,8 @@ def load_library(path: Optional[str] = None):
     lib.ripple_destroy.restype = None
     lib.ripple_version.argtypes = []
     lib.ripple_version.restype = ctypes.c_char_p
-    for name in EXPORTED[:9]:
+    lib.ripple_export_graph_static.argtypes = [vp, vp, vp, i64]
+    for name in EXPORTED[:10]:
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -280,6 +282,21 @@ class Ripple:
         rowptr = np.zeros(self.n + 1, dtype=np.int64)
         col = np.zeros(max(e, 1), dtype=np.int32)
         self._check(self.lib.ripple_export_graph(self.h, rowptr.ctypes.data, col.ctypes.data, col.size))
+        return rowptr, col[: rowptr[-1]]
+
+    def export_graph_static(self) -> Tuple[np.ndarray, np.ndarray]:
+        """Same result as export_graph() through the entry point that allocates no device memory.
+
+        For processes in which every byte of device memory already belongs to a framework's
+        caching allocator, or callers that cannot afford the synchronisation an allocation may
+        imply.  Works for graphs of up to 262 144 vertices and 2 097 152 edges; larger graphs
+        raise RippleError (status ERR_CAPACITY).  The first call on a device performs a one-time
+        address look-up and should come before any stream capture; concurrent calls on one device
+        share the library's fixed staging arrays and must be serialised by the caller."""
+        e = self.stats()["num_edges"]
+        rowptr = np.zeros(self.n + 1, dtype=np.int64)
+        col = np.zeros(max(e, 1), dtype=np.int32)
+        self._check(self.lib.ripple_export_graph_static(self.h, rowptr.ctypes.data, col.ctypes.data, col.size))
         return rowptr, col[: rowptr[-1]]
 
     def stats(self) -> dict:
