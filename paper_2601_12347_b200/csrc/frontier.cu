@@ -167,7 +167,7 @@ __device__ __forceinline__ void set_bit(uint32_t* bitmap, int v) {
 
 constexpr int WALK_CHUNK = 256;  // edges per warp work item
 
-__global__ void k_mark_frontier(Ctl* ctl, int l, int self_term, const int32_t* __restrict__ senders,
+__global__ void k_mark_frontier(Ctl* ctl, int l, int self_term, int walk, const int32_t* __restrict__ senders,
                                 const int64_t* __restrict__ coff, Side out, const Rec* __restrict__ rec,
                                 const int32_t* __restrict__ A_prev, uint32_t* bitmap) {
     if (ctl->abort) return;
@@ -176,7 +176,8 @@ __global__ void k_mark_frontier(Ctl* ctl, int l, int self_term, const int32_t* _
     for (int i = gtid; i < ctl->n_rec; i += gsize) set_bit(bitmap, rec[i].v);
     if (self_term)
         for (int i = gtid; i < ctl->nA[l - 1]; i += gsize) set_bit(bitmap, A_prev[i]);
-    // out-neighbours of the senders of the previous hop
+    // out-neighbours of the senders of the previous hop (the push scatter marks them itself)
+    if (!walk) return;
     const int nC = ctl->nC[l - 1];
     if (nC == 0) return;
     const int64_t E = coff[nC];
@@ -202,10 +203,14 @@ void frontier_seed_features(Ctx* c, int n) {
     bitmap_to_list(c, c->A[0], &c->ctl->nA[0], nullptr);
 }
 
-void frontier_build(Ctx* c, int l, int n) {
-    (void)n;
-    RP_LAUNCH(c, k_mark_frontier, c->n_sm * 8, 256, 0, c->ctl, l, (int)c->self_term, c->Clist[(l - 1) & 1],
-              c->coff, c->side[0], c->rec, c->A[l - 1], c->bitmap);
+// Marks the members of A_l that do not come from walking the senders' out-lists (sinks of edge
+// changes, A_{l-1} for models with a self term) and, if `walk`, those that do.
+void frontier_mark(Ctx* c, int l, bool walk) {
+    RP_LAUNCH(c, k_mark_frontier, walk ? c->n_sm * 8 : c->n_sm * 2, 256, 0, c->ctl, l, (int)c->self_term,
+              (int)walk, c->Clist[(l - 1) & 1], c->coff, c->side[0], c->rec, c->A[l - 1], c->bitmap);
+}
+
+void frontier_compact(Ctx* c, int l) {
     bitmap_to_list(c, c->A[l], &c->ctl->nA[l], &c->ctl->pull_work[l]);
 }
 

@@ -149,7 +149,10 @@ void update_rows(Ctx* c, int l, bool full) {
     p.src_norm = c->src_norm;
     p.deg_out = c->side[0].deg;
     p.deg_out_old = c->deg_out_old;
-    if (pre) { p.addend = c->S[l]; p.ld_add = c->ws[l]; }
+    if (pre) {
+        p.addend = c->S[l]; p.ld_add = c->ws[l];
+        if (!full) { p.addend_rw = c->S[l]; p.addend_delta = c->dS[l]; }   // fold_deltas is skipped for these layers
+    }
     float* dout = (full || l == c->L) ? nullptr : c->D[l & 1];  // the last hop sends nothing
     if (ly.kind == RIPPLE_LAYER_GIN) {
         // hidden = relu(W1^T ((1 + eps) h + x) + b1), kept as compact rows
@@ -157,7 +160,7 @@ void update_rows(Ctx* c, int l, bool full) {
         p.K = ly.ld_in; p.W = ly.W1; p.ldw = ly.ld_hid; p.bias = ly.b1; p.n_cols = ly.ld_hid;
         p.act = RIPPLE_ACT_RELU; p.Hout = c->T; p.ld_o = ly.ld_hid; p.Dout = nullptr;
         launch_update(c, p, ly.tc_main);
-        p.a_mode = A_DENSE; p.epi_mode = EPI_COMMIT; p.addend = nullptr;
+        p.a_mode = A_DENSE; p.epi_mode = EPI_COMMIT; p.addend = nullptr; p.addend_rw = nullptr; p.addend_delta = nullptr;
         p.Hprev = c->T; p.ld_h = ly.ld_hid;
         p.K = ly.ld_hid; p.W = ly.W2; p.ldw = ly.ld_out; p.bias = ly.b2; p.n_cols = ly.ld_out;
         p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = dout;

@@ -36,6 +36,8 @@ struct UpdParams {
     float* Dout;                    // COMMIT: compact delta rows (may be null)
     const float* addend; int ld_add; // rows by id added as row_scale * addend (may be null)
     const float* addend2;           // rows by id added as they are, same leading dimension (may be null)
+    float* addend_rw;               // if set: addend with its pending per-batch sums folded in on the way
+    float* addend_delta;            //   (addend_rw += addend_delta, addend_delta = 0); replaces addend
     int src_norm;
     const int32_t* deg_out;
     const int32_t* deg_out_old;
@@ -85,7 +87,17 @@ __device__ __forceinline__ void upd_epilogue4(const UpdParams& p, int v, int i, 
         float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
         h.x += b.x; h.y += b.y; h.z += b.z; h.w += b.w;
     }
-    if (p.addend) {
+    if (p.addend_rw) {
+        // every (row, column) of the aggregate is touched by exactly one thread, so the batch's
+        // message sums can be folded into it here instead of in a pass of their own
+        float4* sp = reinterpret_cast<float4*>(p.addend_rw + (size_t)v * p.ld_add + col);
+        float4* dp = reinterpret_cast<float4*>(p.addend_delta + (size_t)v * p.ld_add + col);
+        float4 s = *sp, d = *dp;
+        s.x += d.x; s.y += d.y; s.z += d.z; s.w += d.w;
+        *sp = s;
+        *dp = make_float4(0.f, 0.f, 0.f, 0.f);
+        h.x += sc * s.x; h.y += sc * s.y; h.z += sc * s.z; h.w += sc * s.w;
+    } else if (p.addend) {
         float4 s = *reinterpret_cast<const float4*>(p.addend + (size_t)v * p.ld_add + col);
         h.x += sc * s.x; h.y += sc * s.y; h.z += sc * s.z; h.w += sc * s.w;
     }

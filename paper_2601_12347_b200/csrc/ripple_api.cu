@@ -331,9 +331,14 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
     STAMP();  // 1
     // one superstep per hop (Sec. 3.3.1): frontier, send + aggregate, compute + prepare
     for (int l = 1; l <= L; ++l) {
-        frontier_build(c, l, nb);
+        // the push scatter walks the same out-lists as the frontier and marks the sinks itself; the
+        // gather needs the list first
+        const bool pull = c->scatter_mode == RIPPLE_SCATTER_PULL;
+        frontier_mark(c, l, pull);
+        if (pull) frontier_compact(c, l);
         STAMP();
         scatter_layer(c, l, nb);
+        if (!pull) frontier_compact(c, l);
         senders_release(c, l - 1);
         fold_deltas(c, l);
         STAMP();

@@ -161,7 +161,8 @@ cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, int64_t col_capa
 void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, const int32_t* deg,
                   int64_t* out, unsigned long long* total_dev);
 void frontier_seed_features(Ctx* c, int n);             // A_0 from the batch's feature updates
-void frontier_build(Ctx* c, int l, int n);              // A_l from C_{l-1}, edge records, A_{l-1}
+void frontier_mark(Ctx* c, int l, bool walk);           // bitmap of A_l: edge-record sinks, A_{l-1}, and (walk) Out(C_{l-1})
+void frontier_compact(Ctx* c, int l);                   // bitmap -> ascending list A_l
 void senders_build(Ctx* c, int l, int n);               // C_l, posmap, coff, E_{l+1}
 void senders_release(Ctx* c, int l);                    // clear posmap entries of C_l
 

@@ -120,7 +120,7 @@ constexpr int PUSH_CHUNK = 64;  // edges per warp work item
 template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_scatter_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64_t* __restrict__ coff,
-               Side out, const float* __restrict__ D, int ld, float* S) {
+               Side out, const float* __restrict__ D, int ld, float* S, uint32_t* bitmap) {
     if (ctl->abort || ctl->pull[l]) return;
     const int nC = ctl->nC[l - 1];
     if (nC == 0) return;
@@ -158,6 +158,11 @@ k_scatter_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64
                         for (int k = 0; k < NV; ++k) {
                             int q = ql + LPR * k;
                             if (q < nq) red_add_v4(dst + 4 * q, d[k]);
+                        }
+                        // the sink joins the hop's affected set (same walk as the frontier's)
+                        if (ql == 0) {
+                            const uint32_t m = 1u << (v & 31);
+                            if (!(bitmap[v >> 5] & m)) atomicOr(&bitmap[v >> 5], m);
                         }
                     }
                 }
@@ -300,6 +305,7 @@ __global__ void k_fold_deltas(Ctl* ctl, int l, const int32_t* __restrict__ A, in
 }
 
 void fold_deltas(Ctx* c, int l) {
+    if (c->pre[l]) return;   // transformed aggregates are folded inside the row update's epilogue
     RP_LAUNCH(c, k_fold_deltas, c->n_sm * 8, 256, 0, c->ctl, l, c->A[l], c->ws[l], c->S[l], c->dS[l]);
 }
 
@@ -326,7 +332,7 @@ void scatter_layer(Ctx* c, int l, int n) {
         }
     }
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
-#define PUSH(NV, LPR) RP_LAUNCH(c, (k_scatter_push<NV, LPR>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, ld, c->dS[l])
+#define PUSH(NV, LPR) RP_LAUNCH(c, (k_scatter_push<NV, LPR>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, ld, c->dS[l], c->bitmap)
 #define PULL(NV, LPR) RP_LAUNCH(c, (k_scatter_pull<NV, 32>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->posmap, Dm, ld, c->dS[l])
     if (c->scatter_mode != RIPPLE_SCATTER_PULL) RP_WIDTH_DISPATCH(ld, PUSH);
     if (c->scatter_mode == RIPPLE_SCATTER_PULL) RP_WIDTH_DISPATCH(ld, PULL);
