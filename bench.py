@@ -116,6 +116,23 @@ def scatter_bytes(stats, l, ld):
     return stats["senders"][l - 1] * (4 * ld + 8) + 4 * e + e * 8 * ld
 
 
+def max_over_ranks(values_ms, world, device="cuda"):
+    """Every rank's timings replaced by the maximum over ranks (the job is as slow as its slowest
+    replica).  No-op for one rank."""
+    if world <= 1:
+        return list(values_ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values_ms), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_rate(world, batch, steps, ms):
+    """Updates per second of the whole job: every replica processed batch * steps updates."""
+    return world * batch * steps / (ms / 1e3)
+
+
 def make_workload(name, seed):
     w = I.workloads()[name]
     w.seed = seed
@@ -133,7 +150,7 @@ def run_reference(args, rank, world):
     O.build()
     w, src, dst, X, W = make_workload(args.workload, args.seed)
     orc = O.Oracle(w.n, src, dst, X, w.model, W)
-    stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], w.seed)
+    stream = I.make_stream(w, src, dst)
     lat = []
     for s in range(args.warmup + args.steps):
         ups, rows = stream.next_batch(args.batch)
@@ -167,7 +184,7 @@ def cpu_baseline(args, w, src, dst, X, W, budget_s=20.0):
     t0 = time.perf_counter()
     orc = O.Oracle(w.n, src, dst, X, w.model, W)
     setup = time.perf_counter() - t0
-    stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], w.seed)
+    stream = I.make_stream(w, src, dst)
     spent, nb = 0.0, 0
     while spent < budget_s and nb < 50:
         ups, rows = stream.next_batch(args.batch)
@@ -196,7 +213,7 @@ def run_ours(args, rank, world, local_rank):
     rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=max(args.batch, 16),
                        scatter_mode=args.scatter)
     bootstrap_ms = rp.stats()["ms_bootstrap"]
-    stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], seed)
+    stream = I.make_stream(w, src, dst, seed)
     K, Wm = args.steps, args.warmup
     batches = [stream.next_batch(args.batch) for _ in range(Wm + 2 * K)]
 
@@ -268,10 +285,7 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    if world > 1:
-        t = torch.tensor([dev_ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dev_ms, e2e_ms = float(t[0]), float(t[1])
+    dev_ms, e2e_ms = max_over_ranks([dev_ms, e2e_ms], world)
     if rank != 0:
         rp.close()
         if world > 1:
@@ -288,7 +302,7 @@ def run_ours(args, rank, world, local_rank):
                 "ms_per_launch": sc_ms / K,
                 "algorithmic_bytes_per_launch": sc_bytes / K}
     line = {
-        "metric": METRIC, "value": world * args.batch * K / (dev_ms / 1e3), "unit": UNIT,
+        "metric": METRIC, "value": whole_job_rate(world, args.batch, K, dev_ms), "unit": UNIT,
         "n_gpus": world, "steps": K, "warmup": Wm, "ms_per_step": dev_ms / K,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
@@ -297,7 +311,7 @@ def run_ours(args, rank, world, local_rank):
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                    "l2": "working set (aggregate and embedding rows, GBs) far larger than L2; no flush needed"},
         "clocks": clocks,
-        "e2e": {"value": world * args.batch * K / (e2e_ms / 1e3), "unit": UNIT,
+        "e2e": {"value": whole_job_rate(world, args.batch, K, e2e_ms), "unit": UNIT,
                 "h2d_bytes_per_step": h2d // K, "d2h_bytes_per_step": d2h // K},
         "gpu_launches": int(launches),
         "latency_ms": {"p50": 1e3 * pct(lat, 50), "p99": 1e3 * pct(lat, 99), "mean": 1e3 * float(np.mean(lat)),
@@ -333,13 +347,15 @@ def run_table(args):
         L = len(w.model.layers)
         rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=16384, scatter_mode=args.scatter)
         boot = rp.stats()["ms_bootstrap"]
-        stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], args.seed)
+        rp.recompute_full()   # warm: the recompute-everything alternative on the same state
+        full_ms = rp.stats()["ms_bootstrap"]
+        stream = I.make_stream(w, src, dst, args.seed)
         orc = ostream = None
         if not args.no_cpu_baseline:
             from oracle import oracle as O
             O.build()
             orc = O.Oracle(w.n, src, dst, X, w.model, W)
-            ostream = I.UpdateStream(w.n, src, dst, w.model.dims[0], args.seed)
+            ostream = I.make_stream(w, src, dst, args.seed)
         for bsz in w.batch_sizes:
             nb = args.table_batches
             batches = [stream.next_batch(bsz) for _ in range(5 + nb)]
@@ -374,7 +390,7 @@ def run_table(args):
                     "affected": (aff / nb).round(1).tolist(), "active_edges": (act / nb).round(1).tolist(),
                     "last_hop_scatter": {"ms": sc_ms / nb, "algorithmic_GBps": (sc_bytes / 1e9) / (sc_ms / 1e3) if sc_ms else None,
                                          "frac_of_" + peak_kind: ((sc_bytes / 1e9) / (sc_ms / 1e3) / peak) if sc_ms else None},
-                    "bootstrap_ms": boot}
+                    "bootstrap_ms": boot, "full_recompute_ms": full_ms}
             if orc is not None:
                 spent, done = 0.0, 0
                 while spent < args.oracle_seconds and done < nb:

@@ -62,6 +62,8 @@ def _load():
     lib.orc_export_csr.restype = None
     lib.orc_row_from_prev.argtypes = [vp, i32, i32, vp, i64, vp, vp]
     lib.orc_row_from_prev.restype = None
+    lib.orc_apply_structure.argtypes = [vp, vp, i64, i64]
+    lib.orc_apply_structure.restype = i32
     lib.orc_num_threads.argtypes = []
     lib.orc_num_threads.restype = i32
     _lib = lib
@@ -130,6 +132,11 @@ class Oracle:
 
     def apply_scoped(self, ups, feat_rows=None) -> int:
         return self._apply(self.lib.orc_apply_scoped, ups, feat_rows)
+
+    def apply_structure(self, ups, n_rows: int) -> int:
+        """Graph state and affected sets only (no embedding arithmetic; H and S go stale)."""
+        ups = np.ascontiguousarray(ups, dtype=UPDATE_DTYPE)
+        return int(self.lib.orc_apply_structure(self.h, ups.ctypes.data, ups.size, int(n_rows)))
 
     def bootstrap(self):
         self.lib.orc_bootstrap(self.h)

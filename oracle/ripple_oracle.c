@@ -581,6 +581,35 @@ int orc_apply_scoped(oracle_t *o, const update_t *ups, int64_t n, const float *f
     return 0;
 }
 
+/* Graph state and affected sets only: Apply (Sec. 3.3) and the hops of the propagation tree, with
+ * no embedding arithmetic.  The cached H / S are NOT maintained by this call; it exists so that a
+ * test can follow the structure of a large graph batch by batch and check single rows against
+ * the definition with orc_row_from_prev. */
+int orc_apply_structure(oracle_t *o, const update_t *ups, int64_t n, int64_t n_rows) {
+    delta_t dl;
+    int rc = normalise(o, ups, n, n_rows, &dl);
+    if (rc) return rc;
+    int L = o->L, self_term = o->layer[1].kind != KIND_GRAPHCONV;
+    apply_topology(o, &dl);
+    int nA = dl.nF;
+    int *A = (int *)malloc(sizeof(int) * (size_t)(nA + 1));
+    memcpy(A, dl.F, sizeof(int) * (size_t)nA);
+    set_list(o, 0, A, nA);
+    int nC; int *C = changed_senders(o, &dl, A, nA, &nC);
+    for (int l = 1; l <= L; ++l) {
+        int nAn; long walked;
+        int *An = next_affected(o, &dl, C, nC, A, nA, self_term, &nAn, &walked);
+        o->active_edges[l] = walked + dl.n_add + dl.n_del;
+        set_list(o, l, An, nAn);
+        free(A); free(C);
+        A = An; nA = nAn;
+        C = changed_senders(o, &dl, A, nA, &nC);
+    }
+    free(A); free(C);
+    delta_free(&dl);
+    return 0;
+}
+
 /* One row of one layer from a caller-supplied previous-layer matrix (fp32, leading dimension
  * ld) over the oracle's current graph: h^l_v by Eq. 1-2.  Lets a test check any single row of a
  * large state against the definition without recomputing the whole graph. */

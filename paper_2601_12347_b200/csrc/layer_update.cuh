@@ -81,8 +81,18 @@ __device__ __forceinline__ float4 upd_load_a(const UpdParams& p, int v, int i, i
     return a;
 }
 
-// bias, optional addend, activation, then either a compact temp row or commit + delta row
-__device__ __forceinline__ void upd_epilogue4(const UpdParams& p, int v, int i, int col, float4 h, float sc) {
+// true if the epilogue needs the row's previous value (to emit a delta row)
+__device__ __forceinline__ bool upd_needs_old(const UpdParams& p) { return p.epi_mode == EPI_COMMIT && p.Dout; }
+
+__device__ __forceinline__ float4 upd_load_old(const UpdParams& p, int v, int col) {
+    return *reinterpret_cast<const float4*>(p.Hout + (size_t)v * p.ld_o + col);
+}
+
+// bias, optional addend, activation, then either a compact temp row or commit + delta row;
+// `old` is the previously stored value if the caller has prefetched it (has_old)
+__device__ __forceinline__ void upd_epilogue4(const UpdParams& p, int v, int i, int col, float4 h, float sc,
+                                              bool has_old = false,
+                                              float4 old = make_float4(0.f, 0.f, 0.f, 0.f)) {
     if (p.bias) {
         float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
         h.x += b.x; h.y += b.y; h.z += b.z; h.w += b.w;
@@ -114,7 +124,7 @@ __device__ __forceinline__ void upd_epilogue4(const UpdParams& p, int v, int i, 
     }
     float4* dst = reinterpret_cast<float4*>(p.Hout + (size_t)v * p.ld_o + col);
     if (p.Dout) {
-        float4 o = *dst;
+        float4 o = has_old ? old : *dst;
         float cn = 1.f, co = 1.f;
         if (p.src_norm) {
             int dold = p.deg_out_old[v];

@@ -232,6 +232,18 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
             const int b0 = half ? split : 0, b1 = half ? nblk : split;
             const int r = 32 * g + lane, v = row_id[r];
             const float sc = row_scale[r];
+            // the previous values of the row (needed for the delta) are fetched one block ahead, so
+            // that their latency hides behind the tensor-memory load and the stores of the block
+            // before
+            const bool need_old = upd_needs_old(p) && v >= 0;
+            float4 old_cur[4], old_nxt[4];
+            if (need_old && b0 < b1) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int col = b0 * 16 + 4 * q;
+                    if (col < p.n_cols) old_cur[q] = upd_load_old(p, v, col);
+                }
+            }
             for (int blk = b0; blk < b1; ++blk) {
                 uint32_t x[16];
                 const uint32_t taddr = tmem_base + ((uint32_t)(32 * g) << 16) + (uint32_t)(blk * 16);
@@ -242,6 +254,13 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                       "=r"(x[7]), "=r"(x[8]), "=r"(x[9]), "=r"(x[10]), "=r"(x[11]), "=r"(x[12]), "=r"(x[13]),
                       "=r"(x[14]), "=r"(x[15])
                     : "r"(taddr) : "memory");
+                if (need_old && blk + 1 < b1) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int col = (blk + 1) * 16 + 4 * q;
+                        if (col < p.n_cols) old_nxt[q] = upd_load_old(p, v, col);
+                    }
+                }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (v >= 0) {
 #pragma unroll
@@ -251,9 +270,11 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                             upd_epilogue4(p, v, r0 + r, col,
                                           make_float4(__uint_as_float(x[4 * q]), __uint_as_float(x[4 * q + 1]),
                                                       __uint_as_float(x[4 * q + 2]), __uint_as_float(x[4 * q + 3])),
-                                          sc);
+                                          sc, need_old, old_cur[q]);
                     }
                 }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) old_cur[q] = old_nxt[q];
             }
         }
         tc_fence_before();

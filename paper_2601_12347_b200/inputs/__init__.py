@@ -391,9 +391,26 @@ def workloads() -> Dict[str, Workload]:
         # enough to profile (a few GB on the device)
         "mid-2l": Workload("mid-2l", 1_000_000, 30_000_000, "rmat", sage_model([100, 256, 47]), 0,
                            (1000,), 20),
+        "mid-3l": Workload("mid-3l", 1_000_000, 30_000_000, "rmat", sage_model([100, 256, 256, 47]), 0,
+                           (1000,), 20),
         "dense-3l": Workload("dense-3l", n_d, e_d, "rmat", sage_model([100, 256, 256, 47]), 0,
                              (10, 100, 1000, 10000), 100),
+        # hub stress: every endpoint is one of the top-1 % out-degree vertices of the initial graph
+        "dense-3l-hub-feature": Workload("dense-3l-hub-feature", n_d, e_d, "rmat",
+                                         sage_model([100, 256, 256, 47]), 0, (1, 10, 100, 1000), 20,
+                                         {"hubs": True, "mix": (0.0, 0.0, 1.0)}),
+        "dense-3l-hub-delete": Workload("dense-3l-hub-delete", n_d, e_d, "rmat",
+                                        sage_model([100, 256, 256, 47]), 0, (1, 10, 100, 1000), 20,
+                                        {"hubs": True, "mix": (0.1, 0.8, 0.1)}),
     }
+
+
+def make_stream(w: Workload, src: np.ndarray, dst: np.ndarray, seed: Optional[int] = None,
+                stream: str = "updates") -> "UpdateStream":
+    """The update stream of a named workload (hub-restricted for the hub-stress workloads)."""
+    hubs = top_out_degree(w.n, src) if w.extra.get("hubs") else None
+    return UpdateStream(w.n, src, dst, w.model.dims[0], w.seed if seed is None else seed, stream=stream,
+                        mix=w.extra.get("mix", (0.4, 0.4, 0.2)), hubs=hubs)
 
 
 def make_graph(w: Workload) -> Tuple[np.ndarray, np.ndarray]:

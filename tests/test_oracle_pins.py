@@ -527,3 +527,28 @@ def test_tiny_config_invariant_10_batches():
             assert rel_err(o.H(l), full[l]) < 1e-9
         sizes = [o.affected(l).size for l in range(3)]
         assert sizes[0] <= sizes[1] <= sizes[2] <= w.n
+
+
+def test_structure_only_route_matches_incremental_route():
+    """orc_apply_structure follows graph and affected sets exactly like the incremental route."""
+    for name in ("sage_mean", "gcn_wsum"):
+        model = all_models()[name]
+        n, m = 80, 500
+        src, dst = random_graph(n, m, 3)
+        X = I.features(n, model.dims[0], 3)
+        W = I.make_weights(model, 3)
+        a = Oracle(n, src, dst, X, model, W)
+        b = Oracle(n, src, dst, X, model, W, bootstrap=False)
+        stream = I.UpdateStream(n, src, dst, model.dims[0], 3)
+        for _ in range(8):
+            ups, rows = stream.next_batch(15)
+            assert a.apply_incremental(ups, rows) == 0
+            assert b.apply_structure(ups, rows.shape[0]) == 0
+            for l in range(len(model.layers) + 1):
+                assert np.array_equal(a.affected(l), b.affected(l))
+            for l in range(1, len(model.layers) + 1):
+                assert a.active_edges(l) == b.active_edges(l)
+            assert a.counts() == b.counts()
+            ra, ca = a.export_csr()
+            rb, cb = b.export_csr()
+            assert np.array_equal(ra, rb) and np.array_equal(ca, cb)
