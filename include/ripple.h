@@ -113,6 +113,7 @@ typedef struct {
     int32_t pre_transform;/* 0: a layer narrower than its input applies its neighbour matrix to the sender
                              rows before the scatter (messages and the cached aggregate then have the
                              layer's output width); 1: never, aggregates always hold input-width rows    */
+    int32_t no_graphs;    /* non-zero: never replay small batches (<= 512 updates) as a captured CUDA graph     */
     int32_t device;       /* CUDA device ordinal, or -1 for the current device                              */
     void* stream;         /* cudaStream_t to run on (NULL: the library creates its own)                     */
 } ripple_options;
@@ -207,6 +208,10 @@ ripple_status ripple_recompute_full(ripple_ctx* ctx);
 
 /* Counters and timings of the last batch (HOST struct, filled by the call). */
 ripple_status ripple_get_stats(ripple_ctx* ctx, ripple_stats* out);
+
+/* Switches the per-stage CUDA-event timing of ripple_stats on or off.  While it is on, small
+ * batches are launched kernel by kernel instead of as a captured graph. */
+ripple_status ripple_set_timing(ripple_ctx* ctx, int32_t on);
 
 /* Text of the last error on ctx (or of the last failed ripple_create if ctx is NULL). */
 const char* ripple_last_error(ripple_ctx* ctx);

@@ -103,7 +103,7 @@ cudaError_t graph_build(Ctx* c, const int32_t* src, const int32_t* dst, int64_t 
 // ---------------------------------------------------------------------------------------------
 // batch normalisation
 // ---------------------------------------------------------------------------------------------
-__global__ void k_classify(const ripple_update* __restrict__ ups, int n, int n_rows, int N, Ctl* ctl,
+__global__ void k_classify(const ripple_update* __restrict__ ups, int n, int N, Ctl* ctl,
                            unsigned long long* hkeys, int32_t* hseq, int hmask, int32_t* op_slot,
                            int32_t* feat_last) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -116,7 +116,7 @@ __global__ void k_classify(const ripple_update* __restrict__ ups, int n, int n_r
         return;
     }
     bool bad = (unsigned)op.u >= (unsigned)N;
-    if (op.op == RIPPLE_OP_SET_FEATURE) bad |= (unsigned)op.v >= (unsigned)n_rows;
+    if (op.op == RIPPLE_OP_SET_FEATURE) bad |= (unsigned)op.v >= (unsigned)ctl->n_rows;
     else bad |= (unsigned)op.v >= (unsigned)N;
     if (bad) {
         atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_VERTEX_RANGE);
@@ -247,10 +247,10 @@ __global__ void k_plan_check(Ctl* ctl, long long col_size_out, long long col_siz
     }
 }
 
-void graph_batch_classify(Ctx* c, int n, int n_rows) {
+void graph_batch_classify(Ctx* c, int n) {
     if (n <= 0) return;
     const int T = 256;
-    RP_LAUNCH(c, k_classify, div_up(n, T), T, 0, c->ups_dev, n, n_rows, c->N, c->ctl, c->hkeys, c->hseq,
+    RP_LAUNCH(c, k_classify, div_up(n, T), T, 0, c->ups_dev, n, c->N, c->ctl, c->hkeys, c->hseq,
               c->hsize - 1, c->op_slot, c->feat_last);
     int grid = std::min(n, c->n_sm * 8);
     RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, n, c->ctl, c->hseq, c->op_slot, c->feat_last,

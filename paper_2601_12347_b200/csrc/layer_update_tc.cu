@@ -299,12 +299,16 @@ void launch_update_tc(Ctx* c, const UpdParams& p) {
     const int per_sm = std::max<size_t>(1, std::min<size_t>(4, (size_t)(220 * 1024) / (smem + 2048)));
     const int grid = c->n_sm * per_sm;
     if (x3) {
-        cudaFuncSetAttribute(k_update_rows_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         RP_LAUNCH(c, k_update_rows_tc<true>, grid, TC_THREADS, smem, c->ctl, p);
     } else {
-        cudaFuncSetAttribute(k_update_rows_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         RP_LAUNCH(c, k_update_rows_tc<false>, grid, TC_THREADS, smem, c->ctl, p);
     }
+}
+
+void tc_prepare() {
+    const int max_smem = 2 * 2 * (TC_A_BYTES + 256 * 128) + 1024;
+    cudaFuncSetAttribute(k_update_rows_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    cudaFuncSetAttribute(k_update_rows_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
 }
 
 // Transposed, K-contiguous, tf32-split copy of a row-major K x ldw weight block.

@@ -39,13 +39,16 @@ static cudaError_t dev_alloc(T** p, size_t count, int fill_byte = -2) {
     return e;
 }
 
-__global__ void k_ctl_reset(Ctl* ctl, int n_ops) {
+// params[0] = number of ops, params[1] = number of payload rows (device memory, so that a captured
+// launch chain can be replayed for batches that differ in them)
+__global__ void k_ctl_reset(Ctl* ctl, const int* params) {
     unsigned long long keep0 = ctl->pool_next[0], keep1 = ctl->pool_next[1];
     Ctl z;
     memset(&z, 0, sizeof(Ctl));
     z.pool_next[0] = keep0;
     z.pool_next[1] = keep1;
-    z.n_ops = n_ops;
+    z.n_ops = params[0];
+    z.n_rows = params[1];
     *ctl = z;
 }
 
@@ -68,6 +71,9 @@ static void destroy_ctx(Ctx* c) {
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hseq);
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
+    if (c->params_host) cudaFreeHost(c->params_host);
+    cudaFree(c->params_dev);
+    for (auto& g : c->graph_exec) if (g) cudaGraphExecDestroy(g);
     for (auto& e : c->ev) if (e) cudaEventDestroy(e);
     for (auto& e : c->ev_sc) if (e) cudaEventDestroy(e);
     if (c->own_stream && c->stream) cudaStreamDestroy(c->stream);
@@ -88,7 +94,9 @@ static ripple_status sync_and_fetch_ctl(Ctx* c) {
 // full layer-wise inference over the current graph (Eq. 1-2): bootstrap and recompute-all
 static ripple_status run_full(Ctx* c) {
     c->launches = 0;
-    RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, 0);
+    c->params_host[0] = 0; c->params_host[1] = 0;
+    cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream);
+    RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
     if (c->timing) cudaEventRecord(c->ev[0], c->stream);
     for (int l = 1; l <= c->L; ++l) {
         spmm_full(c, l);
@@ -161,6 +169,10 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         c->self_term = layers[0].kind != RIPPLE_LAYER_GRAPHCONV;
         c->src_norm = agg == RIPPLE_AGG_WSUM_GCN;
         CK(dev_alloc(&c->ctl, 1, 0));
+        CK(dev_alloc(&c->params_dev, 2, 0));
+        CK(cudaMallocHost(&c->params_host, 2 * sizeof(int)));
+        c->no_graphs = o.no_graphs;
+        tc_prepare();
         CK(cudaMallocHost(&c->ctl_host, sizeof(Ctl)));
         memset(c->ctl_host, 0, sizeof(Ctl));
         c->n_words = (N + 31) / 32;
@@ -292,38 +304,15 @@ fail_keep_msg:
     return st;
 }
 
-extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update* ups, int64_t n,
-                                            const float* feat_rows, int64_t n_rows, int32_t mem) {
-    Ctx* c = reinterpret_cast<Ctx*>(ctx);
-    if (!c) return RIPPLE_ERR_INVALID_ARG;
-    ripple_status st = RIPPLE_OK;
-    if (n < 0 || n_rows < 0 || (n > 0 && !ups) || (n_rows > 0 && !feat_rows) || (mem != 0 && mem != 1)) {
-        set_err(c, "bad arguments to ripple_apply_batch");
-        return RIPPLE_ERR_INVALID_ARG;
-    }
-    if (n > c->max_batch || n_rows > c->max_batch) {
-        set_err(c, "batch of %lld updates exceeds max_batch = %lld", (long long)n, (long long)c->max_batch);
-        return RIPPLE_ERR_CAPACITY;
-    }
-    cudaSetDevice(c->device);
-    const int nb = (int)n, nr = (int)n_rows, L = c->L;
-    ripple_update* own_ups = c->ups_dev;
-    float* own_feat = c->feat_dev;
-    c->launches = 0;
+// The launch chain of one batch: no host decision inside, every size read on the device.
+static int enqueue_batch(Ctx* c, int nb, bool stamps) {
+    const int L = c->L;
     int evi = 0;
-#define STAMP() do { if (c->timing) cudaEventRecord(c->ev[evi], c->stream); ++evi; } while (0)
-    if (mem == RIPPLE_MEM_HOST) {
-        if (nb) CK(cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, cudaMemcpyHostToDevice, c->stream));
-        if (nr) CK(cudaMemcpyAsync(c->feat_dev, feat_rows, sizeof(float) * (size_t)nr * c->d[0], cudaMemcpyHostToDevice, c->stream));
-    } else {
-        // device inputs are used in place
-        c->ups_dev = const_cast<ripple_update*>(ups);
-        c->feat_dev = const_cast<float*>(feat_rows);
-    }
-    RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, nb);
+#define STAMP() do { if (stamps) cudaEventRecord(c->ev[evi], c->stream); ++evi; } while (0)
+    RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
     STAMP();  // 0
     // Apply (Sec. 3.3): normalise the batch, mutate both adjacency directions, replace features
-    graph_batch_classify(c, nb, nr);
+    graph_batch_classify(c, nb);
     graph_batch_mutate(c, nb);
     frontier_seed_features(c, nb);
     feature_rows(c, nb);
@@ -350,6 +339,70 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
     graph_batch_cleanup(c, nb);
     STAMP();
 #undef STAMP
+    return evi;
+}
+
+// Small batches are launch-bound (about fifty short kernels): their chain is captured once per
+// batch size into a CUDA graph and replayed.  Returns false if this batch must take the direct path.
+static bool launch_batch_graph(Ctx* c, int nb) {
+    if (c->no_graphs || c->timing || nb < 1 || nb > RP_GRAPH_MAX_BATCH) return false;
+    int slot = -1;
+    for (int i = 0; i < RP_GRAPH_SLOTS; ++i)
+        if (c->graph_exec[i] && c->graph_n[i] == nb) slot = i;
+    if (slot < 0) {
+        slot = c->graph_next++ % RP_GRAPH_SLOTS;
+        if (c->graph_exec[slot]) { cudaGraphExecDestroy(c->graph_exec[slot]); c->graph_exec[slot] = nullptr; }
+        cudaGraph_t g = nullptr;
+        if (cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) { c->no_graphs = 1; return false; }
+        c->launches = 0;
+        enqueue_batch(c, nb, false);
+        cudaError_t e = cudaStreamEndCapture(c->stream, &g);
+        if (e == cudaSuccess) e = cudaGraphInstantiate(&c->graph_exec[slot], g, 0);
+        if (g) cudaGraphDestroy(g);
+        if (e != cudaSuccess) { cudaGetLastError(); c->graph_exec[slot] = nullptr; c->no_graphs = 1; return false; }
+        c->graph_n[slot] = nb;
+        c->graph_launches[slot] = c->launches;
+    }
+    c->launches = c->graph_launches[slot];
+    return cudaGraphLaunch(c->graph_exec[slot], c->stream) == cudaSuccess;
+}
+
+extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update* ups, int64_t n,
+                                            const float* feat_rows, int64_t n_rows, int32_t mem) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c) return RIPPLE_ERR_INVALID_ARG;
+    ripple_status st = RIPPLE_OK;
+    if (n < 0 || n_rows < 0 || (n > 0 && !ups) || (n_rows > 0 && !feat_rows) || (mem != 0 && mem != 1)) {
+        set_err(c, "bad arguments to ripple_apply_batch");
+        return RIPPLE_ERR_INVALID_ARG;
+    }
+    if (n > c->max_batch || n_rows > c->max_batch) {
+        set_err(c, "batch of %lld updates exceeds max_batch = %lld", (long long)n, (long long)c->max_batch);
+        return RIPPLE_ERR_CAPACITY;
+    }
+    cudaSetDevice(c->device);
+    const int nb = (int)n, nr = (int)n_rows, L = c->L;
+    ripple_update* own_ups = c->ups_dev;
+    float* own_feat = c->feat_dev;
+    c->launches = 0;
+    int evi = 0;
+    const bool try_graph = !c->no_graphs && !c->timing && nb >= 1 && nb <= RP_GRAPH_MAX_BATCH;
+    const cudaMemcpyKind kind = mem == RIPPLE_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+    if (mem == RIPPLE_MEM_HOST || try_graph) {
+        // a replayed graph reads the library's own staging buffers, so device inputs are copied too
+        if (nb) CK(cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, kind, c->stream));
+        if (nr) CK(cudaMemcpyAsync(c->feat_dev, feat_rows, sizeof(float) * (size_t)nr * c->d[0], kind, c->stream));
+    } else {
+        // device inputs are used in place
+        c->ups_dev = const_cast<ripple_update*>(ups);
+        c->feat_dev = const_cast<float*>(feat_rows);
+    }
+    c->params_host[0] = nb; c->params_host[1] = nr;
+    CK(cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream));
+    if (!try_graph || !launch_batch_graph(c, nb)) {
+        c->launches = 0;
+        evi = enqueue_batch(c, nb, c->timing != 0);
+    }
     c->ups_dev = own_ups;
     c->feat_dev = own_feat;
     st = sync_and_fetch_ctl(c);
@@ -461,6 +514,13 @@ extern "C" ripple_status ripple_get_stats(ripple_ctx* ctx, ripple_stats* out) {
     Ctx* c = reinterpret_cast<Ctx*>(ctx);
     if (!c || !out) return RIPPLE_ERR_INVALID_ARG;
     *out = c->stats;
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_set_timing(ripple_ctx* ctx, int32_t on) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c) return RIPPLE_ERR_INVALID_ARG;
+    c->timing = on ? 1 : 0;
     return RIPPLE_OK;
 }
 

@@ -13,6 +13,8 @@
 
 #define RP_MAXL RIPPLE_MAX_LAYERS
 #define RP_TOMB (-1)
+#define RP_GRAPH_MAX_BATCH 512   // batches up to this size replay a captured launch chain
+#define RP_GRAPH_SLOTS 8
 
 namespace rp {
 
@@ -22,6 +24,7 @@ struct Ctl {
     int err;     // ripple_status recorded on the device
     int err_info;
     int n_ops;
+    int n_rows;  // payload rows of the batch
     int n_rec;   // net edge changes of the batch (|dE+| + |dE-|)
     int n_add, n_del, n_noop_add, n_noop_del, n_superseded, n_feat;
     int n_grow[2];
@@ -130,6 +133,13 @@ struct Ctx {
     // scan scratch
     int64_t* tile_sums;
     int n_tile_sums;
+    int* params_dev;   // {n_ops, n_rows} of the batch being applied
+    int* params_host;  // pinned
+    int no_graphs;
+    cudaGraphExec_t graph_exec[RP_GRAPH_SLOTS];
+    int graph_n[RP_GRAPH_SLOTS];
+    int64_t graph_launches[RP_GRAPH_SLOTS];
+    int graph_next;
     Ctl* ctl;        // device
     Ctl* ctl_host;   // pinned
     ripple_stats stats;
@@ -152,7 +162,7 @@ inline int pad4(int x) { return (x + 3) & ~3; }
 // graph_store.cu
 cudaError_t graph_build(Ctx* c, const int32_t* src_dev, const int32_t* dst_dev, int64_t E,
                         double slack, int64_t pool_edges);
-void graph_batch_classify(Ctx* c, int n, int n_rows);   // validate, dedupe, find net changes, plan
+void graph_batch_classify(Ctx* c, int n);   // validate, dedupe, find net changes, plan
 void graph_batch_mutate(Ctx* c, int n);                 // apply the net changes to both directions
 void graph_batch_cleanup(Ctx* c, int n);                // reset per-batch scratch
 cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, int64_t col_capacity, int64_t* n_edges);
@@ -181,5 +191,6 @@ void extra_sender_rows(Ctx* c, int l, int n);           // deltas of senders who
 
 // layer_update_tc.cu
 cudaError_t tc_weights_build(TcW* out, const float* W_host, int K, int ldw);
+void tc_prepare();   // one-time kernel attributes (not allowed inside a stream capture)
 
 }  // namespace rp

@@ -30,7 +30,7 @@ UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
 EXPORTED = [
     "ripple_create", "ripple_apply_batch", "ripple_get_embeddings", "ripple_get_aggregate",
     "ripple_get_affected", "ripple_export_graph", "ripple_get_degrees", "ripple_recompute_full",
-    "ripple_export_graph_static",
+    "ripple_export_graph_static", "ripple_set_timing",
     "ripple_get_stats", "ripple_last_error", "ripple_destroy", "ripple_version",
 ]
 
@@ -57,7 +57,7 @@ class _Options(ctypes.Structure):
     _fields_ = [("slack", ctypes.c_double), ("pool_edges", ctypes.c_int64),
                 ("max_batch", ctypes.c_int64), ("scatter_mode", ctypes.c_int32),
                 ("gemm_mode", ctypes.c_int32), ("timing", ctypes.c_int32),
-                ("pre_transform", ctypes.c_int32), ("device", ctypes.c_int32), ("stream", ctypes.c_void_p)]
+                ("pre_transform", ctypes.c_int32), ("no_graphs", ctypes.c_int32), ("device", ctypes.c_int32), ("stream", ctypes.c_void_p)]
 
 
 class _Stats(ctypes.Structure):
@@ -108,7 +108,8 @@ def load_library(path: Optional[str] = None):
     lib.ripple_version.argtypes = []
     lib.ripple_version.restype = ctypes.c_char_p
     lib.ripple_export_graph_static.argtypes = [vp, vp, vp, i64]
-    for name in EXPORTED[:10]:
+    lib.ripple_set_timing.argtypes = [vp, i32]
+    for name in EXPORTED[:11]:
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -138,7 +139,7 @@ class Ripple:
     def __init__(self, n: int, src, dst, features, model, weights: Sequence[Dict[str, np.ndarray]],
                  slack: float = 0.0, pool_edges: int = 0, max_batch: int = 0,
                  scatter_mode: int = SCATTER_AUTO, gemm_mode: int = GEMM_AUTO, timing: bool = False,
-                 pre_transform: bool = True, stream=None):
+                 pre_transform: bool = True, graphs: bool = True, stream=None):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -181,6 +182,7 @@ class Ripple:
         opt.slack, opt.pool_edges, opt.max_batch = float(slack), int(pool_edges), int(max_batch)
         opt.scatter_mode, opt.gemm_mode, opt.timing = int(scatter_mode), int(gemm_mode), int(bool(timing))
         opt.pre_transform = 0 if pre_transform else 1
+        opt.no_graphs = 0 if graphs else 1
         opt.device = torch.cuda.current_device()
         self._stream = stream if stream is not None else torch.cuda.Stream()
         opt.stream = self._stream.cuda_stream
@@ -239,6 +241,9 @@ class Ripple:
                 feat_rows = np.ascontiguousarray(feat_rows, dtype=np.float32)
                 nr, fptr = feat_rows.shape[0], feat_rows.ctypes.data
         self._check(self.lib.ripple_apply_batch(self.h, uptr, n, fptr, nr, mem))
+
+    def set_timing(self, on: bool) -> None:
+        self._check(self.lib.ripple_set_timing(self.h, int(bool(on))))
 
     def recompute_full(self) -> None:
         self._check(self.lib.ripple_recompute_full(self.h))
