@@ -149,6 +149,12 @@ k_scatter_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64
             for (int j0 = 0; j0 < cnt_total; j0 += 32) {
                 int mine = j0 + lane < cnt_total ? out.col[base + j0 + lane] : 0;
                 int cnt = min(32, cnt_total - j0);
+                // every sink joins the hop's affected set (same walk as the frontier's): one lane per
+                // edge, 32 edges per instruction
+                if (lane < cnt) {
+                    const uint32_t m = 1u << (mine & 31);
+                    if (!(bitmap[mine >> 5] & m)) atomicOr(&bitmap[mine >> 5], m);
+                }
                 for (int j = 0; j < cnt; j += EPI) {
                     int jj = j + sub;
                     int v = __shfl_sync(FULL, mine, jj & 31);
@@ -159,11 +165,61 @@ k_scatter_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64
                             int q = ql + LPR * k;
                             if (q < nq) red_add_v4(dst + 4 * q, d[k]);
                         }
-                        // the sink joins the hop's affected set (same walk as the frontier's)
-                        if (ql == 0) {
-                            const uint32_t m = 1u << (v & 31);
-                            if (!(bitmap[v >> 5] & m)) atomicOr(&bitmap[v >> 5], m);
-                        }
+                    }
+                }
+            }
+            e = seg_end;
+            ++i;
+        }
+    }
+}
+
+// Packed form for row widths that do not divide a warp (48 floats = 12 lanes, 40 floats = 10):
+// messages are laid end to end over the lanes of consecutive instructions (8 messages over 3
+// instructions for 12 lanes), so every reduction instruction carries 32 active lanes instead of
+// 24.  Lane t of instruction i serves float4 slot (32 i + t) % NQ of message (32 i + t) / NQ.
+template <int NQ>
+__global__ void __launch_bounds__(256)
+k_scatter_push_packed(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64_t* __restrict__ coff,
+                      Side out, const float* __restrict__ D, float* S, uint32_t* bitmap) {
+    constexpr int LCM = NQ == 12 ? 96 : NQ == 10 ? 160 : NQ * 32;
+    constexpr int NI = LCM / 32, G = LCM / NQ, LD = NQ * 4;
+    if (ctl->abort || ctl->pull[l]) return;
+    const int nC = ctl->nC[l - 1];
+    if (nC == 0) return;
+    const int64_t E = coff[nC];
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id();
+    int msg_of[NI], slot_of[NI];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) { msg_of[i] = (32 * i + lane) / NQ; slot_of[i] = (32 * i + lane) % NQ; }
+    for (int64_t e0 = (int64_t)warp * PUSH_CHUNK; e0 < E; e0 += (int64_t)nwarps * PUSH_CHUNK) {
+        const int64_t e1 = min(e0 + PUSH_CHUNK, E);
+        int i = upper_row(coff, nC, e0);
+        int64_t e = e0;
+        while (e < e1) {
+            const int64_t row_end = coff[i + 1];
+            if (row_end <= e) { ++i; continue; }
+            const int64_t seg_end = min(e1, row_end);
+            const int64_t base = out.start[senders[i]] + (e - coff[i]);
+            float4 d[NI];
+            const float4* drow = reinterpret_cast<const float4*>(D + (size_t)i * LD);
+#pragma unroll
+            for (int k = 0; k < NI; ++k) d[k] = __ldg(drow + slot_of[k]);
+            const int cnt_total = (int)(seg_end - e);
+            for (int j0 = 0; j0 < cnt_total; j0 += 32) {
+                int mine = j0 + lane < cnt_total ? out.col[base + j0 + lane] : 0;
+                int cnt = min(32, cnt_total - j0);
+                if (lane < cnt) {
+                    const uint32_t m = 1u << (mine & 31);
+                    if (!(bitmap[mine >> 5] & m)) atomicOr(&bitmap[mine >> 5], m);
+                }
+                for (int g0 = 0; g0 < cnt; g0 += G) {
+#pragma unroll
+                    for (int k = 0; k < NI; ++k) {
+                        const int idx = g0 + msg_of[k];
+                        const int v = __shfl_sync(FULL, mine, idx & 31);
+                        if (idx < cnt) red_add_v4(S + (size_t)v * LD + 4 * slot_of[k], d[k]);
                     }
                 }
             }
@@ -334,7 +390,11 @@ void scatter_layer(Ctx* c, int l, int n) {
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
 #define PUSH(NV, LPR) RP_LAUNCH(c, (k_scatter_push<NV, LPR>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, ld, c->dS[l], c->bitmap)
 #define PULL(NV, LPR) RP_LAUNCH(c, (k_scatter_pull<NV, 32>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->posmap, Dm, ld, c->dS[l])
-    if (c->scatter_mode != RIPPLE_SCATTER_PULL) RP_WIDTH_DISPATCH(ld, PUSH);
+    if (c->scatter_mode != RIPPLE_SCATTER_PULL) {
+        if (ld == 48) RP_LAUNCH(c, k_scatter_push_packed<12>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
+        else if (ld == 40) RP_LAUNCH(c, k_scatter_push_packed<10>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
+        else RP_WIDTH_DISPATCH(ld, PUSH);
+    }
     if (c->scatter_mode == RIPPLE_SCATTER_PULL) RP_WIDTH_DISPATCH(ld, PULL);
 #undef PUSH
 #undef PULL
