@@ -441,3 +441,96 @@ def test_sparse_config_100_consecutive_batches(env, batch):
 @pytest.mark.parametrize("batch", [100, 1000])
 def test_sparse_deep_configs_100_consecutive_batches(env, wname, batch):
     _run_workload(env, wname, batch, 100, 50, row_slack=gin_row_slack(100) if "gin" in wname else 0.0)
+
+
+# ---------------------------------------------------------------------------------------------
+# shapes and sizes at the edges
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dims,kind", [([7, 5], "sage"), ([7, 13, 5], "sage"), ([6, 9], "gcn"), ([3, 11, 2], "gin")])
+def test_odd_widths_single_layer_and_empty_graph(env, dims, kind):
+    """Widths that are not multiples of 4 (padded columns must stay zero), one-layer models, and a
+    graph that starts with no edge at all."""
+    ripple, Oracle = env
+    if kind == "sage":
+        model = I.sage_model(dims, I.AGG_MEAN)
+    elif kind == "gcn":
+        model = I.graphconv_model(dims, I.AGG_WSUM_GCN)
+    else:
+        model = I.gin_model(dims[0], dims[1], len(dims) - 1, eps=0.3)
+    L = len(model.layers)
+    n = 257
+    src = np.zeros(0, dtype=np.int32)
+    dst = np.zeros(0, dtype=np.int32)
+    X = I.features(n, dims[0], 5)
+    W = I.make_weights(model, 5, zero_bias=False)
+    rp = ripple.Ripple(n, src, dst, X, model, W)
+    orc = Oracle(n, src, dst, X, model, W)
+    check_values(rp, orc.full(), L)
+    stream = I.UpdateStream(n, src, dst, dims[0], 5, mix=(0.7, 0.1, 0.2))
+    for b in range(12):
+        ups, rows = stream.next_batch(40)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, L)
+    check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+    for l in range(L + 1):   # padded columns are not exposed: views have exactly the model's widths
+        assert rp.embeddings(l).shape == (n, model.dims[l])
+    rp.close()
+
+
+def test_largest_batch_with_heavy_repetition(env):
+    """A batch of the maximum size (16 384 ops) drawn over few pairs, so that most pairs repeat
+    several times with conflicting ops: the last op per pair and per feature vertex must win."""
+    ripple, Oracle = env
+    model = I.sage_model([10, 12, 6], I.AGG_MEAN)
+    n, m = 400, 3000
+    src, dst = I.er_graph(n, m, 17)
+    X = I.features(n, 10, 17)
+    W = I.make_weights(model, 17)
+    rp = ripple.Ripple(n, src, dst, X, model, W)          # default max_batch = 16384
+    orc = Oracle(n, src, dst, X, model, W)
+    rng = np.random.default_rng(17)
+    for rnd in range(3):
+        b = 16384
+        ups = np.zeros(b, dtype=I.UPDATE_DTYPE)
+        ups["op"] = rng.choice(3, size=b, p=[0.45, 0.45, 0.1])
+        ups["u"] = rng.integers(0, 60, size=b)
+        ups["v"] = rng.integers(0, 60, size=b)
+        nf = int((ups["op"] == I.OP_SET_FEATURE).sum())
+        ups["v"][ups["op"] == I.OP_SET_FEATURE] = np.arange(nf)
+        rows = I.features(nf, 10, 100 + rnd)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, 2)
+        check_values(rp, orc.full(), 2)
+        assert rp.stats()["n_superseded"] > 10000
+    with pytest.raises(ripple.RippleError) as ei:
+        rp.apply_batch(np.zeros(16385, dtype=I.UPDATE_DTYPE))
+    assert ei.value.status == ripple.ERR_CAPACITY
+    rp.close()
+
+
+def test_graph_replay_and_direct_launch_agree(env):
+    """Small batches are replayed from a captured launch chain; the result must be the one the
+    kernel-by-kernel path gives (same graph, same frontiers, embeddings within rounding)."""
+    ripple, Oracle = env
+    n, src, dst, X, model, W = _small(seed=53, name="gcn_wsum_3l")
+    a = ripple.Ripple(n, src, dst, X, model, W, graphs=True)
+    b = ripple.Ripple(n, src, dst, X, model, W, graphs=False)
+    orc = Oracle(n, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 53)
+    for bs in [7, 7, 7, 30, 7, 512, 513, 7]:     # repeated sizes hit the cached graph; 513 is direct
+        ups, rows = stream.next_batch(bs)
+        a.apply_batch(ups, rows)
+        b.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        check_graph(a, orc)
+        check_frontiers(a, orc, 3)
+        check_frontiers(b, orc, 3)
+    ref = orc.full()
+    check_values(a, ref, 3)
+    check_values(b, ref, 3)
+    a.close()
+    b.close()
