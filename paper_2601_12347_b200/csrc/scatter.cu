@@ -35,46 +35,84 @@ __device__ __forceinline__ void add4(float4& a, const float4& x, float c) {
 // bootstrap: S_v for every vertex by gathering over in-edges (Eq. 1)
 // LPR lanes hold one row (NV float4 slots each); a warp works on 32 / LPR in-neighbours at a time.
 // ---------------------------------------------------------------------------------------------
+constexpr int SPMM_HUB_DEGREE = 2048;  // longer in-lists are cut into chunks handled by separate warps
+constexpr int SPMM_HUB_CHUNK = 1024;
+
+// acc += sum over in-list entries [j_begin, j_end) of row v of c_u * M_u; LPR lanes hold one row
+// (NV float4 slots each), a warp works on 32 / LPR neighbours per step, four steps in flight.
 template <int NV, int LPR>
-__global__ void __launch_bounds__(256)
-k_spmm_pull(int N, Side in, const int32_t* __restrict__ deg_out, int src_norm,
-            const float* __restrict__ M, int ld, float* __restrict__ S) {
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+__device__ __forceinline__ void spmm_accumulate(float4 (&acc)[NV], const Side& in, int v, int j_begin, int j_end,
+                                                const int32_t* __restrict__ deg_out, int src_norm,
+                                                const float* __restrict__ M, int ld) {
     const int lane = lane_id(), nq = ld >> 2;
     constexpr int EPI = 32 / LPR;
     const int sub = lane / LPR, ql = lane % LPR;
+    const int64_t base = in.start[v];
+    for (int j0 = j_begin; j0 < j_end; j0 += 32) {
+        int mine = j0 + lane < j_end ? in.col[base + j0 + lane] : 0;
+        int cnt = min(32, j_end - j0);
+        constexpr int UNR = 4;
+        for (int j = 0; j < cnt; j += UNR * EPI) {
+            int u[UNR];
+            float cu[UNR];
+            float4 x[UNR][NV];
+#pragma unroll
+            for (int t = 0; t < UNR; ++t) {
+                const int jj = j + t * EPI + sub;
+                u[t] = __shfl_sync(FULL, mine, jj & 31);
+                cu[t] = 0.f;
+                if (jj < cnt) cu[t] = src_norm ? coef_from_degree(deg_out[u[t]]) : 1.0f;
+                else u[t] = -1;
+            }
+#pragma unroll
+            for (int t = 0; t < UNR; ++t) {
+                const float4* row = reinterpret_cast<const float4*>(M + (size_t)max(u[t], 0) * ld);
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    const int q = ql + LPR * k;
+                    x[t][k] = (u[t] >= 0 && q < nq) ? __ldg(row + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < UNR; ++t)
+#pragma unroll
+                for (int k = 0; k < NV; ++k) add4(acc[k], x[t][k], cu[t]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) {
+            acc[k].x += __shfl_xor_sync(FULL, acc[k].x, o);
+            acc[k].y += __shfl_xor_sync(FULL, acc[k].y, o);
+            acc[k].z += __shfl_xor_sync(FULL, acc[k].z, o);
+            acc[k].w += __shfl_xor_sync(FULL, acc[k].w, o);
+        }
+    }
+}
+
+// One warp per vertex.  A vertex with a very long in-list only zeroes its row here and queues
+// (vertex, chunk) work items for k_spmm_hubs, so that no single warp walks 150 K neighbours.
+template <int NV, int LPR>
+__global__ void __launch_bounds__(256)
+k_spmm_pull(int N, Side in, const int32_t* __restrict__ deg_out, int src_norm,
+            const float* __restrict__ M, int ld, float* __restrict__ S, int2* items, int* n_items) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id(), nq = ld >> 2;
+    const int sub = lane / LPR, ql = lane % LPR;
     for (int v = warp; v < N; v += nwarps) {
+        const int deg = in.deg[v];
         float4 acc[NV];
 #pragma unroll
         for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        const int64_t base = in.start[v];
-        const int deg = in.deg[v];
-        for (int j0 = 0; j0 < deg; j0 += 32) {
-            int mine = j0 + lane < deg ? in.col[base + j0 + lane] : 0;
-            int cnt = min(32, deg - j0);
-            for (int j = 0; j < cnt; j += EPI) {
-                int jj = j + sub;
-                int u = __shfl_sync(FULL, mine, jj & 31);
-                if (jj < cnt) {
-                    float cu = src_norm ? coef_from_degree(deg_out[u]) : 1.0f;
-                    const float4* row = reinterpret_cast<const float4*>(M + (size_t)u * ld);
-#pragma unroll
-                    for (int k = 0; k < NV; ++k) {
-                        int q = ql + LPR * k;
-                        if (q < nq) add4(acc[k], __ldg(row + q), cu);
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int k = 0; k < NV; ++k) {
-#pragma unroll
-            for (int o = LPR; o < 32; o <<= 1) {
-                acc[k].x += __shfl_xor_sync(FULL, acc[k].x, o);
-                acc[k].y += __shfl_xor_sync(FULL, acc[k].y, o);
-                acc[k].z += __shfl_xor_sync(FULL, acc[k].z, o);
-                acc[k].w += __shfl_xor_sync(FULL, acc[k].w, o);
-            }
+        if (deg > SPMM_HUB_DEGREE) {
+            const int nch = (deg + SPMM_HUB_CHUNK - 1) / SPMM_HUB_CHUNK;
+            int first = 0;
+            if (lane == 0) first = atomicAdd(n_items, nch);
+            first = __shfl_sync(FULL, first, 0);
+            for (int ch = lane; ch < nch; ch += 32) items[first + ch] = make_int2(v, ch);
+        } else {
+            spmm_accumulate<NV, LPR>(acc, in, v, 0, deg, deg_out, src_norm, M, ld);
         }
         if (sub == 0) {
             float4* dst = reinterpret_cast<float4*>(S + (size_t)v * ld);
@@ -82,6 +120,32 @@ k_spmm_pull(int N, Side in, const int32_t* __restrict__ deg_out, int src_norm,
             for (int k = 0; k < NV; ++k) {
                 int q = ql + LPR * k;
                 if (q < nq) dst[q] = acc[k];
+            }
+        }
+    }
+}
+
+template <int NV, int LPR>
+__global__ void __launch_bounds__(256)
+k_spmm_hubs(Side in, const int32_t* __restrict__ deg_out, int src_norm, const float* __restrict__ M, int ld,
+            float* S, const int2* __restrict__ items, const int* __restrict__ n_items) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id(), nq = ld >> 2;
+    const int sub = lane / LPR, ql = lane % LPR;
+    const int n = *n_items;
+    for (int it = warp; it < n; it += nwarps) {
+        const int2 w = items[it];
+        const int deg = in.deg[w.x];
+        float4 acc[NV];
+#pragma unroll
+        for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        spmm_accumulate<NV, LPR>(acc, in, w.x, w.y * SPMM_HUB_CHUNK, min(deg, (w.y + 1) * SPMM_HUB_CHUNK), deg_out,
+                                 src_norm, M, ld);
+        if (sub == 0) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                int q = ql + LPR * k;
+                if (q < nq) red_add_v4(S + (size_t)w.x * ld + 4 * q, acc[k]);
             }
         }
     }
@@ -107,7 +171,16 @@ void spmm_full(Ctx* c, int l) {
         M = c->D[0];
     }
     const int grid = c->n_sm * 16, T = 256;
-#define SPMM(NV, LPR) RP_LAUNCH(c, (k_spmm_pull<NV, LPR>), grid, T, 0, c->N, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld, c->S[l])
+    // work items of the long rows live in the degree-prefix buffer, which is idle during a full pass
+    int2* items = reinterpret_cast<int2*>(c->coff);
+    int* n_items = &c->ctl->work_counter[(l - 1) & 7];
+#define SPMM(NV, LPR)                                                                                              \
+    do {                                                                                                           \
+        RP_LAUNCH(c, (k_spmm_pull<NV, LPR>), grid, T, 0, c->N, c->side[1], c->side[0].deg, (int)c->src_norm, M,   \
+                  ld, c->S[l], items, n_items);                                                                    \
+        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), grid, T, 0, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
+                  c->S[l], items, n_items);                                                                        \
+    } while (0)
     RP_WIDTH_DISPATCH(ld, SPMM);
 #undef SPMM
 }
