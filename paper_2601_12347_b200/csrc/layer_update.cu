@@ -116,10 +116,11 @@ void neighbour_transform(Ctx* c, int l, const float* rows_in, int ld_rows, const
     launch_update(c, p, ly.tc_nbr);
 }
 
-// Z^l_v = W_self^T h^{l-1}_v for the rows whose h^{l-1} changed (all rows at bootstrap).  A SAGE
-// layer that is narrower than its input keeps this self projection cached next to the transformed
-// aggregate, so that its affected-row update needs no contraction at all: the projection is
-// recomputed where the layer's input changed (A_{l-1}), not where its output is needed (A_l).
+// Z^l_v = W_self^T h^{l-1}_v for the rows whose h^{l-1} changed (all rows at bootstrap).  SAGE
+// layers keep this self projection cached: it is recomputed where the layer's input changed
+// (A_{l-1}), not where its output is needed (A_l, usually far larger).  The affected-row update
+// then contracts over the aggregate only (half the K of [h || x]); for a layer that also
+// transforms before the scatter nothing is left to contract.
 void self_project(Ctx* c, int l, bool full) {
     if (!c->Z[l]) return;
     const LayerDev& ly = c->layer[l];
@@ -131,7 +132,7 @@ void self_project(Ctx* c, int l, bool full) {
     p.Hprev = c->H[l - 1]; p.ld_h = c->ld[l - 1];
     p.K = ly.ld_in; p.W = ly.W1; p.ldw = ly.ld_out; p.n_cols = ly.ld_out;
     p.act = RIPPLE_ACT_IDENTITY; p.Hout = c->Z[l]; p.ld_o = ly.ld_out;
-    launch_update(c, p, ly.tc_main);
+    launch_update(c, p, ly.tc_self);
 }
 
 void update_rows(Ctx* c, int l, bool full) {
@@ -169,15 +170,17 @@ void update_rows(Ctx* c, int l, bool full) {
     }
     p.epi_mode = EPI_COMMIT;
     if (ly.kind == RIPPLE_LAYER_SAGE) {
-        p.a_mode = pre ? A_SELF : A_CONCAT;
-        p.K = pre ? 0 : 2 * ly.ld_in;   // narrow layer: self projection and aggregate are both cached
-        if (pre) p.addend2 = c->Z[l];
+        p.a_mode = A_AGG;
+        p.K = pre ? 0 : ly.ld_in;       // transformed aggregate: nothing left to multiply
+        p.addend2 = c->Z[l];            // cached W_self^T h_v
     } else {
         p.a_mode = A_AGG;
         p.K = pre ? 0 : ly.ld_in;   // transformed inbox: nothing left to multiply
     }
-    p.W = ly.W1; p.ldw = ly.ld_out; p.bias = ly.b1; p.n_cols = ly.ld_out;
+    p.W = ly.kind == RIPPLE_LAYER_SAGE ? ly.W1 + (size_t)ly.ld_in * ly.ld_out : ly.W1;   // neighbour matrix
+    p.ldw = ly.ld_out; p.bias = ly.b1; p.n_cols = ly.ld_out;
     p.act = ly.act; p.Hout = c->H[l]; p.ld_o = ly.ld_out; p.Dout = dout;
+    if (!pre) p.ld_add = ly.ld_out;   // leading dimension of the cached projection
     launch_update(c, p, ly.tc_main);
 }
 

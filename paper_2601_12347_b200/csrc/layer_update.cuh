@@ -89,10 +89,13 @@ __device__ __forceinline__ float4 upd_load_old(const UpdParams& p, int v, int co
 }
 
 // bias, optional addend, activation, then either a compact temp row or commit + delta row;
-// `old` is the previously stored value if the caller has prefetched it (has_old)
+// `old` / `zpre` are the previously stored value and the addend2 value if the caller has
+// prefetched them (has_old / has_z)
 __device__ __forceinline__ void upd_epilogue4(const UpdParams& p, int v, int i, int col, float4 h, float sc,
                                               bool has_old = false,
-                                              float4 old = make_float4(0.f, 0.f, 0.f, 0.f)) {
+                                              float4 old = make_float4(0.f, 0.f, 0.f, 0.f),
+                                              bool has_z = false,
+                                              float4 zpre = make_float4(0.f, 0.f, 0.f, 0.f)) {
     if (p.bias) {
         float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col));
         h.x += b.x; h.y += b.y; h.z += b.z; h.w += b.w;
@@ -112,7 +115,7 @@ __device__ __forceinline__ void upd_epilogue4(const UpdParams& p, int v, int i, 
         h.x += sc * s.x; h.y += sc * s.y; h.z += sc * s.z; h.w += sc * s.w;
     }
     if (p.addend2) {
-        float4 z = *reinterpret_cast<const float4*>(p.addend2 + (size_t)v * p.ld_add + col);
+        float4 z = has_z ? zpre : *reinterpret_cast<const float4*>(p.addend2 + (size_t)v * p.ld_add + col);
         h.x += z.x; h.y += z.y; h.z += z.z; h.w += z.w;
     }
     if (p.act == RIPPLE_ACT_RELU) {

@@ -84,15 +84,27 @@ __device__ __forceinline__ uint32_t tc_swz(int r, int c) {
 
 __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
 
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// barrier among the loader warps only (the MMA warp never joins it)
+__device__ __forceinline__ void loaders_sync() { asm volatile("bar.sync 1, %0;" ::"n"(TC_THREADS) : "memory"); }
+
+// Warp roles: warps 0..7 ("loaders") stage the operands of every K chunk and run the epilogue;
+// warp 8 issues the MMAs.  Two mbarriers per stage hand the stage back and forth:
+//   full[s]   8 arrivals (one per loader warp, after its stores and proxy fence) -> MMA warp may read
+//   empty[s]  1 arrival (tcgen05.commit of the MMAs that read the stage)         -> loaders may refill
+// so the single-thread MMA issue (a microsecond per chunk) overlaps the loads of the next chunk.
 template <bool X3>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TC_THREADS + 32, 1)
 k_update_rows_tc(Ctl* ctl, UpdParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t mbar[2];
+    __shared__ uint64_t full[2], empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int row_id[TC_M];
     __shared__ float row_scale[TC_M];
-    __shared__ int s_fail;
+    __shared__ volatile int s_fail;
 
     if (ctl->abort) return;
     const int n = upd_rows(p);
@@ -101,6 +113,7 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
     if ((int)blockIdx.x >= row_tiles) return;   // before any allocation
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool is_mma_warp = warp == TC_THREADS / 32;
     const int n_pad = p.n_pad;
     const uint32_t b_bytes = (uint32_t)n_pad * 128u;
     const uint32_t stage_bytes = (X3 ? 2u : 1u) * (TC_A_BYTES + b_bytes);
@@ -109,8 +122,10 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
     while ((int)tmem_cols < n_pad) tmem_cols <<= 1;
 
     if (tid == 0) {
-        mbar_init(&mbar[0], 1);
-        mbar_init(&mbar[1], 1);
+        mbar_init(&full[0], TC_THREADS / 32);
+        mbar_init(&full[1], TC_THREADS / 32);
+        mbar_init(&empty[0], 1);
+        mbar_init(&empty[1], 1);
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -128,34 +143,65 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
     const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n_pad >> 3) << 17) |
                            ((uint32_t)(TC_M >> 4) << 24);
     const int nchunks = p.k_pad / TC_KC;
-    uint32_t uses[2] = {0u, 0u};
-    bool failed = false;
+    uint32_t uses[2] = {0u, 0u};   // how often each stage has been handed over so far (same in every thread)
 
-    for (int tile = blockIdx.x; tile < row_tiles && !failed; tile += gridDim.x) {
-        const int r0 = tile * TC_M;
-        if (tid < TC_M) {
-            int i = r0 + tid, v = -1;
-            float sc = 0.f;
-            if (i < n) {
-                v = p.list ? p.list[i] : i;
-                sc = upd_row_scale(p, v);
+    if (is_mma_warp) {
+        // ---------------- MMA issue ----------------
+        for (int tile = blockIdx.x; tile < row_tiles && !s_fail; tile += gridDim.x) {
+            for (int kc = 0; kc < nchunks; ++kc) {
+                const int s = kc & 1;
+                uint8_t* a_hi = smem + (size_t)s * stage_bytes;
+                uint8_t* a_lo = a_hi + TC_A_BYTES;
+                uint8_t* b_hi = a_hi + (X3 ? 2 : 1) * TC_A_BYTES;
+                uint8_t* b_lo = b_hi + b_bytes;
+                if (lane == 0) {
+                    if (!mbar_wait_bounded(&full[s], uses[s] & 1)) s_fail = 1;
+                    if (!s_fail) {
+                        tc_fence_after();
+                        const uint64_t da_hi = tc_smem_desc(smem_u32(a_hi)), db_hi = tc_smem_desc(smem_u32(b_hi));
+                        const uint64_t da_lo = tc_smem_desc(smem_u32(a_lo)), db_lo = tc_smem_desc(smem_u32(b_lo));
+#pragma unroll
+                        for (int j = 0; j < TC_KC / 8; ++j) {     // one MMA K step = 8 floats = 32 bytes
+                            const uint64_t adv = (uint64_t)((j * 32) >> 4);
+                            tc_mma_tf32(tmem_base, da_hi + adv, db_hi + adv, idesc, (kc | j) != 0);
+                            if (X3) {
+                                tc_mma_tf32(tmem_base, da_lo + adv, db_hi + adv, idesc, 1u);
+                                tc_mma_tf32(tmem_base, da_hi + adv, db_lo + adv, idesc, 1u);
+                            }
+                        }
+                        tc_commit(&empty[s]);
+                    }
+                }
+                __syncwarp();
+                uses[s]++;
+                if (s_fail) break;
             }
-            row_id[tid] = v;
-            row_scale[tid] = sc;
         }
-        __syncthreads();
+    } else {
+        // ---------------- loaders + epilogue ----------------
+        for (int tile = blockIdx.x; tile < row_tiles && !s_fail; tile += gridDim.x) {
+            const int r0 = tile * TC_M;
+            if (tid < TC_M) {
+                int i = r0 + tid, v = -1;
+                float sc = 0.f;
+                if (i < n) {
+                    v = p.list ? p.list[i] : i;
+                    sc = upd_row_scale(p, v);
+                }
+                row_id[tid] = v;
+                row_scale[tid] = sc;
+            }
+            loaders_sync();
 
-        for (int kc = 0; kc < nchunks; ++kc) {
-            const int s = kc & 1;
-            uint8_t* a_hi = smem + (size_t)s * stage_bytes;
-            uint8_t* a_lo = a_hi + TC_A_BYTES;                              // only if X3
-            uint8_t* b_hi = a_hi + (X3 ? 2 : 1) * TC_A_BYTES;
-            uint8_t* b_lo = b_hi + b_bytes;                                 // only if X3
-            // the MMAs that last read this stage must have finished
-            if (uses[s] > 0 && !mbar_wait_bounded(&mbar[s], (uses[s] - 1) & 1)) s_fail = 1;
-            // Staging: every global load of the chunk (gathered A rows, weight rows) is issued before
-            // the first shared-memory store so that all of their latencies overlap.
-            {
+            for (int kc = 0; kc < nchunks; ++kc) {
+                const int s = kc & 1;
+                uint8_t* a_hi = smem + (size_t)s * stage_bytes;
+                uint8_t* a_lo = a_hi + TC_A_BYTES;                              // only if X3
+                uint8_t* b_hi = a_hi + (X3 ? 2 : 1) * TC_A_BYTES;
+                uint8_t* b_lo = b_hi + b_bytes;                                 // only if X3
+                // Every global load of the chunk (gathered A rows, weight rows) is issued before the
+                // stage is even known to be free, and before the first shared-memory store, so that
+                // all latencies overlap.
                 constexpr int A_ITERS = (TC_M * 8) / TC_THREADS;
                 constexpr int B_ITERS = (256 * 8) / TC_THREADS;   // n_pad <= 256
                 float4 ax[A_ITERS], bh[B_ITERS], bl[B_ITERS];
@@ -175,6 +221,8 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                         if (X3) bl[it] = __ldg(reinterpret_cast<const float4*>(p.Wt_lo + g));
                     }
                 }
+                // the MMAs that last read this stage must have finished
+                if (uses[s] > 0 && !mbar_wait_bounded(&empty[s], (uses[s] - 1) & 1)) s_fail = 1;
 #pragma unroll
                 for (int it = 0; it < A_ITERS; ++it) {
                     const int idx = tid + it * TC_THREADS;
@@ -193,95 +241,96 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                         if (X3) *reinterpret_cast<float4*>(b_lo + off) = bl[it];
                     }
                 }
+                fence_async_smem();   // generic-proxy stores -> visible to the tensor core's async proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full[s]);
+                uses[s]++;
+                if (s_fail) break;
             }
-            fence_async_smem();   // generic-proxy stores -> visible to the tensor core's async proxy
-            __syncthreads();
-            if (s_fail) { failed = true; break; }
-            if (tid == 0) {
-                tc_fence_after();
-                const uint64_t da_hi = tc_smem_desc(smem_u32(a_hi)), db_hi = tc_smem_desc(smem_u32(b_hi));
-                const uint64_t da_lo = tc_smem_desc(smem_u32(a_lo)), db_lo = tc_smem_desc(smem_u32(b_lo));
-#pragma unroll
-                for (int j = 0; j < TC_KC / 8; ++j) {     // one MMA K step = 8 floats = 32 bytes
-                    const uint64_t adv = (uint64_t)((j * 32) >> 4);
-                    tc_mma_tf32(tmem_base, da_hi + adv, db_hi + adv, idesc, (kc | j) != 0);
-                    if (X3) {
-                        tc_mma_tf32(tmem_base, da_lo + adv, db_hi + adv, idesc, 1u);
-                        tc_mma_tf32(tmem_base, da_hi + adv, db_lo + adv, idesc, 1u);
-                    }
-                }
-                tc_commit(&mbar[s]);
+            if (s_fail) break;
+            // the last commit covers every MMA of the tile
+            {
+                const int s = (nchunks - 1) & 1;
+                if (!mbar_wait_bounded(&empty[s], (uses[s] - 1) & 1)) s_fail = 1;
             }
-            uses[s]++;
-        }
-        if (failed) break;
-        // the last commit covers every MMA of the tile
-        {
-            const int s = (nchunks - 1) & 1;
-            if (!mbar_wait_bounded(&mbar[s], (uses[s] - 1) & 1)) s_fail = 1;
-        }
-        tc_fence_after();
-        __syncthreads();
-        if (s_fail) { failed = true; break; }
+            if (s_fail) break;
+            tc_fence_after();
 
-        // epilogue: warp w reads lanes 32 (w % 4) .. +31, warps 0-3 the first half of the 16-column
-        // blocks and warps 4-7 the rest; one accumulator row per thread
-        {
-            const int g = warp & 3, half = warp >> 2;
-            const int nblk = n_pad >> 4, split = (nblk + 1) >> 1;
-            const int b0 = half ? split : 0, b1 = half ? nblk : split;
-            const int r = 32 * g + lane, v = row_id[r];
-            const float sc = row_scale[r];
-            // the previous values of the row (needed for the delta) are fetched one block ahead, so
-            // that their latency hides behind the tensor-memory load and the stores of the block
-            // before
-            const bool need_old = upd_needs_old(p) && v >= 0;
-            float4 old_cur[4], old_nxt[4];
-            if (need_old && b0 < b1) {
+            // Epilogue in two steps.  (1) Every thread copies its accumulator row (warp w: tensor-memory
+            // lanes 32 (w % 4).., warps 0-3 the first half of the 16-column blocks, warps 4-7 the rest)
+            // into a row-major tile in shared memory; the operand stages are free now.  (2) Each warp
+            // then takes whole rows, 32 lanes x 16 bytes per pass, so that the previous row, the cached
+            // projection, the delta row and the new row all move in coalesced 512-byte pieces, four
+            // rows in flight.
+            float* tile_s = reinterpret_cast<float*>(smem);
+            const int tstride = n_pad + 4;   // = 4 mod 32: conflict-free 16-byte stores down a column
+            {
+                const int g = warp & 3, half = warp >> 2;
+                const int nblk = n_pad >> 4, split = (nblk + 1) >> 1;
+                const int b0 = half ? split : 0, b1 = half ? nblk : split;
+                const int r = 32 * g + lane;
+                for (int blk = b0; blk < b1; ++blk) {
+                    uint32_t x[16];
+                    const uint32_t taddr = tmem_base + ((uint32_t)(32 * g) << 16) + (uint32_t)(blk * 16);
+                    asm volatile(
+                        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                        : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3]), "=r"(x[4]), "=r"(x[5]), "=r"(x[6]),
+                          "=r"(x[7]), "=r"(x[8]), "=r"(x[9]), "=r"(x[10]), "=r"(x[11]), "=r"(x[12]), "=r"(x[13]),
+                          "=r"(x[14]), "=r"(x[15])
+                        : "r"(taddr) : "memory");
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    float4* dst = reinterpret_cast<float4*>(tile_s + (size_t)r * tstride + blk * 16);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int col = b0 * 16 + 4 * q;
-                    if (col < p.n_cols) old_cur[q] = upd_load_old(p, v, col);
+                    for (int q = 0; q < 4; ++q)
+                        dst[q] = make_float4(__uint_as_float(x[4 * q]), __uint_as_float(x[4 * q + 1]),
+                                             __uint_as_float(x[4 * q + 2]), __uint_as_float(x[4 * q + 3]));
                 }
             }
-            for (int blk = b0; blk < b1; ++blk) {
-                uint32_t x[16];
-                const uint32_t taddr = tmem_base + ((uint32_t)(32 * g) << 16) + (uint32_t)(blk * 16);
-                asm volatile(
-                    "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-                    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-                    : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3]), "=r"(x[4]), "=r"(x[5]), "=r"(x[6]),
-                      "=r"(x[7]), "=r"(x[8]), "=r"(x[9]), "=r"(x[10]), "=r"(x[11]), "=r"(x[12]), "=r"(x[13]),
-                      "=r"(x[14]), "=r"(x[15])
-                    : "r"(taddr) : "memory");
-                if (need_old && blk + 1 < b1) {
+            tc_fence_before();   // accumulators consumed: the MMA warp may overwrite them after our next arrival
+            loaders_sync();
+            {
+                constexpr int RUN = 4;                       // rows in flight per warp
+                const bool need_old = upd_needs_old(p);
+                const bool need_z = p.addend2 != nullptr;
+                const int npass = (p.n_cols + 127) >> 7;     // <= 2
+                for (int rb = warp; rb < TC_M; rb += (TC_THREADS / 32) * RUN) {
+                    int vv[RUN];
+                    float4 oldv[RUN][2], zv[RUN][2];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int col = (blk + 1) * 16 + 4 * q;
-                        if (col < p.n_cols) old_nxt[q] = upd_load_old(p, v, col);
+                    for (int t = 0; t < RUN; ++t) {
+                        const int r = rb + t * (TC_THREADS / 32);
+                        vv[t] = r < TC_M ? row_id[r] : -1;
+#pragma unroll
+                        for (int ps = 0; ps < 2; ++ps) {
+                            const int col = 4 * lane + 128 * ps;
+                            if (vv[t] >= 0 && ps < npass && col < p.n_cols) {
+                                if (need_old) oldv[t][ps] = upd_load_old(p, vv[t], col);
+                                if (need_z) zv[t][ps] = *reinterpret_cast<const float4*>(p.addend2 + (size_t)vv[t] * p.ld_add + col);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int t = 0; t < RUN; ++t) {
+                        const int r = rb + t * (TC_THREADS / 32);
+                        if (vv[t] < 0) continue;
+#pragma unroll
+                        for (int ps = 0; ps < 2; ++ps) {
+                            const int col = 4 * lane + 128 * ps;
+                            if (ps < npass && col < p.n_cols) {
+                                const float4 acc = *reinterpret_cast<const float4*>(tile_s + (size_t)r * tstride + col);
+                                upd_epilogue4(p, vv[t], r0 + r, col, acc, row_scale[r], need_old, oldv[t][ps], need_z, zv[t][ps]);
+                            }
+                        }
                     }
                 }
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (v >= 0) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int col = blk * 16 + 4 * q;
-                        if (col < p.n_cols)
-                            upd_epilogue4(p, v, r0 + r, col,
-                                          make_float4(__uint_as_float(x[4 * q]), __uint_as_float(x[4 * q + 1]),
-                                                      __uint_as_float(x[4 * q + 2]), __uint_as_float(x[4 * q + 3])),
-                                          sc, need_old, old_cur[q]);
-                    }
-                }
-#pragma unroll
-                for (int q = 0; q < 4; ++q) old_cur[q] = old_nxt[q];
             }
+            // the tile buffer (= the operand stages) and row_id are free before the next tile's staging
+            loaders_sync();
         }
-        tc_fence_before();
-        __syncthreads();   // accumulators consumed and row_id free before the next tile
     }
 
-    if (failed && tid == 0) {
+    if (s_fail && lane == 0) {
         atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_TIMEOUT);
         ctl->abort = 1;
     }
@@ -299,9 +348,9 @@ void launch_update_tc(Ctx* c, const UpdParams& p) {
     const int per_sm = std::max<size_t>(1, std::min<size_t>(4, (size_t)(220 * 1024) / (smem + 2048)));
     const int grid = c->n_sm * per_sm;
     if (x3) {
-        RP_LAUNCH(c, k_update_rows_tc<true>, grid, TC_THREADS, smem, c->ctl, p);
+        RP_LAUNCH(c, k_update_rows_tc<true>, grid, TC_THREADS + 32, smem, c->ctl, p);
     } else {
-        RP_LAUNCH(c, k_update_rows_tc<false>, grid, TC_THREADS, smem, c->ctl, p);
+        RP_LAUNCH(c, k_update_rows_tc<false>, grid, TC_THREADS + 32, smem, c->ctl, p);
     }
 }
 

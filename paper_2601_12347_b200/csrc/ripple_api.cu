@@ -65,7 +65,7 @@ static void destroy_ctx(Ctx* c) {
     for (int l = 0; l <= RP_MAXL; ++l) {
         cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->Z[l]); cudaFree(c->A[l]);
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
-        for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2}) { cudaFree(t->hi); cudaFree(t->lo); }
+        for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2, &c->layer[l].tc_self}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
     cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hseq);
@@ -235,7 +235,10 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                 if (o.gemm_mode != RIPPLE_GEMM_FP32) {   // transposed, tf32-split copies for the tensor-core form
                     const float* wn = y.kind == RIPPLE_LAYER_SAGE ? w1.data() + (size_t)ly.ld_in * ly.ld_out : w1.data();
                     if (y.kind == RIPPLE_LAYER_SAGE)
-                        CK(tc_weights_build(&ly.tc_main, w1.data(), c->pre[l] ? ly.ld_in : 2 * ly.ld_in, ly.ld_out));
+                    {   // self part for the cached projection; neighbour part for the affected-row GEMM
+                        CK(tc_weights_build(&ly.tc_self, w1.data(), ly.ld_in, ly.ld_out));
+                        if (!c->pre[l]) CK(tc_weights_build(&ly.tc_main, wn, ly.ld_in, ly.ld_out));
+                    }
                     else if (y.kind == RIPPLE_LAYER_GIN)
                         CK(tc_weights_build(&ly.tc_main, w1.data(), ly.ld_in, ly.ld_hid));
                     else if (!c->pre[l])
@@ -259,7 +262,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             max_ld = std::max(max_ld, c->ld[l]);
             CK(dev_alloc(&c->H[l], (size_t)N * c->ld[l], 0));
             if (l > 0) { CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0)); CK(dev_alloc(&c->dS[l], (size_t)N * c->ws[l], 0));
-                         if (c->pre[l] && c->layer[l].kind == RIPPLE_LAYER_SAGE) CK(dev_alloc(&c->Z[l], (size_t)N * c->ws[l], 0)); }
+                         if (c->layer[l].kind == RIPPLE_LAYER_SAGE) CK(dev_alloc(&c->Z[l], (size_t)N * c->ld[l], 0)); }
             CK(dev_alloc(&c->A[l], (size_t)N + 32));
         }
         CK(cudaMemcpy2D(c->H[0], sizeof(float) * c->ld[0], features, sizeof(float) * c->d[0],

@@ -85,6 +85,7 @@ struct LayerDev {
     TcW tc_main; // weights of the affected-row GEMM (GIN: first matrix)
     TcW tc_nbr;  // neighbour matrix, for layers that transform before the scatter
     TcW tc_2;    // GIN: second matrix
+    TcW tc_self; // SAGE: self matrix, for the cached self projection
 };
 
 struct Ctx {
@@ -102,7 +103,7 @@ struct Ctx {
     Side side[2];
     float* H[RP_MAXL + 1];
     float* S[RP_MAXL + 1];
-    float* Z[RP_MAXL + 1];    // cached self projection W_self^T h^{l-1} of narrow SAGE layers (N x ws), else null
+    float* Z[RP_MAXL + 1];    // cached self projection W_self^T h^{l-1} of SAGE layers (N x ld_l), else null
     float* dS[RP_MAXL + 1];   // per-batch message accumulator, zero outside a batch (same shape as S)
     float* T;          // GIN hidden rows (compact, N x ld_hid)
     float* D[2];       // delta rows, ping-pong (compact, N x max ld)
