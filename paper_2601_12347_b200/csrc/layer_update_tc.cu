@@ -84,6 +84,10 @@ __device__ __forceinline__ uint32_t tc_swz(int r, int c) {
 
 __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
 
+__device__ __forceinline__ void cp_async16(uint32_t smem_addr, const float* gptr) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr), "l"(gptr) : "memory");
+}
+
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -193,36 +197,44 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
             }
             loaders_sync();
 
+            // The gathered A rows come from DRAM, the weights from L2: A is therefore loaded one chunk
+            // further ahead (registers), so that two chunks of row gathers are in flight.
+            constexpr int A_ITERS = (TC_M * 8) / TC_THREADS;
+            constexpr int B_ITERS = (256 * 8) / TC_THREADS;   // n_pad <= 256
+            float4 ax[A_ITERS], ax_next[A_ITERS];
+            auto load_a = [&](int kc, float4 (&dst)[A_ITERS]) {
+#pragma unroll
+                for (int it = 0; it < A_ITERS; ++it) {   // 128 rows x 8 chunks of 16 bytes, by vertex id
+                    const int idx = tid + it * TC_THREADS, r = idx >> 3, c = idx & 7;
+                    const int v = row_id[r], k = kc * TC_KC + c * 4;
+                    dst[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (v >= 0 && k < p.K) dst[it] = upd_load_a(p, v, r0 + r, k, row_scale[r]);
+                }
+            };
+            load_a(0, ax);
             for (int kc = 0; kc < nchunks; ++kc) {
                 const int s = kc & 1;
                 uint8_t* a_hi = smem + (size_t)s * stage_bytes;
                 uint8_t* a_lo = a_hi + TC_A_BYTES;                              // only if X3
                 uint8_t* b_hi = a_hi + (X3 ? 2 : 1) * TC_A_BYTES;
                 uint8_t* b_lo = b_hi + b_bytes;                                 // only if X3
-                // Every global load of the chunk (gathered A rows, weight rows) is issued before the
-                // stage is even known to be free, and before the first shared-memory store, so that
-                // all latencies overlap.
-                constexpr int A_ITERS = (TC_M * 8) / TC_THREADS;
-                constexpr int B_ITERS = (256 * 8) / TC_THREADS;   // n_pad <= 256
-                float4 ax[A_ITERS], bh[B_ITERS], bl[B_ITERS];
+                // next chunk's row gathers first (registers), so that they have a whole iteration to land
+                if (kc + 1 < nchunks) load_a(kc + 1, ax_next);
+                // the MMAs that last read this stage must have finished
+                if (uses[s] > 0 && !mbar_wait_bounded(&empty[s], (uses[s] - 1) & 1)) s_fail = 1;
+                // B: n_pad output columns x 8 chunks of the pre-split transposed weights, copied
+                // asynchronously from L2 straight into their swizzled places
 #pragma unroll
-                for (int it = 0; it < A_ITERS; ++it) {   // A: 128 rows x 8 chunks of 16 bytes, by vertex id
-                    const int idx = tid + it * TC_THREADS, r = idx >> 3, c = idx & 7;
-                    const int v = row_id[r], k = kc * TC_KC + c * 4;
-                    ax[it] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (v >= 0 && k < p.K) ax[it] = upd_load_a(p, v, r0 + r, k, row_scale[r]);
-                }
-#pragma unroll
-                for (int it = 0; it < B_ITERS; ++it) {   // B: n_pad output columns x 8 chunks, pre-split
+                for (int it = 0; it < B_ITERS; ++it) {
                     const int idx = tid + it * TC_THREADS;
                     if (idx < n_pad * 8) {
                         const size_t g = (size_t)(idx >> 3) * p.k_pad + kc * TC_KC + (idx & 7) * 4;
-                        bh[it] = __ldg(reinterpret_cast<const float4*>(p.Wt_hi + g));
-                        if (X3) bl[it] = __ldg(reinterpret_cast<const float4*>(p.Wt_lo + g));
+                        const uint32_t off = tc_swz(idx >> 3, idx & 7);
+                        cp_async16(smem_u32(b_hi + off), p.Wt_hi + g);
+                        if (X3) cp_async16(smem_u32(b_lo + off), p.Wt_lo + g);
                     }
                 }
-                // the MMAs that last read this stage must have finished
-                if (uses[s] > 0 && !mbar_wait_bounded(&empty[s], (uses[s] - 1) & 1)) s_fail = 1;
+                asm volatile("cp.async.commit_group;" ::: "memory");
 #pragma unroll
                 for (int it = 0; it < A_ITERS; ++it) {
                     const int idx = tid + it * TC_THREADS;
@@ -232,19 +244,13 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                     *reinterpret_cast<float4*>(a_hi + off) = h;
                     if (X3) *reinterpret_cast<float4*>(a_lo + off) = make_float4(x.x - h.x, x.y - h.y, x.z - h.z, x.w - h.w);
                 }
-#pragma unroll
-                for (int it = 0; it < B_ITERS; ++it) {
-                    const int idx = tid + it * TC_THREADS;
-                    if (idx < n_pad * 8) {
-                        const uint32_t off = tc_swz(idx >> 3, idx & 7);
-                        *reinterpret_cast<float4*>(b_hi + off) = bh[it];
-                        if (X3) *reinterpret_cast<float4*>(b_lo + off) = bl[it];
-                    }
-                }
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
                 fence_async_smem();   // generic-proxy stores -> visible to the tensor core's async proxy
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&full[s]);
                 uses[s]++;
+#pragma unroll
+                for (int it = 0; it < A_ITERS; ++it) ax[it] = ax_next[it];
                 if (s_fail) break;
             }
             if (s_fail) break;
