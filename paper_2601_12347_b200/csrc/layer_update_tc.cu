@@ -211,19 +211,14 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                     if (v >= 0 && k < p.K) dst[it] = upd_load_a(p, v, r0 + r, k, row_scale[r]);
                 }
             };
-            load_a(0, ax);
-            for (int kc = 0; kc < nchunks; ++kc) {
+            // asynchronous copy of chunk kc's pre-split transposed weights (n_pad output columns x 8
+            // pieces of 16 bytes, hi and lo) from L2 straight into their swizzled places in stage kc & 1;
+            // the MMAs that last read that stage must have finished
+            auto copy_b = [&](int kc) {
                 const int s = kc & 1;
-                uint8_t* a_hi = smem + (size_t)s * stage_bytes;
-                uint8_t* a_lo = a_hi + TC_A_BYTES;                              // only if X3
-                uint8_t* b_hi = a_hi + (X3 ? 2 : 1) * TC_A_BYTES;
-                uint8_t* b_lo = b_hi + b_bytes;                                 // only if X3
-                // next chunk's row gathers first (registers), so that they have a whole iteration to land
-                if (kc + 1 < nchunks) load_a(kc + 1, ax_next);
-                // the MMAs that last read this stage must have finished
+                uint8_t* b_hi = smem + (size_t)s * stage_bytes + (X3 ? 2 : 1) * TC_A_BYTES;
+                uint8_t* b_lo = b_hi + b_bytes;
                 if (uses[s] > 0 && !mbar_wait_bounded(&empty[s], (uses[s] - 1) & 1)) s_fail = 1;
-                // B: n_pad output columns x 8 chunks of the pre-split transposed weights, copied
-                // asynchronously from L2 straight into their swizzled places
 #pragma unroll
                 for (int it = 0; it < B_ITERS; ++it) {
                     const int idx = tid + it * TC_THREADS;
@@ -235,6 +230,15 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                     }
                 }
                 asm volatile("cp.async.commit_group;" ::: "memory");
+            };
+            load_a(0, ax);
+            copy_b(0);
+            for (int kc = 0; kc < nchunks; ++kc) {
+                const int s = kc & 1;
+                uint8_t* a_hi = smem + (size_t)s * stage_bytes;
+                uint8_t* a_lo = a_hi + TC_A_BYTES;                              // only if X3
+                // next chunk's row gathers first (registers), so that they have a whole iteration to land
+                if (kc + 1 < nchunks) load_a(kc + 1, ax_next);
 #pragma unroll
                 for (int it = 0; it < A_ITERS; ++it) {
                     const int idx = tid + it * TC_THREADS;
@@ -244,11 +248,13 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                     *reinterpret_cast<float4*>(a_hi + off) = h;
                     if (X3) *reinterpret_cast<float4*>(a_lo + off) = make_float4(x.x - h.x, x.y - h.y, x.z - h.z, x.w - h.w);
                 }
-                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                asm volatile("cp.async.wait_group 0;" ::: "memory");   // this chunk's weights have landed
                 fence_async_smem();   // generic-proxy stores -> visible to the tensor core's async proxy
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&full[s]);
                 uses[s]++;
+                // the next chunk's weights travel while its rows are split and stored
+                if (kc + 1 < nchunks) copy_b(kc + 1);
 #pragma unroll
                 for (int it = 0; it < A_ITERS; ++it) ax[it] = ax_next[it];
                 if (s_fail) break;
