@@ -1,4 +1,4 @@
-// Affected-row layer update (Compute + Prepare of Sec. 3.3.1): gather [h^{l-1}_v || x_v] for the
+// Affected-row layer update (Compute + Prepare of Sec. 3.3.1): gather the inputs of Update^l for the
 // rows of A_l, multiply by the layer weights, add bias, apply the activation, write h^l_v in
 // place and emit the delta row D_v = c_new h_new - c_old h_old for the next hop (Sec. 3.3.3).
 //
@@ -86,6 +86,21 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
     }
 }
 
+// K = 0: the layer's self projection and transformed aggregate are both cached, so the update is
+// elementwise (bias + cached terms + activation); one thread per 16-byte piece of a row
+__global__ void __launch_bounds__(256)
+k_update_rows_elementwise(const Ctl* ctl, UpdParams p) {
+    if (ctl->abort) return;
+    const int n = upd_rows(p), nq = p.n_cols >> 2;
+    const long long total = (long long)n * nq;
+    for (long long it = blockIdx.x * (long long)blockDim.x + threadIdx.x; it < total;
+         it += (long long)gridDim.x * blockDim.x) {
+        const int i = (int)(it / nq), q = (int)(it - (long long)i * nq);
+        const int v = p.list ? p.list[i] : i;
+        upd_epilogue4(p, v, i, 4 * q, make_float4(0.f, 0.f, 0.f, 0.f), upd_row_scale(p, v));
+    }
+}
+
 // launches both forms; exactly one of them does the work (decided on the device)
 static void launch_update(Ctx* c, UpdParams& p, const TcW& tw) {
     p.tc_mode = TC_OFF;
@@ -95,6 +110,10 @@ static void launch_update(Ctx* c, UpdParams& p, const TcW& tw) {
         p.tc_mode = c->gemm_mode == RIPPLE_GEMM_TF32 ? TC_TF32 : TC_TF32X3;
         p.tc_min_rows = 1024;
         p.Wt_hi = tw.hi; p.Wt_lo = tw.lo; p.k_pad = tw.k_pad; p.n_pad = tw.n_pad;
+    }
+    if (p.K == 0) {
+        RP_LAUNCH(c, k_update_rows_elementwise, c->n_sm * 8, 256, 0, c->ctl, p);
+        return;
     }
     RP_LAUNCH(c, k_update_rows, c->n_sm * 4, 256, 0, c->ctl, p);
     if (p.tc_mode != TC_OFF) launch_update_tc(c, p);

@@ -7,7 +7,8 @@
 
 namespace rp {
 
-enum { A_CONCAT = 0, A_SUM = 1, A_AGG = 2, A_DENSE = 3, A_SELF = 4 };
+// A operand: SUM = alpha h_v + scale S_v (GIN); AGG = scale S_v; DENSE = compact rows; SELF = alpha h_v
+enum { A_SUM = 1, A_AGG = 2, A_DENSE = 3, A_SELF = 4 };
 enum { EPI_COMMIT = 0, EPI_TEMP = 1 };
 enum { TC_OFF = 0, TC_TF32X3 = 1, TC_TF32 = 2 };
 
@@ -17,12 +18,12 @@ struct UpdParams {
     int n_host;
     int a_mode, epi_mode;
     // A operand
-    const float* Hprev; int ld_h;   // previous-layer rows (CONCAT, SUM, SELF) or dense rows (DENSE)
+    const float* Hprev; int ld_h;   // previous-layer rows (SUM, SELF) or dense rows (DENSE)
     const float* S; int ld_s;       // aggregate rows
     float alpha;                    // SUM, SELF: factor on the self row
     int agg;                        // sink-side normalisation
     const int32_t* deg_in;
-    int K;                          // reduction length (CONCAT: 2 * ld_h)
+    int K;                          // reduction length
     // B operand
     const float* W; int ldw;        // K x ldw, row-major (SIMT form)
     const float* Wt_hi;             // tensor-core form: transposed (n_pad x k_pad, K contiguous), split
@@ -69,10 +70,7 @@ __device__ __forceinline__ float4 upd_load_a(const UpdParams& p, int v, int i, i
         float4 h = __ldg(reinterpret_cast<const float4*>(p.Hprev + (size_t)v * p.ld_h + k));
         return make_float4(p.alpha * h.x, p.alpha * h.y, p.alpha * h.z, p.alpha * h.w);
     }
-    if (p.a_mode == A_CONCAT && k < p.ld_h)
-        return __ldg(reinterpret_cast<const float4*>(p.Hprev + (size_t)v * p.ld_h + k));
-    const int ks = p.a_mode == A_CONCAT ? k - p.ld_h : k;
-    float4 s = *reinterpret_cast<const float4*>(p.S + (size_t)v * p.ld_s + ks);
+    float4 s = *reinterpret_cast<const float4*>(p.S + (size_t)v * p.ld_s + k);
     float4 a = make_float4(sc * s.x, sc * s.y, sc * s.z, sc * s.w);
     if (p.a_mode == A_SUM) {
         float4 h = __ldg(reinterpret_cast<const float4*>(p.Hprev + (size_t)v * p.ld_h + k));

@@ -356,7 +356,9 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
 void launch_update_tc(Ctx* c, const UpdParams& p) {
     const bool x3 = p.tc_mode == TC_TF32X3;
     const size_t stage = (size_t)(x3 ? 2 : 1) * (TC_A_BYTES + (size_t)p.n_pad * 128);
-    const size_t smem = 2 * stage + 1024;
+    // two operand stages, reused by the epilogue as a 128 x (n_pad + 4) fp32 tile
+    const size_t tile = (size_t)TC_M * (p.n_pad + 4) * sizeof(float);
+    const size_t smem = std::max(2 * stage, tile) + 1024;
     const int per_sm = std::max<size_t>(1, std::min<size_t>(4, (size_t)(220 * 1024) / (smem + 2048)));
     const int grid = c->n_sm * per_sm;
     if (x3) {

@@ -22,7 +22,6 @@ namespace rp {
 struct Ctl {
     int abort;   // set by validation / planning: the batch is rejected, mutate nothing
     int err;     // ripple_status recorded on the device
-    int err_info;
     int n_ops;
     int n_rows;  // payload rows of the batch
     int n_rec;   // net edge changes of the batch (|dE+| + |dE-|)
@@ -78,7 +77,7 @@ struct LayerDev {
     int kind, d_in, d_hid, d_out, act;
     float eps;
     int ld_in, ld_hid, ld_out;  // padded widths (multiples of 4)
-    float* W1;   // SAGE: [W_self; W_neigh] (2 d_in x ld_out); GRAPHCONV: d_in x ld_out; GIN: d_in x ld_hid
+    float* W1;   // SAGE: [W_self; W_neigh] (2 ld_in x ld_out); GRAPHCONV: ld_in x ld_out; GIN: ld_in x ld_hid
     float* b1;   // ld_out (SAGE, GRAPHCONV) or ld_hid (GIN)
     float* W2;   // GIN: d_hid x ld_out
     float* b2;   // GIN: ld_out
@@ -123,8 +122,6 @@ struct Ctx {
     // batch staging
     ripple_update* ups_dev;
     float* feat_dev;
-    ripple_update* ups_pin;
-    float* feat_pin;
     unsigned long long* hkeys; // pair hash table
     int32_t* hseq;
     int32_t* op_slot;

@@ -534,3 +534,58 @@ def test_graph_replay_and_direct_launch_agree(env):
     check_values(b, ref, 3)
     a.close()
     b.close()
+
+
+@pytest.mark.parametrize("mix", [(0.0, 0.0, 1.0), (0.1, 0.8, 0.1)], ids=["hub-feature-only", "hub-delete-heavy"])
+def test_hub_stress_streams(env, mix):
+    """Every endpoint among the top-1 % out-degree vertices: frontiers saturate within two hops and
+    the same few long rows are searched, shrunk and walked again and again."""
+    ripple, Oracle = env
+    w = I.workloads()["sparse"]
+    src, dst = I.make_graph(w)
+    model = I.sage_model([24, 32, 32, 8], I.AGG_MEAN)
+    X = I.features(w.n, 24, 2)
+    W = I.make_weights(model, 2)
+    hubs = I.top_out_degree(w.n, src)
+    rp = ripple.Ripple(w.n, src, dst, X, model, W)
+    orc = Oracle(w.n, src, dst, X, model, W)
+    stream = I.UpdateStream(w.n, src, dst, 24, 2, mix=mix, hubs=hubs)
+    for b in range(6):
+        ups, rows = stream.next_batch(300)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        check_frontiers(rp, orc, 3)
+    check_graph(rp, orc)
+    st = rp.stats()
+    assert st["affected"][3] > 0.3 * w.n          # saturated: a third of all vertices and more
+    check_values(rp, orc.full(), 3, [None] + [orc.full_S(l) for l in range(1, 4)])
+    rp.close()
+
+
+def test_gemm_modes_and_their_tolerances(env):
+    """Wide layers with enough rows take the tensor-core path.  Default (TF32 with a 3-term split)
+    and forced fp32 SIMT must both meet 1e-4; plain TF32 is allowed 2e-2 and must still be close."""
+    ripple, Oracle = env
+    model = I.sage_model([64, 160, 128, 32], I.AGG_MEAN)
+    n, m = 5000, 60000
+    src, dst = I.er_graph(n, m, 29)
+    X = I.features(n, 64, 29)
+    W = I.make_weights(model, 29, zero_bias=False)
+    orc = Oracle(n, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, 64, 29)
+    batches = [stream.next_batch(400) for _ in range(4)]
+    for ups, rows in batches:
+        assert orc.apply_incremental(ups, rows) == 0
+    ref = orc.full()
+    assert orc.affected(2).size >= 1024               # the incremental path reaches the tensor-core form too
+    errs = {}
+    for name, mode, tol in (("auto", ripple.GEMM_AUTO, 1e-4), ("fp32", ripple.GEMM_FP32, 1e-4),
+                            ("tf32", ripple.GEMM_TF32, 2e-2)):
+        rp = ripple.Ripple(n, src, dst, X, model, W, gemm_mode=mode)
+        for ups, rows in batches:
+            rp.apply_batch(ups, rows)
+        check_frontiers(rp, orc, 3)
+        errs[name] = max(max_err(rp.embeddings(l).cpu().numpy(), ref[l]) for l in range(4))
+        assert errs[name] <= tol, (name, errs[name])
+        rp.close()
+    assert errs["tf32"] > 10 * errs["auto"]           # the single-pass form really is the coarser one
