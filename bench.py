@@ -295,10 +295,11 @@ def run_ours(args, rank, world, local_rank):
     e2e_ms = e0.elapsed_time(e1)
 
     dev_ms, e2e_ms = max_over_ranks([dev_ms, e2e_ms], world)
+    if world > 1:   # the replicas are done with each other; rank 0 alone reports
+        dist.barrier()
+        dist.destroy_process_group()
     if rank != 0:
         rp.close()
-        if world > 1:
-            dist.destroy_process_group()
         return
 
     peak, peak_kind = load_peaks()
@@ -345,8 +346,6 @@ def run_ours(args, rank, world, local_rank):
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args, w, src, dst, X, W)
     print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
 
 
 def run_table(args):

@@ -589,3 +589,45 @@ def test_gemm_modes_and_their_tolerances(env):
         assert errs[name] <= tol, (name, errs[name])
         rp.close()
     assert errs["tf32"] > 10 * errs["auto"]           # the single-pass form really is the coarser one
+
+
+def test_mixed_growth_and_deletion_in_the_same_rows(env):
+    """Batches that delete from and add to the same few rows at once, with almost no slack, so that
+    rows are compacted, relocated into the overflow pool and appended to within one batch."""
+    ripple, Oracle = env
+    model = I.graphconv_model([6, 8, 4], I.AGG_WSUM_GCN)
+    n = 900
+    rng = np.random.default_rng(3)
+    hubs = np.arange(8)
+    present = set()
+    for h in hubs:                                   # every hub starts with ~200 out- and in-edges
+        for v in rng.choice(np.arange(8, n), size=200, replace=False):
+            present.add((int(h), int(v)))
+            present.add((int(v), int(h)))
+    src = np.array([a for a, _ in sorted(present)], dtype=np.int32)
+    dst = np.array([b for _, b in sorted(present)], dtype=np.int32)
+    X = I.features(n, 6, 3)
+    W = I.make_weights(model, 3)
+    rp = ripple.Ripple(n, src, dst, X, model, W, slack=0.01, pool_edges=200000)
+    orc = Oracle(n, src, dst, X, model, W)
+    for b in range(12):
+        recs = []
+        cur = sorted(present)
+        for idx in rng.choice(len(cur), size=150, replace=False):      # deletions spread over the hub rows
+            recs.append((I.OP_DEL_EDGE, cur[idx][0], cur[idx][1]))
+            present.discard(cur[idx])
+        while len(recs) < 450:                                          # twice as many additions to the same rows
+            h, v = int(rng.choice(hubs)), int(rng.integers(8, n))
+            p = (h, v) if rng.random() < 0.5 else (v, h)
+            if p not in present and all(p != (r[1], r[2]) for r in recs):
+                recs.append((I.OP_ADD_EDGE, p[0], p[1]))
+                present.add(p)
+        order = rng.permutation(len(recs))
+        ups = ups_array([recs[i] for i in order])
+        rp.apply_batch(ups)
+        assert orc.apply_incremental(ups) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, 2)
+    assert rp.stats()["pool_used"] > 0 and rp.stats()["num_edges"] == len(present)
+    check_values(rp, orc.full(), 2)
+    rp.close()
