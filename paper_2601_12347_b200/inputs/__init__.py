@@ -115,9 +115,10 @@ def rmat_graph(n: int, m: int, seed: int, a: float = 0.57, b: float = 0.19, c: f
     scale = max(1, int(np.ceil(np.log2(n))))
     keys = np.empty(0, dtype=np.int64)
     drawn = 0
+    yield_ = 1.0 / 1.35        # distinct new pairs per candidate, re-estimated after every round
     while keys.size < m:
         need = m - keys.size
-        cnt = int(need * (1.35 if keys.size == 0 else 2.0)) + 1024
+        cnt = int(need * 1.35) + 1024 if drawn == 0 else int(need / max(yield_, 0.02) * 1.05) + 1024
         u = np.empty(cnt, dtype=np.int32)
         v = np.empty(cnt, dtype=np.int32)
         lib.rmat_pairs(ctypes.c_uint64(seed), ctypes.c_uint64(drawn), cnt, scale, a, b, c,
@@ -126,12 +127,9 @@ def rmat_graph(n: int, m: int, seed: int, a: float = 0.57, b: float = 0.19, c: f
         ok = (u < n) & (v < n) & (u != v)
         k = u[ok].astype(np.int64) * n + v[ok]
         del u, v, ok
-        k = _sorted_unique(k)
-        if keys.size:
-            k = k[~np.isin(k, keys, assume_unique=True)]
-            keys = np.union1d(keys, k)
-        else:
-            keys = k
+        before = keys.size
+        keys = _sorted_unique(np.concatenate([keys, k])) if before else _sorted_unique(k)
+        yield_ = max(keys.size - before, 1) / cnt
     if keys.size > m:
         drop = _rng(seed, "drop").choice(keys.size, size=keys.size - m, replace=False)
         mask = np.ones(keys.size, dtype=bool)
@@ -395,6 +393,14 @@ def workloads() -> Dict[str, Workload]:
                            (1000,), 20),
         "dense-3l": Workload("dense-3l", n_d, e_d, "rmat", sage_model([100, 256, 256, 47]), 0,
                              (10, 100, 1000, 10000), 100),
+        "dense-4l": Workload("dense-4l", n_d, e_d, "rmat", sage_model([100, 256, 256, 256, 47]), 0,
+                             (100, 1000), 20),
+        # ultra-dense second graph shaped like the paper's social-network dataset (Table 2: 233 K
+        # vertices, 114.9 M edges, average in-degree 492, 602 features, 41 classes)
+        "reddit-2l": Workload("reddit-2l", 232_965, 114_900_000, "rmat", sage_model([602, 256, 41]), 0,
+                              (10, 100, 1000), 20),
+        "reddit-4l": Workload("reddit-4l", 232_965, 114_900_000, "rmat",
+                              sage_model([602, 256, 256, 256, 41]), 0, (100, 1000), 20),
         # hub stress: every endpoint is one of the top-1 % out-degree vertices of the initial graph
         "dense-3l-hub-feature": Workload("dense-3l-hub-feature", n_d, e_d, "rmat",
                                          sage_model([100, 256, 256, 47]), 0, (1, 10, 100, 1000), 20,

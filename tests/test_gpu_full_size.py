@@ -1,5 +1,6 @@
 """Parity at full size, in the launch configuration bench.py times (dense graph, 2-layer
-GraphSAGE-mean 100-256-47, batches of 1000).
+GraphSAGE-mean 100-256-47, batches of 1000), and on the ultra-dense second graph (233 K vertices,
+114.9 M edges, 602 features).
 
 The oracle cannot recompute 2.4 M x 256 embeddings per batch in test time, so here
   * graph state, affected sets and counters are compared exactly, batch by batch, against the
@@ -19,7 +20,8 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-4
 
 
-def test_dense_2l_batch_1000_sampled_rows():
+@pytest.mark.parametrize("wname,n_batches", [("dense-2l", 3), ("reddit-2l", 2)])
+def test_full_size_batch_1000_sampled_rows(wname, n_batches):
     import torch
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
@@ -28,7 +30,7 @@ def test_dense_2l_batch_1000_sampled_rows():
     from paper_2601_12347_b200 import ripple
     from oracle.oracle import Oracle
     torch.cuda.set_device(0)
-    w = I.workloads()["dense-2l"]
+    w = I.workloads()[wname]
     src, dst = I.make_graph(w)
     X = I.features(w.n, w.model.dims[0], w.seed)
     W = I.make_weights(w.model, w.seed)
@@ -37,7 +39,7 @@ def test_dense_2l_batch_1000_sampled_rows():
     orc = Oracle(w.n, src, dst, X, w.model, W, bootstrap=False)
     stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], w.seed)
     feat_now = {}
-    for b in range(3):
+    for b in range(n_batches):
         ups, rows = stream.next_batch(1000)
         rp.apply_batch(ups, rows)
         assert orc.apply_structure(ups, rows.shape[0]) == 0
@@ -79,5 +81,5 @@ def test_dense_2l_batch_1000_sampled_rows():
             err = float(np.max(np.abs(H[l][v].astype(np.float64) - ref) / (1.0 + np.abs(ref))))
             worst = max(worst, err)
             assert err <= TOL, f"layer {l}, vertex {v} (in-degree {odi[v]}): err {err}"
-    print(f"dense-2l sampled rows: {len(sample)} vertices x {L} layers, worst err {worst:.2e}")
+    print(f"{wname} sampled rows: {len(sample)} vertices x {L} layers, worst err {worst:.2e}")
     rp.close()
