@@ -361,13 +361,14 @@ def run_table(args):
     for name in args.table.split(","):
         w, src, dst, X, W = make_workload(name, args.seed)
         L = len(w.model.layers)
-        rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=16384, scatter_mode=args.scatter)
+        rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=16384, scatter_mode=args.scatter,
+                           regather_threshold=args.regather_threshold)
         boot = rp.stats()["ms_bootstrap"]
         rp.recompute_full()   # warm: the recompute-everything alternative on the same state
         full_ms = rp.stats()["ms_bootstrap"]
         stream = I.make_stream(w, src, dst, args.seed)
         orc = ostream = None
-        if not args.no_cpu_baseline:
+        if not args.no_cpu_baseline and args.oracle_seconds > 0:
             from oracle import oracle as O
             O.build()
             orc = O.Oracle(w.n, src, dst, X, w.model, W)
@@ -383,6 +384,7 @@ def run_table(args):
             lat, sc_ms, sc_bytes = [], 0.0, 0
             stage = {"graph": 0.0, "frontier": 0.0, "scatter": 0.0, "update": 0.0}
             aff, act = np.zeros(L + 1), np.zeros(L + 1)
+            hop = {k: np.zeros(L + 1) for k in ("scatter", "update", "regather", "rebuilt")}
             rp.set_timing(False)
             for i, (u, r) in enumerate(pinned):
                 if i == 5 + nb:
@@ -402,6 +404,10 @@ def run_table(args):
                     stage["scatter"] += s["ms_scatter"][l]
                     stage["update"] += s["ms_update"][l]
                 sc_ms += s["ms_scatter_kernel"][L]
+                hop["scatter"] += np.array(s["ms_scatter"][: L + 1])
+                hop["update"] += np.array(s["ms_update"][: L + 1])
+                hop["regather"] += np.array(s["ms_regather"][: L + 1])
+                hop["rebuilt"] += np.array(s["scatter_pull"][: L + 1]) == 2
                 sc_bytes += scatter_bytes(s, L, s["message_width"][L])
                 aff += np.array(s["affected"][: L + 1])
                 act += np.array(s["active_edges"][: L + 1])
@@ -412,6 +418,7 @@ def run_table(args):
                     "affected": (aff / nt).round(1).tolist(), "active_edges": (act / nt).round(1).tolist(),
                     "last_hop_scatter": {"ms": sc_ms / nt, "algorithmic_GBps": (sc_bytes / 1e9) / (sc_ms / 1e3) if sc_ms else None,
                                          "frac_of_" + peak_kind: ((sc_bytes / 1e9) / (sc_ms / 1e3) / peak) if sc_ms else None},
+                    "hop_ms": {k: (v[1:] / nt).round(3).tolist() for k, v in hop.items()},
                     "bootstrap_ms": boot, "full_recompute_ms": full_ms}
             if orc is not None:
                 spent, done = 0.0, 0
@@ -435,6 +442,8 @@ def main():
     ap.add_argument("--table", default="", help="comma-separated workloads: print one line per batch size")
     ap.add_argument("--table-batches", type=int, default=100)
     ap.add_argument("--oracle-seconds", type=float, default=10.0)
+    ap.add_argument("--regather-threshold", type=float, default=0.0,
+                    help="share of all edges from which a hop rebuilds its aggregates (0: library default, <0: never)")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)

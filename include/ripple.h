@@ -60,11 +60,19 @@ typedef enum { RIPPLE_LAYER_SAGE = 0, RIPPLE_LAYER_GRAPHCONV = 1, RIPPLE_LAYER_G
 
 typedef enum { RIPPLE_ACT_IDENTITY = 0, RIPPLE_ACT_RELU = 1 } ripple_act;
 
-/* The three update types on this path (of the five of Sec. 3.1). */
-typedef enum { RIPPLE_OP_ADD_EDGE = 0, RIPPLE_OP_DEL_EDGE = 1, RIPPLE_OP_SET_FEATURE = 2 } ripple_op;
+/* The update types of Sec. 3.1.  Vertex ids live in [0, num_vertices) for the life of the context:
+ * num_vertices is a capacity.
+ *   - Vertex deletion (Sec. 3.2): DEL_VERTEX removes, at its position in the batch, every edge
+ *     that has u as an endpoint and replaces u's feature row by zeros; propagation starts from u
+ *     as root (the sinks of the removed edges and u itself are affected).  The id stays valid.
+ *   - Vertex addition arrives, as in Sec. 4.1, as the edge addition that first names an unused
+ *     id (plus a SET_FEATURE for its row); an unused id is an isolated vertex with a zero row. */
+typedef enum {
+    RIPPLE_OP_ADD_EDGE = 0, RIPPLE_OP_DEL_EDGE = 1, RIPPLE_OP_SET_FEATURE = 2, RIPPLE_OP_DEL_VERTEX = 3
+} ripple_op;
 
 /* One update.  ADD_EDGE / DEL_EDGE: edge (u, v).  SET_FEATURE: vertex u takes row `v` of the
- * batch's feature payload. */
+ * batch's feature payload.  DEL_VERTEX: vertex u (v is ignored). */
 typedef struct {
     int32_t op;
     int32_t u;
@@ -99,7 +107,14 @@ typedef struct {
     const float* bb;
 } ripple_layer;
 
-typedef enum { RIPPLE_SCATTER_AUTO = 0, RIPPLE_SCATTER_PUSH = 1, RIPPLE_SCATTER_PULL = 2 } ripple_scatter_mode;
+/* How hop l brings the cached aggregates S^l up to date.  PUSH / PULL: delta messages (Sec. 3.3.1),
+ * scattered along the senders' out-edges or gathered per affected sink.  REGATHER: the aggregates
+ * of the affected vertices are rebuilt from their in-lists (the scoped recomputation of Sec. 3.2,
+ * for this hop only).  AUTO: PUSH, except that a hop whose senders own at least
+ * regather_threshold of all edges rebuilds. */
+typedef enum {
+    RIPPLE_SCATTER_AUTO = 0, RIPPLE_SCATTER_PUSH = 1, RIPPLE_SCATTER_PULL = 2, RIPPLE_SCATTER_REGATHER = 3
+} ripple_scatter_mode;
 typedef enum { RIPPLE_GEMM_AUTO = 0, RIPPLE_GEMM_FP32 = 1, RIPPLE_GEMM_TF32 = 2 } ripple_gemm_mode;
 
 /* Zero-initialise for defaults. */
@@ -116,6 +131,8 @@ typedef struct {
     int32_t no_graphs;    /* non-zero: never replay small batches (<= 512 updates) as a captured CUDA graph     */
     int32_t device;       /* CUDA device ordinal, or -1 for the current device                              */
     void* stream;         /* cudaStream_t to run on (NULL: the library creates its own)                     */
+    float regather_threshold; /* AUTO only: a hop rebuilds its aggregates once its messages number at least
+                             this share of all edges.  0: default (0.7); < 0: never                       */
 } ripple_options;
 
 typedef struct {
@@ -127,7 +144,7 @@ typedef struct {
     int64_t affected[RIPPLE_MAX_LAYERS + 1];      /* |A_l|, l = 0..L                                      */
     int64_t senders[RIPPLE_MAX_LAYERS + 1];       /* |C_l|: vertices whose outgoing message changed       */
     int64_t active_edges[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: edges carrying a message at hop l          */
-    int32_t scatter_pull[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: 1 if hop l gathered over in-edges          */
+    int32_t scatter_pull[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: 0 push, 1 pull, 2 aggregates rebuilt       */
     int64_t in_edges[RIPPLE_MAX_LAYERS + 1];      /* l = 1..L: in-edges of A_l (what a gather walks)      */
     int32_t message_width[RIPPLE_MAX_LAYERS + 1]; /* l = 1..L: floats per message / aggregate row (padded) */
     int64_t pool_used, pool_size;                 /* overflow pool, edges, out-direction                  */
@@ -137,8 +154,10 @@ typedef struct {
     float ms_scatter[RIPPLE_MAX_LAYERS + 1];
     float ms_update[RIPPLE_MAX_LAYERS + 1];
     float ms_scatter_kernel[RIPPLE_MAX_LAYERS + 1]; /* the push or pull kernel alone, l = 1..L               */
+    float ms_regather[RIPPLE_MAX_LAYERS + 1];     /* the gather of a rebuilding hop alone, l = 1..L       */
     float ms_bootstrap;                           /* last ripple_create / ripple_recompute_full           */
     int64_t gpu_launches;                         /* kernels launched by the last call                    */
+    int64_t n_expanded;                           /* last batch: edge deletions generated by vertex deletions */
 } ripple_stats;
 
 /* Sec. 3.1 (preliminaries): the bootstrap embeddings exist before updates arrive.  Builds the
@@ -154,7 +173,12 @@ ripple_status ripple_create(const ripple_graph* g, const float* features, int32_
  * in order (the last operation on a pair, and the last payload of a vertex, win; adding an
  * existing edge or deleting a missing one is counted and ignored), then propagates the changes
  * through all L layers.  ups and feat_rows (n_rows x d0, leading dimension d0) are HOST|DEVICE
- * per `mem`.  Returns after the embeddings are up to date.  n = 0 is valid. */
+ * per `mem`.  Returns after the embeddings are up to date.  n = 0 is valid.
+ * A DEL_VERTEX is expanded on the device into one DEL_EDGE per incident edge; the given and the
+ * generated operations together must not exceed max_batch (else CAPACITY, nothing is changed).
+ * An explicit operation on an edge of u that precedes DEL_VERTEX(u) is superseded by it; one that
+ * follows it acts on the emptied vertex.  Only the given operations are counted in n_superseded
+ * and the no-op counters; edges removed by a vertex deletion are counted in n_deleted. */
 ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update* ups, int64_t n,
                                  const float* feat_rows, int64_t n_rows, int32_t mem);
 

@@ -22,7 +22,12 @@
  *     both from the current graph; a source whose out-degree changed re-sends at every hop;
  *   - "affected" is structural: it follows from the recurrence alone, never from values;
  *   - within a batch the last operation on a pair wins; adding an existing edge or deleting a
- *     missing one changes nothing; the last feature payload of a vertex wins.
+ *     missing one changes nothing; the last feature payload of a vertex wins;
+ *   - deleting a vertex (Sec. 3.2: "a delete of all edges incident upon" it, then propagation from
+ *     it as root) removes, at that point of the batch, every edge that has it as an endpoint and
+ *     replaces its feature row by zeros; the id stays addressable, so later operations of the same
+ *     or a later batch may attach edges or features to it again (a vertex addition, which the
+ *     paper models as the edge addition that creates the endpoint, Sec. 4.1);
  *
  * Parity with the authors' own program is unpinned for the mean and weighted-sum degree handling
  * (the paper gives no formula); parity with the definition (orc_full) is pinned for all of it.
@@ -40,7 +45,7 @@
 enum { KIND_SAGE = 0, KIND_GRAPHCONV = 1, KIND_GIN = 2 };
 enum { AGG_SUM = 0, AGG_MEAN = 1, AGG_WSUM_GCN = 2 };
 enum { ACT_IDENTITY = 0, ACT_RELU = 1 };
-enum { OP_ADD_EDGE = 0, OP_DEL_EDGE = 1, OP_SET_FEATURE = 2 };
+enum { OP_ADD_EDGE = 0, OP_DEL_EDGE = 1, OP_SET_FEATURE = 2, OP_DEL_VERTEX = 3 };
 
 typedef struct { int32_t op, u, v; } update_t;
 
@@ -296,28 +301,58 @@ typedef struct {
     int nF;
 } delta_t;
 
+/* last explicit edge operation on (u, v) in the sorted table, or NULL */
+static const eop_t *eop_last(const eop_t *eo, int ne, int u, int v) {
+    int lo = 0, hi = ne;   /* first entry with (u', v') > (u, v) */
+    while (lo < hi) {
+        int mid = (lo + hi) / 2;
+        if (eo[mid].u < u || (eo[mid].u == u && eo[mid].v <= v)) lo = mid + 1; else hi = mid;
+    }
+    if (lo == 0 || eo[lo - 1].u != u || eo[lo - 1].v != v) return NULL;
+    return &eo[lo - 1];
+}
+
+/* Net effect of applying the operations one after the other:
+ *   - an edge operation is the final word on its pair if no later edge operation names the pair
+ *     and neither endpoint is deleted later; it then adds / deletes the edge or is a counted no-op;
+ *     every other edge operation is counted as superseded;
+ *   - a vertex deletion removes every edge of E_old at that vertex whose pair has no final word;
+ *   - the last of {feature replacement, deletion} of a vertex fixes its row (deletion: zeros). */
 static int normalise(oracle_t *o, const update_t *ups, int64_t n, int64_t n_rows, delta_t *dl) {
     memset(dl, 0, sizeof(*dl));
     for (int64_t i = 0; i < n; ++i) {
-        if (ups[i].op < 0 || ups[i].op > 2) return -1;
+        if (ups[i].op < 0 || ups[i].op > 3) return -1;
         if (ups[i].u < 0 || ups[i].u >= o->N) return -2;
+        if (ups[i].op == OP_DEL_VERTEX) continue;
         if (ups[i].op == OP_SET_FEATURE) { if (ups[i].v < 0 || ups[i].v >= n_rows) return -1; }
         else if (ups[i].v < 0 || ups[i].v >= o->N) return -2;
     }
     eop_t *eo = (eop_t *)malloc(sizeof(eop_t) * (size_t)(n + 1));
     fop_t *fo = (fop_t *)malloc(sizeof(fop_t) * (size_t)(n + 1));
-    int ne = 0, nf = 0;
+    int *gone = (int *)malloc(sizeof(int) * (size_t)(n + 1));   /* deleted vertices, one entry per deletion */
+    int ne = 0, nf = 0, ng = 0;
+    int *vdel = NULL;   /* position of the last deletion of each vertex, -1 if none */
     for (int64_t i = 0; i < n; ++i) {
-        if (ups[i].op == OP_SET_FEATURE) { fo[nf].v = ups[i].u; fo[nf].seq = (int)i; fo[nf].row = ups[i].v; nf++; }
-        else { eo[ne].u = ups[i].u; eo[ne].v = ups[i].v; eo[ne].seq = (int)i; eo[ne].op = ups[i].op; ne++; }
+        if (ups[i].op == OP_DEL_VERTEX) {
+            if (!vdel) { vdel = (int *)malloc(sizeof(int) * (size_t)o->N); for (int v = 0; v < o->N; ++v) vdel[v] = -1; }
+            vdel[ups[i].u] = (int)i;
+            gone[ng++] = ups[i].u;
+            fo[nf].v = ups[i].u; fo[nf].seq = (int)i; fo[nf].row = -1; nf++;
+        } else if (ups[i].op == OP_SET_FEATURE) {
+            fo[nf].v = ups[i].u; fo[nf].seq = (int)i; fo[nf].row = ups[i].v; nf++;
+        } else { eo[ne].u = ups[i].u; eo[ne].v = ups[i].v; eo[ne].seq = (int)i; eo[ne].op = ups[i].op; ne++; }
     }
     qsort(eo, (size_t)ne, sizeof(eop_t), cmp_eop);
     qsort(fo, (size_t)nf, sizeof(fop_t), cmp_fop);
+    size_t del_cap = (size_t)ne + 1;
+    for (int i = 0; i < ng; ++i) del_cap += (size_t)o->out[gone[i]].n + (size_t)o->in[gone[i]].n;
     dl->add = (pair_t *)malloc(sizeof(pair_t) * (size_t)(ne + 1));
-    dl->del = (pair_t *)malloc(sizeof(pair_t) * (size_t)(ne + 1));
+    dl->del = (pair_t *)malloc(sizeof(pair_t) * del_cap);
     o->noop_add = o->noop_del = o->superseded = 0;
+#define FINAL_WORD(e) (!vdel || ((e)->seq > vdel[(e)->u] && (e)->seq > vdel[(e)->v]))
     for (int i = 0; i < ne; ++i) {
         if (i + 1 < ne && eo[i + 1].u == eo[i].u && eo[i + 1].v == eo[i].v) { o->superseded++; continue; }
+        if (!FINAL_WORD(&eo[i])) { o->superseded++; continue; }
         int present = ivec_find(&o->out[eo[i].u], eo[i].v) >= 0;
         if (eo[i].op == OP_ADD_EDGE) {
             if (present) o->noop_add++;
@@ -327,6 +362,27 @@ static int normalise(oracle_t *o, const update_t *ups, int64_t n, int64_t n_rows
             else { dl->del[dl->n_del].u = eo[i].u; dl->del[dl->n_del].v = eo[i].v; dl->n_del++; }
         }
     }
+    if (ng) {
+        for (int i = 0; i < ng; ++i) {
+            int w = gone[i];
+            for (int side = 0; side < 2; ++side) {
+                const ivec *r = side ? &o->in[w] : &o->out[w];
+                for (int j = 0; j < r->n; ++j) {
+                    int u = side ? r->a[j] : w, v = side ? w : r->a[j];
+                    const eop_t *e = eop_last(eo, ne, u, v);
+                    if (e && FINAL_WORD(e)) continue;   /* a later operation on the pair decided */
+                    dl->del[dl->n_del].u = u; dl->del[dl->n_del].v = v; dl->n_del++;
+                }
+            }
+        }
+        /* a pair is met once per deleted endpoint and per list it is in: keep one copy */
+        qsort(dl->del, (size_t)dl->n_del, sizeof(pair_t), cmp_pair);
+        int k = 0;
+        for (int i = 0; i < dl->n_del; ++i)
+            if (k == 0 || dl->del[k - 1].u != dl->del[i].u || dl->del[k - 1].v != dl->del[i].v) dl->del[k++] = dl->del[i];
+        dl->n_del = k;
+    }
+#undef FINAL_WORD
     dl->F = (int *)malloc(sizeof(int) * (size_t)(nf + 1));
     dl->Frow = (int *)malloc(sizeof(int) * (size_t)(nf + 1));
     for (int i = 0; i < nf; ++i) {
@@ -334,7 +390,7 @@ static int normalise(oracle_t *o, const update_t *ups, int64_t n, int64_t n_rows
         dl->F[dl->nF] = fo[i].v; dl->Frow[dl->nF] = fo[i].row; dl->nF++;
     }
     o->n_added = dl->n_add; o->n_deleted = dl->n_del;
-    free(eo); free(fo);
+    free(eo); free(fo); free(gone); free(vdel);
     return 0;
 }
 
@@ -465,8 +521,8 @@ int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const flo
     for (int i = 0; i < nA; ++i) {
         double *row = o->H[0] + (size_t)A[i] * d0;
         memcpy(oldA + (size_t)i * d0, row, sizeof(double) * (size_t)d0);
-        const float *src = feat_rows + (size_t)dl.Frow[i] * d0;
-        for (int k = 0; k < d0; ++k) row[k] = (double)src[k];
+        const float *src = dl.Frow[i] >= 0 ? feat_rows + (size_t)dl.Frow[i] * d0 : NULL;   /* deleted vertex: zeros */
+        for (int k = 0; k < d0; ++k) row[k] = src ? (double)src[k] : 0.0;
     }
     set_list(o, 0, A, nA);
     int nC; int *C = changed_senders(o, &dl, A, nA, &nC);
@@ -554,8 +610,8 @@ int orc_apply_scoped(oracle_t *o, const update_t *ups, int64_t n, const float *f
     memcpy(A, dl.F, sizeof(int) * (size_t)nA);
     for (int i = 0; i < nA; ++i) {
         double *row = o->H[0] + (size_t)A[i] * d0;
-        const float *src = feat_rows + (size_t)dl.Frow[i] * d0;
-        for (int k = 0; k < d0; ++k) row[k] = (double)src[k];
+        const float *src = dl.Frow[i] >= 0 ? feat_rows + (size_t)dl.Frow[i] * d0 : NULL;   /* deleted vertex: zeros */
+        for (int k = 0; k < d0; ++k) row[k] = src ? (double)src[k] : 0.0;
     }
     set_list(o, 0, A, nA);
     int nC; int *C = changed_senders(o, &dl, A, nA, &nC);

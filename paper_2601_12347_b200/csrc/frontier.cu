@@ -198,6 +198,59 @@ __global__ void k_mark_frontier(Ctl* ctl, int l, int self_term, int walk, const 
     }
 }
 
+// Rebuilding hops mark bottom-up (the direction switch of a frontier search that has reached most
+// of the graph): v belongs to Out_new(C_{l-1}) iff one of its in-neighbours is a sender.  With the
+// senders owning most edges the first few probes of the position map settle almost every vertex,
+// where walking the senders' out-lists would look up the bitmap once per edge (measured 1.2 ms on
+// 123 M edges against 0.1 ms).  Four lanes per vertex probe the first 64 in-neighbours; the few
+// vertices still undecided with longer lists are queued for a warp each.
+constexpr int BU_LANES = 4, BU_FIRST = 64;
+
+__global__ void __launch_bounds__(256)
+k_mark_bottom_up(Ctl* ctl, int l, int N, Side in, const int32_t* __restrict__ posmap, uint32_t* bitmap,
+                 int32_t* overflow, int* n_overflow) {
+    if (ctl->abort || !ctl->regather[l]) return;
+    const int gtid = blockIdx.x * blockDim.x + threadIdx.x, groups = (gridDim.x * blockDim.x) / BU_LANES;
+    const int sub = threadIdx.x & (BU_LANES - 1);
+    const unsigned group = 0xFu << ((threadIdx.x & 31) & ~(BU_LANES - 1));   // the four lanes that share a vertex
+    for (int v = gtid / BU_LANES; v < N; v += groups) {
+        const int deg = in.deg[v];
+        if (deg == 0 || (bitmap[v >> 5] & (1u << (v & 31)))) continue;   // same outcome in all four lanes
+        const int64_t base = in.start[v];
+        const int lim = min(deg, BU_FIRST);
+        bool hit = false;
+        for (int j0 = 0; j0 < lim && !hit; j0 += BU_LANES) {
+            const int j = j0 + sub;
+            const bool mine = j < lim && posmap[in.col[base + j]] >= 0;
+            hit = __any_sync(group, mine);
+        }
+        if (sub == 0) {
+            if (hit) set_bit(bitmap, v);
+            else if (deg > BU_FIRST) overflow[atomicAdd(n_overflow, 1)] = v;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+k_mark_bottom_up_long(Ctl* ctl, int l, Side in, const int32_t* __restrict__ posmap, uint32_t* bitmap,
+                      const int32_t* __restrict__ overflow, const int* __restrict__ n_overflow) {
+    if (ctl->abort || !ctl->regather[l]) return;
+    const int n = *n_overflow;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id();
+    for (int i = warp; i < n; i += nwarps) {
+        const int v = overflow[i];
+        const int deg = in.deg[v];
+        const int64_t base = in.start[v];
+        bool hit = false;
+        for (int j0 = BU_FIRST; j0 < deg && !hit; j0 += 32) {
+            bool mine = j0 + lane < deg && posmap[in.col[base + j0 + lane]] >= 0;
+            hit = __any_sync(FULL, mine);
+        }
+        if (hit && lane == 0) set_bit(bitmap, v);
+    }
+}
+
 void frontier_seed_features(Ctx* c, int n) {
     (void)n;
     bitmap_to_list(c, c->A[0], &c->ctl->nA[0], nullptr);
@@ -208,6 +261,14 @@ void frontier_seed_features(Ctx* c, int n) {
 void frontier_mark(Ctx* c, int l, bool walk) {
     RP_LAUNCH(c, k_mark_frontier, walk ? c->n_sm * 8 : c->n_sm * 2, 256, 0, c->ctl, l, (int)c->self_term,
               (int)walk, c->Clist[(l - 1) & 1], c->coff, c->side[0], c->rec, c->A[l - 1], c->bitmap);
+    const bool may_rebuild = c->scatter_mode == RIPPLE_SCATTER_REGATHER ||
+                             (c->scatter_mode == RIPPLE_SCATTER_AUTO && c->regather_threshold[l] > 0.f);
+    if (!may_rebuild) return;
+    // the list A_l is not built yet: its buffer holds the queue of undecided long rows
+    RP_LAUNCH(c, k_mark_bottom_up, c->n_sm * 8, 256, 0, c->ctl, l, c->N, c->side[1], c->posmap, c->bitmap, c->A[l],
+              &c->ctl->n_long[l]);
+    RP_LAUNCH(c, k_mark_bottom_up_long, c->n_sm * 4, 256, 0, c->ctl, l, c->side[1], c->posmap, c->bitmap, c->A[l],
+              &c->ctl->n_long[l]);
 }
 
 void frontier_compact(Ctx* c, int l) {

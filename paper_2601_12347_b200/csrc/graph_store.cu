@@ -103,43 +103,102 @@ cudaError_t graph_build(Ctx* c, const int32_t* src, const int32_t* dst, int64_t 
 // ---------------------------------------------------------------------------------------------
 // batch normalisation
 // ---------------------------------------------------------------------------------------------
-__global__ void k_classify(const ripple_update* __restrict__ ups, int n, int N, Ctl* ctl,
-                           unsigned long long* hkeys, int32_t* hseq, int hmask, int32_t* op_slot,
-                           int32_t* feat_last) {
-    int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    ripple_update op = ups[i];
-    op_slot[i] = -1;
-    if (op.op < 0 || op.op > 2) {
-        atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_INVALID_ARG);
-        ctl->abort = 1;
-        return;
-    }
-    bool bad = (unsigned)op.u >= (unsigned)N;
-    if (op.op == RIPPLE_OP_SET_FEATURE) bad |= (unsigned)op.v >= (unsigned)ctl->n_rows;
-    else bad |= (unsigned)op.v >= (unsigned)N;
-    if (bad) {
-        atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_VERTEX_RANGE);
-        ctl->abort = 1;
-        return;
-    }
-    if (op.op == RIPPLE_OP_SET_FEATURE) {
-        atomicMax(&feat_last[op.u], i);
-        return;
-    }
-    unsigned long long key = (unsigned long long)op.u * (unsigned long long)N + (unsigned long long)op.v + 1ull;
-    int h = (int)(mix64(key) & (unsigned long long)hmask);
-    for (int probe = 0; probe <= hmask; ++probe) {
-        unsigned long long prev = atomicCAS(&hkeys[h], 0ull, key);
-        if (prev == 0ull || prev == key) {
-            atomicMax(&hseq[h], i);
-            op_slot[i] = h;
-            return;
+// number of operations after vertex deletions have been expanded into edge deletions
+__device__ __forceinline__ int ops_total(const Ctl* ctl) {
+    return ctl->n_ops + (ctl->expand_failed ? 0 : (int)ctl->n_extra);
+}
+
+// Vertex deletion (Sec. 3.2): "a delete of all edges incident upon" the vertex.  Each deletion
+// reserves room behind the caller's operations for one edge deletion per stored out- and
+// in-neighbour; the generated operations carry the deletion's position in the batch, so that the
+// last-operation-wins rule orders them against the explicit operations on the same pairs.
+__global__ void k_expand_plan(const ripple_update* __restrict__ ups, int N, long long capacity, Ctl* ctl,
+                              Side out, Side in, int2* vjobs) {
+    const int n = ctl->n_ops;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const ripple_update op = ups[i];
+        if (op.op != RIPPLE_OP_DEL_VERTEX || (unsigned)op.u >= (unsigned)N) continue;
+        const unsigned long long cnt = (unsigned long long)out.deg[op.u] + (unsigned long long)in.deg[op.u];
+        const unsigned long long base = atomicAdd(&ctl->n_extra, cnt);
+        if ((unsigned long long)n + base + cnt > (unsigned long long)capacity) {
+            atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_CAPACITY);
+            ctl->expand_failed = 1;
+            ctl->abort = 1;
+            continue;
         }
-        h = (h + 1) & hmask;
+        vjobs[atomicAdd(&ctl->n_vjobs, 1)] = make_int2(i, n + (int)base);
     }
-    atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_CAPACITY);  // table full: cannot happen with hsize >= 2 max_batch
-    ctl->abort = 1;
+}
+
+__global__ void k_expand_copy(ripple_update* ups, int32_t* op_seq, Ctl* ctl, Side out, Side in,
+                              const int2* __restrict__ vjobs) {
+    if (ctl->abort) return;
+    const int nj = ctl->n_vjobs;
+    for (int j = blockIdx.x; j < nj; j += gridDim.x) {
+        const int2 job = vjobs[j];
+        const int w = ups[job.x].u;
+        const int dout = out.deg[w], din = in.deg[w];
+        const int64_t bo = out.start[w], bi = in.start[w];
+        for (int k = threadIdx.x; k < dout + din; k += blockDim.x) {
+            ripple_update g;
+            g.op = RIPPLE_OP_DEL_EDGE;
+            if (k < dout) { g.u = w; g.v = out.col[bo + k]; }
+            else { g.u = in.col[bi + (k - dout)]; g.v = w; }
+            ups[job.y + k] = g;
+            op_seq[job.y + k] = job.x;
+        }
+    }
+}
+
+__global__ void k_classify(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, int N,
+                           Ctl* ctl, unsigned long long* hkeys, unsigned long long* hwin, int hmask,
+                           int32_t* op_slot, int32_t* feat_last, int32_t* vdel_seq) {
+    const int n = ops_total(ctl), n_given = ctl->n_ops;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        ripple_update op = ups[i];
+        op_slot[i] = -1;
+        if (op.op < 0 || op.op > 3) {
+            atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_INVALID_ARG);
+            ctl->abort = 1;
+            continue;
+        }
+        bool bad = (unsigned)op.u >= (unsigned)N;
+        if (op.op == RIPPLE_OP_SET_FEATURE) bad |= (unsigned)op.v >= (unsigned)ctl->n_rows;
+        else if (op.op != RIPPLE_OP_DEL_VERTEX) bad |= (unsigned)op.v >= (unsigned)N;
+        if (bad) {
+            atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_VERTEX_RANGE);
+            ctl->abort = 1;
+            continue;
+        }
+        if (op.op == RIPPLE_OP_SET_FEATURE) {
+            atomicMax(&feat_last[op.u], i);
+            continue;
+        }
+        if (op.op == RIPPLE_OP_DEL_VERTEX) {   // also the last word on the vertex's feature row so far
+            atomicMax(&feat_last[op.u], i);
+            atomicMax(&vdel_seq[op.u], i);
+            continue;
+        }
+        const int seq = i < n_given ? i : op_seq[i];
+        const unsigned long long mine = ((unsigned long long)(seq + 1) << 32) | (unsigned)i;
+        unsigned long long key = (unsigned long long)op.u * (unsigned long long)N + (unsigned long long)op.v + 1ull;
+        int h = (int)(mix64(key) & (unsigned long long)hmask);
+        bool placed = false;
+        for (int probe = 0; probe <= hmask; ++probe) {
+            unsigned long long prev = atomicCAS(&hkeys[h], 0ull, key);
+            if (prev == 0ull || prev == key) {
+                atomicMax(&hwin[h], mine);
+                op_slot[i] = h;
+                placed = true;
+                break;
+            }
+            h = (h + 1) & hmask;
+        }
+        if (!placed) {   // table full: cannot happen with hsize >= 2 max_batch
+            atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_CAPACITY);
+            ctl->abort = 1;
+        }
+    }
 }
 
 // Position of x in row [base, base + deg), or -1; the whole block calls this.  Rows start on
@@ -168,24 +227,29 @@ __device__ __forceinline__ int block_find(const int32_t* __restrict__ col, int64
 }
 
 // One block per op: winners are compared with the stored graph and become records or no-ops.
+// An explicit edge operation that precedes the deletion of one of its endpoints is superseded by
+// it (for stored edges the generated deletion already wins the slot; for pairs that are not stored
+// nothing was generated, hence the explicit test).  Only the caller's operations are counted.
 __global__ void __launch_bounds__(256)
-k_resolve(const ripple_update* __restrict__ ups, int n, Ctl* ctl,
-          const int32_t* __restrict__ hseq, const int32_t* __restrict__ op_slot,
-          const int32_t* __restrict__ feat_last, Side out, Side in, Rec* rec,
-          uint32_t* bitmap) {
+k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, Ctl* ctl,
+          const unsigned long long* __restrict__ hwin, const int32_t* __restrict__ op_slot,
+          const int32_t* __restrict__ feat_last, const int32_t* __restrict__ vdel_seq, Side out, Side in,
+          Rec* rec, uint32_t* bitmap) {
     __shared__ int s_found;
     if (ctl->abort) return;
+    const int n = ops_total(ctl), n_given = ctl->n_ops;
     for (int i = blockIdx.x; i < n; i += gridDim.x) {
         ripple_update op = ups[i];
-        if (op.op == RIPPLE_OP_SET_FEATURE) {
+        if (op.op == RIPPLE_OP_SET_FEATURE || op.op == RIPPLE_OP_DEL_VERTEX) {
             if (threadIdx.x == 0 && feat_last[op.u] == i) {
                 atomicAdd(&ctl->n_feat, 1);
                 atomicOr(&bitmap[op.u >> 5], 1u << (op.u & 31));
             }
             continue;
         }
-        if (hseq[op_slot[i]] != i) {
-            if (threadIdx.x == 0) atomicAdd(&ctl->n_superseded, 1);
+        const int seq = i < n_given ? i : op_seq[i];
+        if ((int)(unsigned)hwin[op_slot[i]] != i || seq < max(vdel_seq[op.u], vdel_seq[op.v])) {
+            if (threadIdx.x == 0 && i < n_given) atomicAdd(&ctl->n_superseded, 1);
             continue;
         }
         int j_out = block_find(out.col, out.start[op.u], out.deg[op.u], op.v, &s_found);
@@ -247,14 +311,21 @@ __global__ void k_plan_check(Ctl* ctl, long long col_size_out, long long col_siz
     }
 }
 
+// n sizes the launches (the number of operations given, or the batch capacity if vertex deletions
+// may multiply them); the kernels read the actual counts from the control block
 void graph_batch_classify(Ctx* c, int n) {
     if (n <= 0) return;
     const int T = 256;
-    RP_LAUNCH(c, k_classify, div_up(n, T), T, 0, c->ups_dev, n, c->N, c->ctl, c->hkeys, c->hseq,
-              c->hsize - 1, c->op_slot, c->feat_last);
+    const int grid_ops = std::min(div_up(n, T), c->n_sm * 8);
+    RP_LAUNCH(c, k_expand_plan, grid_ops, T, 0, c->ups_dev, c->N, (long long)c->max_batch, c->ctl, c->side[0],
+              c->side[1], c->vjobs);
+    RP_LAUNCH(c, k_expand_copy, std::min(n, c->n_sm * 4), T, 0, c->ups_dev, c->op_seq, c->ctl, c->side[0],
+              c->side[1], c->vjobs);
+    RP_LAUNCH(c, k_classify, grid_ops, T, 0, c->ups_dev, c->op_seq, c->N, c->ctl, c->hkeys, c->hwin,
+              c->hsize - 1, c->op_slot, c->feat_last, c->vdel_seq);
     int grid = std::min(n, c->n_sm * 8);
-    RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, n, c->ctl, c->hseq, c->op_slot, c->feat_last,
-              c->side[0], c->side[1], c->rec, c->bitmap);
+    RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, c->op_seq, c->ctl, c->hwin, c->op_slot, c->feat_last,
+              c->vdel_seq, c->side[0], c->side[1], c->rec, c->bitmap);
     RP_LAUNCH(c, k_plan_growth, std::min(div_up(2 * n, T), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[0],
               c->side[1], c->grow_list[0], c->grow_list[1]);
     RP_LAUNCH(c, k_plan_check, 1, 1, 0, c->ctl, (long long)c->side[0].col_size, (long long)c->side[1].col_size);
@@ -391,18 +462,22 @@ void graph_batch_mutate(Ctx* c, int n) {
 // ---------------------------------------------------------------------------------------------
 // per-batch scratch back to its resting state (runs for rejected batches too)
 // ---------------------------------------------------------------------------------------------
-__global__ void k_cleanup(const ripple_update* __restrict__ ups, int n, int N, Ctl* ctl,
+__global__ void k_cleanup(const ripple_update* __restrict__ ups, int N, Ctl* ctl,
                           const Rec* __restrict__ rec, Side out, Side in, unsigned long long* hkeys,
-                          int32_t* hseq, const int32_t* __restrict__ op_slot, int32_t* feat_last,
-                          int32_t* deg_out_old, uint32_t* bitmap) {
-    int n_rec = ctl->n_rec;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-        ripple_update op = ups[i];
-        int slot = op_slot[i];
-        if (slot >= 0) { hkeys[slot] = 0ull; hseq[slot] = -1; }
-        if (op.op == RIPPLE_OP_SET_FEATURE && (unsigned)op.u < (unsigned)N) {
-            feat_last[op.u] = -1;
-            if (ctl->abort) atomicAnd(&bitmap[op.u >> 5], ~(1u << (op.u & 31)));
+                          unsigned long long* hwin, const int32_t* __restrict__ op_slot, int32_t* feat_last,
+                          int32_t* vdel_seq, int32_t* deg_out_old, uint32_t* bitmap) {
+    const int n_rec = ctl->n_rec, n = ops_total(ctl);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && !ctl->abort) ctl->num_edges += ctl->n_add - ctl->n_del;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < max(n, n_rec); i += gridDim.x * blockDim.x) {
+        if (i < n) {
+            ripple_update op = ups[i];
+            int slot = op_slot[i];
+            if (slot >= 0) { hkeys[slot] = 0ull; hwin[slot] = 0ull; }
+            if ((op.op == RIPPLE_OP_SET_FEATURE || op.op == RIPPLE_OP_DEL_VERTEX) && (unsigned)op.u < (unsigned)N) {
+                feat_last[op.u] = -1;
+                if (op.op == RIPPLE_OP_DEL_VERTEX) vdel_seq[op.u] = -1;
+                if (ctl->abort) atomicAnd(&bitmap[op.u >> 5], ~(1u << (op.u & 31)));
+            }
         }
         if (i < n_rec) {
             const Rec& x = rec[i];
@@ -416,8 +491,9 @@ __global__ void k_cleanup(const ripple_update* __restrict__ ups, int n, int N, C
 void graph_batch_cleanup(Ctx* c, int n) {
     if (n <= 0) return;
     const int T = 256;
-    RP_LAUNCH(c, k_cleanup, std::min(div_up(n, T), c->n_sm * 8), T, 0, c->ups_dev, n, c->N, c->ctl, c->rec,
-              c->side[0], c->side[1], c->hkeys, c->hseq, c->op_slot, c->feat_last, c->deg_out_old, c->bitmap);
+    RP_LAUNCH(c, k_cleanup, std::min(div_up(n, T), c->n_sm * 8), T, 0, c->ups_dev, c->N, c->ctl, c->rec,
+              c->side[0], c->side[1], c->hkeys, c->hwin, c->op_slot, c->feat_last, c->vdel_seq, c->deg_out_old,
+              c->bitmap);
 }
 
 // ---------------------------------------------------------------------------------------------

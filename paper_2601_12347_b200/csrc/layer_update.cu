@@ -135,6 +135,25 @@ void neighbour_transform(Ctx* c, int l, const float* rows_in, int ld_rows, const
     launch_update(c, p, ly.tc_nbr);
 }
 
+// Layers that transform before the scatter keep P^l_u = W_n^T h^{l-1}_u for every vertex.  For the
+// senders of hop l (rows whose h^{l-1}, or whose source coefficient, changed) this recomputes the
+// row, commits it and emits the transformed delta message c_new P_new - c_old P_old as a compact
+// row.  Because the next batch subtracts exactly the value cached here, the deltas of successive
+// batches telescope: the aggregate tracks the cached rows without a rounding drift of its own.
+void sender_transform(Ctx* c, int l) {
+    const LayerDev& ly = c->layer[l];
+    UpdParams p{};
+    p.list = c->Clist[(l - 1) & 1]; p.n_dev = &c->ctl->nC[l - 1]; p.n_host = 0;
+    p.a_mode = A_SELF; p.epi_mode = EPI_COMMIT; p.alpha = 1.0f;
+    p.Hprev = c->H[l - 1]; p.ld_h = c->ld[l - 1];
+    p.K = ly.ld_in;
+    p.W = ly.kind == RIPPLE_LAYER_SAGE ? ly.W1 + (size_t)ly.ld_in * ly.ld_out : ly.W1;
+    p.ldw = c->ws[l]; p.bias = nullptr; p.n_cols = c->ws[l];
+    p.act = RIPPLE_ACT_IDENTITY; p.Hout = c->P[l]; p.ld_o = c->ws[l]; p.Dout = c->Dt;
+    p.src_norm = c->src_norm; p.deg_out = c->side[0].deg; p.deg_out_old = c->deg_out_old;
+    launch_update(c, p, ly.tc_nbr);
+}
+
 // Z^l_v = W_self^T h^{l-1}_v for the rows whose h^{l-1} changed (all rows at bootstrap).  SAGE
 // layers keep this self projection cached: it is recomputed where the layer's input changed
 // (A_{l-1}), not where its output is needed (A_l, usually far larger).  The affected-row update
@@ -215,14 +234,16 @@ __global__ void k_feature_rows(Ctl* ctl, const ripple_update* __restrict__ ups, 
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     for (int i = warp; i < n; i += nwarps) {
         const int v = A0[i];
-        const float* src = feat + (size_t)ups[feat_last[v]].v * d0;
+        const ripple_update last = ups[feat_last[v]];
+        // the last word on the row is either a payload row or the vertex's deletion (zeros)
+        const float* src = last.op == RIPPLE_OP_SET_FEATURE ? feat + (size_t)last.v * d0 : nullptr;
         float cn = 1.f, co = 1.f;
         if (src_norm) {
             cn = coef_deg(deg_out[v]);
             co = deg_out_old[v] >= 0 ? coef_deg(deg_out_old[v]) : cn;
         }
         for (int k = lane_id(); k < ld; k += 32) {
-            float x = k < d0 ? src[k] : 0.f;
+            float x = (src && k < d0) ? src[k] : 0.f;
             float o = H0[(size_t)v * ld + k];
             D[(size_t)i * ld + k] = cn * x - co * o;
             H0[(size_t)v * ld + k] = x;

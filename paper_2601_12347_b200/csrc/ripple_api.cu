@@ -47,6 +47,7 @@ __global__ void k_ctl_reset(Ctl* ctl, const int* params) {
     memset(&z, 0, sizeof(Ctl));
     z.pool_next[0] = keep0;
     z.pool_next[1] = keep1;
+    z.num_edges = ctl->num_edges;
     z.n_ops = params[0];
     z.n_rows = params[1];
     *ctl = z;
@@ -63,12 +64,12 @@ static void destroy_ctx(Ctx* c) {
         cudaFree(c->grow_list[s]); cudaFree(c->D[s]); cudaFree(c->Clist[s]);
     }
     for (int l = 0; l <= RP_MAXL; ++l) {
-        cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->Z[l]); cudaFree(c->A[l]);
+        cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->Z[l]); cudaFree(c->P[l]); cudaFree(c->A[l]);
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
         for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2, &c->layer[l].tc_self}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
     cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->posmap); cudaFree(c->deg_out_old);
-    cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hseq);
+    cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
     if (c->params_host) cudaFreeHost(c->params_host);
@@ -76,6 +77,7 @@ static void destroy_ctx(Ctx* c) {
     for (auto& g : c->graph_exec) if (g) cudaGraphExecDestroy(g);
     for (auto& e : c->ev) if (e) cudaEventDestroy(e);
     for (auto& e : c->ev_sc) if (e) cudaEventDestroy(e);
+    for (auto& e : c->ev_rg) if (e) cudaEventDestroy(e);
     if (c->own_stream && c->stream) cudaStreamDestroy(c->stream);
     delete c;
 }
@@ -180,6 +182,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         CK(dev_alloc(&c->tile_sums, (size_t)c->n_tile_sums, 0));
         for (auto& e : c->ev) CK(cudaEventCreate(&e));
         for (auto& e : c->ev_sc) CK(cudaEventCreate(&e));
+        for (auto& e : c->ev_rg) CK(cudaEventCreate(&e));
 
         // graph
         if (E > 0 && g->mem == RIPPLE_MEM_HOST) {
@@ -232,6 +235,9 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                 const int target = y.kind == RIPPLE_LAYER_GIN ? ly.ld_hid : ly.ld_out;
                 c->pre[l] = o.pre_transform == 0 && target < ly.ld_in;
                 c->ws[l] = c->pre[l] ? target : ly.ld_in;
+                // measured: a gathered row costs about half of a row delivered as a reduction
+                c->regather_threshold[l] = o.regather_threshold > 0.f ? o.regather_threshold
+                                           : o.regather_threshold < 0.f ? -1.f : 0.7f;
                 if (o.gemm_mode != RIPPLE_GEMM_FP32) {   // transposed, tf32-split copies for the tensor-core form
                     const float* wn = y.kind == RIPPLE_LAYER_SAGE ? w1.data() + (size_t)ly.ld_in * ly.ld_out : w1.data();
                     if (y.kind == RIPPLE_LAYER_SAGE)
@@ -262,7 +268,8 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             max_ld = std::max(max_ld, c->ld[l]);
             CK(dev_alloc(&c->H[l], (size_t)N * c->ld[l], 0));
             if (l > 0) { CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0)); CK(dev_alloc(&c->dS[l], (size_t)N * c->ws[l], 0));
-                         if (c->layer[l].kind == RIPPLE_LAYER_SAGE) CK(dev_alloc(&c->Z[l], (size_t)N * c->ld[l], 0)); }
+                         if (c->layer[l].kind == RIPPLE_LAYER_SAGE) CK(dev_alloc(&c->Z[l], (size_t)N * c->ld[l], 0));
+                         if (c->pre[l]) CK(dev_alloc(&c->P[l], (size_t)N * c->ws[l], 0)); }
             CK(dev_alloc(&c->A[l], (size_t)N + 32));
         }
         CK(cudaMemcpy2D(c->H[0], sizeof(float) * c->ld[0], features, sizeof(float) * c->d[0],
@@ -277,7 +284,9 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             CK(dev_alloc(&c->Clist[s], (size_t)N + 32));
             CK(dev_alloc(&c->grow_list[s], (size_t)o.max_batch));
         }
-        CK(dev_alloc(&c->coff, (size_t)N + 2, 0));
+        // degree prefix of a sender list; also the (vertex, chunk) work items of long in-lists during a
+        // gather: at most 1.5 items per 1024 stored edges
+        CK(dev_alloc(&c->coff, std::max((size_t)N + 2, (size_t)(c->side[1].col_size / 680) + 64), 0));
         CK(dev_alloc(&c->bitmap, (size_t)c->n_words + 256, 0));
         CK(dev_alloc(&c->posmap, (size_t)N, 0xFF));
         CK(dev_alloc(&c->deg_out_old, (size_t)N, 0xFF));
@@ -288,11 +297,18 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         c->hsize = 1024;
         while (c->hsize < 4 * o.max_batch) c->hsize <<= 1;
         CK(dev_alloc(&c->hkeys, (size_t)c->hsize, 0));
-        CK(dev_alloc(&c->hseq, (size_t)c->hsize, 0xFF));
+        CK(dev_alloc(&c->hwin, (size_t)c->hsize, 0));
+        CK(dev_alloc(&c->op_seq, (size_t)o.max_batch));
+        CK(dev_alloc(&c->vdel_seq, (size_t)N, 0xFF));
+        CK(dev_alloc(&c->vjobs, (size_t)o.max_batch));
         CK(dev_alloc(&c->op_slot, (size_t)o.max_batch));
         CK(dev_alloc(&c->rec, (size_t)o.max_batch));
         CK(cudaDeviceSynchronize());
 
+        {
+            const long long e0 = (long long)E;
+            CK(cudaMemcpy(&c->ctl->num_edges, &e0, sizeof(e0), cudaMemcpyHostToDevice));
+        }
         st = run_full(c);
         if (st) { memcpy(g_create_err, c->err, sizeof(g_create_err)); goto fail_keep_msg; }
         c->stats.num_layers = L;
@@ -323,9 +339,11 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
     STAMP();  // 1
     // one superstep per hop (Sec. 3.3.1): frontier, send + aggregate, compute + prepare
     for (int l = 1; l <= L; ++l) {
-        // the push scatter walks the same out-lists as the frontier and marks the sinks itself; the
-        // gather needs the list first
+        // The push scatter walks the same out-lists as the frontier and marks the sinks itself; the
+        // gathering forms need the list A_l first, so the frontier walk is a pass of its own for them
+        // (decided per hop on the device for the rebuilding form).
         const bool pull = c->scatter_mode == RIPPLE_SCATTER_PULL;
+        choose_direction(c, l);
         frontier_mark(c, l, pull);
         if (pull) frontier_compact(c, l);
         STAMP();
@@ -333,6 +351,7 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
         if (!pull) frontier_compact(c, l);
         senders_release(c, l - 1);
         fold_deltas(c, l);
+        regather_layer(c, l);
         STAMP();
         self_project(c, l, false);
         update_rows(c, l, false);
@@ -385,28 +404,33 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
     }
     cudaSetDevice(c->device);
     const int nb = (int)n, nr = (int)n_rows, L = c->L;
-    ripple_update* own_ups = c->ups_dev;
     float* own_feat = c->feat_dev;
     c->launches = 0;
     int evi = 0;
-    const bool try_graph = !c->no_graphs && !c->timing && nb >= 1 && nb <= RP_GRAPH_MAX_BATCH;
+    // A vertex deletion becomes one edge deletion per incident edge on the device.  Launches are
+    // sized from the number of operations, so a host batch that holds one is given the geometry
+    // of a full batch (device batches are not inspected and keep the geometry of n: still
+    // correct, since every kernel strides over the counts it reads from the control block).
+    bool wide = false;
+    if (mem == RIPPLE_MEM_HOST)
+        for (int i = 0; i < nb && !wide; ++i) wide = ups[i].op == RIPPLE_OP_DEL_VERTEX;
+    const int ng = wide ? (int)c->max_batch : nb;
+    const bool try_graph = !wide && !c->no_graphs && !c->timing && nb >= 1 && nb <= RP_GRAPH_MAX_BATCH;
     const cudaMemcpyKind kind = mem == RIPPLE_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+    // operations are always staged: generated edge deletions are appended behind them
+    if (nb) CK(cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, kind, c->stream));
     if (mem == RIPPLE_MEM_HOST || try_graph) {
-        // a replayed graph reads the library's own staging buffers, so device inputs are copied too
-        if (nb) CK(cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, kind, c->stream));
+        // a replayed graph reads the library's own staging buffers, so device payload rows are copied too
         if (nr) CK(cudaMemcpyAsync(c->feat_dev, feat_rows, sizeof(float) * (size_t)nr * c->d[0], kind, c->stream));
     } else {
-        // device inputs are used in place
-        c->ups_dev = const_cast<ripple_update*>(ups);
-        c->feat_dev = const_cast<float*>(feat_rows);
+        c->feat_dev = const_cast<float*>(feat_rows);   // device payload rows are read in place
     }
     c->params_host[0] = nb; c->params_host[1] = nr;
     CK(cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream));
     if (!try_graph || !launch_batch_graph(c, nb)) {
         c->launches = 0;
-        evi = enqueue_batch(c, nb, c->timing != 0);
+        evi = enqueue_batch(c, ng, c->timing != 0);
     }
-    c->ups_dev = own_ups;
     c->feat_dev = own_feat;
     st = sync_and_fetch_ctl(c);
     if (st) return st;
@@ -418,20 +442,22 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
         if (h.err) {
             st = (ripple_status)h.err;
             set_err(c, st == RIPPLE_ERR_VERTEX_RANGE ? "batch rejected: vertex id or payload row out of range"
-                       : st == RIPPLE_ERR_CAPACITY   ? "batch rejected: overflow edge pool exhausted"
+                       : st == RIPPLE_ERR_CAPACITY   ? (h.expand_failed ? "batch rejected: vertex deletions expand to more than max_batch operations"
+                                                                         : "batch rejected: overflow edge pool exhausted")
                                                      : "batch rejected: unknown op code");
-            s.n_added = s.n_deleted = s.n_noop_add = s.n_noop_del = s.n_superseded = s.n_feature = 0;
+            s.n_added = s.n_deleted = s.n_noop_add = s.n_noop_del = s.n_superseded = s.n_feature = s.n_expanded = 0;
             for (int l = 0; l <= L; ++l) s.affected[l] = s.senders[l] = s.active_edges[l] = 0;
             return st;
         }
         s.n_added = h.n_add; s.n_deleted = h.n_del; s.n_noop_add = h.n_noop_add; s.n_noop_del = h.n_noop_del;
         s.n_superseded = h.n_superseded; s.n_feature = h.n_feat;
+        s.n_expanded = (int64_t)h.n_extra;
         s.num_edges += h.n_add - h.n_del;
         for (int l = 0; l <= L; ++l) {
             s.affected[l] = h.nA[l];
             s.senders[l] = h.nC[l];
             s.active_edges[l] = l ? (int64_t)h.E[l] + h.n_rec : 0;
-            s.scatter_pull[l] = h.pull[l];
+            s.scatter_pull[l] = h.regather[l] ? 2 : h.pull[l];
             s.in_edges[l] = (int64_t)h.pull_work[l];
             s.message_width[l] = l ? c->ws[l] : 0;
         }
@@ -446,12 +472,13 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
                 cudaEventElapsedTime(&s.ms_scatter[l], c->ev[b + 1], c->ev[b + 2]);
                 cudaEventElapsedTime(&s.ms_update[l], c->ev[b + 2], c->ev[b + 3]);
                 cudaEventElapsedTime(&s.ms_scatter_kernel[l], c->ev_sc[2 * l], c->ev_sc[2 * l + 1]);
+                s.ms_regather[l] = 0.f;
+                if (h.regather[l]) cudaEventElapsedTime(&s.ms_regather[l], c->ev_rg[2 * l], c->ev_rg[2 * l + 1]);
             }
         }
     }
     return RIPPLE_OK;
 fail:
-    c->ups_dev = own_ups;
     c->feat_dev = own_feat;
     return st;
 }

@@ -22,7 +22,10 @@ namespace rp {
 struct Ctl {
     int abort;   // set by validation / planning: the batch is rejected, mutate nothing
     int err;     // ripple_status recorded on the device
-    int n_ops;
+    int n_ops;   // operations given by the caller
+    unsigned long long n_extra;  // edge deletions generated from vertex deletions (they follow the given ops)
+    int expand_failed;           // the generated operations did not fit: none of them is used
+    int n_vjobs;
     int n_rows;  // payload rows of the batch
     int n_rec;   // net edge changes of the batch (|dE+| + |dE-|)
     int n_add, n_del, n_noop_add, n_noop_del, n_superseded, n_feat;
@@ -34,6 +37,9 @@ struct Ctl {
     unsigned long long E[RP_MAXL + 1];          // out-edges of C_{l-1} (+ edge records): message count of hop l
     unsigned long long pull_work[RP_MAXL + 1];  // in-edges of A_l
     int pull[RP_MAXL + 1];
+    int regather[RP_MAXL + 1];        // hop l rebuilds the aggregates of A_l from their in-lists instead of adding deltas
+    int n_long[RP_MAXL + 1];          // bottom-up marking: vertices whose long in-list is scanned by a warp
+    long long num_edges;              // current edge count (kept across batches)
     int work_counter[8];              // dynamic work distribution tickets (reset by the consumer)
 };
 
@@ -96,6 +102,7 @@ struct Ctx {
     int64_t E0;
     int64_t max_batch;
     int scatter_mode, gemm_mode, timing;
+    float regather_threshold[RP_MAXL + 1];  // per hop: share of all edges from which the hop rebuilds its aggregates
     int n_sm;
     LayerDev layer[RP_MAXL + 1];
     int d[RP_MAXL + 1], ld[RP_MAXL + 1];
@@ -103,6 +110,7 @@ struct Ctx {
     float* H[RP_MAXL + 1];
     float* S[RP_MAXL + 1];
     float* Z[RP_MAXL + 1];    // cached self projection W_self^T h^{l-1} of SAGE layers (N x ld_l), else null
+    float* P[RP_MAXL + 1];    // cached neighbour projection W_n^T h^{l-1} of layers that transform before the scatter (N x ws_l), else null
     float* dS[RP_MAXL + 1];   // per-batch message accumulator, zero outside a batch (same shape as S)
     float* T;          // GIN hidden rows (compact, N x ld_hid)
     float* D[2];       // delta rows, ping-pong (compact, N x max ld)
@@ -123,7 +131,10 @@ struct Ctx {
     ripple_update* ups_dev;
     float* feat_dev;
     unsigned long long* hkeys; // pair hash table
-    int32_t* hseq;
+    unsigned long long* hwin;  // per hash slot: (position in the batch + 1) << 32 | op index of the winning op
+    int32_t* op_seq;           // generated ops: position in the batch of the vertex deletion they come from
+    int32_t* vdel_seq;         // vertex -> position of its last deletion in the batch, or -1
+    int2* vjobs;               // (op index, first generated slot) per vertex deletion
     int32_t* op_slot;
     int hsize;
     Rec* rec;
@@ -143,6 +154,7 @@ struct Ctx {
     ripple_stats stats;
     cudaEvent_t ev[4 + 3 * (RP_MAXL + 1) + 2];
     cudaEvent_t ev_sc[2 * (RP_MAXL + 1)];  // tight brackets around each hop's main scatter kernel
+    cudaEvent_t ev_rg[2 * (RP_MAXL + 1)];  // ... and around the gather of a rebuilding hop
     int64_t launches;
     char err[512];
 };
@@ -176,12 +188,15 @@ void senders_release(Ctx* c, int l);                    // clear posmap entries 
 
 // scatter.cu
 void spmm_full(Ctx* c, int l);                          // S^l for every vertex (bootstrap)
+void choose_direction(Ctx* c, int l);                   // delta or rebuilding form of hop l (device-side decision)
 void scatter_layer(Ctx* c, int l, int n);               // delta messages of hop l into dS^l
+void regather_layer(Ctx* c, int l);                     // rebuilding form: S^l rows of A_l gathered anew
 void fold_deltas(Ctx* c, int l);                        // S^l += dS^l, dS^l = 0 on the rows of A_l
 
 // layer_update.cu
 void update_rows(Ctx* c, int l, bool full);             // re-apply Update^l + activation, emit deltas
 void self_project(Ctx* c, int l, bool full);            // refresh the cached self projection of a narrow SAGE layer
+void sender_transform(Ctx* c, int l);                   // P^l rows of the senders of hop l, and their transformed deltas
 void neighbour_transform(Ctx* c, int l, const float* rows_in, int ld_rows, const int* n_dev, int n_host,
                          float* rows_out);              // compact rows times the layer's neighbour matrix
 void feature_rows(Ctx* c, int n);                       // hop 0: overwrite feature rows, emit deltas

@@ -167,8 +167,8 @@ void spmm_full(Ctx* c, int l) {
     const int ld = c->ws[l];
     const float* M = c->H[l - 1];
     if (c->pre[l]) {
-        neighbour_transform(c, l, c->H[l - 1], c->ld[l - 1], nullptr, c->N, c->D[0]);
-        M = c->D[0];
+        neighbour_transform(c, l, c->H[l - 1], c->ld[l - 1], nullptr, c->N, c->P[l]);
+        M = c->P[l];
     }
     const int grid = c->n_sm * 16, T = 256;
     // work items of the long rows live in the degree-prefix buffer, which is idle during a full pass
@@ -194,7 +194,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_scatter_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64_t* __restrict__ coff,
                Side out, const float* __restrict__ D, int ld, float* S, uint32_t* bitmap) {
-    if (ctl->abort || ctl->pull[l]) return;
+    if (ctl->abort || ctl->pull[l] || ctl->regather[l]) return;
     const int nC = ctl->nC[l - 1];
     if (nC == 0) return;
     const int64_t E = coff[nC];
@@ -257,7 +257,7 @@ k_scatter_push_packed(Ctl* ctl, int l, const int32_t* __restrict__ senders, cons
                       Side out, const float* __restrict__ D, float* S, uint32_t* bitmap) {
     constexpr int LCM = NQ == 12 ? 96 : NQ == 10 ? 160 : NQ * 32;
     constexpr int NI = LCM / 32, G = LCM / NQ, LD = NQ * 4;
-    if (ctl->abort || ctl->pull[l]) return;
+    if (ctl->abort || ctl->pull[l] || ctl->regather[l]) return;
     const int nC = ctl->nC[l - 1];
     if (nC == 0) return;
     const int64_t E = coff[nC];
@@ -309,7 +309,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_scatter_pull(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_t* __restrict__ posmap,
                const float* __restrict__ D, int ld, float* S) {
-    if (ctl->abort || !ctl->pull[l]) return;
+    if (ctl->abort || !ctl->pull[l] || ctl->regather[l]) return;
     const int nA = ctl->nA[l];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
@@ -357,10 +357,10 @@ k_scatter_pull(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const in
 // ---------------------------------------------------------------------------------------------
 // M_u = c_old h_old = c_new h_new - D_u for a sender, c h otherwise; one warp per record, compact
 // rows in record order (row width = that of the previous layer's embeddings).
-__global__ void k_record_rows(Ctl* ctl, const Rec* __restrict__ rec, int src_norm,
+__global__ void k_record_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, int src_norm,
                               const int32_t* __restrict__ deg_out, const int32_t* __restrict__ posmap,
                               const float* __restrict__ Hprev, const float* __restrict__ D, int ld, float* M) {
-    if (ctl->abort) return;
+    if (ctl->abort || ctl->regather[l]) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
@@ -383,9 +383,9 @@ __global__ void k_record_rows(Ctl* ctl, const Rec* __restrict__ rec, int src_nor
 }
 
 // S_v += sign * M_r for every record r (row width = inbox width)
-__global__ void k_scatter_records(Ctl* ctl, const Rec* __restrict__ rec, const float* __restrict__ M,
+__global__ void k_scatter_records(Ctl* ctl, int l, const Rec* __restrict__ rec, const float* __restrict__ M,
                                   int ld, float* S) {
-    if (ctl->abort) return;
+    if (ctl->abort || ctl->regather[l]) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
@@ -400,14 +400,101 @@ __global__ void k_scatter_records(Ctl* ctl, const Rec* __restrict__ rec, const f
     }
 }
 
-// Direction of hop l, decided on the device.  Measured on the dense R-MAT graph (123.7 M edges):
-// pushing 22 M messages of 256 floats takes 5.4 ms where gathering them over the in-lists of the
-// 1.15 M affected sinks takes 6.0 ms, and on a saturated hop (122 M messages of 48 floats over
-// 123.7 M in-edges) pushing is several times faster than the gather, whose per-edge position
-// lookup and dependent row loads leave it latency-bound.  So the automatic choice is to push;
-// the gather stays selectable for comparison.
-__global__ void k_choose_direction(Ctl* ctl, int l, int mode) {
+// ---------------------------------------------------------------------------------------------
+// rebuilding hop (scoped recomputation of the aggregates, the "RC" strategy of Sec. 3.2 applied to
+// one hop): S_v of every affected vertex is gathered again over In_new(v) from the current rows
+// ---------------------------------------------------------------------------------------------
+template <int NV, int LPR>
+__global__ void __launch_bounds__(256)
+k_regather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_t* __restrict__ deg_out,
+           int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, int2* items, int* n_items) {
+    if (ctl->abort || !ctl->regather[l]) return;
+    const int nA = ctl->nA[l];
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id(), nq = ld >> 2;
+    const int sub = lane / LPR, ql = lane % LPR;
+    for (int i = warp; i < nA; i += nwarps) {
+        const int v = A[i];
+        const int deg = in.deg[v];
+        float4 acc[NV];
+#pragma unroll
+        for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (deg > SPMM_HUB_DEGREE) {   // zero the row here, chunks are added by k_spmm_hubs
+            const int nch = (deg + SPMM_HUB_CHUNK - 1) / SPMM_HUB_CHUNK;
+            int first = 0;
+            if (lane == 0) first = atomicAdd(n_items, nch);
+            first = __shfl_sync(FULL, first, 0);
+            for (int ch = lane; ch < nch; ch += 32) items[first + ch] = make_int2(v, ch);
+        } else {
+            spmm_accumulate<NV, LPR>(acc, in, v, 0, deg, deg_out, src_norm, M, ld);
+        }
+        if (sub == 0) {
+            float4* dst = reinterpret_cast<float4*>(S + (size_t)v * ld);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                int q = ql + LPR * k;
+                if (q < nq) dst[q] = acc[k];
+            }
+        }
+    }
+}
+
+// A sink that lost at least as many in-edges as it keeps is rebuilt from its in-list, whatever
+// form the hop takes: subtracting most of a sum leaves the rounding of the large old value on the
+// small new one (a hub emptied by a vertex deletion kept 2e-3 where exact zeros belong), while
+// gathering the survivors costs no more than the deletions did.  One warp per such row; its
+// pending message sums are dropped with it.
+template <int NV, int LPR>
+__global__ void __launch_bounds__(256)
+k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int32_t* __restrict__ deg_out,
+                int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, float* __restrict__ dS) {
+    if (ctl->abort || ctl->regather[l]) return;
+    const int n = ctl->n_rec;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id(), nq = ld >> 2;
+    const int sub = lane / LPR, ql = lane % LPR;
+    for (int r = warp; r < n; r += nwarps) {
+        if (!rec[r].rep[1]) continue;          // one record per distinct sink
+        const int v = rec[r].v;
+        const int deg = in.deg[v], lost = in.cnt_del[v];
+        if (lost == 0 || lost < deg) continue;
+        float4 acc[NV];
+#pragma unroll
+        for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        spmm_accumulate<NV, LPR>(acc, in, v, 0, deg, deg_out, src_norm, M, ld);
+        if (sub == 0) {
+            float4* dst = reinterpret_cast<float4*>(S + (size_t)v * ld);
+            float4* pend = reinterpret_cast<float4*>(dS + (size_t)v * ld);
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                int q = ql + LPR * k;
+                if (q < nq) { dst[q] = acc[k]; pend[q] = make_float4(0.f, 0.f, 0.f, 0.f); }
+            }
+        }
+    }
+}
+
+// Form of hop l, decided on the device once the senders and their out-degree sum are known.
+//
+// Delta form: the out-edges of the senders each carry one message, added to the sink's aggregate
+// by a vector reduction (push), or gathered per sink over the senders among its in-neighbours
+// (pull; measured slower at every size because of the per-edge membership lookup, kept
+// selectable for comparison).
+//
+// Rebuilding form: once the senders' out-edges are most of the graph, reading every in-edge of
+// the affected sinks once and overwriting their aggregates costs less than one reduction per
+// message: a gathered row is a plain load, a delivered message a read-modify-write in L2.  The
+// rebuilt aggregate also sheds whatever rounding the deltas had left in it.  threshold = the
+// share of all edges above which the hop rebuilds (<= 0: never).
+__global__ void k_choose_direction(Ctl* ctl, int l, int mode, float threshold) {
+    const int nC = ctl->nC[l - 1];
+    int re = 0;
+    if (mode == RIPPLE_SCATTER_REGATHER) re = 1;
+    else if (mode == RIPPLE_SCATTER_AUTO && threshold > 0.f)
+        re = (double)(ctl->E[l] + (unsigned long long)ctl->n_rec) >= (double)threshold * (double)ctl->num_edges && ctl->num_edges > 0;
+    if (nC == 0 && ctl->n_rec == 0) re = 0;
     ctl->pull[l] = mode == RIPPLE_SCATTER_PULL;
+    ctl->regather[l] = re;
 }
 
 // Messages of one batch are first summed among themselves in dS (zero outside a batch) and reach
@@ -416,7 +503,7 @@ __global__ void k_choose_direction(Ctl* ctl, int l, int mode) {
 // the aggregate's magnitude, and the error random-walks with the number of messages (measured
 // drift 1e-4 of the value after 100 batches).  Folding keeps it at one rounding per row and batch.
 __global__ void k_fold_deltas(Ctl* ctl, int l, const int32_t* __restrict__ A, int ld, float* S, float* dS) {
-    if (ctl->abort) return;
+    if (ctl->abort || ctl->regather[l]) return;   // a rebuilt aggregate has no pending sums
     const int n = ctl->nA[l];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
@@ -438,6 +525,11 @@ void fold_deltas(Ctx* c, int l) {
     RP_LAUNCH(c, k_fold_deltas, c->n_sm * 8, 256, 0, c->ctl, l, c->A[l], c->ws[l], c->S[l], c->dS[l]);
 }
 
+void choose_direction(Ctx* c, int l) {
+    RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode, c->regather_threshold[l]);
+}
+
+// delta form of hop l (does nothing on the device if the hop rebuilds)
 void scatter_layer(Ctx* c, int l, int n) {
     const int ld_prev = c->ld[l - 1];
     const int ld = c->ws[l];
@@ -445,25 +537,26 @@ void scatter_layer(Ctx* c, int l, int n) {
     const int32_t* senders = c->Clist[(l - 1) & 1];
     const int T = 256;
     const int grid = c->n_sm * 8;
-    RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode);
-    // records need the untransformed delta rows and the position map of C_{l-1}
-    if (n > 0)
-        RP_LAUNCH(c, k_record_rows, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, c->rec,
-                  (int)c->src_norm, c->side[0].deg, c->posmap, c->H[l - 1], D, ld_prev, c->M);
+    // Edge records: M_r = c_old m_old of the record's source = c_new m_new - D_u for a sender.  A
+    // layer that transforms first keeps m = P^l rows up to date for the senders, whatever form the
+    // hop takes, and builds its records from them directly.
     const float* Dm = D;
     const float* Mm = c->M;
     if (c->pre[l]) {
-        neighbour_transform(c, l, D, ld_prev, &c->ctl->nC[l - 1], 0, c->Dt);
+        sender_transform(c, l);
         Dm = c->Dt;
-        if (n > 0) {
-            neighbour_transform(c, l, c->M, ld_prev, &c->ctl->n_rec, 0, c->Mt);
-            Mm = c->Mt;
-        }
+        Mm = c->Mt;
+        if (n > 0)
+            RP_LAUNCH(c, k_record_rows, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec,
+                      (int)c->src_norm, c->side[0].deg, c->posmap, c->P[l], c->Dt, ld, c->Mt);
+    } else if (n > 0) {
+        RP_LAUNCH(c, k_record_rows, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec,
+                  (int)c->src_norm, c->side[0].deg, c->posmap, c->H[l - 1], D, ld_prev, c->M);
     }
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
 #define PUSH(NV, LPR) RP_LAUNCH(c, (k_scatter_push<NV, LPR>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, ld, c->dS[l], c->bitmap)
 #define PULL(NV, LPR) RP_LAUNCH(c, (k_scatter_pull<NV, 32>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->posmap, Dm, ld, c->dS[l])
-    if (c->scatter_mode != RIPPLE_SCATTER_PULL) {
+    if (c->scatter_mode == RIPPLE_SCATTER_AUTO || c->scatter_mode == RIPPLE_SCATTER_PUSH) {
         if (ld == 48) RP_LAUNCH(c, k_scatter_push_packed<12>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
         else if (ld == 40) RP_LAUNCH(c, k_scatter_push_packed<10>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
         else RP_WIDTH_DISPATCH(ld, PUSH);
@@ -472,9 +565,36 @@ void scatter_layer(Ctx* c, int l, int n) {
 #undef PUSH
 #undef PULL
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
-    if (n > 0)
-        RP_LAUNCH(c, k_scatter_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, c->rec, Mm, ld,
+    if (n > 0) {
+        RP_LAUNCH(c, k_scatter_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, Mm, ld,
                   c->dS[l]);
+        const float* rows = c->pre[l] ? c->P[l] : c->H[l - 1];
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l])
+        RP_WIDTH_DISPATCH(ld, ROWS);
+#undef ROWS
+    }
+}
+
+// rebuilding form of hop l (does nothing on the device unless the hop rebuilds); needs the list A_l
+void regather_layer(Ctx* c, int l) {
+    if (c->scatter_mode != RIPPLE_SCATTER_AUTO && c->scatter_mode != RIPPLE_SCATTER_REGATHER) return;
+    if (c->scatter_mode == RIPPLE_SCATTER_AUTO && c->regather_threshold[l] <= 0.f) return;
+    const int ld = c->ws[l];
+    const float* M = c->pre[l] ? c->P[l] : c->H[l - 1];   // P^l rows of the senders are already current
+    const int grid = c->n_sm * 16, T = 256;
+    int2* items = reinterpret_cast<int2*>(c->coff);   // the degree prefix of the senders is no longer needed
+    int* n_items = &c->ctl->work_counter[(l - 1) & 7];
+    if (c->timing) cudaEventRecord(c->ev_rg[2 * l], c->stream);
+#define REGATHER(NV, LPR)                                                                                          \
+    do {                                                                                                           \
+        RP_LAUNCH(c, (k_regather<NV, LPR>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->side[0].deg,           \
+                  (int)c->src_norm, M, ld, c->S[l], items, n_items);                                               \
+        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), grid, T, 0, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
+                  c->S[l], items, n_items);                                                                        \
+    } while (0)
+    RP_WIDTH_DISPATCH(ld, REGATHER);
+#undef REGATHER
+    if (c->timing) cudaEventRecord(c->ev_rg[2 * l + 1], c->stream);
 }
 
 }  // namespace rp

@@ -20,6 +20,7 @@ import numpy as np
 OP_ADD_EDGE = 0
 OP_DEL_EDGE = 1
 OP_SET_FEATURE = 2
+OP_DEL_VERTEX = 3
 
 # one update record: for edge ops (u, v) = (source, sink); for a feature update u is the vertex
 # and v the index of its row in the batch's feature payload

@@ -21,8 +21,8 @@ MEM_HOST, MEM_DEVICE = 0, 1
 AGG_SUM, AGG_MEAN, AGG_WSUM_GCN = 0, 1, 2
 LAYER_SAGE, LAYER_GRAPHCONV, LAYER_GIN = 0, 1, 2
 ACT_IDENTITY, ACT_RELU = 0, 1
-OP_ADD_EDGE, OP_DEL_EDGE, OP_SET_FEATURE = 0, 1, 2
-SCATTER_AUTO, SCATTER_PUSH, SCATTER_PULL = 0, 1, 2
+OP_ADD_EDGE, OP_DEL_EDGE, OP_SET_FEATURE, OP_DEL_VERTEX = 0, 1, 2, 3
+SCATTER_AUTO, SCATTER_PUSH, SCATTER_PULL, SCATTER_REGATHER = 0, 1, 2, 3
 GEMM_AUTO, GEMM_FP32, GEMM_TF32 = 0, 1, 2
 
 UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
@@ -57,7 +57,8 @@ class _Options(ctypes.Structure):
     _fields_ = [("slack", ctypes.c_double), ("pool_edges", ctypes.c_int64),
                 ("max_batch", ctypes.c_int64), ("scatter_mode", ctypes.c_int32),
                 ("gemm_mode", ctypes.c_int32), ("timing", ctypes.c_int32),
-                ("pre_transform", ctypes.c_int32), ("no_graphs", ctypes.c_int32), ("device", ctypes.c_int32), ("stream", ctypes.c_void_p)]
+                ("pre_transform", ctypes.c_int32), ("no_graphs", ctypes.c_int32), ("device", ctypes.c_int32), ("stream", ctypes.c_void_p),
+                ("regather_threshold", ctypes.c_float)]
 
 
 class _Stats(ctypes.Structure):
@@ -73,7 +74,7 @@ class _Stats(ctypes.Structure):
                 ("pool_used", ctypes.c_int64), ("pool_size", ctypes.c_int64),
                 ("ms_total", ctypes.c_float), ("ms_graph", ctypes.c_float),
                 ("ms_frontier", _F), ("ms_scatter", _F), ("ms_update", _F),
-                ("ms_scatter_kernel", _F), ("ms_bootstrap", ctypes.c_float), ("gpu_launches", ctypes.c_int64)]
+                ("ms_scatter_kernel", _F), ("ms_regather", _F), ("ms_bootstrap", ctypes.c_float), ("gpu_launches", ctypes.c_int64), ("n_expanded", ctypes.c_int64)]
 
 
 _lib = None
@@ -139,7 +140,8 @@ class Ripple:
     def __init__(self, n: int, src, dst, features, model, weights: Sequence[Dict[str, np.ndarray]],
                  slack: float = 0.0, pool_edges: int = 0, max_batch: int = 0,
                  scatter_mode: int = SCATTER_AUTO, gemm_mode: int = GEMM_AUTO, timing: bool = False,
-                 pre_transform: bool = True, graphs: bool = True, stream=None):
+                 pre_transform: bool = True, graphs: bool = True, stream=None,
+                 regather_threshold: float = 0.0):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -183,6 +185,7 @@ class Ripple:
         opt.scatter_mode, opt.gemm_mode, opt.timing = int(scatter_mode), int(gemm_mode), int(bool(timing))
         opt.pre_transform = 0 if pre_transform else 1
         opt.no_graphs = 0 if graphs else 1
+        opt.regather_threshold = float(regather_threshold)
         opt.device = torch.cuda.current_device()
         self._stream = stream if stream is not None else torch.cuda.Stream()
         opt.stream = self._stream.cuda_stream
@@ -311,9 +314,9 @@ class Ripple:
         out = {k: getattr(s, k) for k in ("num_layers", "num_edges", "n_ops", "n_added", "n_deleted",
                                           "n_noop_add", "n_noop_del", "n_superseded", "n_feature",
                                           "pool_used", "pool_size", "ms_total", "ms_graph",
-                                          "ms_bootstrap", "gpu_launches")}
+                                          "ms_bootstrap", "gpu_launches", "n_expanded")}
         for k in ("affected", "senders", "active_edges", "scatter_pull", "in_edges", "message_width", "ms_frontier", "ms_scatter",
-                  "ms_update", "ms_scatter_kernel"):
+                  "ms_update", "ms_scatter_kernel", "ms_regather"):
             out[k] = list(getattr(s, k))[: L + 1]
         return out
 

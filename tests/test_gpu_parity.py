@@ -153,7 +153,7 @@ def test_tiny_config_every_batch_against_full_recompute(env):
 
 
 @pytest.mark.parametrize("name", list(small_models().keys()))
-@pytest.mark.parametrize("mode", ["auto", "push", "pull", "push-notransform"])
+@pytest.mark.parametrize("mode", ["auto", "push", "pull", "push-notransform", "regather", "auto-mixed"])
 def test_every_model_kind_and_scatter_direction(env, name, mode):
     ripple, Oracle = env
     model = small_models()[name]
@@ -169,22 +169,32 @@ def test_every_model_kind_and_scatter_direction(env, name, mode):
     X = I.features(n, model.dims[0], 3)
     W = I.make_weights(model, 3, zero_bias=False)
     sm = {"auto": ripple.SCATTER_AUTO, "push": ripple.SCATTER_PUSH, "pull": ripple.SCATTER_PULL,
-          "push-notransform": ripple.SCATTER_PUSH}[mode]
-    rp = ripple.Ripple(n, src, dst, X, model, W, scatter_mode=sm, pre_transform=mode != "push-notransform")
+          "push-notransform": ripple.SCATTER_PUSH, "regather": ripple.SCATTER_REGATHER,
+          "auto-mixed": ripple.SCATTER_AUTO}[mode]
+    # auto-mixed: a hop rebuilds its aggregates once its messages reach 5 % of the edges, so that
+    # pushing and rebuilding hops alternate within a batch and from batch to batch
+    rp = ripple.Ripple(n, src, dst, X, model, W, scatter_mode=sm, pre_transform=mode != "push-notransform",
+                       regather_threshold=0.05 if mode == "auto-mixed" else 0.0)
     narrowing = any((ly.d_hidden or ly.d_out) + 3 < ly.d_in for ly in model.layers)
     assert any(rp.aggregate(l)[1] for l in range(1, L + 1)) == (narrowing and mode != "push-notransform")
     orc = Oracle(n, src, dst, X, model, W)
     stream = I.UpdateStream(n, src, dst, model.dims[0], 3)
     sizes = [1, 1, 2, 7, 33, 100, 1, 250, 64, 5] * 3
+    forms = set()
     for b, bs in enumerate(sizes):
         ups, rows = stream.next_batch(bs)
         rp.apply_batch(ups, rows)
         assert orc.apply_incremental(ups, rows) == 0
         check_graph(rp, orc)
         check_frontiers(rp, orc, L)
+        forms.update(rp.stats()["scatter_pull"][1:L + 1])
         if b % 5 == 4 or b == len(sizes) - 1:
             check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
     st = rp.stats()
+    if mode == "regather":
+        assert forms == {2}
+    if mode == "auto-mixed":
+        assert forms == {0, 2}
     if mode == "pull":
         assert all(st["scatter_pull"][l] == 1 for l in range(1, L + 1))
     if mode.startswith("push"):
@@ -559,6 +569,42 @@ def test_hub_stress_streams(env, mix):
     st = rp.stats()
     assert st["affected"][3] > 0.3 * w.n          # saturated: a third of all vertices and more
     check_values(rp, orc.full(), 3, [None] + [orc.full_S(l) for l in range(1, 4)])
+    rp.close()
+
+
+def test_rebuilding_hops_with_long_in_lists(env):
+    """Default settings on a graph where two sinks have in-lists long enough to be gathered in
+    chunks by separate warps; wide layers, so that saturated hops rebuild their aggregates."""
+    ripple, Oracle = env
+    model = I.sage_model([20, 128, 128, 128, 12], I.AGG_MEAN)
+    L = 4
+    n = 6000
+    src, dst = I.er_graph(n, 30000, 11)
+    have = set(zip(src.tolist(), dst.tolist()))
+    extra = [(u, 7) for u in range(100, 5100) if (u, 7) not in have]
+    extra += [(u, 9) for u in range(0, 2300) if (u, 9) not in have and u != 9]
+    extra += [(7, v) for v in range(200, 3200) if (7, v) not in have]      # and a hub that reaches half the graph
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    X = I.features(n, 20, 11)
+    W = I.make_weights(model, 11, zero_bias=False)
+    rp = ripple.Ripple(n, src, dst, X, model, W)
+    orc = Oracle(n, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, 20, 11)
+    forms = set()
+    for b, bs in enumerate([1, 20, 300, 5, 1000, 50, 2, 400]):
+        ups, rows = stream.next_batch(bs)
+        if b == 3:   # touch the hub directly: its 3000 out-edges carry a message, then everything does
+            if rows.shape[0] == 0:
+                rows = I.features(1, 20, 99)
+            ups = np.concatenate([ups, ups_array([(I.OP_SET_FEATURE, 7, 0)])])
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, L)
+        forms.update(rp.stats()["scatter_pull"][1:L + 1])
+        check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+    assert forms == {0, 2}, forms
     rp.close()
 
 

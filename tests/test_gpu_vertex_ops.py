@@ -1,0 +1,145 @@
+"""Vertex deletion and re-creation on the GPU against the oracle (Sec. 3.2: a vertex deletion
+deletes every incident edge and propagates from the vertex as root; Sec. 4.1: a vertex addition
+arrives as the edge addition that names the new endpoint)."""
+import os
+import sys
+
+import numpy as np
+import pytest
+
+sys.path.insert(0, os.path.dirname(__file__))
+import test_gpu_parity as G  # noqa: E402  (env fixture, graph / frontier / value checks)
+from test_gpu_parity import env  # noqa: E402,F401
+from test_oracle_vertex_ops import random_batch  # noqa: E402
+
+from paper_2601_12347_b200 import inputs as I  # noqa: E402
+
+pytestmark = pytest.mark.gpu
+
+
+def edge_set(src, dst):
+    return set(zip(src.tolist(), dst.tolist()))
+
+
+@pytest.mark.parametrize("name", list(G.small_models().keys()))
+def test_colliding_batches_with_vertex_deletions(env, name):
+    """Edge operations before and after the deletion of their endpoints, repeated deletions,
+    feature rows overridden by a deletion and the other way round."""
+    ripple, Oracle = env
+    model = G.small_models()[name]
+    L = len(model.layers)
+    n, m = 300, 2500
+    src, dst = I.er_graph(n, m, 5)
+    X = I.features(n, model.dims[0], 5)
+    W = I.make_weights(model, 5, zero_bias=False)
+    rp = ripple.Ripple(n, src, dst, X, model, W)
+    orc = Oracle(n, src, dst, X, model, W)
+    rng = np.random.default_rng(5)
+    edges = edge_set(src, dst)
+    seen_expanded = 0
+    for b in range(24):
+        rows = I.features(6, model.dims[0], 700 + b)
+        recs = random_batch(rng, n, edges, int(rng.integers(1, 60)), 6, p_vertex=0.1)
+        ups = G.ups_array(recs)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        G.check_graph(rp, orc)
+        G.check_frontiers(rp, orc, L)
+        seen_expanded += rp.stats()["n_expanded"]
+        rowptr, col = orc.export_csr()
+        edges = {(u, int(col[j])) for u in range(n) for j in range(rowptr[u], rowptr[u + 1])}
+        if b % 4 == 3:
+            G.check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+    assert seen_expanded > 0
+    rp.close()
+
+
+@pytest.mark.parametrize("mem", ["host", "device"])
+def test_hub_deletion_and_recreation(env, mem):
+    """A vertex with thousands of in- and out-edges is deleted (host batch: full-batch launch
+    geometry; device batch: geometry of the few given operations, replayed as a captured graph),
+    then re-created under the same id."""
+    import torch
+    ripple, Oracle = env
+    model = I.sage_model([12, 64, 24, 8], I.AGG_MEAN)
+    L = 3
+    n = 5000
+    src, dst = I.er_graph(n, 20000, 9)
+    have = edge_set(src, dst)
+    hub = 17
+    extra = [(hub, v) for v in range(100, 2600) if (hub, v) not in have]
+    extra += [(u, hub) for u in range(1000, 4200) if (u, hub) not in have and u != hub]
+    extra += [(hub, hub)]
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    X = I.features(n, 12, 9)
+    W = I.make_weights(model, 9, zero_bias=False)
+    rp = ripple.Ripple(n, src, dst, X, model, W, max_batch=8192)
+    orc = Oracle(n, src, dst, X, model, W)
+    rows = I.features(2, 12, 99)
+
+    def apply(recs):
+        ups = G.ups_array(recs)
+        if mem == "device":
+            u = torch.from_numpy(np.stack([ups["op"], ups["u"], ups["v"]], axis=1).astype(np.int32)).cuda()
+            rp.apply_batch(u, torch.from_numpy(rows).cuda())
+        else:
+            rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        G.check_graph(rp, orc)
+        G.check_frontiers(rp, orc, L)
+        G.check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+
+    do, di = rp.degrees()
+    deg = int(do[hub]) + int(di[hub])
+    assert deg > 5000
+    apply([(I.OP_ADD_EDGE, 3, 4), (I.OP_DEL_VERTEX, hub, 0), (I.OP_SET_FEATURE, 8, 1)])
+    st = rp.stats()
+    assert st["n_expanded"] == deg and st["n_deleted"] == deg - 1     # the self-loop is stored in both lists
+    do, di = rp.degrees()
+    assert int(do[hub]) == 0 and int(di[hub]) == 0
+    assert float(rp.embeddings(0)[hub].abs().max()) == 0.0
+    # the same id comes back: features first, then edges in both directions
+    apply([(I.OP_SET_FEATURE, hub, 0), (I.OP_ADD_EDGE, hub, 5), (I.OP_ADD_EDGE, 6, hub), (I.OP_ADD_EDGE, hub, hub)])
+    assert rp.stats()["n_added"] == 3
+    # deleted again together with a neighbour, with edge operations on both sides of the deletions
+    apply([(I.OP_ADD_EDGE, hub, 7), (I.OP_DEL_VERTEX, hub, 0), (I.OP_DEL_VERTEX, 5, 0), (I.OP_ADD_EDGE, hub, 9),
+           (I.OP_DEL_VERTEX, hub, 0), (I.OP_ADD_EDGE, 5, hub)])
+    rp.close()
+
+
+def test_expansion_beyond_the_batch_capacity_is_rejected(env):
+    ripple, Oracle = env
+    model = I.sage_model([8, 16, 4], I.AGG_SUM)
+    n = 2000
+    src, dst = I.er_graph(n, 6000, 13)
+    have = edge_set(src, dst)
+    extra = [(1, v) for v in range(2, 1500) if (1, v) not in have]
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    X = I.features(n, 8, 13)
+    W = I.make_weights(model, 13)
+    rp = ripple.Ripple(n, src, dst, X, model, W, max_batch=1024)
+    orc = Oracle(n, src, dst, X, model, W)
+    before = [rp.embeddings(l).clone() for l in range(3)]
+    ups = G.ups_array([(I.OP_ADD_EDGE, 5, 6), (I.OP_DEL_VERTEX, 1, 0), (I.OP_SET_FEATURE, 9, 0)])
+    with pytest.raises(ripple.RippleError) as ei:
+        rp.apply_batch(ups, I.features(1, 8, 1))
+    assert ei.value.status == ripple.ERR_CAPACITY and "max_batch" in str(ei.value)
+    G.check_graph(rp, orc)
+    for l in range(3):
+        assert bool((rp.embeddings(l) == before[l]).all())
+    # the context is still usable, and a deletion that fits goes through
+    small = int(np.argmin(np.bincount(src, minlength=n) + np.bincount(dst, minlength=n) + (np.arange(n) == 1) * 10**6))
+    ups = G.ups_array([(I.OP_DEL_VERTEX, small, 0), (I.OP_ADD_EDGE, 5, 6)])
+    rp.apply_batch(ups, None)
+    assert orc.apply_incremental(ups, None) == 0
+    G.check_graph(rp, orc)
+    G.check_frontiers(rp, orc, 2)
+    G.check_values(rp, orc.full(), 2)
+    # out-of-range vertex: rejected like any other bad id
+    with pytest.raises(ripple.RippleError) as ei:
+        rp.apply_batch(G.ups_array([(I.OP_DEL_VERTEX, n, 0)]), None)
+    assert ei.value.status == ripple.ERR_VERTEX_RANGE
+    G.check_graph(rp, orc)
+    rp.close()
