@@ -1,16 +1,18 @@
 // Tensor-core form of the affected-row layer update for sm_100a: tcgen05.mma (kind::tf32) with
 // the accumulator tile in tensor memory.
 //
-// One CTA owns tiles of 128 affected rows x all (<= 256) output columns.  Per 32-float K chunk the
-// CTA's threads gather the A rows by vertex id (applying the sink normalisation or the GIN self
-// factor on the way), split every fp32 value x into hi = x with the 13 low mantissa bits cleared
-// (exactly representable in tf32) and lo = x - hi, and store both into shared memory in the
-// K-major 128-byte-swizzle layout the tensor core reads; the transposed weights arrive pre-split
-// the same way.  One elected thread then issues hi*hi + lo*hi + hi*lo (three MMAs per 8-float K
-// step), which reproduces the fp32 product to about 2^-21 relative, and commits to an mbarrier
-// so that the next-but-one chunk can reuse the stage.  With tc_mode = TC_TF32 only hi*hi is
-// issued (plain TF32, 2^-11).  The epilogue reads the accumulators back with tcgen05.ld, one row
-// per thread, and runs the same fused bias / activation / delta / commit code as the SIMT form.
+// One persistent CTA per SM takes tiles of 128 affected rows x all (<= 256) output columns, in
+// passes of at most 128 columns.  Per 32-float K chunk the loader warps gather the A rows by vertex
+// id (applying the sink normalisation or the GIN self factor on the way), split every fp32 value x
+// into hi = x with the 13 low mantissa bits cleared (exactly representable in tf32) and lo = x - hi,
+// and store both into shared memory in the K-major 128-byte-swizzle layout the tensor core reads;
+// the transposed weights arrive pre-split the same way (cp.async from L2, two steps ahead).  One
+// elected thread issues hi*hi + lo*hi + hi*lo (three MMAs per 8-float K step), which reproduces
+// the fp32 product to about 2^-21 relative, and commits to an mbarrier so that the stage can be
+// refilled.  With tc_mode = TC_TF32 only hi*hi is issued (plain TF32, 2^-11).  Accumulators are
+// double-buffered in tensor memory; four epilogue warps read a finished tile back with tcgen05.ld
+// and run the same fused bias / activation / delta / commit code as the SIMT form while the next
+// tile's main loop is already running.
 //
 // Every wait is bounded: if an mbarrier does not complete within the spin limit the CTA records
 // RIPPLE_ERR_TIMEOUT in the control block, frees its tensor memory and returns.
@@ -92,22 +94,52 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// barrier among the loader warps only (the MMA warp never joins it)
+// barrier among the loader warps only (the other roles never join it)
 __device__ __forceinline__ void loaders_sync() { asm volatile("bar.sync 1, %0;" ::"n"(TC_THREADS) : "memory"); }
 
-// Warp roles: warps 0..7 ("loaders") stage the operands of every K chunk and run the epilogue;
-// warp 8 issues the MMAs.  Two mbarriers per stage hand the stage back and forth:
-//   full[s]   8 arrivals (one per loader warp, after its stores and proxy fence) -> MMA warp may read
-//   empty[s]  1 arrival (tcgen05.commit of the MMAs that read the stage)         -> loaders may refill
-// so the single-thread MMA issue (a microsecond per chunk) overlaps the loads of the next chunk.
+// the same barrier, returning whether any loader thread passed a non-zero flag: a decision every
+// loader thread takes alike (a thread that left the loop alone would strand the others here)
+__device__ __forceinline__ bool loaders_sync_any(int flag) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 1, %2, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(out) : "r"(flag), "n"(TC_THREADS) : "memory");
+    return out != 0;
+}
+
+// warp-uniform view of the failure flag
+__device__ __forceinline__ bool warp_failed(volatile int* flag) { return __any_sync(0xffffffffu, *flag != 0); }
+
+constexpr int TC_STAGES = 2;
+constexpr int TC_NH = 256;                 // output columns per MMA pass (all of them: n_pad <= 256)
+constexpr int TC_EPI_WARPS = 8;             // two per tensor-memory lane quarter, alternating column slabs
+constexpr int TC_ALL_THREADS = TC_THREADS + 32 + 32 * TC_EPI_WARPS;
+constexpr int TC_SLAB = 16;                // columns per epilogue step
+constexpr int TC_SLAB_LD = TC_SLAB + 4;    // 20 floats: 16-byte stores of 8 consecutive rows fall on distinct banks
+
+// Warp roles.  Warps 0..7 ("loaders") stage the operands, warp 8 issues the MMAs, warps 9..16 run
+// the epilogue.  Every K chunk of a tile (128 rows x all output columns) is one step and takes one
+// of two operand stages; the step counter runs on across tiles, so the loads of the next tile
+// start while the last MMAs of this one are still in flight.
+// Accumulators are double-buffered in tensor memory: the epilogue of tile t overlaps the main
+// loop of tile t + 1.  Barriers (all waits bounded):
+//   full[s]        8 arrivals (one per loader warp, after its stores and proxy fence) -> MMA warp may read
+//   empty[s]       tcgen05.commit of the MMAs that read stage s                      -> loaders may refill
+//   acc_full[b]    tcgen05.commit after the last MMA of a tile into buffer b         -> epilogue may read
+//   acc_empty[b]   8 arrivals (one per epilogue warp, accumulators read)             -> MMA warp may overwrite
+// Weights of step g + 1 are requested (cp.async from L2) as soon as step g has been handed over;
+// the gathered A rows are prefetched one step ahead in registers.
 template <bool X3>
-__global__ void __launch_bounds__(TC_THREADS + 32, 1)
+__global__ void __launch_bounds__(TC_ALL_THREADS, 1)
 k_update_rows_tc(Ctl* ctl, UpdParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full[2], empty[2];
+    __shared__ uint64_t full[TC_STAGES], empty[TC_STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
-    __shared__ int row_id[TC_M];
-    __shared__ float row_scale[TC_M];
+    __shared__ int row_id[2][TC_M];
+    __shared__ float row_scale[2][TC_M];
     __shared__ volatile int s_fail;
 
     if (ctl->abort) return;
@@ -117,19 +149,21 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
     if ((int)blockIdx.x >= row_tiles) return;   // before any allocation
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool is_loader = warp < TC_THREADS / 32;
     const bool is_mma_warp = warp == TC_THREADS / 32;
     const int n_pad = p.n_pad;
-    const uint32_t b_bytes = (uint32_t)n_pad * 128u;
-    const uint32_t stage_bytes = (X3 ? 2u : 1u) * (TC_A_BYTES + b_bytes);
+    const int n_pass = (n_pad + TC_NH - 1) / TC_NH;
+    constexpr uint32_t B_BYTES = TC_NH * 128u;
+    constexpr uint32_t STAGE_BYTES = (X3 ? 2u : 1u) * (TC_A_BYTES + B_BYTES);
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < n_pad) tmem_cols <<= 1;
+    float* slabs = reinterpret_cast<float*>(smem + TC_STAGES * STAGE_BYTES);   // one 32-row slab per epilogue warp
+    uint32_t buf_cols = 32;
+    while ((int)buf_cols < n_pad) buf_cols <<= 1;
+    const uint32_t tmem_cols = 2 * buf_cols;
 
     if (tid == 0) {
-        mbar_init(&full[0], TC_THREADS / 32);
-        mbar_init(&full[1], TC_THREADS / 32);
-        mbar_init(&empty[0], 1);
-        mbar_init(&empty[1], 1);
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(&full[s], TC_THREADS / 32); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], TC_EPI_WARPS); }
         s_fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -143,202 +177,220 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
     tc_fence_after();
     const uint32_t tmem_base = tmem_slot;
 
-    // instruction descriptor: fp32 accumulate, tf32 x tf32, both K-major, N = n_pad, M = 128
-    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n_pad >> 3) << 17) |
-                           ((uint32_t)(TC_M >> 4) << 24);
     const int nchunks = p.k_pad / TC_KC;
-    uint32_t uses[2] = {0u, 0u};   // how often each stage has been handed over so far (same in every thread)
+    const int steps_per_tile = n_pass * nchunks;
+    const int my_tiles = (row_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int total_steps = my_tiles * steps_per_tile;
 
     if (is_mma_warp) {
         // ---------------- MMA issue ----------------
-        for (int tile = blockIdx.x; tile < row_tiles && !s_fail; tile += gridDim.x) {
-            for (int kc = 0; kc < nchunks; ++kc) {
-                const int s = kc & 1;
-                uint8_t* a_hi = smem + (size_t)s * stage_bytes;
-                uint8_t* a_lo = a_hi + TC_A_BYTES;
-                uint8_t* b_hi = a_hi + (X3 ? 2 : 1) * TC_A_BYTES;
-                uint8_t* b_lo = b_hi + b_bytes;
-                if (lane == 0) {
-                    if (!mbar_wait_bounded(&full[s], uses[s] & 1)) s_fail = 1;
-                    if (!s_fail) {
-                        tc_fence_after();
-                        const uint64_t da_hi = tc_smem_desc(smem_u32(a_hi)), db_hi = tc_smem_desc(smem_u32(b_hi));
-                        const uint64_t da_lo = tc_smem_desc(smem_u32(a_lo)), db_lo = tc_smem_desc(smem_u32(b_lo));
+        int g = 0;
+        bool failed = false;
+        for (int lt = 0; lt < my_tiles && !failed; ++lt) {
+            const int b = lt & 1, ub = lt >> 1;
+            // the epilogue must have drained this accumulator buffer (tile lt - 2)
+            if (lane == 0 && ub > 0 && !mbar_wait_bounded(&acc_empty[b], (ub - 1) & 1)) s_fail = 1;
+            __syncwarp();
+            if ((failed = warp_failed(&s_fail))) break;
+            tc_fence_after();
+            for (int ps = 0; ps < n_pass && !failed; ++ps) {
+                const int ncol = min(TC_NH, n_pad - ps * TC_NH);
+                // instruction descriptor: fp32 accumulate, tf32 x tf32, both K-major, N = ncol, M = 128
+                const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(ncol >> 3) << 17) |
+                                       ((uint32_t)(TC_M >> 4) << 24);
+                const uint32_t d_addr = tmem_base + (uint32_t)b * buf_cols + (uint32_t)(ps * TC_NH);
+                for (int kc = 0; kc < nchunks; ++kc, ++g) {
+                    const int s = g % TC_STAGES;
+                    const uint32_t u = (uint32_t)(g / TC_STAGES);
+                    uint8_t* a_hi = smem + (size_t)s * STAGE_BYTES;
+                    uint8_t* a_lo = a_hi + TC_A_BYTES;
+                    uint8_t* b_hi = a_hi + (X3 ? 2 : 1) * TC_A_BYTES;
+                    uint8_t* b_lo = b_hi + B_BYTES;
+                    if (lane == 0) {
+                        if (!mbar_wait_bounded(&full[s], u & 1)) s_fail = 1;
+                        if (!s_fail) {
+                            tc_fence_after();
+                            const uint64_t da_hi = tc_smem_desc(smem_u32(a_hi)), db_hi = tc_smem_desc(smem_u32(b_hi));
+                            const uint64_t da_lo = tc_smem_desc(smem_u32(a_lo)), db_lo = tc_smem_desc(smem_u32(b_lo));
 #pragma unroll
-                        for (int j = 0; j < TC_KC / 8; ++j) {     // one MMA K step = 8 floats = 32 bytes
-                            const uint64_t adv = (uint64_t)((j * 32) >> 4);
-                            tc_mma_tf32(tmem_base, da_hi + adv, db_hi + adv, idesc, (kc | j) != 0);
-                            if (X3) {
-                                tc_mma_tf32(tmem_base, da_lo + adv, db_hi + adv, idesc, 1u);
-                                tc_mma_tf32(tmem_base, da_hi + adv, db_lo + adv, idesc, 1u);
+                            for (int j = 0; j < TC_KC / 8; ++j) {     // one MMA K step = 8 floats = 32 bytes
+                                const uint64_t adv = (uint64_t)((j * 32) >> 4);
+                                tc_mma_tf32(d_addr, da_hi + adv, db_hi + adv, idesc, (kc | j) != 0);
+                                if (X3) {
+                                    tc_mma_tf32(d_addr, da_lo + adv, db_hi + adv, idesc, 1u);
+                                    tc_mma_tf32(d_addr, da_hi + adv, db_lo + adv, idesc, 1u);
+                                }
                             }
+                            tc_commit(&empty[s]);
+                            if (ps == n_pass - 1 && kc == nchunks - 1) tc_commit(&acc_full[b]);
                         }
-                        tc_commit(&empty[s]);
                     }
+                    __syncwarp();
+                    if ((failed = warp_failed(&s_fail))) break;
                 }
-                __syncwarp();
-                uses[s]++;
-                if (s_fail) break;
             }
         }
-    } else {
-        // ---------------- loaders + epilogue ----------------
-        for (int tile = blockIdx.x; tile < row_tiles && !s_fail; tile += gridDim.x) {
-            const int r0 = tile * TC_M;
+    } else if (is_loader) {
+        // ---------------- operand staging ----------------
+        constexpr int A_ITERS = (TC_M * 8) / TC_THREADS;
+        constexpr int B_ITERS = (TC_NH * 8) / TC_THREADS;
+        auto write_ids = [&](int lt) {   // vertex ids and sink scales of local tile lt, buffer lt & 1
             if (tid < TC_M) {
-                int i = r0 + tid, v = -1;
+                const int i = ((int)blockIdx.x + lt * (int)gridDim.x) * TC_M + tid;
+                int v = -1;
                 float sc = 0.f;
-                if (i < n) {
+                if (lt < my_tiles && i < n) {
                     v = p.list ? p.list[i] : i;
                     sc = upd_row_scale(p, v);
                 }
-                row_id[tid] = v;
-                row_scale[tid] = sc;
+                row_id[lt & 1][tid] = v;
+                row_scale[lt & 1][tid] = sc;
             }
-            loaders_sync();
-
-            // The gathered A rows come from DRAM, the weights from L2: A is therefore loaded one chunk
-            // further ahead (registers), so that two chunks of row gathers are in flight.
-            constexpr int A_ITERS = (TC_M * 8) / TC_THREADS;
-            constexpr int B_ITERS = (256 * 8) / TC_THREADS;   // n_pad <= 256
-            float4 ax[A_ITERS], ax_next[A_ITERS];
-            auto load_a = [&](int kc, float4 (&dst)[A_ITERS]) {
+        };
+        float4 ax[A_ITERS], ax_next[A_ITERS];
+        auto load_a = [&](int g, float4 (&dst)[A_ITERS]) {   // 128 rows x 8 pieces of 16 bytes, by vertex id
+            const int lt = g / steps_per_tile, kc = (g - lt * steps_per_tile) % nchunks, b = lt & 1;
+            const int r0 = ((int)blockIdx.x + lt * (int)gridDim.x) * TC_M;
 #pragma unroll
-                for (int it = 0; it < A_ITERS; ++it) {   // 128 rows x 8 chunks of 16 bytes, by vertex id
-                    const int idx = tid + it * TC_THREADS, r = idx >> 3, c = idx & 7;
-                    const int v = row_id[r], k = kc * TC_KC + c * 4;
-                    dst[it] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (v >= 0 && k < p.K) dst[it] = upd_load_a(p, v, r0 + r, k, row_scale[r]);
-                }
-            };
-            // asynchronous copy of chunk kc's pre-split transposed weights (n_pad output columns x 8
-            // pieces of 16 bytes, hi and lo) from L2 straight into their swizzled places in stage kc & 1;
-            // the MMAs that last read that stage must have finished
-            auto copy_b = [&](int kc) {
-                const int s = kc & 1;
-                uint8_t* b_hi = smem + (size_t)s * stage_bytes + (X3 ? 2 : 1) * TC_A_BYTES;
-                uint8_t* b_lo = b_hi + b_bytes;
-                if (uses[s] > 0 && !mbar_wait_bounded(&empty[s], (uses[s] - 1) & 1)) s_fail = 1;
+            for (int it = 0; it < A_ITERS; ++it) {
+                const int idx = tid + it * TC_THREADS, r = idx >> 3, c = idx & 7;
+                const int v = row_id[b][r], k = kc * TC_KC + c * 4;
+                dst[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (v >= 0 && k < p.K) dst[it] = upd_load_a(p, v, r0 + r, k, row_scale[b][r]);
+            }
+        };
+        // asynchronous copy of step g's pre-split transposed weights (<= 128 output columns x 8 pieces
+        // of 16 bytes, hi and lo) from L2 straight into their swizzled places in stage g % 3; the MMAs
+        // that last read that stage must have finished.  Always closes one copy group.
+        auto copy_b = [&](int g) {
+            if (g < total_steps) {
+                const int s = g % TC_STAGES;
+                const uint32_t u = (uint32_t)(g / TC_STAGES);
+                if (u > 0 && !s_fail && !mbar_wait_bounded(&empty[s], (u - 1) & 1)) s_fail = 1;
+                const int r = g % steps_per_tile, ps = r / nchunks, kc = r - ps * nchunks;
+                const int ncol = min(TC_NH, n_pad - ps * TC_NH);
+                uint8_t* b_hi = smem + (size_t)s * STAGE_BYTES + (X3 ? 2 : 1) * TC_A_BYTES;
+                uint8_t* b_lo = b_hi + B_BYTES;
 #pragma unroll
                 for (int it = 0; it < B_ITERS; ++it) {
                     const int idx = tid + it * TC_THREADS;
-                    if (idx < n_pad * 8) {
-                        const size_t g = (size_t)(idx >> 3) * p.k_pad + kc * TC_KC + (idx & 7) * 4;
+                    if (idx < ncol * 8) {
+                        const size_t go = (size_t)(ps * TC_NH + (idx >> 3)) * p.k_pad + kc * TC_KC + (idx & 7) * 4;
                         const uint32_t off = tc_swz(idx >> 3, idx & 7);
-                        cp_async16(smem_u32(b_hi + off), p.Wt_hi + g);
-                        if (X3) cp_async16(smem_u32(b_lo + off), p.Wt_lo + g);
+                        cp_async16(smem_u32(b_hi + off), p.Wt_hi + go);
+                        if (X3) cp_async16(smem_u32(b_lo + off), p.Wt_lo + go);
                     }
                 }
-                asm volatile("cp.async.commit_group;" ::: "memory");
-            };
-            load_a(0, ax);
-            copy_b(0);
-            for (int kc = 0; kc < nchunks; ++kc) {
-                const int s = kc & 1;
-                uint8_t* a_hi = smem + (size_t)s * stage_bytes;
-                uint8_t* a_lo = a_hi + TC_A_BYTES;                              // only if X3
-                // next chunk's row gathers first (registers), so that they have a whole iteration to land
-                if (kc + 1 < nchunks) load_a(kc + 1, ax_next);
-#pragma unroll
-                for (int it = 0; it < A_ITERS; ++it) {
-                    const int idx = tid + it * TC_THREADS;
-                    const uint32_t off = tc_swz(idx >> 3, idx & 7);
-                    const float4 x = ax[it];
-                    const float4 h = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
-                    *reinterpret_cast<float4*>(a_hi + off) = h;
-                    if (X3) *reinterpret_cast<float4*>(a_lo + off) = make_float4(x.x - h.x, x.y - h.y, x.z - h.z, x.w - h.w);
-                }
-                asm volatile("cp.async.wait_group 0;" ::: "memory");   // this chunk's weights have landed
-                fence_async_smem();   // generic-proxy stores -> visible to the tensor core's async proxy
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&full[s]);
-                uses[s]++;
-                // the next chunk's weights travel while its rows are split and stored
-                if (kc + 1 < nchunks) copy_b(kc + 1);
-#pragma unroll
-                for (int it = 0; it < A_ITERS; ++it) ax[it] = ax_next[it];
-                if (s_fail) break;
             }
-            if (s_fail) break;
-            // the last commit covers every MMA of the tile
-            {
-                const int s = (nchunks - 1) & 1;
-                if (!mbar_wait_bounded(&empty[s], (uses[s] - 1) & 1)) s_fail = 1;
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        write_ids(0);
+        write_ids(1);
+        loaders_sync();
+        load_a(0, ax);
+        copy_b(0);
+        for (int g = 0; g < total_steps; ++g) {
+            const int s = g % TC_STAGES;
+            const int lt = g / steps_per_tile;
+            if (lt >= 1 && g == lt * steps_per_tile) {
+                // ids of the tile after this one; their buffer last served tile lt - 1, fully staged by now
+                write_ids(lt + 1);
+                if (loaders_sync_any(s_fail)) break;   // the only place the loaders leave early, all together
             }
-            if (s_fail) break;
+            uint8_t* a_hi = smem + (size_t)s * STAGE_BYTES;
+            uint8_t* a_lo = a_hi + TC_A_BYTES;                              // only if X3
+            // next step's row gathers first (registers), so that they have a whole step to land
+            if (g + 1 < total_steps) load_a(g + 1, ax_next);
+#pragma unroll
+            for (int it = 0; it < A_ITERS; ++it) {
+                const int idx = tid + it * TC_THREADS;
+                const uint32_t off = tc_swz(idx >> 3, idx & 7);
+                const float4 x = ax[it];
+                const float4 h = make_float4(tf32_hi(x.x), tf32_hi(x.y), tf32_hi(x.z), tf32_hi(x.w));
+                *reinterpret_cast<float4*>(a_hi + off) = h;
+                if (X3) *reinterpret_cast<float4*>(a_lo + off) = make_float4(x.x - h.x, x.y - h.y, x.z - h.z, x.w - h.w);
+            }
+            asm volatile("cp.async.wait_group 0;" ::: "memory");   // this step's weights have landed
+            fence_async_smem();   // generic-proxy stores -> visible to the tensor core's async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full[s]);
+            copy_b(g + 1);   // travels while the next step's rows are split and stored
+#pragma unroll
+            for (int it = 0; it < A_ITERS; ++it) ax[it] = ax_next[it];
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    } else {
+        // ---------------- epilogue ----------------
+        // A warp's index modulo 4 fixes the tensor-memory lanes it may read: rows 32 q .. 32 q + 31 of the
+        // tile, shared by two warps that take alternate 16-column slabs.  Per slab every lane pulls
+        // its own row's 16 accumulators, the warp turns them through a small shared-memory slab, and
+        // then each pass handles 8 rows x 64 bytes, so that the previous row, the cached projection,
+        // the delta row and the new row move in whole sectors; the loads of all 4 passes are issued
+        // before the first is used.
+        const int q = warp & 3;
+        const int ew = warp - (TC_THREADS / 32 + 1);     // 0..7
+        const int parity = ew >> 2;                      // which of the quarter's two warps: even or odd slabs
+        float* slab = slabs + (size_t)ew * 32 * TC_SLAB_LD;
+        const bool need_old = upd_needs_old(p);
+        const bool need_z = p.addend2 != nullptr;
+        const int sub_r = lane >> 2, sub_c = 4 * (lane & 3);   // 8 rows x 64 bytes per pass
+        for (int lt = 0; lt < my_tiles; ++lt) {
+            const int b = lt & 1, ub = lt >> 1;
+            const int r0 = ((int)blockIdx.x + lt * (int)gridDim.x) * TC_M + 32 * q;
+            int v_own = -1;
+            float sc_own = 0.f;
+            if (r0 + lane < n) {
+                v_own = p.list ? p.list[r0 + lane] : r0 + lane;
+                sc_own = upd_row_scale(p, v_own);
+            }
+            if (lane == 0 && !mbar_wait_bounded(&acc_full[b], ub & 1)) s_fail = 1;
+            __syncwarp();
+            if (warp_failed(&s_fail)) break;
             tc_fence_after();
-
-            // Epilogue in two steps.  (1) Every thread copies its accumulator row (warp w: tensor-memory
-            // lanes 32 (w % 4).., warps 0-3 the first half of the 16-column blocks, warps 4-7 the rest)
-            // into a row-major tile in shared memory; the operand stages are free now.  (2) Each warp
-            // then takes whole rows, 32 lanes x 16 bytes per pass, so that the previous row, the cached
-            // projection, the delta row and the new row all move in coalesced 512-byte pieces, four
-            // rows in flight.
-            float* tile_s = reinterpret_cast<float*>(smem);
-            const int tstride = n_pad + 4;   // = 4 mod 32: conflict-free 16-byte stores down a column
-            {
-                const int g = warp & 3, half = warp >> 2;
-                const int nblk = n_pad >> 4, split = (nblk + 1) >> 1;
-                const int b0 = half ? split : 0, b1 = half ? nblk : split;
-                const int r = 32 * g + lane;
-                for (int blk = b0; blk < b1; ++blk) {
-                    uint32_t x[16];
-                    const uint32_t taddr = tmem_base + ((uint32_t)(32 * g) << 16) + (uint32_t)(blk * 16);
-                    asm volatile(
-                        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-                        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-                        : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3]), "=r"(x[4]), "=r"(x[5]), "=r"(x[6]),
-                          "=r"(x[7]), "=r"(x[8]), "=r"(x[9]), "=r"(x[10]), "=r"(x[11]), "=r"(x[12]), "=r"(x[13]),
-                          "=r"(x[14]), "=r"(x[15])
-                        : "r"(taddr) : "memory");
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    float4* dst = reinterpret_cast<float4*>(tile_s + (size_t)r * tstride + blk * 16);
+            for (int c0 = parity * TC_SLAB; c0 < p.n_cols; c0 += 2 * TC_SLAB) {
+                uint32_t x[16];
+                const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)b * buf_cols + (uint32_t)c0;
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                    : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3]), "=r"(x[4]), "=r"(x[5]), "=r"(x[6]),
+                      "=r"(x[7]), "=r"(x[8]), "=r"(x[9]), "=r"(x[10]), "=r"(x[11]), "=r"(x[12]), "=r"(x[13]),
+                      "=r"(x[14]), "=r"(x[15])
+                    : "r"(taddr) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                float4* mine = reinterpret_cast<float4*>(slab + (size_t)lane * TC_SLAB_LD);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        dst[q] = make_float4(__uint_as_float(x[4 * q]), __uint_as_float(x[4 * q + 1]),
-                                             __uint_as_float(x[4 * q + 2]), __uint_as_float(x[4 * q + 3]));
-                }
-            }
-            tc_fence_before();   // accumulators consumed: the MMA warp may overwrite them after our next arrival
-            loaders_sync();
-            {
-                constexpr int RUN = 4;                       // rows in flight per warp
-                const bool need_old = upd_needs_old(p);
-                const bool need_z = p.addend2 != nullptr;
-                const int npass = (p.n_cols + 127) >> 7;     // <= 2
-                for (int rb = warp; rb < TC_M; rb += (TC_THREADS / 32) * RUN) {
-                    int vv[RUN];
-                    float4 oldv[RUN][2], zv[RUN][2];
+                for (int j = 0; j < 4; ++j)
+                    mine[j] = make_float4(__uint_as_float(x[4 * j]), __uint_as_float(x[4 * j + 1]),
+                                          __uint_as_float(x[4 * j + 2]), __uint_as_float(x[4 * j + 3]));
+                __syncwarp();
+                const int col = c0 + sub_c;
+                int vv[4];
+                float ss[4];
+                float4 oldv[4], zv[4];
 #pragma unroll
-                    for (int t = 0; t < RUN; ++t) {
-                        const int r = rb + t * (TC_THREADS / 32);
-                        vv[t] = r < TC_M ? row_id[r] : -1;
-#pragma unroll
-                        for (int ps = 0; ps < 2; ++ps) {
-                            const int col = 4 * lane + 128 * ps;
-                            if (vv[t] >= 0 && ps < npass && col < p.n_cols) {
-                                if (need_old) oldv[t][ps] = upd_load_old(p, vv[t], col);
-                                if (need_z) zv[t][ps] = *reinterpret_cast<const float4*>(p.addend2 + (size_t)vv[t] * p.ld_add + col);
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int t = 0; t < RUN; ++t) {
-                        const int r = rb + t * (TC_THREADS / 32);
-                        if (vv[t] < 0) continue;
-#pragma unroll
-                        for (int ps = 0; ps < 2; ++ps) {
-                            const int col = 4 * lane + 128 * ps;
-                            if (ps < npass && col < p.n_cols) {
-                                const float4 acc = *reinterpret_cast<const float4*>(tile_s + (size_t)r * tstride + col);
-                                upd_epilogue4(p, vv[t], r0 + r, col, acc, row_scale[r], need_old, oldv[t][ps], need_z, zv[t][ps]);
-                            }
-                        }
+                for (int t = 0; t < 4; ++t) {
+                    const int rr = 8 * t + sub_r;
+                    vv[t] = __shfl_sync(FULL, v_own, rr);
+                    ss[t] = __shfl_sync(FULL, sc_own, rr);
+                    if (vv[t] >= 0 && col < p.n_cols) {
+                        if (need_old) oldv[t] = upd_load_old(p, vv[t], col);
+                        if (need_z) zv[t] = *reinterpret_cast<const float4*>(p.addend2 + (size_t)vv[t] * p.ld_add + col);
                     }
                 }
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int rr = 8 * t + sub_r;
+                    if (vv[t] >= 0 && col < p.n_cols) {
+                        const float4 acc = *reinterpret_cast<const float4*>(slab + (size_t)rr * TC_SLAB_LD + sub_c);
+                        upd_epilogue4(p, vv[t], r0 + rr, col, acc, ss[t], need_old, oldv[t], need_z, zv[t]);
+                    }
+                }
+                __syncwarp();   // the slab is rewritten by the next step
             }
-            // the tile buffer (= the operand stages) and row_id are free before the next tile's staging
-            loaders_sync();
+            tc_fence_before();   // accumulators consumed: the MMA warp may overwrite them after this arrival
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[b]);
         }
     }
 
@@ -353,25 +405,25 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
     }
 }
 
+static size_t tc_smem_bytes(bool x3) {
+    const size_t stage = (size_t)(x3 ? 2 : 1) * (TC_A_BYTES + (size_t)TC_NH * 128);
+    return TC_STAGES * stage + (size_t)TC_EPI_WARPS * 32 * TC_SLAB_LD * sizeof(float) + 1024;
+}
+
 void launch_update_tc(Ctx* c, const UpdParams& p) {
     const bool x3 = p.tc_mode == TC_TF32X3;
-    const size_t stage = (size_t)(x3 ? 2 : 1) * (TC_A_BYTES + (size_t)p.n_pad * 128);
-    // two operand stages, reused by the epilogue as a 128 x (n_pad + 4) fp32 tile
-    const size_t tile = (size_t)TC_M * (p.n_pad + 4) * sizeof(float);
-    const size_t smem = std::max(2 * stage, tile) + 1024;
-    const int per_sm = std::max<size_t>(1, std::min<size_t>(4, (size_t)(220 * 1024) / (smem + 2048)));
-    const int grid = c->n_sm * per_sm;
+    // one persistent CTA per SM: three operand stages and the epilogue slabs fill its shared memory
+    const int grid = c->n_sm;
     if (x3) {
-        RP_LAUNCH(c, k_update_rows_tc<true>, grid, TC_THREADS + 32, smem, c->ctl, p);
+        RP_LAUNCH(c, k_update_rows_tc<true>, grid, TC_ALL_THREADS, tc_smem_bytes(true), c->ctl, p);
     } else {
-        RP_LAUNCH(c, k_update_rows_tc<false>, grid, TC_THREADS + 32, smem, c->ctl, p);
+        RP_LAUNCH(c, k_update_rows_tc<false>, grid, TC_ALL_THREADS, tc_smem_bytes(false), c->ctl, p);
     }
 }
 
 void tc_prepare() {
-    const int max_smem = 2 * 2 * (TC_A_BYTES + 256 * 128) + 1024;
-    cudaFuncSetAttribute(k_update_rows_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
-    cudaFuncSetAttribute(k_update_rows_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    cudaFuncSetAttribute(k_update_rows_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(true));
+    cudaFuncSetAttribute(k_update_rows_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem_bytes(false));
 }
 
 // Transposed, K-contiguous, tf32-split copy of a row-major K x ldw weight block.
