@@ -317,10 +317,12 @@ void graph_batch_classify(Ctx* c, int n) {
     if (n <= 0) return;
     const int T = 256;
     const int grid_ops = std::min(div_up(n, T), c->n_sm * 8);
-    RP_LAUNCH(c, k_expand_plan, grid_ops, T, 0, c->ups_dev, c->N, (long long)c->max_batch, c->ctl, c->side[0],
-              c->side[1], c->vjobs);
-    RP_LAUNCH(c, k_expand_copy, std::min(n, c->n_sm * 4), T, 0, c->ups_dev, c->op_seq, c->ctl, c->side[0],
-              c->side[1], c->vjobs);
+    if (c->may_expand) {   // a host batch known to hold no vertex deletion skips the expansion
+        RP_LAUNCH(c, k_expand_plan, grid_ops, T, 0, c->ups_dev, c->N, (long long)c->max_batch, c->ctl, c->side[0],
+                  c->side[1], c->vjobs);
+        RP_LAUNCH(c, k_expand_copy, std::min(n, c->n_sm * 4), T, 0, c->ups_dev, c->op_seq, c->ctl, c->side[0],
+                  c->side[1], c->vjobs);
+    }
     RP_LAUNCH(c, k_classify, grid_ops, T, 0, c->ups_dev, c->op_seq, c->N, c->ctl, c->hkeys, c->hwin,
               c->hsize - 1, c->op_slot, c->feat_last, c->vdel_seq);
     int grid = std::min(n, c->n_sm * 8);

@@ -368,9 +368,10 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
 // batch size into a CUDA graph and replayed.  Returns false if this batch must take the direct path.
 static bool launch_batch_graph(Ctx* c, int nb) {
     if (c->no_graphs || c->timing || nb < 1 || nb > RP_GRAPH_MAX_BATCH) return false;
+    const int key = 2 * nb + (c->may_expand ? 1 : 0);   // the captured chain differs with the expansion kernels
     int slot = -1;
     for (int i = 0; i < RP_GRAPH_SLOTS; ++i)
-        if (c->graph_exec[i] && c->graph_n[i] == nb) slot = i;
+        if (c->graph_exec[i] && c->graph_n[i] == key) slot = i;
     if (slot < 0) {
         slot = c->graph_next++ % RP_GRAPH_SLOTS;
         if (c->graph_exec[slot]) { cudaGraphExecDestroy(c->graph_exec[slot]); c->graph_exec[slot] = nullptr; }
@@ -382,7 +383,7 @@ static bool launch_batch_graph(Ctx* c, int nb) {
         if (e == cudaSuccess) e = cudaGraphInstantiate(&c->graph_exec[slot], g, 0);
         if (g) cudaGraphDestroy(g);
         if (e != cudaSuccess) { cudaGetLastError(); c->graph_exec[slot] = nullptr; c->no_graphs = 1; return false; }
-        c->graph_n[slot] = nb;
+        c->graph_n[slot] = key;
         c->graph_launches[slot] = c->launches;
     }
     c->launches = c->graph_launches[slot];
@@ -415,6 +416,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
     if (mem == RIPPLE_MEM_HOST)
         for (int i = 0; i < nb && !wide; ++i) wide = ups[i].op == RIPPLE_OP_DEL_VERTEX;
     const int ng = wide ? (int)c->max_batch : nb;
+    c->may_expand = wide || mem != RIPPLE_MEM_HOST;
     const bool try_graph = !wide && !c->no_graphs && !c->timing && nb >= 1 && nb <= RP_GRAPH_MAX_BATCH;
     const cudaMemcpyKind kind = mem == RIPPLE_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
     // operations are always staged: generated edge deletions are appended behind them

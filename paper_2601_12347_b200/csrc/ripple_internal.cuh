@@ -102,6 +102,7 @@ struct Ctx {
     int64_t E0;
     int64_t max_batch;
     int scatter_mode, gemm_mode, timing;
+    int may_expand;   // the batch being enqueued may hold vertex deletions (always assumed for device batches)
     float regather_threshold[RP_MAXL + 1];  // per hop: share of all edges from which the hop rebuilds its aggregates
     int n_sm;
     LayerDev layer[RP_MAXL + 1];

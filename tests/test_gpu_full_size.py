@@ -1,6 +1,7 @@
 """Parity at full size, in the launch configuration bench.py times (dense graph, 2-layer
 GraphSAGE-mean 100-256-47, batches of 1000), and on the ultra-dense second graph (233 K vertices,
-114.9 M edges, 602 features).
+114.9 M edges, 602 features), each also with a deeper model whose saturated hops rebuild their
+aggregates and whose wide layers run on the tensor-core update.
 
 The oracle cannot recompute 2.4 M x 256 embeddings per batch in test time, so here
   * graph state, affected sets and counters are compared exactly, batch by batch, against the
@@ -20,7 +21,7 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-4
 
 
-@pytest.mark.parametrize("wname,n_batches", [("dense-2l", 3), ("reddit-2l", 2)])
+@pytest.mark.parametrize("wname,n_batches", [("dense-2l", 3), ("reddit-2l", 2), ("dense-3l", 2), ("reddit-4l", 2)])
 def test_full_size_batch_1000_sampled_rows(wname, n_batches):
     import torch
     if not torch.cuda.is_available():
@@ -39,6 +40,7 @@ def test_full_size_batch_1000_sampled_rows(wname, n_batches):
     orc = Oracle(w.n, src, dst, X, w.model, W, bootstrap=False)
     stream = I.UpdateStream(w.n, src, dst, w.model.dims[0], w.seed)
     feat_now = {}
+    forms = set()
     for b in range(n_batches):
         ups, rows = stream.next_batch(1000)
         rp.apply_batch(ups, rows)
@@ -51,8 +53,11 @@ def test_full_size_batch_1000_sampled_rows(wname, n_batches):
             (c["added"], c["deleted"], c["noop_add"], c["noop_del"])
         for l in range(1, L + 1):
             assert st["active_edges"][l] == orc.active_edges(l)
+        forms.update(st["scatter_pull"][1:L + 1])
         for r in ups[ups["op"] == I.OP_SET_FEATURE]:
             feat_now[int(r["u"])] = rows[int(r["v"])]
+    if L >= 3:   # saturated hops rebuilt their aggregates, the others pushed deltas
+        assert forms == {0, 2}, forms
     # graph state, bit-exact
     rowptr, col = rp.export_graph()
     orp, ocol = orc.export_csr()
@@ -72,6 +77,7 @@ def test_full_size_batch_1000_sampled_rows(wname, n_batches):
     sample |= set(np.argsort(odi)[-40:].tolist())                      # largest in-degree hubs
     sample |= set(np.argsort(odo)[-10:].tolist())
     sample |= set(orc.affected(1)[:200].tolist()) | set(orc.affected(2)[:300].tolist())
+    sample |= set(orc.affected(L)[-300:].tolist())
     sample |= set(np.nonzero(odi == 0)[0][:50].tolist())                # rows with an empty aggregate
     worst = 0.0
     for l in range(1, L + 1):
