@@ -43,7 +43,7 @@
 #include <string.h>
 
 enum { KIND_SAGE = 0, KIND_GRAPHCONV = 1, KIND_GIN = 2 };
-enum { AGG_SUM = 0, AGG_MEAN = 1, AGG_WSUM_GCN = 2 };
+enum { AGG_SUM = 0, AGG_MEAN = 1, AGG_WSUM_GCN = 2, AGG_MAX = 3 };
 enum { ACT_IDENTITY = 0, ACT_RELU = 1 };
 enum { OP_ADD_EDGE = 0, OP_DEL_EDGE = 1, OP_SET_FEATURE = 2, OP_DEL_VERTEX = 3 };
 
@@ -116,7 +116,7 @@ static double coef_src(const oracle_t *o, int deg_out) {
 
 /* Sink-side normalisation applied to S_v at compute time (Table 1: mean, weighted sum). */
 static double norm_sink(const oracle_t *o, int deg_in) {
-    if (o->agg == AGG_SUM) return 1.0;
+    if (o->agg == AGG_SUM || o->agg == AGG_MAX) return 1.0;
     if (deg_in <= 0) return 0.0;
     return o->agg == AGG_MEAN ? 1.0 / (double)deg_in : 1.0 / sqrt((double)deg_in);
 }
@@ -164,6 +164,13 @@ static void layer_row(const layer_t *ly, const double *hprev, const double *Srow
 static void aggregate_row(const oracle_t *o, int v, const double *Hprev, int K, double *Srow) {
     for (int k = 0; k < K; ++k) Srow[k] = 0.0;
     const ivec *in = &o->in[v];
+    if (o->agg == AGG_MAX) { /* element-wise maximum over the in-neighbours; no in-neighbour: zeros */
+        for (int i = 0; i < in->n; ++i) {
+            const double *h = Hprev + (size_t)in->a[i] * K;
+            for (int k = 0; k < K; ++k) if (i == 0 || h[k] > Srow[k]) Srow[k] = h[k];
+        }
+        return;
+    }
     for (int i = 0; i < in->n; ++i) {
         int u = in->a[i];
         double c = coef_src(o, o->out[u].n);
@@ -501,6 +508,141 @@ static const srcinfo_t *source_find(const srcinfo_t *t, int n, int u) {
 
 /* O-inc: incremental propagation of one batch (Sec. 3.3).  Returns 0, or <0 if the batch is
  * rejected (nothing changed). */
+/* ------------------------------------------------------------------------------------------ */
+/* Monotonic aggregation (Sec. 3.4.2), max, for models without a self term (GraphConv).  A message
+ * <old, new> from a changed in-neighbour, <-, new> along an added edge or <old, -> along a deleted
+ * one leads, per element, to one of three actions at the sink:
+ *   - new exceeds the cached maximum: the cache is raised to it (incremental);
+ *   - old was the cached maximum and new is smaller (or the edge is gone): the maximum is no longer
+ *     known, the sink recomputes it over all current in-neighbours;
+ *   - otherwise nothing happens.
+ * A sink whose cached row ends up unchanged is not affected and sends nothing on (the pruning of
+ * Sec. 6.3).  "Changed" is decided on the values rounded to single precision, the precision of the
+ * embeddings this oracle is compared with. */
+static int differs_f32(const double *a, const double *b, int n) {
+    for (int k = 0; k < n; ++k) if ((float)a[k] != (float)b[k]) return 1;
+    return 0;
+}
+
+static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *feat_rows) {
+    int L = o->L, N = o->N;
+    int d0 = o->d[0];
+    /* in-degree before the batch: a sink that had no in-neighbour caches zeros, not a maximum */
+    int *din_old = (int *)malloc(sizeof(int) * (size_t)N);
+    for (int v = 0; v < N; ++v) din_old[v] = o->in[v].n;
+    for (int i = 0; i < dl->n_add; ++i) din_old[dl->add[i].v]--;
+    for (int i = 0; i < dl->n_del; ++i) din_old[dl->del[i].v]++;
+
+    int nA = dl->nF;
+    int *A = (int *)malloc(sizeof(int) * (size_t)(nA + 1));
+    memcpy(A, dl->F, sizeof(int) * (size_t)nA);
+    double *oldA = (double *)malloc(sizeof(double) * ((size_t)nA * (size_t)d0 + 1));
+    for (int i = 0; i < nA; ++i) {
+        double *row = o->H[0] + (size_t)A[i] * d0;
+        memcpy(oldA + (size_t)i * d0, row, sizeof(double) * (size_t)d0);
+        const float *src = dl->Frow[i] >= 0 ? feat_rows + (size_t)dl->Frow[i] * d0 : NULL;
+        for (int k = 0; k < d0; ++k) row[k] = src ? (double)src[k] : 0.0;
+    }
+    set_list(o, 0, A, nA);
+
+    int *snap_of = (int *)malloc(sizeof(int) * (size_t)N);   /* vertex -> its saved row, or -1 */
+    for (int v = 0; v < N; ++v) snap_of[v] = -1;
+    unsigned char *need = (unsigned char *)calloc((size_t)N, 1);
+
+    for (int l = 1; l <= L; ++l) {
+        int K = o->d[l - 1], J = o->d[l];
+        const double *Hp = o->H[l - 1];
+        double *S = o->S[l];
+        /* senders: rows of A_{l-1} that really changed */
+        int nC = 0;
+        int *C = (int *)malloc(sizeof(int) * (size_t)(nA + 1));
+        int *Cold = (int *)malloc(sizeof(int) * (size_t)(nA + 1));   /* index of the sender's old row */
+        for (int i = 0; i < nA; ++i)
+            if (differs_f32(Hp + (size_t)A[i] * K, oldA + (size_t)i * K, K)) { C[nC] = A[i]; Cold[nC] = i; nC++; }
+
+        int cap = 1024, nT = 0;              /* touched sinks and their rows before this hop */
+        int *T = (int *)malloc(sizeof(int) * (size_t)cap);
+        double *snap = (double *)malloc(sizeof(double) * (size_t)cap * (size_t)K);
+        long walked = 0;
+#define TOUCH(v)                                                                                   \
+        do {                                                                                       \
+            if (snap_of[v] < 0) {                                                                  \
+                if (nT == cap) { cap *= 2; T = (int *)realloc(T, sizeof(int) * (size_t)cap);       \
+                                 snap = (double *)realloc(snap, sizeof(double) * (size_t)cap * (size_t)K); } \
+                memcpy(snap + (size_t)nT * K, S + (size_t)(v) * K, sizeof(double) * (size_t)K);    \
+                snap_of[v] = nT; T[nT++] = (v);                                                    \
+            }                                                                                      \
+        } while (0)
+        /* <old, new> along the surviving out-edges of the senders */
+        for (int i = 0; i < nC; ++i) {
+            int u = C[i];
+            const double *hnew = Hp + (size_t)u * K, *hold = oldA + (size_t)Cold[i] * K;
+            const ivec *r = &o->out[u];
+            walked += r->n;
+            for (int j = 0; j < r->n; ++j) {
+                int v = r->a[j];
+                pair_t p = { u, v };
+                if (dl->n_add && bsearch(&p, dl->add, (size_t)dl->n_add, sizeof(pair_t), cmp_pair)) continue;
+                double *Sv = S + (size_t)v * K;
+                for (int k = 0; k < K; ++k) {
+                    if (hnew[k] > Sv[k]) { TOUCH(v); Sv[k] = hnew[k]; }
+                    else if (hold[k] == Sv[k] && hnew[k] < hold[k]) need[v] = 1;
+                }
+            }
+        }
+        /* <-, new> along added edges */
+        for (int i = 0; i < dl->n_add; ++i) {
+            int u = dl->add[i].u, v = dl->add[i].v;
+            if (din_old[v] == 0) { need[v] = 1; continue; }
+            const double *hnew = Hp + (size_t)u * K;
+            double *Sv = S + (size_t)v * K;
+            for (int k = 0; k < K; ++k) if (hnew[k] > Sv[k]) { TOUCH(v); Sv[k] = hnew[k]; }
+        }
+        /* <old, -> along deleted edges */
+        for (int i = 0; i < dl->n_del; ++i) {
+            int u = dl->del[i].u, v = dl->del[i].v;
+            int ia = find_sorted(A, nA, u);
+            const double *hold = ia >= 0 ? oldA + (size_t)ia * K : Hp + (size_t)u * K;
+            const double *Sv = S + (size_t)v * K;
+            if (o->in[v].n == 0) need[v] = 1;
+            for (int k = 0; k < K && !need[v]; ++k) if (hold[k] == Sv[k]) need[v] = 1;
+        }
+        /* recomputation of the sinks whose maximum is no longer known */
+        for (int v = 0; v < N; ++v) {
+            if (!need[v]) continue;
+            need[v] = 0;
+            TOUCH(v);
+            aggregate_row(o, v, Hp, K, S + (size_t)v * K);
+        }
+#undef TOUCH
+        o->active_edges[l] = walked + dl->n_add + dl->n_del;
+        /* affected = cached row changed */
+        int nAn = 0;
+        int *An = (int *)malloc(sizeof(int) * (size_t)(nT + 1));
+        for (int t = 0; t < nT; ++t) {
+            int v = T[t];
+            if (differs_f32(S + (size_t)v * K, snap + (size_t)t * K, K)) An[nAn++] = v;
+            snap_of[v] = -1;
+        }
+        qsort(An, (size_t)nAn, sizeof(int), cmp_int);
+        free(T); free(snap); free(C); free(Cold);
+
+        double *oldAn = (double *)malloc(sizeof(double) * ((size_t)nAn * (size_t)J + 1));
+#pragma omp parallel for schedule(dynamic, 64)
+        for (int i = 0; i < nAn; ++i) {
+            int v = An[i];
+            double *row = o->H[l] + (size_t)v * J;
+            memcpy(oldAn + (size_t)i * J, row, sizeof(double) * (size_t)J);
+            layer_row(&o->layer[l], Hp + (size_t)v * K, S + (size_t)v * K, 1.0, row);
+        }
+        set_list(o, l, An, nAn);
+        free(A); free(oldA);
+        A = An; nA = nAn; oldA = oldAn;
+    }
+    free(A); free(oldA); free(din_old); free(snap_of); free(need);
+    return 0;
+}
+
 int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const float *feat_rows,
                           int64_t n_rows) {
     delta_t dl;
@@ -508,6 +650,13 @@ int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const flo
     if (rc) return rc;
     int L = o->L, self_term = o->layer[1].kind != KIND_GRAPHCONV;
 
+    if (o->agg == AGG_MAX) {
+        if (self_term) { delta_free(&dl); return -3; }   /* built for models without a self term only */
+        apply_topology(o, &dl);
+        rc = apply_incremental_max(o, &dl, feat_rows);
+        delta_free(&dl);
+        return rc;
+    }
     apply_topology(o, &dl);
     /* old source coefficients of the endpoints whose out-degree changed */
     int nsrc; srcinfo_t *srcs = source_table(o, &dl, &nsrc);

@@ -33,6 +33,7 @@ KIND_GIN = 2       # h = act(W2 relu(W1 ((1+eps) h_v + agg_v) + b1) + b2)
 AGG_SUM = 0
 AGG_MEAN = 1
 AGG_WSUM_GCN = 2   # coefficient 1/sqrt(deg_out(u) * deg_in(v))
+AGG_MAX = 3        # element-wise maximum over the in-neighbours (monotonic; zeros if there are none)
 
 ACT_IDENTITY = 0
 ACT_RELU = 1
