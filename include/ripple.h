@@ -49,8 +49,14 @@ typedef enum {
 typedef enum { RIPPLE_MEM_HOST = 0, RIPPLE_MEM_DEVICE = 1 } ripple_mem;
 
 /* Aggregators of Table 1.  WSUM_GCN is the weighted sum with alpha_uv = 1/sqrt(deg_out(u) deg_in(v))
- * taken from the current graph and recomputed whenever a degree changes. */
-typedef enum { RIPPLE_AGG_SUM = 0, RIPPLE_AGG_MEAN = 1, RIPPLE_AGG_WSUM_GCN = 2 } ripple_agg;
+ * taken from the current graph and recomputed whenever a degree changes.
+ * MAX (Sec. 3.4.2, monotonic aggregation): element-wise maximum over the in-neighbours, zeros for a
+ * vertex without in-neighbours; GRAPHCONV layers only.  Its batches run hybrid-incrementally:
+ * a message carries the sender's old and new row, a sink raises its cached maximum, recomputes it
+ * over all in-neighbours, or ignores the message; a sink whose cached maximum did not change is
+ * not affected and propagates nothing (ripple_get_affected then lists exactly the vertices whose
+ * cached maximum changed; ripple_stats.senders those whose embedding changed). */
+typedef enum { RIPPLE_AGG_SUM = 0, RIPPLE_AGG_MEAN = 1, RIPPLE_AGG_WSUM_GCN = 2, RIPPLE_AGG_MAX = 3 } ripple_agg;
 
 /* Update functions (Eq. 2) of the model families of Sec. 6.1.1, x_v = normalised aggregate:
  *   SAGE       h = act(Wa^T h_v + Wb^T x_v + ba)                         (self term)

@@ -149,12 +149,16 @@ __global__ void k_bitmap_compact(uint32_t* bitmap, int n_words, const int* __res
     if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) *count_out = tile_base + total;
 }
 
-static void bitmap_to_list(Ctx* c, int32_t* list, int* count_dev, unsigned long long* pull_work) {
+void bitmap_to_list_from(Ctx* c, uint32_t* bitmap, int32_t* list, int* count_dev, unsigned long long* pull_work) {
     int tiles = div_up(c->n_words, CMP_T);
     int* tile_cnt = reinterpret_cast<int*>(c->tile_sums);  // scan scratch is free here
-    RP_LAUNCH(c, k_bitmap_tile_counts, tiles, CMP_T, 0, c->bitmap, c->n_words, tile_cnt);
-    RP_LAUNCH(c, k_bitmap_compact, tiles, CMP_T, 0, c->bitmap, c->n_words, tile_cnt, list, count_dev,
+    RP_LAUNCH(c, k_bitmap_tile_counts, tiles, CMP_T, 0, bitmap, c->n_words, tile_cnt);
+    RP_LAUNCH(c, k_bitmap_compact, tiles, CMP_T, 0, bitmap, c->n_words, tile_cnt, list, count_dev,
               pull_work ? c->side[1].deg : nullptr, pull_work);
+}
+
+static void bitmap_to_list(Ctx* c, int32_t* list, int* count_dev, unsigned long long* pull_work) {
+    bitmap_to_list_from(c, c->bitmap, list, count_dev, pull_work);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -193,6 +193,7 @@ void update_rows(Ctx* c, int l, bool full) {
         if (!full) { p.addend_rw = c->S[l]; p.addend_delta = c->dS[l]; }   // fold_deltas is skipped for these layers
     }
     float* dout = (full || l == c->L) ? nullptr : c->D[l & 1];  // the last hop sends nothing
+    p.dout_old = c->agg == RIPPLE_AGG_MAX;
     if (ly.kind == RIPPLE_LAYER_GIN) {
         // hidden = relu(W1^T ((1 + eps) h + x) + b1), kept as compact rows
         p.a_mode = pre ? A_SELF : A_SUM; p.epi_mode = EPI_TEMP; p.alpha = 1.0f + ly.eps;
@@ -228,7 +229,7 @@ void update_rows(Ctx* c, int l, bool full) {
 __global__ void k_feature_rows(Ctl* ctl, const ripple_update* __restrict__ ups, const float* __restrict__ feat,
                                int d0, const int32_t* __restrict__ A0, const int32_t* __restrict__ feat_last,
                                int src_norm, const int32_t* __restrict__ deg_out,
-                               const int32_t* __restrict__ deg_out_old, float* H0, int ld, float* D) {
+                               const int32_t* __restrict__ deg_out_old, float* H0, int ld, float* D, int keep_old) {
     if (ctl->abort) return;
     const int n = ctl->nA[0];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -245,7 +246,7 @@ __global__ void k_feature_rows(Ctl* ctl, const ripple_update* __restrict__ ups, 
         for (int k = lane_id(); k < ld; k += 32) {
             float x = (src && k < d0) ? src[k] : 0.f;
             float o = H0[(size_t)v * ld + k];
-            D[(size_t)i * ld + k] = cn * x - co * o;
+            D[(size_t)i * ld + k] = keep_old ? o : cn * x - co * o;
             H0[(size_t)v * ld + k] = x;
         }
     }
@@ -255,7 +256,7 @@ void feature_rows(Ctx* c, int n) {
     if (n <= 0) return;
     RP_LAUNCH(c, k_feature_rows, std::min(div_up(n, 8), c->n_sm * 8), 256, 0, c->ctl, c->ups_dev, c->feat_dev,
               c->d[0], c->A[0], c->feat_last, (int)c->src_norm, c->side[0].deg, c->deg_out_old, c->H[0],
-              c->ld[0], c->D[0]);
+              c->ld[0], c->D[0], (int)(c->agg == RIPPLE_AGG_MAX));
 }
 
 // ---------------------------------------------------------------------------------------------

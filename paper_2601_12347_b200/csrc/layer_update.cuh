@@ -39,6 +39,7 @@ struct UpdParams {
     const float* addend2;           // rows by id added as they are, same leading dimension (may be null)
     float* addend_rw;               // if set: addend with its pending per-batch sums folded in on the way
     float* addend_delta;            //   (addend_rw += addend_delta, addend_delta = 0); replaces addend
+    int dout_old;                   // Dout receives the row's previous value instead of a delta (monotonic aggregation)
     int src_norm;
     const int32_t* deg_out;
     const int32_t* deg_out_old;
@@ -133,7 +134,8 @@ __device__ __forceinline__ void upd_epilogue4(const UpdParams& p, int v, int i, 
             co = dold >= 0 ? coef_deg(dold) : cn;
         }
         *reinterpret_cast<float4*>(p.Dout + (size_t)i * p.ld_o + col) =
-            make_float4(cn * h.x - co * o.x, cn * h.y - co * o.y, cn * h.z - co * o.z, cn * h.w - co * o.w);
+            p.dout_old ? o
+                       : make_float4(cn * h.x - co * o.x, cn * h.y - co * o.y, cn * h.z - co * o.z, cn * h.w - co * o.w);
     }
     *dst = h;
 }

@@ -1,0 +1,379 @@
+// Monotonic aggregation (Sec. 3.4.2), max, for models without a self term.
+//
+// The cached aggregate S^l_v is the element-wise maximum of h^{l-1}_u over In(v) (zeros if v has no
+// in-neighbour).  A local delta cannot update it; instead a message carries the sender's old and
+// new row, <old, new>, and the sink takes one of three actions per element:
+//   raise       new > cached maximum: the cache moves up to it (an atomic maximum);
+//   invalidate  old == cached maximum and new < old (or the edge is gone): the maximum is no longer
+//               known, the sink is queued and recomputes its row over all current in-neighbours;
+//   nothing     otherwise.
+// A sink whose cached row ends up unchanged is not affected: it is not recomputed and sends
+// nothing on.  Senders of the next hop are the affected rows whose embedding really changed.
+#include "device_utils.cuh"
+#include "ripple_internal.cuh"
+
+#include <algorithm>
+#include <cfloat>
+
+namespace rp {
+
+constexpr int MAX_HUB_DEGREE = 4096;   // longer in-lists are recomputed by a whole block
+constexpr int MAX_CHUNK = 64;          // edges per warp work item of the message walk
+
+__device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
+
+// atomic maximum of an IEEE float: non-negative values order like signed integers, negative ones
+// like unsigned integers in reverse
+__device__ __forceinline__ void atomic_max_f32(float* addr, float val) {
+    if (val >= 0.f) atomicMax(reinterpret_cast<int*>(addr), __float_as_int(val));
+    else atomicMin(reinterpret_cast<unsigned int*>(addr), __float_as_uint(val));
+}
+
+__device__ __forceinline__ void mark_bit(uint32_t* bitmap, int v) {
+    const uint32_t m = 1u << (v & 31);
+    if (!(bitmap[v >> 5] & m)) atomicOr(&bitmap[v >> 5], m);
+}
+
+__device__ __forceinline__ float4 max4(const float4& a, const float4& b) {
+    return make_float4(fmaxf(a.x, b.x), fmaxf(a.y, b.y), fmaxf(a.z, b.z), fmaxf(a.w, b.w));
+}
+
+// acc = max(acc, rows of the in-neighbours [j_begin, j_end) of v); LPR lanes hold one row (NV float4
+// slots each), a warp works on 32 / LPR neighbours per step; on return every lane group holds the
+// maximum over all groups
+template <int NV, int LPR>
+__device__ __forceinline__ void max_accumulate(float4 (&acc)[NV], const Side& in, int v, int j_begin, int j_end,
+                                               const float* __restrict__ M, int ld) {
+    const int lane = lane_id(), nq = ld >> 2;
+    constexpr int EPI = 32 / LPR;
+    const int sub = lane / LPR, ql = lane % LPR;
+    const int64_t base = in.start[v];
+    for (int j0 = j_begin; j0 < j_end; j0 += 32) {
+        const int mine = j0 + lane < j_end ? in.col[base + j0 + lane] : 0;
+        const int cnt = min(32, j_end - j0);
+        for (int j = 0; j < cnt; j += EPI) {
+            const int jj = j + sub;
+            const int u = __shfl_sync(FULL, mine, jj & 31);
+            if (jj < cnt) {
+                const float4* row = reinterpret_cast<const float4*>(M + (size_t)u * ld);
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    const int q = ql + LPR * k;
+                    if (q < nq) acc[k] = max4(acc[k], __ldg(row + q));
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) {
+            acc[k].x = fmaxf(acc[k].x, __shfl_xor_sync(FULL, acc[k].x, o));
+            acc[k].y = fmaxf(acc[k].y, __shfl_xor_sync(FULL, acc[k].y, o));
+            acc[k].z = fmaxf(acc[k].z, __shfl_xor_sync(FULL, acc[k].z, o));
+            acc[k].w = fmaxf(acc[k].w, __shfl_xor_sync(FULL, acc[k].w, o));
+        }
+    }
+}
+
+template <int NV>
+__device__ __forceinline__ void fill(float4 (&acc)[NV], float x) {
+#pragma unroll
+    for (int k = 0; k < NV; ++k) acc[k] = make_float4(x, x, x, x);
+}
+
+// ---------------------------------------------------------------------------------------------
+// the maximum of one row over its whole in-list: a warp, or for long lists a block
+// ---------------------------------------------------------------------------------------------
+// mode 0 (bootstrap): rows = all vertices, the result is stored.
+// mode 1 (recomputation): rows = list; the result is compared with the cached row, stored if it
+//         differs, and the vertex is marked affected.
+template <int NV, int LPR>
+__global__ void __launch_bounds__(256)
+k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const int* n_dev, int n_host, Side in,
+           const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA, int32_t* long_rows,
+           int* n_long) {
+    if (ctl->abort) return;
+    const int n = n_dev ? *n_dev : n_host;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id(), nq = ld >> 2;
+    const int sub = lane / LPR, ql = lane % LPR;
+    for (int i = warp; i < n; i += nwarps) {
+        const int v = list ? list[i] : i;
+        const int deg = in.deg[v];
+        if (deg > MAX_HUB_DEGREE) {
+            if (lane == 0) long_rows[atomicAdd(n_long, 1)] = v;
+            continue;
+        }
+        float4 acc[NV];
+        fill<NV>(acc, deg > 0 ? neg_inf() : 0.f);
+        max_accumulate<NV, LPR>(acc, in, v, 0, deg, M, ld);
+        float4* dst = reinterpret_cast<float4*>(S + (size_t)v * ld);
+        bool differs = false;
+        if (sub == 0) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int q = ql + LPR * k;
+                if (q < nq) {
+                    if (mode) {
+                        const float4 o = dst[q];
+                        differs |= o.x != acc[k].x || o.y != acc[k].y || o.z != acc[k].z || o.w != acc[k].w;
+                    }
+                    dst[q] = acc[k];
+                }
+            }
+        }
+        if (mode && __any_sync(FULL, differs) && lane == 0) mark_bit(bitmapA, v);
+    }
+    (void)l;
+}
+
+// one block per long row: every warp takes a strided share of the in-list, the partial rows meet in
+// shared memory
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_max_long_rows(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const int* __restrict__ n_long, Side in,
+                const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA) {
+    extern __shared__ float part[];   // 8 warps x ld floats
+    __shared__ int s_differs;
+    if (ctl->abort) return;
+    const int n = *n_long;
+    const int warp = threadIdx.x >> 5, lane = lane_id(), nq = ld >> 2;
+    for (int i = blockIdx.x; i < n; i += gridDim.x) {
+        const int v = long_rows[i];
+        const int deg = in.deg[v];
+        float4 acc[NV];
+        fill<NV>(acc, neg_inf());
+        for (int j0 = warp * 1024; j0 < deg; j0 += 8 * 1024)
+            max_accumulate<NV, 32>(acc, in, v, j0, min(deg, j0 + 1024), M, ld);
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+            const int q = lane + 32 * k;
+            if (q < nq) reinterpret_cast<float4*>(part + (size_t)warp * ld)[q] = acc[k];
+        }
+        if (threadIdx.x == 0) s_differs = 0;
+        __syncthreads();
+        bool differs = false;
+        for (int q = threadIdx.x; q < nq; q += blockDim.x) {
+            float4 m = reinterpret_cast<const float4*>(part)[q];
+            for (int w = 1; w < 8; ++w) m = max4(m, reinterpret_cast<const float4*>(part + (size_t)w * ld)[q]);
+            float4* dst = reinterpret_cast<float4*>(S + (size_t)v * ld) + q;
+            if (mode) {
+                const float4 o = *dst;
+                differs |= o.x != m.x || o.y != m.y || o.z != m.z || o.w != m.w;
+            }
+            *dst = m;
+        }
+        if (differs) s_differs = 1;
+        __syncthreads();
+        if (mode && threadIdx.x == 0 && s_differs) mark_bit(bitmapA, v);
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// messages <old, new> along the out-edges of the senders
+// ---------------------------------------------------------------------------------------------
+// in-degree of v before the batch: a sink that had no in-neighbour caches zeros, not a maximum
+__device__ __forceinline__ int deg_in_before(const Side& in, int v) {
+    return in.deg[v] - in.cnt_add[v] + in.cnt_del[v];
+}
+
+template <int NV, int LPR>
+__global__ void __launch_bounds__(256)
+k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32_t* __restrict__ old_idx,
+               const int64_t* __restrict__ coff, Side out, Side in, const float* __restrict__ Hprev,
+               const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR) {
+    if (ctl->abort) return;
+    const int nC = ctl->nC[l - 1];
+    if (nC == 0) return;
+    const int64_t E = coff[nC];
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id(), nq = ld >> 2;
+    constexpr int EPI = 32 / LPR;
+    const int sub = lane / LPR, ql = lane % LPR;
+    const unsigned group = LPR == 32 ? FULL : (((1u << LPR) - 1u) << (sub * LPR));
+    for (int64_t e0 = (int64_t)warp * MAX_CHUNK; e0 < E; e0 += (int64_t)nwarps * MAX_CHUNK) {
+        const int64_t e1 = min(e0 + MAX_CHUNK, E);
+        int i = upper_row(coff, nC, e0);
+        int64_t e = e0;
+        while (e < e1) {
+            const int64_t row_end = coff[i + 1];
+            if (row_end <= e) { ++i; continue; }
+            const int64_t seg_end = min(e1, row_end);
+            const int u = senders[i];
+            const int64_t base = out.start[u] + (e - coff[i]);
+            const int cnt = (int)(seg_end - e);
+            float4 hn[NV], ho[NV];
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int q = ql + LPR * k;
+                hn[k] = q < nq ? __ldg(reinterpret_cast<const float4*>(Hprev + (size_t)u * ld) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                ho[k] = q < nq ? __ldg(reinterpret_cast<const float4*>(Old + (size_t)old_idx[i] * ld) + q) : hn[k];
+            }
+            for (int j = 0; j < cnt; j += EPI) {
+                const int jj = j + sub;
+                const bool live = jj < cnt;
+                const int v = live ? out.col[base + jj] : 0;
+                bool raise = false, invalid = false;
+                if (live) {
+                    if (deg_in_before(in, v) == 0) invalid = true;   // zeros cached: gather the real maximum
+                    else {
+                        float* srow = S + (size_t)v * ld;
+#pragma unroll
+                        for (int k = 0; k < NV; ++k) {
+                            const int q = ql + LPR * k;
+                            if (q < nq) {
+                                const float4 s = *reinterpret_cast<const float4*>(srow + 4 * q);
+                                const float nn[4] = {hn[k].x, hn[k].y, hn[k].z, hn[k].w};
+                                const float oo[4] = {ho[k].x, ho[k].y, ho[k].z, ho[k].w};
+                                const float ss[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) {
+                                    if (nn[t] > ss[t]) { atomic_max_f32(srow + 4 * q + t, nn[t]); raise = true; }
+                                    else if (oo[t] == ss[t] && nn[t] < oo[t]) invalid = true;
+                                }
+                            }
+                        }
+                    }
+                }
+                raise = __any_sync(group, raise);
+                invalid = __any_sync(group, invalid);
+                if (live && ql == 0) {
+                    if (raise) mark_bit(bitmapA, v);
+                    if (invalid) mark_bit(bitmapR, v);
+                }
+            }
+            e = seg_end;
+            ++i;
+        }
+    }
+}
+
+// edge records: <-, new> along an added edge, <old, -> along a deleted one; one warp per record
+__global__ void k_max_records(Ctl* ctl, const Rec* __restrict__ rec, Side in, const int32_t* __restrict__ posmap,
+                              const int32_t* __restrict__ old_idx, const float* __restrict__ Hprev,
+                              const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR) {
+    if (ctl->abort) return;
+    const int n = ctl->n_rec;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id();
+    for (int r = warp; r < n; r += nwarps) {
+        const int u = rec[r].u, v = rec[r].v;
+        float* srow = S + (size_t)v * ld;
+        bool raise = false, invalid = false;
+        if (rec[r].sign > 0) {
+            if (deg_in_before(in, v) == 0) invalid = true;
+            else
+                for (int k = lane; k < ld; k += 32) {
+                    const float x = Hprev[(size_t)u * ld + k];
+                    if (x > srow[k]) { atomic_max_f32(srow + k, x); raise = true; }
+                }
+        } else {
+            if (in.deg[v] == 0) invalid = true;
+            else {
+                const int p = posmap[u];
+                const float* orow = p >= 0 ? Old + (size_t)old_idx[p] * ld : Hprev + (size_t)u * ld;
+                for (int k = lane; k < ld; k += 32) invalid |= orow[k] == srow[k];
+            }
+        }
+        raise = __any_sync(FULL, raise);
+        invalid = __any_sync(FULL, invalid);
+        if (lane == 0) {
+            if (raise) mark_bit(bitmapA, v);
+            if (invalid) mark_bit(bitmapR, v);
+        }
+    }
+}
+
+// senders of the next hop: affected rows whose embedding really changed (old rows are kept compact,
+// in the order of A_l); one warp per affected row
+__global__ void k_max_senders(Ctl* ctl, int l, const int32_t* __restrict__ A, const float* __restrict__ H,
+                              const float* __restrict__ Old, int ld, int32_t* senders, int32_t* old_idx,
+                              int32_t* posmap) {
+    if (ctl->abort) return;
+    const int n = ctl->nA[l];
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id();
+    for (int i = warp; i < n; i += nwarps) {
+        const int v = A[i];
+        bool differs = false;
+        for (int k = lane; k < ld; k += 32) differs |= H[(size_t)v * ld + k] != Old[(size_t)i * ld + k];
+        if (__any_sync(FULL, differs) && lane == 0) {
+            const int idx = atomicAdd(&ctl->nC[l], 1);
+            senders[idx] = v;
+            old_idx[idx] = i;
+            posmap[v] = idx;
+        }
+    }
+}
+
+#define RP_MAX_DISPATCH(ld, CALL)                         \
+    do {                                                  \
+        const int nv_ = div_up((ld), 128);                \
+        if ((ld) <= 32) { CALL(1, 8); }                   \
+        else if ((ld) <= 64) { CALL(1, 16); }             \
+        else if (nv_ <= 1) { CALL(1, 32); }               \
+        else if (nv_ <= 2) { CALL(2, 32); }               \
+        else if (nv_ <= 4) { CALL(4, 32); }               \
+        else { CALL(8, 32); }                             \
+    } while (0)
+
+static void launch_long_rows(Ctx* c, int mode, const float* M, int ld, float* S, int32_t* long_rows, int* n_long) {
+    const int nv = div_up(ld, 128);
+    const size_t smem = (size_t)8 * ld * sizeof(float);
+#define LONG(NV) RP_LAUNCH(c, k_max_long_rows<NV>, c->n_sm, 256, smem, c->ctl, mode, long_rows, n_long, c->side[1], M, ld, S, c->bitmap)
+    if (nv <= 1) LONG(1); else if (nv <= 2) LONG(2); else if (nv <= 4) LONG(4); else LONG(8);
+#undef LONG
+}
+
+// bootstrap: S^l_v for every vertex
+void max_full(Ctx* c, int l) {
+    const int ld = c->ws[l];
+    int32_t* long_rows = c->Clist[0];
+    int* n_long = &c->ctl->work_counter[(l - 1) & 7];
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 16, 256, 0, c->ctl, l, 0, (const int32_t*)nullptr, (const int*)nullptr, c->N, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long)
+    RP_MAX_DISPATCH(ld, ROWS);
+#undef ROWS
+    launch_long_rows(c, 0, c->H[l - 1], ld, c->S[l], long_rows, n_long);
+}
+
+// hop l of a batch: messages, recomputation of the invalidated sinks, the list A_l
+void max_hop(Ctx* c, int l, int n) {
+    const int ld = c->ws[l];
+    const float* Old = c->D[(l - 1) & 1];            // previous values of the rows of A_{l-1}, in its order
+    const int32_t* senders = c->Clist[(l - 1) & 1];
+    const int T = 256;
+#define MSG(NV, LPR) RP_LAUNCH(c, (k_max_messages<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, senders, c->old_idx, c->coff, c->side[0], c->side[1], c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2)
+    if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
+    RP_MAX_DISPATCH(ld, MSG);
+#undef MSG
+    if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
+    if (n > 0)
+        RP_LAUNCH(c, k_max_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[1], c->posmap,
+                  c->old_idx, c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2);
+    // invalidated sinks -> list (the buffer of A_l serves until A_l itself is compacted), then their rows
+    int32_t* rlist = c->A[l];
+    int* n_r = &c->ctl->n_long[l];
+    bitmap_to_list_from(c, c->bitmap2, rlist, n_r, nullptr);
+    int32_t* long_rows = c->Clist[l & 1];            // the next hop's sender list is not built yet
+    int* n_long = &c->ctl->work_counter[(l - 1) & 7];
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, 1, rlist, n_r, 0, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long)
+    RP_MAX_DISPATCH(ld, ROWS);
+#undef ROWS
+    launch_long_rows(c, 1, c->H[l - 1], ld, c->S[l], long_rows, n_long);
+}
+
+// senders of hop l + 1 (l = 0: the vertices whose feature row really changed)
+void max_senders_build(Ctx* c, int l) {
+    int32_t* senders = c->Clist[l & 1];
+    RP_LAUNCH(c, k_max_senders, c->n_sm * 8, 256, 0, c->ctl, l, c->A[l], c->H[l], c->D[l & 1], c->ld[l], senders,
+              c->old_idx, c->posmap);
+    scan_degrees(c, senders, &c->ctl->nC[l], 0, c->side[0].deg, c->coff, &c->ctl->E[l + 1]);
+}
+
+void max_prepare() {
+    cudaFuncSetAttribute(k_max_long_rows<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 1024 * (int)sizeof(float));
+}
+
+}  // namespace rp

@@ -68,7 +68,7 @@ static void destroy_ctx(Ctx* c) {
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
         for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2, &c->layer[l].tc_self}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
-    cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->posmap); cudaFree(c->deg_out_old);
+    cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
@@ -101,7 +101,8 @@ static ripple_status run_full(Ctx* c) {
     RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
     if (c->timing) cudaEventRecord(c->ev[0], c->stream);
     for (int l = 1; l <= c->L; ++l) {
-        spmm_full(c, l);
+        if (c->agg == RIPPLE_AGG_MAX) max_full(c, l);
+        else spmm_full(c, l);
         self_project(c, l, true);
         update_rows(c, l, true);
     }
@@ -129,7 +130,11 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
     g_create_err[0] = 0;
     if (!g || !features || !layers || !out) { set_err(nullptr, "null argument"); return st; }
     if (L < 1 || L > RP_MAXL) { set_err(nullptr, "L must be in 1..%d", RP_MAXL); return st; }
-    if (agg < 0 || agg > 2) { set_err(nullptr, "unknown aggregator %d", agg); return st; }
+    if (agg < 0 || agg > 3) { set_err(nullptr, "unknown aggregator %d", agg); return st; }
+    if (agg == RIPPLE_AGG_MAX && layers[0].kind != RIPPLE_LAYER_GRAPHCONV) {
+        set_err(nullptr, "the max aggregator is built for layers without a self term (GRAPHCONV) only");
+        return st;
+    }
     if (g->num_vertices < 1 || g->num_vertices > 0x7fffffff - 64 || g->num_edges < 0 ||
         (g->num_edges > 0 && (!g->src || !g->dst))) {
         set_err(nullptr, "bad graph description");
@@ -175,6 +180,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         CK(cudaMallocHost(&c->params_host, 2 * sizeof(int)));
         c->no_graphs = o.no_graphs;
         tc_prepare();
+        max_prepare();
         CK(cudaMallocHost(&c->ctl_host, sizeof(Ctl)));
         memset(c->ctl_host, 0, sizeof(Ctl));
         c->n_words = (N + 31) / 32;
@@ -233,7 +239,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             {
                 // a layer narrower than its input transforms the few sender rows before the scatter
                 const int target = y.kind == RIPPLE_LAYER_GIN ? ly.ld_hid : ly.ld_out;
-                c->pre[l] = o.pre_transform == 0 && target < ly.ld_in;
+                c->pre[l] = o.pre_transform == 0 && target < ly.ld_in && agg != RIPPLE_AGG_MAX;   // a maximum does not commute with the matrix
                 c->ws[l] = c->pre[l] ? target : ly.ld_in;
                 // measured: a gathered row costs about half of a row delivered as a reduction
                 c->regather_threshold[l] = o.regather_threshold > 0.f ? o.regather_threshold
@@ -267,7 +273,8 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         for (int l = 0; l <= L; ++l) {
             max_ld = std::max(max_ld, c->ld[l]);
             CK(dev_alloc(&c->H[l], (size_t)N * c->ld[l], 0));
-            if (l > 0) { CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0)); CK(dev_alloc(&c->dS[l], (size_t)N * c->ws[l], 0));
+            if (l > 0) { CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0));
+                         if (agg != RIPPLE_AGG_MAX) CK(dev_alloc(&c->dS[l], (size_t)N * c->ws[l], 0));
                          if (c->layer[l].kind == RIPPLE_LAYER_SAGE) CK(dev_alloc(&c->Z[l], (size_t)N * c->ld[l], 0));
                          if (c->pre[l]) CK(dev_alloc(&c->P[l], (size_t)N * c->ws[l], 0)); }
             CK(dev_alloc(&c->A[l], (size_t)N + 32));
@@ -288,6 +295,10 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         // gather: at most 1.5 items per 1024 stored edges
         CK(dev_alloc(&c->coff, std::max((size_t)N + 2, (size_t)(c->side[1].col_size / 680) + 64), 0));
         CK(dev_alloc(&c->bitmap, (size_t)c->n_words + 256, 0));
+        if (agg == RIPPLE_AGG_MAX) {
+            CK(dev_alloc(&c->bitmap2, (size_t)c->n_words + 256, 0));
+            CK(dev_alloc(&c->old_idx, (size_t)N + 32));
+        }
         CK(dev_alloc(&c->posmap, (size_t)N, 0xFF));
         CK(dev_alloc(&c->deg_out_old, (size_t)N, 0xFF));
         CK(dev_alloc(&c->feat_last, (size_t)N, 0xFF));
@@ -335,10 +346,24 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
     graph_batch_mutate(c, nb);
     frontier_seed_features(c, nb);
     feature_rows(c, nb);
-    senders_build(c, 0, nb);
+    if (c->agg == RIPPLE_AGG_MAX) max_senders_build(c, 0);
+    else senders_build(c, 0, nb);
     STAMP();  // 1
+    if (c->agg == RIPPLE_AGG_MAX) {
+        // hybrid-incremental hops of a monotonic aggregator (Sec. 3.4.2)
+        for (int l = 1; l <= L; ++l) {
+            STAMP();
+            max_hop(c, l, nb);
+            frontier_compact(c, l);
+            senders_release(c, l - 1);
+            STAMP();
+            update_rows(c, l, false);
+            if (l < L) max_senders_build(c, l);
+            STAMP();
+        }
+    }
     // one superstep per hop (Sec. 3.3.1): frontier, send + aggregate, compute + prepare
-    for (int l = 1; l <= L; ++l) {
+    for (int l = 1; l <= L && c->agg != RIPPLE_AGG_MAX; ++l) {
         // The push scatter walks the same out-lists as the frontier and marks the sinks itself; the
         // gathering forms need the list A_l first, so the frontier walk is a pass of its own for them
         // (decided per hop on the device for the rebuilding form).

@@ -111,6 +111,8 @@ struct Ctx {
     float* H[RP_MAXL + 1];
     float* S[RP_MAXL + 1];
     float* Z[RP_MAXL + 1];    // cached self projection W_self^T h^{l-1} of SAGE layers (N x ld_l), else null
+    uint32_t* bitmap2;         // monotonic aggregation: sinks whose cached maximum must be recomputed
+    int32_t* old_idx;          // monotonic aggregation: sender -> index of its previous row among the rows of A_{l-1}
     float* P[RP_MAXL + 1];    // cached neighbour projection W_n^T h^{l-1} of layers that transform before the scatter (N x ws_l), else null
     float* dS[RP_MAXL + 1];   // per-batch message accumulator, zero outside a batch (same shape as S)
     float* T;          // GIN hidden rows (compact, N x ld_hid)
@@ -189,6 +191,12 @@ void senders_release(Ctx* c, int l);                    // clear posmap entries 
 
 // scatter.cu
 void spmm_full(Ctx* c, int l);                          // S^l for every vertex (bootstrap)
+void bitmap_to_list_from(Ctx* c, uint32_t* bitmap, int32_t* list, int* count_dev, unsigned long long* pull_work);
+// monotonic.cu (max aggregation, Sec. 3.4.2)
+void max_full(Ctx* c, int l);                           // bootstrap: cached maxima of every vertex
+void max_hop(Ctx* c, int l, int n);                     // messages <old, new>, recomputation of invalidated sinks
+void max_senders_build(Ctx* c, int l);                  // rows of A_l whose embedding changed, with their out-degree prefix
+void max_prepare();
 void choose_direction(Ctx* c, int l);                   // delta or rebuilding form of hop l (device-side decision)
 void scatter_layer(Ctx* c, int l, int n);               // delta messages of hop l into dS^l
 void regather_layer(Ctx* c, int l);                     // rebuilding form: S^l rows of A_l gathered anew

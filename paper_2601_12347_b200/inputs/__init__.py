@@ -403,6 +403,11 @@ def workloads() -> Dict[str, Workload]:
                               (10, 100, 1000), 20),
         "reddit-4l": Workload("reddit-4l", 232_965, 114_900_000, "rmat",
                               sage_model([602, 256, 256, 256, 41]), 0, (100, 1000), 20),
+        # GraphConv with max (the paper's GC-X workload, Sec. 6.1): hybrid-incremental propagation
+        "sparse-gcx": Workload("sparse-gcx", n_s, e_s, "rmat", graphconv_model([128, 256, 40], AGG_MAX), 0,
+                               (1, 10, 100, 1000), 100),
+        "dense-gcx-2l": Workload("dense-gcx-2l", n_d, e_d, "rmat", graphconv_model([100, 256, 47], AGG_MAX), 0,
+                                 (10, 100, 1000), 20),
         # hub stress: every endpoint is one of the top-1 % out-degree vertices of the initial graph
         "dense-3l-hub-feature": Workload("dense-3l-hub-feature", n_d, e_d, "rmat",
                                          sage_model([100, 256, 256, 47]), 0, (1, 10, 100, 1000), 20,
