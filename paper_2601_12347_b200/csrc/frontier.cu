@@ -265,9 +265,7 @@ void frontier_seed_features(Ctx* c, int n) {
 void frontier_mark(Ctx* c, int l, bool walk) {
     RP_LAUNCH(c, k_mark_frontier, walk ? c->n_sm * 8 : c->n_sm * 2, 256, 0, c->ctl, l, (int)c->self_term,
               (int)walk, c->Clist[(l - 1) & 1], c->coff, c->side[0], c->rec, c->A[l - 1], c->bitmap);
-    const bool may_rebuild = c->scatter_mode == RIPPLE_SCATTER_REGATHER ||
-                             (c->scatter_mode == RIPPLE_SCATTER_AUTO && c->regather_threshold[l] > 0.f);
-    if (!may_rebuild) return;
+    if (!c->rebuild_armed[l]) return;
     // the list A_l is not built yet: its buffer holds the queue of undecided long rows
     RP_LAUNCH(c, k_mark_bottom_up, c->n_sm * 8, 256, 0, c->ctl, l, c->N, c->side[1], c->posmap, c->bitmap, c->A[l],
               &c->ctl->n_long[l]);

@@ -83,6 +83,31 @@ __device__ __forceinline__ void fill(float4 (&acc)[NV], float x) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Invalidated elements.  A sink with thousands of in-neighbours is rarely invalidated in more than
+// a few of its elements (a changed neighbour is the maximiser of about d / deg_in of them), and
+// gathering whole rows for it would move hundreds of bytes per neighbour where a few suffice.  The
+// messages therefore record WHICH elements lost their maximiser (a bit mask per row); a row with
+// at most MAX_EL such elements re-reads only those, any other row is gathered in full.
+// ---------------------------------------------------------------------------------------------
+constexpr int MAX_EL = 16;
+
+// set elements of a row's mask -> ascending indices; returns their number, or -1 if there are more
+// than MAX_EL (or the whole row was flagged).  Same result in every thread.
+__device__ __forceinline__ int mask_elements(const uint32_t* __restrict__ mask, int mw, int ld, int (&el)[MAX_EL]) {
+    int cnt = 0;
+    for (int w = 0; w < mw; ++w) {
+        uint32_t bits = mask[w];
+        while (bits) {
+            const int e = (w << 5) + __ffs(bits) - 1;
+            bits &= bits - 1;
+            if (e >= ld || cnt == MAX_EL) return -1;
+            el[cnt++] = e;
+        }
+    }
+    return cnt;
+}
+
+// ---------------------------------------------------------------------------------------------
 // the maximum of one row over its whole in-list: a warp, or for long lists a block
 // ---------------------------------------------------------------------------------------------
 // mode 0 (bootstrap): rows = all vertices, the result is stored.
@@ -92,7 +117,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const int* n_dev, int n_host, Side in,
            const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA, int32_t* long_rows,
-           int* n_long) {
+           int* n_long, uint32_t* invmask, int mw) {
     if (ctl->abort) return;
     const int n = n_dev ? *n_dev : n_host;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -104,6 +129,40 @@ k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const in
         if (deg > MAX_HUB_DEGREE) {
             if (lane == 0) long_rows[atomicAdd(n_long, 1)] = v;
             continue;
+        }
+        if (mode) {   // few invalidated elements: re-read only those
+            uint32_t* mask = invmask + (size_t)v * mw;
+            int el[MAX_EL];
+            const int cnt = mask_elements(mask, mw, ld, el);
+            __syncwarp();
+            for (int w = lane; w < mw; w += 32) mask[w] = 0u;
+            if (cnt >= 0 && deg > 0) {
+                float acc[MAX_EL];
+#pragma unroll
+                for (int t = 0; t < MAX_EL; ++t) acc[t] = neg_inf();
+                const int64_t base = in.start[v];
+                for (int j = lane; j < deg; j += 32) {
+                    const float* row = M + (size_t)in.col[base + j] * ld;
+#pragma unroll
+                    for (int t = 0; t < MAX_EL; ++t)
+                        if (t < cnt) acc[t] = fmaxf(acc[t], __ldg(row + el[t]));
+                }
+                bool differs = false;
+#pragma unroll
+                for (int t = 0; t < MAX_EL; ++t) {
+                    if (t < cnt) {
+                        float m = acc[t];
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o));
+                        if (lane == 0) {
+                            float* dst = S + (size_t)v * ld + el[t];
+                            if (*dst != m) { *dst = m; differs = true; }
+                        }
+                    }
+                }
+                if (lane == 0 && differs) mark_bit(bitmapA, v);
+                continue;
+            }
         }
         float4 acc[NV];
         fill<NV>(acc, deg > 0 ? neg_inf() : 0.f);
@@ -133,7 +192,8 @@ k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const in
 template <int NV>
 __global__ void __launch_bounds__(256)
 k_max_long_rows(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const int* __restrict__ n_long, Side in,
-                const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA) {
+                const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA, uint32_t* invmask,
+                int mw) {
     extern __shared__ float part[];   // 8 warps x ld floats
     __shared__ int s_differs;
     if (ctl->abort) return;
@@ -142,6 +202,44 @@ k_max_long_rows(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const
     for (int i = blockIdx.x; i < n; i += gridDim.x) {
         const int v = long_rows[i];
         const int deg = in.deg[v];
+        if (mode) {   // few invalidated elements: every thread strides over the in-list for those alone
+            uint32_t* mask = invmask + (size_t)v * mw;
+            int el[MAX_EL];
+            const int cnt = mask_elements(mask, mw, ld, el);
+            __syncthreads();
+            for (int w = threadIdx.x; w < mw; w += blockDim.x) mask[w] = 0u;
+            if (cnt >= 0) {
+                float acc[MAX_EL];
+#pragma unroll
+                for (int t = 0; t < MAX_EL; ++t) acc[t] = neg_inf();
+                const int64_t base = in.start[v];
+                for (int j = threadIdx.x; j < deg; j += blockDim.x) {
+                    const float* row = M + (size_t)in.col[base + j] * ld;
+#pragma unroll
+                    for (int t = 0; t < MAX_EL; ++t)
+                        if (t < cnt) acc[t] = fmaxf(acc[t], __ldg(row + el[t]));
+                }
+#pragma unroll
+                for (int t = 0; t < MAX_EL; ++t) {
+                    float m = acc[t];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o));
+                    if (lane == 0) part[warp * MAX_EL + t] = m;
+                }
+                if (threadIdx.x == 0) s_differs = 0;
+                __syncthreads();
+                if ((int)threadIdx.x < cnt) {
+                    float m = part[threadIdx.x];
+                    for (int w = 1; w < 8; ++w) m = fmaxf(m, part[w * MAX_EL + threadIdx.x]);
+                    float* dst = S + (size_t)v * ld + el[threadIdx.x];
+                    if (*dst != m) { *dst = m; s_differs = 1; }
+                }
+                __syncthreads();
+                if (threadIdx.x == 0 && s_differs) mark_bit(bitmapA, v);
+                __syncthreads();
+                continue;
+            }
+        }
         float4 acc[NV];
         fill<NV>(acc, neg_inf());
         for (int j0 = warp * 1024; j0 < deg; j0 += 8 * 1024)
@@ -183,7 +281,8 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32_t* __restrict__ old_idx,
                const int64_t* __restrict__ coff, Side out, Side in, const float* __restrict__ Hprev,
-               const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR) {
+               const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR,
+               uint32_t* invmask, int mw) {
     if (ctl->abort) return;
     const int nC = ctl->nC[l - 1];
     if (nC == 0) return;
@@ -217,8 +316,11 @@ k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32
                 const int v = live ? out.col[base + jj] : 0;
                 bool raise = false, invalid = false;
                 if (live) {
-                    if (deg_in_before(in, v) == 0) invalid = true;   // zeros cached: gather the real maximum
-                    else {
+                    uint32_t* mask = invmask + (size_t)v * mw;
+                    if (deg_in_before(in, v) == 0) {   // zeros cached: gather the real maximum, every element
+                        invalid = true;
+                        for (int w = ql; w < mw; w += LPR) atomicOr(&mask[w], 0xffffffffu);
+                    } else {
                         float* srow = S + (size_t)v * ld;
 #pragma unroll
                         for (int k = 0; k < NV; ++k) {
@@ -231,7 +333,11 @@ k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32
 #pragma unroll
                                 for (int t = 0; t < 4; ++t) {
                                     if (nn[t] > ss[t]) { atomic_max_f32(srow + 4 * q + t, nn[t]); raise = true; }
-                                    else if (oo[t] == ss[t] && nn[t] < oo[t]) invalid = true;
+                                    else if (oo[t] == ss[t] && nn[t] < oo[t]) {
+                                        invalid = true;
+                                        const int e_ = 4 * q + t;
+                                        atomicOr(&mask[e_ >> 5], 1u << (e_ & 31));
+                                    }
                                 }
                             }
                         }
@@ -253,7 +359,8 @@ k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32
 // edge records: <-, new> along an added edge, <old, -> along a deleted one; one warp per record
 __global__ void k_max_records(Ctl* ctl, const Rec* __restrict__ rec, Side in, const int32_t* __restrict__ posmap,
                               const int32_t* __restrict__ old_idx, const float* __restrict__ Hprev,
-                              const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR) {
+                              const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR,
+                              uint32_t* invmask, int mw) {
     if (ctl->abort) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -261,21 +368,27 @@ __global__ void k_max_records(Ctl* ctl, const Rec* __restrict__ rec, Side in, co
     for (int r = warp; r < n; r += nwarps) {
         const int u = rec[r].u, v = rec[r].v;
         float* srow = S + (size_t)v * ld;
-        bool raise = false, invalid = false;
+        uint32_t* mask = invmask + (size_t)v * mw;
+        bool raise = false, invalid = false, whole = false;
         if (rec[r].sign > 0) {
-            if (deg_in_before(in, v) == 0) invalid = true;
+            if (deg_in_before(in, v) == 0) whole = true;
             else
                 for (int k = lane; k < ld; k += 32) {
                     const float x = Hprev[(size_t)u * ld + k];
                     if (x > srow[k]) { atomic_max_f32(srow + k, x); raise = true; }
                 }
         } else {
-            if (in.deg[v] == 0) invalid = true;
+            if (in.deg[v] == 0) whole = true;
             else {
                 const int p = posmap[u];
                 const float* orow = p >= 0 ? Old + (size_t)old_idx[p] * ld : Hprev + (size_t)u * ld;
-                for (int k = lane; k < ld; k += 32) invalid |= orow[k] == srow[k];
+                for (int k = lane; k < ld; k += 32)
+                    if (orow[k] == srow[k]) { invalid = true; atomicOr(&mask[k >> 5], 1u << (k & 31)); }
             }
+        }
+        if (whole) {   // every element
+            invalid = true;
+            for (int w = lane; w < mw; w += 32) atomicOr(&mask[w], 0xffffffffu);
         }
         raise = __any_sync(FULL, raise);
         invalid = __any_sync(FULL, invalid);
@@ -321,8 +434,8 @@ __global__ void k_max_senders(Ctl* ctl, int l, const int32_t* __restrict__ A, co
 
 static void launch_long_rows(Ctx* c, int mode, const float* M, int ld, float* S, int32_t* long_rows, int* n_long) {
     const int nv = div_up(ld, 128);
-    const size_t smem = (size_t)8 * ld * sizeof(float);
-#define LONG(NV) RP_LAUNCH(c, k_max_long_rows<NV>, c->n_sm, 256, smem, c->ctl, mode, long_rows, n_long, c->side[1], M, ld, S, c->bitmap)
+    const size_t smem = (size_t)8 * std::max(ld, MAX_EL) * sizeof(float);
+#define LONG(NV) RP_LAUNCH(c, k_max_long_rows<NV>, c->n_sm, 256, smem, c->ctl, mode, long_rows, n_long, c->side[1], M, ld, S, c->bitmap, c->invmask, c->mw)
     if (nv <= 1) LONG(1); else if (nv <= 2) LONG(2); else if (nv <= 4) LONG(4); else LONG(8);
 #undef LONG
 }
@@ -332,7 +445,7 @@ void max_full(Ctx* c, int l) {
     const int ld = c->ws[l];
     int32_t* long_rows = c->Clist[0];
     int* n_long = &c->ctl->work_counter[(l - 1) & 7];
-#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 16, 256, 0, c->ctl, l, 0, (const int32_t*)nullptr, (const int*)nullptr, c->N, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long)
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 16, 256, 0, c->ctl, l, 0, (const int32_t*)nullptr, (const int*)nullptr, c->N, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw)
     RP_MAX_DISPATCH(ld, ROWS);
 #undef ROWS
     launch_long_rows(c, 0, c->H[l - 1], ld, c->S[l], long_rows, n_long);
@@ -344,21 +457,21 @@ void max_hop(Ctx* c, int l, int n) {
     const float* Old = c->D[(l - 1) & 1];            // previous values of the rows of A_{l-1}, in its order
     const int32_t* senders = c->Clist[(l - 1) & 1];
     const int T = 256;
-#define MSG(NV, LPR) RP_LAUNCH(c, (k_max_messages<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, senders, c->old_idx, c->coff, c->side[0], c->side[1], c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2)
+#define MSG(NV, LPR) RP_LAUNCH(c, (k_max_messages<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, senders, c->old_idx, c->coff, c->side[0], c->side[1], c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2, c->invmask, c->mw)
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
     RP_MAX_DISPATCH(ld, MSG);
 #undef MSG
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
     if (n > 0)
         RP_LAUNCH(c, k_max_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[1], c->posmap,
-                  c->old_idx, c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2);
+                  c->old_idx, c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2, c->invmask, c->mw);
     // invalidated sinks -> list (the buffer of A_l serves until A_l itself is compacted), then their rows
     int32_t* rlist = c->A[l];
     int* n_r = &c->ctl->n_long[l];
     bitmap_to_list_from(c, c->bitmap2, rlist, n_r, nullptr);
     int32_t* long_rows = c->Clist[l & 1];            // the next hop's sender list is not built yet
     int* n_long = &c->ctl->work_counter[(l - 1) & 7];
-#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, 1, rlist, n_r, 0, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long)
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, 1, rlist, n_r, 0, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw)
     RP_MAX_DISPATCH(ld, ROWS);
 #undef ROWS
     launch_long_rows(c, 1, c->H[l - 1], ld, c->S[l], long_rows, n_long);

@@ -68,7 +68,7 @@ static void destroy_ctx(Ctx* c) {
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
         for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2, &c->layer[l].tc_self}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
-    cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->posmap); cudaFree(c->deg_out_old);
+    cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->invmask); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
@@ -298,6 +298,8 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         if (agg == RIPPLE_AGG_MAX) {
             CK(dev_alloc(&c->bitmap2, (size_t)c->n_words + 256, 0));
             CK(dev_alloc(&c->old_idx, (size_t)N + 32));
+            c->mw = (max_ld + 31) / 32;
+            CK(dev_alloc(&c->invmask, (size_t)N * c->mw, 0));
         }
         CK(dev_alloc(&c->posmap, (size_t)N, 0xFF));
         CK(dev_alloc(&c->deg_out_old, (size_t)N, 0xFF));
@@ -389,11 +391,31 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
     return evi;
 }
 
+// The choice between pushing and rebuilding a hop is taken on the device, but the kernels of the
+// rebuilding form (bottom-up marking, gather) only need to be in the chain when the choice can
+// fall on them.  A hop is armed if the last batch brought it within a factor two of the threshold,
+// or if nothing comparable is known (first batch, much larger batch).  An unarmed hop pushes even
+// if it turns out saturated: slower for that one batch, never wrong, and armed for the next.
+static void arm_rebuild(Ctx* c, int nb) {
+    const bool no_history = c->batches_done == 0 || nb > 4 * std::max(c->last_nb, 1);
+    for (int l = 1; l <= c->L; ++l) {
+        bool armed = false;
+        if (c->agg == RIPPLE_AGG_MAX) armed = false;
+        else if (c->scatter_mode == RIPPLE_SCATTER_REGATHER) armed = true;
+        else if (c->scatter_mode == RIPPLE_SCATTER_AUTO && c->regather_threshold[l] > 0.f)
+            armed = no_history || (double)c->stats.active_edges[l] >=
+                                      0.5 * (double)c->regather_threshold[l] * (double)c->stats.num_edges;
+        c->rebuild_armed[l] = armed;
+    }
+}
+
 // Small batches are launch-bound (about fifty short kernels): their chain is captured once per
 // batch size into a CUDA graph and replayed.  Returns false if this batch must take the direct path.
 static bool launch_batch_graph(Ctx* c, int nb) {
     if (c->no_graphs || c->timing || nb < 1 || nb > RP_GRAPH_MAX_BATCH) return false;
-    const int key = 2 * nb + (c->may_expand ? 1 : 0);   // the captured chain differs with the expansion kernels
+    // the captured chain differs with the expansion kernels and with the hops whose rebuilding form is enqueued
+    int key = 2 * nb + (c->may_expand ? 1 : 0);
+    for (int l = 1; l <= c->L; ++l) key = 2 * key + (c->rebuild_armed[l] ? 1 : 0);
     int slot = -1;
     for (int i = 0; i < RP_GRAPH_SLOTS; ++i)
         if (c->graph_exec[i] && c->graph_n[i] == key) slot = i;
@@ -442,6 +464,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
         for (int i = 0; i < nb && !wide; ++i) wide = ups[i].op == RIPPLE_OP_DEL_VERTEX;
     const int ng = wide ? (int)c->max_batch : nb;
     c->may_expand = wide || mem != RIPPLE_MEM_HOST;
+    arm_rebuild(c, nb);
     const bool try_graph = !wide && !c->no_graphs && !c->timing && nb >= 1 && nb <= RP_GRAPH_MAX_BATCH;
     const cudaMemcpyKind kind = mem == RIPPLE_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
     // operations are always staged: generated edge deletions are appended behind them
@@ -478,6 +501,8 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
         }
         s.n_added = h.n_add; s.n_deleted = h.n_del; s.n_noop_add = h.n_noop_add; s.n_noop_del = h.n_noop_del;
         s.n_superseded = h.n_superseded; s.n_feature = h.n_feat;
+        c->batches_done++;
+        c->last_nb = nb;
         s.n_expanded = (int64_t)h.n_extra;
         s.num_edges += h.n_add - h.n_del;
         for (int l = 0; l <= L; ++l) {

@@ -102,6 +102,9 @@ struct Ctx {
     int64_t E0;
     int64_t max_batch;
     int scatter_mode, gemm_mode, timing;
+    int rebuild_armed[RP_MAXL + 1];   // per hop: the rebuilding form is enqueued for this batch (see arm_rebuild)
+    long long batches_done;
+    int last_nb;
     int may_expand;   // the batch being enqueued may hold vertex deletions (always assumed for device batches)
     float regather_threshold[RP_MAXL + 1];  // per hop: share of all edges from which the hop rebuilds its aggregates
     int n_sm;
@@ -112,6 +115,8 @@ struct Ctx {
     float* S[RP_MAXL + 1];
     float* Z[RP_MAXL + 1];    // cached self projection W_self^T h^{l-1} of SAGE layers (N x ld_l), else null
     uint32_t* bitmap2;         // monotonic aggregation: sinks whose cached maximum must be recomputed
+    uint32_t* invmask;         // monotonic aggregation: per vertex, mw words: elements whose maximiser was lost
+    int mw;
     int32_t* old_idx;          // monotonic aggregation: sender -> index of its previous row among the rows of A_{l-1}
     float* P[RP_MAXL + 1];    // cached neighbour projection W_n^T h^{l-1} of layers that transform before the scatter (N x ws_l), else null
     float* dS[RP_MAXL + 1];   // per-batch message accumulator, zero outside a batch (same shape as S)

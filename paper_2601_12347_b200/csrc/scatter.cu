@@ -526,7 +526,8 @@ void fold_deltas(Ctx* c, int l) {
 }
 
 void choose_direction(Ctx* c, int l) {
-    RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode, c->regather_threshold[l]);
+    RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode,
+              c->rebuild_armed[l] ? c->regather_threshold[l] : -1.f);
 }
 
 // delta form of hop l (does nothing on the device if the hop rebuilds)
@@ -577,8 +578,7 @@ void scatter_layer(Ctx* c, int l, int n) {
 
 // rebuilding form of hop l (does nothing on the device unless the hop rebuilds); needs the list A_l
 void regather_layer(Ctx* c, int l) {
-    if (c->scatter_mode != RIPPLE_SCATTER_AUTO && c->scatter_mode != RIPPLE_SCATTER_REGATHER) return;
-    if (c->scatter_mode == RIPPLE_SCATTER_AUTO && c->regather_threshold[l] <= 0.f) return;
+    if (!c->rebuild_armed[l]) return;
     const int ld = c->ws[l];
     const float* M = c->pre[l] ? c->P[l] : c->H[l - 1];   // P^l rows of the senders are already current
     const int grid = c->n_sm * 16, T = 256;
