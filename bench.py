@@ -351,7 +351,7 @@ def run_ours(args, rank, world, local_rank):
 def run_table(args):
     """One JSON line per (workload, batch size): latency percentiles over 100 consecutive batches
     through the C ABI from pinned host buffers, stage times, frontier sizes, the last hop's scatter
-    rate, and the oracle on a bounded sample of the same stream.  Feeds the table in the benchmark spec."""
+    rate, and the oracle on a bounded sample of the same stream."""
     import torch
     from paper_2601_12347_b200 import build as B
     from paper_2601_12347_b200 import ripple
@@ -361,7 +361,8 @@ def run_table(args):
     for name in args.table.split(","):
         w, src, dst, X, W = make_workload(name, args.seed)
         L = len(w.model.layers)
-        rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=16384, scatter_mode=args.scatter,
+        rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=w.extra.get("max_batch", 16384),
+                           scatter_mode=args.scatter,
                            regather_threshold=args.regather_threshold)
         boot = rp.stats()["ms_bootstrap"]
         rp.recompute_full()   # warm: the recompute-everything alternative on the same state

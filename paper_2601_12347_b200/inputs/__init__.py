@@ -245,6 +245,9 @@ class UpdateStream:
     With `hubs` given (an array of vertex ids), endpoints are restricted to hubs: additions join
     two hubs, a deletion removes a uniform current out-edge of a uniformly drawn hub, feature
     updates name hubs.
+
+    A fourth entry in `mix` is the share of vertex deletions (a uniform vertex; every edge at it
+    goes, its feature row becomes zeros; the id may be named again by later updates).
     """
 
     def __init__(self, n: int, src: np.ndarray, dst: np.ndarray, d0: int, seed: int,
@@ -261,6 +264,9 @@ class UpdateStream:
         self.added_pos: Dict[int, int] = {}
         self.hubs = None if hubs is None else np.asarray(hubs, dtype=np.int64)
         self.n_edges = self.e0
+        self.init_in_keys = None
+        if self.mix.size > 3 and self.mix[3] > 0:   # in-edge index, only needed to delete vertices
+            self.init_in_keys = np.sort(dst.astype(np.int64) * self.n + src.astype(np.int64))
 
     # -- membership ---------------------------------------------------------------------
     def _in_init(self, key: int) -> bool:
@@ -285,6 +291,17 @@ class UpdateStream:
                     self.added[i] = last
                     self.added_pos[last] = i
         self.n_edges += 1 if present else -1
+
+    def _remove_vertex(self, w: int) -> None:
+        n = self.n
+        lo, hi = np.searchsorted(self.init_keys, [w * n, (w + 1) * n])
+        keys = [int(k) for k in self.init_keys[lo:hi]]
+        lo, hi = np.searchsorted(self.init_in_keys, [w * n, (w + 1) * n])
+        keys += [int(k % n) * n + w for k in self.init_in_keys[lo:hi]]
+        keys += [k for k in self.added if k // n == w or k % n == w]
+        for key in set(keys):
+            if self._present(key):
+                self._set(key, False)
 
     # -- draws --------------------------------------------------------------------------
     def _draw_vertex(self) -> int:
@@ -319,7 +336,7 @@ class UpdateStream:
 
     def next_batch(self, b: int) -> Tuple[np.ndarray, np.ndarray]:
         """Returns (updates[b] of UPDATE_DTYPE, feature_rows[n_feat, d0] fp32)."""
-        kinds = self.rng.choice(3, size=b, p=self.mix)
+        kinds = self.rng.choice(self.mix.size, size=b, p=self.mix)
         ups = np.zeros(b, dtype=UPDATE_DTYPE)
         rows: List[np.ndarray] = []
         in_batch = set()
@@ -331,7 +348,9 @@ class UpdateStream:
                     k = OP_ADD_EDGE
             if k == OP_ADD_EDGE:
                 key = self._draw_add(in_batch)
-            if k == OP_SET_FEATURE:
+            if k == OP_DEL_VERTEX:
+                ups[i] = (OP_DEL_VERTEX, self._draw_vertex(), 0)
+            elif k == OP_SET_FEATURE:
                 while True:
                     v = self._draw_vertex()
                     if v not in feat_seen:
@@ -342,9 +361,14 @@ class UpdateStream:
             else:
                 in_batch.add(key)
                 ups[i] = (k, key // self.n, key % self.n)
+        # the stream's own record of the graph, operation by operation
         for rec in ups:
-            if rec["op"] != OP_SET_FEATURE:
-                self._set(int(rec["u"]) * self.n + int(rec["v"]), rec["op"] == OP_ADD_EDGE)
+            if rec["op"] == OP_DEL_VERTEX:
+                self._remove_vertex(int(rec["u"]))
+            elif rec["op"] != OP_SET_FEATURE:
+                key, want = int(rec["u"]) * self.n + int(rec["v"]), rec["op"] == OP_ADD_EDGE
+                if self._present(key) != want:
+                    self._set(key, bool(want))
         feat = np.stack(rows) if rows else np.zeros((0, self.d0), dtype=np.float32)
         return ups, np.ascontiguousarray(feat, dtype=np.float32)
 
@@ -408,6 +432,9 @@ def workloads() -> Dict[str, Workload]:
                                (1, 10, 100, 1000), 100),
         "dense-gcx-2l": Workload("dense-gcx-2l", n_d, e_d, "rmat", graphconv_model([100, 256, 47], AGG_MAX), 0,
                                  (10, 100, 1000), 20),
+        # all five update types of Sec. 3.1: 2 % of the updates delete a vertex
+        "sparse-vdel": Workload("sparse-vdel", n_s, e_s, "rmat", sage_model([128, 256, 40]), 0, (100, 1000), 100,
+                                {"mix": (0.39, 0.39, 0.2, 0.02), "max_batch": 65536}),
         # hub stress: every endpoint is one of the top-1 % out-degree vertices of the initial graph
         "dense-3l-hub-feature": Workload("dense-3l-hub-feature", n_d, e_d, "rmat",
                                          sage_model([100, 256, 256, 47]), 0, (1, 10, 100, 1000), 20,

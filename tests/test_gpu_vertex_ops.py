@@ -143,3 +143,32 @@ def test_expansion_beyond_the_batch_capacity_is_rejected(env):
     assert ei.value.status == ripple.ERR_VERTEX_RANGE
     G.check_graph(rp, orc)
     rp.close()
+
+
+@pytest.mark.parametrize("batch", [100, 1000])
+def test_all_five_update_types_100_consecutive_batches(env, batch):
+    """The sparse workload with 2 % vertex deletions in the stream (Sec. 3.1: five update types)."""
+    ripple, Oracle = env
+    w = I.workloads()["sparse-vdel"]
+    src, dst = I.make_graph(w)
+    X = I.features(w.n, w.model.dims[0], w.seed)
+    W = I.make_weights(w.model, w.seed)
+    L = len(w.model.layers)
+    rp = ripple.Ripple(w.n, src, dst, X, w.model, W, max_batch=w.extra["max_batch"])
+    orc = Oracle(w.n, src, dst, X, w.model, W)
+    stream = I.make_stream(w, src, dst)
+    expanded = 0
+    for b in range(100):
+        ups, rows = stream.next_batch(batch)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        G.check_frontiers(rp, orc, L)
+        expanded += rp.stats()["n_expanded"]
+        if b % 25 == 24:
+            G.check_graph(rp, orc)
+            G.check_values(rp, [orc.H(l) for l in range(L + 1)], L)
+    assert expanded > 0
+    G.check_graph(rp, orc)
+    G.check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+    assert rp.stats()["num_edges"] == stream.n_edges
+    rp.close()

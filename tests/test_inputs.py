@@ -78,3 +78,28 @@ def test_hub_stream_only_touches_hubs():
         assert int(r["u"]) in hs
         if r["op"] == I.OP_ADD_EDGE:
             assert int(r["v"]) in hs
+
+
+def test_stream_with_vertex_deletions_keeps_a_consistent_record():
+    """The four-type stream's own record of the graph equals a literal replay of its batches."""
+    n = 300
+    src, dst = I.er_graph(n, 3000, 1)
+    st = I.UpdateStream(n, src, dst, 4, 1, mix=(0.35, 0.35, 0.2, 0.1))
+    E = set(zip(src.tolist(), dst.tolist()))
+    seen = 0
+    for _ in range(20):
+        ups, rows = st.next_batch(40)
+        for r in ups:
+            op, u, v = int(r["op"]), int(r["u"]), int(r["v"])
+            if op == I.OP_ADD_EDGE:
+                E.add((u, v))
+            elif op == I.OP_DEL_EDGE:
+                E.discard((u, v))
+            elif op == I.OP_DEL_VERTEX:
+                E = {p for p in E if u not in p}
+                seen += 1
+        cur = {(int(k) // n, int(k) % n) for k in st.init_keys if st._present(int(k))}
+        cur |= {(k // n, k % n) for k in st.added}
+        assert cur == E and st.n_edges == len(E)
+        assert rows.shape[0] == int((ups["op"] == I.OP_SET_FEATURE).sum())
+    assert seen > 0
