@@ -50,13 +50,15 @@ typedef enum { RIPPLE_MEM_HOST = 0, RIPPLE_MEM_DEVICE = 1 } ripple_mem;
 
 /* Aggregators of Table 1.  WSUM_GCN is the weighted sum with alpha_uv = 1/sqrt(deg_out(u) deg_in(v))
  * taken from the current graph and recomputed whenever a degree changes.
- * MAX (Sec. 3.4.2, monotonic aggregation): element-wise maximum over the in-neighbours, zeros for a
- * vertex without in-neighbours; GRAPHCONV layers only.  Its batches run hybrid-incrementally:
+ * MAX, MIN (Sec. 3.4.2, monotonic aggregation): element-wise maximum / minimum over the in-neighbours,
+ * zeros for a vertex without in-neighbours; GRAPHCONV layers only.  Its batches run hybrid-incrementally:
  * a message carries the sender's old and new row, a sink raises its cached maximum, recomputes it
  * over all in-neighbours, or ignores the message; a sink whose cached maximum did not change is
  * not affected and propagates nothing (ripple_get_affected then lists exactly the vertices whose
  * cached maximum changed; ripple_stats.senders those whose embedding changed). */
-typedef enum { RIPPLE_AGG_SUM = 0, RIPPLE_AGG_MEAN = 1, RIPPLE_AGG_WSUM_GCN = 2, RIPPLE_AGG_MAX = 3 } ripple_agg;
+typedef enum {
+    RIPPLE_AGG_SUM = 0, RIPPLE_AGG_MEAN = 1, RIPPLE_AGG_WSUM_GCN = 2, RIPPLE_AGG_MAX = 3, RIPPLE_AGG_MIN = 4
+} ripple_agg;
 
 /* Update functions (Eq. 2) of the model families of Sec. 6.1.1, x_v = normalised aggregate:
  *   SAGE       h = act(Wa^T h_v + Wb^T x_v + ba)                         (self term)
@@ -138,7 +140,8 @@ typedef struct {
     int32_t device;       /* CUDA device ordinal, or -1 for the current device                              */
     void* stream;         /* cudaStream_t to run on (NULL: the library creates its own)                     */
     float regather_threshold; /* AUTO only: a hop rebuilds its aggregates once its messages number at least
-                             this share of all edges.  0: default (0.7); < 0: never                       */
+                             this share of all edges.  0: default (0.6 for aggregate rows of 128 floats
+                             or more, else 0.7); < 0: never                       */
 } ripple_options;
 
 typedef struct {

@@ -43,7 +43,8 @@
 #include <string.h>
 
 enum { KIND_SAGE = 0, KIND_GRAPHCONV = 1, KIND_GIN = 2 };
-enum { AGG_SUM = 0, AGG_MEAN = 1, AGG_WSUM_GCN = 2, AGG_MAX = 3 };
+enum { AGG_SUM = 0, AGG_MEAN = 1, AGG_WSUM_GCN = 2, AGG_MAX = 3, AGG_MIN = 4 };
+#define MONOTONIC(agg) ((agg) == AGG_MAX || (agg) == AGG_MIN)
 enum { ACT_IDENTITY = 0, ACT_RELU = 1 };
 enum { OP_ADD_EDGE = 0, OP_DEL_EDGE = 1, OP_SET_FEATURE = 2, OP_DEL_VERTEX = 3 };
 
@@ -116,7 +117,7 @@ static double coef_src(const oracle_t *o, int deg_out) {
 
 /* Sink-side normalisation applied to S_v at compute time (Table 1: mean, weighted sum). */
 static double norm_sink(const oracle_t *o, int deg_in) {
-    if (o->agg == AGG_SUM || o->agg == AGG_MAX) return 1.0;
+    if (o->agg == AGG_SUM || MONOTONIC(o->agg)) return 1.0;
     if (deg_in <= 0) return 0.0;
     return o->agg == AGG_MEAN ? 1.0 / (double)deg_in : 1.0 / sqrt((double)deg_in);
 }
@@ -164,10 +165,12 @@ static void layer_row(const layer_t *ly, const double *hprev, const double *Srow
 static void aggregate_row(const oracle_t *o, int v, const double *Hprev, int K, double *Srow) {
     for (int k = 0; k < K; ++k) Srow[k] = 0.0;
     const ivec *in = &o->in[v];
-    if (o->agg == AGG_MAX) { /* element-wise maximum over the in-neighbours; no in-neighbour: zeros */
+    if (MONOTONIC(o->agg)) { /* element-wise maximum (minimum) over the in-neighbours; none: zeros */
+        int is_min = o->agg == AGG_MIN;
         for (int i = 0; i < in->n; ++i) {
             const double *h = Hprev + (size_t)in->a[i] * K;
-            for (int k = 0; k < K; ++k) if (i == 0 || h[k] > Srow[k]) Srow[k] = h[k];
+            for (int k = 0; k < K; ++k)
+                if (i == 0 || (is_min ? h[k] < Srow[k] : h[k] > Srow[k])) Srow[k] = h[k];
         }
         return;
     }
@@ -509,7 +512,8 @@ static const srcinfo_t *source_find(const srcinfo_t *t, int n, int u) {
 /* O-inc: incremental propagation of one batch (Sec. 3.3).  Returns 0, or <0 if the batch is
  * rejected (nothing changed). */
 /* ------------------------------------------------------------------------------------------ */
-/* Monotonic aggregation (Sec. 3.4.2), max, for models without a self term (GraphConv).  A message
+/* Monotonic aggregation (Sec. 3.4.2), max (min is its mirror image: read "exceeds" as "is below"
+ * and so on), for models without a self term (GraphConv).  A message
  * <old, new> from a changed in-neighbour, <-, new> along an added edge or <old, -> along a deleted
  * one leads, per element, to one of three actions at the sink:
  *   - new exceeds the cached maximum: the cache is raised to it (incremental);
@@ -527,6 +531,8 @@ static int differs_f32(const double *a, const double *b, int n) {
 static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *feat_rows) {
     int L = o->L, N = o->N;
     int d0 = o->d[0];
+    int is_min = o->agg == AGG_MIN;
+#define BEATS(a, b) (is_min ? (a) < (b) : (a) > (b))   /* a improves on b */
     /* in-degree before the batch: a sink that had no in-neighbour caches zeros, not a maximum */
     int *din_old = (int *)malloc(sizeof(int) * (size_t)N);
     for (int v = 0; v < N; ++v) din_old[v] = o->in[v].n;
@@ -585,8 +591,8 @@ static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *fe
                 if (dl->n_add && bsearch(&p, dl->add, (size_t)dl->n_add, sizeof(pair_t), cmp_pair)) continue;
                 double *Sv = S + (size_t)v * K;
                 for (int k = 0; k < K; ++k) {
-                    if (hnew[k] > Sv[k]) { TOUCH(v); Sv[k] = hnew[k]; }
-                    else if (hold[k] == Sv[k] && hnew[k] < hold[k]) need[v] = 1;
+                    if (BEATS(hnew[k], Sv[k])) { TOUCH(v); Sv[k] = hnew[k]; }
+                    else if (hold[k] == Sv[k] && BEATS(hold[k], hnew[k])) need[v] = 1;
                 }
             }
         }
@@ -596,7 +602,7 @@ static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *fe
             if (din_old[v] == 0) { need[v] = 1; continue; }
             const double *hnew = Hp + (size_t)u * K;
             double *Sv = S + (size_t)v * K;
-            for (int k = 0; k < K; ++k) if (hnew[k] > Sv[k]) { TOUCH(v); Sv[k] = hnew[k]; }
+            for (int k = 0; k < K; ++k) if (BEATS(hnew[k], Sv[k])) { TOUCH(v); Sv[k] = hnew[k]; }
         }
         /* <old, -> along deleted edges */
         for (int i = 0; i < dl->n_del; ++i) {
@@ -639,6 +645,7 @@ static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *fe
         free(A); free(oldA);
         A = An; nA = nAn; oldA = oldAn;
     }
+#undef BEATS
     free(A); free(oldA); free(din_old); free(snap_of); free(need);
     return 0;
 }
@@ -650,7 +657,7 @@ int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const flo
     if (rc) return rc;
     int L = o->L, self_term = o->layer[1].kind != KIND_GRAPHCONV;
 
-    if (o->agg == AGG_MAX) {
+    if (MONOTONIC(o->agg)) {
         if (self_term) { delta_free(&dl); return -3; }   /* built for models without a self term only */
         apply_topology(o, &dl);
         rc = apply_incremental_max(o, &dl, feat_rows);

@@ -193,7 +193,7 @@ void update_rows(Ctx* c, int l, bool full) {
         if (!full) { p.addend_rw = c->S[l]; p.addend_delta = c->dS[l]; }   // fold_deltas is skipped for these layers
     }
     float* dout = (full || l == c->L) ? nullptr : c->D[l & 1];  // the last hop sends nothing
-    p.dout_old = c->agg == RIPPLE_AGG_MAX;
+    p.dout_old = rp_monotonic(c->agg);
     if (ly.kind == RIPPLE_LAYER_GIN) {
         // hidden = relu(W1^T ((1 + eps) h + x) + b1), kept as compact rows
         p.a_mode = pre ? A_SELF : A_SUM; p.epi_mode = EPI_TEMP; p.alpha = 1.0f + ly.eps;
@@ -256,7 +256,7 @@ void feature_rows(Ctx* c, int n) {
     if (n <= 0) return;
     RP_LAUNCH(c, k_feature_rows, std::min(div_up(n, 8), c->n_sm * 8), 256, 0, c->ctl, c->ups_dev, c->feat_dev,
               c->d[0], c->A[0], c->feat_last, (int)c->src_norm, c->side[0].deg, c->deg_out_old, c->H[0],
-              c->ld[0], c->D[0], (int)(c->agg == RIPPLE_AGG_MAX));
+              c->ld[0], c->D[0], (int)(rp_monotonic(c->agg)));
 }
 
 // ---------------------------------------------------------------------------------------------

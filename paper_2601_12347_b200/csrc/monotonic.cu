@@ -20,13 +20,22 @@ namespace rp {
 constexpr int MAX_HUB_DEGREE = 4096;   // longer in-lists are recomputed by a whole block
 constexpr int MAX_CHUNK = 64;          // edges per warp work item of the message walk
 
-__device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
+// The same code serves min: every comparison goes through these helpers (is_min = 0: maximum).
+// worst() is the value every real one improves on.
+__device__ __forceinline__ float worst(int is_min) { return __int_as_float(is_min ? 0x7f800000 : 0xff800000); }
+__device__ __forceinline__ float pick(float a, float b, int is_min) { return is_min ? fminf(a, b) : fmaxf(a, b); }
+__device__ __forceinline__ bool beats(float a, float b, int is_min) { return is_min ? a < b : a > b; }
 
-// atomic maximum of an IEEE float: non-negative values order like signed integers, negative ones
-// like unsigned integers in reverse
-__device__ __forceinline__ void atomic_max_f32(float* addr, float val) {
-    if (val >= 0.f) atomicMax(reinterpret_cast<int*>(addr), __float_as_int(val));
-    else atomicMin(reinterpret_cast<unsigned int*>(addr), __float_as_uint(val));
+// atomic maximum / minimum of an IEEE float: non-negative values order like signed integers,
+// negative ones like unsigned integers in reverse
+__device__ __forceinline__ void atomic_pick_f32(float* addr, float val, int is_min) {
+    if (!is_min) {
+        if (val >= 0.f) atomicMax(reinterpret_cast<int*>(addr), __float_as_int(val));
+        else atomicMin(reinterpret_cast<unsigned int*>(addr), __float_as_uint(val));
+    } else {
+        if (val >= 0.f) atomicMin(reinterpret_cast<int*>(addr), __float_as_int(val));
+        else atomicMax(reinterpret_cast<unsigned int*>(addr), __float_as_uint(val));
+    }
 }
 
 __device__ __forceinline__ void mark_bit(uint32_t* bitmap, int v) {
@@ -34,8 +43,8 @@ __device__ __forceinline__ void mark_bit(uint32_t* bitmap, int v) {
     if (!(bitmap[v >> 5] & m)) atomicOr(&bitmap[v >> 5], m);
 }
 
-__device__ __forceinline__ float4 max4(const float4& a, const float4& b) {
-    return make_float4(fmaxf(a.x, b.x), fmaxf(a.y, b.y), fmaxf(a.z, b.z), fmaxf(a.w, b.w));
+__device__ __forceinline__ float4 pick4(const float4& a, const float4& b, int is_min) {
+    return make_float4(pick(a.x, b.x, is_min), pick(a.y, b.y, is_min), pick(a.z, b.z, is_min), pick(a.w, b.w, is_min));
 }
 
 // acc = max(acc, rows of the in-neighbours [j_begin, j_end) of v); LPR lanes hold one row (NV float4
@@ -43,7 +52,7 @@ __device__ __forceinline__ float4 max4(const float4& a, const float4& b) {
 // maximum over all groups
 template <int NV, int LPR>
 __device__ __forceinline__ void max_accumulate(float4 (&acc)[NV], const Side& in, int v, int j_begin, int j_end,
-                                               const float* __restrict__ M, int ld) {
+                                               const float* __restrict__ M, int ld, int is_min) {
     const int lane = lane_id(), nq = ld >> 2;
     constexpr int EPI = 32 / LPR;
     const int sub = lane / LPR, ql = lane % LPR;
@@ -59,7 +68,7 @@ __device__ __forceinline__ void max_accumulate(float4 (&acc)[NV], const Side& in
 #pragma unroll
                 for (int k = 0; k < NV; ++k) {
                     const int q = ql + LPR * k;
-                    if (q < nq) acc[k] = max4(acc[k], __ldg(row + q));
+                    if (q < nq) acc[k] = pick4(acc[k], __ldg(row + q), is_min);
                 }
             }
         }
@@ -68,10 +77,10 @@ __device__ __forceinline__ void max_accumulate(float4 (&acc)[NV], const Side& in
     for (int k = 0; k < NV; ++k) {
 #pragma unroll
         for (int o = LPR; o < 32; o <<= 1) {
-            acc[k].x = fmaxf(acc[k].x, __shfl_xor_sync(FULL, acc[k].x, o));
-            acc[k].y = fmaxf(acc[k].y, __shfl_xor_sync(FULL, acc[k].y, o));
-            acc[k].z = fmaxf(acc[k].z, __shfl_xor_sync(FULL, acc[k].z, o));
-            acc[k].w = fmaxf(acc[k].w, __shfl_xor_sync(FULL, acc[k].w, o));
+            acc[k].x = pick(acc[k].x, __shfl_xor_sync(FULL, acc[k].x, o), is_min);
+            acc[k].y = pick(acc[k].y, __shfl_xor_sync(FULL, acc[k].y, o), is_min);
+            acc[k].z = pick(acc[k].z, __shfl_xor_sync(FULL, acc[k].z, o), is_min);
+            acc[k].w = pick(acc[k].w, __shfl_xor_sync(FULL, acc[k].w, o), is_min);
         }
     }
 }
@@ -117,7 +126,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const int* n_dev, int n_host, Side in,
            const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA, int32_t* long_rows,
-           int* n_long, uint32_t* invmask, int mw) {
+           int* n_long, uint32_t* invmask, int mw, int is_min) {
     if (ctl->abort) return;
     const int n = n_dev ? *n_dev : n_host;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -139,13 +148,13 @@ k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const in
             if (cnt >= 0 && deg > 0) {
                 float acc[MAX_EL];
 #pragma unroll
-                for (int t = 0; t < MAX_EL; ++t) acc[t] = neg_inf();
+                for (int t = 0; t < MAX_EL; ++t) acc[t] = worst(is_min);
                 const int64_t base = in.start[v];
                 for (int j = lane; j < deg; j += 32) {
                     const float* row = M + (size_t)in.col[base + j] * ld;
 #pragma unroll
                     for (int t = 0; t < MAX_EL; ++t)
-                        if (t < cnt) acc[t] = fmaxf(acc[t], __ldg(row + el[t]));
+                        if (t < cnt) acc[t] = pick(acc[t], __ldg(row + el[t]), is_min);
                 }
                 bool differs = false;
 #pragma unroll
@@ -153,7 +162,7 @@ k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const in
                     if (t < cnt) {
                         float m = acc[t];
 #pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o));
+                        for (int o = 16; o > 0; o >>= 1) m = pick(m, __shfl_xor_sync(FULL, m, o), is_min);
                         if (lane == 0) {
                             float* dst = S + (size_t)v * ld + el[t];
                             if (*dst != m) { *dst = m; differs = true; }
@@ -165,8 +174,8 @@ k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const in
             }
         }
         float4 acc[NV];
-        fill<NV>(acc, deg > 0 ? neg_inf() : 0.f);
-        max_accumulate<NV, LPR>(acc, in, v, 0, deg, M, ld);
+        fill<NV>(acc, deg > 0 ? worst(is_min) : 0.f);
+        max_accumulate<NV, LPR>(acc, in, v, 0, deg, M, ld, is_min);
         float4* dst = reinterpret_cast<float4*>(S + (size_t)v * ld);
         bool differs = false;
         if (sub == 0) {
@@ -193,7 +202,7 @@ template <int NV>
 __global__ void __launch_bounds__(256)
 k_max_long_rows(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const int* __restrict__ n_long, Side in,
                 const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA, uint32_t* invmask,
-                int mw) {
+                int mw, int is_min) {
     extern __shared__ float part[];   // 8 warps x ld floats
     __shared__ int s_differs;
     if (ctl->abort) return;
@@ -211,26 +220,26 @@ k_max_long_rows(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const
             if (cnt >= 0) {
                 float acc[MAX_EL];
 #pragma unroll
-                for (int t = 0; t < MAX_EL; ++t) acc[t] = neg_inf();
+                for (int t = 0; t < MAX_EL; ++t) acc[t] = worst(is_min);
                 const int64_t base = in.start[v];
                 for (int j = threadIdx.x; j < deg; j += blockDim.x) {
                     const float* row = M + (size_t)in.col[base + j] * ld;
 #pragma unroll
                     for (int t = 0; t < MAX_EL; ++t)
-                        if (t < cnt) acc[t] = fmaxf(acc[t], __ldg(row + el[t]));
+                        if (t < cnt) acc[t] = pick(acc[t], __ldg(row + el[t]), is_min);
                 }
 #pragma unroll
                 for (int t = 0; t < MAX_EL; ++t) {
                     float m = acc[t];
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o));
+                    for (int o = 16; o > 0; o >>= 1) m = pick(m, __shfl_xor_sync(FULL, m, o), is_min);
                     if (lane == 0) part[warp * MAX_EL + t] = m;
                 }
                 if (threadIdx.x == 0) s_differs = 0;
                 __syncthreads();
                 if ((int)threadIdx.x < cnt) {
                     float m = part[threadIdx.x];
-                    for (int w = 1; w < 8; ++w) m = fmaxf(m, part[w * MAX_EL + threadIdx.x]);
+                    for (int w = 1; w < 8; ++w) m = pick(m, part[w * MAX_EL + threadIdx.x], is_min);
                     float* dst = S + (size_t)v * ld + el[threadIdx.x];
                     if (*dst != m) { *dst = m; s_differs = 1; }
                 }
@@ -241,9 +250,9 @@ k_max_long_rows(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const
             }
         }
         float4 acc[NV];
-        fill<NV>(acc, neg_inf());
+        fill<NV>(acc, worst(is_min));
         for (int j0 = warp * 1024; j0 < deg; j0 += 8 * 1024)
-            max_accumulate<NV, 32>(acc, in, v, j0, min(deg, j0 + 1024), M, ld);
+            max_accumulate<NV, 32>(acc, in, v, j0, min(deg, j0 + 1024), M, ld, is_min);
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             const int q = lane + 32 * k;
@@ -254,7 +263,7 @@ k_max_long_rows(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const
         bool differs = false;
         for (int q = threadIdx.x; q < nq; q += blockDim.x) {
             float4 m = reinterpret_cast<const float4*>(part)[q];
-            for (int w = 1; w < 8; ++w) m = max4(m, reinterpret_cast<const float4*>(part + (size_t)w * ld)[q]);
+            for (int w = 1; w < 8; ++w) m = pick4(m, reinterpret_cast<const float4*>(part + (size_t)w * ld)[q], is_min);
             float4* dst = reinterpret_cast<float4*>(S + (size_t)v * ld) + q;
             if (mode) {
                 const float4 o = *dst;
@@ -282,7 +291,7 @@ __global__ void __launch_bounds__(256)
 k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32_t* __restrict__ old_idx,
                const int64_t* __restrict__ coff, Side out, Side in, const float* __restrict__ Hprev,
                const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR,
-               uint32_t* invmask, int mw) {
+               uint32_t* invmask, int mw, int is_min) {
     if (ctl->abort) return;
     const int nC = ctl->nC[l - 1];
     if (nC == 0) return;
@@ -332,8 +341,8 @@ k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32
                                 const float ss[4] = {s.x, s.y, s.z, s.w};
 #pragma unroll
                                 for (int t = 0; t < 4; ++t) {
-                                    if (nn[t] > ss[t]) { atomic_max_f32(srow + 4 * q + t, nn[t]); raise = true; }
-                                    else if (oo[t] == ss[t] && nn[t] < oo[t]) {
+                                    if (beats(nn[t], ss[t], is_min)) { atomic_pick_f32(srow + 4 * q + t, nn[t], is_min); raise = true; }
+                                    else if (oo[t] == ss[t] && beats(oo[t], nn[t], is_min)) {
                                         invalid = true;
                                         const int e_ = 4 * q + t;
                                         atomicOr(&mask[e_ >> 5], 1u << (e_ & 31));
@@ -360,7 +369,7 @@ k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32
 __global__ void k_max_records(Ctl* ctl, const Rec* __restrict__ rec, Side in, const int32_t* __restrict__ posmap,
                               const int32_t* __restrict__ old_idx, const float* __restrict__ Hprev,
                               const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR,
-                              uint32_t* invmask, int mw) {
+                              uint32_t* invmask, int mw, int is_min) {
     if (ctl->abort) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -375,7 +384,7 @@ __global__ void k_max_records(Ctl* ctl, const Rec* __restrict__ rec, Side in, co
             else
                 for (int k = lane; k < ld; k += 32) {
                     const float x = Hprev[(size_t)u * ld + k];
-                    if (x > srow[k]) { atomic_max_f32(srow + k, x); raise = true; }
+                    if (beats(x, srow[k], is_min)) { atomic_pick_f32(srow + k, x, is_min); raise = true; }
                 }
         } else {
             if (in.deg[v] == 0) whole = true;
@@ -435,7 +444,7 @@ __global__ void k_max_senders(Ctl* ctl, int l, const int32_t* __restrict__ A, co
 static void launch_long_rows(Ctx* c, int mode, const float* M, int ld, float* S, int32_t* long_rows, int* n_long) {
     const int nv = div_up(ld, 128);
     const size_t smem = (size_t)8 * std::max(ld, MAX_EL) * sizeof(float);
-#define LONG(NV) RP_LAUNCH(c, k_max_long_rows<NV>, c->n_sm, 256, smem, c->ctl, mode, long_rows, n_long, c->side[1], M, ld, S, c->bitmap, c->invmask, c->mw)
+#define LONG(NV) RP_LAUNCH(c, k_max_long_rows<NV>, c->n_sm, 256, smem, c->ctl, mode, long_rows, n_long, c->side[1], M, ld, S, c->bitmap, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
     if (nv <= 1) LONG(1); else if (nv <= 2) LONG(2); else if (nv <= 4) LONG(4); else LONG(8);
 #undef LONG
 }
@@ -445,7 +454,7 @@ void max_full(Ctx* c, int l) {
     const int ld = c->ws[l];
     int32_t* long_rows = c->Clist[0];
     int* n_long = &c->ctl->work_counter[(l - 1) & 7];
-#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 16, 256, 0, c->ctl, l, 0, (const int32_t*)nullptr, (const int*)nullptr, c->N, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw)
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 16, 256, 0, c->ctl, l, 0, (const int32_t*)nullptr, (const int*)nullptr, c->N, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
     RP_MAX_DISPATCH(ld, ROWS);
 #undef ROWS
     launch_long_rows(c, 0, c->H[l - 1], ld, c->S[l], long_rows, n_long);
@@ -457,21 +466,21 @@ void max_hop(Ctx* c, int l, int n) {
     const float* Old = c->D[(l - 1) & 1];            // previous values of the rows of A_{l-1}, in its order
     const int32_t* senders = c->Clist[(l - 1) & 1];
     const int T = 256;
-#define MSG(NV, LPR) RP_LAUNCH(c, (k_max_messages<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, senders, c->old_idx, c->coff, c->side[0], c->side[1], c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2, c->invmask, c->mw)
+#define MSG(NV, LPR) RP_LAUNCH(c, (k_max_messages<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, senders, c->old_idx, c->coff, c->side[0], c->side[1], c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
     RP_MAX_DISPATCH(ld, MSG);
 #undef MSG
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
     if (n > 0)
         RP_LAUNCH(c, k_max_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[1], c->posmap,
-                  c->old_idx, c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2, c->invmask, c->mw);
+                  c->old_idx, c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN));
     // invalidated sinks -> list (the buffer of A_l serves until A_l itself is compacted), then their rows
     int32_t* rlist = c->A[l];
     int* n_r = &c->ctl->n_long[l];
     bitmap_to_list_from(c, c->bitmap2, rlist, n_r, nullptr);
     int32_t* long_rows = c->Clist[l & 1];            // the next hop's sender list is not built yet
     int* n_long = &c->ctl->work_counter[(l - 1) & 7];
-#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, 1, rlist, n_r, 0, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw)
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, 1, rlist, n_r, 0, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
     RP_MAX_DISPATCH(ld, ROWS);
 #undef ROWS
     launch_long_rows(c, 1, c->H[l - 1], ld, c->S[l], long_rows, n_long);

@@ -18,6 +18,9 @@
 
 namespace rp {
 
+// monotonic aggregators (Sec. 3.4.2) take the hybrid-incremental path
+inline bool rp_monotonic(int agg) { return agg == RIPPLE_AGG_MAX || agg == RIPPLE_AGG_MIN; }
+
 // ---- device-resident control block -----------------------------------------------------------
 struct Ctl {
     int abort;   // set by validation / planning: the batch is rejected, mutate nothing

@@ -34,6 +34,7 @@ AGG_SUM = 0
 AGG_MEAN = 1
 AGG_WSUM_GCN = 2   # coefficient 1/sqrt(deg_out(u) * deg_in(v))
 AGG_MAX = 3        # element-wise maximum over the in-neighbours (monotonic; zeros if there are none)
+AGG_MIN = 4        # element-wise minimum, likewise
 
 ACT_IDENTITY = 0
 ACT_RELU = 1

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libripple.so")
 MAX_LAYERS = 8
 OK, ERR_INVALID_ARG, ERR_VERTEX_RANGE, ERR_CAPACITY, ERR_OOM, ERR_CUDA, ERR_TIMEOUT = range(7)
 MEM_HOST, MEM_DEVICE = 0, 1
-AGG_SUM, AGG_MEAN, AGG_WSUM_GCN, AGG_MAX = 0, 1, 2, 3
+AGG_SUM, AGG_MEAN, AGG_WSUM_GCN, AGG_MAX, AGG_MIN = 0, 1, 2, 3, 4
 LAYER_SAGE, LAYER_GRAPHCONV, LAYER_GIN = 0, 1, 2
 ACT_IDENTITY, ACT_RELU = 0, 1
 OP_ADD_EDGE, OP_DEL_EDGE, OP_SET_FEATURE, OP_DEL_VERTEX = 0, 1, 2, 3

@@ -1,4 +1,4 @@
-"""Monotonic (max) aggregation on the GPU against the oracle: Sec. 3.4.2, hybrid-incremental
+"""Monotonic (max, min) aggregation on the GPU against the oracle: Sec. 3.4.2, hybrid-incremental
 propagation with pruning.  Graph state, affected sets (= vertices whose cached maximum changed) and
 counters are compared exactly; embeddings and cached maxima within 1e-4 (1 + |ref|)."""
 import os
@@ -42,10 +42,11 @@ def run(env, n, src, dst, model, seed, batches, **kw):
     return pruned
 
 
+@pytest.mark.parametrize("agg", [I.AGG_MAX, I.AGG_MIN], ids=["max", "min"])
 @pytest.mark.parametrize("dims", [[18, 36, 10], [18, 36, 20, 10], [7, 5], [40, 16, 24]])
 @pytest.mark.parametrize("graphs", [True, False], ids=["replayed", "direct"])
-def test_small_models_with_every_update_type(env, dims, graphs):
-    model = I.graphconv_model(dims, I.AGG_MAX)
+def test_small_models_with_every_update_type(env, dims, graphs, agg):
+    model = I.graphconv_model(dims, agg)
     n, m = 600, 5000
     src, dst = I.er_graph(n, m, 7)
     stream = I.UpdateStream(n, src, dst, dims[0], 7)
@@ -63,10 +64,11 @@ def test_small_models_with_every_update_type(env, dims, graphs):
     run(env, n, src, dst, model, 7, batches, graphs=graphs)
 
 
-def test_pruning_wide_layers_and_long_in_lists(env):
+@pytest.mark.parametrize("agg", [I.AGG_MAX, I.AGG_MIN], ids=["max", "min"])
+def test_pruning_wide_layers_and_long_in_lists(env, agg):
     """256-column layers (tensor-core update with old rows kept for the messages), two sinks whose
     in-lists are recomputed by a whole block, and a hub whose out-list reaches half the graph."""
-    model = I.graphconv_model([24, 256, 256, 12], I.AGG_MAX)
+    model = I.graphconv_model([24, 256, 256, 12], agg)
     n = 9000
     src, dst = I.er_graph(n, 45000, 3)
     have = set(zip(src.tolist(), dst.tolist()))

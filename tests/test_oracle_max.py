@@ -16,8 +16,9 @@ from oracle.oracle import Oracle  # noqa: E402
 
 
 def dense_full_max(n, src, dst, X, model, weights):
-    """GraphConv with an element-wise maximum over the in-neighbours, written with an explicit
-    n x n adjacency matrix: x_v = max_{u : A[u, v]} h_u (zeros if v has no in-neighbour)."""
+    """GraphConv with an element-wise maximum (minimum) over the in-neighbours, written with an
+    explicit n x n adjacency matrix: x_v = max_{u : A[u, v]} h_u (zeros if v has no in-neighbour)."""
+    red = np.min if model.agg == I.AGG_MIN else np.max
     A = np.zeros((n, n), dtype=bool)
     A[src, dst] = True
     H = [X.astype(np.float64)]
@@ -26,19 +27,23 @@ def dense_full_max(n, src, dst, X, model, weights):
         for v in range(n):
             nb = np.nonzero(A[:, v])[0]
             if nb.size:
-                agg[v] = H[-1][nb].max(axis=0)
+                agg[v] = red(H[-1][nb], axis=0)
         Z = agg @ w["Wa"].astype(np.float64) + w["ba"]
         H.append(np.maximum(Z, 0.0) if ly.act == I.ACT_RELU else Z)
     return H
 
 
-def max_model(dims):
-    return I.graphconv_model(dims, I.AGG_MAX)
+def max_model(dims, agg=I.AGG_MAX):
+    return I.graphconv_model(dims, agg)
 
 
+AGGS = [I.AGG_MAX, I.AGG_MIN]
+
+
+@pytest.mark.parametrize("agg", AGGS, ids=["max", "min"])
 @pytest.mark.parametrize("seed", [0, 1, 2])
-def test_full_matches_dense_definition(seed):
-    m = max_model([5, 6, 4, 3])
+def test_full_matches_dense_definition(seed, agg):
+    m = max_model([5, 6, 4, 3], agg)
     n = 14
     src, dst = P.random_graph(n, 30, seed)
     X = I.features(n, 5, seed)
@@ -53,7 +58,8 @@ def test_full_matches_dense_definition(seed):
     assert np.all(o.full_S(1)[deg_in == 0] == 0.0)
     v = int(np.argmax(deg_in))
     nb = src[dst == v]
-    assert np.array_equal(o.full_S(1)[v], X[nb].astype(np.float64).max(axis=0))
+    red = np.min if agg == I.AGG_MIN else np.max
+    assert np.array_equal(o.full_S(1)[v], red(X[nb].astype(np.float64), axis=0))
 
 
 def _three_cases():
@@ -87,9 +93,10 @@ def test_worked_cases_of_the_paper(case):
     assert np.array_equal(o.affected(1), want)             # an unchanged maximum is not propagated
 
 
+@pytest.mark.parametrize("agg", AGGS, ids=["max", "min"])
 @pytest.mark.parametrize("seed", [0, 1, 2, 3])
-def test_hybrid_incremental_equals_full_recompute(seed):
-    m = max_model([6, 8, 5, 4])
+def test_hybrid_incremental_equals_full_recompute(seed, agg):
+    m = max_model([6, 8, 5, 4], agg)
     L = 3
     n = 40
     src, dst = P.random_graph(n, 150, 60 + seed)
@@ -160,3 +167,26 @@ def test_models_with_a_self_term_are_refused():
     src, dst = P.random_graph(10, 20, 1)
     o = Oracle(10, src, dst, I.features(10, 4, 1), m, I.make_weights(m, 1))
     assert o.apply_incremental(P.ups_array([(I.OP_ADD_EDGE, 0, 1)])) != 0
+
+
+def test_min_is_the_mirror_image_of_max():
+    """With the identity activation, negating features and the first layer's weights turns a
+    min model into the max model of the negated inputs: the two oracles must agree row by row."""
+    n = 30
+    src, dst = P.random_graph(n, 100, 5)
+    X = I.features(n, 4, 5)
+    mmax, mmin = max_model([4, 3], I.AGG_MAX), max_model([4, 3], I.AGG_MIN)
+    for ly in mmax.layers + mmin.layers:
+        ly.act = I.ACT_IDENTITY
+    W = I.make_weights(mmax, 5, zero_bias=False)
+    Wneg = [{"Wa": -W[0]["Wa"], "ba": W[0]["ba"]}]
+    omax = Oracle(n, src, dst, -X, mmax, Wneg)
+    omin = Oracle(n, src, dst, X, mmin, W)
+    assert np.array_equal(omax.H(1), omin.H(1)) and np.array_equal(omax.S(1), -omin.S(1))
+    rows = I.features(3, 4, 6)
+    recs = [(I.OP_SET_FEATURE, 2, 0), (I.OP_DEL_EDGE, int(src[0]), int(dst[0])), (I.OP_ADD_EDGE, 1, 7),
+            (I.OP_SET_FEATURE, 9, 1), (I.OP_DEL_VERTEX, 11, 0)]
+    assert omax.apply_incremental(P.ups_array(recs), -rows) == 0
+    assert omin.apply_incremental(P.ups_array(recs), rows) == 0
+    assert np.array_equal(omax.H(1), omin.H(1)) and np.array_equal(omax.S(1), -omin.S(1))
+    assert np.array_equal(omax.affected(1), omin.affected(1))
