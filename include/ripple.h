@@ -51,11 +51,12 @@ typedef enum { RIPPLE_MEM_HOST = 0, RIPPLE_MEM_DEVICE = 1 } ripple_mem;
 /* Aggregators of Table 1.  WSUM_GCN is the weighted sum with alpha_uv = 1/sqrt(deg_out(u) deg_in(v))
  * taken from the current graph and recomputed whenever a degree changes.
  * MAX, MIN (Sec. 3.4.2, monotonic aggregation): element-wise maximum / minimum over the in-neighbours,
- * zeros for a vertex without in-neighbours; GRAPHCONV layers only.  Its batches run hybrid-incrementally:
+ * zeros for a vertex without in-neighbours; GRAPHCONV and SAGE layers.  Its batches run hybrid-incrementally:
  * a message carries the sender's old and new row, a sink raises its cached maximum, recomputes it
  * over all in-neighbours, or ignores the message; a sink whose cached maximum did not change is
  * not affected and propagates nothing (ripple_get_affected then lists exactly the vertices whose
- * cached maximum changed; ripple_stats.senders those whose embedding changed). */
+ * cached maximum changed -- for SAGE also those whose own previous-layer row changed;
+ * ripple_stats.senders those whose embedding changed). */
 typedef enum {
     RIPPLE_AGG_SUM = 0, RIPPLE_AGG_MEAN = 1, RIPPLE_AGG_WSUM_GCN = 2, RIPPLE_AGG_MAX = 3, RIPPLE_AGG_MIN = 4
 } ripple_agg;

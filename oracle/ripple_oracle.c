@@ -513,7 +513,7 @@ static const srcinfo_t *source_find(const srcinfo_t *t, int n, int u) {
  * rejected (nothing changed). */
 /* ------------------------------------------------------------------------------------------ */
 /* Monotonic aggregation (Sec. 3.4.2), max (min is its mirror image: read "exceeds" as "is below"
- * and so on), for models without a self term (GraphConv).  A message
+ * and so on), for GraphConv and SAGE layers.  A message
  * <old, new> from a changed in-neighbour, <-, new> along an added edge or <old, -> along a deleted
  * one leads, per element, to one of three actions at the sink:
  *   - new exceeds the cached maximum: the cache is raised to it (incremental);
@@ -521,7 +521,7 @@ static const srcinfo_t *source_find(const srcinfo_t *t, int n, int u) {
  *     known, the sink recomputes it over all current in-neighbours;
  *   - otherwise nothing happens.
  * A sink whose cached row ends up unchanged is not affected and sends nothing on (the pruning of
- * Sec. 6.3).  "Changed" is decided on the values rounded to single precision, the precision of the
+ * Sec. 6.3); with a self term a vertex is also affected when its own previous-layer row changed.  "Changed" is decided on the values rounded to single precision, the precision of the
  * embeddings this oracle is compared with. */
 static int differs_f32(const double *a, const double *b, int n) {
     for (int k = 0; k < n; ++k) if ((float)a[k] != (float)b[k]) return 1;
@@ -529,7 +529,7 @@ static int differs_f32(const double *a, const double *b, int n) {
 }
 
 static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *feat_rows) {
-    int L = o->L, N = o->N;
+    int L = o->L, N = o->N, self_term = o->layer[1].kind != KIND_GRAPHCONV;
     int d0 = o->d[0];
     int is_min = o->agg == AGG_MIN;
 #define BEATS(a, b) (is_min ? (a) < (b) : (a) > (b))   /* a improves on b */
@@ -630,6 +630,14 @@ static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *fe
             if (differs_f32(S + (size_t)v * K, snap + (size_t)t * K, K)) An[nAn++] = v;
             snap_of[v] = -1;
         }
+        /* with a self term a vertex whose own h^{l-1} changed recomputes h^l as well */
+        if (self_term) {
+            for (int t = 0; t < nAn; ++t) o->mark[An[t]] = 1;
+            An = (int *)realloc(An, sizeof(int) * (size_t)(nAn + nC + 1));
+            int base = nAn;
+            for (int i = 0; i < nC; ++i) if (!o->mark[C[i]]) An[nAn++] = C[i];
+            for (int t = 0; t < base; ++t) o->mark[An[t]] = 0;
+        }
         qsort(An, (size_t)nAn, sizeof(int), cmp_int);
         free(T); free(snap); free(C); free(Cold);
 
@@ -658,7 +666,7 @@ int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const flo
     int L = o->L, self_term = o->layer[1].kind != KIND_GRAPHCONV;
 
     if (MONOTONIC(o->agg)) {
-        if (self_term) { delta_free(&dl); return -3; }   /* built for models without a self term only */
+        if (o->layer[1].kind == KIND_GIN) { delta_free(&dl); return -3; }   /* GraphConv and SAGE layers only */
         apply_topology(o, &dl);
         rc = apply_incremental_max(o, &dl, feat_rows);
         delta_free(&dl);

@@ -1,4 +1,4 @@
-// Monotonic aggregation (Sec. 3.4.2), max, for models without a self term.
+// Monotonic aggregation (Sec. 3.4.2), max and min, for GraphConv and SAGE layers.
 //
 // The cached aggregate S^l_v is the element-wise maximum of h^{l-1}_u over In(v) (zeros if v has no
 // in-neighbour).  A local delta cannot update it; instead a message carries the sender's old and
@@ -8,7 +8,7 @@
 //               known, the sink is queued and recomputes its row over all current in-neighbours;
 //   nothing     otherwise.
 // A sink whose cached row ends up unchanged is not affected: it is not recomputed and sends
-// nothing on.  Senders of the next hop are the affected rows whose embedding really changed.
+// nothing on (with a self term it is also affected when its own previous-layer row changed).  Senders of the next hop are the affected rows whose embedding really changed.
 #include "device_utils.cuh"
 #include "ripple_internal.cuh"
 
@@ -408,6 +408,13 @@ __global__ void k_max_records(Ctl* ctl, const Rec* __restrict__ rec, Side in, co
     }
 }
 
+// self term: a vertex whose own previous-layer row changed recomputes its embedding as well
+__global__ void k_max_mark_self(Ctl* ctl, int l, const int32_t* __restrict__ senders, uint32_t* bitmapA) {
+    if (ctl->abort) return;
+    const int n = ctl->nC[l - 1];
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) mark_bit(bitmapA, senders[i]);
+}
+
 // senders of the next hop: affected rows whose embedding really changed (old rows are kept compact,
 // in the order of A_l); one warp per affected row
 __global__ void k_max_senders(Ctl* ctl, int l, const int32_t* __restrict__ A, const float* __restrict__ H,
@@ -430,17 +437,6 @@ __global__ void k_max_senders(Ctl* ctl, int l, const int32_t* __restrict__ A, co
     }
 }
 
-#define RP_MAX_DISPATCH(ld, CALL)                         \
-    do {                                                  \
-        const int nv_ = div_up((ld), 128);                \
-        if ((ld) <= 32) { CALL(1, 8); }                   \
-        else if ((ld) <= 64) { CALL(1, 16); }             \
-        else if (nv_ <= 1) { CALL(1, 32); }               \
-        else if (nv_ <= 2) { CALL(2, 32); }               \
-        else if (nv_ <= 4) { CALL(4, 32); }               \
-        else { CALL(8, 32); }                             \
-    } while (0)
-
 static void launch_long_rows(Ctx* c, int mode, const float* M, int ld, float* S, int32_t* long_rows, int* n_long) {
     const int nv = div_up(ld, 128);
     const size_t smem = (size_t)8 * std::max(ld, MAX_EL) * sizeof(float);
@@ -455,7 +451,7 @@ void max_full(Ctx* c, int l) {
     int32_t* long_rows = c->Clist[0];
     int* n_long = &c->ctl->work_counter[(l - 1) & 7];
 #define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 16, 256, 0, c->ctl, l, 0, (const int32_t*)nullptr, (const int*)nullptr, c->N, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
-    RP_MAX_DISPATCH(ld, ROWS);
+    RP_WIDTH_DISPATCH(ld, ROWS);
 #undef ROWS
     launch_long_rows(c, 0, c->H[l - 1], ld, c->S[l], long_rows, n_long);
 }
@@ -468,7 +464,7 @@ void max_hop(Ctx* c, int l, int n) {
     const int T = 256;
 #define MSG(NV, LPR) RP_LAUNCH(c, (k_max_messages<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, senders, c->old_idx, c->coff, c->side[0], c->side[1], c->H[l - 1], Old, ld, c->S[l], c->bitmap, c->bitmap2, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
-    RP_MAX_DISPATCH(ld, MSG);
+    RP_WIDTH_DISPATCH(ld, MSG);
 #undef MSG
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
     if (n > 0)
@@ -481,9 +477,10 @@ void max_hop(Ctx* c, int l, int n) {
     int32_t* long_rows = c->Clist[l & 1];            // the next hop's sender list is not built yet
     int* n_long = &c->ctl->work_counter[(l - 1) & 7];
 #define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, 1, rlist, n_r, 0, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
-    RP_MAX_DISPATCH(ld, ROWS);
+    RP_WIDTH_DISPATCH(ld, ROWS);
 #undef ROWS
     launch_long_rows(c, 1, c->H[l - 1], ld, c->S[l], long_rows, n_long);
+    if (c->self_term) RP_LAUNCH(c, k_max_mark_self, c->n_sm * 2, T, 0, c->ctl, l, senders, c->bitmap);
 }
 
 // senders of hop l + 1 (l = 0: the vertices whose feature row really changed)

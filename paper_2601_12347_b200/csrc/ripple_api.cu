@@ -131,8 +131,8 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
     if (!g || !features || !layers || !out) { set_err(nullptr, "null argument"); return st; }
     if (L < 1 || L > RP_MAXL) { set_err(nullptr, "L must be in 1..%d", RP_MAXL); return st; }
     if (agg < 0 || agg > 4) { set_err(nullptr, "unknown aggregator %d", agg); return st; }
-    if (rp_monotonic(agg) && layers[0].kind != RIPPLE_LAYER_GRAPHCONV) {
-        set_err(nullptr, "the max and min aggregators are built for layers without a self term (GRAPHCONV) only");
+    if (rp_monotonic(agg) && layers[0].kind == RIPPLE_LAYER_GIN) {
+        set_err(nullptr, "the max and min aggregators are built for GRAPHCONV and SAGE layers");
         return st;
     }
     if (g->num_vertices < 1 || g->num_vertices > 0x7fffffff - 64 || g->num_edges < 0 ||
@@ -361,6 +361,7 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
             frontier_compact(c, l);
             senders_release(c, l - 1);
             STAMP();
+            self_project(c, l, false);
             update_rows(c, l, false);
             if (l < L) max_senders_build(c, l);
             STAMP();

@@ -180,6 +180,18 @@ inline int pad4(int x) { return (x + 3) & ~3; }
         (ctx)->launches++;                                                      \
     } while (0)
 
+// dispatch on row width: ld <= 32 floats -> 8 lanes per row, <= 64 -> 16, else whole warp
+#define RP_WIDTH_DISPATCH(ld, CALL)                       \
+    do {                                                  \
+        const int nv_ = div_up((ld), 128);                \
+        if ((ld) <= 32) { CALL(1, 8); }                   \
+        else if ((ld) <= 64) { CALL(1, 16); }             \
+        else if (nv_ <= 1) { CALL(1, 32); }               \
+        else if (nv_ <= 2) { CALL(2, 32); }               \
+        else if (nv_ <= 4) { CALL(4, 32); }               \
+        else { CALL(8, 32); }                             \
+    } while (0)
+
 // graph_store.cu
 cudaError_t graph_build(Ctx* c, const int32_t* src_dev, const int32_t* dst_dev, int64_t E,
                         double slack, int64_t pool_edges);

@@ -151,18 +151,6 @@ k_spmm_hubs(Side in, const int32_t* __restrict__ deg_out, int src_norm, const fl
     }
 }
 
-// dispatch on row width: ld <= 32 floats -> 8 lanes per row, <= 64 -> 16, else whole warp
-#define RP_WIDTH_DISPATCH(ld, CALL)                       \
-    do {                                                  \
-        const int nv_ = div_up((ld), 128);                \
-        if ((ld) <= 32) { CALL(1, 8); }                   \
-        else if ((ld) <= 64) { CALL(1, 16); }             \
-        else if (nv_ <= 1) { CALL(1, 32); }               \
-        else if (nv_ <= 2) { CALL(2, 32); }               \
-        else if (nv_ <= 4) { CALL(4, 32); }               \
-        else { CALL(8, 32); }                             \
-    } while (0)
-
 void spmm_full(Ctx* c, int l) {
     const int ld = c->ws[l];
     const float* M = c->H[l - 1];

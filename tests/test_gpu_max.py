@@ -92,10 +92,33 @@ def test_pruning_wide_layers_and_long_in_lists(env, agg):
     assert pruned > 0     # some messages changed no cached maximum and were not propagated
 
 
-def test_models_with_a_self_term_are_refused(env):
+def test_gin_layers_are_refused(env):
     ripple, _ = env
-    model = I.sage_model([8, 8, 4], I.AGG_MAX)
+    model = I.gin_model(8, 8, 2)
+    model.agg = I.AGG_MAX
     src, dst = I.er_graph(50, 200, 1)
     with pytest.raises(ripple.RippleError) as ei:
         ripple.Ripple(50, src, dst, I.features(50, 8, 1), model, I.make_weights(model, 1))
     assert ei.value.status == ripple.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("agg", [I.AGG_MAX, I.AGG_MIN], ids=["max", "min"])
+@pytest.mark.parametrize("dims", [[18, 36, 10], [18, 36, 20, 10], [24, 256, 12]])
+def test_self_term_with_a_monotonic_aggregator(env, dims, agg):
+    """SAGE layers with max / min pooling: affected = cached row changed, or own input row changed."""
+    model = I.sage_model(dims, agg)
+    n, m = 2500, 20000
+    src, dst = I.er_graph(n, m, 11)
+    stream = I.UpdateStream(n, src, dst, dims[0], 11)
+    rng = np.random.default_rng(11)
+
+    def batches(orc):
+        for b, bs in enumerate([1, 3, 40, 7, 400, 1, 64, 1500, 120]):
+            if b % 3 == 2:
+                rowptr, col = orc.export_csr()
+                edges = {(u, int(col[j])) for u in range(n) for j in range(rowptr[u], rowptr[u + 1])}
+                yield G.ups_array(random_batch(rng, n, edges, bs, 6, p_vertex=0.05)), I.features(6, dims[0], 300 + b)
+            else:
+                yield stream.next_batch(bs)
+
+    run(env, n, src, dst, model, 11, batches, max_batch=4096)

@@ -162,11 +162,66 @@ def test_empty_in_list_transitions_and_negative_maxima():
     assert np.array_equal(o.H(1), full[1])
 
 
-def test_models_with_a_self_term_are_refused():
-    m = I.sage_model([4, 4, 4], I.AGG_MAX)
+def test_gin_layers_are_refused():
+    m = I.gin_model(4, 4, 2)
+    m.agg = I.AGG_MAX
     src, dst = P.random_graph(10, 20, 1)
     o = Oracle(10, src, dst, I.features(10, 4, 1), m, I.make_weights(m, 1))
     assert o.apply_incremental(P.ups_array([(I.OP_ADD_EDGE, 0, 1)])) != 0
+
+
+def dense_full_sage_max(n, src, dst, X, model, weights):
+    A = np.zeros((n, n), dtype=bool)
+    A[src, dst] = True
+    red = np.min if model.agg == I.AGG_MIN else np.max
+    H = [X.astype(np.float64)]
+    for ly, w in zip(model.layers, weights):
+        agg = np.zeros((n, H[-1].shape[1]))
+        for v in range(n):
+            nb = np.nonzero(A[:, v])[0]
+            if nb.size:
+                agg[v] = red(H[-1][nb], axis=0)
+        Z = H[-1] @ w["Wa"].astype(np.float64) + agg @ w["Wb"].astype(np.float64) + w["ba"]
+        H.append(np.maximum(Z, 0.0) if ly.act == I.ACT_RELU else Z)
+    return H
+
+
+@pytest.mark.parametrize("agg", AGGS, ids=["max", "min"])
+@pytest.mark.parametrize("seed", [0, 1])
+def test_self_term_with_a_monotonic_aggregator(seed, agg):
+    """SAGE layers: h = act(W_self h_v + W_neigh max_u h_u + b).  A vertex is affected when its
+    cached maximum or its own previous-layer row changed."""
+    m = I.sage_model([6, 8, 5, 4], agg)
+    L, n = 3, 40
+    src, dst = P.random_graph(n, 150, 70 + seed)
+    X = I.features(n, 6, seed)
+    W = I.make_weights(m, seed, zero_bias=False)
+    o = Oracle(n, src, dst, X, m, W)
+    edges = set(zip(src.tolist(), dst.tolist()))
+    Xcur = X.copy()
+    rng = np.random.default_rng(seed)
+    o.full()
+    for b in range(10):
+        rows = I.features(5, 6, 400 + 20 * seed + b)
+        recs = random_batch(rng, n, edges, int(rng.integers(1, 12)), 5, p_vertex=0.08)
+        S_old = [None] + [o.full_S(l).copy() for l in range(1, L + 1)]
+        H_old = [o.H(l).copy() for l in range(L + 1)]
+        edges, feat = replay(edges, recs)
+        for v, r in feat.items():
+            Xcur[v] = rows[r] if r >= 0 else 0.0
+        assert o.apply_incremental(P.ups_array(recs), rows) == 0
+        e = sorted(edges)
+        ref = dense_full_sage_max(n, np.array([a for a, _ in e], dtype=np.int32),
+                                  np.array([c for _, c in e], dtype=np.int32), Xcur, m, W)
+        o.full()
+        for l in range(L + 1):
+            assert P.rel_err(o.H(l), ref[l]) < 1e-12, (seed, b, l)
+        for l in range(1, L + 1):
+            S_new = o.full_S(l)
+            assert np.array_equal(o.S(l), S_new)
+            changed = set(np.nonzero(np.any(S_new != S_old[l], axis=1))[0].tolist())
+            own = set(np.nonzero(np.any(o.H(l - 1).astype(np.float32) != H_old[l - 1].astype(np.float32), axis=1))[0].tolist())
+            assert set(o.affected(l).tolist()) == changed | own, (seed, b, l)
 
 
 def test_min_is_the_mirror_image_of_max():
