@@ -343,6 +343,25 @@ def run_ours(args, rank, world, local_rank):
     rp.close()
     del rp
     torch.cuda.empty_cache()
+    if pulls == 0 and sc_ms > 0 and msgs >= 1:
+        # The push scatter is made of 16-byte vector reductions that mostly land in L2.  The same
+        # number of reductions of the same row width into pseudo-random rows, timed alone, gives the
+        # ceiling of that path on this GPU: with a window that fits L2, and with a window of the
+        # size of the aggregate matrix (every row its own DRAM line).
+        payload = msgs * ld_last * 4
+        ms_l2 = ripple.probe_reduction_rate(max(1, (64 << 20) // (ld_last * 4)), ld_last, int(msgs))
+        ms_ws = ripple.probe_reduction_rate(w.n, ld_last, int(msgs))
+        got = payload / 1e9 / (sc_ms / K / 1e3)
+        roofline["reduction_path"] = {
+            "payload_GBps_achieved": got,
+            "probe_64MB_window_GBps": payload / 1e9 / (ms_l2 / 1e3),
+            "probe_aggregate_sized_window_GBps": payload / 1e9 / (ms_ws / 1e3),
+            "frac_of_64MB_probe": got / (payload / 1e9 / (ms_l2 / 1e3)),
+            "note": "payload = messages x row bytes (one reduction each, no read counted); the probes issue the "
+                    "same count of red.global.add.v4.f32 rows, and nothing else, into uniformly random rows of a "
+                    "zeroed window; a fraction above 1 means the scatter, whose sinks are skewed towards popular "
+                    "rows, retires reductions faster than the bare loop does on uniform rows: no headroom left "
+                    "on this path"}
     if not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(args, w, src, dst, X, W)
     print(json.dumps(line), flush=True)

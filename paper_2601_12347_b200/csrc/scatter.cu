@@ -585,4 +585,52 @@ void regather_layer(Ctx* c, int l) {
     if (c->timing) cudaEventRecord(c->ev_rg[2 * l + 1], c->stream);
 }
 
+// ---------------------------------------------------------------------------------------------
+// diagnostic: the rate at which the device retires the 16-byte vector reductions the push scatter
+// is made of, on rows drawn pseudo-randomly from a window of n_rows rows
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_probe_reductions(float* buf, long long n_rows, int nq, long long n_messages, unsigned long long seed) {
+    const long long total = n_messages * nq;
+    for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total;
+         t += (long long)gridDim.x * blockDim.x) {
+        const long long m = t / nq;
+        const int q = (int)(t - m * nq);
+        const long long row = (long long)(mix64((unsigned long long)m + seed) % (unsigned long long)n_rows);
+        red_add_v4(buf + (size_t)row * (4 * nq) + 4 * q, make_float4(1.f, 1.f, 1.f, 1.f));
+    }
+}
+
 }  // namespace rp
+
+extern "C" ripple_status ripple_probe_reduction_rate(int32_t device, int64_t n_rows, int32_t row_floats,
+                                                     int64_t n_messages, float* ms_out) {
+    if (n_rows < 1 || row_floats < 4 || (row_floats & 3) || n_messages < 1 || !ms_out) return RIPPLE_ERR_INVALID_ARG;
+    if (device >= 0 && cudaSetDevice(device) != cudaSuccess) return RIPPLE_ERR_CUDA;
+    float* buf = nullptr;
+    const size_t bytes = sizeof(float) * (size_t)n_rows * (size_t)row_floats;
+    if (cudaMalloc(&buf, bytes) != cudaSuccess) { cudaGetLastError(); return RIPPLE_ERR_OOM; }
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0);
+    cudaEventCreate(&e1);
+    int n_sm = 1;
+    cudaGetDevice(&device);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device);
+    cudaMemset(buf, 0, bytes);
+    float best = 0.f;
+    for (int rep = 0; rep < 4; ++rep) {   // the first pass warms up
+        cudaEventRecord(e0);
+        rp::k_probe_reductions<<<n_sm * 8, 256>>>(buf, n_rows, row_floats / 4, n_messages, 0x9E37ull * (rep + 1));
+        cudaEventRecord(e1);
+        cudaEventSynchronize(e1);
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        if (rep > 0 && (best == 0.f || ms < best)) best = ms;
+    }
+    cudaError_t e = cudaGetLastError();
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    cudaFree(buf);
+    *ms_out = best;
+    return e == cudaSuccess ? RIPPLE_OK : RIPPLE_ERR_CUDA;
+}

@@ -30,7 +30,7 @@ UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
 EXPORTED = [
     "ripple_create", "ripple_apply_batch", "ripple_get_embeddings", "ripple_get_aggregate",
     "ripple_get_affected", "ripple_export_graph", "ripple_get_degrees", "ripple_recompute_full",
-    "ripple_export_graph_static", "ripple_set_timing",
+    "ripple_export_graph_static", "ripple_set_timing", "ripple_probe_reduction_rate",
     "ripple_get_stats", "ripple_last_error", "ripple_destroy", "ripple_version",
 ]
 
@@ -110,7 +110,8 @@ def load_library(path: Optional[str] = None):
     lib.ripple_version.restype = ctypes.c_char_p
     lib.ripple_export_graph_static.argtypes = [vp, vp, vp, i64]
     lib.ripple_set_timing.argtypes = [vp, i32]
-    for name in EXPORTED[:11]:
+    lib.ripple_probe_reduction_rate.argtypes = [i32, i64, i32, i64, P(ctypes.c_float)]
+    for name in EXPORTED[:12]:
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -319,6 +320,17 @@ class Ripple:
                   "ms_update", "ms_scatter_kernel", "ms_regather"):
             out[k] = list(getattr(s, k))[: L + 1]
         return out
+
+
+def probe_reduction_rate(n_rows: int, row_floats: int, n_messages: int, device: int = -1) -> float:
+    """Milliseconds for n_messages rows of row_floats floats issued as 16-byte vector reductions
+    into pseudo-random rows of a window of n_rows rows (best of three passes)."""
+    lib = load_library()
+    ms = ctypes.c_float()
+    st = lib.ripple_probe_reduction_rate(int(device), int(n_rows), int(row_floats), int(n_messages), ctypes.byref(ms))
+    if st:
+        raise RippleError(st, "reduction probe failed")
+    return float(ms.value)
 
 
 def version() -> str:

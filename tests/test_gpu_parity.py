@@ -677,3 +677,12 @@ def test_mixed_growth_and_deletion_in_the_same_rows(env):
     assert rp.stats()["pool_used"] > 0 and rp.stats()["num_edges"] == len(present)
     check_values(rp, orc.full(), 2)
     rp.close()
+
+
+def test_reduction_probe_runs_and_rejects_bad_arguments(env):
+    ripple, _ = env
+    assert ripple.probe_reduction_rate(1000, 48, 20000) > 0.0
+    for bad in [(0, 48, 10), (10, 6, 10), (10, 48, 0)]:
+        with pytest.raises(ripple.RippleError) as ei:
+            ripple.probe_reduction_rate(*bad)
+        assert ei.value.status == ripple.ERR_INVALID_ARG
