@@ -142,7 +142,8 @@ typedef struct {
     void* stream;         /* cudaStream_t to run on (NULL: the library creates its own)                     */
     float regather_threshold; /* AUTO only: a hop rebuilds its aggregates once its messages number at least
                              this share of all edges.  0: default (0.6 for aggregate rows of 128 floats
-                             or more, else 0.7); < 0: never                       */
+                             or more, else 0.7, and never for hops of fewer than 4 Mi messages,
+                             where pushing is as fast); < 0: never                       */
 } ripple_options;
 
 typedef struct {

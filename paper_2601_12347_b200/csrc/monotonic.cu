@@ -17,7 +17,7 @@
 
 namespace rp {
 
-constexpr int MAX_HUB_DEGREE = 4096;   // longer in-lists are recomputed by a whole block
+constexpr int MAX_HUB_DEGREE = 1024;   // longer in-lists are recomputed by a whole block
 constexpr int MAX_CHUNK = 64;          // edges per warp work item of the message walk
 
 // The same code serves min: every comparison goes through these helpers (is_min = 0: maximum).

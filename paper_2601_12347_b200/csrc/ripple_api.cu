@@ -243,6 +243,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                 c->ws[l] = c->pre[l] ? target : ly.ld_in;
                 // measured on the dense graph: rebuilding every aggregate costs 0.60 of pushing a message
                 // along every edge at 256 floats per row (15.7 against 26 ms) and 0.67 at 48 (4.3 / 6.4 ms)
+                c->regather_min_messages = o.regather_threshold > 0.f ? 0 : (4ll << 20);
                 c->regather_threshold[l] = o.regather_threshold > 0.f ? o.regather_threshold
                                            : o.regather_threshold < 0.f ? -1.f
                                            : c->ws[l] >= 128 ? 0.6f : 0.7f;
@@ -294,8 +295,8 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             CK(dev_alloc(&c->grow_list[s], (size_t)o.max_batch));
         }
         // degree prefix of a sender list; also the (vertex, chunk) work items of long in-lists during a
-        // gather: at most 1.5 items per 1024 stored edges
-        CK(dev_alloc(&c->coff, std::max((size_t)N + 2, (size_t)(c->side[1].col_size / 680) + 64), 0));
+        // gather: a row of more than 256 entries gives at most 2 items per 256 of them
+        CK(dev_alloc(&c->coff, std::max((size_t)N + 2, (size_t)(c->side[1].col_size / 128) + 64), 0));
         CK(dev_alloc(&c->bitmap, (size_t)c->n_words + 256, 0));
         if (rp_monotonic(agg)) {
             CK(dev_alloc(&c->bitmap2, (size_t)c->n_words + 256, 0));
@@ -406,8 +407,9 @@ static void arm_rebuild(Ctx* c, int nb) {
         if (rp_monotonic(c->agg)) armed = false;
         else if (c->scatter_mode == RIPPLE_SCATTER_REGATHER) armed = true;
         else if (c->scatter_mode == RIPPLE_SCATTER_AUTO && c->regather_threshold[l] > 0.f)
-            armed = no_history || (double)c->stats.active_edges[l] >=
-                                      0.5 * (double)c->regather_threshold[l] * (double)c->stats.num_edges;
+            armed = (no_history || (double)c->stats.active_edges[l] >=
+                                       0.5 * (double)c->regather_threshold[l] * (double)c->stats.num_edges) &&
+                    c->stats.num_edges + c->max_batch >= c->regather_min_messages;
         c->rebuild_armed[l] = armed;
     }
 }

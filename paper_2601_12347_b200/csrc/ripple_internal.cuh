@@ -109,6 +109,7 @@ struct Ctx {
     long long batches_done;
     int last_nb;
     int may_expand;   // the batch being enqueued may hold vertex deletions (always assumed for device batches)
+    long long regather_min_messages;   // default threshold only: hops with fewer messages always push
     float regather_threshold[RP_MAXL + 1];  // per hop: share of all edges from which the hop rebuilds its aggregates
     int n_sm;
     LayerDev layer[RP_MAXL + 1];

@@ -35,8 +35,11 @@ __device__ __forceinline__ void add4(float4& a, const float4& x, float c) {
 // bootstrap: S_v for every vertex by gathering over in-edges (Eq. 1)
 // LPR lanes hold one row (NV float4 slots each); a warp works on 32 / LPR in-neighbours at a time.
 // ---------------------------------------------------------------------------------------------
-constexpr int SPMM_HUB_DEGREE = 2048;  // longer in-lists are cut into chunks handled by separate warps
-constexpr int SPMM_HUB_CHUNK = 1024;
+// In-lists longer than this are cut into chunks handled by separate warps.  A warp gathers about
+// three neighbours per microsecond at 256 floats per row, so one 2048-neighbour row used to keep a
+// single warp busy for 0.7 ms, longer than everything else of a hop on the sparse graph.
+constexpr int SPMM_HUB_DEGREE = 256;
+constexpr int SPMM_HUB_CHUNK = 256;
 
 // acc += sum over in-list entries [j_begin, j_end) of row v of c_u * M_u; LPR lanes hold one row
 // (NV float4 slots each), a warp works on 32 / LPR neighbours per step, four steps in flight.
@@ -91,8 +94,8 @@ __device__ __forceinline__ void spmm_accumulate(float4 (&acc)[NV], const Side& i
     }
 }
 
-// One warp per vertex.  A vertex with a very long in-list only zeroes its row here and queues
-// (vertex, chunk) work items for k_spmm_hubs, so that no single warp walks 150 K neighbours.
+// One warp per vertex.  A vertex with a long in-list only zeroes its row here and queues
+// (vertex, chunk) work items for k_spmm_hubs, so that no single warp walks thousands of neighbours.
 template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_spmm_pull(int N, Side in, const int32_t* __restrict__ deg_out, int src_norm,
@@ -473,13 +476,19 @@ k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int
 // the affected sinks once and overwriting their aggregates costs less than one reduction per
 // message: a gathered row is a plain load, a delivered message a read-modify-write in L2.  The
 // rebuilt aggregate also sheds whatever rounding the deltas had left in it.  threshold = the
-// share of all edges above which the hop rebuilds (<= 0: never).
-__global__ void k_choose_direction(Ctl* ctl, int l, int mode, float threshold) {
+// share of all edges above which the hop rebuilds (<= 0: never).  With the default threshold a hop
+// of fewer than min_messages messages pushes regardless: on a graph of a million edges neither
+// form is throughput-bound, and the edge-balanced push is the more parallel of the two (measured
+// on the sparse graph, 256 floats per row: 0.24 ms pushed, 0.26 to 0.47 ms rebuilt).
+__global__ void k_choose_direction(Ctl* ctl, int l, int mode, float threshold, long long min_messages) {
     const int nC = ctl->nC[l - 1];
     int re = 0;
     if (mode == RIPPLE_SCATTER_REGATHER) re = 1;
-    else if (mode == RIPPLE_SCATTER_AUTO && threshold > 0.f)
-        re = (double)(ctl->E[l] + (unsigned long long)ctl->n_rec) >= (double)threshold * (double)ctl->num_edges && ctl->num_edges > 0;
+    else if (mode == RIPPLE_SCATTER_AUTO && threshold > 0.f) {
+        const unsigned long long msgs = ctl->E[l] + (unsigned long long)ctl->n_rec;
+        re = (double)msgs >= (double)threshold * (double)ctl->num_edges && ctl->num_edges > 0 &&
+             msgs >= (unsigned long long)min_messages;
+    }
     if (nC == 0 && ctl->n_rec == 0) re = 0;
     ctl->pull[l] = mode == RIPPLE_SCATTER_PULL;
     ctl->regather[l] = re;
@@ -515,7 +524,7 @@ void fold_deltas(Ctx* c, int l) {
 
 void choose_direction(Ctx* c, int l) {
     RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode,
-              c->rebuild_armed[l] ? c->regather_threshold[l] : -1.f);
+              c->rebuild_armed[l] ? c->regather_threshold[l] : -1.f, c->regather_min_messages);
 }
 
 // delta form of hop l (does nothing on the device if the hop rebuilds)

@@ -573,8 +573,8 @@ def test_hub_stress_streams(env, mix):
 
 
 def test_rebuilding_hops_with_long_in_lists(env):
-    """Default settings on a graph where two sinks have in-lists long enough to be gathered in
-    chunks by separate warps; wide layers, so that saturated hops rebuild their aggregates."""
+    """A graph where two sinks have in-lists long enough to be gathered in chunks by separate warps;
+    saturated hops rebuild their aggregates (by default only hops of millions of messages would)."""
     ripple, Oracle = env
     model = I.sage_model([20, 128, 128, 128, 12], I.AGG_MEAN)
     L = 4
@@ -588,7 +588,7 @@ def test_rebuilding_hops_with_long_in_lists(env):
     dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
     X = I.features(n, 20, 11)
     W = I.make_weights(model, 11, zero_bias=False)
-    rp = ripple.Ripple(n, src, dst, X, model, W)
+    rp = ripple.Ripple(n, src, dst, X, model, W, regather_threshold=0.65)   # an explicit threshold also applies to small hops
     orc = Oracle(n, src, dst, X, model, W)
     stream = I.UpdateStream(n, src, dst, 20, 11)
     forms = set()
