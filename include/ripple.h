@@ -134,15 +134,17 @@ typedef struct {
     int32_t scatter_mode; /* ripple_scatter_mode: how delta messages reach the aggregates                   */
     int32_t gemm_mode;    /* ripple_gemm_mode: arithmetic of the affected-row layer update                  */
     int32_t timing;       /* non-zero: record per-stage CUDA-event times into ripple_stats                  */
-    int32_t pre_transform;/* 0: a layer narrower than its input applies its neighbour matrix to the sender
+    int32_t pre_transform;/* 0: a layer not wider than its input applies its neighbour matrix to the sender
                              rows before the scatter (messages and the cached aggregate then have the
-                             layer's output width); 1: never, aggregates always hold input-width rows    */
+                             layer's output width; for equal widths only where nothing but that product
+                             would be left per affected row: SAGE, GRAPHCONV); 1: never, aggregates
+                             always hold input-width rows                                                */
     int32_t no_graphs;    /* non-zero: never replay small batches (<= 512 updates) as a captured CUDA graph     */
     int32_t device;       /* CUDA device ordinal, or -1 for the current device                              */
     void* stream;         /* cudaStream_t to run on (NULL: the library creates its own)                     */
     float regather_threshold; /* AUTO only: a hop rebuilds its aggregates once its messages number at least
-                             this share of all edges.  0: default (0.6 for aggregate rows of 128 floats
-                             or more, else 0.7, and never for hops of fewer than 4 Mi messages,
+                             this share of all edges.  0: default (0.5 for aggregate rows of 128 floats
+                             or more, else 0.55, and never for hops of fewer than 4 Mi messages,
                              where pushing is as fast); < 0: never                       */
 } ripple_options;
 

@@ -239,14 +239,19 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             {
                 // a layer narrower than its input transforms the few sender rows before the scatter
                 const int target = y.kind == RIPPLE_LAYER_GIN ? ly.ld_hid : ly.ld_out;
-                c->pre[l] = o.pre_transform == 0 && target < ly.ld_in && !rp_monotonic(agg);   // a maximum does not commute with the matrix
+                // Also for equal widths where nothing but the matrix product is left per affected row
+                // (SAGE with its cached self projection, GraphConv): the product then runs over the
+                // senders of the hop, the affected rows of the hop before, which are far fewer.
+                // Not for max / min: a maximum does not commute with the matrix.
+                c->pre[l] = o.pre_transform == 0 && !rp_monotonic(agg) &&
+                            (target < ly.ld_in || (target == ly.ld_in && y.kind != RIPPLE_LAYER_GIN));
                 c->ws[l] = c->pre[l] ? target : ly.ld_in;
-                // measured on the dense graph: rebuilding every aggregate costs 0.60 of pushing a message
-                // along every edge at 256 floats per row (15.7 against 26 ms) and 0.67 at 48 (4.3 / 6.4 ms)
+                // measured on the dense graph: rebuilding every aggregate costs 0.47 of pushing a message
+                // along every edge at 256 floats per row (12.1 against 26 ms) and 0.54 at 48 (3.5 / 6.4 ms)
                 c->regather_min_messages = o.regather_threshold > 0.f ? 0 : (4ll << 20);
                 c->regather_threshold[l] = o.regather_threshold > 0.f ? o.regather_threshold
                                            : o.regather_threshold < 0.f ? -1.f
-                                           : c->ws[l] >= 128 ? 0.6f : 0.7f;
+                                           : c->ws[l] >= 128 ? 0.5f : 0.55f;
                 if (o.gemm_mode != RIPPLE_GEMM_FP32) {   // transposed, tf32-split copies for the tensor-core form
                     const float* wn = y.kind == RIPPLE_LAYER_SAGE ? w1.data() + (size_t)ly.ld_in * ly.ld_out : w1.data();
                     if (y.kind == RIPPLE_LAYER_SAGE)
