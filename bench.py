@@ -28,7 +28,7 @@ if ROOT not in sys.path:
 
 from paper_2601_12347_b200 import inputs as I  # noqa: E402
 
-NCU_DRAM_BYTES_PER_MESSAGE = 36.0
+NCU_DRAM_BYTES_PER_MESSAGE = 38.0
 METRIC = "updates_per_sec"
 UNIT = "updates/s"
 
@@ -305,7 +305,7 @@ def run_ours(args, rank, world, local_rank):
     peak, peak_kind = load_peaks()
     achieved = (sc_bytes / 1e9) / (sc_ms / 1e3) if sc_ms > 0 else None
     # DRAM traffic of the push kernel from the ncu capture in profiles/scatter_push_mid2l_b1000_ncu_full.txt
-    # (a 1 M-vertex graph of the same kind: the full-size case is too large to capture): 36 bytes per
+    # (a 1 M-vertex graph of the same kind: the full-size case is too large to capture): 38 bytes per
     # message, scaled by this run's messages per launch
     msgs = float(sizes["active_edges"][L]) / K
     traffic = NCU_DRAM_BYTES_PER_MESSAGE * msgs if (pulls == 0 and ld_last == 48) else None
@@ -313,7 +313,7 @@ def run_ours(args, rank, world, local_rank):
                 "frac": (achieved / peak) if achieved else None, "traffic": traffic,
                 "note": "algorithmic bytes count one read + one write of the sink's aggregate row per message; "
                         "most messages hit rows already in L2, so measured DRAM traffic is ~10x lower and the "
-                        "kernel's limiter is the L2 reduction path (ncu: L1TEX 70 %, L2 57 %, DRAM 11 %)",
+                        "kernel's limiter is the L2 reduction path (ncu: L1TEX 80 %, L2 58 %, DRAM 11 %)",
                 "kernel": f"{'k_scatter_pull' if pulls * 2 > K else 'k_scatter_push'} (hop {L}, row width {ld_last} floats)",
                 "pull_steps": int(pulls),
                 "peak_source": f"of {peak_kind}",
