@@ -43,7 +43,7 @@ typedef enum {
     RIPPLE_ERR_CAPACITY = 3,     /* batch larger than max_batch, or overflow edge pool exhausted  */
     RIPPLE_ERR_OOM = 4,          /* device allocation failed                                     */
     RIPPLE_ERR_CUDA = 5,         /* a CUDA runtime call failed                                   */
-    RIPPLE_ERR_TIMEOUT = 6       /* a bounded device-side wait gave up                           */
+    RIPPLE_ERR_TIMEOUT = 6       /* a bounded device-side wait gave up; destroy the context      */
 } ripple_status;
 
 typedef enum { RIPPLE_MEM_HOST = 0, RIPPLE_MEM_DEVICE = 1 } ripple_mem;

@@ -109,6 +109,7 @@ static void launch_update(Ctx* c, UpdParams& p, const TcW& tw) {
     if (tw.hi && c->gemm_mode != RIPPLE_GEMM_FP32 && p.K > 0 && tw.n_pad >= 128) {
         p.tc_mode = c->gemm_mode == RIPPLE_GEMM_TF32 ? TC_TF32 : TC_TF32X3;
         p.tc_min_rows = 1024;
+        p.tc_withhold = c->debug_tc_withhold;
         p.Wt_hi = tw.hi; p.Wt_lo = tw.lo; p.k_pad = tw.k_pad; p.n_pad = tw.n_pad;
     }
     if (p.K == 0) {

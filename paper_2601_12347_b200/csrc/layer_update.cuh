@@ -46,6 +46,7 @@ struct UpdParams {
     // form selection (decided on the device from the row count)
     int tc_mode;                    // TC_OFF: SIMT only
     int tc_min_rows;
+    int tc_withhold;                // diagnostic: the tensor-core kernel never signals its first finished tile
 };
 
 __device__ __forceinline__ float coef_deg(int deg) { return deg > 0 ? 1.0f / sqrtf((float)deg) : 0.0f; }

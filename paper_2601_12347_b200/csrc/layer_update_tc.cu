@@ -36,10 +36,10 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
 
-// true once the phase with the given parity has completed; gives up after TC_SPIN_LIMIT polls
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+// true once the phase with the given parity has completed; gives up after `limit` polls
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit) {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t it = 0; it < TC_SPIN_LIMIT; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -148,6 +148,8 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
     const int row_tiles = (n + TC_M - 1) / TC_M;
     if ((int)blockIdx.x >= row_tiles) return;   // before any allocation
 
+    // the diagnostic that withholds a completion also shortens the waits, so that they run out in milliseconds
+    const uint32_t spin_limit = p.tc_withhold ? (1u << 16) : TC_SPIN_LIMIT;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const bool is_loader = warp < TC_THREADS / 32;
     const bool is_mma_warp = warp == TC_THREADS / 32;
@@ -189,7 +191,7 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
         for (int lt = 0; lt < my_tiles && !failed; ++lt) {
             const int b = lt & 1, ub = lt >> 1;
             // the epilogue must have drained this accumulator buffer (tile lt - 2)
-            if (lane == 0 && ub > 0 && !mbar_wait_bounded(&acc_empty[b], (ub - 1) & 1)) s_fail = 1;
+            if (lane == 0 && ub > 0 && !mbar_wait_bounded(&acc_empty[b], (ub - 1) & 1, spin_limit)) s_fail = 1;
             __syncwarp();
             if ((failed = warp_failed(&s_fail))) break;
             tc_fence_after();
@@ -207,7 +209,7 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                     uint8_t* b_hi = a_hi + (X3 ? 2 : 1) * TC_A_BYTES;
                     uint8_t* b_lo = b_hi + B_BYTES;
                     if (lane == 0) {
-                        if (!mbar_wait_bounded(&full[s], u & 1)) s_fail = 1;
+                        if (!mbar_wait_bounded(&full[s], u & 1, spin_limit)) s_fail = 1;
                         if (!s_fail) {
                             tc_fence_after();
                             const uint64_t da_hi = tc_smem_desc(smem_u32(a_hi)), db_hi = tc_smem_desc(smem_u32(b_hi));
@@ -222,7 +224,9 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                                 }
                             }
                             tc_commit(&empty[s]);
-                            if (ps == n_pass - 1 && kc == nchunks - 1) tc_commit(&acc_full[b]);
+                            // (diagnostic: with tc_withhold the first tile is never reported finished, so that
+                            // the epilogue's bounded wait runs out and the status path can be exercised)
+                            if (ps == n_pass - 1 && kc == nchunks - 1 && !(p.tc_withhold && lt == 0)) tc_commit(&acc_full[b]);
                         }
                     }
                     __syncwarp();
@@ -266,7 +270,7 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
             if (g < total_steps) {
                 const int s = g % TC_STAGES;
                 const uint32_t u = (uint32_t)(g / TC_STAGES);
-                if (u > 0 && !s_fail && !mbar_wait_bounded(&empty[s], (u - 1) & 1)) s_fail = 1;
+                if (u > 0 && !s_fail && !mbar_wait_bounded(&empty[s], (u - 1) & 1, spin_limit)) s_fail = 1;
                 const int r = g % steps_per_tile, ps = r / nchunks, kc = r - ps * nchunks;
                 const int ncol = min(TC_NH, n_pad - ps * TC_NH);
                 uint8_t* b_hi = smem + (size_t)s * STAGE_BYTES + (X3 ? 2 : 1) * TC_A_BYTES;
@@ -343,7 +347,7 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
                 v_own = p.list ? p.list[r0 + lane] : r0 + lane;
                 sc_own = upd_row_scale(p, v_own);
             }
-            if (lane == 0 && !mbar_wait_bounded(&acc_full[b], ub & 1)) s_fail = 1;
+            if (lane == 0 && !mbar_wait_bounded(&acc_full[b], ub & 1, spin_limit)) s_fail = 1;
             __syncwarp();
             if (warp_failed(&s_fail)) break;
             tc_fence_after();

@@ -5,6 +5,7 @@
 #include <algorithm>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -96,6 +97,7 @@ static ripple_status sync_and_fetch_ctl(Ctx* c) {
 // full layer-wise inference over the current graph (Eq. 1-2): bootstrap and recompute-all
 static ripple_status run_full(Ctx* c) {
     c->launches = 0;
+    c->debug_tc_withhold = 0;
     c->params_host[0] = 0; c->params_host[1] = 0;
     cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream);
     RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
@@ -474,6 +476,10 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
         for (int i = 0; i < nb && !wide; ++i) wide = ups[i].op == RIPPLE_OP_DEL_VERTEX;
     const int ng = wide ? (int)c->max_batch : nb;
     c->may_expand = wide || mem != RIPPLE_MEM_HOST;
+    {   // diagnostic: a wait that nothing ends, to exercise the time-out path without faulting the device
+        const char* e = getenv("RIPPLE_DEBUG_TC_WITHHOLD");
+        c->debug_tc_withhold = e && e[0] == '1';
+    }
     arm_rebuild(c, nb);
     const bool try_graph = !wide && !c->no_graphs && !c->timing && nb >= 1 && nb <= RP_GRAPH_MAX_BATCH;
     const cudaMemcpyKind kind = mem == RIPPLE_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
@@ -504,6 +510,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
             set_err(c, st == RIPPLE_ERR_VERTEX_RANGE ? "batch rejected: vertex id or payload row out of range"
                        : st == RIPPLE_ERR_CAPACITY   ? (h.expand_failed ? "batch rejected: vertex deletions expand to more than max_batch operations"
                                                                          : "batch rejected: overflow edge pool exhausted")
+                       : st == RIPPLE_ERR_TIMEOUT    ? "a bounded device-side wait gave up; the embeddings are no longer consistent: destroy the context"
                                                      : "batch rejected: unknown op code");
             s.n_added = s.n_deleted = s.n_noop_add = s.n_noop_del = s.n_superseded = s.n_feature = s.n_expanded = 0;
             for (int l = 0; l <= L; ++l) s.affected[l] = s.senders[l] = s.active_edges[l] = 0;

@@ -108,6 +108,7 @@ struct Ctx {
     int rebuild_armed[RP_MAXL + 1];   // per hop: the rebuilding form is enqueued for this batch (see arm_rebuild)
     long long batches_done;
     int last_nb;
+    int debug_tc_withhold;   // diagnostic (environment RIPPLE_DEBUG_TC_WITHHOLD=1): see ripple_create
     int may_expand;   // the batch being enqueued may hold vertex deletions (always assumed for device batches)
     long long regather_min_messages;   // default threshold only: hops with fewer messages always push
     float regather_threshold[RP_MAXL + 1];  // per hop: share of all edges from which the hop rebuilds its aggregates

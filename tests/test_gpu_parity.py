@@ -686,3 +686,39 @@ def test_reduction_probe_runs_and_rejects_bad_arguments(env):
         with pytest.raises(ripple.RippleError) as ei:
             ripple.probe_reduction_rate(*bad)
         assert ei.value.status == ripple.ERR_INVALID_ARG
+
+
+def test_bounded_wait_reports_a_timeout_and_the_device_stays_usable(env, monkeypatch):
+    """Failure detection without a fault: the tensor-core update is told (diagnostic environment
+    switch) never to signal its first finished tile, so the epilogue's bounded wait runs out.  The
+    call must come back with RIPPLE_ERR_TIMEOUT, and the device must go on answering."""
+    ripple, Oracle = env
+    model = I.sage_model([24, 256, 256, 12], I.AGG_MEAN)
+    n = 9000
+    src, dst = I.er_graph(n, 45000, 3)
+    have = set(zip(src.tolist(), dst.tolist()))
+    extra = [(7, v) for v in range(200, 4700) if (7, v) not in have]
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    X = I.features(n, 24, 3)
+    W = I.make_weights(model, 3, zero_bias=False)
+    stream = I.UpdateStream(n, src, dst, 24, 3)
+    rp = ripple.Ripple(n, src, dst, X, model, W, max_batch=4096)
+    ups, rows = stream.next_batch(1500)
+    rp.apply_batch(ups, rows)                                   # a normal batch first
+    assert max(rp.stats()["affected"]) >= 1024                  # enough rows for the tensor-core form
+    monkeypatch.setenv("RIPPLE_DEBUG_TC_WITHHOLD", "1")
+    ups2, rows2 = stream.next_batch(1500)
+    with pytest.raises(ripple.RippleError) as ei:
+        rp.apply_batch(ups2, rows2)
+    assert ei.value.status == ripple.ERR_TIMEOUT and "wait gave up" in str(ei.value)
+    monkeypatch.delenv("RIPPLE_DEBUG_TC_WITHHOLD")
+    rp.close()
+    # the device still answers: a fresh context over the same inputs is correct
+    rp = ripple.Ripple(n, src, dst, X, model, W, max_batch=4096)
+    orc = Oracle(n, src, dst, X, model, W)
+    rp.apply_batch(ups, rows)
+    assert orc.apply_incremental(ups, rows) == 0
+    check_graph(rp, orc)
+    check_values(rp, orc.full(), 3)
+    rp.close()
