@@ -10,6 +10,17 @@ constexpr unsigned FULL = 0xffffffffu;
 
 __device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
 
+// First statement of every kernel.  The kernels of a batch are launched with programmatic stream
+// serialisation: a kernel may be scheduled while its predecessor is still running, so that launch
+// latency overlaps execution (a batch is a chain of some fifty short kernels).  The wait returns
+// once every prerequisite grid has completed and its memory operations are visible, so nothing a
+// kernel reads can be stale; the trigger then lets the successor be scheduled in turn.  Without a
+// programmatic dependency both instructions are no-ops.
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // inclusive warp scan
 template <typename T>
 __device__ __forceinline__ T warp_inclusive_scan(T x) {

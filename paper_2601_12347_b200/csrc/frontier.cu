@@ -26,6 +26,7 @@ __device__ __forceinline__ int scan_count(const int* n_dev, int n_host) { return
 
 __global__ void k_scan_tiles(const int32_t* __restrict__ list, const int* n_dev, int n_host,
                              const int32_t* __restrict__ deg, int64_t* tile_sums) {
+    pdl_enter();
     __shared__ int64_t scratch[33];
     int n = scan_count(n_dev, n_host);
     int n_tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
@@ -45,6 +46,7 @@ __global__ void k_scan_tiles(const int32_t* __restrict__ list, const int* n_dev,
 
 __global__ void k_scan_tile_sums(const int* n_dev, int n_host, int64_t* tile_sums, int64_t* out,
                                  unsigned long long* total_dev) {
+    pdl_enter();
     __shared__ int64_t scratch[33];
     int n = scan_count(n_dev, n_host);
     int n_tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
@@ -66,6 +68,7 @@ __global__ void k_scan_tile_sums(const int* n_dev, int n_host, int64_t* tile_sum
 __global__ void k_scan_write(const int32_t* __restrict__ list, const int* n_dev, int n_host,
                              const int32_t* __restrict__ deg, const int64_t* __restrict__ tile_sums,
                              int64_t* out) {
+    pdl_enter();
     __shared__ int64_t scratch[33];
     int n = scan_count(n_dev, n_host);
     int n_tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
@@ -106,6 +109,7 @@ void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, con
 constexpr int CMP_T = 256;  // one word per thread
 
 __global__ void k_bitmap_tile_counts(const uint32_t* __restrict__ bitmap, int n_words, int* tile_cnt) {
+    pdl_enter();
     __shared__ int scratch[33];
     int w = blockIdx.x * CMP_T + threadIdx.x;
     int pc = w < n_words ? __popc(bitmap[w]) : 0;
@@ -117,6 +121,7 @@ __global__ void k_bitmap_tile_counts(const uint32_t* __restrict__ bitmap, int n_
 __global__ void k_bitmap_compact(uint32_t* bitmap, int n_words, const int* __restrict__ tile_cnt,
                                  int32_t* list, int* count_out, const int32_t* __restrict__ deg_in,
                                  unsigned long long* pull_work) {
+    pdl_enter();
     __shared__ int scratch[33];
     __shared__ int tile_base;
     __shared__ unsigned long long work;
@@ -174,6 +179,7 @@ constexpr int WALK_CHUNK = 256;  // edges per warp work item
 __global__ void k_mark_frontier(Ctl* ctl, int l, int self_term, int walk, const int32_t* __restrict__ senders,
                                 const int64_t* __restrict__ coff, Side out, const Rec* __restrict__ rec,
                                 const int32_t* __restrict__ A_prev, uint32_t* bitmap) {
+    pdl_enter();
     if (ctl->abort) return;
     const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gsize = gridDim.x * blockDim.x;
     // sinks of net edge changes are affected at every hop
@@ -213,6 +219,7 @@ constexpr int BU_LANES = 4, BU_FIRST = 64;
 __global__ void __launch_bounds__(256)
 k_mark_bottom_up(Ctl* ctl, int l, int N, Side in, const int32_t* __restrict__ posmap, uint32_t* bitmap,
                  int32_t* overflow, int* n_overflow) {
+    pdl_enter();
     if (ctl->abort || !ctl->regather[l]) return;
     const int gtid = blockIdx.x * blockDim.x + threadIdx.x, groups = (gridDim.x * blockDim.x) / BU_LANES;
     const int sub = threadIdx.x & (BU_LANES - 1);
@@ -238,6 +245,7 @@ k_mark_bottom_up(Ctl* ctl, int l, int N, Side in, const int32_t* __restrict__ po
 __global__ void __launch_bounds__(256)
 k_mark_bottom_up_long(Ctl* ctl, int l, Side in, const int32_t* __restrict__ posmap, uint32_t* bitmap,
                       const int32_t* __restrict__ overflow, const int* __restrict__ n_overflow) {
+    pdl_enter();
     if (ctl->abort || !ctl->regather[l]) return;
     const int n = *n_overflow;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -282,6 +290,7 @@ void frontier_compact(Ctx* c, int l) {
 // ---------------------------------------------------------------------------------------------
 __global__ void k_senders_from_affected(Ctl* ctl, int l, const int32_t* __restrict__ A, int32_t* senders,
                                         int32_t* posmap) {
+    pdl_enter();
     if (ctl->abort) return;
     int n = ctl->nA[l];
     if (blockIdx.x == 0 && threadIdx.x == 0) ctl->nC[l] = n;
@@ -293,6 +302,7 @@ __global__ void k_senders_from_affected(Ctl* ctl, int l, const int32_t* __restri
 }
 
 __global__ void k_senders_release(Ctl* ctl, int l, const int32_t* __restrict__ senders, int32_t* posmap) {
+    pdl_enter();
     int n = ctl->nC[l];
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
         posmap[senders[i]] = -1;

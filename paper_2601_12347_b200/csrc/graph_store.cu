@@ -25,6 +25,7 @@ namespace rp {
 // ---------------------------------------------------------------------------------------------
 __global__ void k_count_degrees(const int32_t* __restrict__ src, const int32_t* __restrict__ dst,
                                 int64_t E, int N, int32_t* deg_out, int32_t* deg_in, Ctl* ctl) {
+    pdl_enter();
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < E;
          e += (int64_t)gridDim.x * blockDim.x) {
         int u = src[e], v = dst[e];
@@ -38,6 +39,7 @@ __global__ void k_count_degrees(const int32_t* __restrict__ src, const int32_t* 
 }
 
 __global__ void k_capacities(int N, const int32_t* __restrict__ deg, int32_t* cap, float slack) {
+    pdl_enter();
     int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v >= N) return;
     int d = deg[v];
@@ -47,6 +49,7 @@ __global__ void k_capacities(int N, const int32_t* __restrict__ deg, int32_t* ca
 
 __global__ void k_fill_rows(const int32_t* __restrict__ src, const int32_t* __restrict__ dst,
                             int64_t E, int N, Side out, Side in) {
+    pdl_enter();
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < E;
          e += (int64_t)gridDim.x * blockDim.x) {
         int u = src[e], v = dst[e];
@@ -114,6 +117,7 @@ __device__ __forceinline__ int ops_total(const Ctl* ctl) {
 // last-operation-wins rule orders them against the explicit operations on the same pairs.
 __global__ void k_expand_plan(const ripple_update* __restrict__ ups, int N, long long capacity, Ctl* ctl,
                               Side out, Side in, int2* vjobs) {
+    pdl_enter();
     const int n = ctl->n_ops;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
         const ripple_update op = ups[i];
@@ -132,6 +136,7 @@ __global__ void k_expand_plan(const ripple_update* __restrict__ ups, int N, long
 
 __global__ void k_expand_copy(ripple_update* ups, int32_t* op_seq, Ctl* ctl, Side out, Side in,
                               const int2* __restrict__ vjobs) {
+    pdl_enter();
     if (ctl->abort) return;
     const int nj = ctl->n_vjobs;
     for (int j = blockIdx.x; j < nj; j += gridDim.x) {
@@ -153,6 +158,7 @@ __global__ void k_expand_copy(ripple_update* ups, int32_t* op_seq, Ctl* ctl, Sid
 __global__ void k_classify(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, int N,
                            Ctl* ctl, unsigned long long* hkeys, unsigned long long* hwin, int hmask,
                            int32_t* op_slot, int32_t* feat_last, int32_t* vdel_seq) {
+    pdl_enter();
     const int n = ops_total(ctl), n_given = ctl->n_ops;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
         ripple_update op = ups[i];
@@ -235,6 +241,7 @@ k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_
           const unsigned long long* __restrict__ hwin, const int32_t* __restrict__ op_slot,
           const int32_t* __restrict__ feat_last, const int32_t* __restrict__ vdel_seq, Side out, Side in,
           Rec* rec, uint32_t* bitmap) {
+    pdl_enter();
     __shared__ int s_found;
     if (ctl->abort) return;
     const int n = ops_total(ctl), n_given = ctl->n_ops;
@@ -285,6 +292,7 @@ __device__ __forceinline__ int grown_capacity(int cap, int need) {
 // Rows whose additions do not fit: list them and add up the pool entries they will take.
 __global__ void k_plan_growth(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
                               int32_t* grow_out, int32_t* grow_in) {
+    pdl_enter();
     if (ctl->abort) return;
     int n = ctl->n_rec;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * n; i += gridDim.x * blockDim.x) {
@@ -303,6 +311,7 @@ __global__ void k_plan_growth(Ctl* ctl, const Rec* __restrict__ rec, Side out, S
 }
 
 __global__ void k_plan_check(Ctl* ctl, long long col_size_out, long long col_size_in) {
+    pdl_enter();
     if (ctl->abort) return;
     if (ctl->pool_next[0] + ctl->pool_need[0] > (unsigned long long)col_size_out ||
         ctl->pool_next[1] + ctl->pool_need[1] > (unsigned long long)col_size_in) {
@@ -341,6 +350,7 @@ void graph_batch_classify(Ctx* c, int n) {
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * n_; i += gridDim.x * blockDim.x)
 
 __global__ void k_del_mark(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
+    pdl_enter();
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -353,6 +363,7 @@ __global__ void k_del_mark(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side
 }
 
 __global__ void k_del_tail_read(Ctl* ctl, Rec* rec, Side out, Side in) {
+    pdl_enter();
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -366,6 +377,7 @@ __global__ void k_del_tail_read(Ctl* ctl, Rec* rec, Side out, Side in) {
 }
 
 __global__ void k_del_tail_pack(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
+    pdl_enter();
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -380,6 +392,7 @@ __global__ void k_del_tail_pack(Ctl* ctl, const Rec* __restrict__ rec, Side out,
 }
 
 __global__ void k_del_fill(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
+    pdl_enter();
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -397,6 +410,7 @@ __global__ void k_del_fill(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side
 // One warp per growing row: take a block from the pool, move the row, double its capacity.
 __global__ void k_grow_rows(Ctl* ctl, Side out, Side in, const int32_t* __restrict__ grow_out,
                             const int32_t* __restrict__ grow_in) {
+    pdl_enter();
     if (ctl->abort) return;
     int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -419,6 +433,7 @@ __global__ void k_grow_rows(Ctl* ctl, Side out, Side in, const int32_t* __restri
 }
 
 __global__ void k_add_write(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
+    pdl_enter();
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -433,6 +448,7 @@ __global__ void k_add_write(Ctl* ctl, const Rec* __restrict__ rec, Side out, Sid
 
 __global__ void k_commit_degrees(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
                                  int32_t* deg_out_old) {
+    pdl_enter();
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -468,6 +484,7 @@ __global__ void k_cleanup(const ripple_update* __restrict__ ups, int N, Ctl* ctl
                           const Rec* __restrict__ rec, Side out, Side in, unsigned long long* hkeys,
                           unsigned long long* hwin, const int32_t* __restrict__ op_slot, int32_t* feat_last,
                           int32_t* vdel_seq, int32_t* deg_out_old, uint32_t* bitmap) {
+    pdl_enter();
     const int n_rec = ctl->n_rec, n = ops_total(ctl);
     if (blockIdx.x == 0 && threadIdx.x == 0 && !ctl->abort) ctl->num_edges += ctl->n_add - ctl->n_del;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < max(n, n_rec); i += gridDim.x * blockDim.x) {
@@ -502,6 +519,7 @@ void graph_batch_cleanup(Ctx* c, int n) {
 // canonical export (parity checks)
 // ---------------------------------------------------------------------------------------------
 __global__ void k_export_rows(int N, Side out, const int64_t* __restrict__ rowptr, int32_t* col) {
+    pdl_enter();
     int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int nwarps = (gridDim.x * blockDim.x) >> 5;
     for (int v = warp; v < N; v += nwarps) {

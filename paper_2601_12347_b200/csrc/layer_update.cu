@@ -16,6 +16,7 @@ constexpr int BM = 64, BN = 64, BK = 16, TM = 4, TN = 4;
 
 __global__ void __launch_bounds__(256)
 k_update_rows(const Ctl* ctl, UpdParams p) {
+    pdl_enter();
     if (ctl->abort) return;
     __shared__ __align__(16) float As[BK][BM + 4];
     __shared__ __align__(16) float Bs[BK][BN];
@@ -90,6 +91,7 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
 // elementwise (bias + cached terms + activation); one thread per 16-byte piece of a row
 __global__ void __launch_bounds__(256)
 k_update_rows_elementwise(const Ctl* ctl, UpdParams p) {
+    pdl_enter();
     if (ctl->abort) return;
     const int n = upd_rows(p), nq = p.n_cols >> 2;
     const long long total = (long long)n * nq;
@@ -231,6 +233,7 @@ __global__ void k_feature_rows(Ctl* ctl, const ripple_update* __restrict__ ups, 
                                int d0, const int32_t* __restrict__ A0, const int32_t* __restrict__ feat_last,
                                int src_norm, const int32_t* __restrict__ deg_out,
                                const int32_t* __restrict__ deg_out_old, float* H0, int ld, float* D, int keep_old) {
+    pdl_enter();
     if (ctl->abort) return;
     const int n = ctl->nA[0];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -266,6 +269,7 @@ void feature_rows(Ctx* c, int n) {
 __global__ void k_extra_senders(Ctl* ctl, int l, const Rec* __restrict__ rec, int32_t* senders,
                                 int32_t* posmap, const int32_t* __restrict__ deg_out,
                                 const float* __restrict__ H, int ld, float* D) {
+    pdl_enter();
     if (ctl->abort) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;

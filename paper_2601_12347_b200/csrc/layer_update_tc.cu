@@ -135,6 +135,7 @@ constexpr int TC_SLAB_LD = TC_SLAB + 4;    // 20 floats: 16-byte stores of 8 con
 template <bool X3>
 __global__ void __launch_bounds__(TC_ALL_THREADS, 1)
 k_update_rows_tc(Ctl* ctl, UpdParams p) {
+    pdl_enter();
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full[TC_STAGES], empty[TC_STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;

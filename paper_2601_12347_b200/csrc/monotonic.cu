@@ -127,6 +127,7 @@ __global__ void __launch_bounds__(256)
 k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const int* n_dev, int n_host, Side in,
            const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA, int32_t* long_rows,
            int* n_long, uint32_t* invmask, int mw, int is_min) {
+    pdl_enter();
     if (ctl->abort) return;
     const int n = n_dev ? *n_dev : n_host;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -203,6 +204,7 @@ __global__ void __launch_bounds__(256)
 k_max_long_rows(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const int* __restrict__ n_long, Side in,
                 const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA, uint32_t* invmask,
                 int mw, int is_min) {
+    pdl_enter();
     extern __shared__ float part[];   // 8 warps x ld floats
     __shared__ int s_differs;
     if (ctl->abort) return;
@@ -292,6 +294,7 @@ k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32
                const int64_t* __restrict__ coff, Side out, Side in, const float* __restrict__ Hprev,
                const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR,
                uint32_t* invmask, int mw, int is_min) {
+    pdl_enter();
     if (ctl->abort) return;
     const int nC = ctl->nC[l - 1];
     if (nC == 0) return;
@@ -370,6 +373,7 @@ __global__ void k_max_records(Ctl* ctl, const Rec* __restrict__ rec, Side in, co
                               const int32_t* __restrict__ old_idx, const float* __restrict__ Hprev,
                               const float* __restrict__ Old, int ld, float* S, uint32_t* bitmapA, uint32_t* bitmapR,
                               uint32_t* invmask, int mw, int is_min) {
+    pdl_enter();
     if (ctl->abort) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -410,6 +414,7 @@ __global__ void k_max_records(Ctl* ctl, const Rec* __restrict__ rec, Side in, co
 
 // self term: a vertex whose own previous-layer row changed recomputes its embedding as well
 __global__ void k_max_mark_self(Ctl* ctl, int l, const int32_t* __restrict__ senders, uint32_t* bitmapA) {
+    pdl_enter();
     if (ctl->abort) return;
     const int n = ctl->nC[l - 1];
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) mark_bit(bitmapA, senders[i]);
@@ -420,6 +425,7 @@ __global__ void k_max_mark_self(Ctl* ctl, int l, const int32_t* __restrict__ sen
 __global__ void k_max_senders(Ctl* ctl, int l, const int32_t* __restrict__ A, const float* __restrict__ H,
                               const float* __restrict__ Old, int ld, int32_t* senders, int32_t* old_idx,
                               int32_t* posmap) {
+    pdl_enter();
     if (ctl->abort) return;
     const int n = ctl->nA[l];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;

@@ -1,5 +1,6 @@
 // C ABI of the ripple library: argument checks, device state set-up, and the per-batch launch
 // chain.  See include/ripple.h for the contract of every entry point.
+#include "device_utils.cuh"
 #include "ripple_internal.cuh"
 
 #include <algorithm>
@@ -43,6 +44,7 @@ static cudaError_t dev_alloc(T** p, size_t count, int fill_byte = -2) {
 // params[0] = number of ops, params[1] = number of payload rows (device memory, so that a captured
 // launch chain can be replayed for batches that differ in them)
 __global__ void k_ctl_reset(Ctl* ctl, const int* params) {
+    pdl_enter();
     unsigned long long keep0 = ctl->pool_next[0], keep1 = ctl->pool_next[1];
     Ctl z;
     memset(&z, 0, sizeof(Ctl));
@@ -181,6 +183,10 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         CK(dev_alloc(&c->params_dev, 2, 0));
         CK(cudaMallocHost(&c->params_host, 2 * sizeof(int)));
         c->no_graphs = o.no_graphs;
+        {
+            const char* e = getenv("RIPPLE_NO_PDL");
+            c->pdl = !(e && e[0] == '1');
+        }
         tc_prepare();
         max_prepare();
         CK(cudaMallocHost(&c->ctl_host, sizeof(Ctl)));

@@ -109,6 +109,7 @@ struct Ctx {
     long long batches_done;
     int last_nb;
     int debug_tc_withhold;   // diagnostic (environment RIPPLE_DEBUG_TC_WITHHOLD=1): see ripple_create
+    int pdl;                 // launch with programmatic stream serialisation (off: environment RIPPLE_NO_PDL=1)
     int may_expand;   // the batch being enqueued may hold vertex deletions (always assumed for device batches)
     long long regather_min_messages;   // default threshold only: hops with fewer messages always push
     float regather_threshold[RP_MAXL + 1];  // per hop: share of all edges from which the hop rebuilds its aggregates
@@ -176,10 +177,22 @@ struct Ctx {
 inline int div_up(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 inline int pad4(int x) { return (x + 3) & ~3; }
 
-#define RP_LAUNCH(ctx, kernel, grid, block, smem, ...)                         \
-    do {                                                                        \
-        kernel<<<(grid), (block), (smem), (ctx)->stream>>>(__VA_ARGS__);        \
-        (ctx)->launches++;                                                      \
+// Every kernel of the library goes through this: programmatic stream serialisation (see pdl_enter)
+// unless switched off for the context.
+#define RP_LAUNCH(ctx, kernel, grid, block, smem, ...)                                            \
+    do {                                                                                           \
+        cudaLaunchConfig_t cfg_ = {};                                                              \
+        cfg_.gridDim = dim3((unsigned)(grid));                                                     \
+        cfg_.blockDim = dim3((unsigned)(block));                                                   \
+        cfg_.dynamicSmemBytes = (size_t)(smem);                                                    \
+        cfg_.stream = (ctx)->stream;                                                               \
+        cudaLaunchAttribute attr_[1];                                                              \
+        attr_[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                          \
+        attr_[0].val.programmaticStreamSerializationAllowed = 1;                                   \
+        cfg_.attrs = attr_;                                                                        \
+        cfg_.numAttrs = (ctx)->pdl ? 1 : 0;                                                        \
+        cudaLaunchKernelEx(&cfg_, kernel, __VA_ARGS__);                                            \
+        (ctx)->launches++;                                                                         \
     } while (0)
 
 // dispatch on row width: ld <= 32 floats -> 8 lanes per row, <= 64 -> 16, else whole warp

@@ -100,6 +100,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_spmm_pull(int N, Side in, const int32_t* __restrict__ deg_out, int src_norm,
             const float* __restrict__ M, int ld, float* __restrict__ S, int2* items, int* n_items) {
+    pdl_enter();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
     const int sub = lane / LPR, ql = lane % LPR;
@@ -132,6 +133,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_spmm_hubs(Side in, const int32_t* __restrict__ deg_out, int src_norm, const float* __restrict__ M, int ld,
             float* S, const int2* __restrict__ items, const int* __restrict__ n_items) {
+    pdl_enter();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
     const int sub = lane / LPR, ql = lane % LPR;
@@ -185,6 +187,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_scatter_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64_t* __restrict__ coff,
                Side out, const float* __restrict__ D, int ld, float* S, uint32_t* bitmap) {
+    pdl_enter();
     if (ctl->abort || ctl->pull[l] || ctl->regather[l]) return;
     const int nC = ctl->nC[l - 1];
     if (nC == 0) return;
@@ -246,6 +249,7 @@ template <int NQ>
 __global__ void __launch_bounds__(256)
 k_scatter_push_packed(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64_t* __restrict__ coff,
                       Side out, const float* __restrict__ D, float* S, uint32_t* bitmap) {
+    pdl_enter();
     constexpr int LCM = NQ == 12 ? 96 : NQ == 10 ? 160 : NQ * 32;
     constexpr int NI = LCM / 32, G = LCM / NQ, LD = NQ * 4;
     if (ctl->abort || ctl->pull[l] || ctl->regather[l]) return;
@@ -300,6 +304,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_scatter_pull(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_t* __restrict__ posmap,
                const float* __restrict__ D, int ld, float* S) {
+    pdl_enter();
     if (ctl->abort || !ctl->pull[l] || ctl->regather[l]) return;
     const int nA = ctl->nA[l];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -351,6 +356,7 @@ k_scatter_pull(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const in
 __global__ void k_record_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, int src_norm,
                               const int32_t* __restrict__ deg_out, const int32_t* __restrict__ posmap,
                               const float* __restrict__ Hprev, const float* __restrict__ D, int ld, float* M) {
+    pdl_enter();
     if (ctl->abort || ctl->regather[l]) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -376,6 +382,7 @@ __global__ void k_record_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, int 
 // S_v += sign * M_r for every record r (row width = inbox width)
 __global__ void k_scatter_records(Ctl* ctl, int l, const Rec* __restrict__ rec, const float* __restrict__ M,
                                   int ld, float* S) {
+    pdl_enter();
     if (ctl->abort || ctl->regather[l]) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -399,6 +406,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_regather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_t* __restrict__ deg_out,
            int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, int2* items, int* n_items) {
+    pdl_enter();
     if (ctl->abort || !ctl->regather[l]) return;
     const int nA = ctl->nA[l];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -439,6 +447,7 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int32_t* __restrict__ deg_out,
                 int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, float* __restrict__ dS) {
+    pdl_enter();
     if (ctl->abort || ctl->regather[l]) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -481,6 +490,7 @@ k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int
 // form is throughput-bound, and the edge-balanced push is the more parallel of the two (measured
 // on the sparse graph, 256 floats per row: 0.24 ms pushed, 0.26 to 0.47 ms rebuilt).
 __global__ void k_choose_direction(Ctl* ctl, int l, int mode, float threshold, long long min_messages) {
+    pdl_enter();
     const int nC = ctl->nC[l - 1];
     int re = 0;
     if (mode == RIPPLE_SCATTER_REGATHER) re = 1;
@@ -500,6 +510,7 @@ __global__ void k_choose_direction(Ctl* ctl, int l, int mode, float threshold, l
 // the aggregate's magnitude, and the error random-walks with the number of messages (measured
 // drift 1e-4 of the value after 100 batches).  Folding keeps it at one rounding per row and batch.
 __global__ void k_fold_deltas(Ctl* ctl, int l, const int32_t* __restrict__ A, int ld, float* S, float* dS) {
+    pdl_enter();
     if (ctl->abort || ctl->regather[l]) return;   // a rebuilt aggregate has no pending sums
     const int n = ctl->nA[l];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -600,6 +611,7 @@ void regather_layer(Ctx* c, int l) {
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 k_probe_reductions(float* buf, long long n_rows, int nq, long long n_messages, unsigned long long seed) {
+    pdl_enter();
     const long long total = n_messages * nq;
     for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total;
          t += (long long)gridDim.x * blockDim.x) {
