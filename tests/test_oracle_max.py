@@ -245,3 +245,25 @@ def test_min_is_the_mirror_image_of_max():
     assert omin.apply_incremental(P.ups_array(recs), rows) == 0
     assert np.array_equal(omax.H(1), omin.H(1)) and np.array_equal(omax.S(1), -omin.S(1))
     assert np.array_equal(omax.affected(1), omin.affected(1))
+
+
+@pytest.mark.parametrize("agg", AGGS, ids=["max", "min"])
+def test_scoped_recompute_route_agrees_for_monotonic_aggregators(agg):
+    """The scoped route (Sec. 3.2) recomputes every structurally reachable vertex; its embeddings must
+    equal full recomputation, and its affected sets must contain the pruned ones of the hybrid route."""
+    m = max_model([6, 8, 4], agg)
+    n = 40
+    src, dst = P.random_graph(n, 150, 8)
+    X = I.features(n, 6, 8)
+    W = I.make_weights(m, 8, zero_bias=False)
+    a, b = Oracle(n, src, dst, X, m, W), Oracle(n, src, dst, X, m, W)
+    stream = I.UpdateStream(n, src, dst, 6, 8)
+    for _ in range(6):
+        ups, rows = stream.next_batch(5)
+        assert a.apply_incremental(ups, rows) == 0
+        assert b.apply_scoped(ups, rows) == 0
+        full = a.full()
+        for l in range(3):
+            assert P.rel_err(a.H(l), full[l]) < 1e-12 and P.rel_err(b.H(l), full[l]) < 1e-12
+        for l in range(1, 3):
+            assert set(a.affected(l).tolist()) <= set(b.affected(l).tolist())
