@@ -136,7 +136,7 @@ k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const in
     for (int i = warp; i < n; i += nwarps) {
         const int v = list ? list[i] : i;
         const int deg = in.deg[v];
-        if (deg > MAX_HUB_DEGREE) {
+        if (deg > (mode ? MAX_HUB_DEGREE : 4 * MAX_HUB_DEGREE)) {   // a full pass has rows enough to keep every warp busy
             if (lane == 0) long_rows[atomicAdd(n_long, 1)] = v;
             continue;
         }
@@ -446,7 +446,7 @@ __global__ void k_max_senders(Ctl* ctl, int l, const int32_t* __restrict__ A, co
 static void launch_long_rows(Ctx* c, int mode, const float* M, int ld, float* S, int32_t* long_rows, int* n_long) {
     const int nv = div_up(ld, 128);
     const size_t smem = (size_t)8 * std::max(ld, MAX_EL) * sizeof(float);
-#define LONG(NV) RP_LAUNCH(c, k_max_long_rows<NV>, c->n_sm, 256, smem, c->ctl, mode, long_rows, n_long, c->side[1], M, ld, S, c->bitmap, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
+#define LONG(NV) RP_LAUNCH(c, k_max_long_rows<NV>, c->n_sm * 8, 256, smem, c->ctl, mode, long_rows, n_long, c->side[1], M, ld, S, c->bitmap, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
     if (nv <= 1) LONG(1); else if (nv <= 2) LONG(2); else if (nv <= 4) LONG(4); else LONG(8);
 #undef LONG
 }
