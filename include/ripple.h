@@ -139,7 +139,8 @@ typedef struct {
                              layer's output width; for equal widths only where nothing but that product
                              would be left per affected row: SAGE, GRAPHCONV); 1: never, aggregates
                              always hold input-width rows                                                */
-    int32_t no_graphs;    /* non-zero: never replay small batches (<= 512 updates) as a captured CUDA graph     */
+    int32_t no_graphs;    /* non-zero: never replay small batches (<= 512 updates; a batch size is captured
+                             the second time it is seen) as a CUDA graph                                  */
     int32_t device;       /* CUDA device ordinal, or -1 for the current device                              */
     void* stream;         /* cudaStream_t to run on (NULL: the library creates its own)                     */
     float regather_threshold; /* AUTO only: a hop rebuilds its aggregates once its messages number at least

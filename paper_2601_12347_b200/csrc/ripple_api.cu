@@ -438,6 +438,17 @@ static bool launch_batch_graph(Ctx* c, int nb) {
     for (int i = 0; i < RP_GRAPH_SLOTS; ++i)
         if (c->graph_exec[i] && c->graph_n[i] == key) slot = i;
     if (slot < 0) {
+        // Capturing costs a millisecond or more: only a chain that keeps coming back is worth it.  A
+        // stream whose batch sizes never repeat is launched kernel by kernel.
+        int seen = -1;
+        for (int i = 0; i < RP_GRAPH_SEEN; ++i)
+            if (c->seen_key[i] == key) seen = i;
+        if (seen < 0) {
+            seen = c->seen_next++ % RP_GRAPH_SEEN;
+            c->seen_key[seen] = key;
+            c->seen_count[seen] = 0;
+        }
+        if (++c->seen_count[seen] < 2) return false;
         slot = c->graph_next++ % RP_GRAPH_SLOTS;
         if (c->graph_exec[slot]) { cudaGraphExecDestroy(c->graph_exec[slot]); c->graph_exec[slot] = nullptr; }
         cudaGraph_t g = nullptr;

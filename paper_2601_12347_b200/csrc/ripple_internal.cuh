@@ -15,6 +15,7 @@
 #define RP_TOMB (-1)
 #define RP_GRAPH_MAX_BATCH 512   // batches up to this size replay a captured launch chain
 #define RP_GRAPH_SLOTS 8
+#define RP_GRAPH_SEEN 32    // recently seen chain keys: a chain is captured at its second appearance
 
 namespace rp {
 
@@ -163,6 +164,9 @@ struct Ctx {
     int graph_n[RP_GRAPH_SLOTS];
     int64_t graph_launches[RP_GRAPH_SLOTS];
     int graph_next;
+    int seen_key[RP_GRAPH_SEEN];
+    int seen_count[RP_GRAPH_SEEN];
+    int seen_next;
     Ctl* ctl;        // device
     Ctl* ctl_host;   // pinned
     ripple_stats stats;

@@ -105,6 +105,10 @@ def test_hub_deletion_and_recreation(env, mem):
     # deleted again together with a neighbour, with edge operations on both sides of the deletions
     apply([(I.OP_ADD_EDGE, hub, 7), (I.OP_DEL_VERTEX, hub, 0), (I.OP_DEL_VERTEX, 5, 0), (I.OP_ADD_EDGE, hub, 9),
            (I.OP_DEL_VERTEX, hub, 0), (I.OP_ADD_EDGE, 5, hub)])
+    # three more batches of three operations: a chain is captured at its second appearance and
+    # replayed from the third on, here with a vertex deletion inside the replayed batch
+    apply([(I.OP_ADD_EDGE, 20, 21), (I.OP_DEL_VERTEX, 30, 0), (I.OP_SET_FEATURE, 31, 0)])
+    apply([(I.OP_ADD_EDGE, 22, 23), (I.OP_DEL_VERTEX, 32, 0), (I.OP_SET_FEATURE, 33, 1)])
     rp.close()
 
 
