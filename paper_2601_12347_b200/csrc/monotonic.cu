@@ -60,17 +60,32 @@ __device__ __forceinline__ void max_accumulate(float4 (&acc)[NV], const Side& in
     for (int j0 = j_begin; j0 < j_end; j0 += 32) {
         const int mine = j0 + lane < j_end ? in.col[base + j0 + lane] : 0;
         const int cnt = min(32, j_end - j0);
-        for (int j = 0; j < cnt; j += EPI) {
-            const int jj = j + sub;
-            const int u = __shfl_sync(FULL, mine, jj & 31);
-            if (jj < cnt) {
-                const float4* row = reinterpret_cast<const float4*>(M + (size_t)u * ld);
+        constexpr int UNR = 4;   // neighbour rows in flight per lane group
+        for (int j = 0; j < cnt; j += UNR * EPI) {
+            int u[UNR];
+            float4 x[UNR][NV];
+#pragma unroll
+            for (int t = 0; t < UNR; ++t) {
+                const int jj = j + t * EPI + sub;
+                u[t] = __shfl_sync(FULL, mine, jj & 31);
+                if (jj >= cnt) u[t] = -1;
+            }
+#pragma unroll
+            for (int t = 0; t < UNR; ++t) {
+                const float4* row = reinterpret_cast<const float4*>(M + (size_t)max(u[t], 0) * ld);
 #pragma unroll
                 for (int k = 0; k < NV; ++k) {
                     const int q = ql + LPR * k;
-                    if (q < nq) acc[k] = pick4(acc[k], __ldg(row + q), is_min);
+                    if (u[t] >= 0 && q < nq) x[t][k] = __ldg(row + q);
                 }
             }
+#pragma unroll
+            for (int t = 0; t < UNR; ++t)
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    const int q = ql + LPR * k;
+                    if (u[t] >= 0 && q < nq) acc[k] = pick4(acc[k], x[t][k], is_min);
+                }
         }
     }
 #pragma unroll
