@@ -122,3 +122,28 @@ def test_self_term_with_a_monotonic_aggregator(env, dims, agg):
                 yield stream.next_batch(bs)
 
     run(env, n, src, dst, model, 11, batches, max_batch=4096)
+
+
+@pytest.mark.parametrize("batch", [100, 1000])
+def test_sparse_gcx_100_consecutive_batches(env, batch):
+    """The GC-X workload on the sparse graph: 100 consecutive batches, affected lists and counters
+    exact after every batch, embeddings and cached maxima within tolerance every 25 batches."""
+    ripple, Oracle = env
+    w = I.workloads()["sparse-gcx"]
+    src, dst = I.make_graph(w)
+    X = I.features(w.n, w.model.dims[0], w.seed)
+    W = I.make_weights(w.model, w.seed)
+    L = len(w.model.layers)
+    rp = ripple.Ripple(w.n, src, dst, X, w.model, W)
+    orc = Oracle(w.n, src, dst, X, w.model, W)
+    stream = I.make_stream(w, src, dst)
+    for b in range(100):
+        ups, rows = stream.next_batch(batch)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        G.check_frontiers(rp, orc, L)
+        if b % 25 == 24:
+            G.check_graph(rp, orc)
+            G.check_values(rp, [orc.H(l) for l in range(L + 1)], L, [None] + [orc.S(l) for l in range(1, L + 1)])
+    G.check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+    rp.close()
