@@ -534,6 +534,8 @@ void fold_deltas(Ctx* c, int l) {
 }
 
 void choose_direction(Ctx* c, int l) {
+    // nothing to decide for a pushing hop: the control block's flags are already zero after its reset
+    if (!c->rebuild_armed[l] && (c->scatter_mode == RIPPLE_SCATTER_AUTO || c->scatter_mode == RIPPLE_SCATTER_PUSH)) return;
     RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode,
               c->rebuild_armed[l] ? c->regather_threshold[l] : -1.f, c->regather_min_messages);
 }
