@@ -431,6 +431,8 @@ def workloads() -> Dict[str, Workload]:
         # GraphConv with max (the paper's GC-X workload, Sec. 6.1): hybrid-incremental propagation
         "sparse-gcx": Workload("sparse-gcx", n_s, e_s, "rmat", graphconv_model([128, 256, 40], AGG_MAX), 0,
                                (1, 10, 100, 1000), 100),
+        "mid-gcx-2l": Workload("mid-gcx-2l", 1_000_000, 30_000_000, "rmat", graphconv_model([100, 256, 47], AGG_MAX), 0,
+                               (1000,), 20),
         "dense-gcx-2l": Workload("dense-gcx-2l", n_d, e_d, "rmat", graphconv_model([100, 256, 47], AGG_MAX), 0,
                                  (10, 100, 1000), 20),
         # all five update types of Sec. 3.1: 2 % of the updates delete a vertex
