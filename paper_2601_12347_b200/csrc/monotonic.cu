@@ -337,14 +337,36 @@ k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32
                 hn[k] = q < nq ? __ldg(reinterpret_cast<const float4*>(Hprev + (size_t)u * ld) + q) : make_float4(0.f, 0.f, 0.f, 0.f);
                 ho[k] = q < nq ? __ldg(reinterpret_cast<const float4*>(Old + (size_t)old_idx[i] * ld) + q) : hn[k];
             }
-            for (int j = 0; j < cnt; j += EPI) {
+            // the sink of the next edge, its in-degree before the batch and its cached row are fetched
+            // while the current edge is classified (every edge is a dependent chain of loads otherwise)
+            int v_nx = 0, db_nx = 1;
+            bool live_nx = false;
+            float4 s_nx[NV];
+            auto fetch = [&](int j) {
                 const int jj = j + sub;
-                const bool live = jj < cnt;
-                const int v = live ? out.col[base + jj] : 0;
+                live_nx = jj < cnt;
+                v_nx = live_nx ? out.col[base + jj] : 0;
+                db_nx = live_nx ? deg_in_before(in, v_nx) : 1;
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    const int q = ql + LPR * k;
+                    s_nx[k] = (live_nx && db_nx != 0 && q < nq)
+                                  ? *reinterpret_cast<const float4*>(S + (size_t)v_nx * ld + 4 * q)
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            };
+            fetch(0);
+            for (int j = 0; j < cnt; j += EPI) {
+                const int v = v_nx, db = db_nx;
+                const bool live = live_nx;
+                float4 s_cur[NV];
+#pragma unroll
+                for (int k = 0; k < NV; ++k) s_cur[k] = s_nx[k];
+                if (j + EPI < cnt) fetch(j + EPI);
                 bool raise = false, invalid = false;
                 if (live) {
                     uint32_t* mask = invmask + (size_t)v * mw;
-                    if (deg_in_before(in, v) == 0) {   // zeros cached: gather the real maximum, every element
+                    if (db == 0) {   // zeros cached: gather the real maximum, every element
                         invalid = true;
                         for (int w = ql; w < mw; w += LPR) atomicOr(&mask[w], 0xffffffffu);
                     } else {
@@ -353,7 +375,7 @@ k_max_messages(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int32
                         for (int k = 0; k < NV; ++k) {
                             const int q = ql + LPR * k;
                             if (q < nq) {
-                                const float4 s = *reinterpret_cast<const float4*>(srow + 4 * q);
+                                const float4 s = s_cur[k];
                                 const float nn[4] = {hn[k].x, hn[k].y, hn[k].z, hn[k].w};
                                 const float oo[4] = {ho[k].x, ho[k].y, ho[k].z, ho[k].w};
                                 const float ss[4] = {s.x, s.y, s.z, s.w};
