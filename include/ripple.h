@@ -256,7 +256,6 @@ const char* ripple_last_error(ripple_ctx* ctx);
 
 void ripple_destroy(ripple_ctx* ctx);
 
-/* Library version string. */
 /* Diagnostic for the roofline of the push scatter (the paper has no counterpart): issues n_messages
  * rows of row_floats floats (a multiple of 4) as 16-byte vector reductions, red.global.add.v4.f32,
  * into rows drawn pseudo-randomly from a zeroed scratch window of n_rows rows, and returns the best
@@ -266,6 +265,7 @@ void ripple_destroy(ripple_ctx* ctx);
 ripple_status ripple_probe_reduction_rate(int32_t device, int64_t n_rows, int32_t row_floats,
                                           int64_t n_messages, float* ms_out);
 
+/* Library version string. */
 const char* ripple_version(void);
 
 #ifdef __cplusplus

@@ -23,8 +23,8 @@
  *   - "affected" is structural: it follows from the recurrence alone, never from values;
  *   - within a batch the last operation on a pair wins; adding an existing edge or deleting a
  *     missing one changes nothing; the last feature payload of a vertex wins;
- *   - deleting a vertex (Sec. 3.2: "a delete of all edges incident upon" it, then propagation from
- *     it as root) removes, at that point of the batch, every edge that has it as an endpoint and
+ *   - deleting a vertex (Sec. 3.2: all of its incident edges are deleted, then updates propagate
+ *     from it as root) removes, at that point of the batch, every edge that has it as an endpoint and
  *     replaces its feature row by zeros; the id stays addressable, so later operations of the same
  *     or a later batch may attach edges or features to it again (a vertex addition, which the
  *     paper models as the edge addition that creates the endpoint, Sec. 4.1);
@@ -509,8 +509,6 @@ static const srcinfo_t *source_find(const srcinfo_t *t, int n, int u) {
     return (const srcinfo_t *)bsearch(&key, t, (size_t)n, sizeof(srcinfo_t), cmp_srcinfo);
 }
 
-/* O-inc: incremental propagation of one batch (Sec. 3.3).  Returns 0, or <0 if the batch is
- * rejected (nothing changed). */
 /* ------------------------------------------------------------------------------------------ */
 /* Monotonic aggregation (Sec. 3.4.2), max (min is its mirror image: read "exceeds" as "is below"
  * and so on), for GraphConv and SAGE layers.  A message
@@ -658,6 +656,8 @@ static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *fe
     return 0;
 }
 
+/* O-inc: incremental propagation of one batch (Sec. 3.3).  Returns 0, or <0 if the batch is
+ * rejected (nothing changed). */
 int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const float *feat_rows,
                           int64_t n_rows) {
     delta_t dl;

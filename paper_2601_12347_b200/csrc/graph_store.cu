@@ -111,7 +111,7 @@ __device__ __forceinline__ int ops_total(const Ctl* ctl) {
     return ctl->n_ops + (ctl->expand_failed ? 0 : (int)ctl->n_extra);
 }
 
-// Vertex deletion (Sec. 3.2): "a delete of all edges incident upon" the vertex.  Each deletion
+// Vertex deletion (Sec. 3.2): every edge that has the vertex as an endpoint goes.  Each deletion
 // reserves room behind the caller's operations for one edge deletion per stored out- and
 // in-neighbour; the generated operations carry the deletion's position in the batch, so that the
 // last-operation-wins rule orders them against the explicit operations on the same pairs.
@@ -570,6 +570,7 @@ cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, int64_t col_capa
 // process exits.  In host code the arrays' names are host-side stand-ins, not device addresses:
 // the addresses the kernel receives come from cudaGetSymbolAddress, taken once per device.
 #include <cstdio>
+#include <cstring>
 #include <mutex>
 
 namespace rp {
@@ -622,9 +623,11 @@ extern "C" ripple_status ripple_export_graph_static(ripple_ctx* ctx, int64_t* ro
     cudaError_t e = cudaSetDevice(c->device);
     StaticScratch sc;
     if (!e) e = static_scratch(c->device, &sc);
-    // degrees land in the tail of the caller's rowptr buffer and are widened in place, front to back
-    int32_t* deg = reinterpret_cast<int32_t*>(rowptr + N + 1) - N;
-    if (!e) e = cudaMemcpyAsync(deg, c->side[0].deg, sizeof(int32_t) * (size_t)N, cudaMemcpyDeviceToHost, c->stream);
+    // degrees land, as raw bytes, in the tail of the caller's rowptr buffer and are widened in place,
+    // front to back: entry v is read (memcpy, so that no int64 object is ever read through an int32
+    // pointer) before the store to rowptr[v + 1] can reach its bytes
+    unsigned char* deg_bytes = reinterpret_cast<unsigned char*>(rowptr + N + 1) - sizeof(int32_t) * (size_t)N;
+    if (!e) e = cudaMemcpyAsync(deg_bytes, c->side[0].deg, sizeof(int32_t) * (size_t)N, cudaMemcpyDeviceToHost, c->stream);
     if (!e) e = cudaStreamSynchronize(c->stream);
     if (e) {
         snprintf(c->err, sizeof(c->err), "ripple_export_graph_static: %s", cudaGetErrorString(e));
@@ -632,8 +635,9 @@ extern "C" ripple_status ripple_export_graph_static(ripple_ctx* ctx, int64_t* ro
     }
     rowptr[0] = 0;
     for (int v = 0; v < N; ++v) {
-        int64_t d = deg[v];
-        rowptr[v + 1] = rowptr[v] + d;
+        int32_t d;
+        memcpy(&d, deg_bytes + sizeof(int32_t) * (size_t)v, sizeof(int32_t));
+        rowptr[v + 1] = rowptr[v] + (int64_t)d;
     }
     const int64_t E = rowptr[N];
     if (E > STATIC_MAX_EDGES) {

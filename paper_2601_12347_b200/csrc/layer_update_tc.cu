@@ -10,7 +10,7 @@
 // elected thread issues hi*hi + lo*hi + hi*lo (three MMAs per 8-float K step), which reproduces
 // the fp32 product to about 2^-21 relative, and commits to an mbarrier so that the stage can be
 // refilled.  With tc_mode = TC_TF32 only hi*hi is issued (plain TF32, 2^-11).  Accumulators are
-// double-buffered in tensor memory; four epilogue warps read a finished tile back with tcgen05.ld
+// double-buffered in tensor memory; eight epilogue warps read a finished tile back with tcgen05.ld
 // and run the same fused bias / activation / delta / commit code as the SIMT form while the next
 // tile's main loop is already running.
 //
@@ -265,7 +265,7 @@ k_update_rows_tc(Ctl* ctl, UpdParams p) {
             }
         };
         // asynchronous copy of step g's pre-split transposed weights (<= 128 output columns x 8 pieces
-        // of 16 bytes, hi and lo) from L2 straight into their swizzled places in stage g % 3; the MMAs
+        // of 16 bytes, hi and lo) from L2 straight into their swizzled places in stage g % TC_STAGES; the MMAs
         // that last read that stage must have finished.  Always closes one copy group.
         auto copy_b = [&](int g) {
             if (g < total_steps) {
@@ -417,7 +417,7 @@ static size_t tc_smem_bytes(bool x3) {
 
 void launch_update_tc(Ctx* c, const UpdParams& p) {
     const bool x3 = p.tc_mode == TC_TF32X3;
-    // one persistent CTA per SM: three operand stages and the epilogue slabs fill its shared memory
+    // one persistent CTA per SM: the operand stages and the epilogue slabs fill its shared memory
     const int grid = c->n_sm;
     if (x3) {
         RP_LAUNCH(c, k_update_rows_tc<true>, grid, TC_ALL_THREADS, tc_smem_bytes(true), c->ctl, p);

@@ -51,7 +51,14 @@ def test_static_export_equals_allocating_export_on_consecutive_calls(ripple):
         got_rp, got_col = rp.export_graph_static()
         assert np.array_equal(got_rp, want_rp)
         assert np.array_equal(got_col, want_col)
+        # from the second call on nothing may be allocated on the device: not by the library, and not
+        # behind its back by the CUDA runtime on its behalf (the first call may have paid one-time
+        # costs of the context, such as loading the kernel)
+        import torch
+        free_before, _ = torch.cuda.mem_get_info()
         again_rp, again_col = rp.export_graph_static()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before, "the allocation-free export changed the amount of free device memory"
         assert np.array_equal(again_rp, want_rp) and np.array_equal(again_col, want_col)
         want_src = np.repeat(np.arange(n, dtype=np.int32), np.diff(want_rp)).astype(np.int32)
         want_dst = want_col.astype(np.int32)
@@ -73,4 +80,25 @@ def test_static_export_rejects_graphs_beyond_its_limit(ripple):
     assert "262144" in str(ei.value) and "vertices" in str(ei.value)
     rowptr, col = rp.export_graph()     # the allocating entry point still serves it
     assert rowptr[-1] == 1000
+    rp.close()
+
+
+def test_static_export_rejects_too_many_edges_on_a_small_vertex_set(ripple):
+    """The second limit: few enough vertices, but more edges than the fixed column array holds."""
+    model = I.sage_model([4, 4], I.AGG_SUM)
+    n = 4096
+    u = np.repeat(np.arange(2048, dtype=np.int32), 1100)
+    v = np.tile(np.arange(1100, dtype=np.int32), 2048)
+    keep = u != v
+    src, dst = u[keep], v[keep]
+    assert n <= (1 << 18) and src.size > (1 << 21)
+    X = np.zeros((n, 4), dtype=np.float32)
+    W = I.make_weights(model, 0)
+    rp = ripple.Ripple(n, src, dst, X, model, W)
+    with pytest.raises(ripple.RippleError) as ei:
+        rp.export_graph_static()
+    assert ei.value.status == ripple.ERR_CAPACITY
+    assert "2097152" in str(ei.value) and "edges" in str(ei.value)
+    rowptr, col = rp.export_graph()
+    assert rowptr[-1] == src.size
     rp.close()
