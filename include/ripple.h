@@ -147,6 +147,15 @@ typedef struct {
                              this share of all edges.  0: default (0.5 for aggregate rows of 128 floats
                              or more, else 0.55, and never for hops of fewer than 4 Mi messages,
                              where pushing is as fast); < 0: never                       */
+    float rebuild_budget; /* A cached aggregate row is updated by one fp32 addition per batch, and each
+                             addition rounds at the magnitude the row has at that moment.  The library
+                             adds these roundings up per row (as a sum of squares, in units of one
+                             rounding of the row's largest entry) and gathers the row anew from its
+                             in-list once the total exceeds rebuild_budget roundings of the row's
+                             present largest entry: a row that keeps its size is gathered anew every
+                             rebuild_budget^2 batches that touch it, a row that lost a large term (an
+                             edge from a hub deleted) at once.  0: default (8); < 0: never.  Applies to
+                             aggregates of input-width rows and to all aggregates of RIPPLE_AGG_SUM.   */
 } ripple_options;
 
 typedef struct {
@@ -172,6 +181,8 @@ typedef struct {
     float ms_bootstrap;                           /* last ripple_create / ripple_recompute_full           */
     int64_t gpu_launches;                         /* kernels launched by the last call                    */
     int64_t n_expanded;                           /* last batch: edge deletions generated by vertex deletions */
+    int64_t rows_rebuilt[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: aggregate rows gathered anew because their
+                                                     rounding budget ran out (ripple_options.rebuild_budget) */
 } ripple_stats;
 
 /* Sec. 3.1 (preliminaries): the bootstrap embeddings exist before updates arrive.  Builds the

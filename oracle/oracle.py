@@ -42,7 +42,7 @@ def _load():
     for name in ("orc_full", "orc_bootstrap"):
         getattr(lib, name).argtypes = [vp]
         getattr(lib, name).restype = None
-    for name in ("orc_apply_incremental", "orc_apply_scoped"):
+    for name in ("orc_apply_incremental", "orc_apply_incremental_pull", "orc_apply_scoped"):
         getattr(lib, name).argtypes = [vp, vp, i64, vp, i64]
         getattr(lib, name).restype = i32
     for name in ("orc_H", "orc_S", "orc_full_H", "orc_full_S"):
@@ -127,8 +127,12 @@ class Oracle:
         feat_rows = np.ascontiguousarray(feat_rows, dtype=np.float32)
         return int(fn(self.h, ups.ctypes.data, ups.size, feat_rows.ctypes.data, feat_rows.shape[0]))
 
-    def apply_incremental(self, ups, feat_rows=None) -> int:
-        return self._apply(self.lib.orc_apply_incremental, ups, feat_rows)
+    def apply_incremental(self, ups, feat_rows=None, pull: bool = False) -> int:
+        """The incremental algorithm.  pull: messages are gathered per affected sink on all host
+        cores instead of being pushed along the senders' out-lists by one thread; only the order
+        of the additions differs."""
+        fn = self.lib.orc_apply_incremental_pull if pull else self.lib.orc_apply_incremental
+        return self._apply(fn, ups, feat_rows)
 
     def apply_scoped(self, ups, feat_rows=None) -> int:
         return self._apply(self.lib.orc_apply_scoped, ups, feat_rows)

@@ -657,9 +657,16 @@ static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *fe
 }
 
 /* O-inc: incremental propagation of one batch (Sec. 3.3).  Returns 0, or <0 if the batch is
- * rejected (nothing changed). */
-int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const float *feat_rows,
-                          int64_t n_rows) {
+ * rejected (nothing changed).
+ * pull = 0: every sender walks its out-list and adds its message to each sink's inbox, one thread
+ *           (the order in which the paper states Send and Aggregate, Sec. 3.3.1).
+ * pull = 1: the same messages, delivered the other way round: every hop-l vertex walks its in-list
+ *           and sums the messages of the senders it finds there.  Summation is order-free
+ *           (Sec. 3.3.3), every sink of a message is a hop-l vertex (A_l contains Out_new(C_{l-1})),
+ *           and no two vertices write the same inbox row, so the sinks run in parallel without
+ *           atomics.  Only the order of the additions differs from pull = 0. */
+static int apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const float *feat_rows,
+                             int64_t n_rows, int pull) {
     delta_t dl;
     int rc = normalise(o, ups, n, n_rows, &dl);
     if (rc) return rc;
@@ -690,12 +697,17 @@ int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const flo
     }
     set_list(o, 0, A, nA);
     int nC; int *C = changed_senders(o, &dl, A, nA, &nC);
+    int *sender_pos = NULL;   /* pull form: vertex -> index of its message, or -1 */
+    if (pull) {
+        sender_pos = (int *)malloc(sizeof(int) * (size_t)o->N);
+        for (int v = 0; v < o->N; ++v) sender_pos[v] = -1;
+    }
 
     for (int l = 1; l <= L; ++l) { /* one BSP superstep per hop (Sec. 3.3.1) */
         int K = o->d[l - 1], J = o->d[l];
         const double *Hp = o->H[l - 1];
         double *S = o->S[l];
-        double *m = (double *)malloc(sizeof(double) * (size_t)K);
+        double *m = (double *)malloc(sizeof(double) * (size_t)K * (size_t)(pull ? nC + 1 : 1));
         int nAn; long walked;
         int *An = next_affected(o, &dl, C, nC, A, nA, self_term, &nAn, &walked);
         o->active_edges[l] = walked + dl.n_add + dl.n_del;
@@ -712,7 +724,9 @@ int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const flo
             int has_add = 0;
             const srcinfo_t *si = source_find(srcs, nsrc, u);
             if (si) { cold = si->c_old; has_add = si->n_add > 0; }
-            for (int k = 0; k < K; ++k) m[k] = cnew * hnew[k] - cold * hold[k];
+            double *mu = pull ? m + (size_t)i * K : m;
+            for (int k = 0; k < K; ++k) mu[k] = cnew * hnew[k] - cold * hold[k];
+            if (pull) { sender_pos[u] = i; continue; }
             const ivec *r = &o->out[u];
             for (int j = 0; j < r->n; ++j) {
                 int v = r->a[j];
@@ -720,6 +734,23 @@ int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const flo
                 double *Sv = S + (size_t)v * K;
                 for (int k = 0; k < K; ++k) Sv[k] += m[k];
             }
+        }
+        if (pull) {
+#pragma omp parallel for schedule(dynamic, 64)
+            for (int i = 0; i < nAn; ++i) {
+                int v = An[i];
+                double *Sv = S + (size_t)v * K;
+                const ivec *r = &o->in[v];
+                for (int j = 0; j < r->n; ++j) {
+                    int u = r->a[j], p = sender_pos[u];
+                    if (p < 0) continue;
+                    /* an edge added by this batch carries no delta message */
+                    if (dl.n_add) { pair_t e = { u, v }; if (bsearch(&e, dl.add, (size_t)dl.n_add, sizeof(pair_t), cmp_pair)) continue; }
+                    const double *mu = m + (size_t)p * K;
+                    for (int k = 0; k < K; ++k) Sv[k] += mu[k];
+                }
+            }
+            for (int i = 0; i < nC; ++i) sender_pos[C[i]] = -1;
         }
         /* added edge: the old contribution is taken as 0, so the whole new term arrives */
         for (int i = 0; i < dl.n_add; ++i) {
@@ -754,9 +785,20 @@ int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const flo
         A = An; nA = nAn; oldA = oldAn;
         C = changed_senders(o, &dl, A, nA, &nC);
     }
-    free(A); free(oldA); free(C); free(srcs);
+    free(A); free(oldA); free(C); free(srcs); free(sender_pos);
     delta_free(&dl);
     return 0;
+}
+
+int orc_apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const float *feat_rows,
+                          int64_t n_rows) {
+    return apply_incremental(o, ups, n, feat_rows, n_rows, 0);
+}
+
+/* The incremental algorithm with Send + Aggregate in pull form on all host cores (see apply_incremental). */
+int orc_apply_incremental_pull(oracle_t *o, const update_t *ups, int64_t n, const float *feat_rows,
+                               int64_t n_rows) {
+    return apply_incremental(o, ups, n, feat_rows, n_rows, 1);
 }
 
 /* O-rc: layer-wise recompute scoped to the affected sets (Sec. 3.2): every affected vertex pulls

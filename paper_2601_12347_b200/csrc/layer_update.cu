@@ -193,7 +193,7 @@ void update_rows(Ctx* c, int l, bool full) {
     p.deg_out_old = c->deg_out_old;
     if (pre) {
         p.addend = c->S[l]; p.ld_add = c->ws[l];
-        if (!full) { p.addend_rw = c->S[l]; p.addend_delta = c->dS[l]; }   // fold_deltas is skipped for these layers
+        if (!full && c->fused_fold[l]) { p.addend_rw = c->S[l]; p.addend_delta = c->dS[l]; }   // fold_deltas is skipped for these layers
     }
     float* dout = (full || l == c->L) ? nullptr : c->D[l & 1];  // the last hop sends nothing
     p.dout_old = rp_monotonic(c->agg);

@@ -67,7 +67,7 @@ static void destroy_ctx(Ctx* c) {
         cudaFree(c->grow_list[s]); cudaFree(c->D[s]); cudaFree(c->Clist[s]);
     }
     for (int l = 0; l <= RP_MAXL; ++l) {
-        cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->Z[l]); cudaFree(c->P[l]); cudaFree(c->A[l]);
+        cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->Eb[l]); cudaFree(c->Z[l]); cudaFree(c->P[l]); cudaFree(c->A[l]);
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
         for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2, &c->layer[l].tc_self}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
@@ -107,6 +107,7 @@ static ripple_status run_full(Ctx* c) {
     for (int l = 1; l <= c->L; ++l) {
         if (rp_monotonic(c->agg)) max_full(c, l);
         else spmm_full(c, l);
+        if (c->Eb[l]) cudaMemsetAsync(c->Eb[l], 0, sizeof(float) * (size_t)c->N, c->stream);   // every row freshly gathered
         self_project(c, l, true);
         update_rows(c, l, true);
     }
@@ -177,6 +178,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         c->N = N; c->L = L; c->agg = agg; c->E0 = E;
         c->max_batch = o.max_batch;
         c->scatter_mode = o.scatter_mode; c->gemm_mode = o.gemm_mode; c->timing = o.timing;
+        c->rebuild_tau2 = o.rebuild_budget > 0.f ? o.rebuild_budget * o.rebuild_budget : 64.f;
         c->self_term = layers[0].kind != RIPPLE_LAYER_GRAPHCONV;
         c->src_norm = agg == RIPPLE_AGG_WSUM_GCN;
         CK(dev_alloc(&c->ctl, 1, 0));
@@ -254,6 +256,11 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                 c->pre[l] = o.pre_transform == 0 && !rp_monotonic(agg) &&
                             (target < ly.ld_in || (target == ly.ld_in && y.kind != RIPPLE_LAYER_GIN));
                 c->ws[l] = c->pre[l] ? target : ly.ld_in;
+                // Transformed aggregates are folded inside the update's epilogue, which sees a row in
+                // pieces and keeps no rounding budget for it.  That is left to the normalised
+                // aggregators, whose rows stay of one size; an unnormalised sum folds in a pass of its
+                // own, with the budget.
+                c->fused_fold[l] = c->pre[l] && agg != RIPPLE_AGG_SUM;
                 // measured on the dense graph: rebuilding every aggregate costs 0.47 of pushing a message
                 // along every edge at 256 floats per row (12.1 against 26 ms) and 0.54 at 48 (3.5 / 6.4 ms)
                 c->regather_min_messages = o.regather_threshold > 0.f ? 0 : (4ll << 20);
@@ -291,6 +298,8 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             CK(dev_alloc(&c->H[l], (size_t)N * c->ld[l], 0));
             if (l > 0) { CK(dev_alloc(&c->S[l], (size_t)N * c->ws[l], 0));
                          if (!rp_monotonic(agg)) CK(dev_alloc(&c->dS[l], (size_t)N * c->ws[l], 0));
+                         if (!rp_monotonic(agg) && !c->fused_fold[l] && o.rebuild_budget >= 0.f)
+                             CK(dev_alloc(&c->Eb[l], (size_t)N, 0));
                          if (c->layer[l].kind == RIPPLE_LAYER_SAGE) CK(dev_alloc(&c->Z[l], (size_t)N * c->ld[l], 0));
                          if (c->pre[l]) CK(dev_alloc(&c->P[l], (size_t)N * c->ws[l], 0)); }
             CK(dev_alloc(&c->A[l], (size_t)N + 32));
@@ -530,7 +539,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
                        : st == RIPPLE_ERR_TIMEOUT    ? "a bounded device-side wait gave up; the embeddings are no longer consistent: destroy the context"
                                                      : "batch rejected: unknown op code");
             s.n_added = s.n_deleted = s.n_noop_add = s.n_noop_del = s.n_superseded = s.n_feature = s.n_expanded = 0;
-            for (int l = 0; l <= L; ++l) s.affected[l] = s.senders[l] = s.active_edges[l] = 0;
+            for (int l = 0; l <= L; ++l) s.affected[l] = s.senders[l] = s.active_edges[l] = s.rows_rebuilt[l] = 0;
             return st;
         }
         s.n_added = h.n_add; s.n_deleted = h.n_del; s.n_noop_add = h.n_noop_add; s.n_noop_del = h.n_noop_del;
@@ -546,6 +555,7 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
             s.scatter_pull[l] = h.regather[l] ? 2 : h.pull[l];
             s.in_edges[l] = (int64_t)h.pull_work[l];
             s.message_width[l] = l ? c->ws[l] : 0;
+            s.rows_rebuilt[l] = h.n_rebuilt[l];
         }
         s.pool_used = (int64_t)h.pool_next[0] - c->side[0].base_end;
         s.pool_size = c->side[0].col_size - c->side[0].base_end;

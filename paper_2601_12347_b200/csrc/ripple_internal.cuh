@@ -43,6 +43,8 @@ struct Ctl {
     int pull[RP_MAXL + 1];
     int regather[RP_MAXL + 1];        // hop l rebuilds the aggregates of A_l from their in-lists instead of adding deltas
     int n_long[RP_MAXL + 1];          // bottom-up marking: vertices whose long in-list is scanned by a warp
+    int n_rebuilt[RP_MAXL + 1];       // aggregate rows of hop l gathered anew because their rounding budget ran out
+    int rebuild_items[RP_MAXL + 1];   // (vertex, chunk) work items of the long rows among them
     long long num_edges;              // current edge count (kept across batches)
     int work_counter[8];              // dynamic work distribution tickets (reset by the consumer)
 };
@@ -127,6 +129,9 @@ struct Ctx {
     int32_t* old_idx;          // monotonic aggregation: sender -> index of its previous row among the rows of A_{l-1}
     float* P[RP_MAXL + 1];    // cached neighbour projection W_n^T h^{l-1} of layers that transform before the scatter (N x ws_l), else null
     float* dS[RP_MAXL + 1];   // per-batch message accumulator, zero outside a batch (same shape as S)
+    float* Eb[RP_MAXL + 1];   // per vertex: rounding budget spent on S^l_v since the row was last gathered (see k_fold_deltas), or null
+    bool fused_fold[RP_MAXL + 1];   // S^l += dS^l happens inside the row update's epilogue (no budget kept)
+    float rebuild_tau2;       // square of the budget, in roundings of the row's largest entry
     float* T;          // GIN hidden rows (compact, N x ld_hid)
     float* D[2];       // delta rows, ping-pong (compact, N x max ld)
     float* Dt;         // delta rows after the neighbour transform (compact, N x max inbox width)

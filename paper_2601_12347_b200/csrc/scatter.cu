@@ -405,7 +405,8 @@ __global__ void k_scatter_records(Ctl* ctl, int l, const Rec* __restrict__ rec, 
 template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_regather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_t* __restrict__ deg_out,
-           int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, int2* items, int* n_items) {
+           int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, int2* items, int* n_items,
+           float* budget) {
     pdl_enter();
     if (ctl->abort || !ctl->regather[l]) return;
     const int nA = ctl->nA[l];
@@ -435,6 +436,7 @@ k_regather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_
                 if (q < nq) dst[q] = acc[k];
             }
         }
+        if (budget && lane == 0) budget[v] = 0.f;   // a freshly gathered row has spent nothing
     }
 }
 
@@ -446,7 +448,8 @@ k_regather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_
 template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int32_t* __restrict__ deg_out,
-                int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, float* __restrict__ dS) {
+                int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, float* __restrict__ dS,
+                float* budget) {
     pdl_enter();
     if (ctl->abort || ctl->regather[l]) return;
     const int n = ctl->n_rec;
@@ -471,6 +474,7 @@ k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int
                 if (q < nq) { dst[q] = acc[k]; pend[q] = make_float4(0.f, 0.f, 0.f, 0.f); }
             }
         }
+        if (budget && lane == 0) budget[v] = 0.f;
     }
 }
 
@@ -509,28 +513,94 @@ __global__ void k_choose_direction(Ctl* ctl, int l, int mode, float threshold, l
 // thousands of small messages per batch; adding each of them to it directly rounds every time at
 // the aggregate's magnitude, and the error random-walks with the number of messages (measured
 // drift 1e-4 of the value after 100 batches).  Folding keeps it at one rounding per row and batch.
-__global__ void k_fold_deltas(Ctl* ctl, int l, const int32_t* __restrict__ A, int ld, float* S, float* dS) {
+//
+// Even that one rounding per batch adds up, and it is taken at the magnitude the row has at the
+// time: a sink that loses the edge from a hub keeps, on its now small aggregate, the rounding of
+// the large value it held before (on the unnormalised-sum stack rows differ by four orders of
+// magnitude).  So every row keeps a budget: the sum over its folds of max|S_v|^2, in units of one
+// fp32 rounding.  Once that exceeds tau^2 max|S_v,new|^2 the row is gathered anew from its in-list
+// (Sec. 3.2's scoped recomputation, for this one row) and the budget starts again.  tau^2 is
+// scaled per vertex by a fixed factor in [0.5, 1), so that rows touched by every batch do not all
+// come due in the same batch.  Rows of at most SPMM_HUB_DEGREE in-neighbours are gathered by the
+// warp that folded them; longer ones are zeroed and queued as chunks for k_spmm_hubs.
+template <int NV, int LPR>
+__global__ void __launch_bounds__(256)
+k_fold_deltas(Ctl* ctl, int l, const int32_t* __restrict__ A, int ld, float* S, float* dS, float* budget,
+              float tau2, Side in, const int32_t* __restrict__ deg_out, int src_norm,
+              const float* __restrict__ M, int2* items) {
     pdl_enter();
     if (ctl->abort || ctl->regather[l]) return;   // a rebuilt aggregate has no pending sums
     const int n = ctl->nA[l];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
+    const int sub = lane / LPR, ql = lane % LPR;
     for (int i = warp; i < n; i += nwarps) {
-        const size_t off = (size_t)A[i] * ld;
+        const int v = A[i];
+        const size_t off = (size_t)v * ld;
         float4* s = reinterpret_cast<float4*>(S + off);
         float4* d = reinterpret_cast<float4*>(dS + off);
+        float m_old = 0.f, m_new = 0.f;
         for (int q = lane; q < nq; q += 32) {
             float4 x = s[q], y = d[q];
+            m_old = fmaxf(m_old, fmaxf(fmaxf(fabsf(x.x), fabsf(x.y)), fmaxf(fabsf(x.z), fabsf(x.w))));
             x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
+            m_new = fmaxf(m_new, fmaxf(fmaxf(fabsf(x.x), fabsf(x.y)), fmaxf(fabsf(x.z), fabsf(x.w))));
             s[q] = x;
             d[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
+        if (!budget) continue;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            m_old = fmaxf(m_old, __shfl_xor_sync(FULL, m_old, o));
+            m_new = fmaxf(m_new, __shfl_xor_sync(FULL, m_new, o));
+        }
+        const float m = fmaxf(m_old, m_new);
+        const float spent = budget[v] + m * m;
+        const float limit = tau2 * (0.5f + (float)(mix64((uint64_t)v) & 255u) * (1.0f / 512.0f)) * m_new * m_new;
+        if (!(spent > limit)) {     // also taken when anything overflowed to inf or nan: then never rebuild-loop
+            if (lane == 0) budget[v] = spent;
+            continue;
+        }
+        __syncwarp();   // the fold's stores are ordered before the gather's
+        const int deg = in.deg[v];
+        float4 acc[NV];
+#pragma unroll
+        for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (deg > SPMM_HUB_DEGREE) {
+            const int nch = (deg + SPMM_HUB_CHUNK - 1) / SPMM_HUB_CHUNK;
+            int first = 0;
+            if (lane == 0) first = atomicAdd(&ctl->rebuild_items[l], nch);
+            first = __shfl_sync(FULL, first, 0);
+            for (int ch = lane; ch < nch; ch += 32) items[first + ch] = make_int2(v, ch);
+        } else {
+            spmm_accumulate<NV, LPR>(acc, in, v, 0, deg, deg_out, src_norm, M, ld);
+        }
+        if (sub == 0) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                int q = ql + LPR * k;
+                if (q < nq) s[q] = acc[k];
+            }
+        }
+        if (lane == 0) { budget[v] = 0.f; atomicAdd(&ctl->n_rebuilt[l], 1); }
     }
 }
 
 void fold_deltas(Ctx* c, int l) {
-    if (c->pre[l]) return;   // transformed aggregates are folded inside the row update's epilogue
-    RP_LAUNCH(c, k_fold_deltas, c->n_sm * 8, 256, 0, c->ctl, l, c->A[l], c->ws[l], c->S[l], c->dS[l]);
+    if (c->fused_fold[l]) return;   // folded inside the row update's epilogue
+    const float* M = c->pre[l] ? c->P[l] : c->H[l - 1];
+    int2* items = reinterpret_cast<int2*>(c->coff);   // the degree prefix of the senders is no longer needed
+    const int ld = c->ws[l];
+#define FOLD(NV, LPR)                                                                                             \
+    do {                                                                                                           \
+        RP_LAUNCH(c, (k_fold_deltas<NV, LPR>), c->n_sm * 8, 256, 0, c->ctl, l, c->A[l], ld, c->S[l], c->dS[l],    \
+                  c->Eb[l], c->rebuild_tau2, c->side[1], c->side[0].deg, (int)c->src_norm, M, items);              \
+        if (c->Eb[l])                                                                                              \
+            RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), c->n_sm * 8, 256, 0, c->side[1], c->side[0].deg,                 \
+                      (int)c->src_norm, M, ld, c->S[l], items, &c->ctl->rebuild_items[l]);                         \
+    } while (0)
+    RP_WIDTH_DISPATCH(ld, FOLD);
+#undef FOLD
 }
 
 void choose_direction(Ctx* c, int l) {
@@ -580,7 +650,7 @@ void scatter_layer(Ctx* c, int l, int n) {
         RP_LAUNCH(c, k_scatter_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, Mm, ld,
                   c->dS[l]);
         const float* rows = c->pre[l] ? c->P[l] : c->H[l - 1];
-#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l])
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l], c->Eb[l])
         RP_WIDTH_DISPATCH(ld, ROWS);
 #undef ROWS
     }
@@ -598,7 +668,7 @@ void regather_layer(Ctx* c, int l) {
 #define REGATHER(NV, LPR)                                                                                          \
     do {                                                                                                           \
         RP_LAUNCH(c, (k_regather<NV, LPR>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->side[0].deg,           \
-                  (int)c->src_norm, M, ld, c->S[l], items, n_items);                                               \
+                  (int)c->src_norm, M, ld, c->S[l], items, n_items, c->Eb[l]);                                     \
         RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), grid, T, 0, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
                   c->S[l], items, n_items);                                                                        \
     } while (0)

@@ -58,7 +58,7 @@ class _Options(ctypes.Structure):
                 ("max_batch", ctypes.c_int64), ("scatter_mode", ctypes.c_int32),
                 ("gemm_mode", ctypes.c_int32), ("timing", ctypes.c_int32),
                 ("pre_transform", ctypes.c_int32), ("no_graphs", ctypes.c_int32), ("device", ctypes.c_int32), ("stream", ctypes.c_void_p),
-                ("regather_threshold", ctypes.c_float)]
+                ("regather_threshold", ctypes.c_float), ("rebuild_budget", ctypes.c_float)]
 
 
 class _Stats(ctypes.Structure):
@@ -74,7 +74,8 @@ class _Stats(ctypes.Structure):
                 ("pool_used", ctypes.c_int64), ("pool_size", ctypes.c_int64),
                 ("ms_total", ctypes.c_float), ("ms_graph", ctypes.c_float),
                 ("ms_frontier", _F), ("ms_scatter", _F), ("ms_update", _F),
-                ("ms_scatter_kernel", _F), ("ms_regather", _F), ("ms_bootstrap", ctypes.c_float), ("gpu_launches", ctypes.c_int64), ("n_expanded", ctypes.c_int64)]
+                ("ms_scatter_kernel", _F), ("ms_regather", _F), ("ms_bootstrap", ctypes.c_float), ("gpu_launches", ctypes.c_int64), ("n_expanded", ctypes.c_int64),
+                ("rows_rebuilt", _A)]
 
 
 _lib = None
@@ -142,7 +143,7 @@ class Ripple:
                  slack: float = 0.0, pool_edges: int = 0, max_batch: int = 0,
                  scatter_mode: int = SCATTER_AUTO, gemm_mode: int = GEMM_AUTO, timing: bool = False,
                  pre_transform: bool = True, graphs: bool = True, stream=None,
-                 regather_threshold: float = 0.0):
+                 regather_threshold: float = 0.0, rebuild_budget: float = 0.0):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -187,6 +188,7 @@ class Ripple:
         opt.pre_transform = 0 if pre_transform else 1
         opt.no_graphs = 0 if graphs else 1
         opt.regather_threshold = float(regather_threshold)
+        opt.rebuild_budget = float(rebuild_budget)
         opt.device = torch.cuda.current_device()
         self._stream = stream if stream is not None else torch.cuda.Stream()
         opt.stream = self._stream.cuda_stream
@@ -316,7 +318,7 @@ class Ripple:
                                           "n_noop_add", "n_noop_del", "n_superseded", "n_feature",
                                           "pool_used", "pool_size", "ms_total", "ms_graph",
                                           "ms_bootstrap", "gpu_launches", "n_expanded")}
-        for k in ("affected", "senders", "active_edges", "scatter_pull", "in_edges", "message_width", "ms_frontier", "ms_scatter",
+        for k in ("affected", "senders", "active_edges", "scatter_pull", "in_edges", "message_width", "rows_rebuilt", "ms_frontier", "ms_scatter",
                   "ms_update", "ms_scatter_kernel", "ms_regather"):
             out[k] = list(getattr(s, k))[: L + 1]
         return out

@@ -1,0 +1,58 @@
+"""What any fp32 evaluation of the unnormalised-sum GIN stack achieves against the fp64 oracle.
+
+The stack of the sparse-deep configuration (GIN-sum, eps = 0, 128-256-256-256 on the R-MAT graph with
+169 343 vertices) is evaluated here by its plain definition (Eq. 1-2), once, non-incrementally, in
+fp32 with NumPy / SciPy on the CPU: S = A^T H, h = W2^T relu(W1^T (h + S) + b1) + b2.  Nothing of the
+CUDA path is involved.  Its distance from the fp64 oracle is the floor that the parity tests of that
+configuration build their tolerance on (tests/tolerances.py): it pins that floor to something other
+than the CUDA path's own measurements.
+"""
+import numpy as np
+import pytest
+import scipy.sparse as sp
+
+from paper_2601_12347_b200 import inputs as I
+from oracle.oracle import Oracle
+from tolerances import GIN_FP32_FLOOR, TOL
+
+
+@pytest.fixture(scope="module")
+def gin_state():
+    w = I.workloads()["sparse-deep-gin"]
+    src, dst = I.make_graph(w)
+    X = I.features(w.n, w.model.dims[0], w.seed)
+    W = I.make_weights(w.model, w.seed)
+    orc = Oracle(w.n, src, dst, X, w.model, W)
+    return w, src, dst, X, W, orc
+
+
+def fp32_stack(w, src, dst, X, W):
+    A_t = sp.csr_matrix((np.ones(src.size, dtype=np.float32), (dst, src)), shape=(w.n, w.n))
+    H = [X.astype(np.float32)]
+    for ly, wl in zip(w.model.layers, W):
+        h = H[-1]
+        S = (A_t @ h).astype(np.float32)
+        z = np.maximum((np.float32(1.0 + ly.eps) * h + S) @ wl["Wa"] + wl["ba"], 0).astype(np.float32)
+        out = (z @ wl["Wb"] + wl["bb"]).astype(np.float32)
+        H.append(np.maximum(out, 0) if ly.act == I.ACT_RELU else out)
+    return H
+
+
+def test_fp32_floor_of_the_gin_sum_stack(gin_state):
+    w, src, dst, X, W, orc = gin_state
+    H32 = fp32_stack(w, src, dst, X, W)
+    plain, frac = [], []
+    for l in range(1, len(H32)):
+        ref = orc.H(l)
+        err = np.abs(H32[l].astype(np.float64) - ref)
+        plain.append(float(np.max(err / (1.0 + np.abs(ref)))))
+        frac.append(float(np.max(err / np.maximum(np.max(np.abs(ref), axis=1, keepdims=True), 1e-30))))
+    print("fp32 evaluation vs fp64 oracle: north_star criterion", plain, "fraction of row maximum", frac)
+    # the floor the GPU tolerance is built on: not understated, and not inflated either
+    for f in frac:
+        assert GIN_FP32_FLOOR / 4 <= f <= GIN_FP32_FLOOR, f
+    # the plain bound is out of reach of fp32 from the second layer on (rows of 3e4 and 2e6)
+    assert plain[1] > 10 * TOL and plain[2] > 50 * TOL
+    # and the reason is the row magnitude, not a bug of this evaluation: relative to the row's
+    # largest entry every layer is at a few fp32 roundings
+    assert max(frac) < 64 * 2.0 ** -24

@@ -7,10 +7,9 @@ import numpy as np
 import pytest
 
 from paper_2601_12347_b200 import inputs as I
+from tolerances import GIN_ROW_SLACK, TOL
 
 pytestmark = pytest.mark.gpu
-
-TOL = 1e-4
 
 
 @pytest.fixture(scope="module")
@@ -26,33 +25,14 @@ def env():
     return ripple, Oracle
 
 
-# Extra slack for the unnormalised-sum GIN stack, as a fraction of the largest |ref| in the row.
-# On the skewed R-MAT graph its rows grow to 1e4 (layer 2) and 1e6 (layer 3) and are all-positive
-# (sums of ReLU outputs) while the Glorot weights have mixed signs, so every one of the six matrix
-# products cancels by about sqrt(K) = 16: an element that ends up O(1) carries the rounding of
-# 1e6-sized partial sums, and any relative error already in the cached aggregate is amplified by
-# that condition number at each product.  No fp32 path can meet 1e-4 (1 + |ref|) on such elements.
-# Measured, as a fraction of the row maximum: 2e-6 right after the bootstrap; 1e-5 (B = 100) and
-# 8e-5 (B = 1000) after 100 batches, each batch adding one fresh fp32 rounding to every aggregate
-# row it touches (a random walk).  Bound: 3e-5 sqrt(1 + batches) of the row maximum.
-def gin_row_slack(n_batches):
-    return 3e-5 * float(np.sqrt(1.0 + n_batches))
-
-
-# A second effect of the same stack: when an edge from a hub is deleted, its contribution (1e4 at
-# layer 2) is subtracted from the sink's cached aggregate; what remains of a now small row carries
-# the fp32 rounding of the removed term, eps32 * 1e4 = 1e-3 absolute, whatever the row's present
-# size (measured: 1.3e-3 on a layer-3 row whose largest entry is 0.36).  This is a property of
-# incremental subtraction in fp32, not of a kernel.  Bound: 16 * 2^-24 * max |H^{l-1}|, absolute.
-def gin_abs_slack(ref_prev):
-    return 16.0 * 2.0 ** -24 * float(np.max(np.abs(ref_prev)))
-
-
-def max_err(got, ref, row_slack=0.0, abs_slack=0.0):
+# The unnormalised-sum GIN stack gets, on top of the benchmark spec bound, GIN_ROW_SLACK of the row's largest
+# |ref|: four times what a plain fp32 evaluation of the stack achieves, independent of the number of
+# batches (derivation and the CPU measurement behind it: tests/tolerances.py, tests/test_fp32_floor.py).
+def max_err(got, ref, row_slack=0.0):
     got = np.asarray(got, dtype=np.float64)
     if not ref.size:
         return 0.0
-    den = 1.0 + np.abs(ref) + abs_slack / TOL
+    den = 1.0 + np.abs(ref)
     if row_slack:
         den = den + (row_slack / TOL) * np.max(np.abs(ref), axis=1, keepdims=True)
     return float(np.max(np.abs(got - ref) / den))
@@ -87,8 +67,7 @@ def check_values(rp, refH, L, refS=None, tol=TOL, row_slack=0.0):
     lost or doubled message is an O(1) error and still fails)."""
     worst = 0.0
     for l in range(L + 1):
-        e = max_err(rp.embeddings(l).cpu().numpy(), refH[l], row_slack,
-                    gin_abs_slack(refH[l - 1]) if (row_slack and l > 0) else 0.0)
+        e = max_err(rp.embeddings(l).cpu().numpy(), refH[l], row_slack)
         assert e <= tol, f"H^{l}: max err {e}"
         worst = max(worst, e)
     if refS is not None:
@@ -104,7 +83,6 @@ def check_values(rp, refH, L, refS=None, tol=TOL, row_slack=0.0):
             den = 1.0 + np.abs(want)
             if row_slack:
                 den = den + (row_slack / TOL) * np.max(np.abs(want), axis=1, keepdims=True)
-                den = den + gin_abs_slack(refH[l - 1]) / TOL
             e = float(np.max(np.abs(got - want) / (den * scale)))
             assert e <= tol, f"S^{l}: max scaled err {e}"
     return worst
@@ -450,7 +428,7 @@ def test_sparse_config_100_consecutive_batches(env, batch):
 @pytest.mark.parametrize("wname", ["sparse-deep-gin", "sparse-deep-gcn"])
 @pytest.mark.parametrize("batch", [100, 1000])
 def test_sparse_deep_configs_100_consecutive_batches(env, wname, batch):
-    _run_workload(env, wname, batch, 100, 50, row_slack=gin_row_slack(100) if "gin" in wname else 0.0)
+    _run_workload(env, wname, batch, 100, 50, row_slack=GIN_ROW_SLACK if "gin" in wname else 0.0)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -605,6 +583,63 @@ def test_rebuilding_hops_with_long_in_lists(env):
         forms.update(rp.stats()["scatter_pull"][1:L + 1])
         check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
     assert forms == {0, 2}, forms
+    rp.close()
+
+
+def test_rounding_budget_gathers_rows_anew(env):
+    """Every fold of a batch's messages into a cached aggregate rounds at the row's magnitude of the
+    moment.  A sink that loses the edge from a vertex with a huge row keeps that rounding on its now
+    small aggregate unless the row is gathered anew; rows that are touched again and again come due
+    after a fixed number of folds, the long ones through the chunked gather."""
+    ripple, Oracle = env
+    model = I.graphconv_model([16, 24, 8], I.AGG_SUM)
+    n = 3000
+    src, dst = I.er_graph(n, 20000, 21)
+    have = set(zip(src.tolist(), dst.tolist()))
+    extra = [(7, v) for v in range(200, 700) if (7, v) not in have]            # a source with a huge row
+    extra += [(u, 9) for u in range(500, 2800) if (u, 9) not in have]          # a sink with a long in-list
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    X = I.features(n, 16, 21)
+    X[7] *= 1e6
+    W = I.make_weights(model, 21)
+    victims = [(7, v) for v in range(200, 230)]
+    ups = ups_array([(I.OP_DEL_EDGE, a, b) for a, b in victims])
+    sinks = np.array([b for _, b in victims])
+    err = {}
+    for name, budget in (("default", 0.0), ("never", -1.0)):
+        rp = ripple.Ripple(n, src, dst, X, model, W, rebuild_budget=budget)
+        orc = Oracle(n, src, dst, X, model, W)
+        rp.apply_batch(ups)
+        assert orc.apply_incremental(ups) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, 2)
+        got = rp.aggregate(1)[0].cpu().numpy().astype(np.float64)[sinks]
+        orc.full()
+        want = orc.full_S(1)[sinks]
+        err[name] = float(np.max(np.abs(got - want) / np.max(np.abs(want), axis=1, keepdims=True)))
+        if name == "default":
+            assert rp.stats()["rows_rebuilt"][1] >= len(victims)
+            check_values(rp, orc.full(), 2, [None] + [orc.full_S(l) for l in range(1, 3)])
+        else:
+            assert rp.stats()["rows_rebuilt"][1] == 0
+        rp.close()
+    assert err["default"] <= 64 * 2.0 ** -24, err            # a few roundings of the row as it now is
+    assert err["never"] > 100 * err["default"], err          # what the budget is there to prevent
+    # steady touching: with a budget of 2 roundings every touched row comes due every few batches,
+    # sink 9 (2300 in-neighbours) through the chunked gather
+    rp = ripple.Ripple(n, src, dst, X, model, W, rebuild_budget=2.0)
+    orc = Oracle(n, src, dst, X, model, W)
+    rebuilt = 0
+    for b in range(12):
+        rows = I.features(3, 16, 300 + b)
+        bu = ups_array([(I.OP_SET_FEATURE, 600 + b % 2, 0), (I.OP_SET_FEATURE, 1200, 1), (I.OP_SET_FEATURE, 2000 + b, 2)])
+        rp.apply_batch(bu, rows)
+        assert orc.apply_incremental(bu, rows) == 0
+        check_frontiers(rp, orc, 2)
+        rebuilt += sum(rp.stats()["rows_rebuilt"])
+    assert rebuilt > 12
+    check_values(rp, orc.full(), 2, [None] + [orc.full_S(l) for l in range(1, 3)])
     rp.close()
 
 

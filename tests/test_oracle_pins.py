@@ -240,8 +240,9 @@ def test_worked_example_affected_sets(route):
 # ---------------------------------------------------------------------------------------------
 # the defining invariant, every model, many batches
 # ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("pull", [False, True], ids=["push", "pull"])
 @pytest.mark.parametrize("name", list(all_models().keys()))
-def test_incremental_equals_full_recompute_every_batch(name):
+def test_incremental_equals_full_recompute_every_batch(name, pull):
     model = all_models()[name]
     n, m = 60, 400
     src, dst = random_graph(n, m, 11)
@@ -253,7 +254,7 @@ def test_incremental_equals_full_recompute_every_batch(name):
     e = m
     for b in range(12):
         ups, rows = stream.next_batch(1 + 3 * b)
-        assert inc.apply_incremental(ups, rows) == 0
+        assert inc.apply_incremental(ups, rows, pull=pull) == 0
         assert rc.apply_scoped(ups, rows) == 0
         c = inc.counts()
         e += c["added"] - c["deleted"]
@@ -278,9 +279,10 @@ def model_layers(model):
     return len(model.layers)
 
 
+@pytest.mark.parametrize("pull", [False, True], ids=["push", "pull"])
 @pytest.mark.parametrize("name", ["sage_mean", "gc_sum", "gcn_wsum", "gin"])
-@pytest.mark.parametrize("op", ["add", "del", "feat"])
-def test_single_update_rules(name, op):
+@pytest.mark.parametrize("op", ["add", "del", "feat", "feat+add+del"])
+def test_single_update_rules(name, op, pull):
     """One update per batch: added edge (old contribution 0), deleted edge (new contribution 0),
     changed vertex (new minus old) -- Sec. 3.3.3."""
     model = all_models()[name]
@@ -298,13 +300,24 @@ def test_single_update_rules(name, op):
         u, v = int(src[17]), int(dst[17])
         ups, rows = ups_array([(I.OP_DEL_EDGE, u, v)]), None
         src2, dst2, X2 = np.delete(src, 17), np.delete(dst, 17), X
-    else:
+    elif op == "feat":
         rows = I.features(1, model.dims[0], 99)
         ups = ups_array([(I.OP_SET_FEATURE, 9, 0)])
         X2 = X.copy()
         X2[9] = rows[0]
         src2, dst2 = src, dst
-    assert o.apply_incremental(ups, rows) == 0
+    else:
+        # the three rules meet at one source: its row changes, it gains an edge (the whole new term
+        # arrives, and no delta message travels along that edge) and loses one (the whole old term leaves)
+        u = int(src[17])
+        w = int(dst[17])
+        v = next(b for b in range(n) if b != u and (u, b) not in present)
+        rows = I.features(1, model.dims[0], 98)
+        ups = ups_array([(I.OP_SET_FEATURE, u, 0), (I.OP_ADD_EDGE, u, v), (I.OP_DEL_EDGE, u, w)])
+        X2 = X.copy()
+        X2[u] = rows[0]
+        src2, dst2 = np.append(np.delete(src, 17), u), np.append(np.delete(dst, 17), v)
+    assert o.apply_incremental(ups, rows, pull=pull) == 0
     ref = dense_full(n, src2.astype(np.int32), dst2.astype(np.int32), X2, model, W)
     for l in range(len(ref)):
         assert rel_err(o.H(l), ref[l]) < 1e-10, (name, op, l)

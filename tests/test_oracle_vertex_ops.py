@@ -82,7 +82,7 @@ def test_net_effect_equals_literal_replay(name, seed):
         rows = I.features(4, model.dims[0], 1000 + 10 * seed + b)
         recs = random_batch(rng, n, edges, int(rng.integers(1, 25)), 4)
         new_edges, feat = replay(edges, recs)
-        assert o.apply_incremental(P.ups_array(recs), rows) == 0
+        assert o.apply_incremental(P.ups_array(recs), rows, pull=(seed + b) % 2 == 1) == 0   # both delivery orders
         assert edges_of(o) == new_edges, (name, seed, b)
         c = o.counts()
         assert c["added"] == len(new_edges - edges) and c["deleted"] == len(edges - new_edges)

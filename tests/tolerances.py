@@ -1,0 +1,26 @@
+"""Tolerances shared by the parity tests, with where each number comes from.
+
+the benchmark spec tolerance for fp32 embeddings: max |got - ref| <= 1e-4 (1 + |ref|), ref = the oracle's fp64
+full recomputation.
+
+The unnormalised-sum GIN stack of the sparse-deep configuration cannot meet that bound with ANY fp32
+evaluation, incremental or not: on the skewed R-MAT graph its rows grow to 1e2, 3e4 and 2e6 at layers
+1, 2, 3 and are all-positive (sums of ReLU outputs) while the Glorot weights have mixed signs, so every
+matrix product cancels and an element that ends up O(1) carries the rounding of its row's largest
+partial sums.  tests/test_fp32_floor.py evaluates the stack non-incrementally in fp32 on the CPU (NumPy
+and SciPy, the plain definition, no code of the CUDA path) against the fp64 oracle: the error is
+2.0e-6 to 2.3e-6 of the row's largest |ref| at every layer, and 1.2, 17 and 130 times the benchmark spec
+bound at layers 1, 2, 3.  GIN_FP32_FLOOR is that measured floor (the test fails if the measurement leaves
+[GIN_FP32_FLOOR / 4, GIN_FP32_FLOOR]).
+
+The parity tests allow the CUDA path GIN_FLOOR_FACTOR times the floor on top of the benchmark spec bound,
+whatever the number of batches applied:
+    |got - ref| <= 1e-4 (1 + |ref|) + GIN_FLOOR_FACTOR * GIN_FP32_FLOOR * max_row |ref|
+The factor covers the difference between one fresh fp32 evaluation and a state kept incrementally
+within a bounded number of roundings of it (the library gathers an aggregate row anew once the roundings
+spent on it exceed 8 of its largest entry), and the split-TF32 products of the tensor-core update.
+"""
+TOL = 1e-4
+GIN_FP32_FLOOR = 2.5e-6
+GIN_FLOOR_FACTOR = 4.0
+GIN_ROW_SLACK = GIN_FLOOR_FACTOR * GIN_FP32_FLOOR
