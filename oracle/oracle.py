@@ -62,6 +62,8 @@ def _load():
     lib.orc_export_csr.restype = None
     lib.orc_row_from_prev.argtypes = [vp, i32, i32, vp, i64, vp, vp]
     lib.orc_row_from_prev.restype = None
+    lib.orc_rows_from_prev.argtypes = [vp, i32, vp, i64, vp, i64, vp, vp]
+    lib.orc_rows_from_prev.restype = None
     lib.orc_apply_structure.argtypes = [vp, vp, i64, i64]
     lib.orc_apply_structure.restype = i32
     lib.orc_num_threads.argtypes = []
@@ -202,4 +204,14 @@ class Oracle:
         h = np.zeros(self.dims[l], dtype=np.float64)
         self.lib.orc_row_from_prev(self.h, l, int(v), Hprev.ctypes.data, ld, S.ctypes.data,
                                    h.ctypes.data)
+        return S, h
+
+    def rows_from_prev(self, l: int, ids: np.ndarray, Hprev: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+        """row_from_prev for every vertex of ids: (S rows, h rows), fp64, in the order of ids."""
+        assert Hprev.dtype == np.float32 and Hprev.flags.c_contiguous
+        ids = np.ascontiguousarray(ids, dtype=np.int32)
+        S = np.zeros((ids.size, self.dims[l - 1]), dtype=np.float64)
+        h = np.zeros((ids.size, self.dims[l]), dtype=np.float64)
+        self.lib.orc_rows_from_prev(self.h, l, ids.ctypes.data, ids.size, Hprev.ctypes.data,
+                                    Hprev.shape[1], S.ctypes.data, h.ctypes.data)
         return S, h

@@ -891,6 +891,16 @@ void orc_row_from_prev(const oracle_t *o, int l, int v, const float *Hprev, int6
     free(hp);
 }
 
+/* The same for many rows at once (ids[0..n)), one row per thread at a time: S_out is n x d[l-1],
+ * h_out n x d[l]. */
+void orc_rows_from_prev(const oracle_t *o, int l, const int32_t *ids, int64_t n, const float *Hprev,
+                        int64_t ld, double *S_out, double *h_out) {
+    int K = o->d[l - 1], J = o->d[l];
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int64_t i = 0; i < n; ++i)
+        orc_row_from_prev(o, l, ids[i], Hprev, ld, S_out + (size_t)i * K, h_out + (size_t)i * J);
+}
+
 /* ------------------------------------------------------------------------------------------ */
 /* threads the parallel loops (full inference, the compute step) run on */
 int orc_num_threads(void) {

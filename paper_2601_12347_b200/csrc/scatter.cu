@@ -129,11 +129,117 @@ k_spmm_pull(int N, Side in, const int32_t* __restrict__ deg_out, int src_norm,
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Long in-lists: a 256-entry chunk per warp, gathered through a shared-memory ring.
+//
+// A gather is bounded by how many bytes a multiprocessor keeps in flight.  With the rows landing in
+// registers that is four rows per warp, and nothing is requested while the warp adds them up.  Here
+// every lane copies its 16-byte pieces of the next rows asynchronously (cp.async, past L1) into a
+// ring of DEPTH stages in shared memory and adds the oldest stage to its accumulators once it has
+// landed: DEPTH - 1 stages stay in flight per warp the whole time, and no register holds data
+// that is still on its way.  A lane only ever reads back what it copied itself, so the ring needs
+// no barrier, only the copy-group wait.  Stage = one row piece per lane = 32 / LPR rows per warp.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+                 "l"(gsrc)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// stages of the ring: as many as 8 KB per warp (12 KB for the widest rows) allow, and no more than
+// keep the copies within one batch of 32 neighbour ids of the additions
+template <int NV, int LPR>
+struct Ring {
+    static constexpr int EPI = 32 / LPR;
+    static constexpr int DEPTH = NV >= 8 ? 3 : NV == 4 ? 4 : NV == 2 ? 8 : EPI == 4 ? 8 : 12;
+    static constexpr int FLOAT4_PER_WARP = DEPTH * NV * 32;
+    static constexpr size_t BYTES_PER_BLOCK = (size_t)FLOAT4_PER_WARP * 16 * 8;   // 8 warps
+    static_assert((DEPTH - 1) * EPI <= 32, "copies run at most one id batch ahead of the additions");
+    // resident blocks per multiprocessor are set by the ring: fill about 200 KB of shared memory
+    static int grid(int n_sm) { return n_sm * (int)std::max<size_t>(1, std::min<size_t>(8, (200u << 10) / BYTES_PER_BLOCK)); }
+};
+
+// acc += sum over col[0 .. n) of c_u M_u, through this warp's ring
+template <int NV, int LPR>
+__device__ __forceinline__ void gather_ring(float4 (&acc)[NV], const int32_t* __restrict__ col, int n,
+                                            const int32_t* __restrict__ deg_out, int src_norm,
+                                            const float* __restrict__ M, int ld, float4* ring) {
+    constexpr int EPI = Ring<NV, LPR>::EPI, DEPTH = Ring<NV, LPR>::DEPTH;
+    const int lane = lane_id(), nq = ld >> 2;
+    const int sub = lane / LPR, ql = lane % LPR;
+    const int n_stage = (n + EPI - 1) / EPI;
+    // neighbour ids, 32 at a time: the batch being added (a), the next one (b), the one after (c)
+    int id_a = lane < n ? col[lane] : 0;
+    int id_b = 32 + lane < n ? col[32 + lane] : 0;
+    int id_c = 64 + lane < n ? col[64 + lane] : 0;
+    float cf_a = src_norm ? coef_from_degree(deg_out[id_a]) : 1.0f;
+    int base_a = 0;
+    int slot_issue = 0, slot_use = 0;
+    auto issue = [&](int s) {
+        if (s < n_stage) {
+            const int r = s * EPI + sub;
+            const int idreg = s * EPI >= base_a + 32 ? id_b : id_a;
+            const int u = __shfl_sync(FULL, idreg, r & 31);
+            if (r < n) {
+                const float4* row = reinterpret_cast<const float4*>(M + (size_t)u * ld);
+                float4* dst = ring + slot_issue * (NV * 32) + lane;
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    const int q = ql + LPR * k;
+                    if (q < nq) cp_async16(dst + 32 * k, row + q);
+                }
+            }
+        }
+        cp_async_commit();
+        slot_issue = slot_issue + 1 == DEPTH ? 0 : slot_issue + 1;
+    };
+    for (int s = 0; s < DEPTH - 1; ++s) issue(s);
+    for (int s = 0; s < n_stage; ++s) {
+        const int r0 = s * EPI;
+        if (r0 >= base_a + 32) {
+            base_a += 32;
+            id_a = id_b;
+            id_b = id_c;
+            id_c = base_a + 64 + lane < n ? col[base_a + 64 + lane] : 0;
+            if (src_norm) cf_a = coef_from_degree(deg_out[id_a]);
+        }
+        issue(s + DEPTH - 1);
+        cp_async_wait<DEPTH - 1>();
+        const int r = r0 + sub;
+        const float cu = src_norm ? __shfl_sync(FULL, cf_a, r & 31) : 1.0f;
+        if (r < n) {
+            const float4* src = ring + slot_use * (NV * 32) + lane;
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int q = ql + LPR * k;
+                if (q < nq) add4(acc[k], src[32 * k], cu);
+            }
+        }
+        slot_use = slot_use + 1 == DEPTH ? 0 : slot_use + 1;
+    }
+    // every copy that was issued has been waited for; what is still counted are empty groups
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+#pragma unroll
+        for (int o = LPR; o < 32; o <<= 1) {
+            acc[k].x += __shfl_xor_sync(FULL, acc[k].x, o);
+            acc[k].y += __shfl_xor_sync(FULL, acc[k].y, o);
+            acc[k].z += __shfl_xor_sync(FULL, acc[k].z, o);
+            acc[k].w += __shfl_xor_sync(FULL, acc[k].w, o);
+        }
+    }
+}
+
 template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_spmm_hubs(Side in, const int32_t* __restrict__ deg_out, int src_norm, const float* __restrict__ M, int ld,
             float* S, const int2* __restrict__ items, const int* __restrict__ n_items) {
     pdl_enter();
+    extern __shared__ float4 ring_all[];
+    float4* ring = ring_all + (threadIdx.x >> 5) * Ring<NV, LPR>::FLOAT4_PER_WARP;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
     const int sub = lane / LPR, ql = lane % LPR;
@@ -144,8 +250,8 @@ k_spmm_hubs(Side in, const int32_t* __restrict__ deg_out, int src_norm, const fl
         float4 acc[NV];
 #pragma unroll
         for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        spmm_accumulate<NV, LPR>(acc, in, w.x, w.y * SPMM_HUB_CHUNK, min(deg, (w.y + 1) * SPMM_HUB_CHUNK), deg_out,
-                                 src_norm, M, ld);
+        const int j0 = w.y * SPMM_HUB_CHUNK, j1 = min(deg, j0 + SPMM_HUB_CHUNK);
+        gather_ring<NV, LPR>(acc, in.col + in.start[w.x] + j0, j1 - j0, deg_out, src_norm, M, ld, ring);
         if (sub == 0) {
 #pragma unroll
             for (int k = 0; k < NV; ++k) {
@@ -154,6 +260,17 @@ k_spmm_hubs(Side in, const int32_t* __restrict__ deg_out, int src_norm, const fl
             }
         }
     }
+}
+
+// dynamic shared memory of the ring kernels (more than the default limit for wide rows): once per process
+template <int NV, int LPR>
+static void ring_prepare_one() {
+    cudaFuncSetAttribute(k_spmm_hubs<NV, LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)Ring<NV, LPR>::BYTES_PER_BLOCK);
+}
+void gather_prepare() {
+    ring_prepare_one<1, 8>(); ring_prepare_one<1, 16>(); ring_prepare_one<1, 32>();
+    ring_prepare_one<2, 32>(); ring_prepare_one<4, 32>(); ring_prepare_one<8, 32>();
 }
 
 void spmm_full(Ctx* c, int l) {
@@ -171,7 +288,7 @@ void spmm_full(Ctx* c, int l) {
     do {                                                                                                           \
         RP_LAUNCH(c, (k_spmm_pull<NV, LPR>), grid, T, 0, c->N, c->side[1], c->side[0].deg, (int)c->src_norm, M,   \
                   ld, c->S[l], items, n_items);                                                                    \
-        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), grid, T, 0, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
+        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), (Ring<NV, LPR>::grid(c->n_sm)), T, (Ring<NV, LPR>::BYTES_PER_BLOCK), c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
                   c->S[l], items, n_items);                                                                        \
     } while (0)
     RP_WIDTH_DISPATCH(ld, SPMM);
@@ -596,7 +713,7 @@ void fold_deltas(Ctx* c, int l) {
         RP_LAUNCH(c, (k_fold_deltas<NV, LPR>), c->n_sm * 8, 256, 0, c->ctl, l, c->A[l], ld, c->S[l], c->dS[l],    \
                   c->Eb[l], c->rebuild_tau2, c->side[1], c->side[0].deg, (int)c->src_norm, M, items);              \
         if (c->Eb[l])                                                                                              \
-            RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), c->n_sm * 8, 256, 0, c->side[1], c->side[0].deg,                 \
+            RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), (Ring<NV, LPR>::grid(c->n_sm)), 256, (Ring<NV, LPR>::BYTES_PER_BLOCK), c->side[1], c->side[0].deg,                 \
                       (int)c->src_norm, M, ld, c->S[l], items, &c->ctl->rebuild_items[l]);                         \
     } while (0)
     RP_WIDTH_DISPATCH(ld, FOLD);
@@ -669,7 +786,7 @@ void regather_layer(Ctx* c, int l) {
     do {                                                                                                           \
         RP_LAUNCH(c, (k_regather<NV, LPR>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->side[0].deg,           \
                   (int)c->src_norm, M, ld, c->S[l], items, n_items, c->Eb[l]);                                     \
-        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), grid, T, 0, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
+        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), (Ring<NV, LPR>::grid(c->n_sm)), T, (Ring<NV, LPR>::BYTES_PER_BLOCK), c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
                   c->S[l], items, n_items);                                                                        \
     } while (0)
     RP_WIDTH_DISPATCH(ld, REGATHER);

@@ -520,6 +520,11 @@ def test_row_from_prev_matches_full():
         for v in (0, 5, 24):
             S, h = o.row_from_prev(l, v, prev)
             assert np.allclose(h, ref[l][v], rtol=1e-5, atol=1e-6)
+        ids = np.array([24, 0, 5, 5], dtype=np.int32)     # the many-rows form returns the same rows, in order
+        Sm, hm = o.rows_from_prev(l, ids, prev)
+        for i, v in enumerate(ids):
+            S, h = o.row_from_prev(l, int(v), prev)
+            assert np.array_equal(Sm[i], S) and np.array_equal(hm[i], h)
 
 
 # ---------------------------------------------------------------------------------------------
