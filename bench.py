@@ -393,7 +393,7 @@ def run_table(args):
             O.build()
             orc = O.Oracle(w.n, src, dst, X, w.model, W)
             ostream = I.make_stream(w, src, dst, args.seed)
-        for bsz in w.batch_sizes:
+        for bsz in (args.batch_sizes or w.batch_sizes):
             nb = args.table_batches
             nt = min(20, nb)   # extra batches with per-stage event timing (small batches then run ungraphed)
             batches = [stream.next_batch(bsz) for _ in range(5 + nb + nt)]
@@ -461,6 +461,8 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--table", default="", help="comma-separated workloads: print one line per batch size")
     ap.add_argument("--table-batches", type=int, default=100)
+    ap.add_argument("--batch-sizes", type=lambda s: [int(x) for x in s.split(",")], default=None,
+                    help="--table: these batch sizes instead of the workload's own")
     ap.add_argument("--oracle-seconds", type=float, default=10.0)
     ap.add_argument("--regather-threshold", type=float, default=0.0,
                     help="share of all edges from which a hop rebuilds its aggregates (0: library default, <0: never)")

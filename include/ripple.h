@@ -122,7 +122,9 @@ typedef struct {
  * for this hop only).  AUTO: PUSH, except that a hop whose senders own at least
  * regather_threshold of all edges rebuilds. */
 typedef enum {
-    RIPPLE_SCATTER_AUTO = 0, RIPPLE_SCATTER_PUSH = 1, RIPPLE_SCATTER_PULL = 2, RIPPLE_SCATTER_REGATHER = 3
+    RIPPLE_SCATTER_AUTO = 0, RIPPLE_SCATTER_PUSH = 1, RIPPLE_SCATTER_PULL = 2, RIPPLE_SCATTER_REGATHER = 3,
+    RIPPLE_SCATTER_PUSH_BULK = 4 /* PUSH with one bulk reduction of the copy engine per message (cp.reduce.async.bulk)
+                                    instead of 16-byte vector reductions; measured equally fast */
 } ripple_scatter_mode;
 typedef enum { RIPPLE_GEMM_AUTO = 0, RIPPLE_GEMM_FP32 = 1, RIPPLE_GEMM_TF32 = 2 } ripple_gemm_mode;
 
@@ -275,6 +277,15 @@ void ripple_destroy(ripple_ctx* ctx);
  * Allocates and frees its own scratch on `device` (-1: current); touches no context. */
 ripple_status ripple_probe_reduction_rate(int32_t device, int64_t n_rows, int32_t row_floats,
                                           int64_t n_messages, float* ms_out);
+
+/* Diagnostic for the roofline of the gathering kernels (bootstrap aggregation, rebuilding hops; the
+ * paper has no counterpart): reads n_gathers whole rows of row_floats floats (a multiple of 4) from
+ * pseudo-random places of a zeroed scratch window of n_rows rows, eight rows in flight per warp, and
+ * returns the best of three timed passes in *ms_out (HOST).  Index arithmetic only, no index array: the
+ * rate is what the device's memory system gives a row gather at best -- from L2 if the window fits
+ * there, from L2 and DRAM otherwise.  Allocates and frees its own scratch on `device` (-1: current). */
+ripple_status ripple_probe_gather_rate(int32_t device, int64_t n_rows, int32_t row_floats,
+                                       int64_t n_gathers, float* ms_out);
 
 /* Library version string. */
 const char* ripple_version(void);

@@ -190,7 +190,6 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             c->pdl = !(e && e[0] == '1');
         }
         tc_prepare();
-        gather_prepare();
         max_prepare();
         CK(cudaMallocHost(&c->ctl_host, sizeof(Ctl)));
         memset(c->ctl_host, 0, sizeof(Ctl));

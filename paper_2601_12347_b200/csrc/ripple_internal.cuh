@@ -235,7 +235,6 @@ void senders_release(Ctx* c, int l);                    // clear posmap entries 
 
 // scatter.cu
 void spmm_full(Ctx* c, int l);                          // S^l for every vertex (bootstrap)
-void gather_prepare();                                  // one-time kernel attributes of the ring gathers
 void bitmap_to_list_from(Ctx* c, uint32_t* bitmap, int32_t* list, int* count_dev, unsigned long long* pull_work);
 // monotonic.cu (max aggregation, Sec. 3.4.2)
 void max_full(Ctx* c, int l);                           // bootstrap: cached maxima of every vertex

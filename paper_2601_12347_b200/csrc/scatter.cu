@@ -129,117 +129,13 @@ k_spmm_pull(int N, Side in, const int32_t* __restrict__ deg_out, int src_norm,
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// Long in-lists: a 256-entry chunk per warp, gathered through a shared-memory ring.
-//
-// A gather is bounded by how many bytes a multiprocessor keeps in flight.  With the rows landing in
-// registers that is four rows per warp, and nothing is requested while the warp adds them up.  Here
-// every lane copies its 16-byte pieces of the next rows asynchronously (cp.async, past L1) into a
-// ring of DEPTH stages in shared memory and adds the oldest stage to its accumulators once it has
-// landed: DEPTH - 1 stages stay in flight per warp the whole time, and no register holds data
-// that is still on its way.  A lane only ever reads back what it copied itself, so the ring needs
-// no barrier, only the copy-group wait.  Stage = one row piece per lane = 32 / LPR rows per warp.
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
-                 "l"(gsrc)
-                 : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-// stages of the ring: as many as 8 KB per warp (12 KB for the widest rows) allow, and no more than
-// keep the copies within one batch of 32 neighbour ids of the additions
-template <int NV, int LPR>
-struct Ring {
-    static constexpr int EPI = 32 / LPR;
-    static constexpr int DEPTH = NV >= 8 ? 3 : NV == 4 ? 4 : NV == 2 ? 8 : EPI == 4 ? 8 : 12;
-    static constexpr int FLOAT4_PER_WARP = DEPTH * NV * 32;
-    static constexpr size_t BYTES_PER_BLOCK = (size_t)FLOAT4_PER_WARP * 16 * 8;   // 8 warps
-    static_assert((DEPTH - 1) * EPI <= 32, "copies run at most one id batch ahead of the additions");
-    // resident blocks per multiprocessor are set by the ring: fill about 200 KB of shared memory
-    static int grid(int n_sm) { return n_sm * (int)std::max<size_t>(1, std::min<size_t>(8, (200u << 10) / BYTES_PER_BLOCK)); }
-};
-
-// acc += sum over col[0 .. n) of c_u M_u, through this warp's ring
-template <int NV, int LPR>
-__device__ __forceinline__ void gather_ring(float4 (&acc)[NV], const int32_t* __restrict__ col, int n,
-                                            const int32_t* __restrict__ deg_out, int src_norm,
-                                            const float* __restrict__ M, int ld, float4* ring) {
-    constexpr int EPI = Ring<NV, LPR>::EPI, DEPTH = Ring<NV, LPR>::DEPTH;
-    const int lane = lane_id(), nq = ld >> 2;
-    const int sub = lane / LPR, ql = lane % LPR;
-    const int n_stage = (n + EPI - 1) / EPI;
-    // neighbour ids, 32 at a time: the batch being added (a), the next one (b), the one after (c)
-    int id_a = lane < n ? col[lane] : 0;
-    int id_b = 32 + lane < n ? col[32 + lane] : 0;
-    int id_c = 64 + lane < n ? col[64 + lane] : 0;
-    float cf_a = src_norm ? coef_from_degree(deg_out[id_a]) : 1.0f;
-    int base_a = 0;
-    int slot_issue = 0, slot_use = 0;
-    auto issue = [&](int s) {
-        if (s < n_stage) {
-            const int r = s * EPI + sub;
-            const int idreg = s * EPI >= base_a + 32 ? id_b : id_a;
-            const int u = __shfl_sync(FULL, idreg, r & 31);
-            if (r < n) {
-                const float4* row = reinterpret_cast<const float4*>(M + (size_t)u * ld);
-                float4* dst = ring + slot_issue * (NV * 32) + lane;
-#pragma unroll
-                for (int k = 0; k < NV; ++k) {
-                    const int q = ql + LPR * k;
-                    if (q < nq) cp_async16(dst + 32 * k, row + q);
-                }
-            }
-        }
-        cp_async_commit();
-        slot_issue = slot_issue + 1 == DEPTH ? 0 : slot_issue + 1;
-    };
-    for (int s = 0; s < DEPTH - 1; ++s) issue(s);
-    for (int s = 0; s < n_stage; ++s) {
-        const int r0 = s * EPI;
-        if (r0 >= base_a + 32) {
-            base_a += 32;
-            id_a = id_b;
-            id_b = id_c;
-            id_c = base_a + 64 + lane < n ? col[base_a + 64 + lane] : 0;
-            if (src_norm) cf_a = coef_from_degree(deg_out[id_a]);
-        }
-        issue(s + DEPTH - 1);
-        cp_async_wait<DEPTH - 1>();
-        const int r = r0 + sub;
-        const float cu = src_norm ? __shfl_sync(FULL, cf_a, r & 31) : 1.0f;
-        if (r < n) {
-            const float4* src = ring + slot_use * (NV * 32) + lane;
-#pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                const int q = ql + LPR * k;
-                if (q < nq) add4(acc[k], src[32 * k], cu);
-            }
-        }
-        slot_use = slot_use + 1 == DEPTH ? 0 : slot_use + 1;
-    }
-    // every copy that was issued has been waited for; what is still counted are empty groups
-#pragma unroll
-    for (int k = 0; k < NV; ++k) {
-#pragma unroll
-        for (int o = LPR; o < 32; o <<= 1) {
-            acc[k].x += __shfl_xor_sync(FULL, acc[k].x, o);
-            acc[k].y += __shfl_xor_sync(FULL, acc[k].y, o);
-            acc[k].z += __shfl_xor_sync(FULL, acc[k].z, o);
-            acc[k].w += __shfl_xor_sync(FULL, acc[k].w, o);
-        }
-    }
-}
-
+// The chunks of the long in-lists, one warp per 256-entry chunk; chunk sums are added to the row,
+// which the kernel that queued the chunks has zeroed.
 template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_spmm_hubs(Side in, const int32_t* __restrict__ deg_out, int src_norm, const float* __restrict__ M, int ld,
             float* S, const int2* __restrict__ items, const int* __restrict__ n_items) {
     pdl_enter();
-    extern __shared__ float4 ring_all[];
-    float4* ring = ring_all + (threadIdx.x >> 5) * Ring<NV, LPR>::FLOAT4_PER_WARP;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
     const int sub = lane / LPR, ql = lane % LPR;
@@ -250,8 +146,8 @@ k_spmm_hubs(Side in, const int32_t* __restrict__ deg_out, int src_norm, const fl
         float4 acc[NV];
 #pragma unroll
         for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        const int j0 = w.y * SPMM_HUB_CHUNK, j1 = min(deg, j0 + SPMM_HUB_CHUNK);
-        gather_ring<NV, LPR>(acc, in.col + in.start[w.x] + j0, j1 - j0, deg_out, src_norm, M, ld, ring);
+        spmm_accumulate<NV, LPR>(acc, in, w.x, w.y * SPMM_HUB_CHUNK, min(deg, (w.y + 1) * SPMM_HUB_CHUNK), deg_out,
+                                 src_norm, M, ld);
         if (sub == 0) {
 #pragma unroll
             for (int k = 0; k < NV; ++k) {
@@ -260,17 +156,6 @@ k_spmm_hubs(Side in, const int32_t* __restrict__ deg_out, int src_norm, const fl
             }
         }
     }
-}
-
-// dynamic shared memory of the ring kernels (more than the default limit for wide rows): once per process
-template <int NV, int LPR>
-static void ring_prepare_one() {
-    cudaFuncSetAttribute(k_spmm_hubs<NV, LPR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                         (int)Ring<NV, LPR>::BYTES_PER_BLOCK);
-}
-void gather_prepare() {
-    ring_prepare_one<1, 8>(); ring_prepare_one<1, 16>(); ring_prepare_one<1, 32>();
-    ring_prepare_one<2, 32>(); ring_prepare_one<4, 32>(); ring_prepare_one<8, 32>();
 }
 
 void spmm_full(Ctx* c, int l) {
@@ -288,7 +173,7 @@ void spmm_full(Ctx* c, int l) {
     do {                                                                                                           \
         RP_LAUNCH(c, (k_spmm_pull<NV, LPR>), grid, T, 0, c->N, c->side[1], c->side[0].deg, (int)c->src_norm, M,   \
                   ld, c->S[l], items, n_items);                                                                    \
-        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), (Ring<NV, LPR>::grid(c->n_sm)), T, (Ring<NV, LPR>::BYTES_PER_BLOCK), c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
+        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), grid, T, 0, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
                   c->S[l], items, n_items);                                                                        \
     } while (0)
     RP_WIDTH_DISPATCH(ld, SPMM);
@@ -414,6 +299,73 @@ k_scatter_push_packed(Ctl* ctl, int l, const int32_t* __restrict__ senders, cons
     }
 }
 
+// Bulk form of the push scatter: the sender's delta row is staged in shared memory once per work
+// item, and each lane then delivers it along one out-edge with a single bulk reduction
+// (cp.reduce.async.bulk ... add.f32: the copy engine adds the whole row, 16-byte aligned, into the
+// sink's row in global memory).  One instruction per message instead of one per 16 bytes of it.
+// Measured on the dense graph it takes exactly as long as the vector-reduction form (hop 2 at 48
+// floats 1.14 against 1.12 ms, at 256 floats 6.15 against 6.18 ms): the additions are retired by
+// the L2 slices at the same rate whoever issues them, so the form is selectable
+// (RIPPLE_SCATTER_PUSH_BULK), not the default.
+// Every lane closes its bulk operations of a work item into one group; before a staging buffer
+// (two per warp) is rewritten each lane waits until its group that read the buffer has done so,
+// and before the warp leaves, until all its groups have completed.
+constexpr int PUSH_BULK_CHUNK = 128;  // edges per warp work item
+
+__device__ __forceinline__ void bulk_reduce_add_f32(float* gdst, const float* smem_src, uint32_t bytes) {
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(gdst),
+                 "r"((uint32_t)__cvta_generic_to_shared(smem_src)), "r"(bytes)
+                 : "memory");
+}
+
+__global__ void __launch_bounds__(256)
+k_scatter_push_bulk(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64_t* __restrict__ coff,
+                    Side out, const float* __restrict__ D, int ld, float* S, uint32_t* bitmap) {
+    pdl_enter();
+    extern __shared__ __align__(16) float stage_all[];
+    if (ctl->abort || ctl->pull[l] || ctl->regather[l]) return;
+    const int nC = ctl->nC[l - 1];
+    if (nC == 0) return;
+    const int64_t E = coff[nC];
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id(), nq = ld >> 2;
+    float* stage = stage_all + (size_t)(threadIdx.x >> 5) * 2 * ld;
+    int buf = 0;
+    for (int64_t e0 = (int64_t)warp * PUSH_BULK_CHUNK; e0 < E; e0 += (int64_t)nwarps * PUSH_BULK_CHUNK) {
+        const int64_t e1 = min(e0 + PUSH_BULK_CHUNK, E);
+        int i = upper_row(coff, nC, e0);
+        int64_t e = e0;
+        while (e < e1) {
+            const int64_t row_end = coff[i + 1];
+            if (row_end <= e) { ++i; continue; }
+            const int64_t seg_end = min(e1, row_end);
+            const int64_t base = out.start[senders[i]] + (e - coff[i]);
+            // this buffer was last read by the bulk operations of two segments ago
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            __syncwarp();
+            float* row = stage + (size_t)buf * ld;
+            const float4* drow = reinterpret_cast<const float4*>(D + (size_t)i * ld);
+            for (int q = lane; q < nq; q += 32) reinterpret_cast<float4*>(row)[q] = __ldg(drow + q);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the copy engine
+            __syncwarp();
+            const int cnt_total = (int)(seg_end - e);
+            for (int j0 = 0; j0 < cnt_total; j0 += 32) {
+                if (j0 + lane < cnt_total) {
+                    const int v = out.col[base + j0 + lane];
+                    const uint32_t m = 1u << (v & 31);
+                    if (!(bitmap[v >> 5] & m)) atomicOr(&bitmap[v >> 5], m);
+                    bulk_reduce_add_f32(S + (size_t)v * ld, row, (uint32_t)ld * 4u);
+                }
+            }
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            buf ^= 1;
+            e = seg_end;
+            ++i;
+        }
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
 // ---------------------------------------------------------------------------------------------
 // pull scatter
 // ---------------------------------------------------------------------------------------------
@@ -522,8 +474,8 @@ __global__ void k_scatter_records(Ctl* ctl, int l, const Rec* __restrict__ rec, 
 template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_regather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_t* __restrict__ deg_out,
-           int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, int2* items, int* n_items,
-           float* budget) {
+           int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, int2* items,
+           int* n_items, float* budget) {
     pdl_enter();
     if (ctl->abort || !ctl->regather[l]) return;
     const int nA = ctl->nA[l];
@@ -638,19 +590,16 @@ __global__ void k_choose_direction(Ctl* ctl, int l, int mode, float threshold, l
 // fp32 rounding.  Once that exceeds tau^2 max|S_v,new|^2 the row is gathered anew from its in-list
 // (Sec. 3.2's scoped recomputation, for this one row) and the budget starts again.  tau^2 is
 // scaled per vertex by a fixed factor in [0.5, 1), so that rows touched by every batch do not all
-// come due in the same batch.  Rows of at most SPMM_HUB_DEGREE in-neighbours are gathered by the
-// warp that folded them; longer ones are zeroed and queued as chunks for k_spmm_hubs.
-template <int NV, int LPR>
+// come due in the same batch.  A row that comes due is zeroed and its in-list queued, in chunks,
+// for k_spmm_hubs.
 __global__ void __launch_bounds__(256)
 k_fold_deltas(Ctl* ctl, int l, const int32_t* __restrict__ A, int ld, float* S, float* dS, float* budget,
-              float tau2, Side in, const int32_t* __restrict__ deg_out, int src_norm,
-              const float* __restrict__ M, int2* items) {
+              float tau2, const int32_t* __restrict__ deg_in, int2* items) {
     pdl_enter();
     if (ctl->abort || ctl->regather[l]) return;   // a rebuilt aggregate has no pending sums
     const int n = ctl->nA[l];
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
-    const int sub = lane / LPR, ql = lane % LPR;
     for (int i = warp; i < n; i += nwarps) {
         const int v = A[i];
         const size_t off = (size_t)v * ld;
@@ -674,32 +623,23 @@ k_fold_deltas(Ctl* ctl, int l, const int32_t* __restrict__ A, int ld, float* S, 
         const float m = fmaxf(m_old, m_new);
         const float spent = budget[v] + m * m;
         const float limit = tau2 * (0.5f + (float)(mix64((uint64_t)v) & 255u) * (1.0f / 512.0f)) * m_new * m_new;
-        if (!(spent > limit)) {     // also taken when anything overflowed to inf or nan: then never rebuild-loop
+        if (!(spent > limit)) {     // also taken if anything overflowed to inf or nan
             if (lane == 0) budget[v] = spent;
             continue;
         }
-        __syncwarp();   // the fold's stores are ordered before the gather's
-        const int deg = in.deg[v];
-        float4 acc[NV];
-#pragma unroll
-        for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (deg > SPMM_HUB_DEGREE) {
-            const int nch = (deg + SPMM_HUB_CHUNK - 1) / SPMM_HUB_CHUNK;
-            int first = 0;
-            if (lane == 0) first = atomicAdd(&ctl->rebuild_items[l], nch);
-            first = __shfl_sync(FULL, first, 0);
-            for (int ch = lane; ch < nch; ch += 32) items[first + ch] = make_int2(v, ch);
-        } else {
-            spmm_accumulate<NV, LPR>(acc, in, v, 0, deg, deg_out, src_norm, M, ld);
+        // the row comes due: zero it and queue its in-list, in chunks, for k_spmm_hubs
+        __syncwarp();
+        for (int q = lane; q < nq; q += 32) s[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        const int deg = deg_in[v];
+        const int nch = (deg + SPMM_HUB_CHUNK - 1) / SPMM_HUB_CHUNK;
+        int first = 0;
+        if (lane == 0) {
+            if (nch) first = atomicAdd(&ctl->rebuild_items[l], nch);
+            budget[v] = 0.f;
+            atomicAdd(&ctl->n_rebuilt[l], 1);
         }
-        if (sub == 0) {
-#pragma unroll
-            for (int k = 0; k < NV; ++k) {
-                int q = ql + LPR * k;
-                if (q < nq) s[q] = acc[k];
-            }
-        }
-        if (lane == 0) { budget[v] = 0.f; atomicAdd(&ctl->n_rebuilt[l], 1); }
+        first = __shfl_sync(FULL, first, 0);
+        for (int ch = lane; ch < nch; ch += 32) items[first + ch] = make_int2(v, ch);
     }
 }
 
@@ -708,21 +648,20 @@ void fold_deltas(Ctx* c, int l) {
     const float* M = c->pre[l] ? c->P[l] : c->H[l - 1];
     int2* items = reinterpret_cast<int2*>(c->coff);   // the degree prefix of the senders is no longer needed
     const int ld = c->ws[l];
-#define FOLD(NV, LPR)                                                                                             \
-    do {                                                                                                           \
-        RP_LAUNCH(c, (k_fold_deltas<NV, LPR>), c->n_sm * 8, 256, 0, c->ctl, l, c->A[l], ld, c->S[l], c->dS[l],    \
-                  c->Eb[l], c->rebuild_tau2, c->side[1], c->side[0].deg, (int)c->src_norm, M, items);              \
-        if (c->Eb[l])                                                                                              \
-            RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), (Ring<NV, LPR>::grid(c->n_sm)), 256, (Ring<NV, LPR>::BYTES_PER_BLOCK), c->side[1], c->side[0].deg,                 \
-                      (int)c->src_norm, M, ld, c->S[l], items, &c->ctl->rebuild_items[l]);                         \
-    } while (0)
-    RP_WIDTH_DISPATCH(ld, FOLD);
-#undef FOLD
+    RP_LAUNCH(c, k_fold_deltas, c->n_sm * 8, 256, 0, c->ctl, l, c->A[l], ld, c->S[l], c->dS[l], c->Eb[l],
+              c->rebuild_tau2, c->side[1].deg, items);
+    if (!c->Eb[l]) return;
+#define HUBS(NV, LPR)                                                                                              \
+    RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), c->n_sm * 8, 256, 0, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld, \
+              c->S[l], items, &c->ctl->rebuild_items[l])
+    RP_WIDTH_DISPATCH(ld, HUBS);
+#undef HUBS
 }
 
 void choose_direction(Ctx* c, int l) {
     // nothing to decide for a pushing hop: the control block's flags are already zero after its reset
-    if (!c->rebuild_armed[l] && (c->scatter_mode == RIPPLE_SCATTER_AUTO || c->scatter_mode == RIPPLE_SCATTER_PUSH)) return;
+    if (!c->rebuild_armed[l] && (c->scatter_mode == RIPPLE_SCATTER_AUTO || c->scatter_mode == RIPPLE_SCATTER_PUSH ||
+                                 c->scatter_mode == RIPPLE_SCATTER_PUSH_BULK)) return;
     RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode,
               c->rebuild_armed[l] ? c->regather_threshold[l] : -1.f, c->regather_min_messages);
 }
@@ -754,7 +693,11 @@ void scatter_layer(Ctx* c, int l, int n) {
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
 #define PUSH(NV, LPR) RP_LAUNCH(c, (k_scatter_push<NV, LPR>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, ld, c->dS[l], c->bitmap)
 #define PULL(NV, LPR) RP_LAUNCH(c, (k_scatter_pull<NV, 32>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->posmap, Dm, ld, c->dS[l])
-    if (c->scatter_mode == RIPPLE_SCATTER_AUTO || c->scatter_mode == RIPPLE_SCATTER_PUSH) {
+    // (rows too wide for two staging buffers per warp in the default shared-memory allowance take the ordinary form)
+    if (c->scatter_mode == RIPPLE_SCATTER_PUSH_BULK && (size_t)8 * 2 * ld * sizeof(float) <= (48u << 10)) {
+        RP_LAUNCH(c, k_scatter_push_bulk, grid, T, (size_t)8 * 2 * ld * sizeof(float), c->ctl, l, senders, c->coff,
+                  c->side[0], Dm, ld, c->dS[l], c->bitmap);
+    } else if (c->scatter_mode != RIPPLE_SCATTER_PULL && c->scatter_mode != RIPPLE_SCATTER_REGATHER) {
         if (ld == 48) RP_LAUNCH(c, k_scatter_push_packed<12>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
         else if (ld == 40) RP_LAUNCH(c, k_scatter_push_packed<10>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
         else RP_WIDTH_DISPATCH(ld, PUSH);
@@ -786,7 +729,7 @@ void regather_layer(Ctx* c, int l) {
     do {                                                                                                           \
         RP_LAUNCH(c, (k_regather<NV, LPR>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->side[0].deg,           \
                   (int)c->src_norm, M, ld, c->S[l], items, n_items, c->Eb[l]);                                     \
-        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), (Ring<NV, LPR>::grid(c->n_sm)), T, (Ring<NV, LPR>::BYTES_PER_BLOCK), c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
+        RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), grid, T, 0, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
                   c->S[l], items, n_items);                                                                        \
     } while (0)
     RP_WIDTH_DISPATCH(ld, REGATHER);
@@ -811,6 +754,34 @@ k_probe_reductions(float* buf, long long n_rows, int nq, long long n_messages, u
     }
 }
 
+// diagnostic: the rate at which the device serves whole rows read from pseudo-random places of a
+// window of n_rows rows, eight rows in flight per warp and nothing else going on: what a gather
+// over in-lists could reach if its indices cost nothing
+__global__ void __launch_bounds__(256)
+k_probe_gathers(const float* __restrict__ buf, long long n_rows, int nq, long long n_gathers,
+                unsigned long long seed, float* sink) {
+    pdl_enter();
+    const long long warp = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
+    const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id();
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    constexpr int UNR = 8;
+    for (long long g0 = warp * UNR; g0 < n_gathers; g0 += nwarps * UNR) {
+        for (int q0 = 0; q0 < nq; q0 += 32) {
+            float4 x[UNR];
+#pragma unroll
+            for (int t = 0; t < UNR; ++t) {
+                const long long row = (long long)(mix64((unsigned long long)(g0 + t) + seed) % (unsigned long long)n_rows);
+                const float4* p = reinterpret_cast<const float4*>(buf + (size_t)row * (4 * nq));
+                x[t] = (q0 + lane < nq && g0 + t < n_gathers) ? __ldg(p + q0 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int t = 0; t < UNR; ++t) add4(acc, x[t], 1.0f);
+        }
+    }
+    if (acc.x + acc.y + acc.z + acc.w == 12345.678f) sink[0] = acc.x;   // keeps the loads alive
+}
+
 }  // namespace rp
 
 extern "C" ripple_status ripple_probe_reduction_rate(int32_t device, int64_t n_rows, int32_t row_floats,
@@ -831,6 +802,39 @@ extern "C" ripple_status ripple_probe_reduction_rate(int32_t device, int64_t n_r
     for (int rep = 0; rep < 4; ++rep) {   // the first pass warms up
         cudaEventRecord(e0);
         rp::k_probe_reductions<<<n_sm * 8, 256>>>(buf, n_rows, row_floats / 4, n_messages, 0x9E37ull * (rep + 1));
+        cudaEventRecord(e1);
+        cudaEventSynchronize(e1);
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        if (rep > 0 && (best == 0.f || ms < best)) best = ms;
+    }
+    cudaError_t e = cudaGetLastError();
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    cudaFree(buf);
+    *ms_out = best;
+    return e == cudaSuccess ? RIPPLE_OK : RIPPLE_ERR_CUDA;
+}
+
+extern "C" ripple_status ripple_probe_gather_rate(int32_t device, int64_t n_rows, int32_t row_floats,
+                                                  int64_t n_gathers, float* ms_out) {
+    if (n_rows < 1 || row_floats < 4 || (row_floats & 3) || n_gathers < 1 || !ms_out) return RIPPLE_ERR_INVALID_ARG;
+    if (device >= 0 && cudaSetDevice(device) != cudaSuccess) return RIPPLE_ERR_CUDA;
+    float* buf = nullptr;
+    const size_t bytes = sizeof(float) * (size_t)n_rows * (size_t)row_floats;
+    if (cudaMalloc(&buf, bytes + 16) != cudaSuccess) { cudaGetLastError(); return RIPPLE_ERR_OOM; }
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0);
+    cudaEventCreate(&e1);
+    int n_sm = 1;
+    cudaGetDevice(&device);
+    cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device);
+    cudaMemset(buf, 0, bytes + 16);
+    float best = 0.f;
+    for (int rep = 0; rep < 4; ++rep) {   // the first pass warms up
+        cudaEventRecord(e0);
+        rp::k_probe_gathers<<<n_sm * 8, 256>>>(buf, n_rows, row_floats / 4, n_gathers, 0x9E37ull * (rep + 1),
+                                               buf + (size_t)n_rows * row_floats);
         cudaEventRecord(e1);
         cudaEventSynchronize(e1);
         float ms = 0.f;

@@ -13,7 +13,8 @@ from typing import Dict, List, Optional, Sequence, Tuple
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libripple.so")
+# RIPPLE_LIB_PATH: load another build of the library (kernel experiments); default: the in-tree build
+LIB_PATH = os.environ.get("RIPPLE_LIB_PATH") or os.path.join(_HERE, "libripple.so")
 
 MAX_LAYERS = 8
 OK, ERR_INVALID_ARG, ERR_VERTEX_RANGE, ERR_CAPACITY, ERR_OOM, ERR_CUDA, ERR_TIMEOUT = range(7)
@@ -22,7 +23,7 @@ AGG_SUM, AGG_MEAN, AGG_WSUM_GCN, AGG_MAX, AGG_MIN = 0, 1, 2, 3, 4
 LAYER_SAGE, LAYER_GRAPHCONV, LAYER_GIN = 0, 1, 2
 ACT_IDENTITY, ACT_RELU = 0, 1
 OP_ADD_EDGE, OP_DEL_EDGE, OP_SET_FEATURE, OP_DEL_VERTEX = 0, 1, 2, 3
-SCATTER_AUTO, SCATTER_PUSH, SCATTER_PULL, SCATTER_REGATHER = 0, 1, 2, 3
+SCATTER_AUTO, SCATTER_PUSH, SCATTER_PULL, SCATTER_REGATHER, SCATTER_PUSH_BULK = 0, 1, 2, 3, 4
 GEMM_AUTO, GEMM_FP32, GEMM_TF32 = 0, 1, 2
 
 UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
@@ -30,7 +31,7 @@ UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
 EXPORTED = [
     "ripple_create", "ripple_apply_batch", "ripple_get_embeddings", "ripple_get_aggregate",
     "ripple_get_affected", "ripple_export_graph", "ripple_get_degrees", "ripple_recompute_full",
-    "ripple_export_graph_static", "ripple_set_timing", "ripple_probe_reduction_rate",
+    "ripple_export_graph_static", "ripple_set_timing", "ripple_probe_reduction_rate", "ripple_probe_gather_rate",
     "ripple_get_stats", "ripple_last_error", "ripple_destroy", "ripple_version",
 ]
 
@@ -112,7 +113,8 @@ def load_library(path: Optional[str] = None):
     lib.ripple_export_graph_static.argtypes = [vp, vp, vp, i64]
     lib.ripple_set_timing.argtypes = [vp, i32]
     lib.ripple_probe_reduction_rate.argtypes = [i32, i64, i32, i64, P(ctypes.c_float)]
-    for name in EXPORTED[:12]:
+    lib.ripple_probe_gather_rate.argtypes = [i32, i64, i32, i64, P(ctypes.c_float)]
+    for name in EXPORTED[:13]:
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -332,6 +334,17 @@ def probe_reduction_rate(n_rows: int, row_floats: int, n_messages: int, device: 
     st = lib.ripple_probe_reduction_rate(int(device), int(n_rows), int(row_floats), int(n_messages), ctypes.byref(ms))
     if st:
         raise RippleError(st, "reduction probe failed")
+    return float(ms.value)
+
+
+def probe_gather_rate(n_rows: int, row_floats: int, n_gathers: int, device: int = -1) -> float:
+    """Milliseconds for n_gathers whole rows of row_floats floats read from pseudo-random rows of a
+    window of n_rows rows (best of three passes)."""
+    lib = load_library()
+    ms = ctypes.c_float()
+    st = lib.ripple_probe_gather_rate(int(device), int(n_rows), int(row_floats), int(n_gathers), ctypes.byref(ms))
+    if st:
+        raise RippleError(st, "gather probe failed")
     return float(ms.value)
 
 

@@ -131,7 +131,7 @@ def test_tiny_config_every_batch_against_full_recompute(env):
 
 
 @pytest.mark.parametrize("name", list(small_models().keys()))
-@pytest.mark.parametrize("mode", ["auto", "push", "pull", "push-notransform", "regather", "auto-mixed"])
+@pytest.mark.parametrize("mode", ["auto", "push", "pull", "push-notransform", "regather", "auto-mixed", "push-bulk"])
 def test_every_model_kind_and_scatter_direction(env, name, mode):
     ripple, Oracle = env
     model = small_models()[name]
@@ -148,7 +148,7 @@ def test_every_model_kind_and_scatter_direction(env, name, mode):
     W = I.make_weights(model, 3, zero_bias=False)
     sm = {"auto": ripple.SCATTER_AUTO, "push": ripple.SCATTER_PUSH, "pull": ripple.SCATTER_PULL,
           "push-notransform": ripple.SCATTER_PUSH, "regather": ripple.SCATTER_REGATHER,
-          "auto-mixed": ripple.SCATTER_AUTO}[mode]
+          "auto-mixed": ripple.SCATTER_AUTO, "push-bulk": ripple.SCATTER_PUSH_BULK}[mode]
     # auto-mixed: a hop rebuilds its aggregates once its messages reach 5 % of the edges, so that
     # pushing and rebuilding hops alternate within a batch and from batch to batch
     rp = ripple.Ripple(n, src, dst, X, model, W, scatter_mode=sm, pre_transform=mode != "push-notransform",
