@@ -271,12 +271,14 @@ void ripple_destroy(ripple_ctx* ctx);
 
 /* Diagnostic for the roofline of the push scatter (the paper has no counterpart): issues n_messages
  * rows of row_floats floats (a multiple of 4) as 16-byte vector reductions, red.global.add.v4.f32,
- * into rows drawn pseudo-randomly from a zeroed scratch window of n_rows rows, and returns the best
- * of three timed passes in *ms_out (HOST).  A window that fits L2 gives the ceiling of the on-chip
- * reduction path, a window of the size of an aggregate matrix the rate with DRAM behind it.
+ * into rows of a zeroed scratch window of n_rows rows, and returns the best of three timed passes in
+ * *ms_out (HOST).  pattern 0: uniformly random rows; 1: consecutive rows (the best case of the
+ * reduction path); 2: random rows with a popular head (position = u^3 of the window, u uniform).
+ * A window that fits L2 gives the ceiling of the on-chip reduction path, a window of the size of an
+ * aggregate matrix the rate with DRAM behind it.
  * Allocates and frees its own scratch on `device` (-1: current); touches no context. */
 ripple_status ripple_probe_reduction_rate(int32_t device, int64_t n_rows, int32_t row_floats,
-                                          int64_t n_messages, float* ms_out);
+                                          int64_t n_messages, int32_t pattern, float* ms_out);
 
 /* Diagnostic for the roofline of the gathering kernels (bootstrap aggregation, rebuilding hops; the
  * paper has no counterpart): reads n_gathers whole rows of row_floats floats (a multiple of 4) from

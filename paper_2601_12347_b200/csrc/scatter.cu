@@ -742,14 +742,23 @@ void regather_layer(Ctx* c, int l) {
 // is made of, on rows drawn pseudo-randomly from a window of n_rows rows
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-k_probe_reductions(float* buf, long long n_rows, int nq, long long n_messages, unsigned long long seed) {
+k_probe_reductions(float* buf, long long n_rows, int nq, long long n_messages, unsigned long long seed, int pattern) {
     pdl_enter();
     const long long total = n_messages * nq;
     for (long long t = blockIdx.x * (long long)blockDim.x + threadIdx.x; t < total;
          t += (long long)gridDim.x * blockDim.x) {
         const long long m = t / nq;
         const int q = (int)(t - m * nq);
-        const long long row = (long long)(mix64((unsigned long long)m + seed) % (unsigned long long)n_rows);
+        long long row;
+        if (pattern == 1) row = m % n_rows;                                    // consecutive rows
+        else {
+            const unsigned long long h = mix64((unsigned long long)m + seed);
+            row = (long long)(h % (unsigned long long)n_rows);                  // uniformly random rows
+            if (pattern == 2) {                                                 // popular rows: position = u^3
+                const double u = (double)(h >> 11) * (1.0 / 9007199254740992.0);
+                row = (long long)(u * u * u * (double)n_rows);
+            }
+        }
         red_add_v4(buf + (size_t)row * (4 * nq) + 4 * q, make_float4(1.f, 1.f, 1.f, 1.f));
     }
 }
@@ -785,7 +794,8 @@ k_probe_gathers(const float* __restrict__ buf, long long n_rows, int nq, long lo
 }  // namespace rp
 
 extern "C" ripple_status ripple_probe_reduction_rate(int32_t device, int64_t n_rows, int32_t row_floats,
-                                                     int64_t n_messages, float* ms_out) {
+                                                     int64_t n_messages, int32_t pattern, float* ms_out) {
+    if (pattern < 0 || pattern > 2) return RIPPLE_ERR_INVALID_ARG;
     if (n_rows < 1 || row_floats < 4 || (row_floats & 3) || n_messages < 1 || !ms_out) return RIPPLE_ERR_INVALID_ARG;
     if (device >= 0 && cudaSetDevice(device) != cudaSuccess) return RIPPLE_ERR_CUDA;
     float* buf = nullptr;
@@ -801,7 +811,7 @@ extern "C" ripple_status ripple_probe_reduction_rate(int32_t device, int64_t n_r
     float best = 0.f;
     for (int rep = 0; rep < 4; ++rep) {   // the first pass warms up
         cudaEventRecord(e0);
-        rp::k_probe_reductions<<<n_sm * 8, 256>>>(buf, n_rows, row_floats / 4, n_messages, 0x9E37ull * (rep + 1));
+        rp::k_probe_reductions<<<n_sm * 8, 256>>>(buf, n_rows, row_floats / 4, n_messages, 0x9E37ull * (rep + 1), pattern);
         cudaEventRecord(e1);
         cudaEventSynchronize(e1);
         float ms = 0.f;

@@ -112,7 +112,7 @@ def load_library(path: Optional[str] = None):
     lib.ripple_version.restype = ctypes.c_char_p
     lib.ripple_export_graph_static.argtypes = [vp, vp, vp, i64]
     lib.ripple_set_timing.argtypes = [vp, i32]
-    lib.ripple_probe_reduction_rate.argtypes = [i32, i64, i32, i64, P(ctypes.c_float)]
+    lib.ripple_probe_reduction_rate.argtypes = [i32, i64, i32, i64, i32, P(ctypes.c_float)]
     lib.ripple_probe_gather_rate.argtypes = [i32, i64, i32, i64, P(ctypes.c_float)]
     for name in EXPORTED[:13]:
         getattr(lib, name).restype = i32
@@ -326,12 +326,14 @@ class Ripple:
         return out
 
 
-def probe_reduction_rate(n_rows: int, row_floats: int, n_messages: int, device: int = -1) -> float:
+def probe_reduction_rate(n_rows: int, row_floats: int, n_messages: int, pattern: int = 0, device: int = -1) -> float:
     """Milliseconds for n_messages rows of row_floats floats issued as 16-byte vector reductions
-    into pseudo-random rows of a window of n_rows rows (best of three passes)."""
+    into rows of a window of n_rows rows (best of three passes).  pattern 0: uniformly random
+    rows, 1: consecutive rows, 2: random rows with a popular head."""
     lib = load_library()
     ms = ctypes.c_float()
-    st = lib.ripple_probe_reduction_rate(int(device), int(n_rows), int(row_floats), int(n_messages), ctypes.byref(ms))
+    st = lib.ripple_probe_reduction_rate(int(device), int(n_rows), int(row_floats), int(n_messages), int(pattern),
+                                         ctypes.byref(ms))
     if st:
         raise RippleError(st, "reduction probe failed")
     return float(ms.value)

@@ -716,8 +716,10 @@ def test_mixed_growth_and_deletion_in_the_same_rows(env):
 
 def test_reduction_probe_runs_and_rejects_bad_arguments(env):
     ripple, _ = env
-    assert ripple.probe_reduction_rate(1000, 48, 20000) > 0.0
-    for bad in [(0, 48, 10), (10, 6, 10), (10, 48, 0)]:
+    for pattern in (0, 1, 2):
+        assert ripple.probe_reduction_rate(1000, 48, 20000, pattern) > 0.0
+    assert ripple.probe_gather_rate(1000, 48, 20000) > 0.0
+    for bad in [(0, 48, 10), (10, 6, 10), (10, 48, 0), (10, 48, 10, 3)]:
         with pytest.raises(ripple.RippleError) as ei:
             ripple.probe_reduction_rate(*bad)
         assert ei.value.status == ripple.ERR_INVALID_ARG
