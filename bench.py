@@ -473,16 +473,20 @@ def run_table(args):
                 # the dominant kernels of a rebuilding hop: the gather over the in-lists of the affected sinks
                 # (k_regather for short lists, k_spmm_hubs for the chunks of long ones).  It is bounded by the
                 # rate at which L2 serves row gathers: achieved = in-edges x row bytes per second, peak = the
-                # library's gather probe on a window of the source matrix's size (no index traffic at all).
+                # library's gather probe (same lane layout, no index traffic at all) on an L2-resident window
+                # of 64 MB; the same probe on a window of the source matrix's size (uniformly random rows, so
+                # mostly DRAM) is reported beside it.
                 ldw = s["message_width"][L]
                 ms = hop["regather"][L] / hop["rebuilt"][L]
                 edges = hop["in_edges"][L] / hop["rebuilt"][L]
                 got = edges * ldw * 4 / 1e9 / (ms / 1e3)
-                pk = edges * ldw * 4 / 1e9 / (ripple.probe_gather_rate(w.n, ldw, int(edges)) / 1e3)
+                pk = edges * ldw * 4 / 1e9 / (ripple.probe_gather_rate(max(1, (64 << 20) // (ldw * 4)), ldw, int(edges)) / 1e3)
+                pk_big = edges * ldw * 4 / 1e9 / (ripple.probe_gather_rate(w.n, ldw, int(edges)) / 1e3)
                 per_edge = NCU_DRAM_BYTES_PER_IN_EDGE.get((name.split("-")[0], ldw))
                 line["last_hop_gather"] = {
                     "bound": "l2-gather", "kernel": f"k_regather + k_spmm_hubs (hop {L}, row width {ldw} floats)",
                     "ms": ms, "in_edges": edges, "achieved_GBps": got, "peak_GBps": pk, "frac": got / pk,
+                    "probe_uniform_rows_matrix_sized_GBps": pk_big,
                     "traffic": per_edge * edges if per_edge else None,
                     "frac_hbm": (per_edge * edges / 1e9 / (ms / 1e3) / peak) if per_edge else None}
             if orc is not None:

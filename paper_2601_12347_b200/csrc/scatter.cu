@@ -764,25 +764,29 @@ k_probe_reductions(float* buf, long long n_rows, int nq, long long n_messages, u
 }
 
 // diagnostic: the rate at which the device serves whole rows read from pseudo-random places of a
-// window of n_rows rows, eight rows in flight per warp and nothing else going on: what a gather
-// over in-lists could reach if its indices cost nothing
+// window of n_rows rows, with the lane layout of the gathering kernels (LPR lanes per row, 32 / LPR
+// rows per warp instruction), eight instructions in flight per warp and nothing else going on: what
+// a gather over in-lists could reach if its indices cost nothing
+template <int LPR>
 __global__ void __launch_bounds__(256)
-k_probe_gathers(const float* __restrict__ buf, long long n_rows, int nq, long long n_gathers,
+k_probe_gathers(const float* __restrict__ buf, unsigned long long n_rows, int nq, long long n_gathers,
                 unsigned long long seed, float* sink) {
     pdl_enter();
+    constexpr int EPI = 32 / LPR, UNR = 8;
     const long long warp = (blockIdx.x * (long long)blockDim.x + threadIdx.x) >> 5;
     const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
-    const int lane = lane_id();
+    const int lane = lane_id(), sub = lane / LPR, ql = lane % LPR;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    constexpr int UNR = 8;
-    for (long long g0 = warp * UNR; g0 < n_gathers; g0 += nwarps * UNR) {
-        for (int q0 = 0; q0 < nq; q0 += 32) {
+    for (long long g0 = warp * (UNR * EPI); g0 < n_gathers; g0 += nwarps * (UNR * EPI)) {
+        for (int q0 = 0; q0 < nq; q0 += LPR) {
             float4 x[UNR];
 #pragma unroll
             for (int t = 0; t < UNR; ++t) {
-                const long long row = (long long)(mix64((unsigned long long)(g0 + t) + seed) % (unsigned long long)n_rows);
+                const long long g = g0 + t * EPI + sub;
+                // uniform row index without a 64-bit division: high half of hash x n_rows
+                const unsigned long long row = __umul64hi(mix64((unsigned long long)g + seed), n_rows);
                 const float4* p = reinterpret_cast<const float4*>(buf + (size_t)row * (4 * nq));
-                x[t] = (q0 + lane < nq && g0 + t < n_gathers) ? __ldg(p + q0 + lane) : make_float4(0.f, 0.f, 0.f, 0.f);
+                x[t] = (q0 + ql < nq && g < n_gathers) ? __ldg(p + q0 + ql) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
             for (int t = 0; t < UNR; ++t) add4(acc, x[t], 1.0f);
@@ -843,8 +847,12 @@ extern "C" ripple_status ripple_probe_gather_rate(int32_t device, int64_t n_rows
     float best = 0.f;
     for (int rep = 0; rep < 4; ++rep) {   // the first pass warms up
         cudaEventRecord(e0);
-        rp::k_probe_gathers<<<n_sm * 8, 256>>>(buf, n_rows, row_floats / 4, n_gathers, 0x9E37ull * (rep + 1),
-                                               buf + (size_t)n_rows * row_floats);
+        const int nq = row_floats / 4;
+        float* sink = buf + (size_t)n_rows * row_floats;
+        const unsigned long long seed = 0x9E37ull * (rep + 1);
+        if (nq <= 8) rp::k_probe_gathers<8><<<n_sm * 8, 256>>>(buf, (unsigned long long)n_rows, nq, n_gathers, seed, sink);
+        else if (nq <= 16) rp::k_probe_gathers<16><<<n_sm * 8, 256>>>(buf, (unsigned long long)n_rows, nq, n_gathers, seed, sink);
+        else rp::k_probe_gathers<32><<<n_sm * 8, 256>>>(buf, (unsigned long long)n_rows, nq, n_gathers, seed, sink);
         cudaEventRecord(e1);
         cudaEventSynchronize(e1);
         float ms = 0.f;
