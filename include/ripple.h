@@ -172,7 +172,8 @@ typedef struct {
     int32_t scatter_pull[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: 0 push, 1 pull, 2 aggregates rebuilt       */
     int64_t in_edges[RIPPLE_MAX_LAYERS + 1];      /* l = 1..L: in-edges of A_l (what a gather walks)      */
     int32_t message_width[RIPPLE_MAX_LAYERS + 1]; /* l = 1..L: floats per message / aggregate row (padded) */
-    int64_t pool_used, pool_size;                 /* overflow pool, edges, out-direction                  */
+    int64_t pool_used, pool_size;                 /* overflow pool, out-direction, in edges: handed out so far
+                                                     (high-water mark of the never-used part), total size  */
     /* CUDA-event times of the last batch in milliseconds (zero unless options.timing) */
     float ms_total, ms_graph;
     float ms_frontier[RIPPLE_MAX_LAYERS + 1];
@@ -185,6 +186,10 @@ typedef struct {
     int64_t n_expanded;                           /* last batch: edge deletions generated by vertex deletions */
     int64_t rows_rebuilt[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: aggregate rows gathered anew because their
                                                      rounding budget ran out (ripple_options.rebuild_budget) */
+    int64_t pool_free, pool_lost;                 /* out-direction, in edges: room in vacated blocks (of the pool or
+                                                     of the initial layout) that waits for reuse; room that cannot
+                                                     be reused (tails beyond a block's power-of-two part, blocks
+                                                     dropped because a free list was full)                       */
 } ripple_stats;
 
 /* Sec. 3.1 (preliminaries): the bootstrap embeddings exist before updates arrive.  Builds the

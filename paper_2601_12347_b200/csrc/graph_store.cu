@@ -70,7 +70,9 @@ static cudaError_t alloc_side(Side& s, int N) {
         if ((e = cudaMalloc(a, nb))) return e;
         if ((e = cudaMemset(*a, 0, nb))) return e;
     }
-    return cudaSuccess;
+    if ((e = cudaMalloc(&s.free_blk, sizeof(int64_t) * (size_t)RP_POOL_CLASSES * RP_POOL_LIST_CAP))) return e;
+    if ((e = cudaMalloc(&s.free_cnt, sizeof(int32_t) * RP_POOL_CLASSES))) return e;
+    return cudaMemset(s.free_cnt, 0, sizeof(int32_t) * RP_POOL_CLASSES);
 }
 
 cudaError_t graph_build(Ctx* c, const int32_t* src, const int32_t* dst, int64_t E, double slack,
@@ -284,39 +286,86 @@ k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_
     }
 }
 
-__device__ __forceinline__ int grown_capacity(int cap, int need) {
-    int want = max(2 * cap, need + (need >> 2) + 4);
-    return (want + 3) & ~3;
+// ---------------------------------------------------------------------------------------------
+// Blocks of the adjacency store.  A row that outgrows its block moves to one of at least twice the
+// size; a row left with less than a quarter of a (not small) block in use moves to a smaller one.
+// Blocks handed out after the initial layout have power-of-two sizes (class k = 2^k entries) and
+// come from the class's free list of vacated blocks if it has one, else from the never-used tail
+// of the array (the overflow pool).  A vacated block -- of the pool or of the initial layout -- goes
+// onto the list of the largest class that fits into it.  Within a kernel the lists are either
+// taken from (k_grow_rows) or added to (k_commit_degrees), never both, so a plain counter per list
+// is enough.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int class_for_request(int want) {   // smallest class that holds `want` entries
+    int k = RP_POOL_MIN_CLASS;
+    while ((1 << k) < want) ++k;
+    return k;
 }
 
-// Rows whose additions do not fit: list them and add up the pool entries they will take.
+__device__ __forceinline__ int class_of_block(int cap) {       // largest class that fits into `cap` entries, or -1
+    if (cap < (1 << RP_POOL_MIN_CLASS)) return -1;
+    return 31 - __clz(cap);
+}
+
+__device__ __forceinline__ int grown_class(int cap, int need) {
+    return class_for_request(max(2 * cap, need + (need >> 2) + 4));
+}
+
+__device__ __forceinline__ bool wants_smaller_block(int cap, int need) { return cap >= 64 && 4 * need <= cap; }
+
+__device__ __forceinline__ int shrunk_class(int need) { return class_for_request(2 * need + 8); }
+
+// takes a block of class k from the free list; -1 if the list is empty
+__device__ __forceinline__ long long take_block(const Side& sd, int k) {
+    const int old = atomicSub(&sd.free_cnt[k], 1);
+    if (old >= 1) return sd.free_blk[(size_t)k * RP_POOL_LIST_CAP + (old - 1)];
+    atomicAdd(&sd.free_cnt[k], 1);
+    return -1;
+}
+
+// Rows whose additions do not fit: list them and count the blocks they will take, by class.  Rows
+// that deletions leave nearly empty: list them for a move to a smaller block.
 __global__ void k_plan_growth(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
-                              int32_t* grow_out, int32_t* grow_in) {
+                              int32_t* grow_out, int32_t* grow_in, int32_t* shrink_out, int32_t* shrink_in) {
     pdl_enter();
     if (ctl->abort) return;
     int n = ctl->n_rec;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * n; i += gridDim.x * blockDim.x) {
         int s = i & 1;
         const Rec& x = rec[i >> 1];
-        if (x.sign < 0 || x.rank[s] != 0) continue;
+        if (x.rank[s] != 0) continue;   // one record per row and kind of change
         const Side& sd = s ? in : out;
         int row = s ? x.v : x.u;
         int need = sd.deg[row] - sd.cnt_del[row] + sd.cnt_add[row];
-        if (need > sd.cap[row]) {
-            int g = atomicAdd(&ctl->n_grow[s], 1);
-            (s ? grow_in : grow_out)[g] = row;
-            atomicAdd(&ctl->pool_need[s], (unsigned long long)grown_capacity(sd.cap[row], need));
+        if (x.sign > 0) {
+            if (need > sd.cap[row]) {
+                int g = atomicAdd(&ctl->n_grow[s], 1);
+                (s ? grow_in : grow_out)[g] = row;
+                atomicAdd(&ctl->grow_demand[s][grown_class(sd.cap[row], need)], 1);
+            }
+        } else if (need <= sd.cap[row] && wants_smaller_block(sd.cap[row], need)) {
+            int g = atomicAdd(&ctl->n_shrink[s], 1);
+            (s ? shrink_in : shrink_out)[g] = row;
         }
     }
 }
 
-__global__ void k_plan_check(Ctl* ctl, long long col_size_out, long long col_size_in) {
+// what the growing rows cannot take from the free lists must fit into the never-used tail
+__global__ void k_plan_check(Ctl* ctl, Side out, Side in) {
     pdl_enter();
     if (ctl->abort) return;
-    if (ctl->pool_next[0] + ctl->pool_need[0] > (unsigned long long)col_size_out ||
-        ctl->pool_next[1] + ctl->pool_need[1] > (unsigned long long)col_size_in) {
-        ctl->err = (int)RIPPLE_ERR_CAPACITY;
-        ctl->abort = 1;
+    for (int s = 0; s < 2; ++s) {
+        const Side& sd = s ? in : out;
+        unsigned long long need = 0;
+        for (int k = RP_POOL_MIN_CLASS; k < RP_POOL_CLASSES; ++k) {
+            const int short_of = ctl->grow_demand[s][k] - sd.free_cnt[k];
+            if (short_of > 0) need += (unsigned long long)short_of << k;
+        }
+        ctl->pool_need[s] = need;
+        if (ctl->pool_next[s] + need > (unsigned long long)sd.col_size) {
+            ctl->err = (int)RIPPLE_ERR_CAPACITY;
+            ctl->abort = 1;
+        }
     }
 }
 
@@ -338,8 +387,8 @@ void graph_batch_classify(Ctx* c, int n) {
     RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, c->op_seq, c->ctl, c->hwin, c->op_slot, c->feat_last,
               c->vdel_seq, c->side[0], c->side[1], c->rec, c->bitmap);
     RP_LAUNCH(c, k_plan_growth, std::min(div_up(2 * n, T), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[0],
-              c->side[1], c->grow_list[0], c->grow_list[1]);
-    RP_LAUNCH(c, k_plan_check, 1, 1, 0, c->ctl, (long long)c->side[0].col_size, (long long)c->side[1].col_size);
+              c->side[1], c->grow_list[0], c->grow_list[1], c->shrink_list[0], c->shrink_list[1]);
+    RP_LAUNCH(c, k_plan_check, 1, 1, 0, c->ctl, c->side[0], c->side[1]);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -407,28 +456,89 @@ __global__ void k_del_fill(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side
     }
 }
 
-// One warp per growing row: take a block from the pool, move the row, double its capacity.
-__global__ void k_grow_rows(Ctl* ctl, Side out, Side in, const int32_t* __restrict__ grow_out,
-                            const int32_t* __restrict__ grow_in) {
+// Moves rows into new blocks.  Growing rows: a block of the planned class from the free list, else
+// from the never-used tail (the plan has checked that it fits).  One warp per row; a row of more
+// than GROW_BLOCK_ROW entries is left to a second pass in which a whole block copies it.  The last
+// block to finish then moves the shrinking rows, which take from the free lists or from what the
+// growing rows have left of the never-used tail (a row that finds no block stays where it is and
+// is looked at again when it is next touched).  The blocks left behind are noted in moved_start / moved_cap and returned to the free
+// lists by k_commit_degrees.
+constexpr int GROW_BLOCK_ROW = 2048;
+
+__device__ __forceinline__ void move_row(Side& sd, int row, long long off, int ncap, int live, int tid, int nthreads) {
+    const int64_t old = sd.start[row];
+    for (int j = tid; j < live; j += nthreads) sd.col[off + j] = sd.col[old + j];
+}
+
+__global__ void __launch_bounds__(256)
+k_grow_rows(Ctl* ctl, Side out, Side in, const int32_t* __restrict__ grow_out, const int32_t* __restrict__ grow_in,
+            const int32_t* __restrict__ shrink_out, const int32_t* __restrict__ shrink_in, int64_t* moved_start,
+            int32_t* moved_cap) {
     pdl_enter();
     if (ctl->abort) return;
-    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    int nwarps = (gridDim.x * blockDim.x) >> 5;
-    int n0 = ctl->n_grow[0], n1 = ctl->n_grow[1];
-    for (int g = warp; g < n0 + n1; g += nwarps) {
-        int s = g >= n0;
+    __shared__ long long s_off;
+    __shared__ int s_last;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id();
+    const int n0 = ctl->n_grow[0], n1 = ctl->n_grow[1];
+    for (int pass = 0; pass < 2; ++pass) {
+        const int first = pass ? (int)blockIdx.x : warp, step = pass ? (int)gridDim.x : nwarps;
+        for (int g = first; g < n0 + n1; g += step) {
+            const int s = g >= n0;
+            Side& sd = s ? in : out;
+            const int row = s ? grow_in[g - n0] : grow_out[g];
+            const int live = sd.deg[row] - sd.cnt_del[row];
+            if ((live > GROW_BLOCK_ROW) != (pass == 1)) continue;
+            const int k = grown_class(sd.cap[row], live + sd.cnt_add[row]);
+            const int ncap = 1 << k;
+            long long off = 0;
+            if (pass ? threadIdx.x == 0 : lane == 0) {
+                off = take_block(sd, k);
+                if (off >= 0) atomicAdd(&ctl->pool_free[s], (unsigned long long)(-(long long)ncap));
+                else off = (long long)atomicAdd(&ctl->pool_next[s], (unsigned long long)ncap);
+                moved_start[g] = sd.start[row];
+                moved_cap[g] = sd.cap[row];
+                if (pass) s_off = off;
+            }
+            if (pass) { __syncthreads(); off = s_off; move_row(sd, row, off, ncap, live, threadIdx.x, blockDim.x); __syncthreads(); }
+            else { off = __shfl_sync(FULL, off, 0); move_row(sd, row, off, ncap, live, lane, 32); __syncwarp(); }
+            if (pass ? threadIdx.x == 0 : lane == 0) { sd.start[row] = (int64_t)off; sd.cap[row] = ncap; }
+        }
+    }
+    const int m0 = ctl->n_shrink[0], m1 = ctl->n_shrink[1];
+    if (m0 + m1 == 0) return;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(&ctl->grow_done, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int g = threadIdx.x >> 5; g < m0 + m1; g += blockDim.x >> 5) {
+        const int s = g >= m0;
         Side& sd = s ? in : out;
-        int row = s ? grow_in[g - n0] : grow_out[g];
-        int live = sd.deg[row] - sd.cnt_del[row];
-        int need = live + sd.cnt_add[row];
-        int ncap = grown_capacity(sd.cap[row], need);
-        unsigned long long off = 0;
-        if (lane_id() == 0) off = atomicAdd(&ctl->pool_next[s], (unsigned long long)ncap);
+        const int row = s ? shrink_in[g - m0] : shrink_out[g];
+        const int live = sd.deg[row] - sd.cnt_del[row];
+        const int k = shrunk_class(live + sd.cnt_add[row]);
+        const int ncap = 1 << k;
+        long long off = -1;
+        if (lane == 0) {
+            off = take_block(sd, k);
+            if (off >= 0) atomicAdd(&ctl->pool_free[s], (unsigned long long)(-(long long)ncap));
+            else {   // the growing rows have all been served: what is left of the never-used tail may be taken
+                const unsigned long long at = atomicAdd(&ctl->pool_next[s], (unsigned long long)ncap);
+                if (at + (unsigned long long)ncap <= (unsigned long long)sd.col_size) off = (long long)at;
+                else atomicAdd(&ctl->pool_next[s], (unsigned long long)(-(long long)ncap));
+            }
+            moved_start[n0 + n1 + g] = sd.start[row];
+            moved_cap[n0 + n1 + g] = off >= 0 ? sd.cap[row] : 0;   // 0: nothing left behind
+        }
         off = __shfl_sync(FULL, off, 0);
-        int64_t old = sd.start[row];
-        for (int j = lane_id(); j < live; j += 32) sd.col[off + j] = sd.col[old + j];
+        if (off < 0) continue;
+        move_row(sd, row, off, ncap, live, lane, 32);
         __syncwarp();
-        if (lane_id() == 0) { sd.start[row] = (int64_t)off; sd.cap[row] = ncap; }
+        if (lane == 0) { sd.start[row] = (int64_t)off; sd.cap[row] = ncap; }
     }
 }
 
@@ -447,9 +557,29 @@ __global__ void k_add_write(Ctl* ctl, const Rec* __restrict__ rec, Side out, Sid
 }
 
 __global__ void k_commit_degrees(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
-                                 int32_t* deg_out_old) {
+                                 int32_t* deg_out_old, const int64_t* __restrict__ moved_start,
+                                 const int32_t* __restrict__ moved_cap) {
     pdl_enter();
     if (ctl->abort) return;
+    // the blocks that moved rows left behind go onto the free lists
+    const int n0 = ctl->n_grow[0], n1 = ctl->n_grow[1], m0 = ctl->n_shrink[0], m1 = ctl->n_shrink[1];
+    for (int g = blockIdx.x * blockDim.x + threadIdx.x; g < n0 + n1 + m0 + m1; g += gridDim.x * blockDim.x) {
+        const int s = g < n0 + n1 ? g >= n0 : g - n0 - n1 >= m0;
+        const Side& sd = s ? in : out;
+        const int cap = moved_cap[g];
+        if (cap <= 0) continue;
+        const int k = class_of_block(cap);
+        int kept = 0;
+        if (k >= 0) {
+            const int idx = atomicAdd(&sd.free_cnt[k], 1);
+            if (idx < RP_POOL_LIST_CAP) {
+                sd.free_blk[(size_t)k * RP_POOL_LIST_CAP + idx] = moved_start[g];
+                kept = 1 << k;
+            } else atomicSub(&sd.free_cnt[k], 1);
+        }
+        if (kept) atomicAdd(&ctl->pool_free[s], (unsigned long long)kept);
+        if (cap > kept) atomicAdd(&ctl->pool_lost[s], (unsigned long long)(cap - kept));
+    }
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
         const Rec& x = rec[i >> 1];
@@ -472,9 +602,9 @@ void graph_batch_mutate(Ctx* c, int n) {
     RP_LAUNCH(c, k_del_tail_pack, grid, T, 0, c->ctl, c->rec, o, i);
     RP_LAUNCH(c, k_del_fill, grid, T, 0, c->ctl, c->rec, o, i);
     RP_LAUNCH(c, k_grow_rows, std::min(div_up(2 * n, T / 32), c->n_sm * 8), T, 0, c->ctl, o, i,
-              c->grow_list[0], c->grow_list[1]);
+              c->grow_list[0], c->grow_list[1], c->shrink_list[0], c->shrink_list[1], c->moved_start, c->moved_cap);
     RP_LAUNCH(c, k_add_write, grid, T, 0, c->ctl, c->rec, o, i);
-    RP_LAUNCH(c, k_commit_degrees, grid, T, 0, c->ctl, c->rec, o, i, c->deg_out_old);
+    RP_LAUNCH(c, k_commit_degrees, grid, T, 0, c->ctl, c->rec, o, i, c->deg_out_old, c->moved_start, c->moved_cap);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -45,11 +45,13 @@ static cudaError_t dev_alloc(T** p, size_t count, int fill_byte = -2) {
 // launch chain can be replayed for batches that differ in them)
 __global__ void k_ctl_reset(Ctl* ctl, const int* params) {
     pdl_enter();
-    unsigned long long keep0 = ctl->pool_next[0], keep1 = ctl->pool_next[1];
     Ctl z;
     memset(&z, 0, sizeof(Ctl));
-    z.pool_next[0] = keep0;
-    z.pool_next[1] = keep1;
+    for (int s = 0; s < 2; ++s) {
+        z.pool_next[s] = ctl->pool_next[s];
+        z.pool_free[s] = ctl->pool_free[s];
+        z.pool_lost[s] = ctl->pool_lost[s];
+    }
     z.num_edges = ctl->num_edges;
     z.n_ops = params[0];
     z.n_rows = params[1];
@@ -64,7 +66,8 @@ static void destroy_ctx(Ctx* c) {
         Side& sd = c->side[s];
         cudaFree(sd.col); cudaFree(sd.start); cudaFree(sd.cap); cudaFree(sd.deg);
         cudaFree(sd.cnt_del); cudaFree(sd.cnt_add); cudaFree(sd.tick_a); cudaFree(sd.tick_b); cudaFree(sd.touch);
-        cudaFree(c->grow_list[s]); cudaFree(c->D[s]); cudaFree(c->Clist[s]);
+        cudaFree(c->grow_list[s]); cudaFree(c->shrink_list[s]); cudaFree(c->D[s]); cudaFree(c->Clist[s]);
+        cudaFree(sd.free_blk); cudaFree(sd.free_cnt);
     }
     for (int l = 0; l <= RP_MAXL; ++l) {
         cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->Eb[l]); cudaFree(c->Z[l]); cudaFree(c->P[l]); cudaFree(c->A[l]);
@@ -74,6 +77,7 @@ static void destroy_ctx(Ctx* c) {
     cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->invmask); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
+    cudaFree(c->moved_start); cudaFree(c->moved_cap);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
     if (c->params_host) cudaFreeHost(c->params_host);
     cudaFree(c->params_dev);
@@ -315,7 +319,10 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             CK(dev_alloc(&c->D[s], (size_t)N * max_ld));
             CK(dev_alloc(&c->Clist[s], (size_t)N + 32));
             CK(dev_alloc(&c->grow_list[s], (size_t)o.max_batch));
+            CK(dev_alloc(&c->shrink_list[s], (size_t)o.max_batch));
         }
+        CK(dev_alloc(&c->moved_start, (size_t)4 * o.max_batch));
+        CK(dev_alloc(&c->moved_cap, (size_t)4 * o.max_batch));
         // degree prefix of a sender list; also the (vertex, chunk) work items of long in-lists during a
         // gather: a row of more than 256 entries gives at most 2 items per 256 of them
         CK(dev_alloc(&c->coff, std::max((size_t)N + 2, (size_t)(c->side[1].col_size / 128) + 64), 0));
@@ -559,6 +566,8 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
         }
         s.pool_used = (int64_t)h.pool_next[0] - c->side[0].base_end;
         s.pool_size = c->side[0].col_size - c->side[0].base_end;
+        s.pool_free = (int64_t)h.pool_free[0];
+        s.pool_lost = (int64_t)h.pool_lost[0];
         if (c->timing) {
             cudaEventElapsedTime(&s.ms_total, c->ev[0], c->ev[evi - 1]);
             cudaEventElapsedTime(&s.ms_graph, c->ev[0], c->ev[1]);

@@ -16,6 +16,9 @@
 #define RP_GRAPH_MAX_BATCH 512   // batches up to this size replay a captured launch chain
 #define RP_GRAPH_SLOTS 8
 #define RP_GRAPH_SEEN 32    // recently seen chain keys: a chain is captured at its second appearance
+#define RP_POOL_CLASSES 32          // block size classes of the adjacency store: class k holds blocks of 2^k entries
+#define RP_POOL_MIN_CLASS 3         // smallest block that is kept for reuse: 8 entries
+#define RP_POOL_LIST_CAP 16384      // blocks a class's free list can hold
 
 namespace rp {
 
@@ -34,8 +37,14 @@ struct Ctl {
     int n_rec;   // net edge changes of the batch (|dE+| + |dE-|)
     int n_add, n_del, n_noop_add, n_noop_del, n_superseded, n_feat;
     int n_grow[2];
+    int n_shrink[2];                  // rows left with less than a quarter of their capacity in use: moved to a smaller block
+    int grow_demand[2][RP_POOL_CLASSES];   // growing rows per block size class
+    int grow_done;                    // blocks of k_grow_rows that have finished (the last one moves the shrinking rows)
     unsigned long long pool_need[2];
-    unsigned long long pool_next[2];  // next free entry of each side's adjacency array
+    // kept across batches:
+    unsigned long long pool_next[2];  // next entry of each side's adjacency array that was never handed out
+    unsigned long long pool_free[2];  // entries in vacated blocks that wait in the free lists
+    unsigned long long pool_lost[2];  // entries that cannot be reused: tails beyond a block's power-of-two part, overflow of a list
     int nA[RP_MAXL + 1];              // |A_l|
     int nC[RP_MAXL + 1];              // |C_l| (A_l plus sources of edge changes when coefficients depend on them)
     unsigned long long E[RP_MAXL + 1];          // out-edges of C_{l-1} (+ edge records): message count of hop l
@@ -65,6 +74,10 @@ struct Side {
     int32_t* tick_a;
     int32_t* tick_b;
     int32_t* touch;
+    // vacated blocks, by size class: free_blk[k * RP_POOL_LIST_CAP + i], i < free_cnt[k], is the first entry
+    // of a block of 2^k entries.  A kernel either takes blocks or returns them, never both.
+    int64_t* free_blk;
+    int32_t* free_cnt;
 };
 
 // One net edge change.  side 0 = out-list of u (stores v), side 1 = in-list of v (stores u).
@@ -159,6 +172,9 @@ struct Ctx {
     int hsize;
     Rec* rec;
     int32_t* grow_list[2];
+    int32_t* shrink_list[2];
+    int64_t* moved_start;      // per moved row (growing rows of both sides, then shrinking rows): the block it left
+    int32_t* moved_cap;
     // scan scratch
     int64_t* tile_sums;
     int n_tile_sums;

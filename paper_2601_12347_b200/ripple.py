@@ -76,7 +76,7 @@ class _Stats(ctypes.Structure):
                 ("ms_total", ctypes.c_float), ("ms_graph", ctypes.c_float),
                 ("ms_frontier", _F), ("ms_scatter", _F), ("ms_update", _F),
                 ("ms_scatter_kernel", _F), ("ms_regather", _F), ("ms_bootstrap", ctypes.c_float), ("gpu_launches", ctypes.c_int64), ("n_expanded", ctypes.c_int64),
-                ("rows_rebuilt", _A)]
+                ("rows_rebuilt", _A), ("pool_free", ctypes.c_int64), ("pool_lost", ctypes.c_int64)]
 
 
 _lib = None
@@ -318,7 +318,7 @@ class Ripple:
         L = self.L
         out = {k: getattr(s, k) for k in ("num_layers", "num_edges", "n_ops", "n_added", "n_deleted",
                                           "n_noop_add", "n_noop_del", "n_superseded", "n_feature",
-                                          "pool_used", "pool_size", "ms_total", "ms_graph",
+                                          "pool_used", "pool_size", "pool_free", "pool_lost", "ms_total", "ms_graph",
                                           "ms_bootstrap", "gpu_launches", "n_expanded")}
         for k in ("affected", "senders", "active_edges", "scatter_pull", "in_edges", "message_width", "rows_rebuilt", "ms_frontier", "ms_scatter",
                   "ms_update", "ms_scatter_kernel", "ms_regather"):

@@ -339,6 +339,48 @@ def test_rows_outgrow_their_slack_and_the_pool_can_run_out(env):
     rp.close()
 
 
+def test_vacated_blocks_are_reused_so_a_churning_stream_does_not_exhaust_the_pool(env):
+    """One vertex after the other gains 600 out-edges and loses them again.  Every growth moves the
+    row into a larger block and every mass deletion into a smaller one; without reuse of the vacated
+    blocks the small overflow pool would be gone after about twenty vertices.  The live edge count
+    stays flat, so must the pool."""
+    ripple, Oracle = env
+    model = I.graphconv_model([6, 8, 4], I.AGG_MEAN)
+    n = 2000
+    src, dst = I.er_graph(n, 8000, 31)
+    X = I.features(n, 6, 31)
+    W = I.make_weights(model, 31)
+    present = set(zip(src.tolist(), dst.tolist()))
+    rng = np.random.default_rng(31)
+    pool = 24000
+    rp = ripple.Ripple(n, src, dst, X, model, W, slack=0.25, pool_edges=pool)
+    orc = Oracle(n, src, dst, X, model, W)
+    used = []
+    for phase in range(200):            # bump allocation alone would need 200 x 1024 entries
+        v = 100 + phase
+        targets = [int(t) for t in rng.permutation(n)[:620] if t != v and (v, int(t)) not in present][:600]
+        add = ups_array([(I.OP_ADD_EDGE, v, t) for t in targets])
+        rp.apply_batch(add)
+        assert orc.apply_incremental(add) == 0
+        dele = ups_array([(I.OP_DEL_EDGE, v, t) for t in targets])
+        rp.apply_batch(dele)
+        assert orc.apply_incremental(dele) == 0
+        st = rp.stats()
+        used.append(st["pool_used"])
+        assert st["pool_used"] <= st["pool_size"]
+        if phase % 20 == 19:
+            check_graph(rp, orc)
+            check_frontiers(rp, orc, 2)
+    st = rp.stats()
+    assert st["num_edges"] == 8000
+    assert max(used[20:]) <= used[19] + 4096, used[::20]      # flat after the first few vertices
+    assert st["pool_free"] > 0
+    assert st["pool_used"] - st["pool_free"] - st["pool_lost"] < pool // 2
+    check_graph(rp, orc)
+    check_values(rp, orc.full(), 2)
+    rp.close()
+
+
 def test_star_graph_mass_deletion_and_isolated_vertices(env):
     """Degenerate structure: one hub pointing at everyone, most vertices without out-edges;
     deleting most of the hub's edges in one batch exercises the tail logic of the row update."""
