@@ -35,6 +35,12 @@ def _load():
     vp, i32, i64, dbl = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_double
     lib.orc_create.argtypes = [i32, i64, vp, vp, vp, i32, vp, i32]
     lib.orc_create.restype = vp
+    lib.orc_create_weighted.argtypes = [i32, i64, vp, vp, vp, vp, i32, vp, i32]
+    lib.orc_create_weighted.restype = vp
+    lib.orc_set_batch_weights.argtypes = [vp, vp]
+    lib.orc_set_batch_weights.restype = None
+    lib.orc_export_weights.argtypes = [vp, vp]
+    lib.orc_export_weights.restype = None
     lib.orc_set_layer.argtypes = [vp, i32, i32, i32, i32, dbl, vp, vp, vp, vp]
     lib.orc_set_layer.restype = None
     lib.orc_destroy.argtypes = [vp]
@@ -84,7 +90,7 @@ class Oracle:
     """
 
     def __init__(self, n: int, src: np.ndarray, dst: np.ndarray, feat: np.ndarray, model, weights,
-                 bootstrap: bool = True):
+                 bootstrap: bool = True, edge_weights: Optional[np.ndarray] = None):
         lib = _load()
         self.lib = lib
         self.n = int(n)
@@ -95,8 +101,12 @@ class Oracle:
         feat = np.ascontiguousarray(feat, dtype=np.float32)
         assert feat.shape == (self.n, self.dims[0])
         dims = np.asarray(self.dims, dtype=np.int32)
-        self.h = lib.orc_create(self.n, src.size, src.ctypes.data, dst.ctypes.data,
-                                feat.ctypes.data, self.L, dims.ctypes.data, int(model.agg))
+        if edge_weights is not None:
+            edge_weights = np.ascontiguousarray(edge_weights, dtype=np.float32)
+            assert edge_weights.shape == src.shape
+        self.h = lib.orc_create_weighted(self.n, src.size, src.ctypes.data, dst.ctypes.data,
+                                         edge_weights.ctypes.data if edge_weights is not None else None,
+                                         feat.ctypes.data, self.L, dims.ctypes.data, int(model.agg))
         for i, (ly, w) in enumerate(zip(model.layers, weights)):
             def p(name):
                 a = w.get(name)
@@ -122,27 +132,41 @@ class Oracle:
             pass
 
     # ---- updates -----------------------------------------------------------------------
-    def _apply(self, fn, ups: np.ndarray, feat_rows: Optional[np.ndarray]) -> int:
+    def _apply(self, fn, ups: np.ndarray, feat_rows: Optional[np.ndarray], op_weights=None) -> int:
         ups = np.ascontiguousarray(ups, dtype=UPDATE_DTYPE)
         if feat_rows is None:
             feat_rows = np.zeros((0, self.dims[0]), dtype=np.float32)
         feat_rows = np.ascontiguousarray(feat_rows, dtype=np.float32)
-        return int(fn(self.h, ups.ctypes.data, ups.size, feat_rows.ctypes.data, feat_rows.shape[0]))
+        if op_weights is not None:     # one weight per operation; read for edge additions only
+            op_weights = np.ascontiguousarray(op_weights, dtype=np.float32)
+            assert op_weights.shape == (ups.size,)
+            self.lib.orc_set_batch_weights(self.h, op_weights.ctypes.data)
+        try:
+            return int(fn(self.h, ups.ctypes.data, ups.size, feat_rows.ctypes.data, feat_rows.shape[0]))
+        finally:
+            self.lib.orc_set_batch_weights(self.h, None)
 
-    def apply_incremental(self, ups, feat_rows=None, pull: bool = False) -> int:
+    def apply_incremental(self, ups, feat_rows=None, pull: bool = False, op_weights=None) -> int:
         """The incremental algorithm.  pull: messages are gathered per affected sink on all host
         cores instead of being pushed along the senders' out-lists by one thread; only the order
-        of the additions differs."""
+        of the additions differs.  op_weights: the weight of every ADD_EDGE of the batch (an array
+        with one entry per operation) for the weighted sum with per-edge weights."""
         fn = self.lib.orc_apply_incremental_pull if pull else self.lib.orc_apply_incremental
-        return self._apply(fn, ups, feat_rows)
+        return self._apply(fn, ups, feat_rows, op_weights)
 
-    def apply_scoped(self, ups, feat_rows=None) -> int:
-        return self._apply(self.lib.orc_apply_scoped, ups, feat_rows)
+    def apply_scoped(self, ups, feat_rows=None, op_weights=None) -> int:
+        return self._apply(self.lib.orc_apply_scoped, ups, feat_rows, op_weights)
 
-    def apply_structure(self, ups, n_rows: int) -> int:
+    def apply_structure(self, ups, n_rows: int, op_weights=None) -> int:
         """Graph state and affected sets only (no embedding arithmetic; H and S go stale)."""
         ups = np.ascontiguousarray(ups, dtype=UPDATE_DTYPE)
-        return int(self.lib.orc_apply_structure(self.h, ups.ctypes.data, ups.size, int(n_rows)))
+        if op_weights is not None:
+            op_weights = np.ascontiguousarray(op_weights, dtype=np.float32)
+            self.lib.orc_set_batch_weights(self.h, op_weights.ctypes.data)
+        try:
+            return int(self.lib.orc_apply_structure(self.h, ups.ctypes.data, ups.size, int(n_rows)))
+        finally:
+            self.lib.orc_set_batch_weights(self.h, None)
 
     def bootstrap(self):
         self.lib.orc_bootstrap(self.h)
@@ -195,6 +219,12 @@ class Oracle:
         col = np.zeros(max(1, self.num_edges()), dtype=np.int32)
         self.lib.orc_export_csr(self.h, rowptr.ctypes.data, col.ctypes.data)
         return rowptr, col[: rowptr[-1]]
+
+    def export_weights(self) -> np.ndarray:
+        """The stored weight of every edge, in the order of export_csr()'s column array."""
+        w = np.zeros(max(1, self.num_edges()), dtype=np.float32)
+        self.lib.orc_export_weights(self.h, w.ctypes.data)
+        return w[: self.num_edges()]
 
     def row_from_prev(self, l: int, v: int, Hprev: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
         """(S^l_v, h^l_v) by the layer definition from a caller-supplied fp32 H^{l-1}."""

@@ -43,7 +43,7 @@
 #include <string.h>
 
 enum { KIND_SAGE = 0, KIND_GRAPHCONV = 1, KIND_GIN = 2 };
-enum { AGG_SUM = 0, AGG_MEAN = 1, AGG_WSUM_GCN = 2, AGG_MAX = 3, AGG_MIN = 4 };
+enum { AGG_SUM = 0, AGG_MEAN = 1, AGG_WSUM_GCN = 2, AGG_MAX = 3, AGG_MIN = 4, AGG_WSUM_EDGE = 5 };
 #define MONOTONIC(agg) ((agg) == AGG_MAX || (agg) == AGG_MIN)
 enum { ACT_IDENTITY = 0, ACT_RELU = 1 };
 enum { OP_ADD_EDGE = 0, OP_DEL_EDGE = 1, OP_SET_FEATURE = 2, OP_DEL_VERTEX = 3 };
@@ -56,12 +56,15 @@ typedef struct {
     double *Wa, *Wb, *ba, *bb; /* input-major: Wa[k * d_next + j] */
 } layer_t;
 
-typedef struct { int *a; int n, cap; } ivec; /* ascending neighbour ids */
+/* ascending neighbour ids; w: the stored weight of each edge (weighted sum with per-edge weights only, else NULL) */
+typedef struct { int *a; float *w; int n, cap; } ivec;
 
-typedef struct { int u, v; } pair_t;
+typedef struct { int u, v; float w; } pair_t;   /* w: weight of an added edge / weight a deleted edge had */
 
 typedef struct {
     int N, L, agg;
+    int weighted;      /* every edge carries a stored weight alpha_uv (Table 1, weighted sum) */
+    const float *op_w; /* weights of the batch being applied, one per operation (read for ADD_EDGE only), or NULL = 1 */
     int *d;            /* d[0..L] widths */
     layer_t *layer;    /* layer[1..L] */
     ivec *out, *in;
@@ -91,14 +94,20 @@ static int ivec_find(const ivec *r, int x) { /* index of x or -1 */
     return (lo < r->n && r->a[lo] == x) ? lo : -1;
 }
 
-static void ivec_insert(ivec *r, int x) {
+static void ivec_insert(ivec *r, int x, int weighted, float w) {
     if (r->n == r->cap) {
         r->cap = r->cap ? 2 * r->cap : 4;
         r->a = (int *)realloc(r->a, sizeof(int) * (size_t)r->cap);
+        if (weighted) r->w = (float *)realloc(r->w, sizeof(float) * (size_t)r->cap);
     }
     int i = r->n;
-    while (i > 0 && r->a[i - 1] > x) { r->a[i] = r->a[i - 1]; --i; }
+    while (i > 0 && r->a[i - 1] > x) {
+        r->a[i] = r->a[i - 1];
+        if (weighted) r->w[i] = r->w[i - 1];
+        --i;
+    }
     r->a[i] = x;
+    if (weighted) r->w[i] = w;
     r->n++;
 }
 
@@ -106,6 +115,7 @@ static void ivec_erase(ivec *r, int x) {
     int i = ivec_find(r, x);
     if (i < 0) return;
     memmove(r->a + i, r->a + i + 1, sizeof(int) * (size_t)(r->n - i - 1));
+    if (r->w) memmove(r->w + i, r->w + i + 1, sizeof(float) * (size_t)(r->n - i - 1));
     r->n--;
 }
 
@@ -115,9 +125,16 @@ static double coef_src(const oracle_t *o, int deg_out) {
     return deg_out > 0 ? 1.0 / sqrt((double)deg_out) : 0.0;
 }
 
+/* Coefficient of the i-th in-edge (u, v) of v inside S_v: the edge's stored weight alpha_uv for the
+ * weighted sum with per-edge weights (Table 1), else the source-side coefficient c_u. */
+static double in_edge_coef(const oracle_t *o, int v, int i) {
+    if (o->weighted) return (double)o->in[v].w[i];
+    return coef_src(o, o->out[o->in[v].a[i]].n);
+}
+
 /* Sink-side normalisation applied to S_v at compute time (Table 1: mean, weighted sum). */
 static double norm_sink(const oracle_t *o, int deg_in) {
-    if (o->agg == AGG_SUM || MONOTONIC(o->agg)) return 1.0;
+    if (o->agg == AGG_SUM || o->agg == AGG_WSUM_EDGE || MONOTONIC(o->agg)) return 1.0;
     if (deg_in <= 0) return 0.0;
     return o->agg == AGG_MEAN ? 1.0 / (double)deg_in : 1.0 / sqrt((double)deg_in);
 }
@@ -176,17 +193,33 @@ static void aggregate_row(const oracle_t *o, int v, const double *Hprev, int K, 
     }
     for (int i = 0; i < in->n; ++i) {
         int u = in->a[i];
-        double c = coef_src(o, o->out[u].n);
+        double c = in_edge_coef(o, v, i);
         const double *h = Hprev + (size_t)u * K;
         for (int k = 0; k < K; ++k) Srow[k] += c * h[k];
     }
 }
 
 /* ------------------------------------------------------------------------------------------ */
-oracle_t *orc_create(int N, int64_t E, const int32_t *src, const int32_t *dst, const float *feat,
-                     int L, const int *dims, int agg) {
+typedef struct { int id; float w; } idw_t;
+static int cmp_idw(const void *a, const void *b) {
+    int x = ((const idw_t *)a)->id, y = ((const idw_t *)b)->id;
+    return (x > y) - (x < y);
+}
+static void sort_list(ivec *r) {   /* ascending ids, weights (if any) moving with them */
+    if (!r->w) { qsort(r->a, (size_t)r->n, sizeof(int), cmp_int); return; }
+    idw_t *t = (idw_t *)malloc(sizeof(idw_t) * (size_t)(r->n + 1));
+    for (int i = 0; i < r->n; ++i) { t[i].id = r->a[i]; t[i].w = r->w[i]; }
+    qsort(t, (size_t)r->n, sizeof(idw_t), cmp_idw);
+    for (int i = 0; i < r->n; ++i) { r->a[i] = t[i].id; r->w[i] = t[i].w; }
+    free(t);
+}
+
+/* weight: one stored weight per edge (required for the weighted sum with per-edge weights), or NULL */
+oracle_t *orc_create_weighted(int N, int64_t E, const int32_t *src, const int32_t *dst, const float *weight,
+                              const float *feat, int L, const int *dims, int agg) {
     oracle_t *o = (oracle_t *)calloc(1, sizeof(oracle_t));
     o->N = N; o->L = L; o->agg = agg;
+    o->weighted = agg == AGG_WSUM_EDGE;
     o->d = (int *)malloc(sizeof(int) * (size_t)(L + 1));
     memcpy(o->d, dims, sizeof(int) * (size_t)(L + 1));
     o->layer = (layer_t *)calloc((size_t)L + 1, sizeof(layer_t));
@@ -196,15 +229,20 @@ oracle_t *orc_create(int N, int64_t E, const int32_t *src, const int32_t *dst, c
     for (int v = 0; v < N; ++v) {
         if (o->out[v].cap) o->out[v].a = (int *)malloc(sizeof(int) * (size_t)o->out[v].cap);
         if (o->in[v].cap) o->in[v].a = (int *)malloc(sizeof(int) * (size_t)o->in[v].cap);
+        if (o->weighted && o->out[v].cap) o->out[v].w = (float *)malloc(sizeof(float) * (size_t)o->out[v].cap);
+        if (o->weighted && o->in[v].cap) o->in[v].w = (float *)malloc(sizeof(float) * (size_t)o->in[v].cap);
     }
     for (int64_t e = 0; e < E; ++e) {
-        ivec *r = &o->out[src[e]]; r->a[r->n++] = dst[e];
-        ivec *c = &o->in[dst[e]];  c->a[c->n++] = src[e];
+        ivec *r = &o->out[src[e]];
+        ivec *c = &o->in[dst[e]];
+        if (o->weighted) { r->w[r->n] = weight ? weight[e] : 1.0f; c->w[c->n] = weight ? weight[e] : 1.0f; }
+        r->a[r->n++] = dst[e];
+        c->a[c->n++] = src[e];
     }
 #pragma omp parallel for schedule(dynamic, 1024)
     for (int v = 0; v < N; ++v) {
-        qsort(o->out[v].a, (size_t)o->out[v].n, sizeof(int), cmp_int);
-        qsort(o->in[v].a, (size_t)o->in[v].n, sizeof(int), cmp_int);
+        sort_list(&o->out[v]);
+        sort_list(&o->in[v]);
     }
     o->H = (double **)calloc((size_t)L + 1, sizeof(double *));
     o->S = (double **)calloc((size_t)L + 1, sizeof(double *));
@@ -220,6 +258,11 @@ oracle_t *orc_create(int N, int64_t E, const int32_t *src, const int32_t *dst, c
     }
     for (size_t i = 0; i < (size_t)N * (size_t)dims[0]; ++i) o->H[0][i] = (double)feat[i];
     return o;
+}
+
+oracle_t *orc_create(int N, int64_t E, const int32_t *src, const int32_t *dst, const float *feat,
+                     int L, const int *dims, int agg) {
+    return orc_create_weighted(N, E, src, dst, NULL, feat, L, dims, agg);
 }
 
 static double *widen(const float *x, size_t n) {
@@ -247,7 +290,7 @@ void orc_set_layer(oracle_t *o, int l, int kind, int d_hid, int act, double eps,
 
 void orc_destroy(oracle_t *o) {
     if (!o) return;
-    for (int v = 0; v < o->N; ++v) { free(o->out[v].a); free(o->in[v].a); }
+    for (int v = 0; v < o->N; ++v) { free(o->out[v].a); free(o->in[v].a); free(o->out[v].w); free(o->in[v].w); }
     for (int l = 0; l <= o->L; ++l) {
         free(o->H[l]); free(o->S[l]); free(o->FH[l]); free(o->FS[l]); free(o->A[l]);
         free(o->layer[l].Wa); free(o->layer[l].Wb); free(o->layer[l].ba); free(o->layer[l].bb);
@@ -363,13 +406,21 @@ static int normalise(oracle_t *o, const update_t *ups, int64_t n, int64_t n_rows
     for (int i = 0; i < ne; ++i) {
         if (i + 1 < ne && eo[i + 1].u == eo[i].u && eo[i + 1].v == eo[i].v) { o->superseded++; continue; }
         if (!FINAL_WORD(&eo[i])) { o->superseded++; continue; }
-        int present = ivec_find(&o->out[eo[i].u], eo[i].v) >= 0;
-        if (eo[i].op == OP_ADD_EDGE) {
+        int at = ivec_find(&o->out[eo[i].u], eo[i].v), present = at >= 0;
+        if (eo[i].op == OP_ADD_EDGE) {   /* an edge that exists keeps the weight it has */
             if (present) o->noop_add++;
-            else { dl->add[dl->n_add].u = eo[i].u; dl->add[dl->n_add].v = eo[i].v; dl->n_add++; }
+            else {
+                dl->add[dl->n_add].u = eo[i].u; dl->add[dl->n_add].v = eo[i].v;
+                dl->add[dl->n_add].w = o->op_w ? o->op_w[eo[i].seq] : 1.0f;
+                dl->n_add++;
+            }
         } else {
             if (!present) o->noop_del++;
-            else { dl->del[dl->n_del].u = eo[i].u; dl->del[dl->n_del].v = eo[i].v; dl->n_del++; }
+            else {
+                dl->del[dl->n_del].u = eo[i].u; dl->del[dl->n_del].v = eo[i].v;
+                dl->del[dl->n_del].w = o->weighted ? o->out[eo[i].u].w[at] : 1.0f;
+                dl->n_del++;
+            }
         }
     }
     if (ng) {
@@ -381,7 +432,9 @@ static int normalise(oracle_t *o, const update_t *ups, int64_t n, int64_t n_rows
                     int u = side ? r->a[j] : w, v = side ? w : r->a[j];
                     const eop_t *e = eop_last(eo, ne, u, v);
                     if (e && FINAL_WORD(e)) continue;   /* a later operation on the pair decided */
-                    dl->del[dl->n_del].u = u; dl->del[dl->n_del].v = v; dl->n_del++;
+                    dl->del[dl->n_del].u = u; dl->del[dl->n_del].v = v;
+                    dl->del[dl->n_del].w = o->weighted ? r->w[j] : 1.0f;
+                    dl->n_del++;
                 }
             }
         }
@@ -463,8 +516,8 @@ static int *changed_senders(oracle_t *o, const delta_t *dl, const int *A, int nA
 /* Apply: mutate topology and features (Sec. 3.3, first step of the lifecycle). */
 static void apply_topology(oracle_t *o, const delta_t *dl) {
     for (int i = 0; i < dl->n_add; ++i) {
-        ivec_insert(&o->out[dl->add[i].u], dl->add[i].v);
-        ivec_insert(&o->in[dl->add[i].v], dl->add[i].u);
+        ivec_insert(&o->out[dl->add[i].u], dl->add[i].v, o->weighted, dl->add[i].w);
+        ivec_insert(&o->in[dl->add[i].v], dl->add[i].u, o->weighted, dl->add[i].w);
     }
     for (int i = 0; i < dl->n_del; ++i) {
         ivec_erase(&o->out[dl->del[i].u], dl->del[i].v);
@@ -585,7 +638,7 @@ static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *fe
             walked += r->n;
             for (int j = 0; j < r->n; ++j) {
                 int v = r->a[j];
-                pair_t p = { u, v };
+                pair_t p = { u, v, 0.f };
                 if (dl->n_add && bsearch(&p, dl->add, (size_t)dl->n_add, sizeof(pair_t), cmp_pair)) continue;
                 double *Sv = S + (size_t)v * K;
                 for (int k = 0; k < K; ++k) {
@@ -730,9 +783,10 @@ static int apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const 
             const ivec *r = &o->out[u];
             for (int j = 0; j < r->n; ++j) {
                 int v = r->a[j];
-                if (has_add) { pair_t p = { u, v }; if (bsearch(&p, dl.add, (size_t)dl.n_add, sizeof(pair_t), cmp_pair)) continue; }
+                if (has_add) { pair_t p = { u, v, 0.f }; if (bsearch(&p, dl.add, (size_t)dl.n_add, sizeof(pair_t), cmp_pair)) continue; }
                 double *Sv = S + (size_t)v * K;
-                for (int k = 0; k < K; ++k) Sv[k] += m[k];
+                double a = o->weighted ? (double)r->w[j] : 1.0;   /* the edge's weight scales the message (Sec. 3.3.3) */
+                for (int k = 0; k < K; ++k) Sv[k] += a * m[k];
             }
         }
         if (pull) {
@@ -745,9 +799,10 @@ static int apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const 
                     int u = r->a[j], p = sender_pos[u];
                     if (p < 0) continue;
                     /* an edge added by this batch carries no delta message */
-                    if (dl.n_add) { pair_t e = { u, v }; if (bsearch(&e, dl.add, (size_t)dl.n_add, sizeof(pair_t), cmp_pair)) continue; }
+                    if (dl.n_add) { pair_t e = { u, v, 0.f }; if (bsearch(&e, dl.add, (size_t)dl.n_add, sizeof(pair_t), cmp_pair)) continue; }
                     const double *mu = m + (size_t)p * K;
-                    for (int k = 0; k < K; ++k) Sv[k] += mu[k];
+                    double a = o->weighted ? (double)r->w[j] : 1.0;
+                    for (int k = 0; k < K; ++k) Sv[k] += a * mu[k];
                 }
             }
             for (int i = 0; i < nC; ++i) sender_pos[C[i]] = -1;
@@ -755,7 +810,7 @@ static int apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const 
         /* added edge: the old contribution is taken as 0, so the whole new term arrives */
         for (int i = 0; i < dl.n_add; ++i) {
             int u = dl.add[i].u;
-            double cnew = coef_src(o, o->out[u].n);
+            double cnew = coef_src(o, o->out[u].n) * (o->weighted ? (double)dl.add[i].w : 1.0);
             const double *hnew = Hp + (size_t)u * K;
             double *Sv = S + (size_t)dl.add[i].v * K;
             for (int k = 0; k < K; ++k) Sv[k] += cnew * hnew[k];
@@ -765,7 +820,7 @@ static int apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const 
             int u = dl.del[i].u;
             int ia = find_sorted(A, nA, u);
             const double *hold = ia >= 0 ? oldA + (size_t)ia * K : Hp + (size_t)u * K;
-            double cold = source_find(srcs, nsrc, u)->c_old;
+            double cold = source_find(srcs, nsrc, u)->c_old * (o->weighted ? (double)dl.del[i].w : 1.0);
             double *Sv = S + (size_t)dl.del[i].v * K;
             for (int k = 0; k < K; ++k) Sv[k] -= cold * hold[k];
         }
@@ -883,7 +938,7 @@ void orc_row_from_prev(const oracle_t *o, int l, int v, const float *Hprev, int6
     const ivec *in = &o->in[v];
     for (int i = 0; i < in->n; ++i) {
         int u = in->a[i];
-        double c = coef_src(o, o->out[u].n);
+        double c = in_edge_coef(o, v, i);
         const float *h = Hprev + (size_t)u * (size_t)ld;
         for (int k = 0; k < K; ++k) S_out[k] += c * (double)h[k];
     }
@@ -932,6 +987,15 @@ int64_t orc_num_edges(oracle_t *o) {
 void orc_degrees(oracle_t *o, int32_t *deg_out, int32_t *deg_in) {
     for (int v = 0; v < o->N; ++v) { deg_out[v] = o->out[v].n; deg_in[v] = o->in[v].n; }
 }
+void orc_set_batch_weights(oracle_t *o, const float *op_w) { o->op_w = op_w; }
+
+/* the stored weight of every edge, in the order of orc_export_csr's col */
+void orc_export_weights(oracle_t *o, float *w) {
+    int64_t p = 0;
+    for (int v = 0; v < o->N; ++v)
+        for (int j = 0; j < o->out[v].n; ++j) w[p++] = o->weighted ? o->out[v].w[j] : 1.0f;
+}
+
 /* canonical CSR of the out-lists: rowptr[N+1], col sorted within each row */
 void orc_export_csr(oracle_t *o, int64_t *rowptr, int32_t *col) {
     int64_t p = 0;

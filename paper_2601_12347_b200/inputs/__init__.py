@@ -35,13 +35,14 @@ AGG_MEAN = 1
 AGG_WSUM_GCN = 2   # coefficient 1/sqrt(deg_out(u) * deg_in(v))
 AGG_MAX = 3        # element-wise maximum over the in-neighbours (monotonic; zeros if there are none)
 AGG_MIN = 4        # element-wise minimum, likewise
+AGG_WSUM_EDGE = 5  # weighted sum with a stored weight per edge (the paper's GC-W workload)
 
 ACT_IDENTITY = 0
 ACT_RELU = 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SUBSTREAM = {"graph": 1, "features": 2, "weights": 3, "updates": 4, "warmup": 5, "perm": 6,
-              "drop": 7, "order": 8}
+              "drop": 7, "order": 8, "edge_weights": 9, "update_weights": 10}
 
 
 def _rng(seed: int, stream: str) -> np.random.Generator:
@@ -143,6 +144,11 @@ def rmat_graph(n: int, m: int, seed: int, a: float = 0.57, b: float = 0.19, c: f
     src = perm[keys // n][order]
     dst = perm[keys % n][order]
     return np.ascontiguousarray(src, dtype=np.int32), np.ascontiguousarray(dst, dtype=np.int32)
+
+
+def edge_weights(m: int, seed: int, stream: str = "edge_weights") -> np.ndarray:
+    """m fp32 edge weights ~ U(0.1, 1), in the order of the graph's edge arrays."""
+    return _rng(seed, stream).uniform(0.1, 1.0, size=m).astype(np.float32)
 
 
 def features(n: int, d: int, seed: int, stream: str = "features") -> np.ndarray:
@@ -265,6 +271,7 @@ class UpdateStream:
         self.added_pos: Dict[int, int] = {}
         self.hubs = None if hubs is None else np.asarray(hubs, dtype=np.int64)
         self.n_edges = self.e0
+        self.wrng = _rng(seed, "update_weights")   # weights of added edges: a stream of its own
         self.init_in_keys = None
         if self.mix.size > 3 and self.mix[3] > 0:   # in-edge index, only needed to delete vertices
             self.init_in_keys = np.sort(dst.astype(np.int64) * self.n + src.astype(np.int64))
@@ -374,6 +381,12 @@ class UpdateStream:
         return ups, np.ascontiguousarray(feat, dtype=np.float32)
 
 
+    def next_batch_weighted(self, b: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        """next_batch plus one fp32 weight ~ U(0.1, 1) per update (it matters for edge additions only)."""
+        ups, feat = self.next_batch(b)
+        return ups, feat, self.wrng.uniform(0.1, 1.0, size=b).astype(np.float32)
+
+
 def top_out_degree(n: int, src: np.ndarray, frac: float = 0.01) -> np.ndarray:
     """Ids of the ceil(frac * n) vertices of largest out-degree (ties broken by lower id)."""
     deg = np.bincount(src, minlength=n)
@@ -435,6 +448,11 @@ def workloads() -> Dict[str, Workload]:
                                (1000,), 20),
         "dense-gcx-2l": Workload("dense-gcx-2l", n_d, e_d, "rmat", graphconv_model([100, 256, 47], AGG_MAX), 0,
                                  (10, 100, 1000), 20),
+        # GraphConv with a stored weight per edge (the paper's GC-W workload, Sec. 6.1.1)
+        "sparse-gcw": Workload("sparse-gcw", n_s, e_s, "rmat", graphconv_model([128, 256, 40], AGG_WSUM_EDGE), 0,
+                               (1, 10, 100, 1000), 100, {"edge_weights": True}),
+        "dense-gcw-2l": Workload("dense-gcw-2l", n_d, e_d, "rmat", graphconv_model([100, 256, 47], AGG_WSUM_EDGE), 0,
+                                 (100, 1000), 20, {"edge_weights": True}),
         # all five update types of Sec. 3.1: 2 % of the updates delete a vertex
         "sparse-vdel": Workload("sparse-vdel", n_s, e_s, "rmat", sage_model([128, 256, 40]), 0, (100, 1000), 100,
                                 {"mix": (0.39, 0.39, 0.2, 0.02), "max_batch": 65536}),
