@@ -149,7 +149,17 @@ def make_workload(name, seed):
     src, dst = I.make_graph(w)
     X = I.features(w.n, w.model.dims[0], w.seed)
     W = I.make_weights(w.model, w.seed)
+    # workloads whose edges carry stored weights: one weight per initial edge, one per operation of a batch
+    w.edge_w = I.edge_weights(src.size, w.seed) if w.extra.get("edge_weights") else None
     return w, src, dst, X, W
+
+
+def draw_batch(stream, w, b):
+    """(ups, rows, op_weights or None) of the next batch of the workload's stream"""
+    if w.edge_w is not None:
+        return stream.next_batch_weighted(b)
+    ups, rows = stream.next_batch(b)
+    return ups, rows, None
 
 
 def run_reference(args, rank, world):
@@ -159,18 +169,19 @@ def run_reference(args, rank, world):
     from oracle import oracle as O
     O.build()
     w, src, dst, X, W = make_workload(args.workload, args.seed)
-    orc = O.Oracle(w.n, src, dst, X, w.model, W)
+    orc = O.Oracle(w.n, src, dst, X, w.model, W, edge_weights=w.edge_w)
     stream = I.make_stream(w, src, dst)
     lat = []
     # a step is one batch; if full batches would take the run beyond a few minutes, every step after
     # the first applies a bounded sample of its batch instead (the first n_sample updates)
     n_sample, budget_s = args.batch, 150.0
     for s in range(args.warmup + args.steps):
-        ups, rows = stream.next_batch(args.batch)
+        ups, rows, ow = draw_batch(stream, w, args.batch)
         if n_sample < args.batch:
             ups = ups[:n_sample]
+            ow = ow[:n_sample] if ow is not None else None
         t0 = time.perf_counter()
-        assert orc.apply_incremental(ups, rows) == 0
+        assert orc.apply_incremental(ups, rows, op_weights=ow) == 0
         dt = time.perf_counter() - t0
         if s == 0 and dt * (args.warmup + args.steps) > budget_s:
             n_sample = max(1, int(args.batch * budget_s / (dt * (args.warmup + args.steps))))
@@ -200,14 +211,14 @@ def cpu_baseline(args, w, src, dst, X, W, budget_s=20.0):
     from oracle import oracle as O
     O.build()
     t0 = time.perf_counter()
-    orc = O.Oracle(w.n, src, dst, X, w.model, W)
+    orc = O.Oracle(w.n, src, dst, X, w.model, W, edge_weights=w.edge_w)
     setup = time.perf_counter() - t0
     stream = I.make_stream(w, src, dst)
     spent, nb = 0.0, 0
     while spent < budget_s and nb < 50:
-        ups, rows = stream.next_batch(args.batch)
+        ups, rows, ow = draw_batch(stream, w, args.batch)
         t0 = time.perf_counter()
-        assert orc.apply_incremental(ups, rows) == 0
+        assert orc.apply_incremental(ups, rows, op_weights=ow) == 0
         spent += time.perf_counter() - t0
         nb += 1
     orc.close()
@@ -229,19 +240,19 @@ def run_ours(args, rank, world, local_rank):
     w, src, dst, X, W = make_workload(args.workload, seed)
     L = len(w.model.layers)
     rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=max(args.batch, 16),
-                       scatter_mode=args.scatter)
+                       scatter_mode=args.scatter, edge_weights=w.edge_w)
     bootstrap_ms = rp.stats()["ms_bootstrap"]
     stream = I.make_stream(w, src, dst, seed)
     K, Wm = args.steps, args.warmup
-    batches = [stream.next_batch(args.batch) for _ in range(Wm + 2 * K)]
+    batches = [draw_batch(stream, w, args.batch) for _ in range(Wm + 2 * K)]
 
-    def to_dev(ups, rows):
+    def to_dev(ups, rows, ow):
         u = torch.from_numpy(np.stack([ups["op"], ups["u"], ups["v"]], axis=1).astype(np.int32)).cuda()
-        return u, torch.from_numpy(rows).cuda()
+        return u, torch.from_numpy(rows).cuda(), (torch.from_numpy(ow).cuda() if ow is not None else None)
 
-    def to_pinned(ups, rows):
+    def to_pinned(ups, rows, ow):
         u = torch.from_numpy(np.stack([ups["op"], ups["u"], ups["v"]], axis=1).astype(np.int32)).pin_memory()
-        return u, torch.from_numpy(rows).pin_memory()
+        return u, torch.from_numpy(rows).pin_memory(), (torch.from_numpy(ow).pin_memory() if ow is not None else None)
 
     dev_batches = [to_dev(*b) for b in batches[: Wm + K]]
     pin_batches = [to_pinned(*b) for b in batches[Wm + K:]]
@@ -295,12 +306,12 @@ def run_ours(args, rank, world, local_rank):
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(st)
-    for u, r in pin_batches:
+    for u, r, ow in pin_batches:
         t0 = time.perf_counter()
-        rp.apply_batch(u, r)
+        rp.apply_batch(u, r, ow)
         ids = rp.affected(L).cpu()        # trigger-style read-out: who changed at the last layer
         lat.append(time.perf_counter() - t0)
-        h2d += u.numel() * 4 + r.numel() * 4
+        h2d += u.numel() * 4 + r.numel() * 4 + (ow.numel() * 4 if ow is not None else 0)
         d2h += ids.numel() * 4
     e1.record(st)
     barrier()
@@ -407,7 +418,7 @@ def run_table(args):
         w, src, dst, X, W = make_workload(name, args.seed)
         L = len(w.model.layers)
         rp = ripple.Ripple(w.n, src, dst, X, w.model, W, timing=True, max_batch=w.extra.get("max_batch", 16384),
-                           scatter_mode=args.scatter,
+                           scatter_mode=args.scatter, edge_weights=w.edge_w,
                            regather_threshold=args.regather_threshold)
         boot = rp.stats()["ms_bootstrap"]
         rp.recompute_full()   # warm: the recompute-everything alternative on the same state
@@ -417,26 +428,27 @@ def run_table(args):
         if not args.no_cpu_baseline and args.oracle_seconds > 0:
             from oracle import oracle as O
             O.build()
-            orc = O.Oracle(w.n, src, dst, X, w.model, W)
+            orc = O.Oracle(w.n, src, dst, X, w.model, W, edge_weights=w.edge_w)
             ostream = I.make_stream(w, src, dst, args.seed)
         for bsz in (args.batch_sizes or w.batch_sizes):
             nb = args.table_batches
             nt = min(20, nb)   # extra batches with per-stage event timing (small batches then run ungraphed)
-            batches = [stream.next_batch(bsz) for _ in range(5 + nb + nt)]
+            batches = [draw_batch(stream, w, bsz) for _ in range(5 + nb + nt)]
             pinned = []
-            for ups, rows in batches:
+            for ups, rows, ow in batches:
                 u = torch.from_numpy(np.stack([ups["op"], ups["u"], ups["v"]], axis=1).astype(np.int32)).pin_memory()
-                pinned.append((u, torch.from_numpy(rows).pin_memory()))
+                pinned.append((u, torch.from_numpy(rows).pin_memory(),
+                               torch.from_numpy(ow).pin_memory() if ow is not None else None))
             lat, sc_ms, sc_bytes = [], 0.0, 0
             stage = {"graph": 0.0, "frontier": 0.0, "scatter": 0.0, "update": 0.0}
             aff, act = np.zeros(L + 1), np.zeros(L + 1)
             hop = {k: np.zeros(L + 1) for k in ("scatter", "update", "regather", "rebuilt", "in_edges", "rows_rebuilt")}
             rp.set_timing(False)
-            for i, (u, r) in enumerate(pinned):
+            for i, (u, r, ow) in enumerate(pinned):
                 if i == 5 + nb:
                     rp.set_timing(True)
                 t0 = time.perf_counter()
-                rp.apply_batch(u, r)
+                rp.apply_batch(u, r, ow)
                 dt = time.perf_counter() - t0
                 if i < 5:
                     continue
@@ -492,9 +504,9 @@ def run_table(args):
             if orc is not None:
                 spent, done = 0.0, 0
                 while spent < args.oracle_seconds and done < nb:
-                    ups, rows = ostream.next_batch(bsz)
+                    ups, rows, ow = draw_batch(ostream, w, bsz)
                     t0 = time.perf_counter()
-                    assert orc.apply_incremental(ups, rows) == 0
+                    assert orc.apply_incremental(ups, rows, op_weights=ow) == 0
                     spent += time.perf_counter() - t0
                     done += 1
                 line["oracle"] = {"updates_per_sec": bsz * done / spent, "batches": done, "cores": O.num_threads()}

@@ -56,9 +56,16 @@ typedef enum { RIPPLE_MEM_HOST = 0, RIPPLE_MEM_DEVICE = 1 } ripple_mem;
  * over all in-neighbours, or ignores the message; a sink whose cached maximum did not change is
  * not affected and propagates nothing (ripple_get_affected then lists exactly the vertices whose
  * cached maximum changed -- for SAGE also those whose own previous-layer row changed;
- * ripple_stats.senders those whose embedding changed). */
+ * ripple_stats.senders those whose embedding changed).
+ * WSUM_EDGE: the weighted sum of Table 1 with a stored weight alpha_uv per edge (the GC-W workload of
+ * Sec. 6.1.1): x_v = sum over in-neighbours u of alpha_uv h_u, no normalisation.  Weights are static:
+ * an edge takes its weight when it is created (ripple_graph.weight, or the per-operation weights of
+ * ripple_apply_batch_weighted) and keeps it for as long as it exists at batch boundaries -- adding an
+ * edge that exists is a counted no-op whatever weight comes with it.  Messages along an edge are scaled
+ * by its weight (Sec. 3.3.3, "other linear aggregators"). */
 typedef enum {
-    RIPPLE_AGG_SUM = 0, RIPPLE_AGG_MEAN = 1, RIPPLE_AGG_WSUM_GCN = 2, RIPPLE_AGG_MAX = 3, RIPPLE_AGG_MIN = 4
+    RIPPLE_AGG_SUM = 0, RIPPLE_AGG_MEAN = 1, RIPPLE_AGG_WSUM_GCN = 2, RIPPLE_AGG_MAX = 3, RIPPLE_AGG_MIN = 4,
+    RIPPLE_AGG_WSUM_EDGE = 5
 } ripple_agg;
 
 /* Update functions (Eq. 2) of the model families of Sec. 6.1.1, x_v = normalised aggregate:
@@ -89,13 +96,15 @@ typedef struct {
 } ripple_update;
 
 /* Initial graph in coordinate form: num_edges distinct pairs (src[i], dst[i]), any order.
- * src / dst: HOST|DEVICE per `mem`.  Duplicate pairs are not allowed (not checked). */
+ * src / dst / weight: HOST|DEVICE per `mem`.  Duplicate pairs are not allowed (not checked).
+ * weight: one fp32 weight per edge, read for RIPPLE_AGG_WSUM_EDGE only (NULL there: all ones). */
 typedef struct {
     int64_t num_vertices;
     int64_t num_edges;
     const int32_t* src;
     const int32_t* dst;
     int32_t mem; /* ripple_mem */
+    const float* weight;
 } ripple_graph;
 
 /* One layer.  Matrices are input-major: Wa[k * cols + j] multiplies input k into output j.
@@ -157,7 +166,8 @@ typedef struct {
                              present largest entry: a row that keeps its size is gathered anew every
                              rebuild_budget^2 batches that touch it, a row that lost a large term (an
                              edge from a hub deleted) at once.  0: default (8); < 0: never.  Applies to
-                             aggregates of input-width rows and to all aggregates of RIPPLE_AGG_SUM.   */
+                             aggregates of input-width rows and to all aggregates of the unnormalised
+                             sums (RIPPLE_AGG_SUM, RIPPLE_AGG_WSUM_EDGE).                                 */
 } ripple_options;
 
 typedef struct {
@@ -214,6 +224,13 @@ ripple_status ripple_create(const ripple_graph* g, const float* features, int32_
 ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update* ups, int64_t n,
                                  const float* feat_rows, int64_t n_rows, int32_t mem);
 
+/* The same for a graph with stored edge weights (RIPPLE_AGG_WSUM_EDGE): edge_weights holds one fp32
+ * weight per operation (HOST|DEVICE per `mem`, n entries), read only where ups[i] is an ADD_EDGE that
+ * creates its edge.  NULL: every new edge gets weight 1. */
+ripple_status ripple_apply_batch_weighted(ripple_ctx* ctx, const ripple_update* ups, int64_t n,
+                                          const float* feat_rows, int64_t n_rows, const float* edge_weights,
+                                          int32_t mem);
+
 /* Sec. 3.1: updated predictions are available right after the batch.  *dev_ptr: DEVICE pointer
  * to H^layer (N x *ld), layer in 0..L. */
 ripple_status ripple_get_embeddings(ripple_ctx* ctx, int32_t layer, const float** dev_ptr, int64_t* ld);
@@ -233,6 +250,11 @@ ripple_status ripple_get_affected(ripple_ctx* ctx, int32_t layer, const int32_t*
 /* Current graph in canonical CSR over out-edges: rowptr (HOST, N + 1 entries), col (HOST,
  * col_capacity >= number of edges, ascending within each row).  For parity checks. */
 ripple_status ripple_export_graph(ripple_ctx* ctx, int64_t* rowptr, int32_t* col, int64_t col_capacity);
+
+/* ripple_export_graph plus the stored weight of every edge, in the order of col (HOST, col_capacity
+ * entries; all ones unless the aggregator is RIPPLE_AGG_WSUM_EDGE). */
+ripple_status ripple_export_graph_weighted(ripple_ctx* ctx, int64_t* rowptr, int32_t* col, float* weight,
+                                           int64_t col_capacity);
 
 /* The same canonical CSR as ripple_export_graph, for callers that must not allocate device
  * memory.  (The paper has no counterpart: this is a property of this library, not of the method.)

@@ -48,7 +48,7 @@ __global__ void k_capacities(int N, const int32_t* __restrict__ deg, int32_t* ca
 }
 
 __global__ void k_fill_rows(const int32_t* __restrict__ src, const int32_t* __restrict__ dst,
-                            int64_t E, int N, Side out, Side in) {
+                            const float* __restrict__ weight, int64_t E, int N, Side out, Side in) {
     pdl_enter();
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < E;
          e += (int64_t)gridDim.x * blockDim.x) {
@@ -58,6 +58,11 @@ __global__ void k_fill_rows(const int32_t* __restrict__ src, const int32_t* __re
         out.col[out.start[u] + p] = v;
         int q = atomicAdd(&in.cnt_add[v], 1);
         in.col[in.start[v] + q] = u;
+        if (out.w) {
+            const float a = weight ? weight[e] : 1.0f;
+            out.w[out.start[u] + p] = a;
+            in.w[in.start[v] + q] = a;
+        }
     }
 }
 
@@ -75,8 +80,8 @@ static cudaError_t alloc_side(Side& s, int N) {
     return cudaMemset(s.free_cnt, 0, sizeof(int32_t) * RP_POOL_CLASSES);
 }
 
-cudaError_t graph_build(Ctx* c, const int32_t* src, const int32_t* dst, int64_t E, double slack,
-                        int64_t pool_edges) {
+cudaError_t graph_build(Ctx* c, const int32_t* src, const int32_t* dst, const float* weight, int64_t E,
+                        double slack, int64_t pool_edges) {
     cudaError_t e;
     const int N = c->N;
     for (int s = 0; s < 2; ++s)
@@ -98,8 +103,9 @@ cudaError_t graph_build(Ctx* c, const int32_t* src, const int32_t* dst, int64_t 
         sd.base_end = (int64_t)c->ctl_host->pool_next[s];
         sd.col_size = sd.base_end + pool_edges;
         if ((e = cudaMalloc(&sd.col, sizeof(int32_t) * (size_t)std::max<int64_t>(sd.col_size, 4)))) return e;
+        if (c->weighted && (e = cudaMalloc(&sd.w, sizeof(float) * (size_t)std::max<int64_t>(sd.col_size, 4)))) return e;
     }
-    if (E > 0) RP_LAUNCH(c, k_fill_rows, grid_e, T, 0, src, dst, E, N, out, in);
+    if (E > 0) RP_LAUNCH(c, k_fill_rows, grid_e, T, 0, src, dst, weight, E, N, out, in);
     for (int s = 0; s < 2; ++s)
         if ((e = cudaMemsetAsync(c->side[s].cnt_add, 0, sizeof(int32_t) * (size_t)N, c->stream))) return e;
     return cudaStreamSynchronize(c->stream);
@@ -242,7 +248,7 @@ __global__ void __launch_bounds__(256)
 k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, Ctl* ctl,
           const unsigned long long* __restrict__ hwin, const int32_t* __restrict__ op_slot,
           const int32_t* __restrict__ feat_last, const int32_t* __restrict__ vdel_seq, Side out, Side in,
-          Rec* rec, uint32_t* bitmap) {
+          Rec* rec, uint32_t* bitmap, const float* __restrict__ op_w) {
     pdl_enter();
     __shared__ int s_found;
     if (ctl->abort) return;
@@ -276,6 +282,9 @@ k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_
             x.u = op.u; x.v = op.v; x.sign = is_add ? 1 : -1;
             x.pos[0] = j_out; x.pos[1] = j_in;
             x.tail_val[0] = x.tail_val[1] = RP_TOMB;
+            x.tail_w[0] = x.tail_w[1] = 0.f;
+            // stored weights: a new edge takes the weight given with its operation, a deleted one had ...
+            x.w = !out.w ? 1.0f : is_add ? ((op_w && i < n_given) ? op_w[i] : 1.0f) : out.w[out.start[op.u] + j_out];
             x.deg_out_old = out.deg[op.u];
             x.rep[0] = atomicAdd(&out.touch[op.u], 1) == 0;
             x.rep[1] = atomicAdd(&in.touch[op.v], 1) == 0;
@@ -385,7 +394,8 @@ void graph_batch_classify(Ctx* c, int n) {
               c->hsize - 1, c->op_slot, c->feat_last, c->vdel_seq);
     int grid = std::min(n, c->n_sm * 8);
     RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, c->op_seq, c->ctl, c->hwin, c->op_slot, c->feat_last,
-              c->vdel_seq, c->side[0], c->side[1], c->rec, c->bitmap);
+              c->vdel_seq, c->side[0], c->side[1], c->rec, c->bitmap,
+              (const float*)(c->has_opw ? c->opw_dev : nullptr));
     RP_LAUNCH(c, k_plan_growth, std::min(div_up(2 * n, T), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[0],
               c->side[1], c->grow_list[0], c->grow_list[1], c->shrink_list[0], c->shrink_list[1]);
     RP_LAUNCH(c, k_plan_check, 1, 1, 0, c->ctl, c->side[0], c->side[1]);
@@ -422,6 +432,7 @@ __global__ void k_del_tail_read(Ctl* ctl, Rec* rec, Side out, Side in) {
         int row = s ? x.v : x.u;
         int new_deg = sd.deg[row] - sd.cnt_del[row];
         x.tail_val[s] = sd.col[sd.start[row] + new_deg + x.rank[s]];
+        if (sd.w) x.tail_w[s] = sd.w[sd.start[row] + new_deg + x.rank[s]];
     }
 }
 
@@ -437,6 +448,7 @@ __global__ void k_del_tail_pack(Ctl* ctl, const Rec* __restrict__ rec, Side out,
         int new_deg = sd.deg[row] - sd.cnt_del[row];
         int t = atomicAdd(&sd.tick_a[row], 1);
         sd.col[sd.start[row] + new_deg + t] = x.tail_val[s];
+        if (sd.w) sd.w[sd.start[row] + new_deg + t] = x.tail_w[s];
     }
 }
 
@@ -453,6 +465,7 @@ __global__ void k_del_fill(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side
         if (x.pos[s] >= new_deg) continue;
         int t = atomicAdd(&sd.tick_b[row], 1);
         sd.col[sd.start[row] + x.pos[s]] = sd.col[sd.start[row] + new_deg + t];
+        if (sd.w) sd.w[sd.start[row] + x.pos[s]] = sd.w[sd.start[row] + new_deg + t];
     }
 }
 
@@ -468,6 +481,8 @@ constexpr int GROW_BLOCK_ROW = 2048;
 __device__ __forceinline__ void move_row(Side& sd, int row, long long off, int ncap, int live, int tid, int nthreads) {
     const int64_t old = sd.start[row];
     for (int j = tid; j < live; j += nthreads) sd.col[off + j] = sd.col[old + j];
+    if (sd.w)
+        for (int j = tid; j < live; j += nthreads) sd.w[off + j] = sd.w[old + j];
 }
 
 __global__ void __launch_bounds__(256)
@@ -553,6 +568,7 @@ __global__ void k_add_write(Ctl* ctl, const Rec* __restrict__ rec, Side out, Sid
         int row = s ? x.v : x.u;
         int live = sd.deg[row] - sd.cnt_del[row];
         sd.col[sd.start[row] + live + x.rank[s]] = s ? x.u : x.v;
+        if (sd.w) sd.w[sd.start[row] + live + x.rank[s]] = x.w;
     }
 }
 
@@ -648,18 +664,21 @@ void graph_batch_cleanup(Ctx* c, int n) {
 // ---------------------------------------------------------------------------------------------
 // canonical export (parity checks)
 // ---------------------------------------------------------------------------------------------
-__global__ void k_export_rows(int N, Side out, const int64_t* __restrict__ rowptr, int32_t* col) {
+__global__ void k_export_rows(int N, Side out, const int64_t* __restrict__ rowptr, int32_t* col, float* weight) {
     pdl_enter();
     int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int nwarps = (gridDim.x * blockDim.x) >> 5;
     for (int v = warp; v < N; v += nwarps) {
         int64_t base = out.start[v], dst = rowptr[v];
         int deg = out.deg[v];
-        for (int j = lane_id(); j < deg; j += 32) col[dst + j] = out.col[base + j];
+        for (int j = lane_id(); j < deg; j += 32) {
+            col[dst + j] = out.col[base + j];
+            if (weight) weight[dst + j] = out.w ? out.w[base + j] : 1.0f;
+        }
     }
 }
 
-cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, int64_t col_capacity, int64_t* n_edges) {
+cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, float* weight, int64_t col_capacity, int64_t* n_edges) {
     cudaError_t e;
     const int N = c->N;
     std::vector<int32_t> deg((size_t)N);
@@ -672,19 +691,40 @@ cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, int64_t col_capa
     if (rowptr[N] == 0) return cudaSuccess;
     int64_t* rp_dev = nullptr;
     int32_t* col_dev = nullptr;
+    float* w_dev = nullptr;
     if ((e = cudaMalloc(&rp_dev, sizeof(int64_t) * ((size_t)N + 1)))) return e;
     if ((e = cudaMalloc(&col_dev, sizeof(int32_t) * (size_t)rowptr[N]))) { cudaFree(rp_dev); return e; }
+    if (weight && (e = cudaMalloc(&w_dev, sizeof(float) * (size_t)rowptr[N]))) { cudaFree(rp_dev); cudaFree(col_dev); return e; }
     e = cudaMemcpyAsync(rp_dev, rowptr, sizeof(int64_t) * ((size_t)N + 1), cudaMemcpyHostToDevice, c->stream);
     if (!e) {
-        RP_LAUNCH(c, k_export_rows, c->n_sm * 8, 256, 0, N, c->side[0], rp_dev, col_dev);
+        RP_LAUNCH(c, k_export_rows, c->n_sm * 8, 256, 0, N, c->side[0], rp_dev, col_dev, w_dev);
         e = cudaMemcpyAsync(col, col_dev, sizeof(int32_t) * (size_t)rowptr[N], cudaMemcpyDeviceToHost, c->stream);
+        if (!e && weight)
+            e = cudaMemcpyAsync(weight, w_dev, sizeof(float) * (size_t)rowptr[N], cudaMemcpyDeviceToHost, c->stream);
     }
     if (!e) e = cudaStreamSynchronize(c->stream);
     cudaFree(rp_dev);
     cudaFree(col_dev);
+    cudaFree(w_dev);
     if (e) return e;
+    if (!weight) {
 #pragma omp parallel for schedule(dynamic, 1024)
-    for (int v = 0; v < N; ++v) std::sort(col + rowptr[v], col + rowptr[v + 1]);
+        for (int v = 0; v < N; ++v) std::sort(col + rowptr[v], col + rowptr[v + 1]);
+        return cudaSuccess;
+    }
+    // rows sorted by neighbour id, the weights moving with their entries
+#pragma omp parallel
+    {
+        std::vector<std::pair<int32_t, float>> tmp;
+#pragma omp for schedule(dynamic, 1024)
+        for (int v = 0; v < N; ++v) {
+            const int64_t b = rowptr[v], n = rowptr[v + 1] - b;
+            tmp.resize((size_t)n);
+            for (int64_t j = 0; j < n; ++j) tmp[(size_t)j] = {col[b + j], weight[b + j]};
+            std::sort(tmp.begin(), tmp.end(), [](const std::pair<int32_t, float>& x, const std::pair<int32_t, float>& y) { return x.first < y.first; });
+            for (int64_t j = 0; j < n; ++j) { col[b + j] = tmp[(size_t)j].first; weight[b + j] = tmp[(size_t)j].second; }
+        }
+    }
     return cudaSuccess;
 }
 
@@ -784,7 +824,7 @@ extern "C" ripple_status ripple_export_graph_static(ripple_ctx* ctx, int64_t* ro
     if (E == 0) return RIPPLE_OK;
     e = cudaMemcpyAsync(sc.rowptr, rowptr, sizeof(int64_t) * ((size_t)N + 1), cudaMemcpyHostToDevice, c->stream);
     if (!e) {
-        k_export_rows<<<c->n_sm * 8, 256, 0, c->stream>>>(N, c->side[0], sc.rowptr, sc.col);
+        k_export_rows<<<c->n_sm * 8, 256, 0, c->stream>>>(N, c->side[0], sc.rowptr, sc.col, nullptr);
         e = cudaGetLastError();
     }
     if (!e) e = cudaMemcpyAsync(col, sc.col, sizeof(int32_t) * (size_t)E, cudaMemcpyDeviceToHost, c->stream);

@@ -64,7 +64,7 @@ static void destroy_ctx(Ctx* c) {
     if (c->stream) cudaStreamSynchronize(c->stream);
     for (int s = 0; s < 2; ++s) {
         Side& sd = c->side[s];
-        cudaFree(sd.col); cudaFree(sd.start); cudaFree(sd.cap); cudaFree(sd.deg);
+        cudaFree(sd.col); cudaFree(sd.w); cudaFree(sd.start); cudaFree(sd.cap); cudaFree(sd.deg);
         cudaFree(sd.cnt_del); cudaFree(sd.cnt_add); cudaFree(sd.tick_a); cudaFree(sd.tick_b); cudaFree(sd.touch);
         cudaFree(c->grow_list[s]); cudaFree(c->shrink_list[s]); cudaFree(c->D[s]); cudaFree(c->Clist[s]);
         cudaFree(sd.free_blk); cudaFree(sd.free_cnt);
@@ -75,7 +75,7 @@ static void destroy_ctx(Ctx* c) {
         for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2, &c->layer[l].tc_self}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
     cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->invmask); cudaFree(c->posmap); cudaFree(c->deg_out_old);
-    cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
+    cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->opw_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
     cudaFree(c->moved_start); cudaFree(c->moved_cap);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
@@ -139,7 +139,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
     g_create_err[0] = 0;
     if (!g || !features || !layers || !out) { set_err(nullptr, "null argument"); return st; }
     if (L < 1 || L > RP_MAXL) { set_err(nullptr, "L must be in 1..%d", RP_MAXL); return st; }
-    if (agg < 0 || agg > 4) { set_err(nullptr, "unknown aggregator %d", agg); return st; }
+    if (agg < 0 || agg > 5) { set_err(nullptr, "unknown aggregator %d", agg); return st; }
     if (rp_monotonic(agg) && layers[0].kind == RIPPLE_LAYER_GIN) {
         set_err(nullptr, "the max and min aggregators are built for GRAPHCONV and SAGE layers");
         return st;
@@ -169,6 +169,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         if (!c) { set_err(nullptr, "host allocation failed"); return RIPPLE_ERR_OOM; }
         memset(static_cast<void*>(c), 0, sizeof(Ctx));
         int32_t *src_dev = nullptr, *dst_dev = nullptr;
+        float* w_dev = nullptr;
         bool own_coo = false;
         const int N = (int)g->num_vertices;
         const int64_t E = g->num_edges;
@@ -185,6 +186,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         c->rebuild_tau2 = o.rebuild_budget > 0.f ? o.rebuild_budget * o.rebuild_budget : 64.f;
         c->self_term = layers[0].kind != RIPPLE_LAYER_GRAPHCONV;
         c->src_norm = agg == RIPPLE_AGG_WSUM_GCN;
+        c->weighted = agg == RIPPLE_AGG_WSUM_EDGE;
         CK(dev_alloc(&c->ctl, 1, 0));
         CK(dev_alloc(&c->params_dev, 2, 0));
         CK(cudaMallocHost(&c->params_host, 2 * sizeof(int)));
@@ -211,13 +213,18 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             CK(dev_alloc(&dst_dev, (size_t)E));
             CK(cudaMemcpyAsync(src_dev, g->src, sizeof(int32_t) * (size_t)E, cudaMemcpyHostToDevice, c->stream));
             CK(cudaMemcpyAsync(dst_dev, g->dst, sizeof(int32_t) * (size_t)E, cudaMemcpyHostToDevice, c->stream));
+            if (c->weighted && g->weight) {
+                CK(dev_alloc(&w_dev, (size_t)E));
+                CK(cudaMemcpyAsync(w_dev, g->weight, sizeof(float) * (size_t)E, cudaMemcpyHostToDevice, c->stream));
+            }
         } else {
             src_dev = const_cast<int32_t*>(g->src);
             dst_dev = const_cast<int32_t*>(g->dst);
+            w_dev = c->weighted ? const_cast<float*>(g->weight) : nullptr;
         }
         {
-            cudaError_t e = graph_build(c, src_dev, dst_dev, E, o.slack, o.pool_edges);
-            if (own_coo) { cudaFree(src_dev); cudaFree(dst_dev); }
+            cudaError_t e = graph_build(c, src_dev, dst_dev, w_dev, E, o.slack, o.pool_edges);
+            if (own_coo) { cudaFree(src_dev); cudaFree(dst_dev); cudaFree(w_dev); }
             CK(e);
             if (c->ctl_host->err) {
                 set_err(nullptr, "an edge endpoint is outside [0, N)");
@@ -264,7 +271,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                 // pieces and keeps no rounding budget for it.  That is left to the normalised
                 // aggregators, whose rows stay of one size; an unnormalised sum folds in a pass of its
                 // own, with the budget.
-                c->fused_fold[l] = c->pre[l] && agg != RIPPLE_AGG_SUM;
+                c->fused_fold[l] = c->pre[l] && agg != RIPPLE_AGG_SUM && agg != RIPPLE_AGG_WSUM_EDGE;
                 // measured on the dense graph: rebuilding every aggregate costs 0.47 of pushing a message
                 // along every edge at 256 floats per row (12.1 against 26 ms) and 0.54 at 48 (3.5 / 6.4 ms)
                 c->regather_min_messages = o.regather_threshold > 0.f ? 0 : (4ll << 20);
@@ -338,6 +345,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         CK(dev_alloc(&c->feat_last, (size_t)N, 0xFF));
         // batch staging
         CK(dev_alloc(&c->ups_dev, (size_t)o.max_batch));
+        if (c->weighted) CK(dev_alloc(&c->opw_dev, (size_t)o.max_batch));
         CK(dev_alloc(&c->feat_dev, (size_t)o.max_batch * c->d[0]));
         c->hsize = 1024;
         while (c->hsize < 4 * o.max_batch) c->hsize <<= 1;
@@ -448,7 +456,7 @@ static void arm_rebuild(Ctx* c, int nb) {
 static bool launch_batch_graph(Ctx* c, int nb) {
     if (c->no_graphs || c->timing || nb < 1 || nb > RP_GRAPH_MAX_BATCH) return false;
     // the captured chain differs with the expansion kernels and with the hops whose rebuilding form is enqueued
-    int key = 2 * nb + (c->may_expand ? 1 : 0);
+    int key = 4 * nb + (c->may_expand ? 1 : 0) + (c->has_opw ? 2 : 0);
     for (int l = 1; l <= c->L; ++l) key = 2 * key + (c->rebuild_armed[l] ? 1 : 0);
     int slot = -1;
     for (int i = 0; i < RP_GRAPH_SLOTS; ++i)
@@ -484,6 +492,12 @@ static bool launch_batch_graph(Ctx* c, int nb) {
 
 extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update* ups, int64_t n,
                                             const float* feat_rows, int64_t n_rows, int32_t mem) {
+    return ripple_apply_batch_weighted(ctx, ups, n, feat_rows, n_rows, nullptr, mem);
+}
+
+extern "C" ripple_status ripple_apply_batch_weighted(ripple_ctx* ctx, const ripple_update* ups, int64_t n,
+                                                     const float* feat_rows, int64_t n_rows,
+                                                     const float* edge_weights, int32_t mem) {
     Ctx* c = reinterpret_cast<Ctx*>(ctx);
     if (!c) return RIPPLE_ERR_INVALID_ARG;
     ripple_status st = RIPPLE_OK;
@@ -518,6 +532,8 @@ extern "C" ripple_status ripple_apply_batch(ripple_ctx* ctx, const ripple_update
     const cudaMemcpyKind kind = mem == RIPPLE_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
     // operations are always staged: generated edge deletions are appended behind them
     if (nb) CK(cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, kind, c->stream));
+    c->has_opw = c->weighted && edge_weights && nb;
+    if (c->has_opw) CK(cudaMemcpyAsync(c->opw_dev, edge_weights, sizeof(float) * (size_t)nb, kind, c->stream));
     if (mem == RIPPLE_MEM_HOST || try_graph) {
         // a replayed graph reads the library's own staging buffers, so device payload rows are copied too
         if (nr) CK(cudaMemcpyAsync(c->feat_dev, feat_rows, sizeof(float) * (size_t)nr * c->d[0], kind, c->stream));
@@ -621,7 +637,22 @@ extern "C" ripple_status ripple_export_graph(ripple_ctx* ctx, int64_t* rowptr, i
     if (!c || !rowptr || (!col && col_capacity > 0)) return RIPPLE_ERR_INVALID_ARG;
     cudaSetDevice(c->device);
     int64_t ne = 0;
-    cudaError_t e = graph_export(c, rowptr, col, col_capacity, &ne);
+    cudaError_t e = graph_export(c, rowptr, col, nullptr, col_capacity, &ne);
+    if (e == cudaErrorInvalidValue) {
+        set_err(c, "col_capacity %lld is smaller than the edge count %lld", (long long)col_capacity, (long long)ne);
+        return RIPPLE_ERR_INVALID_ARG;
+    }
+    if (e) { set_err(c, "export failed: %s", cudaGetErrorString(e)); return RIPPLE_ERR_CUDA; }
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_export_graph_weighted(ripple_ctx* ctx, int64_t* rowptr, int32_t* col, float* weight,
+                                                      int64_t col_capacity) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c || !rowptr || ((!col || !weight) && col_capacity > 0)) return RIPPLE_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    int64_t ne = 0;
+    cudaError_t e = graph_export(c, rowptr, col, weight, col_capacity, &ne);
     if (e == cudaErrorInvalidValue) {
         set_err(c, "col_capacity %lld is smaller than the edge count %lld", (long long)col_capacity, (long long)ne);
         return RIPPLE_ERR_INVALID_ARG;

@@ -63,6 +63,7 @@ struct Ctl {
 // (the tail of the same array) with doubled capacity.
 struct Side {
     int32_t* col;
+    float* w;          // stored weight of every entry of col (weighted sum with per-edge weights), else null
     int64_t* start;
     int32_t* cap;
     int32_t* deg;
@@ -89,6 +90,8 @@ struct Rec {
     int32_t tail_val[2]; // deleted: entry found at tail slot new_deg + rank
     int32_t rep[2];      // 1 for the first record that touched the row
     int32_t deg_out_old; // out-degree of u before the batch
+    float w;             // stored edge weights: weight of the added edge / weight the deleted edge had
+    float tail_w[2];     // deleted: weight found at the tail slot
 };
 
 // transposed (K contiguous), tf32-split copy of a weight block for the tensor-core layer update
@@ -118,6 +121,9 @@ struct Ctx {
     bool own_stream;
     int N, L, agg;
     bool self_term, src_norm;
+    bool weighted;             // every edge carries a stored weight (RIPPLE_AGG_WSUM_EDGE)
+    float* opw_dev;            // batch staging: one weight per operation (weighted only)
+    int has_opw;               // the batch being applied came with weights
     int64_t E0;
     int64_t max_batch;
     int scatter_mode, gemm_mode, timing;
@@ -233,12 +239,12 @@ inline int pad4(int x) { return (x + 3) & ~3; }
     } while (0)
 
 // graph_store.cu
-cudaError_t graph_build(Ctx* c, const int32_t* src_dev, const int32_t* dst_dev, int64_t E,
+cudaError_t graph_build(Ctx* c, const int32_t* src_dev, const int32_t* dst_dev, const float* w_dev, int64_t E,
                         double slack, int64_t pool_edges);
 void graph_batch_classify(Ctx* c, int n);   // validate, dedupe, find net changes, plan
 void graph_batch_mutate(Ctx* c, int n);                 // apply the net changes to both directions
 void graph_batch_cleanup(Ctx* c, int n);                // reset per-batch scratch
-cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, int64_t col_capacity, int64_t* n_edges);
+cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, float* weight, int64_t col_capacity, int64_t* n_edges);
 
 // frontier.cu
 void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, const int32_t* deg,

@@ -53,6 +53,8 @@ __device__ __forceinline__ void spmm_accumulate(float4 (&acc)[NV], const Side& i
     const int64_t base = in.start[v];
     for (int j0 = j_begin; j0 < j_end; j0 += 32) {
         int mine = j0 + lane < j_end ? in.col[base + j0 + lane] : 0;
+        // stored edge weights (weighted sum with per-edge weights): the entry's weight is its coefficient
+        float mine_w = (in.w && j0 + lane < j_end) ? in.w[base + j0 + lane] : 1.0f;
         int cnt = min(32, j_end - j0);
         constexpr int UNR = 4;
         for (int j = 0; j < cnt; j += UNR * EPI) {
@@ -63,8 +65,9 @@ __device__ __forceinline__ void spmm_accumulate(float4 (&acc)[NV], const Side& i
             for (int t = 0; t < UNR; ++t) {
                 const int jj = j + t * EPI + sub;
                 u[t] = __shfl_sync(FULL, mine, jj & 31);
+                const float wj = __shfl_sync(FULL, mine_w, jj & 31);
                 cu[t] = 0.f;
-                if (jj < cnt) cu[t] = src_norm ? coef_from_degree(deg_out[u[t]]) : 1.0f;
+                if (jj < cnt) cu[t] = src_norm ? coef_from_degree(deg_out[u[t]]) : wj;
                 else u[t] = -1;
             }
 #pragma unroll
@@ -217,6 +220,8 @@ k_scatter_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64
             const int cnt_total = (int)(seg_end - e);
             for (int j0 = 0; j0 < cnt_total; j0 += 32) {
                 int mine = j0 + lane < cnt_total ? out.col[base + j0 + lane] : 0;
+                // stored edge weights: the message along an edge is the sender's delta row times the edge's weight
+                float mine_w = (out.w && j0 + lane < cnt_total) ? out.w[base + j0 + lane] : 1.0f;
                 int cnt = min(32, cnt_total - j0);
                 // every sink joins the hop's affected set (same walk as the frontier's): one lane per
                 // edge, 32 edges per instruction
@@ -227,12 +232,13 @@ k_scatter_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64
                 for (int j = 0; j < cnt; j += EPI) {
                     int jj = j + sub;
                     int v = __shfl_sync(FULL, mine, jj & 31);
+                    const float a = __shfl_sync(FULL, mine_w, jj & 31);
                     if (jj < cnt) {
                         float* dst = S + (size_t)v * ld;
 #pragma unroll
                         for (int k = 0; k < NV; ++k) {
                             int q = ql + LPR * k;
-                            if (q < nq) red_add_v4(dst + 4 * q, d[k]);
+                            if (q < nq) red_add_v4(dst + 4 * q, make_float4(a * d[k].x, a * d[k].y, a * d[k].z, a * d[k].w));
                         }
                     }
                 }
@@ -388,18 +394,23 @@ k_scatter_pull(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const in
         bool any = false;
         for (int j0 = 0; j0 < deg; j0 += 32) {
             int p = -1;
-            if (j0 + lane < deg) p = posmap[in.col[base + j0 + lane]];
+            float wj = 1.0f;
+            if (j0 + lane < deg) {
+                p = posmap[in.col[base + j0 + lane]];
+                if (in.w) wj = in.w[base + j0 + lane];
+            }
             unsigned m = __ballot_sync(FULL, p >= 0);
             any |= m != 0;
             while (m) {
                 int j = __ffs(m) - 1;
                 m &= m - 1;
                 int pj = __shfl_sync(FULL, p, j);
+                const float a = __shfl_sync(FULL, wj, j);
                 const float4* drow = reinterpret_cast<const float4*>(D + (size_t)pj * ld);
 #pragma unroll
                 for (int k = 0; k < NV; ++k) {
                     int q = lane + 32 * k;
-                    if (q < nq) add4(acc[k], __ldg(drow + q), 1.0f);
+                    if (q < nq) add4(acc[k], __ldg(drow + q), a);
                 }
             }
         }
@@ -457,7 +468,7 @@ __global__ void k_scatter_records(Ctl* ctl, int l, const Rec* __restrict__ rec, 
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
     for (int r = warp; r < n; r += nwarps) {
-        const float sgn = (float)rec[r].sign;
+        const float sgn = (float)rec[r].sign * rec[r].w;   // (w = 1 unless edges carry stored weights)
         float* dst = S + (size_t)rec[r].v * ld;
         const float4* mrow = reinterpret_cast<const float4*>(M + (size_t)r * ld);
         for (int q = lane; q < nq; q += 32) {
@@ -694,12 +705,12 @@ void scatter_layer(Ctx* c, int l, int n) {
 #define PUSH(NV, LPR) RP_LAUNCH(c, (k_scatter_push<NV, LPR>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, ld, c->dS[l], c->bitmap)
 #define PULL(NV, LPR) RP_LAUNCH(c, (k_scatter_pull<NV, 32>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->posmap, Dm, ld, c->dS[l])
     // (rows too wide for two staging buffers per warp in the default shared-memory allowance take the ordinary form)
-    if (c->scatter_mode == RIPPLE_SCATTER_PUSH_BULK && (size_t)8 * 2 * ld * sizeof(float) <= (48u << 10)) {
+    if (c->scatter_mode == RIPPLE_SCATTER_PUSH_BULK && !c->weighted && (size_t)8 * 2 * ld * sizeof(float) <= (48u << 10)) {
         RP_LAUNCH(c, k_scatter_push_bulk, grid, T, (size_t)8 * 2 * ld * sizeof(float), c->ctl, l, senders, c->coff,
                   c->side[0], Dm, ld, c->dS[l], c->bitmap);
     } else if (c->scatter_mode != RIPPLE_SCATTER_PULL && c->scatter_mode != RIPPLE_SCATTER_REGATHER) {
-        if (ld == 48) RP_LAUNCH(c, k_scatter_push_packed<12>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
-        else if (ld == 40) RP_LAUNCH(c, k_scatter_push_packed<10>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
+        if (ld == 48 && !c->weighted) RP_LAUNCH(c, k_scatter_push_packed<12>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
+        else if (ld == 40 && !c->weighted) RP_LAUNCH(c, k_scatter_push_packed<10>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
         else RP_WIDTH_DISPATCH(ld, PUSH);
     }
     if (c->scatter_mode == RIPPLE_SCATTER_PULL) RP_WIDTH_DISPATCH(ld, PULL);

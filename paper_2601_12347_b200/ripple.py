@@ -19,7 +19,7 @@ LIB_PATH = os.environ.get("RIPPLE_LIB_PATH") or os.path.join(_HERE, "libripple.s
 MAX_LAYERS = 8
 OK, ERR_INVALID_ARG, ERR_VERTEX_RANGE, ERR_CAPACITY, ERR_OOM, ERR_CUDA, ERR_TIMEOUT = range(7)
 MEM_HOST, MEM_DEVICE = 0, 1
-AGG_SUM, AGG_MEAN, AGG_WSUM_GCN, AGG_MAX, AGG_MIN = 0, 1, 2, 3, 4
+AGG_SUM, AGG_MEAN, AGG_WSUM_GCN, AGG_MAX, AGG_MIN, AGG_WSUM_EDGE = 0, 1, 2, 3, 4, 5
 LAYER_SAGE, LAYER_GRAPHCONV, LAYER_GIN = 0, 1, 2
 ACT_IDENTITY, ACT_RELU = 0, 1
 OP_ADD_EDGE, OP_DEL_EDGE, OP_SET_FEATURE, OP_DEL_VERTEX = 0, 1, 2, 3
@@ -29,8 +29,9 @@ GEMM_AUTO, GEMM_FP32, GEMM_TF32 = 0, 1, 2
 UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
 
 EXPORTED = [
-    "ripple_create", "ripple_apply_batch", "ripple_get_embeddings", "ripple_get_aggregate",
-    "ripple_get_affected", "ripple_export_graph", "ripple_get_degrees", "ripple_recompute_full",
+    "ripple_create", "ripple_apply_batch", "ripple_apply_batch_weighted", "ripple_get_embeddings",
+    "ripple_get_aggregate", "ripple_get_affected", "ripple_export_graph", "ripple_export_graph_weighted",
+    "ripple_get_degrees", "ripple_recompute_full",
     "ripple_export_graph_static", "ripple_set_timing", "ripple_probe_reduction_rate", "ripple_probe_gather_rate",
     "ripple_get_stats", "ripple_last_error", "ripple_destroy", "ripple_version",
 ]
@@ -44,7 +45,8 @@ class RippleError(RuntimeError):
 
 class _Graph(ctypes.Structure):
     _fields_ = [("num_vertices", ctypes.c_int64), ("num_edges", ctypes.c_int64),
-                ("src", ctypes.c_void_p), ("dst", ctypes.c_void_p), ("mem", ctypes.c_int32)]
+                ("src", ctypes.c_void_p), ("dst", ctypes.c_void_p), ("mem", ctypes.c_int32),
+                ("weight", ctypes.c_void_p)]
 
 
 class _Layer(ctypes.Structure):
@@ -97,6 +99,8 @@ def load_library(path: Optional[str] = None):
     P = ctypes.POINTER
     lib.ripple_create.argtypes = [P(_Graph), vp, i32, P(_Layer), i32, i32, P(_Options), P(vp)]
     lib.ripple_apply_batch.argtypes = [vp, vp, i64, vp, i64, i32]
+    lib.ripple_apply_batch_weighted.argtypes = [vp, vp, i64, vp, i64, vp, i32]
+    lib.ripple_export_graph_weighted.argtypes = [vp, vp, vp, vp, i64]
     lib.ripple_get_embeddings.argtypes = [vp, i32, P(vp), P(i64)]
     lib.ripple_get_aggregate.argtypes = [vp, i32, P(vp), P(i64), P(i32), P(i32)]
     lib.ripple_get_affected.argtypes = [vp, i32, P(vp), P(i64)]
@@ -114,7 +118,7 @@ def load_library(path: Optional[str] = None):
     lib.ripple_set_timing.argtypes = [vp, i32]
     lib.ripple_probe_reduction_rate.argtypes = [i32, i64, i32, i64, i32, P(ctypes.c_float)]
     lib.ripple_probe_gather_rate.argtypes = [i32, i64, i32, i64, P(ctypes.c_float)]
-    for name in EXPORTED[:13]:
+    for name in EXPORTED[:15]:
         getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -145,7 +149,7 @@ class Ripple:
                  slack: float = 0.0, pool_edges: int = 0, max_batch: int = 0,
                  scatter_mode: int = SCATTER_AUTO, gemm_mode: int = GEMM_AUTO, timing: bool = False,
                  pre_transform: bool = True, graphs: bool = True, stream=None,
-                 regather_threshold: float = 0.0, rebuild_budget: float = 0.0):
+                 regather_threshold: float = 0.0, rebuild_budget: float = 0.0, edge_weights=None):
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -166,6 +170,17 @@ class Ripple:
             dst = np.ascontiguousarray(dst, dtype=np.int32)
             g.num_edges, g.src, g.dst, g.mem = src.size, src.ctypes.data, dst.ctypes.data, MEM_HOST
         keep += [src, dst]
+        if edge_weights is not None:       # one stored weight per edge (AGG_WSUM_EDGE), same memory space as src / dst
+            if _is_torch_cuda(edge_weights):
+                assert g.mem == MEM_DEVICE and edge_weights.dtype == torch.float32
+                edge_weights = edge_weights.contiguous()
+                g.weight = edge_weights.data_ptr()
+            else:
+                assert g.mem == MEM_HOST
+                edge_weights = np.ascontiguousarray(edge_weights, dtype=np.float32)
+                g.weight = edge_weights.ctypes.data
+            assert edge_weights.shape[0] == g.num_edges
+            keep.append(edge_weights)
         if _is_torch_cuda(features):
             assert features.dtype == torch.float32
             features = features.contiguous()
@@ -223,9 +238,10 @@ class Ripple:
         return self._stream
 
     # ---- the hot path ----------------------------------------------------------------------
-    def apply_batch(self, ups, feat_rows=None) -> None:
+    def apply_batch(self, ups, feat_rows=None, op_weights=None) -> None:
         """ups: numpy array of UPDATE_DTYPE (host) or CUDA int32 tensor [n, 3] (device);
-        feat_rows: [n_rows, d0] fp32 in the same memory space."""
+        feat_rows: [n_rows, d0] fp32 in the same memory space; op_weights: [n] fp32 in the same
+        memory space, the weight of every ADD_EDGE (graphs with stored edge weights only)."""
         if _is_torch_cuda(ups):
             ups = ups.contiguous()
             n, uptr, mem = ups.shape[0], ups.data_ptr(), MEM_DEVICE
@@ -248,7 +264,19 @@ class Ripple:
             else:
                 feat_rows = np.ascontiguousarray(feat_rows, dtype=np.float32)
                 nr, fptr = feat_rows.shape[0], feat_rows.ctypes.data
-        self._check(self.lib.ripple_apply_batch(self.h, uptr, n, fptr, nr, mem))
+        if op_weights is None:
+            self._check(self.lib.ripple_apply_batch(self.h, uptr, n, fptr, nr, mem))
+            return
+        if mem == MEM_DEVICE:
+            op_weights = op_weights.contiguous()
+            wptr = op_weights.data_ptr()
+        elif hasattr(op_weights, "numpy"):
+            wptr = op_weights.data_ptr()
+        else:
+            op_weights = np.ascontiguousarray(op_weights, dtype=np.float32)
+            wptr = op_weights.ctypes.data
+        assert op_weights.shape[0] == n
+        self._check(self.lib.ripple_apply_batch_weighted(self.h, uptr, n, fptr, nr, wptr, mem))
 
     def set_timing(self, on: bool) -> None:
         self._check(self.lib.ripple_set_timing(self.h, int(bool(on))))
@@ -296,6 +324,16 @@ class Ripple:
         col = np.zeros(max(e, 1), dtype=np.int32)
         self._check(self.lib.ripple_export_graph(self.h, rowptr.ctypes.data, col.ctypes.data, col.size))
         return rowptr, col[: rowptr[-1]]
+
+    def export_graph_weighted(self) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        """export_graph() plus the stored weight of every edge, in the order of col."""
+        e = self.stats()["num_edges"]
+        rowptr = np.zeros(self.n + 1, dtype=np.int64)
+        col = np.zeros(max(e, 1), dtype=np.int32)
+        w = np.zeros(max(e, 1), dtype=np.float32)
+        self._check(self.lib.ripple_export_graph_weighted(self.h, rowptr.ctypes.data, col.ctypes.data,
+                                                          w.ctypes.data, col.size))
+        return rowptr, col[: rowptr[-1]], w[: rowptr[-1]]
 
     def export_graph_static(self) -> Tuple[np.ndarray, np.ndarray]:
         """Same result as export_graph() through the entry point that allocates no device memory.

@@ -56,3 +56,28 @@ def test_fp32_floor_of_the_gin_sum_stack(gin_state):
     # and the reason is the row magnitude, not a bug of this evaluation: relative to the row's
     # largest entry every layer is at a few fp32 roundings
     assert max(frac) < 64 * 2.0 ** -24
+
+
+def test_fp32_floor_of_the_weighted_sum_stack():
+    """GraphConv with a stored weight per edge (no normalisation) on the same graph: the same floor."""
+    w = I.workloads()["sparse-gcw"]
+    src, dst = I.make_graph(w)
+    ew = I.edge_weights(src.size, w.seed)
+    X = I.features(w.n, w.model.dims[0], w.seed)
+    W = I.make_weights(w.model, w.seed)
+    orc = Oracle(w.n, src, dst, X, w.model, W, edge_weights=ew)
+    A_t = sp.csr_matrix((ew, (dst, src)), shape=(w.n, w.n))
+    H = X.astype(np.float32)
+    plain, frac = [], []
+    for l, (ly, wl) in enumerate(zip(w.model.layers, W), 1):
+        H = ((A_t @ H).astype(np.float32) @ wl["Wa"] + wl["ba"]).astype(np.float32)
+        if ly.act == I.ACT_RELU:
+            H = np.maximum(H, 0)
+        ref = orc.H(l)
+        err = np.abs(H.astype(np.float64) - ref)
+        plain.append(float(np.max(err / (1.0 + np.abs(ref)))))
+        frac.append(float(np.max(err / np.maximum(np.max(np.abs(ref), axis=1, keepdims=True), 1e-30))))
+    print("fp32 evaluation vs fp64 oracle: north_star criterion", plain, "fraction of row maximum", frac)
+    for f in frac:
+        assert GIN_FP32_FLOOR / 4 <= f <= GIN_FP32_FLOOR, f
+    assert plain[1] > 5 * TOL
