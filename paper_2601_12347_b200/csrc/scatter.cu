@@ -253,7 +253,8 @@ k_scatter_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64
 // messages are laid end to end over the lanes of consecutive instructions (8 messages over 3
 // instructions for 12 lanes), so every reduction instruction carries 32 active lanes instead of
 // 24.  Lane t of instruction i serves float4 slot (32 i + t) % NQ of message (32 i + t) / NQ.
-template <int NQ>
+// WEIGHTED: edges carry stored weights, the message along an edge is the delta row times its weight.
+template <int NQ, bool WEIGHTED>
 __global__ void __launch_bounds__(256)
 k_scatter_push_packed(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64_t* __restrict__ coff,
                       Side out, const float* __restrict__ D, float* S, uint32_t* bitmap) {
@@ -285,6 +286,8 @@ k_scatter_push_packed(Ctl* ctl, int l, const int32_t* __restrict__ senders, cons
             const int cnt_total = (int)(seg_end - e);
             for (int j0 = 0; j0 < cnt_total; j0 += 32) {
                 int mine = j0 + lane < cnt_total ? out.col[base + j0 + lane] : 0;
+                float mine_w = 1.0f;
+                if (WEIGHTED && j0 + lane < cnt_total) mine_w = out.w[base + j0 + lane];
                 int cnt = min(32, cnt_total - j0);
                 if (lane < cnt) {
                     const uint32_t m = 1u << (mine & 31);
@@ -295,7 +298,12 @@ k_scatter_push_packed(Ctl* ctl, int l, const int32_t* __restrict__ senders, cons
                     for (int k = 0; k < NI; ++k) {
                         const int idx = g0 + msg_of[k];
                         const int v = __shfl_sync(FULL, mine, idx & 31);
-                        if (idx < cnt) red_add_v4(S + (size_t)v * LD + 4 * slot_of[k], d[k]);
+                        float4 m4 = d[k];
+                        if (WEIGHTED) {
+                            const float a = __shfl_sync(FULL, mine_w, idx & 31);
+                            m4 = make_float4(a * m4.x, a * m4.y, a * m4.z, a * m4.w);
+                        }
+                        if (idx < cnt) red_add_v4(S + (size_t)v * LD + 4 * slot_of[k], m4);
                     }
                 }
             }
@@ -709,8 +717,12 @@ void scatter_layer(Ctx* c, int l, int n) {
         RP_LAUNCH(c, k_scatter_push_bulk, grid, T, (size_t)8 * 2 * ld * sizeof(float), c->ctl, l, senders, c->coff,
                   c->side[0], Dm, ld, c->dS[l], c->bitmap);
     } else if (c->scatter_mode != RIPPLE_SCATTER_PULL && c->scatter_mode != RIPPLE_SCATTER_REGATHER) {
-        if (ld == 48 && !c->weighted) RP_LAUNCH(c, k_scatter_push_packed<12>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
-        else if (ld == 40 && !c->weighted) RP_LAUNCH(c, k_scatter_push_packed<10>, grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap);
+#define PACKED(NQ, WGT) RP_LAUNCH(c, (k_scatter_push_packed<NQ, WGT>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap)
+        if (ld == 48 && c->weighted) PACKED(12, true);
+        else if (ld == 48) PACKED(12, false);
+        else if (ld == 40 && c->weighted) PACKED(10, true);
+        else if (ld == 40) PACKED(10, false);
+#undef PACKED
         else RP_WIDTH_DISPATCH(ld, PUSH);
     }
     if (c->scatter_mode == RIPPLE_SCATTER_PULL) RP_WIDTH_DISPATCH(ld, PULL);

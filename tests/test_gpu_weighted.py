@@ -30,6 +30,8 @@ def weighted_models():
         "gc_2l": I.graphconv_model([18, 36, 10], I.AGG_WSUM_EDGE),
         "gc_3l": I.graphconv_model([18, 36, 20, 10], I.AGG_WSUM_EDGE),
         "sage_2l": I.sage_model([18, 36, 10], I.AGG_WSUM_EDGE),
+        "gc_47": I.graphconv_model([18, 64, 47], I.AGG_WSUM_EDGE),     # messages of 48 and 40 floats take the
+        "gc_40": I.graphconv_model([18, 64, 40], I.AGG_WSUM_EDGE),     # lane-packed form of the push
     }
 
 
