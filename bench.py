@@ -181,7 +181,7 @@ def run_reference(args, rank, world):
             ups = ups[:n_sample]
             ow = ow[:n_sample] if ow is not None else None
         t0 = time.perf_counter()
-        assert orc.apply_incremental(ups, rows, op_weights=ow) == 0
+        assert orc.apply_incremental(ups, rows, pull=True, op_weights=ow) == 0
         dt = time.perf_counter() - t0
         if s == 0 and dt * (args.warmup + args.steps) > budget_s:
             n_sample = max(1, int(args.batch * budget_s / (dt * (args.warmup + args.steps))))
@@ -198,33 +198,42 @@ def run_reference(args, rank, world):
         "config": {"workload": f"{args.workload}, batch {args.batch}", "batch": args.batch,
                    "vertices": w.n, "edges": w.e, "dims": w.model.dims},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": f"{len(lat)} steps of {n_sample} updates (of batches of {args.batch}), incremental route; "
-                                   "message scatter single-threaded, compute step on all cores"},
+                         "sample": f"{len(lat)} steps of {n_sample} updates (of batches of {args.batch}), incremental route, "
+                                   "messages gathered per affected sink on all cores"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "latency_ms": {"p50": 1e3 * pct(lat, 50), "p99": 1e3 * pct(lat, 99)},
     }
     print(json.dumps(line), flush=True)
 
 
-def cpu_baseline(args, w, src, dst, X, W, budget_s=20.0):
-    """The oracle as it stands, timed on the host cores on a bounded sample of the workload."""
+def cpu_baseline(args, w, src, dst, X, W, budget_s=16.0):
+    """The oracle as it stands, timed on the host cores on a bounded sample of the workload: the
+    incremental route with its messages gathered per affected sink on all cores (the faster of its two
+    delivery orders), and, on a shorter sample, with its messages pushed by one thread."""
     from oracle import oracle as O
     O.build()
     t0 = time.perf_counter()
     orc = O.Oracle(w.n, src, dst, X, w.model, W, edge_weights=w.edge_w)
     setup = time.perf_counter() - t0
     stream = I.make_stream(w, src, dst)
-    spent, nb = 0.0, 0
-    while spent < budget_s and nb < 50:
-        ups, rows, ow = draw_batch(stream, w, args.batch)
-        t0 = time.perf_counter()
-        assert orc.apply_incremental(ups, rows, op_weights=ow) == 0
-        spent += time.perf_counter() - t0
-        nb += 1
+    out = {}
+    for pull, budget in ((True, budget_s), (False, budget_s / 2)):
+        spent, nb = 0.0, 0
+        while spent < budget and nb < 50:
+            ups, rows, ow = draw_batch(stream, w, args.batch)
+            t0 = time.perf_counter()
+            assert orc.apply_incremental(ups, rows, pull=pull, op_weights=ow) == 0
+            spent += time.perf_counter() - t0
+            nb += 1
+        out[pull] = (args.batch * nb / spent, nb, spent)
     orc.close()
-    return {"value": args.batch * nb / spent, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
-            "sample": f"first {nb} batches of {args.batch} updates of the same stream "
-                      f"({spent:.1f} s; oracle set-up incl. its own bootstrap {setup:.0f} s, untimed)"}
+    return {"value": out[True][0], "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"incremental route, messages gathered per affected sink on all cores: first {out[True][1]} batches of "
+                      f"{args.batch} updates of the same stream ({out[True][2]:.1f} s); oracle set-up incl. its own "
+                      f"bootstrap {setup:.0f} s, untimed",
+            "single_thread_scatter": {"value": out[False][0], "unit": UNIT,
+                                      "sample": f"the next {out[False][1]} batches with the messages pushed along the "
+                                                f"senders' out-lists by one thread ({out[False][2]:.1f} s)"}}
 
 
 def run_ours(args, rank, world, local_rank):
@@ -506,7 +515,7 @@ def run_table(args):
                 while spent < args.oracle_seconds and done < nb:
                     ups, rows, ow = draw_batch(ostream, w, bsz)
                     t0 = time.perf_counter()
-                    assert orc.apply_incremental(ups, rows, op_weights=ow) == 0
+                    assert orc.apply_incremental(ups, rows, pull=True, op_weights=ow) == 0
                     spent += time.perf_counter() - t0
                     done += 1
                 line["oracle"] = {"updates_per_sec": bsz * done / spent, "batches": done, "cores": O.num_threads()}

@@ -21,9 +21,17 @@ def digest(*arrays) -> str:
     return h.hexdigest()[:32]
 
 
-def checksums():
+SMALL = ("tiny", "sparse", "mid-2l")          # regenerated and compared by the CPU tests
+LARGE = ("dense-2l", "reddit-2l")            # compared where the graphs are generated anyway: the full-size GPU tests
+
+
+def graph_digest(src, dst) -> str:
+    return digest(src, dst)
+
+
+def checksums(names=SMALL):
     out = {}
-    for name in ("tiny", "sparse"):
+    for name in names:
         w = I.workloads()[name]
         src, dst = I.make_graph(w)
         X = I.features(w.n, w.model.dims[0], w.seed)
@@ -33,7 +41,7 @@ def checksums():
         deg = np.bincount(src, minlength=w.n)
         out[name] = {
             "edges": int(src.size),
-            "graph": digest(src, dst),
+            "graph": graph_digest(src, dst),
             "max_out_degree": int(deg.max()),
             "zero_out_degree": int((deg == 0).sum()),
             "features": digest(X[:64]),
@@ -46,5 +54,5 @@ def checksums():
 if __name__ == "__main__":
     path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "generator_checksums.json")
     with open(path, "w") as f:
-        json.dump(checksums(), f, indent=1, sort_keys=True)
+        json.dump(checksums(SMALL + LARGE), f, indent=1, sort_keys=True)
     print("wrote", path)

@@ -61,6 +61,20 @@ def graph_of(wname):
     if key not in _graphs:
         _graphs.clear()          # one large graph on the host at a time
         _graphs[key] = I.make_graph(w)
+        # the generator still draws the graph whose checksum was recorded (tests/golden/generator_checksums.json)
+        import importlib.util
+        import json
+        import os
+        gold = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+        spec = importlib.util.spec_from_file_location("write_generator_checksums",
+                                                      os.path.join(gold, "write_generator_checksums.py"))
+        mod = importlib.util.module_from_spec(spec)
+        spec.loader.exec_module(mod)
+        want = json.load(open(os.path.join(gold, "generator_checksums.json")))
+        for name, rec in want.items():
+            wn = I.workloads()[name]
+            if (wn.graph, wn.n, wn.e, wn.seed) == key:
+                assert mod.graph_digest(*_graphs[key]) == rec["graph"], f"generator output of {name} changed"
     return w, _graphs[key]
 
 
