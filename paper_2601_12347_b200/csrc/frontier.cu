@@ -24,10 +24,14 @@ constexpr int SCAN_TILE = SCAN_T * SCAN_ITEMS;
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ int scan_count(const int* n_dev, int n_host) { return n_dev ? *n_dev : n_host; }
 
+// Tile sums; the last block to finish turns them into exclusive tile prefixes and writes the total
+// (one launch instead of two: the chain of a small batch is bound by the number of launches).
 __global__ void k_scan_tiles(const int32_t* __restrict__ list, const int* n_dev, int n_host,
-                             const int32_t* __restrict__ deg, int64_t* tile_sums) {
+                             const int32_t* __restrict__ deg, int64_t* tile_sums, int64_t* out,
+                             unsigned long long* total_dev, int* done) {
     pdl_enter();
     __shared__ int64_t scratch[33];
+    __shared__ int s_last;
     int n = scan_count(n_dev, n_host);
     int n_tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
@@ -42,14 +46,14 @@ __global__ void k_scan_tiles(const int32_t* __restrict__ list, const int* n_dev,
         if (threadIdx.x == 0) tile_sums[t] = total;
         __syncthreads();
     }
-}
-
-__global__ void k_scan_tile_sums(const int* n_dev, int n_host, int64_t* tile_sums, int64_t* out,
-                                 unsigned long long* total_dev) {
-    pdl_enter();
-    __shared__ int64_t scratch[33];
-    int n = scan_count(n_dev, n_host);
-    int n_tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(done, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) *done = 0;   // ready for the next scan
     int64_t carry = 0;
     for (int t0 = 0; t0 < n_tiles; t0 += blockDim.x) {
         int t = t0 + threadIdx.x;
@@ -98,8 +102,7 @@ void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, con
                   int64_t* out, unsigned long long* total_dev) {
     int max_tiles = std::max(1, div_up(c->N, SCAN_TILE));
     int grid = std::min(max_tiles, c->n_sm * 8);
-    RP_LAUNCH(c, k_scan_tiles, grid, SCAN_T, 0, list, n_dev, n_host, deg, c->tile_sums);
-    RP_LAUNCH(c, k_scan_tile_sums, 1, 1024, 0, n_dev, n_host, c->tile_sums, out, total_dev);
+    RP_LAUNCH(c, k_scan_tiles, grid, SCAN_T, 0, list, n_dev, n_host, deg, c->tile_sums, out, total_dev, c->scan_done);
     RP_LAUNCH(c, k_scan_write, grid, SCAN_T, 0, list, n_dev, n_host, deg, c->tile_sums, out);
 }
 

@@ -334,9 +334,8 @@ __device__ __forceinline__ long long take_block(const Side& sd, int k) {
 
 // Rows whose additions do not fit: list them and count the blocks they will take, by class.  Rows
 // that deletions leave nearly empty: list them for a move to a smaller block.
-__global__ void k_plan_growth(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
+__device__ __forceinline__ void d_plan_growth(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
                               int32_t* grow_out, int32_t* grow_in, int32_t* shrink_out, int32_t* shrink_in) {
-    pdl_enter();
     if (ctl->abort) return;
     int n = ctl->n_rec;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * n; i += gridDim.x * blockDim.x) {
@@ -360,8 +359,7 @@ __global__ void k_plan_growth(Ctl* ctl, const Rec* __restrict__ rec, Side out, S
 }
 
 // what the growing rows cannot take from the free lists must fit into the never-used tail
-__global__ void k_plan_check(Ctl* ctl, Side out, Side in) {
-    pdl_enter();
+__device__ __forceinline__ void d_plan_check(Ctl* ctl, Side out, Side in) {
     if (ctl->abort) return;
     for (int s = 0; s < 2; ++s) {
         const Side& sd = s ? in : out;
@@ -375,6 +373,25 @@ __global__ void k_plan_check(Ctl* ctl, Side out, Side in) {
             ctl->err = (int)RIPPLE_ERR_CAPACITY;
             ctl->abort = 1;
         }
+    }
+}
+
+// Plan: rows that must move, and whether the blocks they need exist.  One launch: the last block to
+// finish the listing does the check.
+__global__ void k_plan(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in, int32_t* grow_out, int32_t* grow_in,
+                       int32_t* shrink_out, int32_t* shrink_in) {
+    pdl_enter();
+    __shared__ int s_last;
+    d_plan_growth(ctl, rec, out, in, grow_out, grow_in, shrink_out, shrink_in);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(&ctl->plan_done, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (s_last && threadIdx.x == 0) {
+        __threadfence();
+        d_plan_check(ctl, out, in);
     }
 }
 
@@ -396,9 +413,8 @@ void graph_batch_classify(Ctx* c, int n) {
     RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, c->op_seq, c->ctl, c->hwin, c->op_slot, c->feat_last,
               c->vdel_seq, c->side[0], c->side[1], c->rec, c->bitmap,
               (const float*)(c->has_opw ? c->opw_dev : nullptr));
-    RP_LAUNCH(c, k_plan_growth, std::min(div_up(2 * n, T), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[0],
+    RP_LAUNCH(c, k_plan, std::min(div_up(2 * n, T), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[0],
               c->side[1], c->grow_list[0], c->grow_list[1], c->shrink_list[0], c->shrink_list[1]);
-    RP_LAUNCH(c, k_plan_check, 1, 1, 0, c->ctl, c->side[0], c->side[1]);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -408,8 +424,7 @@ void graph_batch_classify(Ctx* c, int n) {
     int n_ = (ctl)->n_rec;                                                                        \
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * n_; i += gridDim.x * blockDim.x)
 
-__global__ void k_del_mark(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
-    pdl_enter();
+__device__ __forceinline__ void d_del_mark(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -421,8 +436,7 @@ __global__ void k_del_mark(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side
     }
 }
 
-__global__ void k_del_tail_read(Ctl* ctl, Rec* rec, Side out, Side in) {
-    pdl_enter();
+__device__ __forceinline__ void d_del_tail_read(Ctl* ctl, Rec* rec, Side out, Side in) {
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -436,8 +450,7 @@ __global__ void k_del_tail_read(Ctl* ctl, Rec* rec, Side out, Side in) {
     }
 }
 
-__global__ void k_del_tail_pack(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
-    pdl_enter();
+__device__ __forceinline__ void d_del_tail_pack(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -452,8 +465,7 @@ __global__ void k_del_tail_pack(Ctl* ctl, const Rec* __restrict__ rec, Side out,
     }
 }
 
-__global__ void k_del_fill(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
-    pdl_enter();
+__device__ __forceinline__ void d_del_fill(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -485,11 +497,9 @@ __device__ __forceinline__ void move_row(Side& sd, int row, long long off, int n
         for (int j = tid; j < live; j += nthreads) sd.w[off + j] = sd.w[old + j];
 }
 
-__global__ void __launch_bounds__(256)
-k_grow_rows(Ctl* ctl, Side out, Side in, const int32_t* __restrict__ grow_out, const int32_t* __restrict__ grow_in,
+__device__ __forceinline__ void d_grow_rows(Ctl* ctl, Side out, Side in, const int32_t* __restrict__ grow_out, const int32_t* __restrict__ grow_in,
             const int32_t* __restrict__ shrink_out, const int32_t* __restrict__ shrink_in, int64_t* moved_start,
             int32_t* moved_cap) {
-    pdl_enter();
     if (ctl->abort) return;
     __shared__ long long s_off;
     __shared__ int s_last;
@@ -557,8 +567,7 @@ k_grow_rows(Ctl* ctl, Side out, Side in, const int32_t* __restrict__ grow_out, c
     }
 }
 
-__global__ void k_add_write(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
-    pdl_enter();
+__device__ __forceinline__ void d_add_write(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) {
     if (ctl->abort) return;
     FOR_EACH_REC_SIDE(ctl, i, s, x, sd, row) {
         int s = i & 1;
@@ -572,10 +581,9 @@ __global__ void k_add_write(Ctl* ctl, const Rec* __restrict__ rec, Side out, Sid
     }
 }
 
-__global__ void k_commit_degrees(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
+__device__ __forceinline__ void d_commit_degrees(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
                                  int32_t* deg_out_old, const int64_t* __restrict__ moved_start,
                                  const int32_t* __restrict__ moved_cap) {
-    pdl_enter();
     if (ctl->abort) return;
     // the blocks that moved rows left behind go onto the free lists
     const int n0 = ctl->n_grow[0], n1 = ctl->n_grow[1], m0 = ctl->n_shrink[0], m1 = ctl->n_shrink[1];
@@ -607,12 +615,59 @@ __global__ void k_commit_degrees(Ctl* ctl, const Rec* __restrict__ rec, Side out
     }
 }
 
+// The kernels of the row update, one launch each ...
+__global__ void k_del_mark(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) { pdl_enter(); d_del_mark(ctl, rec, out, in); }
+__global__ void k_del_tail_read(Ctl* ctl, Rec* rec, Side out, Side in) { pdl_enter(); d_del_tail_read(ctl, rec, out, in); }
+__global__ void k_del_tail_pack(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) { pdl_enter(); d_del_tail_pack(ctl, rec, out, in); }
+__global__ void k_del_fill(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) { pdl_enter(); d_del_fill(ctl, rec, out, in); }
+__global__ void __launch_bounds__(256)
+k_grow_rows(Ctl* ctl, Side out, Side in, const int32_t* __restrict__ grow_out, const int32_t* __restrict__ grow_in,
+            const int32_t* __restrict__ shrink_out, const int32_t* __restrict__ shrink_in, int64_t* moved_start,
+            int32_t* moved_cap) {
+    pdl_enter();
+    d_grow_rows(ctl, out, in, grow_out, grow_in, shrink_out, shrink_in, moved_start, moved_cap);
+}
+__global__ void k_add_write(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in) { pdl_enter(); d_add_write(ctl, rec, out, in); }
+__global__ void k_commit_degrees(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in, int32_t* deg_out_old,
+                                 const int64_t* __restrict__ moved_start, const int32_t* __restrict__ moved_cap) {
+    pdl_enter();
+    d_commit_degrees(ctl, rec, out, in, deg_out_old, moved_start, moved_cap);
+}
+
+// ... and all of them in one block, a barrier between the phases, for the batches that are replayed
+// from a captured chain (up to RP_GRAPH_MAX_BATCH operations: a few hundred records at most, which one
+// block handles in a single sweep per phase).  Small batches are bound by the number of launches.
+__global__ void __launch_bounds__(1024)
+k_mutate_small(Ctl* ctl, Rec* rec, Side out, Side in, const int32_t* __restrict__ grow_out,
+               const int32_t* __restrict__ grow_in, const int32_t* __restrict__ shrink_out,
+               const int32_t* __restrict__ shrink_in, int64_t* moved_start, int32_t* moved_cap, int32_t* deg_out_old) {
+    pdl_enter();
+    d_del_mark(ctl, rec, out, in);
+    __syncthreads();
+    d_del_tail_read(ctl, rec, out, in);
+    __syncthreads();
+    d_del_tail_pack(ctl, rec, out, in);
+    __syncthreads();
+    d_del_fill(ctl, rec, out, in);
+    __syncthreads();
+    d_grow_rows(ctl, out, in, grow_out, grow_in, shrink_out, shrink_in, moved_start, moved_cap);
+    __syncthreads();
+    d_add_write(ctl, rec, out, in);
+    __syncthreads();
+    d_commit_degrees(ctl, rec, out, in, deg_out_old, moved_start, moved_cap);
+}
+
 void graph_batch_mutate(Ctx* c, int n) {
     if (n <= 0) return;
     const int T = 256;
     int grid = std::min(div_up(2 * n, T), c->n_sm * 8);
     Side& o = c->side[0];
     Side& i = c->side[1];
+    if (n <= RP_GRAPH_MAX_BATCH) {
+        RP_LAUNCH(c, k_mutate_small, 1, 1024, 0, c->ctl, c->rec, o, i, c->grow_list[0], c->grow_list[1],
+                  c->shrink_list[0], c->shrink_list[1], c->moved_start, c->moved_cap, c->deg_out_old);
+        return;
+    }
     RP_LAUNCH(c, k_del_mark, grid, T, 0, c->ctl, c->rec, o, i);
     RP_LAUNCH(c, k_del_tail_read, grid, T, 0, c->ctl, c->rec, o, i);
     RP_LAUNCH(c, k_del_tail_pack, grid, T, 0, c->ctl, c->rec, o, i);

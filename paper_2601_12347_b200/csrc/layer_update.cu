@@ -12,7 +12,11 @@
 
 namespace rp {
 
-constexpr int BM = 64, BN = 64, BK = 16, TM = 4, TN = 4;
+// K is walked in chunks of 64: every thread has eight independent 16-byte loads in flight per chunk
+// (four pieces of a gathered A row, four of the weights).  With chunks of 16 a small frontier -- a
+// handful of tiles, so nothing to overlap with -- paid one trip to L2 per 16 columns of K: 20 to 27 us
+// for a few dozen rows, half of the latency of a batch of one update.
+constexpr int BM = 64, BN = 64, BK = 64, TM = 4, TN = 4;
 
 __global__ void __launch_bounds__(256)
 k_update_rows(const Ctl* ctl, UpdParams p) {
@@ -47,23 +51,31 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
 #pragma unroll
             for (int b = 0; b < TN; ++b) acc[a][b] = 0.f;
 
-        const int ar = tid >> 2, ak = (tid & 3) * 4;   // A tile: row ar, k offset ak..ak+3
-        const int bk = tid >> 4, bn = (tid & 15) * 4;  // B tile: k row bk, cols bn..bn+3
+        const int ar = tid >> 2, ak = (tid & 3) * 4;   // A tile: row ar, k offsets ak + 16 j .. + 3, j = 0..3
+        const int bk = tid >> 4, bn = (tid & 15) * 4;  // B tile: k rows bk + 16 j, cols bn..bn+3
         for (int k0 = 0; k0 < p.K; k0 += BK) {
-            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-            {
-                const int v = row_id[ar], k = k0 + ak;
-                if (v >= 0 && k < p.K) a = upd_load_a(p, v, r0 + ar, k, row_scale[ar]);
+            float4 a[4], b[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                a[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                const int v = row_id[ar], k = k0 + ak + 16 * j;
+                if (v >= 0 && k < p.K) a[j] = upd_load_a(p, v, r0 + ar, k, row_scale[ar]);
+                b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                const int kb = k0 + bk + 16 * j;
+                if (kb < p.K && c0 + bn < p.n_cols)
+                    b[j] = __ldg(reinterpret_cast<const float4*>(p.W + (size_t)kb * p.ldw + c0 + bn));
             }
-            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (k0 + bk < p.K && c0 + bn < p.n_cols)
-                b = __ldg(reinterpret_cast<const float4*>(p.W + (size_t)(k0 + bk) * p.ldw + c0 + bn));
-            __syncthreads();
-            As[ak + 0][ar] = a.x; As[ak + 1][ar] = a.y; As[ak + 2][ar] = a.z; As[ak + 3][ar] = a.w;
-            *reinterpret_cast<float4*>(&Bs[bk][bn]) = b;
             __syncthreads();
 #pragma unroll
-            for (int k = 0; k < BK; ++k) {
+            for (int j = 0; j < 4; ++j) {
+                As[ak + 16 * j + 0][ar] = a[j].x; As[ak + 16 * j + 1][ar] = a[j].y;
+                As[ak + 16 * j + 2][ar] = a[j].z; As[ak + 16 * j + 3][ar] = a[j].w;
+                *reinterpret_cast<float4*>(&Bs[bk + 16 * j][bn]) = b[j];
+            }
+            __syncthreads();
+            const int kmax = min(BK, p.K - k0);
+#pragma unroll 16
+            for (int k = 0; k < kmax; ++k) {
                 float4 av = *reinterpret_cast<const float4*>(&As[k][ty * TM]);
                 float4 bv = *reinterpret_cast<const float4*>(&Bs[k][tx * TN]);
                 const float ar4[4] = {av.x, av.y, av.z, av.w};
@@ -108,7 +120,9 @@ static void launch_update(Ctx* c, UpdParams& p, const TcW& tw) {
     p.tc_mode = TC_OFF;
     // measured on the dense graph: the tensor-core form wins for wide outputs (256 columns: 5.5 ms
     // against 9.8 ms SIMT) and loses for narrow ones, where staging latency dominates
-    if (tw.hi && c->gemm_mode != RIPPLE_GEMM_FP32 && p.K > 0 && tw.n_pad >= 128) {
+    // The tensor-core twin is only put into the chain when the last batch's frontiers (or a whole-graph pass)
+    // were large enough for it; without it the SIMT form takes whatever comes.
+    if (tw.hi && c->gemm_mode != RIPPLE_GEMM_FP32 && p.K > 0 && tw.n_pad >= 128 && (c->tc_armed || !p.list)) {
         p.tc_mode = c->gemm_mode == RIPPLE_GEMM_TF32 ? TC_TF32 : TC_TF32X3;
         p.tc_min_rows = 1024;
         p.tc_withhold = c->debug_tc_withhold;

@@ -74,9 +74,9 @@ static void destroy_ctx(Ctx* c) {
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
         for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2, &c->layer[l].tc_self}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
-    cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->M); cudaFree(c->Mt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->invmask); cudaFree(c->posmap); cudaFree(c->deg_out_old);
+    cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->invmask); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->opw_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
-    cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->ctl);
+    cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->scan_done); cudaFree(c->ctl);
     cudaFree(c->moved_start); cudaFree(c->moved_cap);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
     if (c->params_host) cudaFreeHost(c->params_host);
@@ -202,6 +202,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         c->n_words = (N + 31) / 32;
         c->n_tile_sums = std::max(div_up(N, 1024) + 2, div_up(c->n_words, 256) + 2);
         CK(dev_alloc(&c->tile_sums, (size_t)c->n_tile_sums, 0));
+        CK(dev_alloc(&c->scan_done, 1, 0));
         for (auto& e : c->ev) CK(cudaEventCreate(&e));
         for (auto& e : c->ev_sc) CK(cudaEventCreate(&e));
         for (auto& e : c->ev_rg) CK(cudaEventCreate(&e));
@@ -320,8 +321,6 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                         feat_mem == RIPPLE_MEM_DEVICE ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice));
         if (max_hid) CK(dev_alloc(&c->T, (size_t)N * max_hid));
         CK(dev_alloc(&c->Dt, (size_t)N * max_ld));
-        CK(dev_alloc(&c->M, (size_t)o.max_batch * max_ld));
-        CK(dev_alloc(&c->Mt, (size_t)o.max_batch * max_ld));
         for (int s = 0; s < 2; ++s) {
             CK(dev_alloc(&c->D[s], (size_t)N * max_ld));
             CK(dev_alloc(&c->Clist[s], (size_t)N + 32));
@@ -417,7 +416,7 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
         STAMP();
         scatter_layer(c, l, nb);
         if (!pull) frontier_compact(c, l);
-        senders_release(c, l - 1);
+        if (nb <= 0) senders_release(c, l - 1);   // (otherwise the last kernel of the hop's delta form clears them)
         fold_deltas(c, l);
         regather_layer(c, l);
         STAMP();
@@ -439,6 +438,9 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
 // if it turns out saturated: slower for that one batch, never wrong, and armed for the next.
 static void arm_rebuild(Ctx* c, int nb) {
     const bool no_history = c->batches_done == 0 || nb > 4 * std::max(c->last_nb, 1);
+    // the tensor-core update takes over from 1024 rows: in the chain if any frontier of the last batch came near
+    c->tc_armed = no_history;
+    for (int l = 0; l <= c->L; ++l) c->tc_armed |= c->stats.affected[l] >= 256 || c->stats.senders[l] >= 256;
     for (int l = 1; l <= c->L; ++l) {
         bool armed = false;
         if (rp_monotonic(c->agg)) armed = false;
@@ -457,6 +459,7 @@ static bool launch_batch_graph(Ctx* c, int nb) {
     if (c->no_graphs || c->timing || nb < 1 || nb > RP_GRAPH_MAX_BATCH) return false;
     // the captured chain differs with the expansion kernels and with the hops whose rebuilding form is enqueued
     int key = 4 * nb + (c->may_expand ? 1 : 0) + (c->has_opw ? 2 : 0);
+    key = 2 * key + (c->tc_armed ? 1 : 0);
     for (int l = 1; l <= c->L; ++l) key = 2 * key + (c->rebuild_armed[l] ? 1 : 0);
     int slot = -1;
     for (int i = 0; i < RP_GRAPH_SLOTS; ++i)

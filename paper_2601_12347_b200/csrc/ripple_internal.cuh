@@ -40,6 +40,7 @@ struct Ctl {
     int n_shrink[2];                  // rows left with less than a quarter of their capacity in use: moved to a smaller block
     int grow_demand[2][RP_POOL_CLASSES];   // growing rows per block size class
     int grow_done;                    // blocks of k_grow_rows that have finished (the last one moves the shrinking rows)
+    int plan_done;                    // blocks of k_plan that have listed their rows (the last one checks the pool)
     unsigned long long pool_need[2];
     // kept across batches:
     unsigned long long pool_next[2];  // next entry of each side's adjacency array that was never handed out
@@ -128,6 +129,7 @@ struct Ctx {
     int64_t max_batch;
     int scatter_mode, gemm_mode, timing;
     int rebuild_armed[RP_MAXL + 1];   // per hop: the rebuilding form is enqueued for this batch (see arm_rebuild)
+    int tc_armed;                     // the tensor-core form of the layer update is enqueued for this batch
     long long batches_done;
     int last_nb;
     int debug_tc_withhold;   // diagnostic (environment RIPPLE_DEBUG_TC_WITHHOLD=1): see ripple_create
@@ -154,8 +156,6 @@ struct Ctx {
     float* T;          // GIN hidden rows (compact, N x ld_hid)
     float* D[2];       // delta rows, ping-pong (compact, N x max ld)
     float* Dt;         // delta rows after the neighbour transform (compact, N x max inbox width)
-    float* M;          // edge-record rows (compact, max_batch x max ld) and their transform
-    float* Mt;
     bool pre[RP_MAXL + 1];   // layer applies its neighbour transform before the scatter
     int ws[RP_MAXL + 1];     // row width (floats, padded) of S^l and of hop-l messages
     int32_t* A[RP_MAXL + 1];   // affected lists
@@ -184,6 +184,7 @@ struct Ctx {
     // scan scratch
     int64_t* tile_sums;
     int n_tile_sums;
+    int* scan_done;    // blocks of a scan's first kernel that have finished (zero between scans)
     int* params_dev;   // {n_ops, n_rows} of the batch being applied
     int* params_host;  // pinned
     int no_graphs;

@@ -439,11 +439,12 @@ k_scatter_pull(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const in
 // ---------------------------------------------------------------------------------------------
 // edge-change records
 // ---------------------------------------------------------------------------------------------
-// M_u = c_old h_old = c_new h_new - D_u for a sender, c h otherwise; one warp per record, compact
-// rows in record order (row width = that of the previous layer's embeddings).
-__global__ void k_record_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, int src_norm,
-                              const int32_t* __restrict__ deg_out, const int32_t* __restrict__ posmap,
-                              const float* __restrict__ Hprev, const float* __restrict__ D, int ld, float* M) {
+// Messages of the net edge changes: S_v += sign * w * M_r with M_r = c_old m_old of the record's
+// source (= c_new m_new - D_u if the source is a sender of this hop, c m otherwise) and w the edge's
+// stored weight (1 without stored weights).  One warp per record; rows have the inbox width.
+__global__ void k_scatter_records(Ctl* ctl, int l, const Rec* __restrict__ rec, int src_norm,
+                                  const int32_t* __restrict__ deg_out, const int32_t* __restrict__ posmap,
+                                  const float* __restrict__ Mrows, const float* __restrict__ D, int ld, float* S) {
     pdl_enter();
     if (ctl->abort || ctl->regather[l]) return;
     const int n = ctl->n_rec;
@@ -452,9 +453,10 @@ __global__ void k_record_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, int 
     for (int r = warp; r < n; r += nwarps) {
         const int u = rec[r].u;
         const int p = posmap[u];
-        const float4* hrow = reinterpret_cast<const float4*>(Hprev + (size_t)u * ld);
+        const float4* hrow = reinterpret_cast<const float4*>(Mrows + (size_t)u * ld);
         const float cn = src_norm ? coef_from_degree(deg_out[u]) : 1.0f;
-        float4* dst = reinterpret_cast<float4*>(M + (size_t)r * ld);
+        const float sgn = (float)rec[r].sign * rec[r].w;
+        float* dst = S + (size_t)rec[r].v * ld;
         for (int q = lane; q < nq; q += 32) {
             float4 h = __ldg(hrow + q);
             float4 m = make_float4(cn * h.x, cn * h.y, cn * h.z, cn * h.w);
@@ -462,25 +464,6 @@ __global__ void k_record_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, int 
                 float4 d = __ldg(reinterpret_cast<const float4*>(D + (size_t)p * ld) + q);
                 m.x -= d.x; m.y -= d.y; m.z -= d.z; m.w -= d.w;
             }
-            dst[q] = m;
-        }
-    }
-}
-
-// S_v += sign * M_r for every record r (row width = inbox width)
-__global__ void k_scatter_records(Ctl* ctl, int l, const Rec* __restrict__ rec, const float* __restrict__ M,
-                                  int ld, float* S) {
-    pdl_enter();
-    if (ctl->abort || ctl->regather[l]) return;
-    const int n = ctl->n_rec;
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
-    const int lane = lane_id(), nq = ld >> 2;
-    for (int r = warp; r < n; r += nwarps) {
-        const float sgn = (float)rec[r].sign * rec[r].w;   // (w = 1 unless edges carry stored weights)
-        float* dst = S + (size_t)rec[r].v * ld;
-        const float4* mrow = reinterpret_cast<const float4*>(M + (size_t)r * ld);
-        for (int q = lane; q < nq; q += 32) {
-            float4 m = __ldg(mrow + q);
             red_add_v4(dst + 4 * q, make_float4(sgn * m.x, sgn * m.y, sgn * m.z, sgn * m.w));
         }
     }
@@ -537,8 +520,14 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int32_t* __restrict__ deg_out,
                 int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, float* __restrict__ dS,
-                float* budget) {
+                float* budget, const int32_t* __restrict__ senders, int32_t* posmap) {
     pdl_enter();
+    // the hop's senders are no longer looked up by anyone: their entries of the position map are cleared
+    // here (the last kernel of the hop's delta form), whatever form the hop takes
+    {
+        const int nC = ctl->nC[l - 1];
+        for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nC; i += gridDim.x * blockDim.x) posmap[senders[i]] = -1;
+    }
     if (ctl->abort || ctl->regather[l]) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -687,7 +676,6 @@ void choose_direction(Ctx* c, int l) {
 
 // delta form of hop l (does nothing on the device if the hop rebuilds)
 void scatter_layer(Ctx* c, int l, int n) {
-    const int ld_prev = c->ld[l - 1];
     const int ld = c->ws[l];
     const float* D = c->D[(l - 1) & 1];
     const int32_t* senders = c->Clist[(l - 1) & 1];
@@ -697,17 +685,11 @@ void scatter_layer(Ctx* c, int l, int n) {
     // layer that transforms first keeps m = P^l rows up to date for the senders, whatever form the
     // hop takes, and builds its records from them directly.
     const float* Dm = D;
-    const float* Mm = c->M;
+    const float* Mrows = c->H[l - 1];
     if (c->pre[l]) {
         sender_transform(c, l);
         Dm = c->Dt;
-        Mm = c->Mt;
-        if (n > 0)
-            RP_LAUNCH(c, k_record_rows, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec,
-                      (int)c->src_norm, c->side[0].deg, c->posmap, c->P[l], c->Dt, ld, c->Mt);
-    } else if (n > 0) {
-        RP_LAUNCH(c, k_record_rows, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec,
-                  (int)c->src_norm, c->side[0].deg, c->posmap, c->H[l - 1], D, ld_prev, c->M);
+        Mrows = c->P[l];
     }
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
 #define PUSH(NV, LPR) RP_LAUNCH(c, (k_scatter_push<NV, LPR>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, ld, c->dS[l], c->bitmap)
@@ -730,10 +712,10 @@ void scatter_layer(Ctx* c, int l, int n) {
 #undef PULL
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
     if (n > 0) {
-        RP_LAUNCH(c, k_scatter_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, Mm, ld,
-                  c->dS[l]);
+        RP_LAUNCH(c, k_scatter_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec,
+                  (int)c->src_norm, c->side[0].deg, c->posmap, Mrows, Dm, ld, c->dS[l]);
         const float* rows = c->pre[l] ? c->P[l] : c->H[l - 1];
-#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l], c->Eb[l])
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l], c->Eb[l], senders, c->posmap)
         RP_WIDTH_DISPATCH(ld, ROWS);
 #undef ROWS
     }
