@@ -26,20 +26,29 @@ __device__ __forceinline__ int scan_count(const int* n_dev, int n_host) { return
 
 // Tile sums; the last block to finish turns them into exclusive tile prefixes and writes the total
 // (one launch instead of two: the chain of a small batch is bound by the number of launches).
+// If `senders` is given the listed vertices are, in the same pass, copied there and entered into the
+// position map, and their number into *n_senders: the sender list of a hop whose senders are exactly
+// the affected vertices (no launch of its own for that).
 __global__ void k_scan_tiles(const int32_t* __restrict__ list, const int* n_dev, int n_host,
                              const int32_t* __restrict__ deg, int64_t* tile_sums, int64_t* out,
-                             unsigned long long* total_dev, int* done) {
+                             unsigned long long* total_dev, int* done, int32_t* senders, int32_t* posmap,
+                             int* n_senders) {
     pdl_enter();
     __shared__ int64_t scratch[33];
     __shared__ int s_last;
     int n = scan_count(n_dev, n_host);
     int n_tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
+    if (senders && blockIdx.x == 0 && threadIdx.x == 0) *n_senders = n;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
         int64_t s = 0;
 #pragma unroll
         for (int k = 0; k < SCAN_ITEMS; ++k) {
             int i = t * SCAN_TILE + k * SCAN_T + threadIdx.x;
-            if (i < n) s += deg[list ? list[i] : i];
+            if (i < n) {
+                const int v = list ? list[i] : i;
+                s += deg[v];
+                if (senders) { senders[i] = v; posmap[v] = i; }
+            }
         }
         int64_t total;
         block_exclusive_scan<int64_t>(s, scratch, total);
@@ -98,12 +107,18 @@ __global__ void k_scan_write(const int32_t* __restrict__ list, const int* n_dev,
     }
 }
 
-void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, const int32_t* deg,
-                  int64_t* out, unsigned long long* total_dev) {
+static void scan_degrees_and_copy(Ctx* c, const int32_t* list, const int* n_dev, int n_host, const int32_t* deg,
+                                  int64_t* out, unsigned long long* total_dev, int32_t* senders, int* n_senders) {
     int max_tiles = std::max(1, div_up(c->N, SCAN_TILE));
     int grid = std::min(max_tiles, c->n_sm * 8);
-    RP_LAUNCH(c, k_scan_tiles, grid, SCAN_T, 0, list, n_dev, n_host, deg, c->tile_sums, out, total_dev, c->scan_done);
+    RP_LAUNCH(c, k_scan_tiles, grid, SCAN_T, 0, list, n_dev, n_host, deg, c->tile_sums, out, total_dev, c->scan_done,
+              senders, c->posmap, n_senders);
     RP_LAUNCH(c, k_scan_write, grid, SCAN_T, 0, list, n_dev, n_host, deg, c->tile_sums, out);
+}
+
+void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, const int32_t* deg,
+                  int64_t* out, unsigned long long* total_dev) {
+    scan_degrees_and_copy(c, list, n_dev, n_host, deg, out, total_dev, nullptr, nullptr);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -273,9 +288,13 @@ void frontier_seed_features(Ctx* c, int n) {
 
 // Marks the members of A_l that do not come from walking the senders' out-lists (sinks of edge
 // changes, A_{l-1} for models with a self term) and, if `walk`, those that do.
-void frontier_mark(Ctx* c, int l, bool walk) {
-    RP_LAUNCH(c, k_mark_frontier, walk ? c->n_sm * 8 : c->n_sm * 2, 256, 0, c->ctl, l, (int)c->self_term,
-              (int)walk, c->Clist[(l - 1) & 1], c->coff, c->side[0], c->rec, c->A[l - 1], c->bitmap);
+void frontier_mark(Ctx* c, int l, bool walk, int n) {
+    // without a walk of its own (the push scatter marks the sinks it reaches) the rest of the marking rides
+    // along with the last kernel of the hop's delta form; an empty batch has nothing to mark
+    if (walk)
+        RP_LAUNCH(c, k_mark_frontier, c->n_sm * 8, 256, 0, c->ctl, l, (int)c->self_term,
+                  (int)walk, c->Clist[(l - 1) & 1], c->coff, c->side[0], c->rec, c->A[l - 1], c->bitmap);
+    (void)n;
     if (!c->rebuild_armed[l]) return;
     // the list A_l is not built yet: its buffer holds the queue of undecided long rows
     RP_LAUNCH(c, k_mark_bottom_up, c->n_sm * 8, 256, 0, c->ctl, l, c->N, c->side[1], c->posmap, c->bitmap, c->A[l],
@@ -313,8 +332,15 @@ __global__ void k_senders_release(Ctl* ctl, int l, const int32_t* __restrict__ s
 
 void senders_build(Ctx* c, int l, int n) {
     int32_t* senders = c->Clist[l & 1];
+    if (!c->src_norm) {
+        // the senders are exactly the affected vertices: listed while their out-degrees are summed
+        // (after a rejected batch every list is empty, so nothing needs the abort flag here)
+        scan_degrees_and_copy(c, c->A[l], &c->ctl->nA[l], 0, c->side[0].deg, c->coff, &c->ctl->E[l + 1], senders,
+                              &c->ctl->nC[l]);
+        return;
+    }
     RP_LAUNCH(c, k_senders_from_affected, c->n_sm * 4, 256, 0, c->ctl, l, c->A[l], senders, c->posmap);
-    if (c->src_norm && n > 0) extra_sender_rows(c, l, n);
+    if (n > 0) extra_sender_rows(c, l, n);
     scan_degrees(c, senders, &c->ctl->nC[l], 0, c->side[0].deg, c->coff, &c->ctl->E[l + 1]);
 }
 

@@ -240,7 +240,14 @@ __device__ __forceinline__ int block_find(const int32_t* __restrict__ col, int64
     return *s_found;
 }
 
+__device__ __forceinline__ void d_plan_growth(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
+                                              int32_t* grow_out, int32_t* grow_in, int32_t* shrink_out,
+                                              int32_t* shrink_in, int tid, int nthreads);
+__device__ __forceinline__ void d_plan_check(Ctl* ctl, Side out, Side in);
+
 // One block per op: winners are compared with the stored graph and become records or no-ops.
+// The last block to finish then plans the row moves (which rows need a new block, and whether the
+// blocks exist): no launch of its own for that.
 // An explicit edge operation that precedes the deletion of one of its endpoints is superseded by
 // it (for stored edges the generated deletion already wins the slot; for pairs that are not stored
 // nothing was generated, hence the explicit test).  Only the caller's operations are counted.
@@ -248,9 +255,11 @@ __global__ void __launch_bounds__(256)
 k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, Ctl* ctl,
           const unsigned long long* __restrict__ hwin, const int32_t* __restrict__ op_slot,
           const int32_t* __restrict__ feat_last, const int32_t* __restrict__ vdel_seq, Side out, Side in,
-          Rec* rec, uint32_t* bitmap, const float* __restrict__ op_w) {
+          Rec* rec, uint32_t* bitmap, const float* __restrict__ op_w, int32_t* grow_out, int32_t* grow_in,
+          int32_t* shrink_out, int32_t* shrink_in) {
     pdl_enter();
     __shared__ int s_found;
+    __shared__ int s_last;
     if (ctl->abort) return;
     const int n = ops_total(ctl), n_given = ctl->n_ops;
     for (int i = blockIdx.x; i < n; i += gridDim.x) {
@@ -293,6 +302,18 @@ k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_
             rec[r] = x;
         }
     }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(&ctl->plan_done, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    d_plan_growth(ctl, rec, out, in, grow_out, grow_in, shrink_out, shrink_in, threadIdx.x, blockDim.x);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) d_plan_check(ctl, out, in);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -335,10 +356,11 @@ __device__ __forceinline__ long long take_block(const Side& sd, int k) {
 // Rows whose additions do not fit: list them and count the blocks they will take, by class.  Rows
 // that deletions leave nearly empty: list them for a move to a smaller block.
 __device__ __forceinline__ void d_plan_growth(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in,
-                              int32_t* grow_out, int32_t* grow_in, int32_t* shrink_out, int32_t* shrink_in) {
+                              int32_t* grow_out, int32_t* grow_in, int32_t* shrink_out, int32_t* shrink_in,
+                              int tid, int nthreads) {
     if (ctl->abort) return;
     int n = ctl->n_rec;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < 2 * n; i += gridDim.x * blockDim.x) {
+    for (int i = tid; i < 2 * n; i += nthreads) {
         int s = i & 1;
         const Rec& x = rec[i >> 1];
         if (x.rank[s] != 0) continue;   // one record per row and kind of change
@@ -376,25 +398,6 @@ __device__ __forceinline__ void d_plan_check(Ctl* ctl, Side out, Side in) {
     }
 }
 
-// Plan: rows that must move, and whether the blocks they need exist.  One launch: the last block to
-// finish the listing does the check.
-__global__ void k_plan(Ctl* ctl, const Rec* __restrict__ rec, Side out, Side in, int32_t* grow_out, int32_t* grow_in,
-                       int32_t* shrink_out, int32_t* shrink_in) {
-    pdl_enter();
-    __shared__ int s_last;
-    d_plan_growth(ctl, rec, out, in, grow_out, grow_in, shrink_out, shrink_in);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        s_last = atomicAdd(&ctl->plan_done, 1) == (int)gridDim.x - 1;
-    }
-    __syncthreads();
-    if (s_last && threadIdx.x == 0) {
-        __threadfence();
-        d_plan_check(ctl, out, in);
-    }
-}
-
 // n sizes the launches (the number of operations given, or the batch capacity if vertex deletions
 // may multiply them); the kernels read the actual counts from the control block
 void graph_batch_classify(Ctx* c, int n) {
@@ -412,9 +415,8 @@ void graph_batch_classify(Ctx* c, int n) {
     int grid = std::min(n, c->n_sm * 8);
     RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, c->op_seq, c->ctl, c->hwin, c->op_slot, c->feat_last,
               c->vdel_seq, c->side[0], c->side[1], c->rec, c->bitmap,
-              (const float*)(c->has_opw ? c->opw_dev : nullptr));
-    RP_LAUNCH(c, k_plan, std::min(div_up(2 * n, T), c->n_sm * 8), T, 0, c->ctl, c->rec, c->side[0],
-              c->side[1], c->grow_list[0], c->grow_list[1], c->shrink_list[0], c->shrink_list[1]);
+              (const float*)(c->has_opw ? c->opw_dev : nullptr), c->grow_list[0], c->grow_list[1],
+              c->shrink_list[0], c->shrink_list[1]);
 }
 
 // ---------------------------------------------------------------------------------------------

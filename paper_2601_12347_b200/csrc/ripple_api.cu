@@ -411,7 +411,7 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
         // (decided per hop on the device for the rebuilding form).
         const bool pull = c->scatter_mode == RIPPLE_SCATTER_PULL;
         choose_direction(c, l);
-        frontier_mark(c, l, pull);
+        frontier_mark(c, l, pull, nb);
         if (pull) frontier_compact(c, l);
         STAMP();
         scatter_layer(c, l, nb);

@@ -40,7 +40,7 @@ struct Ctl {
     int n_shrink[2];                  // rows left with less than a quarter of their capacity in use: moved to a smaller block
     int grow_demand[2][RP_POOL_CLASSES];   // growing rows per block size class
     int grow_done;                    // blocks of k_grow_rows that have finished (the last one moves the shrinking rows)
-    int plan_done;                    // blocks of k_plan that have listed their rows (the last one checks the pool)
+    int plan_done;                    // blocks of k_resolve that have finished (the last one plans the row moves)
     unsigned long long pool_need[2];
     // kept across batches:
     unsigned long long pool_next[2];  // next entry of each side's adjacency array that was never handed out
@@ -251,7 +251,7 @@ cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, float* weight, i
 void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, const int32_t* deg,
                   int64_t* out, unsigned long long* total_dev);
 void frontier_seed_features(Ctx* c, int n);             // A_0 from the batch's feature updates
-void frontier_mark(Ctx* c, int l, bool walk);           // bitmap of A_l: edge-record sinks, A_{l-1}, and (walk) Out(C_{l-1})
+void frontier_mark(Ctx* c, int l, bool walk, int n);    // bitmap of A_l: (walk) edge-record sinks, A_{l-1} and Out(C_{l-1}); rebuilding hops: bottom-up
 void frontier_compact(Ctx* c, int l);                   // bitmap -> ascending list A_l
 void senders_build(Ctx* c, int l, int n);               // C_l, posmap, coff, E_{l+1}
 void senders_release(Ctx* c, int l);                    // clear posmap entries of C_l

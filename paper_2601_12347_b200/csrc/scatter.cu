@@ -520,13 +520,28 @@ template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int32_t* __restrict__ deg_out,
                 int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, float* __restrict__ dS,
-                float* budget, const int32_t* __restrict__ senders, int32_t* posmap) {
+                float* budget, const int32_t* __restrict__ senders, int32_t* posmap, int mark, int self_term,
+                const int32_t* __restrict__ A_prev, uint32_t* bitmap) {
     pdl_enter();
-    // the hop's senders are no longer looked up by anyone: their entries of the position map are cleared
-    // here (the last kernel of the hop's delta form), whatever form the hop takes
+    // Two chores of the hop ride along with this kernel, the last of the hop's delta form, whatever form
+    // the hop takes.  The hop's senders are no longer looked up by anyone: their entries of the position
+    // map are cleared.  And (mark) the members of A_l that no out-list walk finds are marked: the sinks of
+    // net edge changes, and A_{l-1} for models with a self term.
     {
+        const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gsize = gridDim.x * blockDim.x;
         const int nC = ctl->nC[l - 1];
-        for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nC; i += gridDim.x * blockDim.x) posmap[senders[i]] = -1;
+        for (int i = gtid; i < nC; i += gsize) posmap[senders[i]] = -1;
+        if (mark && !ctl->abort) {
+            for (int i = gtid; i < ctl->n_rec; i += gsize) {
+                const int v = rec[i].v;
+                atomicOr(&bitmap[v >> 5], 1u << (v & 31));
+            }
+            if (self_term)
+                for (int i = gtid; i < ctl->nA[l - 1]; i += gsize) {
+                    const int v = A_prev[i];
+                    atomicOr(&bitmap[v >> 5], 1u << (v & 31));
+                }
+        }
     }
     if (ctl->abort || ctl->regather[l]) return;
     const int n = ctl->n_rec;
@@ -715,7 +730,7 @@ void scatter_layer(Ctx* c, int l, int n) {
         RP_LAUNCH(c, k_scatter_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec,
                   (int)c->src_norm, c->side[0].deg, c->posmap, Mrows, Dm, ld, c->dS[l]);
         const float* rows = c->pre[l] ? c->P[l] : c->H[l - 1];
-#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l], c->Eb[l], senders, c->posmap)
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l], c->Eb[l], senders, c->posmap, (int)(c->scatter_mode != RIPPLE_SCATTER_PULL), (int)c->self_term, c->A[l - 1], c->bitmap)
         RP_WIDTH_DISPATCH(ld, ROWS);
 #undef ROWS
     }
