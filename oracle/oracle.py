@@ -51,7 +51,7 @@ def _load():
     for name in ("orc_apply_incremental", "orc_apply_incremental_pull", "orc_apply_scoped"):
         getattr(lib, name).argtypes = [vp, vp, i64, vp, i64]
         getattr(lib, name).restype = i32
-    for name in ("orc_H", "orc_S", "orc_full_H", "orc_full_S"):
+    for name in ("orc_H", "orc_S", "orc_Den", "orc_full_H", "orc_full_S"):
         getattr(lib, name).argtypes = [vp, i32]
         getattr(lib, name).restype = ctypes.POINTER(ctypes.c_double)
     lib.orc_affected.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_int)]
@@ -180,6 +180,10 @@ class Oracle:
 
     def S(self, l: int) -> np.ndarray:
         return self._mat(self.lib.orc_S(self.h, l), self.n, self.dims[l - 1])
+
+    def Den(self, l: int) -> np.ndarray:
+        """Attention layers: the cached denominator sum of every vertex (S holds the numerator)."""
+        return np.ctypeslib.as_array(self.lib.orc_Den(self.h, l), shape=(self.n,))
 
     def full(self) -> List[np.ndarray]:
         """O-full on the current graph and features: [H^0, H^1, .., H^L] (fresh copies)."""

@@ -28,6 +28,12 @@
  *     replaces its feature row by zeros; the id stays addressable, so later operations of the same
  *     or a later batch may attach edges or features to it again (a vertex addition, which the
  *     paper models as the edge addition that creates the endpoint, Sec. 4.1);
+ *   - attention layers (Sec. 3.4.1, Eq. 3): a vertex with no in-neighbour outputs zeros; the cached
+ *     numerator and denominator are the unshifted sums of Eq. 3's terms (the definition route shifts
+ *     by the largest logit, the usual evaluation of a softmax); a vertex whose own row changed at hop
+ *     l-1 is a hop-l vertex (it recomputes there), so the tree grows with a self term; the layer's
+ *     eps is the slope of the logit for negative arguments: 1 gives Eq. 3 as printed, a value below
+ *     1 the leaky rectifier of the architecture that Eq. 3 cites; width in = width out;
  *
  * Parity with the authors' own program is unpinned for the mean and weighted-sum degree handling
  * (the paper gives no formula); parity with the definition (orc_full) is pinned for all of it.
@@ -42,7 +48,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { KIND_SAGE = 0, KIND_GRAPHCONV = 1, KIND_GIN = 2 };
+enum { KIND_SAGE = 0, KIND_GRAPHCONV = 1, KIND_GIN = 2, KIND_GAT = 3 };
 enum { AGG_SUM = 0, AGG_MEAN = 1, AGG_WSUM_GCN = 2, AGG_MAX = 3, AGG_MIN = 4, AGG_WSUM_EDGE = 5 };
 #define MONOTONIC(agg) ((agg) == AGG_MAX || (agg) == AGG_MIN)
 enum { ACT_IDENTITY = 0, ACT_RELU = 1 };
@@ -69,7 +75,8 @@ typedef struct {
     layer_t *layer;    /* layer[1..L] */
     ivec *out, *in;
     double **H;        /* H[0..L]: N x d[l] */
-    double **S;        /* S[1..L]: N x d[l-1], un-normalised aggregate */
+    double **S;        /* S[1..L]: N x d[l-1], un-normalised aggregate (attention: the numerator sum) */
+    double **Den;      /* attention layers, Den[1..L]: N, the denominator sum of Eq. 3 */
     double **FH, **FS; /* buffers of orc_full */
     int **A;           /* A[0..L]: affected sets of the last batch, ascending */
     int *nA;
@@ -248,6 +255,7 @@ oracle_t *orc_create_weighted(int N, int64_t E, const int32_t *src, const int32_
     o->S = (double **)calloc((size_t)L + 1, sizeof(double *));
     o->FH = (double **)calloc((size_t)L + 1, sizeof(double *));
     o->FS = (double **)calloc((size_t)L + 1, sizeof(double *));
+    o->Den = (double **)calloc((size_t)L + 1, sizeof(double *));
     o->A = (int **)calloc((size_t)L + 1, sizeof(int *));
     o->nA = (int *)calloc((size_t)L + 1, sizeof(int));
     o->active_edges = (long *)calloc((size_t)L + 1, sizeof(long));
@@ -255,6 +263,7 @@ oracle_t *orc_create_weighted(int N, int64_t E, const int32_t *src, const int32_
     for (int l = 0; l <= L; ++l) {
         o->H[l] = (double *)calloc((size_t)N * (size_t)dims[l], sizeof(double));
         if (l > 0) o->S[l] = (double *)calloc((size_t)N * (size_t)dims[l - 1], sizeof(double));
+        if (l > 0) o->Den[l] = (double *)calloc((size_t)N, sizeof(double));
     }
     for (size_t i = 0; i < (size_t)N * (size_t)dims[0]; ++i) o->H[0][i] = (double)feat[i];
     return o;
@@ -282,6 +291,8 @@ void orc_set_layer(oracle_t *o, int l, int kind, int d_hid, int act, double eps,
     if (kind == KIND_GIN) {
         ly->Wa = widen(Wa, K * Hd); ly->ba = widen(ba, Hd);
         ly->Wb = widen(Wb, Hd * J); ly->bb = widen(bb, J);
+    } else if (kind == KIND_GAT) {   /* Wa = W (d_in x d_hid), ba = source half of a, bb = sink half of a (Eq. 3) */
+        ly->Wa = widen(Wa, K * Hd); ly->ba = widen(ba, Hd); ly->bb = widen(bb, Hd);
     } else {
         ly->Wa = widen(Wa, K * J); ly->ba = widen(ba, J);
         ly->Wb = kind == KIND_SAGE ? widen(Wb, K * J) : NULL;
@@ -292,16 +303,92 @@ void orc_destroy(oracle_t *o) {
     if (!o) return;
     for (int v = 0; v < o->N; ++v) { free(o->out[v].a); free(o->in[v].a); free(o->out[v].w); free(o->in[v].w); }
     for (int l = 0; l <= o->L; ++l) {
-        free(o->H[l]); free(o->S[l]); free(o->FH[l]); free(o->FS[l]); free(o->A[l]);
+        free(o->H[l]); free(o->S[l]); free(o->FH[l]); free(o->FS[l]); free(o->A[l]); free(o->Den[l]);
         free(o->layer[l].Wa); free(o->layer[l].Wb); free(o->layer[l].ba); free(o->layer[l].bb);
     }
-    free(o->out); free(o->in); free(o->H); free(o->S); free(o->FH); free(o->FS); free(o->A);
+    free(o->out); free(o->in); free(o->H); free(o->S); free(o->FH); free(o->FS); free(o->A); free(o->Den);
     free(o->nA); free(o->layer); free(o->d); free(o->mark); free(o->active_edges); free(o);
 }
 
 /* One whole layer for every vertex (Eq. 1-2): S = aggregate, H = sigma(Update). */
+/* ------------------------------------------------------------------------------------------ */
+/* Attention layers (Sec. 3.4.1, Eq. 3): h^{l+1}_v = sum_{u in In(v)} alpha_uv h^l_u,
+ * alpha_uv = softmax over In(v) of z_uv, z_uv = a . (W h_u || W h_v).  No in-neighbours: zeros. */
+/* z = a . (W h_u || W h_v) as Eq. 3 prints it when eps (the slope for negative arguments) is 1; the
+ * architecture Eq. 3 cites passes that number through a leaky rectifier, which is eps < 1 */
+static double gat_logit(const layer_t *ly, double s_u, double t_v) {
+    double z = s_u + t_v;
+    return z < 0.0 ? ly->eps * z : z;
+}
+
+static double gat_logit_part(const layer_t *ly, const double *a_half, const double *h) {
+    double s = 0.0;   /* a_half . (W h), W h = Wa^T h with Wa input-major */
+    for (int j = 0; j < ly->d_hid; ++j) {
+        double wh = 0.0;
+        for (int k = 0; k < ly->d_in; ++k) wh += ly->Wa[(size_t)k * ly->d_hid + j] * h[k];
+        s += a_half[j] * wh;
+    }
+    return s;
+}
+
+/* the definition for one vertex, with the usual shift by the largest logit */
+static void gat_row_definition(const oracle_t *o, int l, int v, const double *Hprev, double *out) {
+    const layer_t *ly = &o->layer[l];
+    int K = o->d[l - 1];
+    const ivec *in = &o->in[v];
+    for (int k = 0; k < K; ++k) out[k] = 0.0;
+    if (in->n == 0) return;
+    double tv = gat_logit_part(ly, ly->bb, Hprev + (size_t)v * K);
+    double *z = (double *)malloc(sizeof(double) * (size_t)in->n), zmax = -1e300, den = 0.0;
+    for (int i = 0; i < in->n; ++i) {
+        z[i] = gat_logit(ly, gat_logit_part(ly, ly->ba, Hprev + (size_t)in->a[i] * K), tv);
+        if (z[i] > zmax) zmax = z[i];
+    }
+    for (int i = 0; i < in->n; ++i) den += exp(z[i] - zmax);
+    for (int i = 0; i < in->n; ++i) {
+        double alpha = exp(z[i] - zmax) / den;
+        const double *h = Hprev + (size_t)in->a[i] * K;
+        for (int k = 0; k < K; ++k) out[k] += alpha * h[k];
+    }
+    free(z);
+    if (ly->act == ACT_RELU) for (int k = 0; k < K; ++k) out[k] = out[k] > 0.0 ? out[k] : 0.0;
+}
+
+/* numerator and denominator sums of Eq. 3 as the incremental route caches them (no shift) */
+static void gat_sums(const oracle_t *o, int l, int v, const double *Hprev, double *num, double *den) {
+    const layer_t *ly = &o->layer[l];
+    int K = o->d[l - 1];
+    const ivec *in = &o->in[v];
+    for (int k = 0; k < K; ++k) num[k] = 0.0;
+    *den = 0.0;
+    double tv = gat_logit_part(ly, ly->bb, Hprev + (size_t)v * K);
+    for (int i = 0; i < in->n; ++i) {
+        const double *h = Hprev + (size_t)in->a[i] * K;
+        double e = exp(gat_logit(ly, gat_logit_part(ly, ly->ba, h), tv));
+        for (int k = 0; k < K; ++k) num[k] += e * h[k];
+        *den += e;
+    }
+}
+
+static void gat_output(const layer_t *ly, int K, int deg_in, const double *num, double den, double *out) {
+    for (int k = 0; k < K; ++k) {
+        double x = deg_in > 0 ? num[k] / den : 0.0;
+        out[k] = (ly->act == ACT_RELU && x < 0.0) ? 0.0 : x;
+    }
+}
+
 static void full_layer(const oracle_t *o, int l, const double *Hprev, double *S, double *H) {
     int K = o->d[l - 1], J = o->d[l];
+    if (o->layer[l].kind == KIND_GAT) {
+#pragma omp parallel for schedule(dynamic, 256)
+        for (int v = 0; v < o->N; ++v) {
+            double den;
+            gat_sums(o, l, v, Hprev, S + (size_t)v * K, &den);
+            if (S == o->S[l]) o->Den[l][v] = den;          /* the cached state (bootstrap), not the buffers of orc_full */
+            gat_row_definition(o, l, v, Hprev, H + (size_t)v * J);
+        }
+        return;
+    }
 #pragma omp parallel for schedule(dynamic, 256)
     for (int v = 0; v < o->N; ++v) {
         aggregate_row(o, v, Hprev, K, S + (size_t)v * K);
@@ -709,6 +796,95 @@ static int apply_incremental_max(oracle_t *o, const delta_t *dl, const float *fe
     return 0;
 }
 
+/* Hybrid-incremental propagation through attention layers (Sec. 3.4.1).  Every vertex caches the
+ * numerator sum_u exp(z_uv) h_u and the denominator sum_u exp(z_uv) of its output.  A vertex that
+ * was in the tree at hop l-1 (its own h^{l-1} changed, so every z_uv it is the sink of changed) is in
+ * the tree at hop l too and recomputes both sums over all of its in-neighbours; any other hop-l vertex
+ * takes <numerator, denominator> messages: exp(z_new) h_new - exp(z_old) h_old from a changed
+ * in-neighbour, the whole new term along an added edge, minus the whole old term along a deleted one. */
+static int apply_incremental_gat(oracle_t *o, const delta_t *dl, const float *feat_rows) {
+    int L = o->L, d0 = o->d[0];
+    int nA = dl->nF;
+    int *A = (int *)malloc(sizeof(int) * (size_t)(nA + 1));
+    memcpy(A, dl->F, sizeof(int) * (size_t)nA);
+    double *oldA = (double *)malloc(sizeof(double) * ((size_t)nA * (size_t)d0 + 1));
+    for (int i = 0; i < nA; ++i) {
+        double *row = o->H[0] + (size_t)A[i] * d0;
+        memcpy(oldA + (size_t)i * d0, row, sizeof(double) * (size_t)d0);
+        const float *src = dl->Frow[i] >= 0 ? feat_rows + (size_t)dl->Frow[i] * d0 : NULL;
+        for (int k = 0; k < d0; ++k) row[k] = src ? (double)src[k] : 0.0;
+    }
+    set_list(o, 0, A, nA);
+    unsigned char *recomputes = (unsigned char *)calloc((size_t)o->N, 1);
+
+    for (int l = 1; l <= L; ++l) {
+        const layer_t *ly = &o->layer[l];
+        int K = o->d[l - 1];
+        const double *Hp = o->H[l - 1];
+        double *S = o->S[l], *Den = o->Den[l];
+        int nAn; long walked;
+        int *An = next_affected(o, dl, A, nA, A, nA, 1, &nAn, &walked);
+        o->active_edges[l] = walked + dl->n_add + dl->n_del;
+        for (int i = 0; i < nA; ++i) recomputes[A[i]] = 1;
+
+        for (int i = 0; i < nA; ++i) {      /* changed in-neighbour, surviving edge */
+            int u = A[i];
+            const double *hnew = Hp + (size_t)u * K, *hold = oldA + (size_t)i * K;
+            double s_new = gat_logit_part(ly, ly->ba, hnew), s_old = gat_logit_part(ly, ly->ba, hold);
+            const ivec *r = &o->out[u];
+            for (int j = 0; j < r->n; ++j) {
+                int v = r->a[j];
+                if (recomputes[v]) continue;
+                pair_t p = { u, v, 0.f };
+                if (dl->n_add && bsearch(&p, dl->add, (size_t)dl->n_add, sizeof(pair_t), cmp_pair)) continue;
+                double tv = gat_logit_part(ly, ly->bb, Hp + (size_t)v * K);
+                double e_new = exp(gat_logit(ly, s_new, tv)), e_old = exp(gat_logit(ly, s_old, tv));
+                double *Sv = S + (size_t)v * K;
+                for (int k = 0; k < K; ++k) Sv[k] += e_new * hnew[k] - e_old * hold[k];
+                Den[v] += e_new - e_old;
+            }
+        }
+        for (int i = 0; i < dl->n_add; ++i) {   /* added edge: the new term arrives */
+            int u = dl->add[i].u, v = dl->add[i].v;
+            if (recomputes[v]) continue;
+            const double *hnew = Hp + (size_t)u * K;
+            double e = exp(gat_logit(ly, gat_logit_part(ly, ly->ba, hnew), gat_logit_part(ly, ly->bb, Hp + (size_t)v * K)));
+            double *Sv = S + (size_t)v * K;
+            for (int k = 0; k < K; ++k) Sv[k] += e * hnew[k];
+            Den[v] += e;
+        }
+        for (int i = 0; i < dl->n_del; ++i) {   /* deleted edge: the old term leaves */
+            int u = dl->del[i].u, v = dl->del[i].v;
+            if (recomputes[v]) continue;
+            int ia = find_sorted(A, nA, u);
+            const double *hold = ia >= 0 ? oldA + (size_t)ia * K : Hp + (size_t)u * K;
+            double e = exp(gat_logit(ly, gat_logit_part(ly, ly->ba, hold), gat_logit_part(ly, ly->bb, Hp + (size_t)v * K)));
+            double *Sv = S + (size_t)v * K;
+            for (int k = 0; k < K; ++k) Sv[k] -= e * hold[k];
+            Den[v] -= e;
+        }
+#pragma omp parallel for schedule(dynamic, 64)
+        for (int i = 0; i < nA; ++i) {      /* in the tree one hop earlier: recompute */
+            int v = A[i];
+            gat_sums(o, l, v, Hp, S + (size_t)v * K, &Den[v]);
+            recomputes[v] = 0;
+        }
+        double *oldAn = (double *)malloc(sizeof(double) * ((size_t)nAn * (size_t)K + 1));
+        for (int i = 0; i < nAn; ++i) {
+            int v = An[i];
+            double *row = o->H[l] + (size_t)v * K;
+            memcpy(oldAn + (size_t)i * K, row, sizeof(double) * (size_t)K);
+            if (o->in[v].n == 0) { memset(S + (size_t)v * K, 0, sizeof(double) * (size_t)K); Den[v] = 0.0; }
+            gat_output(ly, K, o->in[v].n, S + (size_t)v * K, Den[v], row);
+        }
+        set_list(o, l, An, nAn);
+        free(A); free(oldA);
+        A = An; nA = nAn; oldA = oldAn;
+    }
+    free(A); free(oldA); free(recomputes);
+    return 0;
+}
+
 /* O-inc: incremental propagation of one batch (Sec. 3.3).  Returns 0, or <0 if the batch is
  * rejected (nothing changed).
  * pull = 0: every sender walks its out-list and adds its message to each sink's inbox, one thread
@@ -726,9 +902,15 @@ static int apply_incremental(oracle_t *o, const update_t *ups, int64_t n, const 
     int L = o->L, self_term = o->layer[1].kind != KIND_GRAPHCONV;
 
     if (MONOTONIC(o->agg)) {
-        if (o->layer[1].kind == KIND_GIN) { delta_free(&dl); return -3; }   /* GraphConv and SAGE layers only */
+        if (o->layer[1].kind >= KIND_GIN) { delta_free(&dl); return -3; }   /* GraphConv and SAGE layers only */
         apply_topology(o, &dl);
         rc = apply_incremental_max(o, &dl, feat_rows);
+        delta_free(&dl);
+        return rc;
+    }
+    if (o->layer[1].kind == KIND_GAT) {
+        apply_topology(o, &dl);
+        rc = apply_incremental_gat(o, &dl, feat_rows);
         delta_free(&dl);
         return rc;
     }
@@ -884,6 +1066,11 @@ int orc_apply_scoped(oracle_t *o, const update_t *ups, int64_t n, const float *f
 #pragma omp parallel for schedule(dynamic, 64)
         for (int i = 0; i < nAn; ++i) {
             int v = An[i];
+            if (o->layer[l].kind == KIND_GAT) {
+                gat_sums(o, l, v, o->H[l - 1], o->S[l] + (size_t)v * K, &o->Den[l][v]);
+                gat_row_definition(o, l, v, o->H[l - 1], o->H[l] + (size_t)v * J);
+                continue;
+            }
             aggregate_row(o, v, o->H[l - 1], K, o->S[l] + (size_t)v * K);
             layer_row(&o->layer[l], o->H[l - 1] + (size_t)v * K, o->S[l] + (size_t)v * K,
                       norm_sink(o, o->in[v].n), o->H[l] + (size_t)v * J);
@@ -933,9 +1120,30 @@ int orc_apply_structure(oracle_t *o, const update_t *ups, int64_t n, int64_t n_r
 void orc_row_from_prev(const oracle_t *o, int l, int v, const float *Hprev, int64_t ld,
                        double *S_out, double *h_out) {
     int K = o->d[l - 1];
+    const ivec *in = &o->in[v];
+    if (o->layer[l].kind == KIND_GAT) {   /* Eq. 3 over the widened rows of v and its in-neighbours; S_out: numerator sum */
+        const layer_t *ly = &o->layer[l];
+        double *rows = (double *)malloc(sizeof(double) * (size_t)K * (size_t)(in->n + 1));
+        double *z = (double *)malloc(sizeof(double) * (size_t)(in->n + 1));
+        for (int k = 0; k < K; ++k) { rows[k] = (double)Hprev[(size_t)v * (size_t)ld + k]; S_out[k] = 0.0; h_out[k] = 0.0; }
+        double tv = gat_logit_part(ly, ly->bb, rows), zmax = -1e300, den = 0.0;
+        for (int i = 0; i < in->n; ++i) {
+            double *r = rows + (size_t)(i + 1) * K;
+            for (int k = 0; k < K; ++k) r[k] = (double)Hprev[(size_t)in->a[i] * (size_t)ld + k];
+            z[i] = gat_logit(ly, gat_logit_part(ly, ly->ba, r), tv);
+            if (z[i] > zmax) zmax = z[i];
+        }
+        for (int i = 0; i < in->n; ++i) den += exp(z[i] - zmax);
+        for (int i = 0; i < in->n; ++i) {
+            const double *r = rows + (size_t)(i + 1) * K;
+            for (int k = 0; k < K; ++k) { S_out[k] += exp(z[i]) * r[k]; h_out[k] += exp(z[i] - zmax) / den * r[k]; }
+        }
+        if (ly->act == ACT_RELU) for (int k = 0; k < K; ++k) h_out[k] = h_out[k] > 0.0 ? h_out[k] : 0.0;
+        free(rows); free(z);
+        return;
+    }
     double *hp = (double *)malloc(sizeof(double) * (size_t)K);
     for (int k = 0; k < K; ++k) { S_out[k] = 0.0; hp[k] = (double)Hprev[(size_t)v * (size_t)ld + k]; }
-    const ivec *in = &o->in[v];
     for (int i = 0; i < in->n; ++i) {
         int u = in->a[i];
         double c = in_edge_coef(o, v, i);
@@ -971,6 +1179,7 @@ int orc_num_threads(void) {
 }
 double *orc_H(oracle_t *o, int l) { return o->H[l]; }
 double *orc_S(oracle_t *o, int l) { return o->S[l]; }
+double *orc_Den(oracle_t *o, int l) { return o->Den[l]; }
 double *orc_full_H(oracle_t *o, int l) { return l == 0 ? o->H[0] : o->FH[l]; }
 double *orc_full_S(oracle_t *o, int l) { return o->FS[l]; }
 const int *orc_affected(oracle_t *o, int l, int *n) { *n = o->nA[l]; return o->A[l]; }

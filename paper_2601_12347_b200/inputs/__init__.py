@@ -28,7 +28,8 @@ UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
 
 KIND_SAGE = 0      # h = act(W_self h_v + W_neigh agg_v + b)
 KIND_GRAPHCONV = 1  # h = act(W agg_v + b)            (no self term)
-KIND_GIN = 2       # h = act(W2 relu(W1 ((1+eps) h_v + agg_v) + b1) + b2)
+KIND_GIN = 2
+KIND_GAT = 3       # h = act(W2 relu(W1 ((1+eps) h_v + agg_v) + b1) + b2)
 
 AGG_SUM = 0
 AGG_MEAN = 1
@@ -165,8 +166,8 @@ class LayerSpec:
     d_in: int
     d_out: int
     act: int
-    d_hidden: int = 0          # GIN only: width of the MLP's hidden layer
-    eps: float = 0.0           # GIN only
+    d_hidden: int = 0          # GIN: width of the MLP's hidden layer; attention: width of W h
+    eps: float = 0.0           # GIN: eps; attention: slope of the logit for negative arguments (1 = linear)
 
 
 @dataclass
@@ -207,6 +208,14 @@ def gin_model(d0: int, hidden: int, n_layers: int, eps: float = 0.0,
                                          d_hidden=hidden, eps=eps) for i in range(n_layers)])
 
 
+def gat_model(d: int, n_layers: int, d_att: int = 8, slope: float = 1.0,
+              act: int = ACT_IDENTITY) -> ModelSpec:
+    """Attention layers: every layer keeps the width d (the output is a convex combination of
+    in-neighbour rows); d_att is the width of W h that the attention vector a reads."""
+    return ModelSpec(AGG_SUM, [LayerSpec(KIND_GAT, d, d, act, d_hidden=d_att, eps=slope)
+                               for _ in range(n_layers)])
+
+
 def _glorot(rng: np.random.Generator, fan_in: int, fan_out: int) -> np.ndarray:
     a = np.sqrt(6.0 / (fan_in + fan_out))
     return rng.uniform(-a, a, size=(fan_in, fan_out)).astype(np.float32)
@@ -216,7 +225,7 @@ def make_weights(model: ModelSpec, seed: int, zero_bias: bool = True) -> List[Di
     """Glorot-uniform matrices (input-major: fan_in x fan_out, row-major), one dict per layer.
 
     SAGE: Wa = W_self, Wb = W_neigh, ba.   GraphConv: Wa, ba.   GIN: Wa (d_in x hid), ba,
-    Wb (hid x d_out), bb.  Biases are zero unless zero_bias is False (then small uniform).
+    Wb (hid x d_out), bb.   Attention: Wa = W (d_in x d_att), ba / bb = halves of a (never zeroed).  Biases are zero unless zero_bias is False (then small uniform).
     """
     rng = _rng(seed, "weights")
     out = []
@@ -230,6 +239,10 @@ def make_weights(model: ModelSpec, seed: int, zero_bias: bool = True) -> List[Di
                  "ba": bias(l.d_out)}
         elif l.kind == KIND_GRAPHCONV:
             w = {"Wa": _glorot(rng, l.d_in, l.d_out), "ba": bias(l.d_out)}
+        elif l.kind == KIND_GAT:   # Wa = W (d_in x d_att); ba, bb = the source and sink halves of a
+            a = _glorot(rng, 2 * l.d_hidden, 1).reshape(-1)
+            w = {"Wa": _glorot(rng, l.d_in, l.d_hidden), "ba": a[:l.d_hidden].copy(),
+                 "bb": a[l.d_hidden:].copy()}
         else:
             w = {"Wa": _glorot(rng, l.d_in, l.d_hidden), "ba": bias(l.d_hidden),
                  "Wb": _glorot(rng, l.d_hidden, l.d_out), "bb": bias(l.d_out)}
