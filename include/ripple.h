@@ -71,8 +71,18 @@ typedef enum {
 /* Update functions (Eq. 2) of the model families of Sec. 6.1.1, x_v = normalised aggregate:
  *   SAGE       h = act(Wa^T h_v + Wb^T x_v + ba)                         (self term)
  *   GRAPHCONV  h = act(Wa^T x_v + ba)                                    (no self term)
- *   GIN        h = act(Wb^T relu(Wa^T ((1 + eps) h_v + x_v) + ba) + bb)  (self term) */
-typedef enum { RIPPLE_LAYER_SAGE = 0, RIPPLE_LAYER_GRAPHCONV = 1, RIPPLE_LAYER_GIN = 2 } ripple_layer_kind;
+ *   GIN        h = act(Wb^T relu(Wa^T ((1 + eps) h_v + x_v) + ba) + bb)  (self term)
+ * and the attention layer of Sec. 3.4.1 (Eq. 3), which takes the hybrid-incremental path:
+ *   GAT        h = act(sum over in-neighbours u of alpha_uv h_u),  alpha_uv = softmax over In(v) of z_uv,
+ *              z_uv = rect(ba . (Wa^T h_u) + bb . (Wa^T h_v)),  rect(z) = z for z >= 0 and eps * z below
+ *              (eps = 1: the linear logit Eq. 3 prints; eps < 1: the leaky rectifier of the architecture it
+ *              cites).  ba, bb are the source and sink halves of Eq. 3's vector a.  d_out = d_in; a vertex
+ *              without in-neighbours outputs zeros; agg must be RIPPLE_AGG_SUM (it is not read).
+ *              A vertex whose own row changed at hop l-1 is a hop-l vertex and gathers its sums anew there;
+ *              every other hop-l vertex is updated by <numerator, denominator> messages.
+ *              ripple_get_aggregate: width d_in + 1, columns 0..d_in-1 the numerator sum_u exp(z_uv) h_u,
+ *              column d_in the denominator sum_u exp(z_uv). */
+typedef enum { RIPPLE_LAYER_SAGE = 0, RIPPLE_LAYER_GRAPHCONV = 1, RIPPLE_LAYER_GIN = 2, RIPPLE_LAYER_GAT = 3 } ripple_layer_kind;
 
 typedef enum { RIPPLE_ACT_IDENTITY = 0, RIPPLE_ACT_RELU = 1 } ripple_act;
 
@@ -111,6 +121,7 @@ typedef struct {
  *   SAGE:      Wa = W_self (d_in x d_out), Wb = W_neigh (d_in x d_out), ba (d_out)
  *   GRAPHCONV: Wa (d_in x d_out), ba (d_out)
  *   GIN:       Wa (d_in x d_hidden), ba (d_hidden), Wb (d_hidden x d_out), bb (d_out)
+ *   GAT:       Wa = W (d_in x d_hidden), ba = a_src (d_hidden), bb = a_dst (d_hidden), all required; eps = slope
  * All HOST pointers; biases may be NULL (zero).  d_in of layer l must equal d_out of layer l-1. */
 typedef struct {
     int32_t kind; /* ripple_layer_kind */

@@ -274,7 +274,7 @@ void feature_rows(Ctx* c, int n) {
     if (n <= 0) return;
     RP_LAUNCH(c, k_feature_rows, std::min(div_up(n, 8), c->n_sm * 8), 256, 0, c->ctl, c->ups_dev, c->feat_dev,
               c->d[0], c->A[0], c->feat_last, (int)c->src_norm, c->side[0].deg, c->deg_out_old, c->H[0],
-              c->ld[0], c->D[0], (int)(rp_monotonic(c->agg)));
+              c->ld[0], c->D[0], (int)(rp_monotonic(c->agg) || c->attention));
 }
 
 // ---------------------------------------------------------------------------------------------

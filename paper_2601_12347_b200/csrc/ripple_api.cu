@@ -70,10 +70,12 @@ static void destroy_ctx(Ctx* c) {
         cudaFree(sd.free_blk); cudaFree(sd.free_cnt);
     }
     for (int l = 0; l <= RP_MAXL; ++l) {
+        cudaFree(c->att_s[l]); cudaFree(c->att_t[l]);
         cudaFree(c->H[l]); cudaFree(c->S[l]); cudaFree(c->dS[l]); cudaFree(c->Eb[l]); cudaFree(c->Z[l]); cudaFree(c->P[l]); cudaFree(c->A[l]);
         cudaFree(c->layer[l].W1); cudaFree(c->layer[l].b1); cudaFree(c->layer[l].W2); cudaFree(c->layer[l].b2);
         for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2, &c->layer[l].tc_self}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
+    cudaFree(c->att_so); cudaFree(c->att_items);
     cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->invmask); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->opw_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->scan_done); cudaFree(c->ctl);
@@ -109,6 +111,7 @@ static ripple_status run_full(Ctx* c) {
     RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
     if (c->timing) cudaEventRecord(c->ev[0], c->stream);
     for (int l = 1; l <= c->L; ++l) {
+        if (c->attention) { att_full(c, l); continue; }
         if (rp_monotonic(c->agg)) max_full(c, l);
         else spmm_full(c, l);
         if (c->Eb[l]) cudaMemsetAsync(c->Eb[l], 0, sizeof(float) * (size_t)c->N, c->stream);   // every row freshly gathered
@@ -151,10 +154,12 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
     }
     for (int l = 0; l < L; ++l) {
         const ripple_layer& y = layers[l];
-        bool ok = y.kind >= 0 && y.kind <= 2 && y.d_in >= 1 && y.d_out >= 1 && y.d_in <= 1024 && y.d_out <= 1024 &&
+        bool ok = y.kind >= 0 && y.kind <= 3 && y.d_in >= 1 && y.d_out >= 1 && y.d_in <= 1024 && y.d_out <= 1024 &&
                   (y.act == 0 || y.act == 1) && y.Wa && y.kind == layers[0].kind;
         if (y.kind == RIPPLE_LAYER_SAGE) ok = ok && y.Wb;
         if (y.kind == RIPPLE_LAYER_GIN) ok = ok && y.Wb && y.d_hidden >= 1 && y.d_hidden <= 1024;
+        if (y.kind == RIPPLE_LAYER_GAT)
+            ok = ok && y.ba && y.bb && y.d_hidden >= 1 && y.d_hidden <= 1024 && y.d_out == y.d_in && agg == RIPPLE_AGG_SUM;
         if (l > 0) ok = ok && y.d_in == layers[l - 1].d_out;
         if (!ok) { set_err(nullptr, "bad description of layer %d", l + 1); return st; }
     }
@@ -187,6 +192,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         c->self_term = layers[0].kind != RIPPLE_LAYER_GRAPHCONV;
         c->src_norm = agg == RIPPLE_AGG_WSUM_GCN;
         c->weighted = agg == RIPPLE_AGG_WSUM_EDGE;
+        c->attention = layers[0].kind == RIPPLE_LAYER_GAT;
         CK(dev_alloc(&c->ctl, 1, 0));
         CK(dev_alloc(&c->params_dev, 2, 0));
         CK(cudaMallocHost(&c->params_host, 2 * sizeof(int)));
@@ -251,6 +257,19 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             } else if (y.kind == RIPPLE_LAYER_GRAPHCONV) {
                 w1 = padded_matrix(y.Wa, y.d_in, y.d_out, ly.ld_in, ly.ld_out);
                 b1 = padded_matrix(y.ba, 1, y.d_out, 1, ly.ld_out);
+            } else if (y.kind == RIPPLE_LAYER_GAT) {
+                // a . (W h) = (W a) . h: the two halves of a are folded into W once (Wa is d_in x d_hidden, input-major)
+                w1.assign((size_t)2 * ly.ld_in, 0.f);
+                for (int k = 0; k < y.d_in; ++k) {
+                    double qs = 0.0, qt = 0.0;
+                    for (int j = 0; j < y.d_hidden; ++j) {
+                        qs += (double)y.Wa[(size_t)k * y.d_hidden + j] * (double)y.ba[j];
+                        qt += (double)y.Wa[(size_t)k * y.d_hidden + j] * (double)y.bb[j];
+                    }
+                    w1[k] = (float)qs;
+                    w1[(size_t)ly.ld_in + k] = (float)qt;
+                }
+                b1.assign(1, 0.f);
             } else {
                 w1 = padded_matrix(y.Wa, y.d_in, y.d_hidden, ly.ld_in, ly.ld_hid);
                 b1 = padded_matrix(y.ba, 1, y.d_hidden, 1, ly.ld_hid);
@@ -258,7 +277,12 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                 b2 = padded_matrix(y.bb, 1, y.d_out, 1, ly.ld_out);
                 max_hid = std::max(max_hid, ly.ld_hid);
             }
-            {
+            if (y.kind == RIPPLE_LAYER_GAT) {
+                c->pre[l] = false;
+                c->ws[l] = pad4(y.d_in + 1);   // numerator columns, then the denominator
+                c->fused_fold[l] = false;
+                c->regather_threshold[l] = -1.f;
+            } else {
                 // a layer narrower than its input transforms the few sender rows before the scatter
                 const int target = y.kind == RIPPLE_LAYER_GIN ? ly.ld_hid : ly.ld_out;
                 // Also for equal widths where nothing but the matrix product is left per affected row
@@ -313,13 +337,18 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
                          if (!rp_monotonic(agg) && !c->fused_fold[l] && o.rebuild_budget >= 0.f)
                              CK(dev_alloc(&c->Eb[l], (size_t)N, 0));
                          if (c->layer[l].kind == RIPPLE_LAYER_SAGE) CK(dev_alloc(&c->Z[l], (size_t)N * c->ld[l], 0));
-                         if (c->pre[l]) CK(dev_alloc(&c->P[l], (size_t)N * c->ws[l], 0)); }
+                         if (c->pre[l]) CK(dev_alloc(&c->P[l], (size_t)N * c->ws[l], 0));
+                         if (c->attention) { CK(dev_alloc(&c->att_s[l], (size_t)N, 0)); CK(dev_alloc(&c->att_t[l], (size_t)N, 0)); } }
             CK(dev_alloc(&c->A[l], (size_t)N + 32));
         }
         CK(cudaMemcpy2D(c->H[0], sizeof(float) * c->ld[0], features, sizeof(float) * c->d[0],
                         sizeof(float) * c->d[0], (size_t)N,
                         feat_mem == RIPPLE_MEM_DEVICE ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice));
         if (max_hid) CK(dev_alloc(&c->T, (size_t)N * max_hid));
+        if (c->attention) {
+            CK(dev_alloc(&c->att_so, (size_t)N + 32));
+            CK(dev_alloc(&c->att_items, (size_t)N + (size_t)(c->side[1].col_size / 256) + 64));
+        }
         CK(dev_alloc(&c->Dt, (size_t)N * max_ld));
         for (int s = 0; s < 2; ++s) {
             CK(dev_alloc(&c->D[s], (size_t)N * max_ld));
@@ -404,8 +433,19 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
             STAMP();
         }
     }
+    if (c->attention) {
+        // hybrid-incremental hops of attention layers (Sec. 3.4.1)
+        for (int l = 1; l <= L; ++l) {
+            STAMP();
+            att_hop(c, l, nb);
+            STAMP();
+            att_update(c, l, false);
+            if (l < L) senders_build(c, l, nb);
+            STAMP();
+        }
+    }
     // one superstep per hop (Sec. 3.3.1): frontier, send + aggregate, compute + prepare
-    for (int l = 1; l <= L && !rp_monotonic(c->agg); ++l) {
+    for (int l = 1; l <= L && !rp_monotonic(c->agg) && !c->attention; ++l) {
         // The push scatter walks the same out-lists as the frontier and marks the sinks itself; the
         // gathering forms need the list A_l first, so the frontier walk is a pass of its own for them
         // (decided per hop on the device for the rebuilding form).
@@ -443,7 +483,7 @@ static void arm_rebuild(Ctx* c, int nb) {
     for (int l = 0; l <= c->L; ++l) c->tc_armed |= c->stats.affected[l] >= 256 || c->stats.senders[l] >= 256;
     for (int l = 1; l <= c->L; ++l) {
         bool armed = false;
-        if (rp_monotonic(c->agg)) armed = false;
+        if (rp_monotonic(c->agg) || c->attention) armed = false;
         else if (c->scatter_mode == RIPPLE_SCATTER_REGATHER) armed = true;
         else if (c->scatter_mode == RIPPLE_SCATTER_AUTO && c->regather_threshold[l] > 0.f)
             armed = (no_history || (double)c->stats.active_edges[l] >=
@@ -622,7 +662,7 @@ extern "C" ripple_status ripple_get_aggregate(ripple_ctx* ctx, int32_t layer, co
     *dev_ptr = c->S[layer];
     *ld = c->ws[layer];
     const LayerDev& ly = c->layer[layer];
-    if (width) *width = c->pre[layer] ? (ly.kind == RIPPLE_LAYER_GIN ? ly.d_hid : ly.d_out) : ly.d_in;
+    if (width) *width = c->attention ? ly.d_in + 1 : c->pre[layer] ? (ly.kind == RIPPLE_LAYER_GIN ? ly.d_hid : ly.d_out) : ly.d_in;
     if (transformed) *transformed = c->pre[layer] ? 1 : 0;
     return RIPPLE_OK;
 }

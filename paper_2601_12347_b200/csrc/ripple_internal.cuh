@@ -106,7 +106,8 @@ struct LayerDev {
     int kind, d_in, d_hid, d_out, act;
     float eps;
     int ld_in, ld_hid, ld_out;  // padded widths (multiples of 4)
-    float* W1;   // SAGE: [W_self; W_neigh] (2 ld_in x ld_out); GRAPHCONV: ld_in x ld_out; GIN: ld_in x ld_hid
+    float* W1;   // SAGE: [W_self; W_neigh] (2 ld_in x ld_out); GRAPHCONV: ld_in x ld_out; GIN: ld_in x ld_hid;
+                 // attention: the two logit vectors W a_src, W a_dst (2 x ld_in)
     float* b1;   // ld_out (SAGE, GRAPHCONV) or ld_hid (GIN)
     float* W2;   // GIN: d_hid x ld_out
     float* b2;   // GIN: ld_out
@@ -123,6 +124,7 @@ struct Ctx {
     int N, L, agg;
     bool self_term, src_norm;
     bool weighted;             // every edge carries a stored weight (RIPPLE_AGG_WSUM_EDGE)
+    bool attention;            // attention layers (Sec. 3.4.1): S^l rows hold [numerator | denominator]
     float* opw_dev;            // batch staging: one weight per operation (weighted only)
     int has_opw;               // the batch being applied came with weights
     int64_t E0;
@@ -153,6 +155,10 @@ struct Ctx {
     float* Eb[RP_MAXL + 1];   // per vertex: rounding budget spent on S^l_v since the row was last gathered (see k_fold_deltas), or null
     bool fused_fold[RP_MAXL + 1];   // S^l += dS^l happens inside the row update's epilogue (no budget kept)
     float rebuild_tau2;       // square of the budget, in roundings of the row's largest entry
+    float* att_s[RP_MAXL + 1];   // attention: source half of the logit, (W a_src) . h^{l-1}_v, per vertex
+    float* att_t[RP_MAXL + 1];   // attention: sink half, (W a_dst) . h^{l-1}_v
+    float* att_so;               // attention: source halves the senders of the current hop had before the batch (list order)
+    int2* att_items;             // attention: (vertex, in-list chunk) work items of the rows gathered anew
     float* T;          // GIN hidden rows (compact, N x ld_hid)
     float* D[2];       // delta rows, ping-pong (compact, N x max ld)
     float* Dt;         // delta rows after the neighbour transform (compact, N x max inbox width)
@@ -268,6 +274,11 @@ void choose_direction(Ctx* c, int l);                   // delta or rebuilding f
 void scatter_layer(Ctx* c, int l, int n);               // delta messages of hop l into dS^l
 void regather_layer(Ctx* c, int l);                     // rebuilding form: S^l rows of A_l gathered anew
 void fold_deltas(Ctx* c, int l);                        // S^l += dS^l, dS^l = 0 on the rows of A_l
+
+// attention.cu (attention layers, Sec. 3.4.1)
+void att_full(Ctx* c, int l);                           // bootstrap: logit halves, cached rows, embeddings of every vertex
+void att_hop(Ctx* c, int l, int n);                     // frontier, messages, recomputation: cached rows of A_l
+void att_update(Ctx* c, int l, bool full);              // h^l = numerator / denominator on the rows of A_l; keeps the old rows
 
 // layer_update.cu
 void update_rows(Ctx* c, int l, bool full);             // re-apply Update^l + activation, emit deltas

@@ -20,7 +20,7 @@ MAX_LAYERS = 8
 OK, ERR_INVALID_ARG, ERR_VERTEX_RANGE, ERR_CAPACITY, ERR_OOM, ERR_CUDA, ERR_TIMEOUT = range(7)
 MEM_HOST, MEM_DEVICE = 0, 1
 AGG_SUM, AGG_MEAN, AGG_WSUM_GCN, AGG_MAX, AGG_MIN, AGG_WSUM_EDGE = 0, 1, 2, 3, 4, 5
-LAYER_SAGE, LAYER_GRAPHCONV, LAYER_GIN = 0, 1, 2
+LAYER_SAGE, LAYER_GRAPHCONV, LAYER_GIN, LAYER_GAT = 0, 1, 2, 3
 ACT_IDENTITY, ACT_RELU = 0, 1
 OP_ADD_EDGE, OP_DEL_EDGE, OP_SET_FEATURE, OP_DEL_VERTEX = 0, 1, 2, 3
 SCATTER_AUTO, SCATTER_PUSH, SCATTER_PULL, SCATTER_REGATHER, SCATTER_PUSH_BULK = 0, 1, 2, 3, 4
