@@ -331,17 +331,19 @@ static double gat_logit_part(const layer_t *ly, const double *a_half, const doub
     return s;
 }
 
-/* the definition for one vertex, with the usual shift by the largest logit */
-static void gat_row_definition(const oracle_t *o, int l, int v, const double *Hprev, double *out) {
+/* the definition for one vertex, with the usual shift by the largest logit; sv / tv: the two halves of
+ * the logit for every vertex if the caller has them (whole-graph passes), else NULL */
+static void gat_row_definition(const oracle_t *o, int l, int v, const double *Hprev, const double *sv,
+                               const double *tv_all, double *out) {
     const layer_t *ly = &o->layer[l];
     int K = o->d[l - 1];
     const ivec *in = &o->in[v];
     for (int k = 0; k < K; ++k) out[k] = 0.0;
     if (in->n == 0) return;
-    double tv = gat_logit_part(ly, ly->bb, Hprev + (size_t)v * K);
+    double tv = tv_all ? tv_all[v] : gat_logit_part(ly, ly->bb, Hprev + (size_t)v * K);
     double *z = (double *)malloc(sizeof(double) * (size_t)in->n), zmax = -1e300, den = 0.0;
     for (int i = 0; i < in->n; ++i) {
-        z[i] = gat_logit(ly, gat_logit_part(ly, ly->ba, Hprev + (size_t)in->a[i] * K), tv);
+        z[i] = gat_logit(ly, sv ? sv[in->a[i]] : gat_logit_part(ly, ly->ba, Hprev + (size_t)in->a[i] * K), tv);
         if (z[i] > zmax) zmax = z[i];
     }
     for (int i = 0; i < in->n; ++i) den += exp(z[i] - zmax);
@@ -355,16 +357,17 @@ static void gat_row_definition(const oracle_t *o, int l, int v, const double *Hp
 }
 
 /* numerator and denominator sums of Eq. 3 as the incremental route caches them (no shift) */
-static void gat_sums(const oracle_t *o, int l, int v, const double *Hprev, double *num, double *den) {
+static void gat_sums(const oracle_t *o, int l, int v, const double *Hprev, const double *sv,
+                     const double *tv_all, double *num, double *den) {
     const layer_t *ly = &o->layer[l];
     int K = o->d[l - 1];
     const ivec *in = &o->in[v];
     for (int k = 0; k < K; ++k) num[k] = 0.0;
     *den = 0.0;
-    double tv = gat_logit_part(ly, ly->bb, Hprev + (size_t)v * K);
+    double tv = tv_all ? tv_all[v] : gat_logit_part(ly, ly->bb, Hprev + (size_t)v * K);
     for (int i = 0; i < in->n; ++i) {
         const double *h = Hprev + (size_t)in->a[i] * K;
-        double e = exp(gat_logit(ly, gat_logit_part(ly, ly->ba, h), tv));
+        double e = exp(gat_logit(ly, sv ? sv[in->a[i]] : gat_logit_part(ly, ly->ba, h), tv));
         for (int k = 0; k < K; ++k) num[k] += e * h[k];
         *den += e;
     }
@@ -380,13 +383,20 @@ static void gat_output(const layer_t *ly, int K, int deg_in, const double *num, 
 static void full_layer(const oracle_t *o, int l, const double *Hprev, double *S, double *H) {
     int K = o->d[l - 1], J = o->d[l];
     if (o->layer[l].kind == KIND_GAT) {
+        double *sv = (double *)malloc(sizeof(double) * (size_t)o->N), *tv = (double *)malloc(sizeof(double) * (size_t)o->N);
+#pragma omp parallel for schedule(static)
+        for (int v = 0; v < o->N; ++v) {
+            sv[v] = gat_logit_part(&o->layer[l], o->layer[l].ba, Hprev + (size_t)v * K);
+            tv[v] = gat_logit_part(&o->layer[l], o->layer[l].bb, Hprev + (size_t)v * K);
+        }
 #pragma omp parallel for schedule(dynamic, 256)
         for (int v = 0; v < o->N; ++v) {
             double den;
-            gat_sums(o, l, v, Hprev, S + (size_t)v * K, &den);
+            gat_sums(o, l, v, Hprev, sv, tv, S + (size_t)v * K, &den);
             if (S == o->S[l]) o->Den[l][v] = den;          /* the cached state (bootstrap), not the buffers of orc_full */
-            gat_row_definition(o, l, v, Hprev, H + (size_t)v * J);
+            gat_row_definition(o, l, v, Hprev, sv, tv, H + (size_t)v * J);
         }
+        free(sv); free(tv);
         return;
     }
 #pragma omp parallel for schedule(dynamic, 256)
@@ -866,7 +876,7 @@ static int apply_incremental_gat(oracle_t *o, const delta_t *dl, const float *fe
 #pragma omp parallel for schedule(dynamic, 64)
         for (int i = 0; i < nA; ++i) {      /* in the tree one hop earlier: recompute */
             int v = A[i];
-            gat_sums(o, l, v, Hp, S + (size_t)v * K, &Den[v]);
+            gat_sums(o, l, v, Hp, NULL, NULL, S + (size_t)v * K, &Den[v]);
             recomputes[v] = 0;
         }
         double *oldAn = (double *)malloc(sizeof(double) * ((size_t)nAn * (size_t)K + 1));
@@ -1067,8 +1077,8 @@ int orc_apply_scoped(oracle_t *o, const update_t *ups, int64_t n, const float *f
         for (int i = 0; i < nAn; ++i) {
             int v = An[i];
             if (o->layer[l].kind == KIND_GAT) {
-                gat_sums(o, l, v, o->H[l - 1], o->S[l] + (size_t)v * K, &o->Den[l][v]);
-                gat_row_definition(o, l, v, o->H[l - 1], o->H[l] + (size_t)v * J);
+                gat_sums(o, l, v, o->H[l - 1], NULL, NULL, o->S[l] + (size_t)v * K, &o->Den[l][v]);
+                gat_row_definition(o, l, v, o->H[l - 1], NULL, NULL, o->H[l] + (size_t)v * J);
                 continue;
             }
             aggregate_row(o, v, o->H[l - 1], K, o->S[l] + (size_t)v * K);

@@ -466,6 +466,16 @@ def workloads() -> Dict[str, Workload]:
                                (1, 10, 100, 1000), 100, {"edge_weights": True}),
         "dense-gcw-2l": Workload("dense-gcw-2l", n_d, e_d, "rmat", graphconv_model([100, 256, 47], AGG_WSUM_EDGE), 0,
                                  (100, 1000), 20, {"edge_weights": True}),
+        # attention layers (the paper's GA-A workload, Sec. 6.1.1): hybrid-incremental propagation; the
+        # layer of Eq. 3 keeps its input's width, logits go through the leaky rectifier of the cited architecture
+        "sparse-gat": Workload("sparse-gat", n_s, e_s, "rmat", gat_model(128, 2, d_att=8, slope=0.2), 0,
+                               (1, 10, 100, 1000), 100),
+        "mid-gat-2l": Workload("mid-gat-2l", 1_000_000, 30_000_000, "rmat", gat_model(100, 2, d_att=8, slope=0.2), 0,
+                               (1000,), 20),
+        "dense-gat-2l": Workload("dense-gat-2l", n_d, e_d, "rmat", gat_model(100, 2, d_att=8, slope=0.2), 0,
+                                 (10, 100, 1000), 20),
+        "dense-gat-3l": Workload("dense-gat-3l", n_d, e_d, "rmat", gat_model(100, 3, d_att=8, slope=0.2), 0,
+                                 (100, 1000), 20),
         # all five update types of Sec. 3.1: 2 % of the updates delete a vertex
         "sparse-vdel": Workload("sparse-vdel", n_s, e_s, "rmat", sage_model([128, 256, 40]), 0, (100, 1000), 100,
                                 {"mix": (0.39, 0.39, 0.2, 0.02), "max_batch": 65536}),

@@ -236,6 +236,8 @@ DEEP_CASES = [
     ("dense-3l-hub-feature", 5, [0, 2, 2]),
     ("dense-3l-hub-delete", 5, [0, 2, 2]),
     ("dense-4l", 2, [0, 0, 2, 2]),
+    ("dense-gat-2l", 3, [0, 0]),        # attention layers never take the rebuilding form: recomputation is per vertex
+    ("dense-gat-3l", 2, [0, 0, 0]),
     ("reddit-2l", 2, [0, 2]),
     ("reddit-4l", 2, [0, 2, 2, 2]),
 ]
