@@ -26,7 +26,7 @@
 namespace rp {
 
 constexpr int ATT_CHUNK = 64;     // out-edges per warp work item of the message walk
-constexpr int ATT_GATHER = 256;   // in-list entries per warp work item of a recomputation
+constexpr int ATT_GATHER = 128;   // in-list entries per warp work item of a recomputation
 
 __device__ __forceinline__ float att_weight(float s_u, float t_v, float slope) {
     float z = s_u + t_v;
@@ -161,12 +161,14 @@ __global__ void k_att_records(Ctl* ctl, const Rec* __restrict__ rec, const int32
 }
 
 // Per hop-l vertex (or per vertex, `all`): either fold the accumulated messages into the cached row,
-// keeping the row's rounding budget, or -- the vertex is a sender (its own h^{l-1} changed), the
-// budget has run out, or `all` -- zero the row and queue its in-list, in chunks, for k_att_gather.
+// keeping the row's rounding budget, and write the new embedding row at once; or -- the vertex is a
+// sender (its own h^{l-1} changed), the budget has run out, no in-neighbour is left, or `all` -- zero
+// the row, queue its in-list, in chunks, for k_att_gather and flag the vertex for k_att_update.
 __global__ void __launch_bounds__(256)
 k_att_fold(Ctl* ctl, int l, const int32_t* __restrict__ A, const int* n_dev, int n_host, int all, int ld, float* S,
            float* dS, float* budget, float tau2, const int32_t* __restrict__ deg_in,
-           const int32_t* __restrict__ posmap, int2* items) {
+           const int32_t* __restrict__ posmap, int2* items, int d, int act, float* H, int ld_h, float* Old,
+           uint32_t* gathered) {
     pdl_enter();
     if (ctl->abort) return;
     const int n = n_dev ? *n_dev : n_host;
@@ -189,21 +191,32 @@ k_att_fold(Ctl* ctl, int l, const int32_t* __restrict__ A, const int* n_dev, int
                 s[q] = x;
                 dd[q] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            if (!budget) continue;
+            bool keep = true;
+            if (budget) {
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                m_old = fmaxf(m_old, __shfl_xor_sync(FULL, m_old, o));
-                m_new = fmaxf(m_new, __shfl_xor_sync(FULL, m_new, o));
+                for (int o = 16; o > 0; o >>= 1) {
+                    m_old = fmaxf(m_old, __shfl_xor_sync(FULL, m_old, o));
+                    m_new = fmaxf(m_new, __shfl_xor_sync(FULL, m_new, o));
+                }
+                const float m = fmaxf(m_old, m_new);
+                const float spent = budget[v] + m * m;
+                const float limit = tau2 * (0.5f + (float)(mix64((uint64_t)v) & 255u) * (1.0f / 512.0f)) * m_new * m_new;
+                keep = !(spent > limit);
+                if (keep && lane == 0) budget[v] = spent;
             }
-            const float m = fmaxf(m_old, m_new);
-            const float spent = budget[v] + m * m;
-            const float limit = tau2 * (0.5f + (float)(mix64((uint64_t)v) & 255u) * (1.0f / 512.0f)) * m_new * m_new;
-            if (!(spent > limit)) {
-                if (lane == 0) budget[v] = spent;
+            __syncwarp();
+            if (keep) {   // the row is final: its embedding follows at once
+                const float den = S[off + d];
+                float* hrow = H + (size_t)v * ld_h;
+                for (int k = lane; k < ld_h; k += 32) {
+                    float x = (den > 0.f && k < d) ? S[off + k] / den : 0.f;
+                    if (act == RIPPLE_ACT_RELU) x = fmaxf(x, 0.f);
+                    if (Old) Old[(size_t)i * ld_h + k] = hrow[k];
+                    hrow[k] = x;
+                }
                 continue;
             }
             anew = on_budget = true;
-            __syncwarp();
         }
         for (int q = lane; q < nq; q += 32) {
             s[q] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -216,6 +229,7 @@ k_att_fold(Ctl* ctl, int l, const int32_t* __restrict__ A, const int* n_dev, int
             if (nch) first = atomicAdd(&ctl->rebuild_items[l], nch);
             if (budget) budget[v] = 0.f;
             if (on_budget) atomicAdd(&ctl->n_rebuilt[l], 1);
+            if (gathered) atomicOr(&gathered[v >> 5], 1u << (v & 31));
         }
         first = __shfl_sync(FULL, first, 0);
         for (int ch = lane; ch < nch; ch += 32) items[first + ch] = make_int2(v, ch);
@@ -249,23 +263,36 @@ k_att_gather(Ctl* ctl, int l, const int2* __restrict__ items, Side in, const flo
             const int mine = have ? in.col[base + j0 + lane] : 0;
             const float mine_e = have ? att_weight(att_s[mine], t, slope) : 0.f;
             const int cnt = min(32, j_end - j0);
-            for (int j = 0; j < cnt; j += EPI) {
-                const int jj = j + sub;
-                const int u = __shfl_sync(FULL, mine, jj & 31);
-                const float e = __shfl_sync(FULL, mine_e, jj & 31);
-                if (jj < cnt) {
-                    const float4* row = reinterpret_cast<const float4*>(Hprev + (size_t)u * ld_h);
+            constexpr int UNR = 4;   // neighbour rows in flight per lane group
+            for (int j = 0; j < cnt; j += UNR * EPI) {
+                int u[UNR];
+                float e[UNR];
+                float4 x[UNR][NV];
+#pragma unroll
+                for (int r = 0; r < UNR; ++r) {
+                    const int jj = j + r * EPI + sub;
+                    u[r] = __shfl_sync(FULL, mine, jj & 31);
+                    e[r] = __shfl_sync(FULL, mine_e, jj & 31);
+                    if (jj >= cnt) { u[r] = -1; e[r] = 0.f; }
+                }
+#pragma unroll
+                for (int r = 0; r < UNR; ++r) {
+                    const float4* row = reinterpret_cast<const float4*>(Hprev + (size_t)max(u[r], 0) * ld_h);
 #pragma unroll
                     for (int k = 0; k < NV; ++k) {
                         const int q = ql + LPR * k;
-                        if (q < nq) {
-                            float4 h = q < nqh ? __ldg(row + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-                            float m[4] = {e * h.x, e * h.y, e * h.z, e * h.w};
-                            if (q == qden) m[cden] = e;
-                            acc[k].x += m[0]; acc[k].y += m[1]; acc[k].z += m[2]; acc[k].w += m[3];
-                        }
+                        x[r][k] = (u[r] >= 0 && q < nqh) ? __ldg(row + q) : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
+#pragma unroll
+                for (int r = 0; r < UNR; ++r)
+#pragma unroll
+                    for (int k = 0; k < NV; ++k) {
+                        const int q = ql + LPR * k;
+                        float m[4] = {e[r] * x[r][k].x, e[r] * x[r][k].y, e[r] * x[r][k].z, e[r] * x[r][k].w};
+                        if (q == qden) m[cden] = e[r];
+                        acc[k].x += m[0]; acc[k].y += m[1]; acc[k].z += m[2]; acc[k].w += m[3];
+                    }
             }
         }
 #pragma unroll
@@ -289,10 +316,12 @@ k_att_gather(Ctl* ctl, int l, const int2* __restrict__ items, Side in, const flo
 }
 
 // h^l_v = numerator / denominator (zeros without in-neighbours), activation; the row it replaces is
-// kept, compact and in list order, for the next hop's messages.  One warp per row.
+// kept, compact and in list order, for the next hop's messages.  One warp per row.  With `gathered`
+// only the flagged rows are written (the others got theirs from k_att_fold) and the flags are cleared.
 __global__ void __launch_bounds__(256)
 k_att_update(Ctl* ctl, const int32_t* __restrict__ list, const int* n_dev, int n_host, const float* __restrict__ S,
-             int ld, int d, const int32_t* __restrict__ deg_in, int act, float* H, int ld_h, float* Old) {
+             int ld, int d, const int32_t* __restrict__ deg_in, int act, float* H, int ld_h, float* Old,
+             uint32_t* gathered) {
     pdl_enter();
     if (ctl->abort) return;
     const int n = n_dev ? *n_dev : n_host;
@@ -300,6 +329,11 @@ k_att_update(Ctl* ctl, const int32_t* __restrict__ list, const int* n_dev, int n
     const int lane = lane_id();
     for (int i = warp; i < n; i += nwarps) {
         const int v = list ? list[i] : i;
+        if (gathered) {
+            if (!(gathered[v >> 5] & (1u << (v & 31)))) continue;
+            __syncwarp();
+            if (lane == 0) atomicAnd(&gathered[v >> 5], ~(1u << (v & 31)));
+        }
         const float* srow = S + (size_t)v * ld;
         const float den = srow[d];
         const bool live = deg_in[v] > 0 && den > 0.f;
@@ -327,7 +361,7 @@ void att_update(Ctx* c, int l, bool full) {
     float* old_rows = (full || l == c->L) ? nullptr : c->D[l & 1];   // the last hop sends nothing
     RP_LAUNCH(c, k_att_update, c->n_sm * 8, 256, 0, c->ctl, full ? (const int32_t*)nullptr : c->A[l],
               full ? (const int*)nullptr : &c->ctl->nA[l], c->N, c->S[l], c->ws[l], ly.d_in, c->side[1].deg, ly.act,
-              c->H[l], c->ld[l], old_rows);
+              c->H[l], c->ld[l], old_rows, full ? (uint32_t*)nullptr : c->bitmap);
 }
 
 // bootstrap: logit halves, cached rows and outputs of every vertex
@@ -336,7 +370,8 @@ void att_full(Ctx* c, int l) {
     RP_LAUNCH(c, k_att_scalars, c->n_sm * 8, 256, 0, c->ctl, (const int32_t*)nullptr, (const int*)nullptr, c->N,
               c->H[l - 1], c->ld[l - 1], ly.W1, c->att_s[l], c->att_t[l], (float*)nullptr);
     RP_LAUNCH(c, k_att_fold, c->n_sm * 8, 256, 0, c->ctl, l, (const int32_t*)nullptr, (const int*)nullptr, c->N, 1,
-              c->ws[l], c->S[l], c->dS[l], c->Eb[l], c->rebuild_tau2, c->side[1].deg, c->posmap, c->att_items);
+              c->ws[l], c->S[l], c->dS[l], c->Eb[l], c->rebuild_tau2, c->side[1].deg, c->posmap, c->att_items, ly.d_in,
+              ly.act, c->H[l], c->ld[l], (float*)nullptr, (uint32_t*)nullptr);
     launch_gather(c, l);
     att_update(c, l, true);
 }
@@ -360,7 +395,8 @@ void att_hop(Ctx* c, int l, int n) {
         RP_LAUNCH(c, k_att_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, c->rec, c->posmap,
                   c->H[l - 1], Old, c->ld[l - 1], c->att_so, c->att_s[l], c->att_t[l], ly.eps, ly.d_in, ld, c->dS[l]);
     RP_LAUNCH(c, k_att_fold, c->n_sm * 8, T, 0, c->ctl, l, c->A[l], (const int*)&c->ctl->nA[l], 0, 0, ld, c->S[l],
-              c->dS[l], c->Eb[l], c->rebuild_tau2, c->side[1].deg, c->posmap, c->att_items);
+              c->dS[l], c->Eb[l], c->rebuild_tau2, c->side[1].deg, c->posmap, c->att_items, ly.d_in, ly.act, c->H[l],
+              c->ld[l], l == c->L ? (float*)nullptr : c->D[l & 1], c->bitmap);   // (the bitmap is free between two hops' markings)
     launch_gather(c, l);
     senders_release(c, l - 1);
 }
