@@ -28,8 +28,8 @@ UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
 
 KIND_SAGE = 0      # h = act(W_self h_v + W_neigh agg_v + b)
 KIND_GRAPHCONV = 1  # h = act(W agg_v + b)            (no self term)
-KIND_GIN = 2
-KIND_GAT = 3       # h = act(W2 relu(W1 ((1+eps) h_v + agg_v) + b1) + b2)
+KIND_GIN = 2       # h = act(W2 relu(W1 ((1+eps) h_v + agg_v) + b1) + b2)
+KIND_GAT = 3       # h = act(sum_u softmax_u(z_uv) h_u), z_uv = rect(a_src . W h_u + a_dst . W h_v)   (Eq. 3)
 
 AGG_SUM = 0
 AGG_MEAN = 1
