@@ -179,6 +179,8 @@ typedef struct {
                              edge from a hub deleted) at once.  0: default (8); < 0: never.  Applies to
                              aggregates of input-width rows and to all aggregates of the unnormalised
                              sums (RIPPLE_AGG_SUM, RIPPLE_AGG_WSUM_EDGE).                                 */
+    int32_t n_local;      /* > 0: the context is one worker of a partitioned execution (ripple_part.h): ids
+                             below n_local (a multiple of 32) are its own vertices, the rest halo slots    */
 } ripple_options;
 
 typedef struct {

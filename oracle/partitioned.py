@@ -108,15 +108,14 @@ class Server:
                 if op == OP_ADD_EDGE:
                     self.assign_edge(u, v)
                 pu, pv = int(self.owner[u]), int(self.owner[v])
-                if pu < 0 or pv < 0:
-                    continue                   # deleting an edge of a vertex that was never placed: nothing exists
-                out[pu].append((i, op, u, v, True))
-                if pv != pu:
-                    out[pv].append((i, op, u, v, False))      # the no-compute copy
-                if op == OP_ADD_EDGE and (u, v) not in self.edges:
-                    self.edges.add((u, v)); self.in_degree[v] += 1; self.n_edges += 1
-                elif op == OP_DEL_EDGE and (u, v) in self.edges:
-                    self.edges.discard((u, v)); self.in_degree[v] -= 1; self.n_edges -= 1
+                if pu >= 0 and pv >= 0:        # (deleting an edge of a vertex that was never placed: nothing exists)
+                    out[pu].append((i, op, u, v, True))
+                    if pv != pu:
+                        out[pv].append((i, op, u, v, False))      # the no-compute copy
+                    if op == OP_ADD_EDGE and (u, v) not in self.edges:
+                        self.edges.add((u, v)); self.in_degree[v] += 1; self.n_edges += 1
+                    elif op == OP_DEL_EDGE and (u, v) in self.edges:
+                        self.edges.discard((u, v)); self.in_degree[v] -= 1; self.n_edges -= 1
             else:
                 raise ValueError("only edge additions, edge deletions and feature updates are routed")
             self.seen += 1

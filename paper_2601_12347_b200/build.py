@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libripple.so")
 SOURCES = ["ripple_api.cu", "graph_store.cu", "frontier.cu", "scatter.cu", "layer_update.cu", "layer_update_tc.cu",
-           "monotonic.cu", "attention.cu"]
+           "monotonic.cu", "attention.cu", "partition.cu", "router.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fopenmp,-O2", "-cudart", "static"]
 

@@ -256,7 +256,7 @@ k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_
           const unsigned long long* __restrict__ hwin, const int32_t* __restrict__ op_slot,
           const int32_t* __restrict__ feat_last, const int32_t* __restrict__ vdel_seq, Side out, Side in,
           Rec* rec, uint32_t* bitmap, const float* __restrict__ op_w, int32_t* grow_out, int32_t* grow_in,
-          int32_t* shrink_out, int32_t* shrink_in) {
+          int32_t* shrink_out, int32_t* shrink_in, const uint8_t* __restrict__ silent) {
     pdl_enter();
     __shared__ int s_found;
     __shared__ int s_last;
@@ -295,6 +295,7 @@ k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_
             // stored weights: a new edge takes the weight given with its operation, a deleted one had ...
             x.w = !out.w ? 1.0f : is_add ? ((op_w && i < n_given) ? op_w[i] : 1.0f) : out.w[out.start[op.u] + j_out];
             x.deg_out_old = out.deg[op.u];
+            x.silent = (silent && i < n_given) ? silent[i] : 0;
             x.rep[0] = atomicAdd(&out.touch[op.u], 1) == 0;
             x.rep[1] = atomicAdd(&in.touch[op.v], 1) == 0;
             x.rank[0] = atomicAdd(is_add ? &out.cnt_add[op.u] : &out.cnt_del[op.u], 1);
@@ -416,7 +417,7 @@ void graph_batch_classify(Ctx* c, int n) {
     RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, c->op_seq, c->ctl, c->hwin, c->op_slot, c->feat_last,
               c->vdel_seq, c->side[0], c->side[1], c->rec, c->bitmap,
               (const float*)(c->has_opw ? c->opw_dev : nullptr), c->grow_list[0], c->grow_list[1],
-              c->shrink_list[0], c->shrink_list[1]);
+              c->shrink_list[0], c->shrink_list[1], (const uint8_t*)(c->has_silent ? c->silent_dev : nullptr));
 }
 
 // ---------------------------------------------------------------------------------------------

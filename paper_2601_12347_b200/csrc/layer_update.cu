@@ -289,7 +289,7 @@ __global__ void k_extra_senders(Ctl* ctl, int l, const Rec* __restrict__ rec, in
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     for (int r = warp; r < n; r += nwarps) {
         const Rec x = rec[r];
-        if (!x.rep[0]) continue;           // one record per distinct source
+        if (!x.rep[0] || x.silent) continue;   // one record per distinct source (a no-compute copy names a remote one)
         if (posmap[x.u] >= 0) continue;    // already a sender: its delta came from the row update
         int idx = 0;
         if (lane_id() == 0) idx = atomicAdd(&ctl->nC[l], 1);

@@ -76,6 +76,8 @@ static void destroy_ctx(Ctx* c) {
         for (TcW* t : {&c->layer[l].tc_main, &c->layer[l].tc_nbr, &c->layer[l].tc_2, &c->layer[l].tc_self}) { cudaFree(t->hi); cudaFree(t->lo); }
     }
     cudaFree(c->att_so); cudaFree(c->att_items);
+    cudaFree(c->halo_owner); cudaFree(c->halo_rid); cudaFree(c->silent_dev); cudaFree(c->rows_sent);
+    for (int i = 0; i < c->n_ipc_opened; ++i) cudaIpcCloseMemHandle(c->ipc_opened[i]);
     cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->invmask); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->opw_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
     cudaFree(c->op_slot); cudaFree(c->rec); cudaFree(c->tile_sums); cudaFree(c->scan_done); cudaFree(c->ctl);
@@ -102,6 +104,16 @@ static ripple_status sync_and_fetch_ctl(Ctx* c) {
     return RIPPLE_OK;
 }
 
+// layer l of the full inference: cached aggregates and embeddings of every vertex
+static void full_layer(Ctx* c, int l) {
+    if (c->attention) { att_full(c, l); return; }
+    if (rp_monotonic(c->agg)) max_full(c, l);
+    else spmm_full(c, l);
+    if (c->Eb[l]) cudaMemsetAsync(c->Eb[l], 0, sizeof(float) * (size_t)c->N, c->stream);   // every row freshly gathered
+    self_project(c, l, true);
+    update_rows(c, l, true);
+}
+
 // full layer-wise inference over the current graph (Eq. 1-2): bootstrap and recompute-all
 static ripple_status run_full(Ctx* c) {
     c->launches = 0;
@@ -110,14 +122,7 @@ static ripple_status run_full(Ctx* c) {
     cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream);
     RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
     if (c->timing) cudaEventRecord(c->ev[0], c->stream);
-    for (int l = 1; l <= c->L; ++l) {
-        if (c->attention) { att_full(c, l); continue; }
-        if (rp_monotonic(c->agg)) max_full(c, l);
-        else spmm_full(c, l);
-        if (c->Eb[l]) cudaMemsetAsync(c->Eb[l], 0, sizeof(float) * (size_t)c->N, c->stream);   // every row freshly gathered
-        self_project(c, l, true);
-        update_rows(c, l, true);
-    }
+    for (int l = 1; l <= c->L; ++l) full_layer(c, l);
     if (c->timing) cudaEventRecord(c->ev[1], c->stream);
     ripple_status st = sync_and_fetch_ctl(c);
     if (st) return st;
@@ -168,6 +173,17 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         if (opt) o = *opt;
         if (o.slack <= 0) o.slack = 0.25;
         if (o.max_batch <= 0) o.max_batch = 16384;
+        if (o.n_local != 0) {   // one worker of a partitioned execution
+            const bool linear = agg == RIPPLE_AGG_SUM || agg == RIPPLE_AGG_MEAN || agg == RIPPLE_AGG_WSUM_GCN;
+            if (o.n_local < 0 || (o.n_local & 31) || o.n_local > g->num_vertices || !linear ||
+                layers[0].kind > RIPPLE_LAYER_GIN) {
+                set_err(nullptr, "a partitioned context needs n_local a multiple of 32 within num_vertices, a linear aggregator and SAGE, GRAPHCONV or GIN layers");
+                return st;
+            }
+            o.scatter_mode = RIPPLE_SCATTER_PUSH;   // rows cannot be gathered anew: remote in-neighbours' rows live elsewhere
+            o.rebuild_budget = -1.f;
+            o.no_graphs = 1;
+        }
         if (o.pool_edges <= 0) o.pool_edges = std::max<int64_t>(g->num_edges / 4, 1 << 20);
         o.pool_edges = std::max<int64_t>(o.pool_edges, 4);
         c = new (std::nothrow) Ctx();
@@ -193,6 +209,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         c->src_norm = agg == RIPPLE_AGG_WSUM_GCN;
         c->weighted = agg == RIPPLE_AGG_WSUM_EDGE;
         c->attention = layers[0].kind == RIPPLE_LAYER_GAT;
+        c->n_local = o.n_local;
         CK(dev_alloc(&c->ctl, 1, 0));
         CK(dev_alloc(&c->params_dev, 2, 0));
         CK(cudaMallocHost(&c->params_host, 2 * sizeof(int)));
@@ -384,14 +401,22 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         CK(dev_alloc(&c->vjobs, (size_t)o.max_batch));
         CK(dev_alloc(&c->op_slot, (size_t)o.max_batch));
         CK(dev_alloc(&c->rec, (size_t)o.max_batch));
+        if (c->n_local > 0) {
+            CK(dev_alloc(&c->halo_owner, (size_t)(N - c->n_local), 0xFF));
+            CK(dev_alloc(&c->halo_rid, (size_t)(N - c->n_local), 0xFF));
+            CK(dev_alloc(&c->silent_dev, (size_t)o.max_batch, 0));
+            CK(dev_alloc(&c->rows_sent, (size_t)RP_MAXL + 1, 0));
+        }
         CK(cudaDeviceSynchronize());
 
         {
             const long long e0 = (long long)E;
             CK(cudaMemcpy(&c->ctl->num_edges, &e0, sizeof(e0), cudaMemcpyHostToDevice));
         }
-        st = run_full(c);
-        if (st) { memcpy(g_create_err, c->err, sizeof(g_create_err)); goto fail_keep_msg; }
+        if (c->n_local == 0) {   // (a partitioned context is bootstrapped layer by layer, in step with its peers)
+            st = run_full(c);
+            if (st) { memcpy(g_create_err, c->err, sizeof(g_create_err)); goto fail_keep_msg; }
+        }
         c->stats.num_layers = L;
         c->stats.num_edges = E;
         *out = reinterpret_cast<ripple_ctx*>(c);
@@ -546,6 +571,10 @@ extern "C" ripple_status ripple_apply_batch_weighted(ripple_ctx* ctx, const ripp
     ripple_status st = RIPPLE_OK;
     if (n < 0 || n_rows < 0 || (n > 0 && !ups) || (n_rows > 0 && !feat_rows) || (mem != 0 && mem != 1)) {
         set_err(c, "bad arguments to ripple_apply_batch");
+        return RIPPLE_ERR_INVALID_ARG;
+    }
+    if (c->n_local > 0) {
+        set_err(c, "a partitioned context applies its batches in phases: ripple_part_begin and so on");
         return RIPPLE_ERR_INVALID_ARG;
     }
     if (n > c->max_batch || n_rows > c->max_batch) {
@@ -714,7 +743,7 @@ extern "C" ripple_status ripple_get_degrees(ripple_ctx* ctx, const int32_t** deg
 
 extern "C" ripple_status ripple_recompute_full(ripple_ctx* ctx) {
     Ctx* c = reinterpret_cast<Ctx*>(ctx);
-    if (!c) return RIPPLE_ERR_INVALID_ARG;
+    if (!c || c->n_local > 0) return RIPPLE_ERR_INVALID_ARG;
     cudaSetDevice(c->device);
     return run_full(c);
 }
@@ -739,5 +768,233 @@ extern "C" const char* ripple_last_error(ripple_ctx* ctx) {
 }
 
 extern "C" void ripple_destroy(ripple_ctx* ctx) { destroy_ctx(reinterpret_cast<Ctx*>(ctx)); }
+
+// ---------------------------------------------------------------------------------------------
+// partitioned execution (Sec. 4): one worker's phases; see include/ripple_part.h
+// ---------------------------------------------------------------------------------------------
+static Ctx* worker(ripple_ctx* ctx) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    return (c && c->n_local > 0) ? c : nullptr;
+}
+
+static ripple_status finish_phase(Ctx* c) {
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    if (!e) e = cudaGetLastError();
+    if (e) {
+        set_err(c, "CUDA error in a phase of a partitioned batch: %s", cudaGetErrorString(e));
+        return RIPPLE_ERR_CUDA;
+    }
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_part_exports_get(ripple_ctx* ctx, ripple_part_exports* out) {
+    Ctx* c = worker(ctx);
+    if (!c || !out) return RIPPLE_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    for (int l = 0; l <= c->L; ++l) {
+        out->accumulator[l] = c->dS[l]; out->accumulator_ld[l] = l ? c->ws[l] : 0;
+        out->embeddings[l] = c->H[l]; out->embeddings_ld[l] = c->ld[l];
+    }
+    out->frontier_bitmap = c->bitmap;
+    out->out_degrees = c->side[0].deg;
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_part_set_peer(ripple_ctx* ctx, int32_t rank, const ripple_part_exports* e) {
+    Ctx* c = worker(ctx);
+    if (!c || !e || rank < 0 || rank >= RIPPLE_MAX_PEERS) return RIPPLE_ERR_INVALID_ARG;
+    for (int l = 0; l <= c->L; ++l) {
+        if ((l && e->accumulator_ld[l] != c->ws[l]) || e->embeddings_ld[l] != c->ld[l]) {
+            set_err(c, "peer %d runs another model: row widths differ at layer %d", rank, l);
+            return RIPPLE_ERR_INVALID_ARG;
+        }
+        c->peer_dS[rank][l] = static_cast<float*>(e->accumulator[l]);
+        c->peer_H[rank][l] = static_cast<float*>(e->embeddings[l]);
+    }
+    c->peer_bitmap[rank] = static_cast<uint32_t*>(e->frontier_bitmap);
+    c->peer_deg_out[rank] = static_cast<int32_t*>(e->out_degrees);
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_part_ipc_export(ripple_ctx* ctx, ripple_part_ipc* out) {
+    Ctx* c = worker(ctx);
+    if (!c || !out) return RIPPLE_ERR_INVALID_ARG;
+    static_assert(sizeof(cudaIpcMemHandle_t) == 64, "handle size");
+    cudaSetDevice(c->device);
+    memset(out, 0, sizeof(*out));
+    out->num_layers = c->L;
+    cudaError_t e = cudaIpcGetMemHandle(reinterpret_cast<cudaIpcMemHandle_t*>(out->frontier_bitmap), c->bitmap);
+    if (!e) e = cudaIpcGetMemHandle(reinterpret_cast<cudaIpcMemHandle_t*>(out->out_degrees), c->side[0].deg);
+    for (int l = 0; l <= c->L && !e; ++l) {
+        out->accumulator_ld[l] = l ? c->ws[l] : 0;
+        out->embeddings_ld[l] = c->ld[l];
+        if (l) e = cudaIpcGetMemHandle(reinterpret_cast<cudaIpcMemHandle_t*>(out->accumulator[l]), c->dS[l]);
+        if (!e) e = cudaIpcGetMemHandle(reinterpret_cast<cudaIpcMemHandle_t*>(out->embeddings[l]), c->H[l]);
+    }
+    if (e) { set_err(c, "cudaIpcGetMemHandle failed: %s", cudaGetErrorString(e)); return RIPPLE_ERR_CUDA; }
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_part_ipc_open(ripple_ctx* ctx, int32_t rank, const ripple_part_ipc* in) {
+    Ctx* c = worker(ctx);
+    if (!c || !in || rank < 0 || rank >= RIPPLE_MAX_PEERS || in->num_layers != c->L) return RIPPLE_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    ripple_part_exports ex;
+    memset(&ex, 0, sizeof(ex));
+    auto open = [&](const unsigned char* h, void** p) {
+        cudaIpcMemHandle_t hh;
+        memcpy(&hh, h, sizeof(hh));
+        cudaError_t e = cudaIpcOpenMemHandle(p, hh, cudaIpcMemLazyEnablePeerAccess);
+        if (!e) c->ipc_opened[c->n_ipc_opened++] = *p;
+        return e;
+    };
+    cudaError_t e = open(in->frontier_bitmap, &ex.frontier_bitmap);
+    if (!e) e = open(in->out_degrees, &ex.out_degrees);
+    for (int l = 0; l <= c->L && !e; ++l) {
+        ex.accumulator_ld[l] = in->accumulator_ld[l];
+        ex.embeddings_ld[l] = in->embeddings_ld[l];
+        if (l) e = open(in->accumulator[l], &ex.accumulator[l]);
+        if (!e) e = open(in->embeddings[l], &ex.embeddings[l]);
+    }
+    if (e) { set_err(c, "cudaIpcOpenMemHandle failed: %s", cudaGetErrorString(e)); return RIPPLE_ERR_CUDA; }
+    return ripple_part_set_peer(ctx, rank, &ex);
+}
+
+extern "C" ripple_status ripple_part_set_halos(ripple_ctx* ctx, int32_t first, int32_t count, const int32_t* owner,
+                                               const int32_t* remote_id) {
+    Ctx* c = worker(ctx);
+    if (!c || first < 0 || count < 0 || (count > 0 && (!owner || !remote_id)) ||
+        (int64_t)first + count > (int64_t)c->N - c->n_local)
+        return RIPPLE_ERR_INVALID_ARG;
+    if (count == 0) return RIPPLE_OK;
+    cudaSetDevice(c->device);
+    cudaError_t e = cudaMemcpyAsync(c->halo_owner + first, owner, sizeof(int32_t) * (size_t)count, cudaMemcpyHostToDevice, c->stream);
+    if (!e) e = cudaMemcpyAsync(c->halo_rid + first, remote_id, sizeof(int32_t) * (size_t)count, cudaMemcpyHostToDevice, c->stream);
+    if (!e) e = cudaStreamSynchronize(c->stream);
+    if (e) { set_err(c, "copying the halo table failed: %s", cudaGetErrorString(e)); return RIPPLE_ERR_CUDA; }
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_part_bootstrap_layer(ripple_ctx* ctx, int32_t l) {
+    Ctx* c = worker(ctx);
+    if (!c || l < 1 || l > c->L) return RIPPLE_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    c->launches = 0;
+    c->params_host[0] = 0; c->params_host[1] = 0;
+    cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream);
+    RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
+    part_fetch_halo_rows(c, l - 1);
+    full_layer(c, l);
+    c->stats.num_layers = c->L;
+    c->stats.num_edges = c->E0;
+    return finish_phase(c);
+}
+
+extern "C" ripple_status ripple_part_begin(ripple_ctx* ctx, const ripple_update* ups, int64_t n, const float* feat_rows,
+                                           int64_t n_rows, const uint8_t* no_compute, int32_t mem) {
+    Ctx* c = worker(ctx);
+    if (!c || n < 0 || n_rows < 0 || (n > 0 && !ups) || (n_rows > 0 && !feat_rows) || (mem != 0 && mem != 1))
+        return RIPPLE_ERR_INVALID_ARG;
+    if (n > c->max_batch || n_rows > c->max_batch) {
+        set_err(c, "batch of %lld updates exceeds max_batch = %lld", (long long)n, (long long)c->max_batch);
+        return RIPPLE_ERR_CAPACITY;
+    }
+    if (mem == RIPPLE_MEM_HOST)
+        for (int64_t i = 0; i < n; ++i)
+            if (ups[i].op == RIPPLE_OP_DEL_VERTEX) {
+                set_err(c, "a partitioned context does not take vertex deletions");
+                return RIPPLE_ERR_INVALID_ARG;
+            }
+    cudaSetDevice(c->device);
+    const int nb = (int)n, nr = (int)n_rows;
+    const cudaMemcpyKind kind = mem == RIPPLE_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+    c->launches = 0;
+    c->may_expand = 0;
+    c->has_opw = 0;
+    c->debug_tc_withhold = 0;
+    c->tc_armed = 1;
+    for (int l = 0; l <= c->L; ++l) c->rebuild_armed[l] = 0;
+    if (nb) cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, kind, c->stream);
+    c->has_silent = no_compute && nb;
+    if (c->has_silent) cudaMemcpyAsync(c->silent_dev, no_compute, (size_t)nb, kind, c->stream);
+    if (nr) cudaMemcpyAsync(c->feat_dev, feat_rows, sizeof(float) * (size_t)nr * c->d[0], kind, c->stream);
+    c->params_host[0] = nb; c->params_host[1] = nr;
+    cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream);
+    cudaMemsetAsync(c->rows_sent, 0, sizeof(unsigned long long) * (RP_MAXL + 1), c->stream);
+    // launch geometry for at least one operation: a worker with an empty share still takes part in every hop
+    c->part_nb = std::max(nb, 1);
+    RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
+    graph_batch_classify(c, c->part_nb);
+    graph_batch_mutate(c, c->part_nb);
+    frontier_seed_features(c, c->part_nb);
+    feature_rows(c, c->part_nb);
+    senders_build(c, 0, c->part_nb);
+    ripple_status st = sync_and_fetch_ctl(c);
+    if (st) return st;
+    c->stats.n_ops = nb;
+    if (c->ctl_host->err) {
+        st = (ripple_status)c->ctl_host->err;
+        set_err(c, "batch rejected by a worker (status %d)", (int)st);
+        graph_batch_cleanup(c, c->part_nb);
+        finish_phase(c);
+        return st;
+    }
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_part_hop_send(ripple_ctx* ctx, int32_t l) {
+    Ctx* c = worker(ctx);
+    if (!c || l < 1 || l > c->L) return RIPPLE_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    scatter_layer(c, l, c->part_nb);
+    part_ship(c, l);
+    return finish_phase(c);
+}
+
+extern "C" ripple_status ripple_part_hop_compute(ripple_ctx* ctx, int32_t l) {
+    Ctx* c = worker(ctx);
+    if (!c || l < 1 || l > c->L) return RIPPLE_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    frontier_compact(c, l);
+    fold_deltas(c, l);
+    self_project(c, l, false);
+    update_rows(c, l, false);
+    if (l < c->L) senders_build(c, l, c->part_nb);
+    return finish_phase(c);
+}
+
+extern "C" ripple_status ripple_part_end(ripple_ctx* ctx) {
+    Ctx* c = worker(ctx);
+    if (!c) return RIPPLE_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    graph_batch_cleanup(c, c->part_nb);
+    ripple_status st = sync_and_fetch_ctl(c);
+    if (st) return st;
+    const Ctl& h = *c->ctl_host;
+    ripple_stats& s = c->stats;
+    s.gpu_launches = c->launches;
+    s.n_added = h.n_add; s.n_deleted = h.n_del; s.n_noop_add = h.n_noop_add; s.n_noop_del = h.n_noop_del;
+    s.n_superseded = h.n_superseded; s.n_feature = h.n_feat;
+    s.num_edges += h.n_add - h.n_del;
+    c->batches_done++;
+    for (int l = 0; l <= c->L; ++l) {
+        s.affected[l] = h.nA[l];
+        s.senders[l] = h.nC[l];
+        s.active_edges[l] = l ? (int64_t)h.E[l] + h.n_rec : 0;
+        s.scatter_pull[l] = 0;
+        s.message_width[l] = l ? c->ws[l] : 0;
+    }
+    return RIPPLE_OK;
+}
+
+extern "C" ripple_status ripple_part_rows_sent(ripple_ctx* ctx, int64_t* out) {
+    Ctx* c = worker(ctx);
+    if (!c || !out) return RIPPLE_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    unsigned long long tmp[RP_MAXL + 1];
+    if (cudaMemcpy(tmp, c->rows_sent, sizeof(tmp), cudaMemcpyDeviceToHost) != cudaSuccess) return RIPPLE_ERR_CUDA;
+    for (int l = 0; l <= RP_MAXL; ++l) out[l] = (int64_t)tmp[l];
+    return RIPPLE_OK;
+}
 
 extern "C" const char* ripple_version(void) { return "ripple-b200 0.1 (sm_100a)"; }

@@ -10,6 +10,7 @@
 #include <stdint.h>
 
 #include "../../include/ripple.h"
+#include "../../include/ripple_part.h"
 
 #define RP_MAXL RIPPLE_MAX_LAYERS
 #define RP_TOMB (-1)
@@ -91,6 +92,7 @@ struct Rec {
     int32_t tail_val[2]; // deleted: entry found at tail slot new_deg + rank
     int32_t rep[2];      // 1 for the first record that touched the row
     int32_t deg_out_old; // out-degree of u before the batch
+    int32_t silent;      // partitioned execution: the no-compute copy of a cut edge (the sink's worker sends nothing for it)
     float w;             // stored edge weights: weight of the added edge / weight the deleted edge had
     float tail_w[2];     // deleted: weight found at the tail slot
 };
@@ -125,6 +127,20 @@ struct Ctx {
     bool self_term, src_norm;
     bool weighted;             // every edge carries a stored weight (RIPPLE_AGG_WSUM_EDGE)
     bool attention;            // attention layers (Sec. 3.4.1): S^l rows hold [numerator | denominator]
+    int n_local;               // partitioned execution: ids below are this worker's vertices, the rest halo slots (0: not partitioned)
+    int32_t* halo_owner;       // per halo slot: owning worker, or -1 while unassigned
+    int32_t* halo_rid;         // per halo slot: the vertex's local id at its owner
+    uint8_t* silent_dev;       // batch staging: no-compute flag per operation
+    int has_silent;
+    float* peer_dS[RIPPLE_MAX_PEERS][RP_MAXL + 1];   // peers' message accumulators (device addresses valid here)
+    float* peer_H[RIPPLE_MAX_PEERS][RP_MAXL + 1];
+    uint32_t* peer_bitmap[RIPPLE_MAX_PEERS];
+    int32_t* peer_deg_out[RIPPLE_MAX_PEERS];
+    void* ipc_opened[RIPPLE_MAX_PEERS * (2 * (RP_MAXL + 1) + 2)];   // mappings to close
+    int n_ipc_opened;
+    unsigned long long* rows_sent;   // device, per hop: halo rows shipped by the last batch
+    int part_phase;            // 0 idle, else 1 + the number of phases of the current batch already run
+    int part_nb;
     float* opw_dev;            // batch staging: one weight per operation (weighted only)
     int has_opw;               // the batch being applied came with weights
     int64_t E0;
@@ -279,6 +295,10 @@ void fold_deltas(Ctx* c, int l);                        // S^l += dS^l, dS^l = 0
 void att_full(Ctx* c, int l);                           // bootstrap: logit halves, cached rows, embeddings of every vertex
 void att_hop(Ctx* c, int l, int n);                     // frontier, messages, recomputation: cached rows of A_l
 void att_update(Ctx* c, int l, bool full);              // h^l = numerator / denominator on the rows of A_l; keeps the old rows
+
+// partition.cu (partitioned execution, Sec. 4)
+void part_ship(Ctx* c, int l);             // remote send: halo mailboxes of hop l into their owners' accumulators
+void part_fetch_halo_rows(Ctx* c, int l);  // bootstrap: H^l of every assigned halo slot from its owner
 
 // layer_update.cu
 void update_rows(Ctx* c, int l, bool full);             // re-apply Update^l + activation, emit deltas

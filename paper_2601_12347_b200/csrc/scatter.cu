@@ -451,6 +451,7 @@ __global__ void k_scatter_records(Ctl* ctl, int l, const Rec* __restrict__ rec, 
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
     for (int r = warp; r < n; r += nwarps) {
+        if (rec[r].silent) continue;   // partitioned execution: the source's worker sends for this edge
         const int u = rec[r].u;
         const int p = posmap[u];
         const float4* hrow = reinterpret_cast<const float4*>(Mrows + (size_t)u * ld);
@@ -521,7 +522,7 @@ __global__ void __launch_bounds__(256)
 k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int32_t* __restrict__ deg_out,
                 int src_norm, const float* __restrict__ M, int ld, float* __restrict__ S, float* __restrict__ dS,
                 float* budget, const int32_t* __restrict__ senders, int32_t* posmap, int mark, int self_term,
-                const int32_t* __restrict__ A_prev, uint32_t* bitmap) {
+                const int32_t* __restrict__ A_prev, uint32_t* bitmap, int chores_only) {
     pdl_enter();
     // Two chores of the hop ride along with this kernel, the last of the hop's delta form, whatever form
     // the hop takes.  The hop's senders are no longer looked up by anyone: their entries of the position
@@ -543,7 +544,8 @@ k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int
                 }
         }
     }
-    if (ctl->abort || ctl->regather[l]) return;
+    // (a worker of a partitioned execution cannot gather a row anew: remote in-neighbours' rows live elsewhere)
+    if (ctl->abort || ctl->regather[l] || chores_only) return;
     const int n = ctl->n_rec;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
@@ -730,7 +732,7 @@ void scatter_layer(Ctx* c, int l, int n) {
         RP_LAUNCH(c, k_scatter_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec,
                   (int)c->src_norm, c->side[0].deg, c->posmap, Mrows, Dm, ld, c->dS[l]);
         const float* rows = c->pre[l] ? c->P[l] : c->H[l - 1];
-#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l], c->Eb[l], senders, c->posmap, (int)(c->scatter_mode != RIPPLE_SCATTER_PULL), (int)c->self_term, c->A[l - 1], c->bitmap)
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l], c->Eb[l], senders, c->posmap, (int)(c->scatter_mode != RIPPLE_SCATTER_PULL), (int)c->self_term, c->A[l - 1], c->bitmap, (int)(c->n_local > 0))
         RP_WIDTH_DISPATCH(ld, ROWS);
 #undef ROWS
     }

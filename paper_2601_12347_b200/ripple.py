@@ -35,6 +35,17 @@ EXPORTED = [
     "ripple_export_graph_static", "ripple_set_timing", "ripple_probe_reduction_rate", "ripple_probe_gather_rate",
     "ripple_get_stats", "ripple_last_error", "ripple_destroy", "ripple_version",
 ]
+# partitioned execution (include/ripple_part.h); all but the last six return a status
+EXPORTED_PART = [
+    "ripple_part_exports_get", "ripple_part_set_peer", "ripple_part_ipc_export", "ripple_part_ipc_open",
+    "ripple_part_set_halos", "ripple_part_bootstrap_layer", "ripple_part_begin", "ripple_part_hop_send",
+    "ripple_part_hop_compute", "ripple_part_end", "ripple_part_rows_sent",
+    "ripple_router_create", "ripple_router_partition_shape", "ripple_router_partition_fill",
+    "ripple_router_route", "ripple_router_batch_shape", "ripple_router_batch_fill",
+    "ripple_router_destroy", "ripple_router_owner", "ripple_router_local_id", "ripple_router_global_id",
+    "ripple_router_is_high_degree", "ripple_router_load",
+]
+MAX_PEERS = 16
 
 
 class RippleError(RuntimeError):
@@ -61,7 +72,8 @@ class _Options(ctypes.Structure):
                 ("max_batch", ctypes.c_int64), ("scatter_mode", ctypes.c_int32),
                 ("gemm_mode", ctypes.c_int32), ("timing", ctypes.c_int32),
                 ("pre_transform", ctypes.c_int32), ("no_graphs", ctypes.c_int32), ("device", ctypes.c_int32), ("stream", ctypes.c_void_p),
-                ("regather_threshold", ctypes.c_float), ("rebuild_budget", ctypes.c_float)]
+                ("regather_threshold", ctypes.c_float), ("rebuild_budget", ctypes.c_float),
+                ("n_local", ctypes.c_int32)]
 
 
 class _Stats(ctypes.Structure):
@@ -79,6 +91,20 @@ class _Stats(ctypes.Structure):
                 ("ms_frontier", _F), ("ms_scatter", _F), ("ms_update", _F),
                 ("ms_scatter_kernel", _F), ("ms_regather", _F), ("ms_bootstrap", ctypes.c_float), ("gpu_launches", ctypes.c_int64), ("n_expanded", ctypes.c_int64),
                 ("rows_rebuilt", _A), ("pool_free", ctypes.c_int64), ("pool_lost", ctypes.c_int64)]
+
+
+class _PartExports(ctypes.Structure):
+    _fields_ = [("accumulator", ctypes.c_void_p * (MAX_LAYERS + 1)), ("accumulator_ld", ctypes.c_int64 * (MAX_LAYERS + 1)),
+                ("embeddings", ctypes.c_void_p * (MAX_LAYERS + 1)), ("embeddings_ld", ctypes.c_int64 * (MAX_LAYERS + 1)),
+                ("frontier_bitmap", ctypes.c_void_p), ("out_degrees", ctypes.c_void_p)]
+
+
+class _PartIpc(ctypes.Structure):
+    _fields_ = [("accumulator", (ctypes.c_ubyte * 64) * (MAX_LAYERS + 1)),
+                ("embeddings", (ctypes.c_ubyte * 64) * (MAX_LAYERS + 1)),
+                ("frontier_bitmap", ctypes.c_ubyte * 64), ("out_degrees", ctypes.c_ubyte * 64),
+                ("accumulator_ld", ctypes.c_int64 * (MAX_LAYERS + 1)),
+                ("embeddings_ld", ctypes.c_int64 * (MAX_LAYERS + 1)), ("num_layers", ctypes.c_int32)]
 
 
 _lib = None
@@ -120,6 +146,35 @@ def load_library(path: Optional[str] = None):
     lib.ripple_probe_gather_rate.argtypes = [i32, i64, i32, i64, P(ctypes.c_float)]
     for name in EXPORTED[:15]:
         getattr(lib, name).restype = i32
+    # partitioned execution
+    lib.ripple_part_exports_get.argtypes = [vp, P(_PartExports)]
+    lib.ripple_part_set_peer.argtypes = [vp, i32, P(_PartExports)]
+    lib.ripple_part_ipc_export.argtypes = [vp, P(_PartIpc)]
+    lib.ripple_part_ipc_open.argtypes = [vp, i32, P(_PartIpc)]
+    lib.ripple_part_set_halos.argtypes = [vp, i32, i32, vp, vp]
+    lib.ripple_part_bootstrap_layer.argtypes = [vp, i32]
+    lib.ripple_part_begin.argtypes = [vp, vp, i64, vp, i64, vp, i32]
+    lib.ripple_part_hop_send.argtypes = [vp, i32]
+    lib.ripple_part_hop_compute.argtypes = [vp, i32]
+    lib.ripple_part_end.argtypes = [vp]
+    lib.ripple_part_rows_sent.argtypes = [vp, vp]
+    lib.ripple_router_create.argtypes = [i32, i64, vp, i64, vp, vp, i32, i64, i64, i64, P(vp)]
+    lib.ripple_router_partition_shape.argtypes = [vp, i32, P(i64), P(i64), P(i64), P(i64)]
+    lib.ripple_router_partition_fill.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.ripple_router_route.argtypes = [vp, vp, i64]
+    lib.ripple_router_batch_shape.argtypes = [vp, i32, P(i64), P(i64), P(i64)]
+    lib.ripple_router_batch_fill.argtypes = [vp, i32, vp, vp, vp, P(i32), vp, vp]
+    for name in EXPORTED_PART[:17]:
+        getattr(lib, name).restype = i32
+    lib.ripple_router_destroy.argtypes = [vp]
+    lib.ripple_router_destroy.restype = None
+    for name in ("ripple_router_owner", "ripple_router_local_id", "ripple_router_is_high_degree"):
+        getattr(lib, name).argtypes = [vp, i32]
+        getattr(lib, name).restype = i32
+    lib.ripple_router_global_id.argtypes = [vp, i32, i32]
+    lib.ripple_router_global_id.restype = i32
+    lib.ripple_router_load.argtypes = [vp, i32]
+    lib.ripple_router_load.restype = i64
     _lib = lib
     return lib
 
@@ -149,11 +204,13 @@ class Ripple:
                  slack: float = 0.0, pool_edges: int = 0, max_batch: int = 0,
                  scatter_mode: int = SCATTER_AUTO, gemm_mode: int = GEMM_AUTO, timing: bool = False,
                  pre_transform: bool = True, graphs: bool = True, stream=None,
-                 regather_threshold: float = 0.0, rebuild_budget: float = 0.0, edge_weights=None):
+                 regather_threshold: float = 0.0, rebuild_budget: float = 0.0, edge_weights=None,
+                 n_local: int = 0):
         import torch
         self._torch = torch
         self.lib = load_library()
         self.n = int(n)
+        self.n_local = int(n_local)
         self.model, self.weights = model, weights
         self.L = len(model.layers)
         self.dims = [model.layers[0].d_in] + [l.d_out for l in model.layers]
@@ -206,6 +263,7 @@ class Ripple:
         opt.no_graphs = 0 if graphs else 1
         opt.regather_threshold = float(regather_threshold)
         opt.rebuild_budget = float(rebuild_budget)
+        opt.n_local = int(n_local)     # > 0: one worker of a partitioned execution (see partitioned.py)
         opt.device = torch.cuda.current_device()
         self._stream = stream if stream is not None else torch.cuda.Stream()
         opt.stream = self._stream.cuda_stream

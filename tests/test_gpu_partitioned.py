@@ -1,0 +1,147 @@
+"""Partitioned execution (Sec. 4) on the device: P workers, each a context of its own holding one vertex
+partition, run in one process on one GPU (the phases of a hop run worker after worker; nothing waits
+on the device).  After every batch the rows gathered from the owners must equal the single-machine
+oracle's full recomputation on the global graph, the union of the workers' hop sets the oracle's hop
+sets, and the number of halo rows sent the oracle cluster's (one combined row per worker and remote
+sink)."""
+import numpy as np
+import pytest
+
+from paper_2601_12347_b200 import inputs as I
+from tolerances import TOL
+
+import test_gpu_parity as G
+
+pytestmark = pytest.mark.gpu
+
+env = G.env
+
+MODELS = {
+    "sage_mean": lambda: I.sage_model([18, 36, 10], I.AGG_MEAN),
+    "sage_sum_3l": lambda: I.sage_model([18, 36, 20, 10], I.AGG_SUM),
+    "gc_sum": lambda: I.graphconv_model([18, 36, 10], I.AGG_SUM),
+    "gcn_wsum_3l": lambda: I.graphconv_model([18, 36, 20, 10], I.AGG_WSUM_GCN),
+    "gin_3l": lambda: I.gin_model(18, 24, 3, eps=0.25),
+    "sage_wide": lambda: I.sage_model([40, 160, 24], I.AGG_MEAN),
+}
+
+
+def max_err(got, ref):
+    return float(np.max(np.abs(got.astype(np.float64) - ref) / (1.0 + np.abs(ref)))) if ref.size else 0.0
+
+
+def setup(name, P, n, m, seed, spare=0):
+    from oracle.partitioned import Cluster as OracleCluster
+    from paper_2601_12347_b200.partitioned import Cluster
+    model = MODELS[name]()
+    L = len(model.layers)
+    src, dst = I.er_graph(n, m, seed)
+    have = set(zip(src.tolist(), dst.tolist()))
+    extra = [(0, int(v)) for v in range(1, min(n, 300)) if (0, int(v)) not in have]      # a hub that cuts every partition
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    X = I.features(n + spare, model.dims[0], seed)
+    X[n:] = 0
+    W = I.make_weights(model, seed, zero_bias=False)
+    owner = np.full(n + spare, -1, dtype=np.int32)
+    owner[:n] = np.random.default_rng(seed).integers(0, P, size=n)
+    return model, L, src, dst, X, W, owner, Cluster, OracleCluster
+
+
+@pytest.mark.parametrize("P", [2, 3])
+@pytest.mark.parametrize("name", list(MODELS.keys()))
+def test_workers_compute_what_one_machine_computes(env, name, P):
+    ripple, Oracle = env
+    n = 700
+    model, L, src, dst, X, W, owner, Cluster, OracleCluster = setup(name, P, n, 5000, 3)
+    orc = Oracle(n, src, dst, X, model, W)
+    full = orc.full()
+    ocl = OracleCluster(P, owner, n, src, dst, X, model, W, full, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+    cl = Cluster(P, owner, src, dst, X, model, W)
+    for l in range(L + 1):
+        assert max_err(cl.embeddings(l, n), full[l]) <= TOL, f"bootstrap, layer {l}"
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 3)
+    for b, bs in enumerate([1, 1, 2, 7, 33, 100, 1, 250, 64, 5]):
+        ups, rows = stream.next_batch(bs)
+        cl.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        ocl.apply_batch(ups, rows)
+        for l in range(L + 1):
+            assert np.array_equal(cl.affected(l), orc.affected(l)), (name, P, b, l)
+        assert cl.rows_sent()[1:] == ocl.halo_rows_sent[1:], (name, P, b)
+        if b % 3 == 2 or b == 9:
+            full = orc.full()
+            for l in range(L + 1):
+                assert max_err(cl.embeddings(l, n), full[l]) <= TOL, (name, P, b, l)
+    cl.close()
+
+
+@pytest.mark.parametrize("routing", ["locality", "hash"])
+def test_vertices_created_by_the_stream_are_placed_and_computed(env, routing):
+    ripple, Oracle = env
+    from paper_2601_12347_b200 import partitioned as PT
+    n, spare, P = 400, 40, 3
+    model, L, src, dst, X, W, owner, Cluster, _ = setup("sage_mean", P, n, 3000, 5, spare=spare)
+    orc = Oracle(n + spare, src, dst, X, model, W)
+    cl = Cluster(P, owner, src, dst, X, model, W, routing=PT.ROUTE_LOCALITY if routing == "locality" else PT.ROUTE_HASH,
+                 spare_local=spare)
+    rng = np.random.default_rng(1)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 5)
+    nxt = n
+    for b in range(8):
+        ups, rows = stream.next_batch(20)
+        extra = G.ups_array([(I.OP_ADD_EDGE, nxt, int(rng.integers(0, n))), (I.OP_ADD_EDGE, int(rng.integers(0, n)), nxt + 1),
+                             (I.OP_ADD_EDGE, nxt + 2, nxt + 3), (I.OP_SET_FEATURE, nxt, rows.shape[0])])
+        nxt += 4
+        ups = np.concatenate([ups, extra])
+        rows = np.concatenate([rows, I.features(1, model.dims[0], 100 + b)])
+        cl.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        for l in range(L + 1):
+            assert np.array_equal(cl.affected(l), orc.affected(l)), (b, l)
+    full = orc.full()
+    placed = np.array([cl.router.owner(v) >= 0 for v in range(n + spare)])
+    assert placed[:nxt].all() and not placed[nxt:].any()
+    for l in range(L + 1):
+        assert max_err(cl.embeddings(l, n + spare)[placed], full[l][placed]) <= TOL, l
+    cl.close()
+
+
+def test_one_partition_is_the_single_machine_case(env):
+    ripple, Oracle = env
+    n = 300
+    model, L, src, dst, X, W, owner, Cluster, _ = setup("gc_sum", 1, n, 2000, 9)
+    owner[:] = 0
+    orc = Oracle(n, src, dst, X, model, W)
+    cl = Cluster(1, owner, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 9)
+    for _ in range(5):
+        ups, rows = stream.next_batch(30)
+        cl.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+    assert cl.rows_sent()[1:] == [0] * L
+    full = orc.full()
+    for l in range(L + 1):
+        assert max_err(cl.embeddings(l, n), full[l]) <= TOL
+    cl.close()
+
+
+def test_partitioned_context_refuses_what_it_cannot_do(env):
+    ripple, Oracle = env
+    from paper_2601_12347_b200.partitioned import Cluster
+    n = 200
+    model, L, src, dst, X, W, owner, _, _ = setup("sage_mean", 2, n, 1000, 4)
+    cl = Cluster(2, owner, src, dst, X, model, W)
+    w = cl.workers[0]
+    with pytest.raises(ripple.RippleError):
+        w.apply_batch(G.ups_array([(I.OP_ADD_EDGE, 0, 1)]))
+    with pytest.raises(ripple.RippleError):
+        w.recompute_full()
+    with pytest.raises(ripple.RippleError):
+        w.begin(G.ups_array([(I.OP_DEL_VERTEX, 0, 0)]), None, np.zeros(1, dtype=np.uint8))
+    with pytest.raises(ripple.RippleError):
+        cl.router.route(G.ups_array([(I.OP_DEL_VERTEX, 0, 0)]))
+    cl.close()
+    model = I.graphconv_model([18, 36, 10], I.AGG_MAX)
+    with pytest.raises(ripple.RippleError):
+        Cluster(2, owner, src, dst, X, model, I.make_weights(model, 1))
