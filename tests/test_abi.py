@@ -18,8 +18,8 @@ def lib():
     return ripple.load_library()
 
 
-def header_functions():
-    text = open(os.path.join(ROOT, "include", "ripple.h")).read()
+def header_functions(name="ripple.h"):
+    text = open(os.path.join(ROOT, "include", name)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(ripple_[a-z_]+)\s*\(", text)))
 
@@ -29,6 +29,11 @@ def test_every_declared_symbol_is_exported(lib):
     assert set(names) == set(ripple.EXPORTED)
     for n in names:
         assert getattr(lib, n) is not None
+    part = header_functions("ripple_part.h")
+    assert set(part) == set(ripple.EXPORTED_PART)
+    for n in part:
+        assert getattr(lib, n) is not None
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["ripple.h", "ripple_part.h"]
 
 
 def test_version_and_null_handling(lib):
@@ -49,14 +54,16 @@ def test_struct_sizes_match_the_header(tmp_path):
     import subprocess
     src = tmp_path / "sizes.c"
     src.write_text(
-        '#include <stdio.h>\n#include "ripple.h"\n'
-        'int main(void){printf("%zu %zu %zu %zu %zu\\n", sizeof(ripple_update), sizeof(ripple_graph),'
-        ' sizeof(ripple_layer), sizeof(ripple_options), sizeof(ripple_stats)); return 0;}\n')
+        '#include <stdio.h>\n#include "ripple_part.h"\n'
+        'int main(void){printf("%zu %zu %zu %zu %zu %zu %zu\\n", sizeof(ripple_update), sizeof(ripple_graph),'
+        ' sizeof(ripple_layer), sizeof(ripple_options), sizeof(ripple_stats), sizeof(ripple_part_exports),'
+        ' sizeof(ripple_part_ipc)); return 0;}\n')
     exe = tmp_path / "sizes"
     subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
     got = [int(x) for x in subprocess.check_output([str(exe)]).split()]
     want = [ripple.UPDATE_DTYPE.itemsize] + [ctypes.sizeof(t) for t in
-                                             (ripple._Graph, ripple._Layer, ripple._Options, ripple._Stats)]
+                                             (ripple._Graph, ripple._Layer, ripple._Options, ripple._Stats,
+                                              ripple._PartExports, ripple._PartIpc)]
     assert got == want
 
 
