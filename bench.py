@@ -527,6 +527,78 @@ def run_table(args):
         torch.cuda.empty_cache()
 
 
+def run_partitioned(args):
+    """The partitioned execution (Sec. 4 of the paper) with P workers ON ONE GPU: every phase runs worker
+    after worker, so the wall time per batch is the sum over the workers; beside it the line gives, per
+    batch, the sum over the phases of the slowest worker's time for that phase: what P GPUs would take if
+    the exchange cost nothing beyond what one GPU's memory system charges for it.  Neither is a
+    measurement on NVLink hardware.  Also: combined halo rows sent per hop, and the single-context time on
+    the same stream."""
+    import torch
+    from paper_2601_12347_b200 import build as B
+    from paper_2601_12347_b200 import partitioned as PT
+    from paper_2601_12347_b200 import ripple
+    B.build_library()
+    torch.cuda.set_device(0)
+    Pn = args.partitioned
+    for name in args.table.split(","):
+        w, src, dst, X, W = make_workload(name, args.seed)
+        L = len(w.model.layers)
+        owner = np.random.default_rng(args.seed).integers(0, Pn, size=w.n).astype(np.int32)
+        cl = PT.Cluster(Pn, owner, src, dst, X, w.model, W, max_batch=w.extra.get("max_batch", 16384))
+        rp = ripple.Ripple(w.n, src, dst, X, w.model, W, max_batch=w.extra.get("max_batch", 16384),
+                           scatter_mode=ripple.SCATTER_PUSH, rebuild_budget=-1.0)
+        stream = I.make_stream(w, src, dst, args.seed)
+        for bsz in (args.batch_sizes or w.batch_sizes):
+            nb = args.table_batches
+            wall, model, single = [], [], []
+            sent = np.zeros(L + 1)
+            for i in range(5 + nb):
+                ups, rows = stream.next_batch(bsz)
+                t0 = time.perf_counter()
+                rp.apply_batch(ups, rows)
+                t_single = time.perf_counter() - t0
+                t0 = time.perf_counter()
+                cl.router.route(ups)
+                shares = [cl.router.batch(r) for r in range(Pn)]
+                t_route = time.perf_counter() - t0
+                crit = t_route
+
+                def phase(fn):
+                    worst = 0.0
+                    for r, wk in enumerate(cl.workers):
+                        t1 = time.perf_counter()
+                        fn(r, wk)
+                        worst = max(worst, time.perf_counter() - t1)
+                    return worst
+
+                def begin(r, wk):
+                    lu, nc, row_of, first, ho, hr = shares[r]
+                    if ho.size:
+                        wk.set_halos(first, ho, hr)
+                    wk.begin(lu, rows[row_of] if row_of.size else None, nc)
+
+                crit += phase(begin)
+                for l in range(1, L + 1):
+                    crit += phase(lambda r, wk: wk.hop_send(l))
+                    crit += phase(lambda r, wk: wk.hop_compute(l))
+                crit += phase(lambda r, wk: wk.end())
+                t_wall = time.perf_counter() - t0
+                if i >= 5:
+                    wall.append(t_wall); model.append(crit); single.append(t_single)
+                    sent += np.array(cl.rows_sent())
+            print(json.dumps({
+                "workload": name, "batch": bsz, "batches": nb, "workers": Pn, "placement": "uniformly random owners",
+                "one_gpu_sequential_ms": {"p50": 1e3 * pct(wall, 50), "p99": 1e3 * pct(wall, 99)},
+                "slowest_worker_per_phase_ms": {"p50": 1e3 * pct(model, 50), "p99": 1e3 * pct(model, 99)},
+                "single_context_push_ms": {"p50": 1e3 * pct(single, 50), "p99": 1e3 * pct(single, 99)},
+                "halo_rows_sent_per_hop": (sent[1:] / nb).round(1).tolist(),
+                "note": "all workers on one GPU; not a measurement on NVLink hardware"}), flush=True)
+        cl.close()
+        rp.close()
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--table", default="", help="comma-separated workloads: print one line per batch size")
@@ -544,6 +616,8 @@ def main():
     ap.add_argument("--batch", type=int, default=1000)
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--scatter", type=int, default=0, help="0 auto, 1 push, 2 pull")
+    ap.add_argument("--partitioned", type=int, default=0,
+                    help="with --table: run the workloads as this many workers of the partitioned execution, all on one GPU")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--verbose-steps", action="store_true", help="per timed step: messages and scatter time (stderr)")
     args = ap.parse_args()
@@ -551,7 +625,10 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.table:
+    if args.table and args.partitioned > 0:
+        if rank == 0:
+            run_partitioned(args)
+    elif args.table:
         if rank == 0:
             run_table(args)
     elif args.impl == "reference":
