@@ -17,7 +17,9 @@
 
 namespace rp {
 
-constexpr int MAX_HUB_DEGREE = 1024;   // longer in-lists are recomputed by a whole block
+constexpr int MAX_HUB_DEGREE = 256;    // longer in-lists are recomputed in chunks, one warp per chunk
+constexpr int MAX_HUB_CHUNK = 256;     // in-list entries per chunk
+constexpr int MAX_FULL_PASS_DEGREE = 4096;   // a full pass has rows enough to keep every warp busy: only longer lists are chunked
 constexpr int MAX_CHUNK = 64;          // edges per warp work item of the message walk
 
 // The same code serves min: every comparison goes through these helpers (is_min = 0: maximum).
@@ -151,7 +153,7 @@ k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const in
     for (int i = warp; i < n; i += nwarps) {
         const int v = list ? list[i] : i;
         const int deg = in.deg[v];
-        if (deg > (mode ? MAX_HUB_DEGREE : 4 * MAX_HUB_DEGREE)) {   // a full pass has rows enough to keep every warp busy
+        if (deg > (mode ? MAX_HUB_DEGREE : MAX_FULL_PASS_DEGREE)) {
             if (lane == 0) long_rows[atomicAdd(n_long, 1)] = v;
             continue;
         }
@@ -212,86 +214,113 @@ k_max_rows(Ctl* ctl, int l, int mode, const int32_t* __restrict__ list, const in
     (void)l;
 }
 
-// one block per long row: every warp takes a strided share of the in-list, the partial rows meet in
-// shared memory
-template <int NV>
+// Long rows, in three steps so that a hub's in-list is spread over the whole device instead of one block
+// (a row of 150 000 in-neighbours took a block 4 to 14 ms: the 99th percentile of a batch):
+//   begin   one warp per long row: the row as it is goes to a scratch copy, the elements to be recomputed
+//           (those flagged in the row's mask if they are few, else all) are reset to the worst value, and
+//           the in-list is queued in chunks;
+//   chunks  one warp per (row, chunk): the maximum over the chunk, for those elements, raises the row by
+//           atomic maxima;
+//   end     one warp per long row: compares the row with its scratch copy, marks the vertex affected if
+//           anything differs, clears the mask.
 __global__ void __launch_bounds__(256)
-k_max_long_rows(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const int* __restrict__ n_long, Side in,
-                const float* __restrict__ M, int ld, float* __restrict__ S, uint32_t* bitmapA, uint32_t* invmask,
-                int mw, int is_min) {
+k_max_long_begin(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const int* __restrict__ n_long, Side in,
+                 int ld, float* __restrict__ S, float* __restrict__ saved, const uint32_t* __restrict__ invmask, int mw,
+                 int is_min, int2* items, int* n_items) {
     pdl_enter();
-    extern __shared__ float part[];   // 8 warps x ld floats
-    __shared__ int s_differs;
     if (ctl->abort) return;
     const int n = *n_long;
-    const int warp = threadIdx.x >> 5, lane = lane_id(), nq = ld >> 2;
-    for (int i = blockIdx.x; i < n; i += gridDim.x) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id();
+    for (int i = warp; i < n; i += nwarps) {
         const int v = long_rows[i];
+        float* srow = S + (size_t)v * ld;
+        int el[MAX_EL];
+        const int cnt = mode ? mask_elements(invmask + (size_t)v * mw, mw, ld, el) : -1;
+        for (int k = lane; k < ld; k += 32) {
+            if (mode) saved[(size_t)i * ld + k] = srow[k];
+            if (cnt < 0) srow[k] = worst(is_min);
+        }
+        __syncwarp();   // every element is saved before any is reset
+        if (cnt >= 0 && lane < cnt) srow[el[lane]] = worst(is_min);
+        const int nch = (in.deg[v] + MAX_HUB_CHUNK - 1) / MAX_HUB_CHUNK;
+        int first = 0;
+        if (lane == 0) first = atomicAdd(n_items, nch);
+        first = __shfl_sync(FULL, first, 0);
+        for (int ch = lane; ch < nch; ch += 32) items[first + ch] = make_int2(i, ch);
+    }
+}
+
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_max_long_chunks(Ctl* ctl, int mode, const int32_t* __restrict__ long_rows, const int2* __restrict__ items,
+                  const int* __restrict__ n_items, Side in, const float* __restrict__ M, int ld, float* S,
+                  const uint32_t* __restrict__ invmask, int mw, int is_min) {
+    pdl_enter();
+    if (ctl->abort) return;
+    const int n = *n_items;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id(), nq = ld >> 2;
+    for (int it = warp; it < n; it += nwarps) {
+        const int v = long_rows[items[it].x], ch = items[it].y;
         const int deg = in.deg[v];
-        if (mode) {   // few invalidated elements: every thread strides over the in-list for those alone
-            uint32_t* mask = invmask + (size_t)v * mw;
-            int el[MAX_EL];
-            const int cnt = mask_elements(mask, mw, ld, el);
-            __syncthreads();
-            for (int w = threadIdx.x; w < mw; w += blockDim.x) mask[w] = 0u;
-            if (cnt >= 0) {
-                float acc[MAX_EL];
+        const int j0 = ch * MAX_HUB_CHUNK, j1 = min(deg, j0 + MAX_HUB_CHUNK);
+        float* srow = S + (size_t)v * ld;
+        int el[MAX_EL];
+        const int cnt = mode ? mask_elements(invmask + (size_t)v * mw, mw, ld, el) : -1;
+        if (cnt >= 0) {   // few elements: every lane strides over the chunk for those alone
+            float acc[MAX_EL];
 #pragma unroll
-                for (int t = 0; t < MAX_EL; ++t) acc[t] = worst(is_min);
-                const int64_t base = in.start[v];
-                for (int j = threadIdx.x; j < deg; j += blockDim.x) {
-                    const float* row = M + (size_t)in.col[base + j] * ld;
+            for (int t = 0; t < MAX_EL; ++t) acc[t] = worst(is_min);
+            const int64_t base = in.start[v];
+            for (int j = j0 + lane; j < j1; j += 32) {
+                const float* row = M + (size_t)in.col[base + j] * ld;
 #pragma unroll
-                    for (int t = 0; t < MAX_EL; ++t)
-                        if (t < cnt) acc[t] = pick(acc[t], __ldg(row + el[t]), is_min);
-                }
+                for (int t = 0; t < MAX_EL; ++t)
+                    if (t < cnt) acc[t] = pick(acc[t], __ldg(row + el[t]), is_min);
+            }
 #pragma unroll
-                for (int t = 0; t < MAX_EL; ++t) {
+            for (int t = 0; t < MAX_EL; ++t) {
+                if (t < cnt) {
                     float m = acc[t];
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) m = pick(m, __shfl_xor_sync(FULL, m, o), is_min);
-                    if (lane == 0) part[warp * MAX_EL + t] = m;
+                    if (lane == 0) atomic_pick_f32(srow + el[t], m, is_min);
                 }
-                if (threadIdx.x == 0) s_differs = 0;
-                __syncthreads();
-                if ((int)threadIdx.x < cnt) {
-                    float m = part[threadIdx.x];
-                    for (int w = 1; w < 8; ++w) m = pick(m, part[w * MAX_EL + threadIdx.x], is_min);
-                    float* dst = S + (size_t)v * ld + el[threadIdx.x];
-                    if (*dst != m) { *dst = m; s_differs = 1; }
-                }
-                __syncthreads();
-                if (threadIdx.x == 0 && s_differs) mark_bit(bitmapA, v);
-                __syncthreads();
-                continue;
             }
+            continue;
         }
         float4 acc[NV];
         fill<NV>(acc, worst(is_min));
-        for (int j0 = warp * 1024; j0 < deg; j0 += 8 * 1024)
-            max_accumulate<NV, 32>(acc, in, v, j0, min(deg, j0 + 1024), M, ld, is_min);
+        max_accumulate<NV, 32>(acc, in, v, j0, j1, M, ld, is_min);
 #pragma unroll
         for (int k = 0; k < NV; ++k) {
             const int q = lane + 32 * k;
-            if (q < nq) reinterpret_cast<float4*>(part + (size_t)warp * ld)[q] = acc[k];
-        }
-        if (threadIdx.x == 0) s_differs = 0;
-        __syncthreads();
-        bool differs = false;
-        for (int q = threadIdx.x; q < nq; q += blockDim.x) {
-            float4 m = reinterpret_cast<const float4*>(part)[q];
-            for (int w = 1; w < 8; ++w) m = pick4(m, reinterpret_cast<const float4*>(part + (size_t)w * ld)[q], is_min);
-            float4* dst = reinterpret_cast<float4*>(S + (size_t)v * ld) + q;
-            if (mode) {
-                const float4 o = *dst;
-                differs |= o.x != m.x || o.y != m.y || o.z != m.z || o.w != m.w;
+            if (q < nq) {
+                atomic_pick_f32(srow + 4 * q + 0, acc[k].x, is_min);
+                atomic_pick_f32(srow + 4 * q + 1, acc[k].y, is_min);
+                atomic_pick_f32(srow + 4 * q + 2, acc[k].z, is_min);
+                atomic_pick_f32(srow + 4 * q + 3, acc[k].w, is_min);
             }
-            *dst = m;
         }
-        if (differs) s_differs = 1;
-        __syncthreads();
-        if (mode && threadIdx.x == 0 && s_differs) mark_bit(bitmapA, v);
-        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(256)
+k_max_long_end(Ctl* ctl, const int32_t* __restrict__ long_rows, const int* __restrict__ n_long, int ld,
+               const float* __restrict__ S, const float* __restrict__ saved, uint32_t* bitmapA, uint32_t* invmask,
+               int mw) {
+    pdl_enter();
+    if (ctl->abort) return;
+    const int n = *n_long;
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id();
+    for (int i = warp; i < n; i += nwarps) {
+        const int v = long_rows[i];
+        bool differs = false;
+        for (int k = lane; k < ld; k += 32) differs |= S[(size_t)v * ld + k] != saved[(size_t)i * ld + k];
+        for (int w = lane; w < mw; w += 32) invmask[(size_t)v * mw + w] = 0u;
+        if (__any_sync(FULL, differs) && lane == 0) mark_bit(bitmapA, v);
     }
 }
 
@@ -480,12 +509,19 @@ __global__ void k_max_senders(Ctl* ctl, int l, const int32_t* __restrict__ A, co
     }
 }
 
-static void launch_long_rows(Ctx* c, int mode, const float* M, int ld, float* S, int32_t* long_rows, int* n_long) {
-    const int nv = div_up(ld, 128);
-    const size_t smem = (size_t)8 * std::max(ld, MAX_EL) * sizeof(float);
-#define LONG(NV) RP_LAUNCH(c, k_max_long_rows<NV>, c->n_sm * 8, 256, smem, c->ctl, mode, long_rows, n_long, c->side[1], M, ld, S, c->bitmap, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
-    if (nv <= 1) LONG(1); else if (nv <= 2) LONG(2); else if (nv <= 4) LONG(4); else LONG(8);
-#undef LONG
+static void launch_long_rows(Ctx* c, int l, int mode, const float* M, int ld, float* S, int32_t* long_rows, int* n_long) {
+    const int nv = div_up(ld, 128), is_min = (int)(c->agg == RIPPLE_AGG_MIN);
+    int2* items = reinterpret_cast<int2*>(c->coff);   // the senders' degree prefix is not needed at this point
+    int* n_items = &c->ctl->max_items[l];
+    float* saved = c->Dt;                              // compact scratch rows (no layer transforms before a max)
+    RP_LAUNCH(c, k_max_long_begin, c->n_sm * 2, 256, 0, c->ctl, mode, long_rows, n_long, c->side[1], ld, S, saved,
+              c->invmask, c->mw, is_min, items, n_items);
+#define CHUNKS(NV) RP_LAUNCH(c, k_max_long_chunks<NV>, c->n_sm * 8, 256, 0, c->ctl, mode, long_rows, items, n_items, c->side[1], M, ld, S, c->invmask, c->mw, is_min)
+    if (nv <= 1) CHUNKS(1); else if (nv <= 2) CHUNKS(2); else if (nv <= 4) CHUNKS(4); else CHUNKS(8);
+#undef CHUNKS
+    if (mode)
+        RP_LAUNCH(c, k_max_long_end, c->n_sm * 2, 256, 0, c->ctl, long_rows, n_long, ld, S, saved, c->bitmap,
+                  c->invmask, c->mw);
 }
 
 // bootstrap: S^l_v for every vertex
@@ -496,7 +532,7 @@ void max_full(Ctx* c, int l) {
 #define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 16, 256, 0, c->ctl, l, 0, (const int32_t*)nullptr, (const int*)nullptr, c->N, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
     RP_WIDTH_DISPATCH(ld, ROWS);
 #undef ROWS
-    launch_long_rows(c, 0, c->H[l - 1], ld, c->S[l], long_rows, n_long);
+    launch_long_rows(c, l, 0, c->H[l - 1], ld, c->S[l], long_rows, n_long);
 }
 
 // hop l of a batch: messages, recomputation of the invalidated sinks, the list A_l
@@ -522,7 +558,7 @@ void max_hop(Ctx* c, int l, int n) {
 #define ROWS(NV, LPR) RP_LAUNCH(c, (k_max_rows<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, 1, rlist, n_r, 0, c->side[1], c->H[l - 1], ld, c->S[l], c->bitmap, long_rows, n_long, c->invmask, c->mw, (int)(c->agg == RIPPLE_AGG_MIN))
     RP_WIDTH_DISPATCH(ld, ROWS);
 #undef ROWS
-    launch_long_rows(c, 1, c->H[l - 1], ld, c->S[l], long_rows, n_long);
+    launch_long_rows(c, l, 1, c->H[l - 1], ld, c->S[l], long_rows, n_long);
     if (c->self_term) RP_LAUNCH(c, k_max_mark_self, c->n_sm * 2, T, 0, c->ctl, l, senders, c->bitmap);
 }
 
@@ -534,8 +570,6 @@ void max_senders_build(Ctx* c, int l) {
     scan_degrees(c, senders, &c->ctl->nC[l], 0, c->side[0].deg, c->coff, &c->ctl->E[l + 1]);
 }
 
-void max_prepare() {
-    cudaFuncSetAttribute(k_max_long_rows<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 8 * 1024 * (int)sizeof(float));
-}
+void max_prepare() {}
 
 }  // namespace rp

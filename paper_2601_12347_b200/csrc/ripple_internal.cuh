@@ -56,6 +56,7 @@ struct Ctl {
     int n_long[RP_MAXL + 1];          // bottom-up marking: vertices whose long in-list is scanned by a warp
     int n_rebuilt[RP_MAXL + 1];       // aggregate rows of hop l gathered anew because their rounding budget ran out
     int rebuild_items[RP_MAXL + 1];   // (vertex, chunk) work items of the long rows among them
+    int max_items[RP_MAXL + 1];       // max / min: (long row, chunk) work items of hop l's recomputation
     long long num_edges;              // current edge count (kept across batches)
     int work_counter[8];              // dynamic work distribution tickets (reset by the consumer)
 };
