@@ -314,11 +314,15 @@ def run_ours(args, rank, world, local_rank):
     h2d = d2h = 0
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ids_host = torch.empty(w.n, dtype=torch.int32).pin_memory()   # the read-out lands in pinned memory, like the inputs
     e0.record(st)
     for u, r, ow in pin_batches:
         t0 = time.perf_counter()
         rp.apply_batch(u, r, ow)
-        ids = rp.affected(L).cpu()        # trigger-style read-out: who changed at the last layer
+        dev_ids = rp.affected(L)          # trigger-style read-out: who changed at the last layer
+        ids = ids_host[: dev_ids.numel()]
+        ids.copy_(dev_ids, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
         lat.append(time.perf_counter() - t0)
         h2d += u.numel() * 4 + r.numel() * 4 + (ow.numel() * 4 if ow is not None else 0)
         d2h += ids.numel() * 4
