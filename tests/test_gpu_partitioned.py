@@ -145,3 +145,66 @@ def test_partitioned_context_refuses_what_it_cannot_do(env):
     model = I.graphconv_model([18, 36, 10], I.AGG_MAX)
     with pytest.raises(ripple.RippleError):
         Cluster(2, owner, src, dst, X, model, I.make_weights(model, 1))
+
+
+# ---------------------------------------------------------------------------------------------
+# one worker per process: CUDA IPC mappings of the peers' buffers, barriers between the phases.  Both
+# processes use the one GPU of the test box; their kernels never wait for each other (every phase call
+# returns when its device work is done, the barrier is on the host).
+# ---------------------------------------------------------------------------------------------
+def _ipc_rank(rank, world, port, out):
+    import datetime
+    import os
+    import torch
+    import torch.distributed as dist
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world, timeout=datetime.timedelta(seconds=120))
+    torch.cuda.set_device(0)
+    from oracle.oracle import Oracle
+    from paper_2601_12347_b200.partitioned import DistributedWorker
+    n = 600
+    model = I.sage_model([18, 36, 10], I.AGG_MEAN)
+    src, dst = I.er_graph(n, 4000, 13)
+    X = I.features(n, 18, 13)
+    W = I.make_weights(model, 13, zero_bias=False)
+    owner = np.random.default_rng(13).integers(0, world, size=n).astype(np.int32)
+    dw = DistributedWorker(owner, src, dst, X, model, W)
+    orc = Oracle(n, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, 18, 13)
+    sent = 0
+    for _ in range(6):
+        ups, rows = stream.next_batch(40)
+        dw.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        sent += sum(dw.worker.rows_sent())
+    full = orc.full()
+    nl = dw.worker.n_local
+    gof = np.array([dw.router.global_id(rank, i) for i in range(nl)])
+    worst = 0.0
+    for l in range(3):
+        h = dw.worker.embeddings(l).cpu().numpy()[:nl][gof >= 0].astype(np.float64)
+        ref = full[l][gof[gof >= 0]]
+        worst = max(worst, float(np.max(np.abs(h - ref) / (1.0 + np.abs(ref)))))
+    mine = sorted(gof[dw.worker.affected(2).cpu().numpy()].tolist())
+    out[rank] = (worst, int((gof >= 0).sum()), sent, mine, orc.affected(2).tolist())
+    dist.barrier()
+    dw.close()
+    dist.destroy_process_group()
+
+
+def test_one_worker_per_process_with_ipc_mappings(env):
+    import socket
+    import torch.multiprocessing as mp
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    world = 2
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_ipc_rank, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    assert sum(res[r][1] for r in range(world)) == 600
+    assert all(res[r][0] <= TOL for r in range(world)), [res[r][0] for r in range(world)]
+    assert all(res[r][2] > 0 for r in range(world))                      # rows did cross between the processes
+    assert sorted(res[0][3] + res[1][3]) == res[0][4]                      # the union of the hop sets is the oracle's
