@@ -162,8 +162,11 @@ ripple_status ripple_router_batch_fill(ripple_router* r, int32_t rank, ripple_up
                                        int32_t* row_of, int32_t* first_halo, int32_t* halo_owner,
                                        int32_t* halo_remote_id);
 
-/* Look-ups: owner and local id of a global vertex (-1: not placed); the global id behind a local id of
- * a worker (-1: unused); whether v is in the high in-degree set; vertices placed on a worker. */
+/* Look-ups: the global id behind every local id of a worker as of now (global_of: HOST, capacity >= the
+ * worker's num_vertices entries, -1 for unused ids); owner and local id of a global vertex (-1: not placed);
+ * the global id behind one local id of a worker (-1: unused); whether v is in the high in-degree set;
+ * vertices placed on a worker. */
+ripple_status ripple_router_global_ids(ripple_router* r, int32_t rank, int32_t* global_of, int64_t capacity);
 int32_t ripple_router_owner(ripple_router* r, int32_t v);
 int32_t ripple_router_local_id(ripple_router* r, int32_t v);
 int32_t ripple_router_global_id(ripple_router* r, int32_t rank, int32_t local_id);

@@ -269,6 +269,14 @@ extern "C" ripple_status ripple_router_batch_fill(ripple_router* r, int32_t rank
     return RIPPLE_OK;
 }
 
+extern "C" ripple_status ripple_router_global_ids(ripple_router* r, int32_t rank, int32_t* global_of, int64_t capacity) {
+    if (!r || rank < 0 || rank >= r->P || !global_of) return RIPPLE_ERR_INVALID_ARG;
+    const Part& q = r->part[rank];
+    if (capacity < (int64_t)q.global_of.size()) return RIPPLE_ERR_CAPACITY;
+    std::copy(q.global_of.begin(), q.global_of.end(), global_of);
+    return RIPPLE_OK;
+}
+
 extern "C" int32_t ripple_router_owner(ripple_router* r, int32_t v) {
     return (r && v >= 0 && v < r->N) ? r->owner[v] : -1;
 }

@@ -98,6 +98,14 @@ class Router:
             raise R.RippleError(st, "batch fill")
         return ups[: a.value], nc[: a.value], row_of[: b.value], first.value, ho[: c.value], hr[: c.value]
 
+    def global_ids(self, rank: int, num_vertices: int) -> np.ndarray:
+        """The global id behind every local id of worker `rank` (locals, then halo slots; -1: unused)."""
+        out = np.zeros(int(num_vertices), dtype=np.int32)
+        st = self.lib.ripple_router_global_ids(self.h, int(rank), out.ctypes.data, out.size)
+        if st != R.OK:
+            raise R.RippleError(st, "global ids")
+        return out
+
     def owner(self, v: int) -> int:
         return int(self.lib.ripple_router_owner(self.h, int(v)))
 
@@ -233,17 +241,16 @@ class Cluster:
         out = np.zeros((n, d), dtype=np.float32)
         for r, w in enumerate(self.workers):
             nl = w_n_local(w)
-            gof = np.array([self.router.global_id(r, i) for i in range(nl)], dtype=np.int64)
-            h = w.embeddings(l).cpu().numpy()[:nl]
+            gof = self.router.global_ids(r, w.n)[:nl].astype(np.int64)
+            h = w.embeddings(l)[:nl].cpu().numpy()
             out[gof[gof >= 0]] = h[gof >= 0]
         return out
 
     def affected(self, l: int) -> np.ndarray:
         ids = []
         for r, w in enumerate(self.workers):
-            a = w.affected(l).cpu().numpy()
-            ids += [self.router.global_id(r, int(i)) for i in a]
-        return np.array(sorted(ids), dtype=np.int32)
+            ids.append(self.router.global_ids(r, w.n)[w.affected(l).cpu().numpy()])
+        return np.sort(np.concatenate(ids)).astype(np.int32)
 
     def rows_sent(self) -> List[int]:
         tot = np.zeros(self.L + 1, dtype=np.int64)

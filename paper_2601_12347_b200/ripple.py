@@ -35,13 +35,13 @@ EXPORTED = [
     "ripple_export_graph_static", "ripple_set_timing", "ripple_probe_reduction_rate", "ripple_probe_gather_rate",
     "ripple_get_stats", "ripple_last_error", "ripple_destroy", "ripple_version",
 ]
-# partitioned execution (include/ripple_part.h); all but the last six return a status
+# partitioned execution (include/ripple_part.h); the first 18 return a status
 EXPORTED_PART = [
     "ripple_part_exports_get", "ripple_part_set_peer", "ripple_part_ipc_export", "ripple_part_ipc_open",
     "ripple_part_set_halos", "ripple_part_bootstrap_layer", "ripple_part_begin", "ripple_part_hop_send",
     "ripple_part_hop_compute", "ripple_part_end", "ripple_part_rows_sent",
     "ripple_router_create", "ripple_router_partition_shape", "ripple_router_partition_fill",
-    "ripple_router_route", "ripple_router_batch_shape", "ripple_router_batch_fill",
+    "ripple_router_route", "ripple_router_batch_shape", "ripple_router_batch_fill", "ripple_router_global_ids",
     "ripple_router_destroy", "ripple_router_owner", "ripple_router_local_id", "ripple_router_global_id",
     "ripple_router_is_high_degree", "ripple_router_load",
 ]
@@ -164,7 +164,8 @@ def load_library(path: Optional[str] = None):
     lib.ripple_router_route.argtypes = [vp, vp, i64]
     lib.ripple_router_batch_shape.argtypes = [vp, i32, P(i64), P(i64), P(i64)]
     lib.ripple_router_batch_fill.argtypes = [vp, i32, vp, vp, vp, P(i32), vp, vp]
-    for name in EXPORTED_PART[:17]:
+    lib.ripple_router_global_ids.argtypes = [vp, i32, vp, i64]
+    for name in EXPORTED_PART[:18]:
         getattr(lib, name).restype = i32
     lib.ripple_router_destroy.argtypes = [vp]
     lib.ripple_router_destroy.restype = None

@@ -270,3 +270,41 @@ def test_full_size_batches_of_1000_structure_and_sampled_rows(env, wname, n_batc
     assert np.array_equal(H[0], X_now)
     rp.close()
     orc.close()
+
+
+def test_full_size_two_workers_of_the_partitioned_execution(env):
+    """dense-2l split over two workers (uniformly random owners: the worst cut) on the one GPU: hop sets
+    exact against the oracle's structure route after every batch, sampled rows of the gathered embeddings
+    against the definition."""
+    ripple, Oracle = env
+    from paper_2601_12347_b200.partitioned import Cluster
+    wname = "dense-2l"
+    w, (src, dst) = graph_of(wname)
+    X = I.features(w.n, w.model.dims[0], w.seed)
+    W = I.make_weights(w.model, w.seed)
+    L = len(w.model.layers)
+    owner = np.random.default_rng(w.seed).integers(0, 2, size=w.n).astype(np.int32)
+    cl = Cluster(2, owner, src, dst, X, w.model, W, max_batch=1000)
+    orc = Oracle(w.n, src, dst, X, w.model, W, bootstrap=False)
+    stream = I.make_stream(w, src, dst)
+    for b in range(3):
+        ups, rows = stream.next_batch(1000)
+        cl.apply_batch(ups, rows)
+        assert orc.apply_structure(ups, rows.shape[0]) == 0
+        for l in range(L + 1):
+            assert np.array_equal(cl.affected(l), orc.affected(l)), f"batch {b}: A_{l} differs"
+    sent = cl.rows_sent()
+    assert sent[L] > 100_000, sent
+    H = [np.ascontiguousarray(cl.embeddings(l, w.n)) for l in range(L + 1)]
+    ids, odi = sample_rows(np.random.default_rng(0), w, orc, L, ups)
+    worst = 0.0
+    for l in range(1, L + 1):
+        _, ref = orc.rows_from_prev(l, ids, H[l - 1])
+        err = np.max(np.abs(H[l][ids].astype(np.float64) - ref) / (1.0 + np.abs(ref)), axis=1)
+        i = int(np.argmax(err))
+        assert err[i] <= TOL, f"layer {l}, vertex {ids[i]} (in-degree {odi[ids[i]]}): err {err[i]}"
+        worst = max(worst, float(err[i]))
+    print(f"dense-2l over 2 workers after 3 batches of 1000: {ids.size} sampled rows x {L} layers, worst err {worst:.2e}, "
+          f"halo rows sent in the last batch {sent[1:]}")
+    cl.close()
+    orc.close()
