@@ -290,6 +290,17 @@ ripple_status ripple_export_graph_weighted(ripple_ctx* ctx, int64_t* rowptr, int
  * col HOST, col_capacity >= number of edges, ascending within each row. */
 ripple_status ripple_export_graph_static(ripple_ctx* ctx, int64_t* rowptr, int32_t* col, int64_t col_capacity);
 
+/* Vertex addition beyond the ids the context was created with (Sec. 3.2, Sec. 4.1: a vertex arrives with
+ * the edge addition that first names it): raises the id capacity to num_vertices.  The new ids are isolated
+ * vertices with zero feature rows; their embeddings are those full inference gives an isolated vertex
+ * (the activation of the bias, layer by layer), everything else keeps its bits.  Every device array that
+ * has a row per vertex is re-allocated and copied: pointers obtained earlier from ripple_get_embeddings,
+ * ripple_get_aggregate, ripple_get_affected and ripple_get_degrees are invalid afterwards, captured launch
+ * chains are dropped, and the call costs a copy of the whole state -- reserve in large steps.
+ * INVALID_ARG if num_vertices is not larger than the present capacity or the context is a worker of a
+ * partitioned execution; OOM leaves the context unusable (destroy it). */
+ripple_status ripple_reserve_vertices(ripple_ctx* ctx, int64_t num_vertices);
+
 /* Degree arrays of the current graph: DEVICE, N entries each. */
 ripple_status ripple_get_degrees(ripple_ctx* ctx, const int32_t** deg_out, const int32_t** deg_in);
 

@@ -748,6 +748,129 @@ extern "C" ripple_status ripple_recompute_full(ripple_ctx* ctx) {
     return run_full(c);
 }
 
+// ---------------------------------------------------------------------------------------------
+// growing the vertex set
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+static cudaError_t grow_array(T** p, size_t old_count, size_t new_count, int fill_byte) {
+    if (!*p) return cudaSuccess;
+    T* q = nullptr;
+    cudaError_t e = cudaMalloc(&q, sizeof(T) * std::max<size_t>(new_count, 1));
+    if (e) return e;
+    if ((e = cudaMemset(q, fill_byte, sizeof(T) * new_count))) return e;
+    if ((e = cudaMemcpy(q, *p, sizeof(T) * std::min(old_count, new_count), cudaMemcpyDeviceToDevice))) return e;
+    cudaFree(*p);
+    *p = q;
+    return cudaSuccess;
+}
+
+// ids first .. first + count - 1 into every list a hop reads (A_l, the two sender lists), and their number
+// into the control block: the new vertices are then rows of every hop's update
+__global__ void k_list_new_vertices(Ctl* ctl, int L, int first, int count, int32_t* const* lists, int n_lists) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < count; i += gridDim.x * blockDim.x)
+        for (int k = 0; k < n_lists; ++k) lists[k][i] = first + i;
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        for (int l = 0; l <= L; ++l) { ctl->nA[l] = count; ctl->nC[l] = count; }
+}
+
+extern "C" ripple_status ripple_reserve_vertices(ripple_ctx* ctx, int64_t num_vertices) {
+    Ctx* c = reinterpret_cast<Ctx*>(ctx);
+    if (!c) return RIPPLE_ERR_INVALID_ARG;
+    if (c->n_local > 0 || num_vertices <= c->N || num_vertices > 0x7fffffff - 64) {
+        set_err(c, "ripple_reserve_vertices: %lld is not above the present capacity %d (or the context is a worker of a partitioned execution)",
+                (long long)num_vertices, c->N);
+        return RIPPLE_ERR_INVALID_ARG;
+    }
+    cudaSetDevice(c->device);
+    ripple_status st = RIPPLE_OK;
+    const size_t N0 = (size_t)c->N, N1 = (size_t)num_vertices;
+    const int L = c->L;
+    int max_ld = 0, max_hid = 0;
+    for (int l = 0; l <= L; ++l) max_ld = std::max(max_ld, c->ld[l]);
+    for (int l = 1; l <= L; ++l) if (c->layer[l].kind == RIPPLE_LAYER_GIN) max_hid = std::max(max_hid, c->layer[l].ld_hid);
+    CK(cudaStreamSynchronize(c->stream));
+    for (auto& g : c->graph_exec) if (g) { cudaGraphExecDestroy(g); g = nullptr; }   // captured chains hold the old addresses
+    memset(c->graph_n, 0, sizeof(c->graph_n));
+    memset(c->seen_key, 0, sizeof(c->seen_key));
+    memset(c->seen_count, 0, sizeof(c->seen_count));
+    for (int l = 0; l <= L; ++l) {
+        CK(grow_array(&c->H[l], N0 * c->ld[l], N1 * c->ld[l], 0));
+        CK(grow_array(&c->A[l], N0 + 32, N1 + 32, 0));
+        if (!l) continue;
+        CK(grow_array(&c->S[l], N0 * c->ws[l], N1 * c->ws[l], 0));
+        CK(grow_array(&c->dS[l], N0 * c->ws[l], N1 * c->ws[l], 0));
+        CK(grow_array(&c->Eb[l], N0, N1, 0));
+        CK(grow_array(&c->Z[l], N0 * c->ld[l], N1 * c->ld[l], 0));
+        CK(grow_array(&c->P[l], N0 * c->ws[l], N1 * c->ws[l], 0));
+        CK(grow_array(&c->att_s[l], N0, N1, 0));
+        CK(grow_array(&c->att_t[l], N0, N1, 0));
+    }
+    CK(grow_array(&c->T, N0 * max_hid, N1 * max_hid, 0));
+    CK(grow_array(&c->Dt, N0 * max_ld, N1 * max_ld, 0));
+    for (int s = 0; s < 2; ++s) {
+        CK(grow_array(&c->D[s], N0 * max_ld, N1 * max_ld, 0));
+        CK(grow_array(&c->Clist[s], N0 + 32, N1 + 32, 0));
+        Side& sd = c->side[s];
+        CK(grow_array(&sd.start, N0 + 1, N1 + 1, 0));   // a new row is empty: capacity 0, its first edge takes a block of the pool
+        for (int32_t** a : {&sd.cap, &sd.deg, &sd.cnt_del, &sd.cnt_add, &sd.tick_a, &sd.tick_b, &sd.touch}) CK(grow_array(a, N0, N1, 0));
+    }
+    CK(grow_array(&c->att_so, N0 + 32, N1 + 32, 0));
+    if (c->att_items) CK(grow_array(&c->att_items, N0 + (size_t)(c->side[1].col_size / 256) + 64, N1 + (size_t)(c->side[1].col_size / 256) + 64, 0));
+    {
+        const size_t other = (size_t)(c->side[1].col_size / 128) + 64;
+        CK(grow_array(&c->coff, std::max(N0 + 2, other), std::max(N1 + 2, other), 0));
+    }
+    {
+        const size_t w0 = (size_t)c->n_words + 256, w1 = (N1 + 31) / 32 + 256;
+        CK(grow_array(&c->bitmap, w0, w1, 0));
+        CK(grow_array(&c->bitmap2, w0, w1, 0));
+    }
+    CK(grow_array(&c->old_idx, N0 + 32, N1 + 32, 0));
+    CK(grow_array(&c->invmask, N0 * c->mw, N1 * c->mw, 0));
+    CK(grow_array(&c->posmap, N0, N1, 0xFF));
+    CK(grow_array(&c->deg_out_old, N0, N1, 0xFF));
+    CK(grow_array(&c->feat_last, N0, N1, 0xFF));
+    CK(grow_array(&c->vdel_seq, N0, N1, 0xFF));
+    {
+        const int nt = std::max(div_up((int64_t)N1, 1024) + 2, div_up((int64_t)((N1 + 31) / 32), 256) + 2);
+        CK(grow_array(&c->tile_sums, (size_t)c->n_tile_sums, (size_t)nt, 0));
+        c->n_tile_sums = nt;
+    }
+    c->N = (int)N1;
+    c->n_words = (int)((N1 + 31) / 32);
+    {
+        // embeddings of the new, isolated vertices: every layer's update (and the cached projections it reads)
+        // run over exactly those rows; their aggregates are zero already
+        const int first = (int)N0, count = (int)(N1 - N0);
+        std::vector<int32_t*> lists;
+        for (int l = 0; l <= L; ++l) lists.push_back(c->A[l]);
+        lists.push_back(c->Clist[0]);
+        lists.push_back(c->Clist[1]);
+        int32_t** lists_dev = nullptr;
+        CK(cudaMalloc(&lists_dev, sizeof(int32_t*) * lists.size()));
+        CK(cudaMemcpy(lists_dev, lists.data(), sizeof(int32_t*) * lists.size(), cudaMemcpyHostToDevice));
+        c->launches = 0;
+        c->debug_tc_withhold = 0;
+        c->tc_armed = 1;
+        c->params_host[0] = 0; c->params_host[1] = 0;
+        cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream);
+        RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
+        k_list_new_vertices<<<std::min(div_up(count, 256), c->n_sm * 4), 256, 0, c->stream>>>(c->ctl, L, first, count, lists_dev, (int)lists.size());
+        for (int l = 1; l <= L && !c->attention; ++l) {   // (attention: an isolated vertex outputs zeros and its logit halves are zero)
+            if (c->pre[l]) sender_transform(c, l);
+            self_project(c, l, false);
+            update_rows(c, l, false);
+        }
+        RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
+        st = sync_and_fetch_ctl(c);
+        cudaFree(lists_dev);
+        if (st) return st;
+    }
+    return RIPPLE_OK;
+fail:
+    return st;
+}
+
 extern "C" ripple_status ripple_get_stats(ripple_ctx* ctx, ripple_stats* out) {
     Ctx* c = reinterpret_cast<Ctx*>(ctx);
     if (!c || !out) return RIPPLE_ERR_INVALID_ARG;

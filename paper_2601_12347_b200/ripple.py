@@ -31,7 +31,7 @@ UPDATE_DTYPE = np.dtype([("op", "<i4"), ("u", "<i4"), ("v", "<i4")])
 EXPORTED = [
     "ripple_create", "ripple_apply_batch", "ripple_apply_batch_weighted", "ripple_get_embeddings",
     "ripple_get_aggregate", "ripple_get_affected", "ripple_export_graph", "ripple_export_graph_weighted",
-    "ripple_get_degrees", "ripple_recompute_full",
+    "ripple_get_degrees", "ripple_recompute_full", "ripple_reserve_vertices",
     "ripple_export_graph_static", "ripple_set_timing", "ripple_probe_reduction_rate", "ripple_probe_gather_rate",
     "ripple_get_stats", "ripple_last_error", "ripple_destroy", "ripple_version",
 ]
@@ -144,7 +144,8 @@ def load_library(path: Optional[str] = None):
     lib.ripple_set_timing.argtypes = [vp, i32]
     lib.ripple_probe_reduction_rate.argtypes = [i32, i64, i32, i64, i32, P(ctypes.c_float)]
     lib.ripple_probe_gather_rate.argtypes = [i32, i64, i32, i64, P(ctypes.c_float)]
-    for name in EXPORTED[:15]:
+    lib.ripple_reserve_vertices.argtypes = [vp, i64]
+    for name in EXPORTED[:16]:
         getattr(lib, name).restype = i32
     # partitioned execution
     lib.ripple_part_exports_get.argtypes = [vp, P(_PartExports)]
@@ -339,6 +340,12 @@ class Ripple:
 
     def set_timing(self, on: bool) -> None:
         self._check(self.lib.ripple_set_timing(self.h, int(bool(on))))
+
+    def reserve_vertices(self, n: int) -> None:
+        """Raises the id capacity to n: the new ids are isolated vertices with zero features.  Views
+        obtained earlier (embeddings, aggregate, affected, degrees) are invalid afterwards."""
+        self._check(self.lib.ripple_reserve_vertices(self.h, int(n)))
+        self.n = int(n)
 
     def recompute_full(self) -> None:
         self._check(self.lib.ripple_recompute_full(self.h))

@@ -176,3 +176,69 @@ def test_all_five_update_types_100_consecutive_batches(env, batch):
     G.check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
     assert rp.stats()["num_edges"] == stream.n_edges
     rp.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# growing the vertex set (ripple_reserve_vertices)
+# ---------------------------------------------------------------------------------------------
+def _reserve_models():
+    return {
+        "sage_mean": I.sage_model([18, 36, 10], I.AGG_MEAN),
+        "gc_sum_3l": I.graphconv_model([18, 36, 20, 10], I.AGG_SUM),     # no self term: an isolated vertex still has act(bias) rows
+        "gcn_wsum": I.graphconv_model([18, 36, 10], I.AGG_WSUM_GCN),
+        "gin": I.gin_model(18, 24, 2, eps=0.25),
+        "gc_max": I.graphconv_model([18, 36, 10], I.AGG_MAX),
+        "gat": I.gat_model(20, 2, d_att=4, slope=0.2),
+        "sage_wide": I.sage_model([40, 160, 24], I.AGG_MEAN),
+    }
+
+
+@pytest.mark.parametrize("name", list(_reserve_models().keys()))
+def test_reserved_vertices_are_isolated_vertices_and_can_be_attached(env, name):
+    ripple, Oracle = env
+    model = _reserve_models()[name]
+    L = len(model.layers)
+    n, spare = 500, 70
+    src, dst = I.er_graph(n, 3500, 17)
+    X = I.features(n + spare, model.dims[0], 17)
+    X[n:] = 0
+    W = I.make_weights(model, 17, zero_bias=False)
+    rp = ripple.Ripple(n, src, dst, X[:n], model, W)
+    orc = Oracle(n + spare, src, dst, X, model, W)          # the oracle has had the ids all along, as isolated vertices
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 17)
+    for _ in range(3):                                       # same size three times: a captured chain exists before the growth
+        ups, rows = stream.next_batch(20)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+    before = [rp.embeddings(l).clone() for l in range(L + 1)]
+    with pytest.raises(ripple.RippleError):
+        rp.reserve_vertices(n)
+    rp.reserve_vertices(n + spare)
+    full = orc.full()
+    for l in range(L + 1):
+        got = rp.embeddings(l)
+        assert got.shape[0] == n + spare
+        assert bool((got[:n] == before[l]).all()), "rows of the old vertices changed"
+    G.check_values(rp, full, L)
+    rng = np.random.default_rng(3)
+    nxt = n
+    for b in range(6):
+        ups, rows = stream.next_batch(20)
+        extra = G.ups_array([(I.OP_ADD_EDGE, nxt, int(rng.integers(0, n))), (I.OP_ADD_EDGE, int(rng.integers(0, n)), nxt + 1),
+                             (I.OP_ADD_EDGE, nxt + 2, nxt + 3), (I.OP_SET_FEATURE, nxt, rows.shape[0]),
+                             (I.OP_ADD_EDGE, nxt + 1, nxt)])
+        nxt += 4
+        ups = np.concatenate([ups, extra])
+        rows = np.concatenate([rows, I.features(1, model.dims[0], 200 + b)])
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        G.check_frontiers(rp, orc, L)
+    rowptr, col = rp.export_graph()
+    orp, ocol = orc.export_csr()
+    assert np.array_equal(rowptr, orp) and np.array_equal(col, ocol)
+    G.check_values(rp, orc.full(), L)
+    rp.reserve_vertices(n + spare + 33)                      # once more, to a capacity that is no multiple of 32
+    assert rp.embeddings(L).shape[0] == n + spare + 33
+    rp.apply_batch(G.ups_array([(I.OP_ADD_EDGE, n + spare + 32, 0)]))
+    assert rp.stats()["n_added"] == 1
+    rp.close()
