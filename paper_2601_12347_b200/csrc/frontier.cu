@@ -303,6 +303,75 @@ void frontier_mark(Ctx* c, int l, bool walk, int n) {
               &c->ctl->n_long[l]);
 }
 
+// The frontier of a hop in one block: words of the bitmap are dealt out in contiguous runs, one per thread, so
+// that a block scan of the popcounts places every id.  For batches of a handful of updates on graphs whose
+// bitmap one block can sweep (two launches of the general chain otherwise).
+__global__ void __launch_bounds__(1024)
+k_frontier_small(Ctl* ctl, int l, uint32_t* bitmap, int n_words, int32_t* list, const int32_t* __restrict__ deg_in) {
+    pdl_enter();
+    __shared__ int scratch_i[33];
+    __shared__ unsigned long long s_work;
+    if (ctl->abort) return;
+    if (threadIdx.x == 0) s_work = 0ull;
+    const int per = (n_words + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int w0 = min(n_words, (int)threadIdx.x * per), w1 = min(n_words, w0 + per);
+    int pc = 0;
+    for (int w = w0; w < w1; ++w) pc += __popc(bitmap[w]);
+    int total;
+    int off = block_exclusive_scan<int>(pc, scratch_i, total);
+    unsigned long long work = 0;
+    for (int w = w0; w < w1; ++w) {
+        uint32_t bits = bitmap[w];
+        if (!bits) continue;
+        bitmap[w] = 0u;
+        while (bits) {
+            const int v = (w << 5) + __ffs(bits) - 1;
+            bits &= bits - 1;
+            list[off++] = v;
+            work += (unsigned long long)deg_in[v];
+        }
+    }
+    work = warp_sum(work);
+    if (lane_id() == 0 && work) atomicAdd(&s_work, work);
+    __syncthreads();
+    if (threadIdx.x == 0) { ctl->nA[l] = total; ctl->pull_work[l] = s_work; }
+}
+
+// ... and the sender list made from it (C_l = A_l) with the prefix of the out-degrees, likewise in one block
+__global__ void __launch_bounds__(1024)
+k_senders_small(Ctl* ctl, int l, const int32_t* __restrict__ list, const int32_t* __restrict__ deg_out, int32_t* senders,
+                int32_t* posmap, int64_t* coff) {
+    pdl_enter();
+    __shared__ int64_t scratch_l[33];
+    if (ctl->abort) return;
+    const int total = ctl->nA[l];
+    int64_t carry = 0;
+    for (int i0 = 0; i0 < total; i0 += (int)blockDim.x) {
+        const int i = i0 + (int)threadIdx.x;
+        int v = -1;
+        int64_t d = 0;
+        if (i < total) { v = list[i]; d = deg_out[v]; }
+        int64_t sum;
+        const int64_t ex = block_exclusive_scan<int64_t>(d, scratch_l, sum);
+        if (i < total) { senders[i] = v; posmap[v] = i; coff[i] = carry + ex; }
+        carry += sum;
+    }
+    if (threadIdx.x == 0) {
+        coff[total] = carry;
+        ctl->E[l + 1] = (unsigned long long)carry;
+        ctl->nC[l] = total;
+    }
+}
+
+void frontier_compact_small(Ctx* c, int l) {
+    RP_LAUNCH(c, k_frontier_small, 1, 1024, 0, c->ctl, l, c->bitmap, c->n_words, c->A[l], (const int32_t*)c->side[1].deg);
+}
+
+void senders_build_small(Ctx* c, int l) {
+    RP_LAUNCH(c, k_senders_small, 1, 1024, 0, c->ctl, l, (const int32_t*)c->A[l], (const int32_t*)c->side[0].deg,
+              c->Clist[l & 1], c->posmap, c->coff);
+}
+
 void frontier_compact(Ctx* c, int l) {
     bitmap_to_list(c, c->A[l], &c->ctl->nA[l], &c->ctl->pull_work[l]);
 }

@@ -163,10 +163,9 @@ __global__ void k_expand_copy(ripple_update* ups, int32_t* op_seq, Ctl* ctl, Sid
     }
 }
 
-__global__ void k_classify(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, int N,
-                           Ctl* ctl, unsigned long long* hkeys, unsigned long long* hwin, int hmask,
-                           int32_t* op_slot, int32_t* feat_last, int32_t* vdel_seq) {
-    pdl_enter();
+__device__ __forceinline__ void d_classify(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, int N,
+                                           Ctl* ctl, unsigned long long* hkeys, unsigned long long* hwin, int hmask,
+                                           int32_t* op_slot, int32_t* feat_last, int32_t* vdel_seq) {
     const int n = ops_total(ctl), n_given = ctl->n_ops;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
         ripple_update op = ups[i];
@@ -215,6 +214,13 @@ __global__ void k_classify(const ripple_update* __restrict__ ups, const int32_t*
     }
 }
 
+__global__ void k_classify(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, int N,
+                           Ctl* ctl, unsigned long long* hkeys, unsigned long long* hwin, int hmask,
+                           int32_t* op_slot, int32_t* feat_last, int32_t* vdel_seq) {
+    pdl_enter();
+    d_classify(ups, op_seq, N, ctl, hkeys, hwin, hmask, op_slot, feat_last, vdel_seq);
+}
+
 // Position of x in row [base, base + deg), or -1; the whole block calls this.  Rows start on
 // 16-byte boundaries, so every thread compares four entries per load; a hub row of 150 K entries
 // costs a block of 256 threads about 150 iterations.
@@ -251,13 +257,12 @@ __device__ __forceinline__ void d_plan_check(Ctl* ctl, Side out, Side in);
 // An explicit edge operation that precedes the deletion of one of its endpoints is superseded by
 // it (for stored edges the generated deletion already wins the slot; for pairs that are not stored
 // nothing was generated, hence the explicit test).  Only the caller's operations are counted.
-__global__ void __launch_bounds__(256)
-k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, Ctl* ctl,
+__device__ __forceinline__ void
+d_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, Ctl* ctl,
           const unsigned long long* __restrict__ hwin, const int32_t* __restrict__ op_slot,
           const int32_t* __restrict__ feat_last, const int32_t* __restrict__ vdel_seq, Side out, Side in,
           Rec* rec, uint32_t* bitmap, const float* __restrict__ op_w, int32_t* grow_out, int32_t* grow_in,
           int32_t* shrink_out, int32_t* shrink_in, const uint8_t* __restrict__ silent) {
-    pdl_enter();
     __shared__ int s_found;
     __shared__ int s_last;
     if (ctl->abort) return;
@@ -315,6 +320,17 @@ k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) d_plan_check(ctl, out, in);
+}
+
+__global__ void __launch_bounds__(256)
+k_resolve(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, Ctl* ctl,
+          const unsigned long long* __restrict__ hwin, const int32_t* __restrict__ op_slot,
+          const int32_t* __restrict__ feat_last, const int32_t* __restrict__ vdel_seq, Side out, Side in,
+          Rec* rec, uint32_t* bitmap, const float* __restrict__ op_w, int32_t* grow_out, int32_t* grow_in,
+          int32_t* shrink_out, int32_t* shrink_in, const uint8_t* __restrict__ silent) {
+    pdl_enter();
+    d_resolve(ups, op_seq, ctl, hwin, op_slot, feat_last, vdel_seq, out, in, rec, bitmap, op_w, grow_out, grow_in,
+              shrink_out, shrink_in, silent);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -658,6 +674,102 @@ k_mutate_small(Ctl* ctl, Rec* rec, Side out, Side in, const int32_t* __restrict_
     d_add_write(ctl, rec, out, in);
     __syncthreads();
     d_commit_degrees(ctl, rec, out, in, deg_out_old, moved_start, moved_cap);
+}
+
+// A batch of a handful of updates, none of them a vertex deletion, for models whose hop-0 senders are exactly
+// the vertices with a feature update: control block reset, classification, resolution and planning, the row
+// update, the list A_0 (sorted in shared memory from the winning feature operations: no sweep of the
+// frontier bitmap), the feature rows with their old values or deltas, and the sender list of hop 1 with its
+// out-degree prefix -- nine launches of the general chain -- in one block with barriers in between.
+__global__ void __launch_bounds__(1024)
+k_apply_small(Ctl* ctl, const int* params, const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, int N,
+              unsigned long long* hkeys, unsigned long long* hwin, int hmask, int32_t* op_slot, int32_t* feat_last,
+              int32_t* vdel_seq, Side out, Side in, Rec* rec, uint32_t* bitmap, const float* __restrict__ op_w,
+              int32_t* grow_out, int32_t* grow_in, int32_t* shrink_out, int32_t* shrink_in, int64_t* moved_start,
+              int32_t* moved_cap, int32_t* deg_out_old, const float* __restrict__ feat, int d0, float* H0, int ld,
+              float* D, int keep_old, int32_t* A0, int32_t* senders, int32_t* posmap, int64_t* coff) {
+    pdl_enter();
+    __shared__ int s_ids[RP_TINY_BATCH];
+    __shared__ int s_n;
+    if (threadIdx.x == 0) { d_ctl_reset(ctl, params); s_n = 0; }
+    __syncthreads();
+    d_classify(ups, op_seq, N, ctl, hkeys, hwin, hmask, op_slot, feat_last, vdel_seq);
+    __syncthreads();
+    d_resolve(ups, op_seq, ctl, hwin, op_slot, feat_last, vdel_seq, out, in, rec, bitmap, op_w, grow_out, grow_in,
+              shrink_out, shrink_in, nullptr);
+    __syncthreads();
+    d_del_mark(ctl, rec, out, in);
+    __syncthreads();
+    d_del_tail_read(ctl, rec, out, in);
+    __syncthreads();
+    d_del_tail_pack(ctl, rec, out, in);
+    __syncthreads();
+    d_del_fill(ctl, rec, out, in);
+    __syncthreads();
+    d_grow_rows(ctl, out, in, grow_out, grow_in, shrink_out, shrink_in, moved_start, moved_cap);
+    __syncthreads();
+    d_add_write(ctl, rec, out, in);
+    __syncthreads();
+    d_commit_degrees(ctl, rec, out, in, deg_out_old, moved_start, moved_cap);
+    __syncthreads();
+    if (ctl->abort) return;
+    // A_0: the vertices whose last feature operation this is, ascending
+    const int n = ctl->n_ops;
+    if ((int)threadIdx.x < n) {
+        const ripple_update op = ups[threadIdx.x];
+        if (op.op == RIPPLE_OP_SET_FEATURE && feat_last[op.u] == (int)threadIdx.x) {
+            s_ids[atomicAdd(&s_n, 1)] = op.u;
+            atomicAnd(&bitmap[op.u >> 5], ~(1u << (op.u & 31)));   // (resolution marked it for the general chain's sweep)
+        }
+    }
+    __syncthreads();
+    const int na = s_n;
+    int mine = -1, rank = 0;
+    if ((int)threadIdx.x < na) {
+        mine = s_ids[threadIdx.x];
+        for (int k = 0; k < na; ++k) rank += s_ids[k] < mine;
+    }
+    __syncthreads();
+    if (mine >= 0) { s_ids[rank] = mine; A0[rank] = mine; }
+    if (threadIdx.x == 0) { ctl->nA[0] = na; ctl->nC[0] = na; }
+    __syncthreads();
+    // feature rows: one warp per vertex of A_0
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = warp; i < na; i += (int)(blockDim.x >> 5)) {
+        const int v = s_ids[i];
+        const float* src = feat + (size_t)ups[feat_last[v]].v * d0;
+        for (int k = lane; k < ld; k += 32) {
+            const float x = k < d0 ? src[k] : 0.f;
+            const float o = H0[(size_t)v * ld + k];
+            D[(size_t)i * ld + k] = keep_old ? o : x - o;
+            H0[(size_t)v * ld + k] = x;
+        }
+    }
+    // senders of hop 1 = A_0, with the prefix of their out-degrees
+    if (threadIdx.x == 0) {
+        int64_t sum = 0;
+        for (int i = 0; i < na; ++i) {
+            const int v = s_ids[i];
+            senders[i] = v;
+            posmap[v] = i;
+            coff[i] = sum;
+            sum += out.deg[v];
+        }
+        coff[na] = sum;
+        ctl->E[1] = (unsigned long long)sum;
+    }
+}
+
+void graph_batch_apply_small(Ctx* c, int n) {
+    (void)n;
+    Side& o = c->side[0];
+    Side& i = c->side[1];
+    RP_LAUNCH(c, k_apply_small, 1, 1024, 0, c->ctl, (const int*)c->params_dev, (const ripple_update*)c->ups_dev,
+              (const int32_t*)c->op_seq, c->N, c->hkeys, c->hwin, c->hsize - 1, c->op_slot, c->feat_last, c->vdel_seq, o, i,
+              c->rec, c->bitmap, (const float*)(c->has_opw ? c->opw_dev : nullptr), c->grow_list[0], c->grow_list[1],
+              c->shrink_list[0], c->shrink_list[1], c->moved_start, c->moved_cap, c->deg_out_old,
+              (const float*)c->feat_dev, c->d[0], c->H[0], c->ld[0], c->D[0], (int)c->attention, c->A[0], c->Clist[0],
+              c->posmap, c->coff);
 }
 
 void graph_batch_mutate(Ctx* c, int n) {

@@ -18,6 +18,64 @@ namespace rp {
 // for a few dozen rows, half of the latency of a batch of one update.
 constexpr int BM = 64, BN = 64, BK = 64, TM = 4, TN = 4;
 
+// A frontier of a few rows (a batch of one or two updates at the first hops) is nothing but latency: the tiled
+// form walks K in chunks, each a round trip to L2 behind the last.  For up to FEW_ROWS rows and K up to FEW_K the
+// same kernel takes another route: a block owns 32 output columns, stages the few A rows in shared memory once,
+// its eight warps each take an eighth of K with every weight load independent of the others (one round trip in
+// all), the partial sums meet in shared memory and the ordinary epilogue finishes the rows.
+constexpr int FEW_ROWS = 16, FEW_K = 256, FEW_COLS = 32;
+
+__device__ __forceinline__ bool upd_few(const UpdParams& p, int n) {
+    return n > 0 && n <= FEW_ROWS && p.K > 0 && p.K <= FEW_K;
+}
+
+__device__ __forceinline__ void update_few_rows(const UpdParams& p, int n, float* A_s, float* red, int* row_id,
+                                                float* row_scale) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int kq = p.K >> 2;
+    const int groups = (p.n_cols + FEW_COLS - 1) / FEW_COLS;
+    for (int g = blockIdx.x; g < groups; g += gridDim.x) {
+        __syncthreads();
+        if (tid < n) {
+            const int v = p.list ? p.list[tid] : tid;
+            row_id[tid] = v;
+            row_scale[tid] = upd_row_scale(p, v);
+        }
+        __syncthreads();
+        for (int it = tid; it < n * kq; it += blockDim.x) {
+            const int r = it / kq, k = 4 * (it - r * kq);
+            *reinterpret_cast<float4*>(A_s + r * FEW_K + k) = upd_load_a(p, row_id[r], r, k, row_scale[r]);
+        }
+        __syncthreads();
+        const int c = g * FEW_COLS + lane;
+        const int kper = (p.K + 7) >> 3, k_begin = warp * kper, k_end = min(p.K, k_begin + kper);
+        float acc[FEW_ROWS];
+#pragma unroll
+        for (int r = 0; r < FEW_ROWS; ++r) acc[r] = 0.f;
+#pragma unroll 8
+        for (int k = k_begin; k < k_end; ++k) {
+            const float wv = c < p.n_cols ? __ldg(p.W + (size_t)k * p.ldw + c) : 0.f;
+#pragma unroll
+            for (int r = 0; r < FEW_ROWS; ++r)
+                if (r < n) acc[r] = fmaf(A_s[r * FEW_K + k], wv, acc[r]);
+        }
+#pragma unroll
+        for (int r = 0; r < FEW_ROWS; ++r) red[(warp * FEW_ROWS + r) * FEW_COLS + lane] = acc[r];
+        __syncthreads();
+        if (tid < n * (FEW_COLS / 4)) {
+            const int r = tid / (FEW_COLS / 4), q = tid - r * (FEW_COLS / 4), col = g * FEW_COLS + 4 * q;
+            if (col < p.n_cols) {
+                float4 h = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int w = 0; w < 8; ++w) {
+                    const float4 x = *reinterpret_cast<const float4*>(red + (w * FEW_ROWS + r) * FEW_COLS + 4 * q);
+                    h.x += x.x; h.y += x.y; h.z += x.z; h.w += x.w;
+                }
+                upd_epilogue4(p, row_id[r], r, col, h, row_scale[r]);
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(256)
 k_update_rows(const Ctl* ctl, UpdParams p) {
     pdl_enter();
@@ -28,6 +86,12 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
     __shared__ float row_scale[BM];
     const int n = upd_rows(p);
     if (upd_use_tc(p, n)) return;
+    if (upd_few(p, n)) {
+        static_assert(sizeof(As) >= sizeof(float) * FEW_ROWS * FEW_K && sizeof(Bs) >= sizeof(float) * 8 * FEW_ROWS * FEW_COLS,
+                      "the few-row form borrows the tiles' shared memory");
+        update_few_rows(p, n, &As[0][0], &Bs[0][0], row_id, row_scale);
+        return;
+    }
     const int row_tiles = (n + BM - 1) / BM, col_tiles = (p.n_cols + BN - 1) / BN;
     const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
     for (int tile = blockIdx.x; tile < row_tiles * col_tiles; tile += gridDim.x) {

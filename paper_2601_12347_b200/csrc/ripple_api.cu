@@ -45,17 +45,7 @@ static cudaError_t dev_alloc(T** p, size_t count, int fill_byte = -2) {
 // launch chain can be replayed for batches that differ in them)
 __global__ void k_ctl_reset(Ctl* ctl, const int* params) {
     pdl_enter();
-    Ctl z;
-    memset(&z, 0, sizeof(Ctl));
-    for (int s = 0; s < 2; ++s) {
-        z.pool_next[s] = ctl->pool_next[s];
-        z.pool_free[s] = ctl->pool_free[s];
-        z.pool_lost[s] = ctl->pool_lost[s];
-    }
-    z.num_edges = ctl->num_edges;
-    z.n_ops = params[0];
-    z.n_rows = params[1];
-    *ctl = z;
+    d_ctl_reset(ctl, params);
 }
 
 static void destroy_ctx(Ctx* c) {
@@ -434,15 +424,23 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
     const int L = c->L;
     int evi = 0;
 #define STAMP() do { if (stamps) cudaEventRecord(c->ev[evi], c->stream); ++evi; } while (0)
-    RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
-    STAMP();  // 0
-    // Apply (Sec. 3.3): normalise the batch, mutate both adjacency directions, replace features
-    graph_batch_classify(c, nb);
-    graph_batch_mutate(c, nb);
-    frontier_seed_features(c, nb);
-    feature_rows(c, nb);
-    if (rp_monotonic(c->agg)) max_senders_build(c, 0);
-    else senders_build(c, 0, nb);
+    // A handful of updates: the whole of Apply and the hop-0 sender list in one block (the chain of a small batch
+    // is bound by the number of dependent steps, not by their work); also the merged frontier kernel below.
+    const bool tiny = nb >= 1 && nb <= RP_TINY_BATCH && !c->may_expand && !c->src_norm && !rp_monotonic(c->agg);
+    if (tiny && nb <= RP_TINY_APPLY) {
+        STAMP();  // 0
+        graph_batch_apply_small(c, nb);
+    } else {
+        RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
+        STAMP();  // 0
+        // Apply (Sec. 3.3): normalise the batch, mutate both adjacency directions, replace features
+        graph_batch_classify(c, nb);
+        graph_batch_mutate(c, nb);
+        frontier_seed_features(c, nb);
+        feature_rows(c, nb);
+        if (rp_monotonic(c->agg)) max_senders_build(c, 0);
+        else senders_build(c, 0, nb);
+    }
     STAMP();  // 1
     if (rp_monotonic(c->agg)) {
         // hybrid-incremental hops of a monotonic aggregator (Sec. 3.4.2)
@@ -480,14 +478,18 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
         if (pull) frontier_compact(c, l);
         STAMP();
         scatter_layer(c, l, nb);
-        if (!pull) frontier_compact(c, l);
+        // tiny batches on graphs whose frontier bitmap one block can sweep: A_l, and later the next hop's senders,
+        // by one launch each instead of two
+        const bool merged = tiny && !pull && c->n_words <= RP_TINY_WORDS;
+        if (merged) frontier_compact_small(c, l);
+        else if (!pull) frontier_compact(c, l);
         if (nb <= 0) senders_release(c, l - 1);   // (otherwise the last kernel of the hop's delta form clears them)
         fold_deltas(c, l);
         regather_layer(c, l);
         STAMP();
         self_project(c, l, false);
         update_rows(c, l, false);
-        if (l < L) senders_build(c, l, nb);
+        if (l < L) { if (merged) senders_build_small(c, l); else senders_build(c, l, nb); }
         STAMP();
     }
     graph_batch_cleanup(c, nb);

@@ -8,6 +8,7 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "../../include/ripple.h"
 #include "../../include/ripple_part.h"
@@ -20,6 +21,9 @@
 #define RP_POOL_CLASSES 32          // block size classes of the adjacency store: class k holds blocks of 2^k entries
 #define RP_POOL_MIN_CLASS 3         // smallest block that is kept for reuse: 8 entries
 #define RP_POOL_LIST_CAP 16384      // blocks a class's free list can hold
+#define RP_TINY_BATCH 32            // batches up to this size list their frontiers and senders in one block each
+#define RP_TINY_APPLY 4             // ... and up to this size run the whole of Apply in one block (operations are resolved one after the other there)
+#define RP_TINY_WORDS 16384         // ... and list a hop's frontier in one block if its bitmap has at most this many words
 
 namespace rp {
 
@@ -60,6 +64,22 @@ struct Ctl {
     long long num_edges;              // current edge count (kept across batches)
     int work_counter[8];              // dynamic work distribution tickets (reset by the consumer)
 };
+
+// Start of a batch: everything back to zero except what lives across batches; params[0] = number of
+// operations, params[1] = number of payload rows.
+__device__ __forceinline__ void d_ctl_reset(Ctl* ctl, const int* params) {
+    Ctl z;
+    memset(&z, 0, sizeof(Ctl));
+    for (int s = 0; s < 2; ++s) {
+        z.pool_next[s] = ctl->pool_next[s];
+        z.pool_free[s] = ctl->pool_free[s];
+        z.pool_lost[s] = ctl->pool_lost[s];
+    }
+    z.num_edges = ctl->num_edges;
+    z.n_ops = params[0];
+    z.n_rows = params[1];
+    *ctl = z;
+}
 
 // One direction of the adjacency: row r holds col[start[r] .. start[r] + deg[r]), capacity cap[r].
 // Rows start in the base region; a row that outgrows its slack moves into the overflow pool
@@ -266,6 +286,7 @@ inline int pad4(int x) { return (x + 3) & ~3; }
 cudaError_t graph_build(Ctx* c, const int32_t* src_dev, const int32_t* dst_dev, const float* w_dev, int64_t E,
                         double slack, int64_t pool_edges);
 void graph_batch_classify(Ctx* c, int n);   // validate, dedupe, find net changes, plan
+void graph_batch_apply_small(Ctx* c, int n);            // a handful of updates: control block reset, Apply and the hop-0 senders in one block
 void graph_batch_mutate(Ctx* c, int n);                 // apply the net changes to both directions
 void graph_batch_cleanup(Ctx* c, int n);                // reset per-batch scratch
 cudaError_t graph_export(Ctx* c, int64_t* rowptr, int32_t* col, float* weight, int64_t col_capacity, int64_t* n_edges);
@@ -276,6 +297,8 @@ void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, con
 void frontier_seed_features(Ctx* c, int n);             // A_0 from the batch's feature updates
 void frontier_mark(Ctx* c, int l, bool walk, int n);    // bitmap of A_l: (walk) edge-record sinks, A_{l-1} and Out(C_{l-1}); rebuilding hops: bottom-up
 void frontier_compact(Ctx* c, int l);                   // bitmap -> ascending list A_l
+void frontier_compact_small(Ctx* c, int l);              // the same in one block (tiny batches, small graphs)
+void senders_build_small(Ctx* c, int l);                // C_l = A_l with its degree prefix, in one block
 void senders_build(Ctx* c, int l, int n);               // C_l, posmap, coff, E_{l+1}
 void senders_release(Ctx* c, int l);                    // clear posmap entries of C_l
 
