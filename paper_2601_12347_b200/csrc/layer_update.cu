@@ -18,33 +18,35 @@ namespace rp {
 // for a few dozen rows, half of the latency of a batch of one update.
 constexpr int BM = 64, BN = 64, BK = 64, TM = 4, TN = 4;
 
-// A frontier of a few rows (a batch of one or two updates at the first hops) is nothing but latency: the tiled
-// form walks K in chunks, each a round trip to L2 behind the last.  For up to FEW_ROWS rows and K up to FEW_K the
-// same kernel takes another route: a block owns 32 output columns, stages the few A rows in shared memory once,
-// its eight warps each take an eighth of K with every weight load independent of the others (one round trip in
-// all), the partial sums meet in shared memory and the ordinary epilogue finishes the rows.
-constexpr int FEW_ROWS = 16, FEW_K = 256, FEW_COLS = 32;
+// A frontier of a few rows (a batch of a few updates at the first hops) is nothing but latency: the tiled form
+// walks K in chunks, each a round trip to L2 behind the last.  For up to FEW_MAX rows and K up to FEW_K the same
+// kernel takes another route: a block owns FEW_ROWS rows and 32 output columns, stages its A rows in shared
+// memory once, its eight warps each take an eighth of K with every weight load independent of the others (one
+// round trip in all), the partial sums meet in shared memory and the ordinary epilogue finishes the rows.
+constexpr int FEW_ROWS = 16, FEW_K = 256, FEW_COLS = 32, FEW_MAX = 256;
 
 __device__ __forceinline__ bool upd_few(const UpdParams& p, int n) {
-    return n > 0 && n <= FEW_ROWS && p.K > 0 && p.K <= FEW_K;
+    return n > 0 && n <= FEW_MAX && p.K > 0 && p.K <= FEW_K;
 }
 
-__device__ __forceinline__ void update_few_rows(const UpdParams& p, int n, float* A_s, float* red, int* row_id,
+__device__ __forceinline__ void update_few_rows(const UpdParams& p, int n_all, float* A_s, float* red, int* row_id,
                                                 float* row_scale) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int kq = p.K >> 2;
-    const int groups = (p.n_cols + FEW_COLS - 1) / FEW_COLS;
-    for (int g = blockIdx.x; g < groups; g += gridDim.x) {
+    const int groups = (p.n_cols + FEW_COLS - 1) / FEW_COLS, row_groups = (n_all + FEW_ROWS - 1) / FEW_ROWS;
+    for (int item = blockIdx.x; item < groups * row_groups; item += gridDim.x) {
+        const int g = item % groups, r0 = (item / groups) * FEW_ROWS;
+        const int n = min(FEW_ROWS, n_all - r0);   // rows of this block: compact indices r0 .. r0 + n - 1
         __syncthreads();
         if (tid < n) {
-            const int v = p.list ? p.list[tid] : tid;
+            const int v = p.list ? p.list[r0 + tid] : r0 + tid;
             row_id[tid] = v;
             row_scale[tid] = upd_row_scale(p, v);
         }
         __syncthreads();
         for (int it = tid; it < n * kq; it += blockDim.x) {
             const int r = it / kq, k = 4 * (it - r * kq);
-            *reinterpret_cast<float4*>(A_s + r * FEW_K + k) = upd_load_a(p, row_id[r], r, k, row_scale[r]);
+            *reinterpret_cast<float4*>(A_s + r * FEW_K + k) = upd_load_a(p, row_id[r], r0 + r, k, row_scale[r]);
         }
         __syncthreads();
         const int c = g * FEW_COLS + lane;
@@ -70,7 +72,7 @@ __device__ __forceinline__ void update_few_rows(const UpdParams& p, int n, float
                     const float4 x = *reinterpret_cast<const float4*>(red + (w * FEW_ROWS + r) * FEW_COLS + 4 * q);
                     h.x += x.x; h.y += x.y; h.z += x.z; h.w += x.w;
                 }
-                upd_epilogue4(p, row_id[r], r, col, h, row_scale[r]);
+                upd_epilogue4(p, row_id[r], r0 + r, col, h, row_scale[r]);
             }
         }
     }
