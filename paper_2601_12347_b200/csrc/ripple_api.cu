@@ -74,6 +74,8 @@ static void destroy_ctx(Ctx* c) {
     cudaFree(c->moved_start); cudaFree(c->moved_cap);
     if (c->ctl_host) cudaFreeHost(c->ctl_host);
     if (c->params_host) cudaFreeHost(c->params_host);
+    if (c->stage_host) cudaFreeHost(c->stage_host);
+    cudaFree(c->stage_dev);
     cudaFree(c->params_dev);
     for (auto& g : c->graph_exec) if (g) cudaGraphExecDestroy(g);
     for (auto& e : c->ev) if (e) cudaEventDestroy(e);
@@ -203,6 +205,9 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         CK(dev_alloc(&c->ctl, 1, 0));
         CK(dev_alloc(&c->params_dev, 2, 0));
         CK(cudaMallocHost(&c->params_host, 2 * sizeof(int)));
+        c->stage_bytes = 64 + (size_t)RP_GRAPH_MAX_BATCH * (sizeof(ripple_update) + sizeof(float) + sizeof(float) * (size_t)layers[0].d_in);
+        CK(cudaMallocHost(&c->stage_host, c->stage_bytes));
+        CK(dev_alloc(&c->stage_dev, c->stage_bytes));
         c->no_graphs = o.no_graphs;
         {
             const char* e = getenv("RIPPLE_NO_PDL");
@@ -527,6 +532,7 @@ static bool launch_batch_graph(Ctx* c, int nb) {
     // the captured chain differs with the expansion kernels and with the hops whose rebuilding form is enqueued
     int key = 4 * nb + (c->may_expand ? 1 : 0) + (c->has_opw ? 2 : 0);
     key = 2 * key + (c->tc_armed ? 1 : 0);
+    key = 2 * key + (c->packed_now ? 1 : 0);   // (the chain holds the addresses its kernels read the batch from)
     for (int l = 1; l <= c->L; ++l) key = 2 * key + (c->rebuild_armed[l] ? 1 : 0);
     int slot = -1;
     for (int i = 0; i < RP_GRAPH_SLOTS; ++i)
@@ -586,6 +592,9 @@ extern "C" ripple_status ripple_apply_batch_weighted(ripple_ctx* ctx, const ripp
     cudaSetDevice(c->device);
     const int nb = (int)n, nr = (int)n_rows, L = c->L;
     float* own_feat = c->feat_dev;
+    ripple_update* own_ups = c->ups_dev;
+    float* own_opw = c->opw_dev;
+    int* own_params = c->params_dev;
     c->launches = 0;
     int evi = 0;
     // A vertex deletion becomes one edge deletion per incident edge on the device.  Launches are
@@ -604,23 +613,45 @@ extern "C" ripple_status ripple_apply_batch_weighted(ripple_ctx* ctx, const ripp
     arm_rebuild(c, nb);
     const bool try_graph = !wide && !c->no_graphs && !c->timing && nb >= 1 && nb <= RP_GRAPH_MAX_BATCH;
     const cudaMemcpyKind kind = mem == RIPPLE_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
-    // operations are always staged: generated edge deletions are appended behind them
-    if (nb) CK(cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, kind, c->stream));
     c->has_opw = c->weighted && edge_weights && nb;
-    if (c->has_opw) CK(cudaMemcpyAsync(c->opw_dev, edge_weights, sizeof(float) * (size_t)nb, kind, c->stream));
-    if (mem == RIPPLE_MEM_HOST || try_graph) {
-        // a replayed graph reads the library's own staging buffers, so device payload rows are copied too
-        if (nr) CK(cudaMemcpyAsync(c->feat_dev, feat_rows, sizeof(float) * (size_t)nr * c->d[0], kind, c->stream));
+    // A small host batch without vertex deletions travels in one copy: sizes, operations, weights and payload
+    // rows are packed into pinned memory at offsets that depend on the number of operations alone (a captured
+    // chain holds them), and the kernels read them where they land.
+    const bool packed = mem == RIPPLE_MEM_HOST && !wide && nb >= 1 && nb <= RP_GRAPH_MAX_BATCH && nr <= RP_GRAPH_MAX_BATCH;
+    c->packed_now = packed;
+    if (packed) {
+        auto pad16 = [](size_t x) { return (x + 15) & ~(size_t)15; };
+        const size_t off_ups = 16, off_w = off_ups + pad16(sizeof(ripple_update) * (size_t)nb);
+        const size_t off_rows = off_w + (c->weighted ? pad16(sizeof(float) * (size_t)nb) : 0);
+        const size_t total = off_rows + sizeof(float) * (size_t)nr * c->d[0];
+        int* head = reinterpret_cast<int*>(c->stage_host);
+        head[0] = nb; head[1] = nr;
+        memcpy(c->stage_host + off_ups, ups, sizeof(ripple_update) * (size_t)nb);
+        if (c->has_opw) memcpy(c->stage_host + off_w, edge_weights, sizeof(float) * (size_t)nb);
+        if (nr) memcpy(c->stage_host + off_rows, feat_rows, sizeof(float) * (size_t)nr * c->d[0]);
+        CK(cudaMemcpyAsync(c->stage_dev, c->stage_host, total, cudaMemcpyHostToDevice, c->stream));
+        c->params_dev = reinterpret_cast<int*>(c->stage_dev);
+        c->ups_dev = reinterpret_cast<ripple_update*>(c->stage_dev + off_ups);
+        c->opw_dev = reinterpret_cast<float*>(c->stage_dev + off_w);
+        c->feat_dev = reinterpret_cast<float*>(c->stage_dev + off_rows);
     } else {
-        c->feat_dev = const_cast<float*>(feat_rows);   // device payload rows are read in place
+        // operations are always staged: generated edge deletions are appended behind them
+        if (nb) CK(cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, kind, c->stream));
+        if (c->has_opw) CK(cudaMemcpyAsync(c->opw_dev, edge_weights, sizeof(float) * (size_t)nb, kind, c->stream));
+        if (mem == RIPPLE_MEM_HOST || try_graph) {
+            // a replayed graph reads the library's own staging buffers, so device payload rows are copied too
+            if (nr) CK(cudaMemcpyAsync(c->feat_dev, feat_rows, sizeof(float) * (size_t)nr * c->d[0], kind, c->stream));
+        } else {
+            c->feat_dev = const_cast<float*>(feat_rows);   // device payload rows are read in place
+        }
+        c->params_host[0] = nb; c->params_host[1] = nr;
+        CK(cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream));
     }
-    c->params_host[0] = nb; c->params_host[1] = nr;
-    CK(cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream));
     if (!try_graph || !launch_batch_graph(c, nb)) {
         c->launches = 0;
         evi = enqueue_batch(c, ng, c->timing != 0);
     }
-    c->feat_dev = own_feat;
+    c->feat_dev = own_feat; c->ups_dev = own_ups; c->opw_dev = own_opw; c->params_dev = own_params;
     st = sync_and_fetch_ctl(c);
     if (st) return st;
     {
@@ -674,7 +705,7 @@ extern "C" ripple_status ripple_apply_batch_weighted(ripple_ctx* ctx, const ripp
     }
     return RIPPLE_OK;
 fail:
-    c->feat_dev = own_feat;
+    c->feat_dev = own_feat; c->ups_dev = own_ups; c->opw_dev = own_opw; c->params_dev = own_params;
     return st;
 }
 

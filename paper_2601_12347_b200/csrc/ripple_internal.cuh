@@ -228,6 +228,10 @@ struct Ctx {
     int64_t* tile_sums;
     int n_tile_sums;
     int* scan_done;    // blocks of a scan's first kernel that have finished (zero between scans)
+    char* stage_host;  // pinned: sizes, operations, weights and payload rows of a small host batch, packed for one copy
+    char* stage_dev;
+    size_t stage_bytes;
+    int packed_now;    // the batch being applied arrived through the packed staging buffer
     int* params_dev;   // {n_ops, n_rows} of the batch being applied
     int* params_host;  // pinned
     int no_graphs;
