@@ -591,6 +591,14 @@ extern "C" ripple_status ripple_apply_batch_weighted(ripple_ctx* ctx, const ripp
     }
     cudaSetDevice(c->device);
     const int nb = (int)n, nr = (int)n_rows, L = c->L;
+    if (nb == 0) {   // nothing to apply, nothing to propagate: no device work at all
+        ripple_stats& s = c->stats;
+        s.gpu_launches = 0;
+        s.n_ops = s.n_added = s.n_deleted = s.n_noop_add = s.n_noop_del = s.n_superseded = s.n_feature = s.n_expanded = 0;
+        for (int l = 0; l <= L; ++l) s.affected[l] = s.senders[l] = s.active_edges[l] = s.rows_rebuilt[l] = s.in_edges[l] = 0;
+        s.ms_total = s.ms_graph = 0.f;
+        return RIPPLE_OK;
+    }
     float* own_feat = c->feat_dev;
     ripple_update* own_ups = c->ups_dev;
     float* own_opw = c->opw_dev;
