@@ -30,7 +30,10 @@ Readings where the paper is silent:
   - load(P_i) counts the vertices placed on P_i; ties go to the lowest partition number;
   - the sink's worker learns that the sink is a hop-l vertex from the arrival of the (possibly zero)
     combined message that the source's worker sends for every changed edge at every hop;
-  - vertex deletion is not routed here (the server would need the incident edge lists).
+  - vertex deletion (Sec. 4.3 routes it to the owner and says no more): the server, which keeps the edge
+    lists for this purpose, replaces it at its position in the batch by one edge deletion per incident
+    edge (out-edges in ascending sink order, then in-edges in ascending source order), each routed like
+    any edge deletion, followed by a feature update of the vertex with a row of zeros (payload row -1);
 The numerical rules (delta messages, coefficients, Update) are those of the single-machine method
 (Sec. 3.3); the pin is that the workers' rows equal the single-machine oracle's full recomputation.
 """
@@ -40,7 +43,7 @@ from typing import Dict, List, Tuple
 
 import numpy as np
 
-OP_ADD_EDGE, OP_DEL_EDGE, OP_SET_FEATURE = 0, 1, 2
+OP_ADD_EDGE, OP_DEL_EDGE, OP_SET_FEATURE, OP_DEL_VERTEX = 0, 1, 2, 3
 KIND_SAGE, KIND_GRAPHCONV, KIND_GIN = 0, 1, 2
 AGG_SUM, AGG_MEAN, AGG_WSUM_GCN = 0, 1, 2
 ACT_RELU = 1
@@ -62,6 +65,11 @@ class Server:
         self.hd_refresh = int(hd_refresh)
         self.seen = 0
         self.edges = set(zip(src.tolist(), dst.tolist()))     # to keep in-degrees right under no-op updates
+        self.out_adj: Dict[int, set] = {}                     # edge lists, for the expansion of vertex deletions
+        self.in_adj: Dict[int, set] = {}
+        for u, v in self.edges:
+            self.out_adj.setdefault(u, set()).add(v)
+            self.in_adj.setdefault(v, set()).add(u)
         self.refresh_hd()
 
     def refresh_hd(self):
@@ -96,12 +104,27 @@ class Server:
         if not ev:
             self._place(v, p)
 
+    def _count(self):
+        self.seen += 1
+        if self.seen % self.hd_refresh == 0:
+            self.refresh_hd()
+
     def route(self, ups: np.ndarray) -> List[List[Tuple[int, int, int, int, bool]]]:
-        """Per worker: (position in the batch, op, u, v, compute?) in batch order."""
+        """Per worker: (position in the batch, op, u, v, compute?) in batch order.  A feature update's v is
+        the payload row (-1: a row of zeros, from the expansion of a vertex deletion)."""
         out: List[List[Tuple[int, int, int, int, bool]]] = [[] for _ in range(self.P)]
-        for i, r in enumerate(ups):
-            op, u, v = int(r["op"]), int(r["u"]), int(r["v"])
-            if op == OP_SET_FEATURE:
+        todo = [(i, int(r["op"]), int(r["u"]), int(r["v"])) for i, r in enumerate(ups)]
+        k = 0
+        while k < len(todo):
+            i, op, u, v = todo[k]
+            k += 1
+            if op == OP_DEL_VERTEX:        # replaced, at its position, by the deletions of its edges and a zero row
+                if self.owner[u] >= 0:
+                    gen = [(i, OP_DEL_EDGE, u, x) for x in sorted(self.out_adj.get(u, ()))]
+                    gen += [(i, OP_DEL_EDGE, x, u) for x in sorted(self.in_adj.get(u, ()))]
+                    gen.append((i, OP_SET_FEATURE, u, -1))
+                    todo[k:k] = gen
+            elif op == OP_SET_FEATURE:
                 assert self.owner[u] >= 0, "feature update of a vertex that is not in the graph"
                 out[int(self.owner[u])].append((i, op, u, v, True))
             elif op in (OP_ADD_EDGE, OP_DEL_EDGE):
@@ -114,13 +137,13 @@ class Server:
                         out[pv].append((i, op, u, v, False))      # the no-compute copy
                     if op == OP_ADD_EDGE and (u, v) not in self.edges:
                         self.edges.add((u, v)); self.in_degree[v] += 1; self.n_edges += 1
+                        self.out_adj.setdefault(u, set()).add(v); self.in_adj.setdefault(v, set()).add(u)
                     elif op == OP_DEL_EDGE and (u, v) in self.edges:
                         self.edges.discard((u, v)); self.in_degree[v] -= 1; self.n_edges -= 1
+                        self.out_adj[u].discard(v); self.in_adj[v].discard(u)
             else:
-                raise ValueError("only edge additions, edge deletions and feature updates are routed")
-            self.seen += 1
-            if self.seen % self.hd_refresh == 0:
-                self.refresh_hd()
+                raise ValueError("unknown op code")
+            self._count()
         return out
 
 
@@ -220,7 +243,7 @@ class Worker:
         A, old = [], {}
         for u, row in sorted(last_feat.items()):
             old[u] = self.H[0][u].copy()
-            self.H[0][u] = feat_rows[row].astype(np.float64)
+            self.H[0][u] = feat_rows[row].astype(np.float64) if row >= 0 else np.zeros_like(old[u])
             A.append(u)
         return A, old
 

@@ -221,3 +221,34 @@ def test_combiner_sends_one_row_per_worker_and_remote_sink():
     assert cl.halo_rows_sent[1] == 30          # 90 messages cross the cut, 30 combined rows are sent
     assert orc.active_edges(1) == 90
     assert rel_err(cl.gather(2, n), orc.full()[2]) < 1e-12
+
+
+# ---------------------------------------------------------------------------------------------
+# vertex deletion: expanded by the server
+# ---------------------------------------------------------------------------------------------
+def test_vertex_deletion_is_replaced_by_its_edge_deletions_and_a_zero_row():
+    s = _server()
+    r = s.route(ups_array([(I.OP_DEL_VERTEX, 3, 0)]))          # in-edges from 0, 1, 2 (partition 0) and 4, 5 (partition 1)
+    assert r[0] == [(0, I.OP_DEL_EDGE, 0, 3, True), (0, I.OP_DEL_EDGE, 1, 3, True), (0, I.OP_DEL_EDGE, 2, 3, True),
+                    (0, I.OP_DEL_EDGE, 4, 3, False), (0, I.OP_DEL_EDGE, 5, 3, False), (0, I.OP_SET_FEATURE, 3, -1, True)]
+    assert r[1] == [(0, I.OP_DEL_EDGE, 4, 3, True), (0, I.OP_DEL_EDGE, 5, 3, True)]
+    assert s.in_degree[3] == 0 and s.n_edges == 1
+    r = s.route(ups_array([(I.OP_ADD_EDGE, 6, 3), (I.OP_DEL_VERTEX, 6, 0)]))   # an edge added earlier in the batch goes too
+    assert (1, I.OP_DEL_EDGE, 6, 3, True) in r[1] and (1, I.OP_DEL_EDGE, 6, 7, True) in r[1]
+    assert s.n_edges == 0
+
+
+@pytest.mark.parametrize("P", [2, 3])
+@pytest.mark.parametrize("name", ["sage_mean", "gcn_wsum_3l", "gin"])
+def test_cluster_with_vertex_deletions_equals_single_machine(name, P):
+    n = 60
+    model, src, dst, orc, cl, L = _cluster(name, P, n=n)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 7, mix=(0.35, 0.35, 0.2, 0.1))
+    for b in range(10):
+        ups, rows = stream.next_batch(1 + 4 * (b % 3))
+        cl.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        full = orc.full()
+        for l in range(L + 1):
+            assert rel_err(cl.gather(l, n), full[l]) < 1e-9, (name, P, b, l)
+            assert cl.affected[l] == orc.affected(l).tolist(), (name, P, b, l)
