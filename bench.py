@@ -580,7 +580,7 @@ def run_partitioned(args):
                     lu, nc, row_of, first, ho, hr = shares[r]
                     if ho.size:
                         wk.set_halos(first, ho, hr)
-                    wk.begin(lu, rows[row_of] if row_of.size else None, nc)
+                    wk.begin(lu, PT.payload_rows(rows, row_of, wk.dims[0]), nc)
 
                 crit += phase(begin)
                 for l in range(1, L + 1):

@@ -26,8 +26,8 @@
  *                          process and no routing messages exist.
  *
  * What a partitioned context supports: the linear aggregators SUM, MEAN, WSUM_GCN with SAGE, GRAPHCONV
- * and GIN layers; edge additions, edge deletions and feature replacements (a vertex deletion would need
- * the router to know the vertex's incident edges: RIPPLE_ERR_INVALID_ARG).  Hops always take the delta
+ * and GIN layers; edge additions, edge deletions and feature replacements (the router turns a vertex
+ * deletion into these; a worker given one answers RIPPLE_ERR_INVALID_ARG).  Hops always take the delta
  * form (push); the rounding budget is off (a row cannot be gathered anew without its remote
  * in-neighbours' rows).  ripple_apply_batch and ripple_recompute_full are refused on such a context.
  *
@@ -151,7 +151,11 @@ ripple_status ripple_router_partition_fill(ripple_router* r, int32_t rank, int32
  * number of operations, payload rows and halo slots assigned by this batch, and ripple_router_batch_fill
  * the operations in local ids (in batch order), their no-compute flags, for every payload row of the
  * worker the index of the global payload row it is a copy of, and the new halo slots (first slot index
- * in *first_halo).  RIPPLE_ERR_INVALID_ARG (a vertex deletion or an unknown op code) and
+ * in *first_halo).  A payload row index of -1 in row_of stands for a row of zeros.
+ * A vertex deletion (Sec. 4.3 routes it to the owner and says no more) is replaced, at its position in the
+ * batch, by one edge deletion per incident edge -- the router keeps the edge lists for this -- each routed
+ * like any edge deletion, and a feature update of the vertex with a row of zeros; the workers never see
+ * a vertex deletion.  RIPPLE_ERR_INVALID_ARG (an unknown op code) and
  * RIPPLE_ERR_VERTEX_RANGE are found before anything changes.  RIPPLE_ERR_CAPACITY (a worker ran out of
  * local ids or halo slots) and RIPPLE_ERR_INVALID_ARG for a feature update of a vertex that is not placed
  * are found while routing: the batch is then partly routed and the router must be destroyed. */

@@ -11,7 +11,6 @@
 #include <algorithm>
 #include <new>
 #include <unordered_map>
-#include <unordered_set>
 #include <vector>
 
 namespace {
@@ -41,11 +40,49 @@ struct ripple_router {
     std::vector<int32_t> owner, local_id, in_degree;
     std::vector<int64_t> load;
     std::vector<uint8_t> high;
-    std::unordered_set<uint64_t> edges;   // u * N + v: keeps the in-degrees right under no-op updates
     std::vector<Part> part;
     std::vector<int32_t> src0, dst0;      // the initial edges (for ripple_router_partition_fill)
+    // the edge lists: whether an edge exists (in-degrees must not move under no-op updates), and the expansion
+    // of vertex deletions
+    std::vector<std::vector<int32_t>> out_adj, in_adj;
 
-    uint64_t key(int32_t u, int32_t v) const { return (uint64_t)u * (uint64_t)N + (uint64_t)v; }
+    void count_update() { if (++seen % hd_refresh == 0) refresh_high(); }
+    static bool drop(std::vector<int32_t>& a, int32_t x) {
+        for (size_t i = 0; i < a.size(); ++i)
+            if (a[i] == x) { a[i] = a.back(); a.pop_back(); return true; }
+        return false;
+    }
+    bool has_edge(int32_t u, int32_t v) const {   // the shorter of the two lists is searched
+        const std::vector<int32_t>& a = out_adj[u].size() <= in_adj[v].size() ? out_adj[u] : in_adj[v];
+        const int32_t x = &a == &out_adj[u] ? v : u;
+        return std::find(a.begin(), a.end(), x) != a.end();
+    }
+    // routes one edge operation (placing new endpoints first); false: a worker ran out of ids or halo slots
+    bool route_edge(int32_t op, int32_t u, int32_t v) {
+        const bool add = op == RIPPLE_OP_ADD_EDGE;
+        if (add && !assign_edge(u, v)) return false;
+        const int pu = owner[u], pv = owner[v];
+        if (pu < 0 || pv < 0) return true;   // (deleting an edge of a vertex that was never placed: nothing exists)
+        const int32_t lu = id_at(pu, u), lv = id_at(pu, v);
+        if (lu < 0 || lv < 0) return false;
+        part[pu].ops.push_back({op, lu, lv});
+        part[pu].no_compute.push_back(0);
+        if (pv != pu) {
+            const int32_t su = id_at(pv, u), sv = id_at(pv, v);
+            if (su < 0 || sv < 0) return false;
+            part[pv].ops.push_back({op, su, sv});
+            part[pv].no_compute.push_back(1);
+        }
+        if (add && !has_edge(u, v)) { in_degree[v]++; n_edges++; out_adj[u].push_back(v); in_adj[v].push_back(u); }
+        else if (!add && drop(out_adj[u], v)) { in_degree[v]--; n_edges--; drop(in_adj[v], u); }
+        return true;
+    }
+    void route_feature(int32_t u, int32_t row) {
+        Part& q = part[owner[u]];
+        q.ops.push_back({RIPPLE_OP_SET_FEATURE, local_id[u], (int32_t)q.row_of.size()});
+        q.no_compute.push_back(0);
+        q.row_of.push_back(row);
+    }
 
     void refresh_high() {
         const double avg = (double)n_edges / (double)std::max<int64_t>(placed, 1);
@@ -117,6 +154,8 @@ extern "C" ripple_status ripple_router_create(int32_t n_partitions, int64_t num_
     r->high.assign(num_vertices, 0);
     r->load.assign(n_partitions, 0);
     r->part.resize(n_partitions);
+    r->out_adj.resize(num_vertices);
+    r->in_adj.resize(num_vertices);
     std::vector<int64_t> count(n_partitions, 0);
     for (int64_t v = 0; v < num_vertices; ++v) {
         if (owner[v] >= n_partitions) { delete r; return RIPPLE_ERR_INVALID_ARG; }
@@ -139,8 +178,9 @@ extern "C" ripple_status ripple_router_create(int32_t n_partitions, int64_t num_
             delete r;
             return RIPPLE_ERR_VERTEX_RANGE;
         }
-        r->edges.insert(r->key(u, v));
         r->in_degree[v]++;
+        r->out_adj[u].push_back(v);
+        r->in_adj[v].push_back(u);
         if (r->owner[u] != r->owner[v] && (r->id_at(r->owner[u], v) < 0 || r->id_at(r->owner[v], u) < 0)) {
             delete r;
             return RIPPLE_ERR_CAPACITY;
@@ -199,9 +239,9 @@ extern "C" ripple_status ripple_router_route(ripple_router* r, const ripple_upda
     if (!r || n < 0 || (n > 0 && !ups)) return RIPPLE_ERR_INVALID_ARG;
     for (int64_t i = 0; i < n; ++i) {     // checked before anything changes
         const ripple_update& x = ups[i];
-        if (x.op != RIPPLE_OP_ADD_EDGE && x.op != RIPPLE_OP_DEL_EDGE && x.op != RIPPLE_OP_SET_FEATURE) return RIPPLE_ERR_INVALID_ARG;
+        if (x.op < RIPPLE_OP_ADD_EDGE || x.op > RIPPLE_OP_DEL_VERTEX) return RIPPLE_ERR_INVALID_ARG;
         if (x.u < 0 || x.u >= r->N) return RIPPLE_ERR_VERTEX_RANGE;
-        if (x.op != RIPPLE_OP_SET_FEATURE && (x.v < 0 || x.v >= r->N)) return RIPPLE_ERR_VERTEX_RANGE;
+        if ((x.op == RIPPLE_OP_ADD_EDGE || x.op == RIPPLE_OP_DEL_EDGE) && (x.v < 0 || x.v >= r->N)) return RIPPLE_ERR_VERTEX_RANGE;
     }
     for (Part& q : r->part) {
         q.ops.clear(); q.no_compute.clear(); q.row_of.clear();
@@ -210,33 +250,24 @@ extern "C" ripple_status ripple_router_route(ripple_router* r, const ripple_upda
     for (int64_t i = 0; i < n; ++i) {
         const ripple_update& x = ups[i];
         if (x.op == RIPPLE_OP_SET_FEATURE) {
-            const int p = r->owner[x.u];
-            if (p < 0) return RIPPLE_ERR_INVALID_ARG;   // a feature update of a vertex that is not in the graph
-            Part& q = r->part[p];
-            q.ops.push_back({x.op, r->local_id[x.u], (int32_t)q.row_of.size()});
-            q.no_compute.push_back(0);
-            q.row_of.push_back(x.v);
-        } else {
-            const bool add = x.op == RIPPLE_OP_ADD_EDGE;
-            if (add && !r->assign_edge(x.u, x.v)) return RIPPLE_ERR_CAPACITY;
-            const int pu = r->owner[x.u], pv = r->owner[x.v];
-            if (pu >= 0 && pv >= 0) {   // (deleting an edge of a vertex that was never placed: nothing exists)
-                const int32_t lu = r->id_at(pu, x.u), lv = r->id_at(pu, x.v);
-                if (lu < 0 || lv < 0) return RIPPLE_ERR_CAPACITY;
-                r->part[pu].ops.push_back({x.op, lu, lv});
-                r->part[pu].no_compute.push_back(0);
-                if (pv != pu) {
-                    const int32_t su = r->id_at(pv, x.u), sv = r->id_at(pv, x.v);
-                    if (su < 0 || sv < 0) return RIPPLE_ERR_CAPACITY;
-                    r->part[pv].ops.push_back({x.op, su, sv});
-                    r->part[pv].no_compute.push_back(1);
-                }
-                const uint64_t k = r->key(x.u, x.v);
-                if (add && r->edges.insert(k).second) { r->in_degree[x.v]++; r->n_edges++; }
-                else if (!add && r->edges.erase(k)) { r->in_degree[x.v]--; r->n_edges--; }
-            }
+            if (r->owner[x.u] < 0) return RIPPLE_ERR_INVALID_ARG;   // a feature update of a vertex that is not in the graph
+            r->route_feature(x.u, x.v);
+        } else if (x.op == RIPPLE_OP_DEL_VERTEX) {
+            // Replaced, at its position in the batch, by the deletions of the vertex's edges (out-edges in ascending
+            // sink order, then in-edges in ascending source order: every replica generates the same sequence) and a
+            // feature update with a row of zeros (payload row -1).
+            r->count_update();
+            if (r->owner[x.u] < 0) continue;
+            std::vector<int32_t> outs = r->out_adj[x.u], ins = r->in_adj[x.u];
+            std::sort(outs.begin(), outs.end());
+            std::sort(ins.begin(), ins.end());
+            for (int32_t v : outs) { if (!r->route_edge(RIPPLE_OP_DEL_EDGE, x.u, v)) return RIPPLE_ERR_CAPACITY; r->count_update(); }
+            for (int32_t u : ins) { if (!r->route_edge(RIPPLE_OP_DEL_EDGE, u, x.u)) return RIPPLE_ERR_CAPACITY; r->count_update(); }
+            r->route_feature(x.u, -1);
+        } else if (!r->route_edge(x.op, x.u, x.v)) {
+            return RIPPLE_ERR_CAPACITY;
         }
-        if (++r->seen % r->hd_refresh == 0) r->refresh_high();
+        r->count_update();
     }
     return RIPPLE_OK;
 }

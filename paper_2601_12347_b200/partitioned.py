@@ -175,6 +175,18 @@ class Worker(R.Ripple):
         return out[: self.L + 1].tolist()
 
 
+def payload_rows(rows: Optional[np.ndarray], row_of: np.ndarray, d0: int) -> Optional[np.ndarray]:
+    """A worker's payload rows: copies of the batch's rows, zeros where the router says -1 (the feature row
+    of a deleted vertex)."""
+    if not row_of.size:
+        return None
+    out = np.zeros((row_of.size, d0), dtype=np.float32)
+    keep = row_of >= 0
+    if keep.any():
+        out[keep] = rows[row_of[keep]]
+    return out
+
+
 def _make_worker(router: Router, rank: int, X: np.ndarray, model, weights, **kw) -> Tuple[Worker, np.ndarray]:
     n_local, nv, src, dst, gof, ho, hr = router.partition(rank)
     feats = np.zeros((nv, X.shape[1]), dtype=np.float32)
@@ -225,7 +237,7 @@ class Cluster:
             lu, nc, row_of, first, ho, hr = self.router.batch(r)
             if ho.size:
                 w.set_halos(first, ho, hr)
-            w.begin(lu, rows[row_of] if row_of.size else None, nc)
+            w.begin(lu, payload_rows(rows, row_of, w.dims[0]), nc)
         for l in range(1, self.L + 1):
             for w in self.workers:
                 w.hop_send(l)
@@ -293,7 +305,7 @@ class DistributedWorker:
         lu, nc, row_of, first, ho, hr = self.router.batch(self.rank)
         if ho.size:
             self.worker.set_halos(first, ho, hr)
-        self.worker.begin(lu, rows[row_of] if row_of.size else None, nc)
+        self.worker.begin(lu, payload_rows(rows, row_of, self.worker.dims[0]), nc)
         for l in range(1, self.L + 1):
             self.dist.barrier()
             self.worker.hop_send(l)

@@ -139,8 +139,6 @@ def test_partitioned_context_refuses_what_it_cannot_do(env):
         w.recompute_full()
     with pytest.raises(ripple.RippleError):
         w.begin(G.ups_array([(I.OP_DEL_VERTEX, 0, 0)]), None, np.zeros(1, dtype=np.uint8))
-    with pytest.raises(ripple.RippleError):
-        cl.router.route(G.ups_array([(I.OP_DEL_VERTEX, 0, 0)]))
     cl.close()
     model = I.graphconv_model([18, 36, 10], I.AGG_MAX)
     with pytest.raises(ripple.RippleError):
@@ -208,3 +206,27 @@ def test_one_worker_per_process_with_ipc_mappings(env):
     assert all(res[r][0] <= TOL for r in range(world)), [res[r][0] for r in range(world)]
     assert all(res[r][2] > 0 for r in range(world))                      # rows did cross between the processes
     assert sorted(res[0][3] + res[1][3]) == res[0][4]                      # the union of the hop sets is the oracle's
+
+
+@pytest.mark.parametrize("name", ["sage_mean", "gcn_wsum_3l", "gin_3l"])
+def test_vertex_deletions_are_expanded_by_the_router(env, name):
+    """The workers never see a vertex deletion: the router turns it into the deletions of the vertex's edges
+    (cut edges reach both workers) and a zero feature row."""
+    ripple, Oracle = env
+    n, P = 700, 3
+    model, L, src, dst, X, W, owner, Cluster, _ = setup(name, P, n, 5000, 6)
+    orc = Oracle(n, src, dst, X, model, W)
+    cl = Cluster(P, owner, src, dst, X, model, W, max_batch=4096)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 6, mix=(0.38, 0.38, 0.2, 0.04))
+    for b, bs in enumerate([1, 5, 20, 60, 20, 5, 40, 3]):
+        ups, rows = stream.next_batch(bs)
+        if b == 3:
+            ups[10] = (I.OP_DEL_VERTEX, 0, 0)       # the hub whose out-edges cut every partition
+        cl.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        for l in range(L + 1):
+            assert np.array_equal(cl.affected(l), orc.affected(l)), (name, b, l)
+    full = orc.full()
+    for l in range(L + 1):
+        assert max_err(cl.embeddings(l, n), full[l]) <= TOL, (name, l)
+    cl.close()

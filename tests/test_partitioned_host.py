@@ -48,7 +48,7 @@ def test_router_routes_like_the_oracle_server(PT, routing):
     r = PT.Router(3, owner, src, dst, routing=PT.ROUTE_LOCALITY if routing == "locality" else PT.ROUTE_HASH,
                   hd_refresh=50, spare_local=spare, halo_capacity=n + spare)
     s = Server(3, owner, src, dst, routing=routing, hd_refresh=50)
-    stream = I.UpdateStream(n, src, dst, 4, 3)
+    stream = I.UpdateStream(n, src, dst, 4, 3, mix=(0.38, 0.38, 0.2, 0.04))    # vertex deletions too: the router expands them
     rng = np.random.default_rng(5)
     nxt = n
     for b in range(30):
@@ -108,12 +108,12 @@ def test_new_halo_slots_are_reported_with_the_batch_that_creates_them(PT):
     assert r.batch(0)[4].size == 0 and r.batch(0)[3] == 2                # nothing new, next free slot is 2
 
 
-def test_router_refuses_vertex_deletions_bad_ids_and_overflow(PT):
+def test_router_refuses_bad_ids_unknown_ops_and_overflow(PT):
     from paper_2601_12347_b200 import ripple
     owner = np.array([0, 0, 1, 1, -1, -1], dtype=np.int32)
     src, dst = np.array([0], dtype=np.int32), np.array([1], dtype=np.int32)
     r = PT.Router(2, owner, src, dst, halo_capacity=1, spare_local=0)
-    for bad in ([(I.OP_DEL_VERTEX, 0, 0)], [(I.OP_ADD_EDGE, 0, 9)], [(7, 0, 1)]):
+    for bad in ([(I.OP_DEL_VERTEX, 9, 0)], [(I.OP_ADD_EDGE, 0, 9)], [(7, 0, 1)]):
         with pytest.raises(ripple.RippleError):
             r.route(ups_array(bad))
     r.route(ups_array([(I.OP_ADD_EDGE, 0, 2)]))
@@ -158,7 +158,7 @@ def _rank_main(rank, world, port, out):
         ops = [(i, int(x["op"]), router.global_id(rank, int(x["u"])),
                 router.global_id(rank, int(x["v"])) if x["op"] != I.OP_SET_FEATURE else int(x["v"]), bool(c == 0))
                for i, (x, c) in enumerate(zip(lu, nc))]
-        A, old = me.apply(ops, rows[row_of] if row_of.size else rows[:0])
+        A, old = me.apply(ops, PT.payload_rows(rows, row_of, 5) if row_of.size else rows[:0])
         dist.barrier()
         for l in range(1, L + 1):
             halo = me.send(l, A, old)
