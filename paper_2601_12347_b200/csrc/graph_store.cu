@@ -165,12 +165,13 @@ __global__ void k_expand_copy(ripple_update* ups, int32_t* op_seq, Ctl* ctl, Sid
 
 __device__ __forceinline__ void d_classify(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, int N,
                                            Ctl* ctl, unsigned long long* hkeys, unsigned long long* hwin, int hmask,
-                                           int32_t* op_slot, int32_t* feat_last, int32_t* vdel_seq) {
+                                           int32_t* op_slot, int32_t* feat_last, int32_t* vdel_seq, int no_vertex_ops) {
     const int n = ops_total(ctl), n_given = ctl->n_ops;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
         ripple_update op = ups[i];
         op_slot[i] = -1;
-        if (op.op < 0 || op.op > 3) {
+        // (a worker of a partitioned execution takes no vertex deletion: its router has turned them into edge deletions)
+        if (op.op < 0 || op.op > 3 || (no_vertex_ops && op.op == RIPPLE_OP_DEL_VERTEX)) {
             atomicCAS(&ctl->err, 0, (int)RIPPLE_ERR_INVALID_ARG);
             ctl->abort = 1;
             continue;
@@ -216,9 +217,9 @@ __device__ __forceinline__ void d_classify(const ripple_update* __restrict__ ups
 
 __global__ void k_classify(const ripple_update* __restrict__ ups, const int32_t* __restrict__ op_seq, int N,
                            Ctl* ctl, unsigned long long* hkeys, unsigned long long* hwin, int hmask,
-                           int32_t* op_slot, int32_t* feat_last, int32_t* vdel_seq) {
+                           int32_t* op_slot, int32_t* feat_last, int32_t* vdel_seq, int no_vertex_ops) {
     pdl_enter();
-    d_classify(ups, op_seq, N, ctl, hkeys, hwin, hmask, op_slot, feat_last, vdel_seq);
+    d_classify(ups, op_seq, N, ctl, hkeys, hwin, hmask, op_slot, feat_last, vdel_seq, no_vertex_ops);
 }
 
 // Position of x in row [base, base + deg), or -1; the whole block calls this.  Rows start on
@@ -428,7 +429,7 @@ void graph_batch_classify(Ctx* c, int n) {
                   c->side[1], c->vjobs);
     }
     RP_LAUNCH(c, k_classify, grid_ops, T, 0, c->ups_dev, c->op_seq, c->N, c->ctl, c->hkeys, c->hwin,
-              c->hsize - 1, c->op_slot, c->feat_last, c->vdel_seq);
+              c->hsize - 1, c->op_slot, c->feat_last, c->vdel_seq, (int)(c->n_local > 0));
     int grid = std::min(n, c->n_sm * 8);
     RP_LAUNCH(c, k_resolve, grid, T, 0, c->ups_dev, c->op_seq, c->ctl, c->hwin, c->op_slot, c->feat_last,
               c->vdel_seq, c->side[0], c->side[1], c->rec, c->bitmap,
@@ -693,7 +694,7 @@ k_apply_small(Ctl* ctl, const int* params, const ripple_update* __restrict__ ups
     __shared__ int s_n;
     if (threadIdx.x == 0) { d_ctl_reset(ctl, params); s_n = 0; }
     __syncthreads();
-    d_classify(ups, op_seq, N, ctl, hkeys, hwin, hmask, op_slot, feat_last, vdel_seq);
+    d_classify(ups, op_seq, N, ctl, hkeys, hwin, hmask, op_slot, feat_last, vdel_seq, 0);
     __syncthreads();
     d_resolve(ups, op_seq, ctl, hwin, op_slot, feat_last, vdel_seq, out, in, rec, bitmap, op_w, grow_out, grow_in,
               shrink_out, shrink_in, nullptr);
