@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(256)
 k_att_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64_t* __restrict__ coff, Side out,
            const int32_t* __restrict__ posmap, const float* __restrict__ Hprev, const float* __restrict__ Old, int ld_h,
            const float* __restrict__ s_old, const float* __restrict__ att_s, const float* __restrict__ att_t,
-           float slope, int d, int ld, float* dS) {
+           float slope, int d, int ld, float* dS, uint32_t* bitmap) {
     pdl_enter();
     if (ctl->abort) return;
     const int nC = ctl->nC[l - 1];
@@ -109,6 +109,10 @@ k_att_push(Ctl* ctl, int l, const int32_t* __restrict__ senders, const int64_t* 
                 const float mine_t = have ? att_t[mine] : 0.f;
                 const int mine_skip = have ? (posmap[mine] >= 0) : 1;
                 const int cnt = min(32, cnt_total - j0);
+                if (have) {   // every sink joins the hop's frontier: the same walk as the frontier's own
+                    const uint32_t m = 1u << (mine & 31);
+                    if (!(bitmap[mine >> 5] & m)) atomicOr(&bitmap[mine >> 5], m);
+                }
                 for (int j = 0; j < cnt; j += EPI) {
                     const int jj = j + sub;
                     const int v = __shfl_sync(FULL, mine, jj & 31);
@@ -377,23 +381,25 @@ void att_full(Ctx* c, int l) {
 }
 
 // hop l of a batch, up to the cached rows; att_update then writes the embeddings
-void att_hop(Ctx* c, int l, int n) {
+void att_hop(Ctx* c, int l, int n, bool small) {
     const LayerDev& ly = c->layer[l];
     const int ld = c->ws[l], T = 256;
     const int32_t* senders = c->Clist[(l - 1) & 1];   // = A_{l-1}, entered in the position map
     const float* Old = c->D[(l - 1) & 1];             // their rows before this batch, in list order
-    frontier_mark(c, l, true, n);
-    frontier_compact(c, l);
     RP_LAUNCH(c, k_att_scalars, c->n_sm * 4, T, 0, c->ctl, senders, (const int*)&c->ctl->nC[l - 1], 0, c->H[l - 1],
               c->ld[l - 1], ly.W1, c->att_s[l], c->att_t[l], c->att_so);
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
-#define PUSH(NV, LPR) RP_LAUNCH(c, (k_att_push<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, senders, c->coff, c->side[0], c->posmap, c->H[l - 1], Old, c->ld[l - 1], c->att_so, c->att_s[l], c->att_t[l], ly.eps, ly.d_in, ld, c->dS[l])
+#define PUSH(NV, LPR) RP_LAUNCH(c, (k_att_push<NV, LPR>), c->n_sm * 8, T, 0, c->ctl, l, senders, c->coff, c->side[0], c->posmap, c->H[l - 1], Old, c->ld[l - 1], c->att_so, c->att_s[l], c->att_t[l], ly.eps, ly.d_in, ld, c->dS[l], c->bitmap)
     RP_WIDTH_DISPATCH(ld, PUSH);
 #undef PUSH
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
     if (n > 0)
         RP_LAUNCH(c, k_att_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, c->rec, c->posmap,
                   c->H[l - 1], Old, c->ld[l - 1], c->att_so, c->att_s[l], c->att_t[l], ly.eps, ly.d_in, ld, c->dS[l]);
+    // the list A_l: the message walk has marked the sinks it reached, the rest is marked here
+    frontier_mark_extras(c, l);
+    if (small) frontier_compact_small(c, l);   // (a handful of updates on a graph whose bitmap one block can sweep)
+    else frontier_compact(c, l);
     RP_LAUNCH(c, k_att_fold, c->n_sm * 8, T, 0, c->ctl, l, c->A[l], (const int*)&c->ctl->nA[l], 0, 0, ld, c->S[l],
               c->dS[l], c->Eb[l], c->rebuild_tau2, c->side[1].deg, c->posmap, c->att_items, ly.d_in, ly.act, c->H[l],
               c->ld[l], l == c->L ? (float*)nullptr : c->D[l & 1], c->bitmap);   // (the bitmap is free between two hops' markings)

@@ -363,6 +363,12 @@ k_senders_small(Ctl* ctl, int l, const int32_t* __restrict__ list, const int32_t
     }
 }
 
+// the members of A_l that no walk of out-lists finds: sinks of edge changes, A_{l-1} for models with a self term
+void frontier_mark_extras(Ctx* c, int l) {
+    RP_LAUNCH(c, k_mark_frontier, c->n_sm * 2, 256, 0, c->ctl, l, (int)c->self_term, 0, c->Clist[(l - 1) & 1], c->coff,
+              c->side[0], c->rec, c->A[l - 1], c->bitmap);
+}
+
 void frontier_compact_small(Ctx* c, int l) {
     RP_LAUNCH(c, k_frontier_small, 1, 1024, 0, c->ctl, l, c->bitmap, c->n_words, c->A[l], (const int32_t*)c->side[1].deg);
 }

@@ -78,6 +78,11 @@ __device__ __forceinline__ void update_few_rows(const UpdParams& p, int n_all, f
     }
 }
 
+// FEW: the instantiation that small batches launch also holds the few-row form.  Large batches launch the one
+// without it: with the few-row code inlined beside it the tiled form, unchanged in registers and shared memory,
+// made a batch of 1000 updates on the dense graph 0.3 ms slower (1.65 -> 2.0 ms) once the kernels of the chain
+// overlap their launches, and calling the few-row form out of line cost the small batches 10 us of the 30 it saves.
+template <bool FEW>
 __global__ void __launch_bounds__(256)
 k_update_rows(const Ctl* ctl, UpdParams p) {
     pdl_enter();
@@ -88,7 +93,7 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
     __shared__ float row_scale[BM];
     const int n = upd_rows(p);
     if (upd_use_tc(p, n)) return;
-    if (upd_few(p, n)) {
+    if (FEW && upd_few(p, n)) {
         static_assert(sizeof(As) >= sizeof(float) * FEW_ROWS * FEW_K && sizeof(Bs) >= sizeof(float) * 8 * FEW_ROWS * FEW_COLS,
                       "the few-row form borrows the tiles' shared memory");
         update_few_rows(p, n, &As[0][0], &Bs[0][0], row_id, row_scale);
@@ -198,7 +203,8 @@ static void launch_update(Ctx* c, UpdParams& p, const TcW& tw) {
         RP_LAUNCH(c, k_update_rows_elementwise, c->n_sm * 8, 256, 0, c->ctl, p);
         return;
     }
-    RP_LAUNCH(c, k_update_rows, c->n_sm * 4, 256, 0, c->ctl, p);
+    if (c->few_rows_form && p.list) RP_LAUNCH(c, k_update_rows<true>, c->n_sm * 4, 256, 0, c->ctl, p);
+    else RP_LAUNCH(c, k_update_rows<false>, c->n_sm * 4, 256, 0, c->ctl, p);
     if (p.tc_mode != TC_OFF) launch_update_tc(c, p);
 }
 

@@ -464,11 +464,12 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
     if (c->attention) {
         // hybrid-incremental hops of attention layers (Sec. 3.4.1)
         for (int l = 1; l <= L; ++l) {
+            const bool small = tiny && c->n_words <= RP_TINY_WORDS;
             STAMP();
-            att_hop(c, l, nb);
+            att_hop(c, l, nb, small);
             STAMP();
             att_update(c, l, false);
-            if (l < L) senders_build(c, l, nb);
+            if (l < L) { if (small) senders_build_small(c, l); else senders_build(c, l, nb); }
             STAMP();
         }
     }
@@ -627,6 +628,7 @@ extern "C" ripple_status ripple_apply_batch_weighted(ripple_ctx* ctx, const ripp
     // chain holds them), and the kernels read them where they land.
     const bool packed = mem == RIPPLE_MEM_HOST && !wide && nb >= 1 && nb <= RP_GRAPH_MAX_BATCH && nr <= RP_GRAPH_MAX_BATCH;
     c->packed_now = packed;
+    c->few_rows_form = nb <= 128;
     if (packed) {
         auto pad16 = [](size_t x) { return (x + 15) & ~(size_t)15; };
         const size_t off_ups = 16, off_w = off_ups + pad16(sizeof(ripple_update) * (size_t)nb);
@@ -893,6 +895,7 @@ extern "C" ripple_status ripple_reserve_vertices(ripple_ctx* ctx, int64_t num_ve
         c->launches = 0;
         c->debug_tc_withhold = 0;
         c->tc_armed = 1;
+        c->few_rows_form = count <= 256;
         c->params_host[0] = 0; c->params_host[1] = 0;
         cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream);
         RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
@@ -1077,6 +1080,7 @@ extern "C" ripple_status ripple_part_begin(ripple_ctx* ctx, const ripple_update*
     c->has_opw = 0;
     c->debug_tc_withhold = 0;
     c->tc_armed = 1;
+    c->few_rows_form = nb <= 128;
     for (int l = 0; l <= c->L; ++l) c->rebuild_armed[l] = 0;
     if (nb) cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, kind, c->stream);
     c->has_silent = no_compute && nb;

@@ -232,6 +232,7 @@ struct Ctx {
     char* stage_dev;
     size_t stage_bytes;
     int packed_now;    // the batch being applied arrived through the packed staging buffer
+    int few_rows_form; // the batch being applied is small: its row updates carry the few-row form (see k_update_rows)
     int* params_dev;   // {n_ops, n_rows} of the batch being applied
     int* params_host;  // pinned
     int no_graphs;
@@ -300,6 +301,7 @@ void scan_degrees(Ctx* c, const int32_t* list, const int* n_dev, int n_host, con
                   int64_t* out, unsigned long long* total_dev);
 void frontier_seed_features(Ctx* c, int n);             // A_0 from the batch's feature updates
 void frontier_mark(Ctx* c, int l, bool walk, int n);    // bitmap of A_l: (walk) edge-record sinks, A_{l-1} and Out(C_{l-1}); rebuilding hops: bottom-up
+void frontier_mark_extras(Ctx* c, int l);               // marks only what no walk finds (for hops whose message walk marks its sinks itself)
 void frontier_compact(Ctx* c, int l);                   // bitmap -> ascending list A_l
 void frontier_compact_small(Ctx* c, int l);              // the same in one block (tiny batches, small graphs)
 void senders_build_small(Ctx* c, int l);                // C_l = A_l with its degree prefix, in one block
@@ -321,7 +323,7 @@ void fold_deltas(Ctx* c, int l);                        // S^l += dS^l, dS^l = 0
 
 // attention.cu (attention layers, Sec. 3.4.1)
 void att_full(Ctx* c, int l);                           // bootstrap: logit halves, cached rows, embeddings of every vertex
-void att_hop(Ctx* c, int l, int n);                     // frontier, messages, recomputation: cached rows of A_l
+void att_hop(Ctx* c, int l, int n, bool small);         // frontier, messages, recomputation: cached rows of A_l
 void att_update(Ctx* c, int l, bool full);              // h^l = numerator / denominator on the rows of A_l; keeps the old rows
 
 // partition.cu (partitioned execution, Sec. 4)
