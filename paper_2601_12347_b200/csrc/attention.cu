@@ -267,7 +267,7 @@ k_att_gather(Ctl* ctl, int l, const int2* __restrict__ items, Side in, const flo
             const int mine = have ? in.col[base + j0 + lane] : 0;
             const float mine_e = have ? att_weight(att_s[mine], t, slope) : 0.f;
             const int cnt = min(32, j_end - j0);
-            constexpr int UNR = 4;   // neighbour rows in flight per lane group
+            constexpr int UNR = NV == 1 ? 8 : 4;   // neighbour rows in flight per lane group
             for (int j = 0; j < cnt; j += UNR * EPI) {
                 int u[UNR];
                 float e[UNR];
