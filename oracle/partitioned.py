@@ -185,7 +185,7 @@ class Worker:
         self.rank, self.model, self.weights = rank, model, weights
         self.L = len(model.layers)
         self.dims = [model.layers[0].d_in] + [l.d_out for l in model.layers]
-        self.out: Dict[int, set] = {}       # local source -> sinks (global ids, local or halo)
+        self.out: Dict[int, Dict[int, float]] = {}   # local source -> {sink (global id, local or halo): stored edge weight}
         self.deg_in: Dict[int, int] = {}    # local sink -> in-degree over ALL sources (local and remote)
         self.H: List[Dict[int, np.ndarray]] = [dict() for _ in range(self.L + 1)]
         self.S: List[Dict[int, np.ndarray]] = [dict() for _ in range(self.L + 1)]
@@ -196,7 +196,7 @@ class Worker:
 
     def add_vertex(self, v: int, x: np.ndarray):
         """A placed vertex: feature row x, no edges yet; its rows are those of an isolated vertex."""
-        self.out[v] = set()
+        self.out[v] = {}
         self.deg_in[v] = 0
         self.H[0][v] = np.array(x, dtype=np.float64)
         for l in range(1, self.L + 1):
@@ -204,29 +204,31 @@ class Worker:
             self.H[l][v] = _update(self.model.layers[l - 1], self.weights[l - 1], self.H[l - 1][v], self.S[l][v])
 
     # -- apply (Sec. 4.5): topology and features; returns what the hops need -------------------------
-    def apply(self, ops, feat_rows):
-        self.added, self.deleted = [], []          # net edge changes this worker computes for
+    def apply(self, ops, feat_rows, op_w=None):
+        """op_w: one weight per operation of the whole batch (stored edge weights; an added edge takes the
+        weight given with its operation, an edge that exists keeps the one it has), or None: all ones."""
+        self.added, self.deleted = [], []          # net edge changes this worker computes for: (u, v, weight)
         self.old_deg_out: Dict[int, int] = {}
-        last_edge: Dict[Tuple[int, int], Tuple[int, bool]] = {}
+        last_edge: Dict[Tuple[int, int], Tuple[int, bool, int]] = {}
         last_feat: Dict[int, int] = {}
-        for (_, op, u, v, compute) in ops:         # the last operation on a pair / a vertex wins
+        for (i, op, u, v, compute) in ops:         # the last operation on a pair / a vertex wins
             if op == OP_SET_FEATURE:
                 last_feat[u] = v
             else:
-                last_edge[(u, v)] = (op, compute)
-        touched_sinks = set()
-        for (u, v), (op, compute) in sorted(last_edge.items()):
+                last_edge[(u, v)] = (op, compute, i)
+        for (u, v), (op, compute, i) in sorted(last_edge.items()):
             src_local, dst_local = self.is_local(u), self.is_local(v)
             present = (v in self.out[u]) if src_local else None
             if src_local:
                 if op == OP_ADD_EDGE and not present:
                     self.old_deg_out.setdefault(u, len(self.out[u]))
-                    self.out[u].add(v); self.added.append((u, v))
+                    w = float(op_w[i]) if op_w is not None else 1.0
+                    self.out[u][v] = w; self.added.append((u, v, w))
                     if dst_local:
                         self.deg_in[v] += 1
                 elif op == OP_DEL_EDGE and present:
                     self.old_deg_out.setdefault(u, len(self.out[u]))
-                    self.out[u].discard(v); self.deleted.append((u, v))
+                    self.deleted.append((u, v, self.out[u].pop(v)))
                     if dst_local:
                         self.deg_in[v] -= 1
             else:
@@ -263,7 +265,7 @@ class Worker:
         senders = set(A_prev)
         if agg == AGG_WSUM_GCN:
             senders |= set(self.old_deg_out.keys())
-        added = set(self.added)
+        added = {(u, v) for (u, v, _) in self.added}
         for u in sorted(senders):
             hn = self.H[l - 1][u]
             ho = old_prev.get(u, hn)
@@ -272,12 +274,12 @@ class Worker:
             m = cn * hn - co * ho
             for v in sorted(self.out[u]):
                 if (u, v) not in added:
-                    deliver(v, m)
-        for (u, v) in self.added:      # the whole new term arrives
-            deliver(v, _coef(agg, len(self.out[u])) * self.H[l - 1][u])
-        for (u, v) in self.deleted:    # the whole old term leaves
+                    deliver(v, self.out[u][v] * m)     # the edge's stored weight scales the message (Sec. 3.3.3)
+        for (u, v, w) in self.added:      # the whole new term arrives
+            deliver(v, w * _coef(agg, len(self.out[u])) * self.H[l - 1][u])
+        for (u, v, w) in self.deleted:    # the whole old term leaves
             ho = old_prev.get(u, self.H[l - 1][u])
-            deliver(v, -_coef(agg, self.old_deg_out[u]) * ho)
+            deliver(v, -w * _coef(agg, self.old_deg_out[u]) * ho)
         return halo
 
     def receive(self, msgs: Dict[int, np.ndarray]):
@@ -305,7 +307,7 @@ class Cluster:
     """P workers and the server; apply_batch runs the hops with one remote send per hop."""
 
     def __init__(self, n_partitions, owner, n, src, dst, X, model, weights, full_H, full_S,
-                 routing="locality", hd_refresh=500_000):
+                 routing="locality", hd_refresh=500_000, edge_weights=None):
         """full_H / full_S: embeddings and aggregates of the initial graph (the state every worker
         starts from is given, as in Sec. 4.1: computed before the stream starts, then partitioned)."""
         self.P = n_partitions
@@ -319,29 +321,30 @@ class Cluster:
             if p < 0:
                 continue
             w = self.workers[p]
-            w.out[v] = set()
+            w.out[v] = {}
             w.deg_in[v] = 0
             for l in range(L + 1):
                 w.H[l][v] = np.array(full_H[l][v], dtype=np.float64)
                 if l:
                     w.S[l][v] = np.array(full_S[l][v], dtype=np.float64)
-        for u, v in zip(src.tolist(), dst.tolist()):
+        ew = edge_weights.tolist() if edge_weights is not None else [1.0] * int(src.size)
+        for u, v, a in zip(src.tolist(), dst.tolist(), ew):
             pu, pv = int(owner[u]), int(owner[v])
-            self.workers[pu].out[u].add(v)
+            self.workers[pu].out[u][v] = float(a)
             self.workers[pv].deg_in[v] += 1
             if pu != pv:
                 self.workers[pv].remote_in.setdefault(v, set()).add(u)
         self.affected: List[List[int]] = []
         self.halo_rows_sent: List[int] = []
 
-    def apply_batch(self, ups: np.ndarray, feat_rows: np.ndarray):
+    def apply_batch(self, ups: np.ndarray, feat_rows: np.ndarray, op_w=None):
         L = len(self.model.layers)
         before = self.server.owner.copy()
         routed = self.server.route(ups)
         d0 = self.model.layers[0].d_in
         for v in np.nonzero((before < 0) & (self.server.owner >= 0))[0].tolist():   # vertices the batch created
             self.workers[int(self.server.owner[v])].add_vertex(v, np.zeros(d0))
-        state = [w.apply(routed[r], feat_rows) for r, w in enumerate(self.workers)]
+        state = [w.apply(routed[r], feat_rows, op_w) for r, w in enumerate(self.workers)]
         A = [s[0] for s in state]
         old = [s[1] for s in state]
         self.affected = [sorted(sum(A, []))]

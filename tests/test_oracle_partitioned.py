@@ -252,3 +252,29 @@ def test_cluster_with_vertex_deletions_equals_single_machine(name, P):
         for l in range(L + 1):
             assert rel_err(cl.gather(l, n), full[l]) < 1e-9, (name, P, b, l)
             assert cl.affected[l] == orc.affected(l).tolist(), (name, P, b, l)
+
+
+# ---------------------------------------------------------------------------------------------
+# stored edge weights (the paper's GC-W runs distributed too, Sec. 6.3.1)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("P", [2, 3])
+def test_cluster_with_stored_edge_weights_equals_single_machine(P):
+    n = 60
+    model = I.graphconv_model([5, 6, 6, 3], I.AGG_WSUM_EDGE)
+    src, dst = I.er_graph(n, 240, 9)
+    ew = I.edge_weights(src.size, 9)
+    X = I.features(n, 5, 9)
+    W = I.make_weights(model, 9, zero_bias=False)
+    orc = Oracle(n, src, dst, X, model, W, edge_weights=ew)
+    owner = np.random.default_rng(9).integers(0, P, size=n)
+    cl = Cluster(P, owner, n, src, dst, X, model, W, orc.full(), [None] + [orc.full_S(l) for l in (1, 2, 3)],
+                 edge_weights=ew)
+    stream = I.UpdateStream(n, src, dst, 5, 9)
+    for b in range(10):
+        ups, rows, ow = stream.next_batch_weighted(1 + 4 * (b % 3))
+        cl.apply_batch(ups, rows, ow)
+        assert orc.apply_incremental(ups, rows, op_weights=ow) == 0
+        full = orc.full()
+        for l in range(4):
+            assert rel_err(cl.gather(l, n), full[l]) < 1e-10, (P, b, l)
+            assert cl.affected[l] == orc.affected(l).tolist()
