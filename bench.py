@@ -577,7 +577,7 @@ def run_partitioned(args):
                     return worst
 
                 def begin(r, wk):
-                    lu, nc, row_of, first, ho, hr = shares[r]
+                    lu, nc, row_of, first, ho, hr, _ = shares[r]
                     if ho.size:
                         wk.set_halos(first, ho, hr)
                     wk.begin(lu, PT.payload_rows(rows, row_of, wk.dims[0]), nc)

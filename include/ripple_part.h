@@ -25,8 +25,8 @@
  *                          every worker process runs its own replica on the same stream, so no server
  *                          process and no routing messages exist.
  *
- * What a partitioned context supports: the linear aggregators SUM, MEAN, WSUM_GCN with SAGE, GRAPHCONV
- * and GIN layers; edge additions, edge deletions and feature replacements (the router turns a vertex
+ * What a partitioned context supports: the linear aggregators SUM, MEAN, WSUM_GCN and WSUM_EDGE (stored edge
+ * weights: a cut edge keeps its weight at both workers) with SAGE, GRAPHCONV and GIN layers; edge additions, edge deletions and feature replacements (the router turns a vertex
  * deletion into these; a worker given one answers RIPPLE_ERR_INVALID_ARG).  Hops always take the delta
  * form (push); the rounding budget is off (a row cannot be gathered anew without its remote
  * in-neighbours' rows).  ripple_apply_batch and ripple_recompute_full are refused on such a context.
@@ -100,9 +100,10 @@ ripple_status ripple_part_set_halos(ripple_ctx* ctx, int32_t first, int32_t coun
  * when done.  Every worker must have finished layer l - 1 before any worker starts layer l. */
 ripple_status ripple_part_bootstrap_layer(ripple_ctx* ctx, int32_t l);
 
-/* One batch, in phases (Sec. 4.5).  ups / feat_rows / no_compute as in ripple_apply_batch (HOST|DEVICE
- * per mem), in local ids; no_compute[i] != 0 marks the copy of a cut edge that the SINK's worker
- * receives: it updates the adjacency and the degrees and sends nothing (may be NULL: none).
+/* One batch, in phases (Sec. 4.5).  ups / feat_rows / no_compute / edge_weights as in ripple_apply_batch_weighted
+ * (HOST|DEVICE per mem), in local ids; no_compute[i] != 0 marks the copy of a cut edge that the SINK's worker
+ * receives: it updates the adjacency and the degrees and sends nothing (may be NULL: none); edge_weights[i] is the
+ * weight of the edge that operation i adds (RIPPLE_AGG_WSUM_EDGE only; NULL: ones).
  *   begin        Apply: normalise the batch, mutate the partition, replace features, list hop-0 senders
  *   hop_send     l = 1..L: prepare + local send + combine, then the remote send of the halo mailboxes
  *   hop_compute  l = 1..L: aggregate what arrived, update the local hop-l vertices, list the next senders
@@ -111,7 +112,7 @@ ripple_status ripple_part_bootstrap_layer(ripple_ctx* ctx, int32_t l);
  * must have returned from hop_send(l); between hop_compute(l) and hop_send(l + 1) no barrier is needed.
  * A batch rejected by begin (status != OK) must not be followed by the other phases. */
 ripple_status ripple_part_begin(ripple_ctx* ctx, const ripple_update* ups, int64_t n, const float* feat_rows,
-                                int64_t n_rows, const uint8_t* no_compute, int32_t mem);
+                                int64_t n_rows, const uint8_t* no_compute, const float* edge_weights, int32_t mem);
 ripple_status ripple_part_hop_send(ripple_ctx* ctx, int32_t l);
 ripple_status ripple_part_hop_compute(ripple_ctx* ctx, int32_t l);
 ripple_status ripple_part_end(ripple_ctx* ctx);
@@ -141,17 +142,20 @@ void ripple_router_destroy(ripple_router* r);
 ripple_status ripple_router_partition_shape(ripple_router* r, int32_t rank, int64_t* n_local,
                                             int64_t* num_vertices, int64_t* num_edges, int64_t* halos_used);
 
-/* The partition itself, in local ids: src_local / dst_local (num_edges entries), global_of
- * (num_vertices entries: the global id behind every local id, -1 for unused ones), halo_owner /
- * halo_remote_id (halos_used entries, for ripple_part_set_halos). */
+/* The partition itself, in local ids: src_local / dst_local (num_edges entries), edge_of (num_edges entries,
+ * may be NULL: the index, in the arrays given to ripple_router_create, of the edge behind each local edge --
+ * for per-edge data such as stored weights), global_of (num_vertices entries: the global id behind every
+ * local id, -1 for unused ones), halo_owner / halo_remote_id (halos_used entries, for ripple_part_set_halos). */
 ripple_status ripple_router_partition_fill(ripple_router* r, int32_t rank, int32_t* src_local, int32_t* dst_local,
-                                           int32_t* global_of, int32_t* halo_owner, int32_t* halo_remote_id);
+                                           int64_t* edge_of, int32_t* global_of, int32_t* halo_owner,
+                                           int32_t* halo_remote_id);
 
 /* Routes a batch given in global ids.  Afterwards, per worker, ripple_router_batch_shape gives the
  * number of operations, payload rows and halo slots assigned by this batch, and ripple_router_batch_fill
- * the operations in local ids (in batch order), their no-compute flags, for every payload row of the
- * worker the index of the global payload row it is a copy of, and the new halo slots (first slot index
- * in *first_halo).  A payload row index of -1 in row_of stands for a row of zeros.
+ * the operations in local ids (in batch order), their no-compute flags, for every operation the position in
+ * the routed batch of the operation it comes from (op_of, may be NULL: for per-operation data such as edge
+ * weights), for every payload row of the worker the index of the global payload row it is a copy of, and
+ * the new halo slots (first slot index in *first_halo).  A payload row index of -1 in row_of stands for a row of zeros.
  * A vertex deletion (Sec. 4.3 routes it to the owner and says no more) is replaced, at its position in the
  * batch, by one edge deletion per incident edge -- the router keeps the edge lists for this -- each routed
  * like any edge deletion, and a feature update of the vertex with a row of zeros; the workers never see
@@ -163,7 +167,7 @@ ripple_status ripple_router_route(ripple_router* r, const ripple_update* ups, in
 ripple_status ripple_router_batch_shape(ripple_router* r, int32_t rank, int64_t* n_ops, int64_t* n_rows,
                                         int64_t* n_new_halos);
 ripple_status ripple_router_batch_fill(ripple_router* r, int32_t rank, ripple_update* ups_local, uint8_t* no_compute,
-                                       int32_t* row_of, int32_t* first_halo, int32_t* halo_owner,
+                                       int32_t* op_of, int32_t* row_of, int32_t* first_halo, int32_t* halo_owner,
                                        int32_t* halo_remote_id);
 
 /* Look-ups: the global id behind every local id of a worker as of now (global_of: HOST, capacity >= the

@@ -166,7 +166,8 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         if (o.slack <= 0) o.slack = 0.25;
         if (o.max_batch <= 0) o.max_batch = 16384;
         if (o.n_local != 0) {   // one worker of a partitioned execution
-            const bool linear = agg == RIPPLE_AGG_SUM || agg == RIPPLE_AGG_MEAN || agg == RIPPLE_AGG_WSUM_GCN;
+            const bool linear = agg == RIPPLE_AGG_SUM || agg == RIPPLE_AGG_MEAN || agg == RIPPLE_AGG_WSUM_GCN ||
+                                agg == RIPPLE_AGG_WSUM_EDGE;
             if (o.n_local < 0 || (o.n_local & 31) || o.n_local > g->num_vertices || !linear ||
                 layers[0].kind > RIPPLE_LAYER_GIN) {
                 set_err(nullptr, "a partitioned context needs n_local a multiple of 32 within num_vertices, a linear aggregator and SAGE, GRAPHCONV or GIN layers");
@@ -1058,7 +1059,8 @@ extern "C" ripple_status ripple_part_bootstrap_layer(ripple_ctx* ctx, int32_t l)
 }
 
 extern "C" ripple_status ripple_part_begin(ripple_ctx* ctx, const ripple_update* ups, int64_t n, const float* feat_rows,
-                                           int64_t n_rows, const uint8_t* no_compute, int32_t mem) {
+                                           int64_t n_rows, const uint8_t* no_compute, const float* edge_weights,
+                                           int32_t mem) {
     Ctx* c = worker(ctx);
     if (!c || n < 0 || n_rows < 0 || (n > 0 && !ups) || (n_rows > 0 && !feat_rows) || (mem != 0 && mem != 1))
         return RIPPLE_ERR_INVALID_ARG;
@@ -1077,7 +1079,7 @@ extern "C" ripple_status ripple_part_begin(ripple_ctx* ctx, const ripple_update*
     const cudaMemcpyKind kind = mem == RIPPLE_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
     c->launches = 0;
     c->may_expand = 0;
-    c->has_opw = 0;
+    c->has_opw = c->weighted && edge_weights && nb;
     c->debug_tc_withhold = 0;
     c->tc_armed = 1;
     c->few_rows_form = nb <= 128;
@@ -1085,6 +1087,7 @@ extern "C" ripple_status ripple_part_begin(ripple_ctx* ctx, const ripple_update*
     if (nb) cudaMemcpyAsync(c->ups_dev, ups, sizeof(ripple_update) * (size_t)nb, kind, c->stream);
     c->has_silent = no_compute && nb;
     if (c->has_silent) cudaMemcpyAsync(c->silent_dev, no_compute, (size_t)nb, kind, c->stream);
+    if (c->has_opw) cudaMemcpyAsync(c->opw_dev, edge_weights, sizeof(float) * (size_t)nb, kind, c->stream);
     if (nr) cudaMemcpyAsync(c->feat_dev, feat_rows, sizeof(float) * (size_t)nr * c->d[0], kind, c->stream);
     c->params_host[0] = nb; c->params_host[1] = nr;
     cudaMemcpyAsync(c->params_dev, c->params_host, 2 * sizeof(int), cudaMemcpyHostToDevice, c->stream);

@@ -26,6 +26,7 @@ struct Part {
     // the batch being routed
     std::vector<ripple_update> ops;
     std::vector<uint8_t> no_compute;
+    std::vector<int32_t> op_of;      // position in the routed batch of the operation each local operation comes from
     std::vector<int32_t> row_of;
     int64_t first_new_halo = 0;
 };
@@ -46,6 +47,7 @@ struct ripple_router {
     // of vertex deletions
     std::vector<std::vector<int32_t>> out_adj, in_adj;
 
+    int32_t cur_pos = 0;   // position in the batch of the operation being routed
     void count_update() { if (++seen % hd_refresh == 0) refresh_high(); }
     static bool drop(std::vector<int32_t>& a, int32_t x) {
         for (size_t i = 0; i < a.size(); ++i)
@@ -67,11 +69,13 @@ struct ripple_router {
         if (lu < 0 || lv < 0) return false;
         part[pu].ops.push_back({op, lu, lv});
         part[pu].no_compute.push_back(0);
+        part[pu].op_of.push_back(cur_pos);
         if (pv != pu) {
             const int32_t su = id_at(pv, u), sv = id_at(pv, v);
             if (su < 0 || sv < 0) return false;
             part[pv].ops.push_back({op, su, sv});
             part[pv].no_compute.push_back(1);
+            part[pv].op_of.push_back(cur_pos);
         }
         if (add && !has_edge(u, v)) { in_degree[v]++; n_edges++; out_adj[u].push_back(v); in_adj[v].push_back(u); }
         else if (!add && drop(out_adj[u], v)) { in_degree[v]--; n_edges--; drop(in_adj[v], u); }
@@ -81,6 +85,7 @@ struct ripple_router {
         Part& q = part[owner[u]];
         q.ops.push_back({RIPPLE_OP_SET_FEATURE, local_id[u], (int32_t)q.row_of.size()});
         q.no_compute.push_back(0);
+        q.op_of.push_back(cur_pos);
         q.row_of.push_back(row);
     }
 
@@ -213,8 +218,8 @@ extern "C" ripple_status ripple_router_partition_shape(ripple_router* r, int32_t
 }
 
 extern "C" ripple_status ripple_router_partition_fill(ripple_router* r, int32_t rank, int32_t* src_local,
-                                                      int32_t* dst_local, int32_t* global_of, int32_t* halo_owner,
-                                                      int32_t* halo_remote_id) {
+                                                      int32_t* dst_local, int64_t* edge_of, int32_t* global_of,
+                                                      int32_t* halo_owner, int32_t* halo_remote_id) {
     if (!r || rank < 0 || rank >= r->P || !global_of) return RIPPLE_ERR_INVALID_ARG;
     Part& q = r->part[rank];
     int64_t n = 0;
@@ -224,6 +229,7 @@ extern "C" ripple_status ripple_router_partition_fill(ripple_router* r, int32_t 
         if (!src_local || !dst_local) return RIPPLE_ERR_INVALID_ARG;
         src_local[n] = r->id_at(rank, u);
         dst_local[n] = r->id_at(rank, v);
+        if (edge_of) edge_of[n] = (int64_t)e;
         ++n;
     }
     std::copy(q.global_of.begin(), q.global_of.end(), global_of);
@@ -244,11 +250,12 @@ extern "C" ripple_status ripple_router_route(ripple_router* r, const ripple_upda
         if ((x.op == RIPPLE_OP_ADD_EDGE || x.op == RIPPLE_OP_DEL_EDGE) && (x.v < 0 || x.v >= r->N)) return RIPPLE_ERR_VERTEX_RANGE;
     }
     for (Part& q : r->part) {
-        q.ops.clear(); q.no_compute.clear(); q.row_of.clear();
+        q.ops.clear(); q.no_compute.clear(); q.op_of.clear(); q.row_of.clear();
         q.first_new_halo = q.next_halo;
     }
     for (int64_t i = 0; i < n; ++i) {
         const ripple_update& x = ups[i];
+        r->cur_pos = (int32_t)i;
         if (x.op == RIPPLE_OP_SET_FEATURE) {
             if (r->owner[x.u] < 0) return RIPPLE_ERR_INVALID_ARG;   // a feature update of a vertex that is not in the graph
             r->route_feature(x.u, x.v);
@@ -283,13 +290,14 @@ extern "C" ripple_status ripple_router_batch_shape(ripple_router* r, int32_t ran
 }
 
 extern "C" ripple_status ripple_router_batch_fill(ripple_router* r, int32_t rank, ripple_update* ups_local,
-                                                  uint8_t* no_compute, int32_t* row_of, int32_t* first_halo,
-                                                  int32_t* halo_owner, int32_t* halo_remote_id) {
+                                                  uint8_t* no_compute, int32_t* op_of, int32_t* row_of,
+                                                  int32_t* first_halo, int32_t* halo_owner, int32_t* halo_remote_id) {
     if (!r || rank < 0 || rank >= r->P || !first_halo) return RIPPLE_ERR_INVALID_ARG;
     const Part& q = r->part[rank];
     if ((!q.ops.empty() && (!ups_local || !no_compute)) || (!q.row_of.empty() && !row_of)) return RIPPLE_ERR_INVALID_ARG;
     std::copy(q.ops.begin(), q.ops.end(), ups_local);
     std::copy(q.no_compute.begin(), q.no_compute.end(), no_compute);
+    if (op_of) std::copy(q.op_of.begin(), q.op_of.end(), op_of);
     std::copy(q.row_of.begin(), q.row_of.end(), row_of);
     *first_halo = (int32_t)q.first_new_halo;
     for (int64_t h = q.first_new_halo; h < q.next_halo; ++h) {

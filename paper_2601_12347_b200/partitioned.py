@@ -57,7 +57,8 @@ class Router:
             pass
 
     def partition(self, rank: int):
-        """(n_local, num_vertices, src_local, dst_local, global_of, halo_owner, halo_remote_id)."""
+        """(n_local, num_vertices, src_local, dst_local, global_of, halo_owner, halo_remote_id, edge_of):
+        edge_of[i] = index, in the arrays the router was created from, of the edge behind local edge i."""
         a, b, c, d = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
         st = self.lib.ripple_router_partition_shape(self.h, rank, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c),
                                                     ctypes.byref(d))
@@ -68,11 +69,12 @@ class Router:
         gof = np.zeros(b.value, dtype=np.int32)
         ho = np.zeros(max(d.value, 1), dtype=np.int32)
         hr = np.zeros(max(d.value, 1), dtype=np.int32)
-        st = self.lib.ripple_router_partition_fill(self.h, rank, src.ctypes.data, dst.ctypes.data, gof.ctypes.data,
-                                                   ho.ctypes.data, hr.ctypes.data)
+        eof = np.zeros(max(c.value, 1), dtype=np.int64)
+        st = self.lib.ripple_router_partition_fill(self.h, rank, src.ctypes.data, dst.ctypes.data, eof.ctypes.data,
+                                                   gof.ctypes.data, ho.ctypes.data, hr.ctypes.data)
         if st != R.OK:
             raise R.RippleError(st, "partition fill")
-        return a.value, b.value, src[: c.value], dst[: c.value], gof, ho[: d.value], hr[: d.value]
+        return a.value, b.value, src[: c.value], dst[: c.value], gof, ho[: d.value], hr[: d.value], eof[: c.value]
 
     def route(self, ups: np.ndarray) -> None:
         ups = np.ascontiguousarray(ups, dtype=R.UPDATE_DTYPE)
@@ -81,7 +83,8 @@ class Router:
             raise R.RippleError(st, "routing failed")
 
     def batch(self, rank: int):
-        """(ups_local, no_compute, row_of, first_halo, halo_owner, halo_remote_id) of the routed batch."""
+        """(ups_local, no_compute, row_of, first_halo, halo_owner, halo_remote_id, op_of) of the routed batch;
+        op_of[i] = position in the batch of the operation that local operation i comes from."""
         a, b, c = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
         st = self.lib.ripple_router_batch_shape(self.h, rank, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
         if st != R.OK:
@@ -92,11 +95,13 @@ class Router:
         ho = np.zeros(max(c.value, 1), dtype=np.int32)
         hr = np.zeros(max(c.value, 1), dtype=np.int32)
         first = ctypes.c_int32()
-        st = self.lib.ripple_router_batch_fill(self.h, rank, ups.ctypes.data, nc.ctypes.data, row_of.ctypes.data,
-                                               ctypes.byref(first), ho.ctypes.data, hr.ctypes.data)
+        op_of = np.zeros(max(a.value, 1), dtype=np.int32)
+        st = self.lib.ripple_router_batch_fill(self.h, rank, ups.ctypes.data, nc.ctypes.data, op_of.ctypes.data,
+                                               row_of.ctypes.data, ctypes.byref(first), ho.ctypes.data, hr.ctypes.data)
         if st != R.OK:
             raise R.RippleError(st, "batch fill")
-        return ups[: a.value], nc[: a.value], row_of[: b.value], first.value, ho[: c.value], hr[: c.value]
+        return (ups[: a.value], nc[: a.value], row_of[: b.value], first.value, ho[: c.value], hr[: c.value],
+                op_of[: a.value])
 
     def global_ids(self, rank: int, num_vertices: int) -> np.ndarray:
         """The global id behind every local id of worker `rank` (locals, then halo slots; -1: unused)."""
@@ -150,15 +155,20 @@ class Worker(R.Ripple):
     def bootstrap_layer(self, l: int) -> None:
         self._check(self.lib.ripple_part_bootstrap_layer(self.h, int(l)))
 
-    def begin(self, ups: np.ndarray, rows: Optional[np.ndarray], no_compute: np.ndarray) -> None:
+    def begin(self, ups: np.ndarray, rows: Optional[np.ndarray], no_compute: np.ndarray,
+              op_weights: Optional[np.ndarray] = None) -> None:
         ups = np.ascontiguousarray(ups, dtype=R.UPDATE_DTYPE)
         no_compute = np.ascontiguousarray(no_compute, dtype=np.uint8)
+        wptr = None
+        if op_weights is not None and ups.size:
+            op_weights = np.ascontiguousarray(op_weights, dtype=np.float32)
+            wptr = op_weights.ctypes.data
         nr, fptr = 0, None
         if rows is not None and rows.shape[0]:
             rows = np.ascontiguousarray(rows, dtype=np.float32)
             nr, fptr = rows.shape[0], rows.ctypes.data
         self._check(self.lib.ripple_part_begin(self.h, ups.ctypes.data if ups.size else None, ups.size, fptr, nr,
-                                               no_compute.ctypes.data if ups.size else None, R.MEM_HOST))
+                                               no_compute.ctypes.data if ups.size else None, wptr, R.MEM_HOST))
 
     def hop_send(self, l: int) -> None:
         self._check(self.lib.ripple_part_hop_send(self.h, int(l)))
@@ -187,8 +197,10 @@ def payload_rows(rows: Optional[np.ndarray], row_of: np.ndarray, d0: int) -> Opt
     return out
 
 
-def _make_worker(router: Router, rank: int, X: np.ndarray, model, weights, **kw) -> Tuple[Worker, np.ndarray]:
-    n_local, nv, src, dst, gof, ho, hr = router.partition(rank)
+def _make_worker(router: Router, rank: int, X: np.ndarray, model, weights, edge_weights=None, **kw) -> Tuple[Worker, np.ndarray]:
+    n_local, nv, src, dst, gof, ho, hr, edge_of = router.partition(rank)
+    if edge_weights is not None:      # a cut edge is held, with its weight, by both of its workers
+        kw["edge_weights"] = np.ascontiguousarray(edge_weights, dtype=np.float32)[edge_of]
     feats = np.zeros((nv, X.shape[1]), dtype=np.float32)
     own = gof[:n_local]
     feats[: n_local][own >= 0] = X[own[own >= 0]]
@@ -204,7 +216,7 @@ class Cluster:
 
     def __init__(self, n_partitions: int, owner: np.ndarray, src: np.ndarray, dst: np.ndarray, X: np.ndarray,
                  model, weights, routing: int = ROUTE_LOCALITY, hd_refresh: int = 500_000, spare_local: int = 0,
-                 halo_capacity: Optional[int] = None, devices: Optional[Sequence[int]] = None, **kw):
+                 halo_capacity: Optional[int] = None, devices: Optional[Sequence[int]] = None, edge_weights=None, **kw):
         import torch
         self._torch = torch
         self.P = int(n_partitions)
@@ -215,7 +227,7 @@ class Cluster:
         self.workers: List[Worker] = []
         for r in range(self.P):
             with torch.cuda.device(self.devices[r]):
-                w, _ = _make_worker(self.router, r, X, model, weights, **kw)
+                w, _ = _make_worker(self.router, r, X, model, weights, edge_weights=edge_weights, **kw)
             self.workers.append(w)
         exports = [w.exports() for w in self.workers]
         for w in self.workers:
@@ -230,14 +242,16 @@ class Cluster:
             w.close()
         self.router.close()
 
-    def apply_batch(self, ups: np.ndarray, rows: Optional[np.ndarray]) -> None:
-        """ups in global ids.  Every phase runs on all workers before the next begins."""
+    def apply_batch(self, ups: np.ndarray, rows: Optional[np.ndarray], op_weights: Optional[np.ndarray] = None) -> None:
+        """ups in global ids (op_weights: the weight of every added edge, graphs with stored edge weights).  Every
+        phase runs on all workers before the next begins."""
         self.router.route(ups)
         for r, w in enumerate(self.workers):
-            lu, nc, row_of, first, ho, hr = self.router.batch(r)
+            lu, nc, row_of, first, ho, hr, op_of = self.router.batch(r)
             if ho.size:
                 w.set_halos(first, ho, hr)
-            w.begin(lu, payload_rows(rows, row_of, w.dims[0]), nc)
+            w.begin(lu, payload_rows(rows, row_of, w.dims[0]), nc,
+                    np.asarray(op_weights, dtype=np.float32)[op_of] if op_weights is not None else None)
         for l in range(1, self.L + 1):
             for w in self.workers:
                 w.hop_send(l)
@@ -281,13 +295,14 @@ class DistributedWorker:
     rank's share.  Barriers separate the phases; peers are reached through CUDA IPC mappings."""
 
     def __init__(self, owner, src, dst, X, model, weights, routing: int = ROUTE_LOCALITY,
-                 hd_refresh: int = 500_000, spare_local: int = 0, halo_capacity: Optional[int] = None, **kw):
+                 hd_refresh: int = 500_000, spare_local: int = 0, halo_capacity: Optional[int] = None,
+                 edge_weights=None, **kw):
         import torch.distributed as dist
         self.dist = dist
         self.rank, self.P = dist.get_rank(), dist.get_world_size()
         self.L = len(model.layers)
         self.router = Router(self.P, owner, src, dst, routing, hd_refresh, spare_local, halo_capacity)
-        self.worker, _ = _make_worker(self.router, self.rank, X, model, weights, **kw)
+        self.worker, _ = _make_worker(self.router, self.rank, X, model, weights, edge_weights=edge_weights, **kw)
         blobs: List[Optional[bytes]] = [None] * self.P
         dist.all_gather_object(blobs, self.worker.ipc_export())
         for r, blob in enumerate(blobs):
@@ -300,12 +315,13 @@ class DistributedWorker:
             self.worker.bootstrap_layer(l)
         dist.barrier()
 
-    def apply_batch(self, ups: np.ndarray, rows: Optional[np.ndarray]) -> None:
+    def apply_batch(self, ups: np.ndarray, rows: Optional[np.ndarray], op_weights: Optional[np.ndarray] = None) -> None:
         self.router.route(ups)
-        lu, nc, row_of, first, ho, hr = self.router.batch(self.rank)
+        lu, nc, row_of, first, ho, hr, op_of = self.router.batch(self.rank)
         if ho.size:
             self.worker.set_halos(first, ho, hr)
-        self.worker.begin(lu, payload_rows(rows, row_of, self.worker.dims[0]), nc)
+        self.worker.begin(lu, payload_rows(rows, row_of, self.worker.dims[0]), nc,
+                          np.asarray(op_weights, dtype=np.float32)[op_of] if op_weights is not None else None)
         for l in range(1, self.L + 1):
             self.dist.barrier()
             self.worker.hop_send(l)

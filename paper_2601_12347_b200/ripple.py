@@ -154,17 +154,17 @@ def load_library(path: Optional[str] = None):
     lib.ripple_part_ipc_open.argtypes = [vp, i32, P(_PartIpc)]
     lib.ripple_part_set_halos.argtypes = [vp, i32, i32, vp, vp]
     lib.ripple_part_bootstrap_layer.argtypes = [vp, i32]
-    lib.ripple_part_begin.argtypes = [vp, vp, i64, vp, i64, vp, i32]
+    lib.ripple_part_begin.argtypes = [vp, vp, i64, vp, i64, vp, vp, i32]
     lib.ripple_part_hop_send.argtypes = [vp, i32]
     lib.ripple_part_hop_compute.argtypes = [vp, i32]
     lib.ripple_part_end.argtypes = [vp]
     lib.ripple_part_rows_sent.argtypes = [vp, vp]
     lib.ripple_router_create.argtypes = [i32, i64, vp, i64, vp, vp, i32, i64, i64, i64, P(vp)]
     lib.ripple_router_partition_shape.argtypes = [vp, i32, P(i64), P(i64), P(i64), P(i64)]
-    lib.ripple_router_partition_fill.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    lib.ripple_router_partition_fill.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.ripple_router_route.argtypes = [vp, vp, i64]
     lib.ripple_router_batch_shape.argtypes = [vp, i32, P(i64), P(i64), P(i64)]
-    lib.ripple_router_batch_fill.argtypes = [vp, i32, vp, vp, vp, P(i32), vp, vp]
+    lib.ripple_router_batch_fill.argtypes = [vp, i32, vp, vp, vp, vp, P(i32), vp, vp]
     lib.ripple_router_global_ids.argtypes = [vp, i32, vp, i64]
     for name in EXPORTED_PART[:18]:
         getattr(lib, name).restype = i32

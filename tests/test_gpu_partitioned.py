@@ -230,3 +230,48 @@ def test_vertex_deletions_are_expanded_by_the_router(env, name):
     for l in range(L + 1):
         assert max_err(cl.embeddings(l, n), full[l]) <= TOL, (name, l)
     cl.close()
+
+
+@pytest.mark.parametrize("P", [2, 3])
+def test_stored_edge_weights_across_partitions(env, P):
+    """The weighted sum with a stored weight per edge (the paper's GC-W, which Sec. 6.3.1 runs distributed): a cut
+    edge keeps its weight at both workers, messages into halo mailboxes are scaled by it."""
+    ripple, Oracle = env
+    from paper_2601_12347_b200.partitioned import Cluster
+    n = 700
+    model = I.graphconv_model([18, 36, 20, 10], I.AGG_WSUM_EDGE)
+    src, dst = I.er_graph(n, 5000, 8)
+    have = set(zip(src.tolist(), dst.tolist()))
+    extra = [(0, int(v)) for v in range(1, 300) if (0, int(v)) not in have]
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    ew = I.edge_weights(src.size, 8)
+    X = I.features(n, 18, 8)
+    W = I.make_weights(model, 8, zero_bias=False)
+    owner = np.random.default_rng(8).integers(0, P, size=n).astype(np.int32)
+    orc = Oracle(n, src, dst, X, model, W, edge_weights=ew)
+    cl = Cluster(P, owner, src, dst, X, model, W, edge_weights=ew)
+    full = orc.full()
+    for l in range(4):
+        assert max_err(cl.embeddings(l, n), full[l]) <= TOL, f"bootstrap, layer {l}"
+    stream = I.UpdateStream(n, src, dst, 18, 8)
+    for b, bs in enumerate([1, 2, 7, 33, 100, 1, 64]):
+        ups, rows, ow = stream.next_batch_weighted(bs)
+        cl.apply_batch(ups, rows, ow)
+        assert orc.apply_incremental(ups, rows, op_weights=ow) == 0
+        for l in range(4):
+            assert np.array_equal(cl.affected(l), orc.affected(l)), (P, b, l)
+    full = orc.full()
+    for l in range(4):
+        assert max_err(cl.embeddings(l, n), full[l]) <= TOL, (P, l)
+    # the stored weights themselves: every worker's copy of its edges, cut edges included
+    rp_o, col_o = orc.export_csr()
+    w_o = orc.export_weights()
+    want = {(int(u), int(v)): float(a) for u, v, a in zip(np.repeat(np.arange(n), np.diff(rp_o)), col_o, w_o)}
+    for r, wk in enumerate(cl.workers):
+        gof = cl.router.global_ids(r, wk.n)
+        rowptr, col, wts = wk.export_graph_weighted()
+        su = np.repeat(np.arange(wk.n), np.diff(rowptr))
+        for u, v, a in zip(gof[su].tolist(), gof[col].tolist(), wts.tolist()):
+            assert want[(u, v)] == a
+    cl.close()

@@ -61,11 +61,12 @@ def test_router_routes_like_the_oracle_server(PT, routing):
         r.route(ups)
         want = s.route(ups)
         for p in range(3):
-            lu, nc, row_of, _, _, _ = r.batch(p)
+            lu, nc, row_of, _, _, _, op_of = r.batch(p)
             got = [(int(x["op"]), r.global_id(p, int(x["u"])),
                     r.global_id(p, int(x["v"])) if x["op"] != I.OP_SET_FEATURE else int(row_of[x["v"]]), bool(c == 0))
                    for x, c in zip(lu, nc)]
             assert got == [(op, u, v, comp) for (_, op, u, v, comp) in want[p]], (b, p)
+            assert op_of.tolist() == [i for (i, _, _, _, _) in want[p]], (b, p)     # where in the batch each one comes from
     assert all(r.owner(v) == s.owner[v] for v in range(n + spare))
     assert all(r.is_high_degree(v) == (v in s.hd) for v in range(n + spare))
     assert [r.load(p) for p in range(3)] == s.load.tolist()
@@ -76,12 +77,13 @@ def test_partition_holds_every_edge_with_a_local_endpoint_and_halo_tables_point_
     r = PT.Router(3, owner, src, dst)
     seen = set()
     for p in range(3):
-        n_local, nv, ls, ld, gof, ho, hr = r.partition(p)
+        n_local, nv, ls, ld, gof, ho, hr, edge_of = r.partition(p)
         assert n_local % 32 == 0 and nv == n_local + n
         own = gof[:n_local]
         assert sorted(own[own >= 0].tolist()) == np.nonzero(owner == p)[0].tolist()
         assert (np.diff(own[own >= 0]) > 0).all()                      # local ids in ascending global id
         edges = set(zip(gof[ls].tolist(), gof[ld].tolist()))
+        assert np.array_equal(src[edge_of], gof[ls]) and np.array_equal(dst[edge_of], gof[ld])   # the global edge behind each
         want = {(u, v) for u, v in zip(src.tolist(), dst.tolist()) if owner[u] == p or owner[v] == p}
         assert edges == want
         seen |= edges
@@ -99,10 +101,11 @@ def test_new_halo_slots_are_reported_with_the_batch_that_creates_them(PT):
     src, dst = np.array([0], dtype=np.int32), np.array([1], dtype=np.int32)
     r = PT.Router(2, owner, src, dst, halo_capacity=4)
     r.route(ups_array([(I.OP_ADD_EDGE, 0, 2), (I.OP_ADD_EDGE, 1, 2), (I.OP_ADD_EDGE, 3, 0)]))
-    lu, nc, _, first, ho, hr = r.batch(0)
+    lu, nc, _, first, ho, hr, op_of = r.batch(0)
     assert first == 0 and ho.tolist() == [1, 1] and hr.tolist() == [r.local_id(2), r.local_id(3)]
+    assert op_of.tolist() == [0, 1, 2]
     assert nc.tolist() == [0, 0, 1] and lu["v"].tolist()[:2] == [32, 32] and lu["u"].tolist()[2] == 33
-    lu, nc, _, first, ho, hr = r.batch(1)
+    lu, nc, _, first, ho, hr, _ = r.batch(1)
     assert ho.tolist() == [0, 0] and hr.tolist() == [0, 1] and nc.tolist() == [1, 1, 0]
     r.route(ups_array([(I.OP_DEL_EDGE, 0, 2)]))
     assert r.batch(0)[4].size == 0 and r.batch(0)[3] == 2                # nothing new, next free slot is 2
@@ -154,7 +157,7 @@ def _rank_main(rank, world, port, out):
     for b in range(6):
         ups, rows = stream.next_batch(9)
         router.route(ups)
-        lu, nc, row_of, _, _, _ = router.batch(rank)
+        lu, nc, row_of, _, _, _, _ = router.batch(rank)
         ops = [(i, int(x["op"]), router.global_id(rank, int(x["u"])),
                 router.global_id(rank, int(x["v"])) if x["op"] != I.OP_SET_FEATURE else int(x["v"]), bool(c == 0))
                for i, (x, c) in enumerate(zip(lu, nc))]
