@@ -549,18 +549,19 @@ def run_partitioned(args):
         w, src, dst, X, W = make_workload(name, args.seed)
         L = len(w.model.layers)
         owner = np.random.default_rng(args.seed).integers(0, Pn, size=w.n).astype(np.int32)
-        cl = PT.Cluster(Pn, owner, src, dst, X, w.model, W, max_batch=w.extra.get("max_batch", 16384))
+        cl = PT.Cluster(Pn, owner, src, dst, X, w.model, W, max_batch=w.extra.get("max_batch", 16384),
+                        edge_weights=w.edge_w)
         rp = ripple.Ripple(w.n, src, dst, X, w.model, W, max_batch=w.extra.get("max_batch", 16384),
-                           scatter_mode=ripple.SCATTER_PUSH, rebuild_budget=-1.0)
+                           scatter_mode=ripple.SCATTER_PUSH, rebuild_budget=-1.0, edge_weights=w.edge_w)
         stream = I.make_stream(w, src, dst, args.seed)
         for bsz in (args.batch_sizes or w.batch_sizes):
             nb = args.table_batches
             wall, model, single = [], [], []
             sent = np.zeros(L + 1)
             for i in range(5 + nb):
-                ups, rows = stream.next_batch(bsz)
+                ups, rows, ow = draw_batch(stream, w, bsz)
                 t0 = time.perf_counter()
-                rp.apply_batch(ups, rows)
+                rp.apply_batch(ups, rows, ow)
                 t_single = time.perf_counter() - t0
                 t0 = time.perf_counter()
                 cl.router.route(ups)
@@ -577,10 +578,10 @@ def run_partitioned(args):
                     return worst
 
                 def begin(r, wk):
-                    lu, nc, row_of, first, ho, hr, _ = shares[r]
+                    lu, nc, row_of, first, ho, hr, op_of = shares[r]
                     if ho.size:
                         wk.set_halos(first, ho, hr)
-                    wk.begin(lu, PT.payload_rows(rows, row_of, wk.dims[0]), nc)
+                    wk.begin(lu, PT.payload_rows(rows, row_of, wk.dims[0]), nc, ow[op_of] if ow is not None else None)
 
                 crit += phase(begin)
                 for l in range(1, L + 1):

@@ -981,6 +981,19 @@ extern "C" ripple_status ripple_part_set_peer(ripple_ctx* ctx, int32_t rank, con
     }
     c->peer_bitmap[rank] = static_cast<uint32_t*>(e->frontier_bitmap);
     c->peer_deg_out[rank] = static_cast<int32_t*>(e->out_degrees);
+    {   // a peer of the same process on another GPU: its memory must be opened to this device's kernels
+        cudaPointerAttributes at;
+        if (e->frontier_bitmap && cudaPointerGetAttributes(&at, e->frontier_bitmap) == cudaSuccess &&
+            at.type == cudaMemoryTypeDevice && at.device != c->device) {
+            cudaSetDevice(c->device);
+            const cudaError_t pe = cudaDeviceEnablePeerAccess(at.device, 0);
+            if (pe != cudaSuccess && pe != cudaErrorPeerAccessAlreadyEnabled) {
+                set_err(c, "device %d cannot reach the memory of device %d: %s", c->device, at.device, cudaGetErrorString(pe));
+                return RIPPLE_ERR_CUDA;
+            }
+        }
+        cudaGetLastError();
+    }
     return RIPPLE_OK;
 }
 
