@@ -51,7 +51,7 @@ k_part_ship(Ctl* ctl, int l, int n_local, int n_words, uint32_t* bitmap, float* 
             const int lid = (w << 5) + b, h = lid - n_local;
             const int owner = halo_owner[h], rid = halo_rid[h];
             float4* row = reinterpret_cast<float4*>(dS + (size_t)lid * ld);
-            if (owner >= 0) {
+            if (owner >= 0 && peers.dS[owner] && peers.bitmap[owner]) {   // (the host refuses a hop whose peers are not all registered)
                 float* dst = peers.dS[owner] + (size_t)rid * ld;
                 for (int q = lane; q < nq; q += 32) red_add_v4_sys(dst + 4 * q, row[q]);
                 if (lane == 0) atomicOr_system(&peers.bitmap[owner][rid >> 5], 1u << (rid & 31));
@@ -72,7 +72,7 @@ k_part_fetch(int l, int n_local, int n_halo, float* H, int ld, const int32_t* __
     const int lane = lane_id(), nq = ld >> 2;
     for (int h = warp; h < n_halo; h += nwarps) {
         const int owner = halo_owner[h];
-        if (owner < 0) continue;
+        if (owner < 0 || !peers.H[owner]) continue;
         const float4* src = reinterpret_cast<const float4*>(peers.H[owner] + (size_t)halo_rid[h] * ld);
         float4* dst = reinterpret_cast<float4*>(H + (size_t)(n_local + h) * ld);
         float a = 1.f;

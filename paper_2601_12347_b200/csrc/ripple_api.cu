@@ -945,6 +945,17 @@ static Ctx* worker(ripple_ctx* ctx) {
     return (c && c->n_local > 0) ? c : nullptr;
 }
 
+// every worker that owns one of this worker's halo slots must have been registered: the exchange kernels
+// dereference its buffers
+static ripple_status peers_known(Ctx* c) {
+    if (c->halo_owner_mask & ~c->peer_mask) {
+        set_err(c, "halo slots name workers (mask 0x%x) whose buffers have not been registered (ripple_part_set_peer / ripple_part_ipc_open)",
+                c->halo_owner_mask & ~c->peer_mask);
+        return RIPPLE_ERR_INVALID_ARG;
+    }
+    return RIPPLE_OK;
+}
+
 static ripple_status finish_phase(Ctx* c) {
     cudaError_t e = cudaStreamSynchronize(c->stream);
     if (!e) e = cudaGetLastError();
@@ -981,6 +992,7 @@ extern "C" ripple_status ripple_part_set_peer(ripple_ctx* ctx, int32_t rank, con
     }
     c->peer_bitmap[rank] = static_cast<uint32_t*>(e->frontier_bitmap);
     c->peer_deg_out[rank] = static_cast<int32_t*>(e->out_degrees);
+    if (e->frontier_bitmap && e->out_degrees) c->peer_mask |= 1u << rank;
     {   // a peer of the same process on another GPU: its memory must be opened to this device's kernels
         cudaPointerAttributes at;
         if (e->frontier_bitmap && cudaPointerGetAttributes(&at, e->frontier_bitmap) == cudaSuccess &&
@@ -1048,6 +1060,13 @@ extern "C" ripple_status ripple_part_set_halos(ripple_ctx* ctx, int32_t first, i
         (int64_t)first + count > (int64_t)c->N - c->n_local)
         return RIPPLE_ERR_INVALID_ARG;
     if (count == 0) return RIPPLE_OK;
+    for (int32_t i = 0; i < count; ++i) {
+        if (owner[i] < 0 || owner[i] >= RIPPLE_MAX_PEERS || remote_id[i] < 0) {
+            set_err(c, "halo slot %d names worker %d, vertex %d", first + i, owner[i], remote_id[i]);
+            return RIPPLE_ERR_INVALID_ARG;
+        }
+        c->halo_owner_mask |= 1u << owner[i];
+    }
     cudaSetDevice(c->device);
     cudaError_t e = cudaMemcpyAsync(c->halo_owner + first, owner, sizeof(int32_t) * (size_t)count, cudaMemcpyHostToDevice, c->stream);
     if (!e) e = cudaMemcpyAsync(c->halo_rid + first, remote_id, sizeof(int32_t) * (size_t)count, cudaMemcpyHostToDevice, c->stream);
@@ -1059,6 +1078,7 @@ extern "C" ripple_status ripple_part_set_halos(ripple_ctx* ctx, int32_t first, i
 extern "C" ripple_status ripple_part_bootstrap_layer(ripple_ctx* ctx, int32_t l) {
     Ctx* c = worker(ctx);
     if (!c || l < 1 || l > c->L) return RIPPLE_ERR_INVALID_ARG;
+    if (ripple_status ps = peers_known(c)) return ps;
     cudaSetDevice(c->device);
     c->launches = 0;
     c->params_host[0] = 0; c->params_host[1] = 0;
@@ -1129,6 +1149,7 @@ extern "C" ripple_status ripple_part_begin(ripple_ctx* ctx, const ripple_update*
 extern "C" ripple_status ripple_part_hop_send(ripple_ctx* ctx, int32_t l) {
     Ctx* c = worker(ctx);
     if (!c || l < 1 || l > c->L) return RIPPLE_ERR_INVALID_ARG;
+    if (ripple_status ps = peers_known(c)) return ps;
     cudaSetDevice(c->device);
     scatter_layer(c, l, c->part_nb);
     part_ship(c, l);

@@ -159,6 +159,8 @@ struct Ctx {
     int32_t* peer_deg_out[RIPPLE_MAX_PEERS];
     void* ipc_opened[RIPPLE_MAX_PEERS * (2 * (RP_MAXL + 1) + 2)];   // mappings to close
     int n_ipc_opened;
+    unsigned peer_mask;        // workers whose buffers have been registered
+    unsigned halo_owner_mask;  // workers that own at least one assigned halo slot
     unsigned long long* rows_sent;   // device, per hop: halo rows shipped by the last batch
     int part_phase;            // 0 idle, else 1 + the number of phases of the current batch already run
     int part_nb;

@@ -139,6 +139,14 @@ def test_partitioned_context_refuses_what_it_cannot_do(env):
         w.recompute_full()
     with pytest.raises(ripple.RippleError):
         w.begin(G.ups_array([(I.OP_DEL_VERTEX, 0, 0)]), None, np.zeros(1, dtype=np.uint8))
+    # a worker whose halo slots name a peer that was never registered refuses to exchange
+    from paper_2601_12347_b200 import partitioned as PT
+    lone, _ = PT._make_worker(cl.router, 1, X, model, W)
+    with pytest.raises(ripple.RippleError):
+        lone.bootstrap_layer(1)
+    with pytest.raises(ripple.RippleError):
+        lone.set_halos(0, np.array([99], dtype=np.int32), np.array([0], dtype=np.int32))
+    lone.close()
     cl.close()
     model = I.graphconv_model([18, 36, 10], I.AGG_MAX)
     with pytest.raises(ripple.RippleError):
