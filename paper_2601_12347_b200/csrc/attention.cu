@@ -26,7 +26,7 @@
 namespace rp {
 
 constexpr int ATT_CHUNK = 64;     // out-edges per warp work item of the message walk
-constexpr int ATT_GATHER = 128;   // in-list entries per warp work item of a recomputation
+constexpr int ATT_GATHER = RP_ATT_CHUNK;   // in-list entries per warp work item of a recomputation
 
 __device__ __forceinline__ float att_weight(float s_u, float t_v, float slope) {
     float z = s_u + t_v;

@@ -21,6 +21,7 @@
 #define RP_POOL_CLASSES 32          // block size classes of the adjacency store: class k holds blocks of 2^k entries
 #define RP_POOL_MIN_CLASS 3         // smallest block that is kept for reuse: 8 entries
 #define RP_POOL_LIST_CAP 16384      // blocks a class's free list can hold
+#define RP_ATT_CHUNK 128            // attention: in-list entries per work item of a recomputation (sizes the item buffer)
 #define RP_TINY_BATCH 32            // batches up to this size list their frontiers and senders in one block each
 #define RP_TINY_APPLY 4             // ... and up to this size run the whole of Apply in one block (operations are resolved one after the other there)
 #define RP_TINY_WORDS 16384         // ... and list a hop's frontier in one block if its bitmap has at most this many words
