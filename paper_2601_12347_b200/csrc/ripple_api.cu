@@ -373,7 +373,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
         CK(dev_alloc(&c->moved_cap, (size_t)4 * o.max_batch));
         // degree prefix of a sender list; also the (vertex, chunk) work items of long in-lists during a
         // gather: a row of more than 256 entries gives at most 2 items per 256 of them
-        CK(dev_alloc(&c->coff, std::max((size_t)N + 2, (size_t)(c->side[1].col_size / RP_ATT_CHUNK) + 64), 0));
+        CK(dev_alloc(&c->coff, std::max((size_t)N + 2, (size_t)(c->side[1].col_size / 128) + 64), 0));
         CK(dev_alloc(&c->bitmap, (size_t)c->n_words + 256, 0));
         if (rp_monotonic(agg)) {
             CK(dev_alloc(&c->bitmap2, (size_t)c->n_words + 256, 0));
@@ -861,7 +861,7 @@ extern "C" ripple_status ripple_reserve_vertices(ripple_ctx* ctx, int64_t num_ve
     CK(grow_array(&c->att_so, N0 + 32, N1 + 32, 0));
     if (c->att_items) CK(grow_array(&c->att_items, N0 + (size_t)(c->side[1].col_size / RP_ATT_CHUNK) + 64, N1 + (size_t)(c->side[1].col_size / RP_ATT_CHUNK) + 64, 0));
     {
-        const size_t other = (size_t)(c->side[1].col_size / RP_ATT_CHUNK) + 64;
+        const size_t other = (size_t)(c->side[1].col_size / 128) + 64;
         CK(grow_array(&c->coff, std::max(N0 + 2, other), std::max(N1 + 2, other), 0));
     }
     {
