@@ -1,22 +1,24 @@
 /* ripple.h -- C ABI of the B200-native incremental GNN inference library.
  *
  * The library keeps, resident on one GPU, a dynamic directed graph, the vertex features H^0 and
- * the cached per-layer embeddings H^1..H^L of an L-layer GNN with a linear aggregator, and
- * brings them up to date after each batch of updates by incremental propagation: only the
- * vertices of the L-hop propagation tree of the batch are touched, and the result equals full
- * layer-wise inference on the updated graph (RIPPLE++, Sec. 3.1 and Sec. 3.3).
+ * the cached per-layer embeddings H^1..H^L of an L-layer GNN -- with a linear aggregator, or,
+ * hybrid-incrementally, with max / min or attention layers (Sec. 3.4) -- and brings them up to
+ * date after each batch of updates by incremental propagation: only the vertices of the L-hop
+ * propagation tree of the batch are touched, and the result equals full layer-wise inference on
+ * the updated graph (RIPPLE++, Sec. 3.1 and Sec. 3.3).  ripple_part.h holds the calls of the
+ * partitioned execution over several GPUs (Sec. 4).
  *
  * Conventions
  *   - Edge (u, v): u is the source, v the sink; v aggregates over its in-neighbours (Eq. 1).
- *   - The vertex set {0..N-1} is fixed at creation.  The graph is simple and directed; a
- *     self-loop is an ordinary edge.
+ *   - The vertex ids are {0..N-1}, N a capacity given at creation that ripple_reserve_vertices
+ *     can raise.  The graph is simple and directed; a self-loop is an ordinary edge.
  *   - All matrices are fp32, row-major.  Device matrices returned by the library have a leading
  *     dimension `ld` >= width (a multiple of 4 floats); columns beyond the width hold zeros.
  *   - Pointers marked HOST must be dereferenceable by the CPU, DEVICE by the GPU the context
  *     lives on; pointers marked HOST|DEVICE are accompanied by a `ripple_mem` flag.
  *   - The caller owns every buffer it passes in; the library copies what it keeps.  Pointers
  *     handed out by the library are borrowed and stay valid until the next ripple_apply_batch,
- *     ripple_recompute_full or ripple_destroy on the same context.
+ *     ripple_recompute_full, ripple_reserve_vertices or ripple_destroy on the same context.
  *   - Every call returns a ripple_status; nothing aborts or traps.  After a non-zero status,
  *     ripple_last_error() describes it.  A batch that is rejected leaves graph, features and
  *     embeddings exactly as they were.
