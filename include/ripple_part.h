@@ -59,6 +59,7 @@ typedef struct {
     int64_t embeddings_ld[RIPPLE_MAX_LAYERS + 1];
     void* frontier_bitmap;
     void* out_degrees;
+    int64_t num_vertices;   /* local ids of the worker: a halo slot that names a larger one is refused */
 } ripple_part_exports;
 
 /* Opaque handles of the same buffers for another process (CUDA IPC). */
@@ -69,6 +70,7 @@ typedef struct {
     unsigned char out_degrees[64];
     int64_t accumulator_ld[RIPPLE_MAX_LAYERS + 1];
     int64_t embeddings_ld[RIPPLE_MAX_LAYERS + 1];
+    int64_t num_vertices;
     int32_t num_layers;
 } ripple_part_ipc;
 

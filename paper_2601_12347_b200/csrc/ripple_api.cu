@@ -67,6 +67,7 @@ static void destroy_ctx(Ctx* c) {
     }
     cudaFree(c->att_so); cudaFree(c->att_items);
     cudaFree(c->halo_owner); cudaFree(c->halo_rid); cudaFree(c->silent_dev); cudaFree(c->rows_sent);
+    free(c->halo_owner_h); free(c->halo_rid_h);
     for (int i = 0; i < c->n_ipc_opened; ++i) cudaIpcCloseMemHandle(c->ipc_opened[i]);
     cudaFree(c->T); cudaFree(c->Dt); cudaFree(c->coff); cudaFree(c->bitmap); cudaFree(c->bitmap2); cudaFree(c->old_idx); cudaFree(c->invmask); cudaFree(c->posmap); cudaFree(c->deg_out_old);
     cudaFree(c->feat_last); cudaFree(c->ups_dev); cudaFree(c->opw_dev); cudaFree(c->feat_dev); cudaFree(c->hkeys); cudaFree(c->hwin); cudaFree(c->op_seq); cudaFree(c->vdel_seq); cudaFree(c->vjobs);
@@ -402,6 +403,10 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             CK(dev_alloc(&c->halo_rid, (size_t)(N - c->n_local), 0xFF));
             CK(dev_alloc(&c->silent_dev, (size_t)o.max_batch, 0));
             CK(dev_alloc(&c->rows_sent, (size_t)RP_MAXL + 1, 0));
+            c->halo_owner_h = static_cast<int32_t*>(malloc(sizeof(int32_t) * (size_t)std::max(N - c->n_local, 1)));
+            c->halo_rid_h = static_cast<int32_t*>(malloc(sizeof(int32_t) * (size_t)std::max(N - c->n_local, 1)));
+            if (!c->halo_owner_h || !c->halo_rid_h) { set_err(nullptr, "host allocation failed"); st = RIPPLE_ERR_OOM; goto fail; }
+            for (int h = 0; h < N - c->n_local; ++h) c->halo_owner_h[h] = -1;
         }
         CK(cudaDeviceSynchronize());
 
@@ -953,6 +958,16 @@ static ripple_status peers_known(Ctx* c) {
                 c->halo_owner_mask & ~c->peer_mask);
         return RIPPLE_ERR_INVALID_ARG;
     }
+    if (c->halo_dirty) {   // no halo slot may name a vertex its owner does not have
+        for (int h = 0; h < c->halo_hi; ++h) {
+            const int o = c->halo_owner_h[h];
+            if (o >= 0 && (int64_t)c->halo_rid_h[h] >= c->peer_n[o]) {
+                set_err(c, "halo slot %d names vertex %d of worker %d, which has %lld", h, c->halo_rid_h[h], o, (long long)c->peer_n[o]);
+                return RIPPLE_ERR_VERTEX_RANGE;
+            }
+        }
+        c->halo_dirty = 0;
+    }
     return RIPPLE_OK;
 }
 
@@ -976,6 +991,7 @@ extern "C" ripple_status ripple_part_exports_get(ripple_ctx* ctx, ripple_part_ex
     }
     out->frontier_bitmap = c->bitmap;
     out->out_degrees = c->side[0].deg;
+    out->num_vertices = c->N;
     return RIPPLE_OK;
 }
 
@@ -993,6 +1009,8 @@ extern "C" ripple_status ripple_part_set_peer(ripple_ctx* ctx, int32_t rank, con
     c->peer_bitmap[rank] = static_cast<uint32_t*>(e->frontier_bitmap);
     c->peer_deg_out[rank] = static_cast<int32_t*>(e->out_degrees);
     if (e->frontier_bitmap && e->out_degrees) c->peer_mask |= 1u << rank;
+    c->peer_n[rank] = e->num_vertices;
+    c->halo_dirty = 1;
     {   // a peer of the same process on another GPU: its memory must be opened to this device's kernels
         cudaPointerAttributes at;
         if (e->frontier_bitmap && cudaPointerGetAttributes(&at, e->frontier_bitmap) == cudaSuccess &&
@@ -1016,6 +1034,7 @@ extern "C" ripple_status ripple_part_ipc_export(ripple_ctx* ctx, ripple_part_ipc
     cudaSetDevice(c->device);
     memset(out, 0, sizeof(*out));
     out->num_layers = c->L;
+    out->num_vertices = c->N;
     cudaError_t e = cudaIpcGetMemHandle(reinterpret_cast<cudaIpcMemHandle_t*>(out->frontier_bitmap), c->bitmap);
     if (!e) e = cudaIpcGetMemHandle(reinterpret_cast<cudaIpcMemHandle_t*>(out->out_degrees), c->side[0].deg);
     for (int l = 0; l <= c->L && !e; ++l) {
@@ -1041,6 +1060,7 @@ extern "C" ripple_status ripple_part_ipc_open(ripple_ctx* ctx, int32_t rank, con
         if (!e) c->ipc_opened[c->n_ipc_opened++] = *p;
         return e;
     };
+    ex.num_vertices = in->num_vertices;
     cudaError_t e = open(in->frontier_bitmap, &ex.frontier_bitmap);
     if (!e) e = open(in->out_degrees, &ex.out_degrees);
     for (int l = 0; l <= c->L && !e; ++l) {
@@ -1066,7 +1086,11 @@ extern "C" ripple_status ripple_part_set_halos(ripple_ctx* ctx, int32_t first, i
             return RIPPLE_ERR_INVALID_ARG;
         }
         c->halo_owner_mask |= 1u << owner[i];
+        c->halo_owner_h[first + i] = owner[i];
+        c->halo_rid_h[first + i] = remote_id[i];
     }
+    c->halo_hi = std::max(c->halo_hi, first + count);
+    c->halo_dirty = 1;
     cudaSetDevice(c->device);
     cudaError_t e = cudaMemcpyAsync(c->halo_owner + first, owner, sizeof(int32_t) * (size_t)count, cudaMemcpyHostToDevice, c->stream);
     if (!e) e = cudaMemcpyAsync(c->halo_rid + first, remote_id, sizeof(int32_t) * (size_t)count, cudaMemcpyHostToDevice, c->stream);

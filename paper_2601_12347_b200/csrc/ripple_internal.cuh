@@ -160,6 +160,11 @@ struct Ctx {
     int32_t* peer_deg_out[RIPPLE_MAX_PEERS];
     void* ipc_opened[RIPPLE_MAX_PEERS * (2 * (RP_MAXL + 1) + 2)];   // mappings to close
     int n_ipc_opened;
+    int32_t* halo_owner_h;     // host copies of the halo table, to check it against the peers' sizes
+    int32_t* halo_rid_h;
+    int halo_hi;               // halo slots below this index may be assigned
+    int halo_dirty;            // the table or the peer set changed since it was last checked
+    int64_t peer_n[RIPPLE_MAX_PEERS];   // local ids of every registered worker
     unsigned peer_mask;        // workers whose buffers have been registered
     unsigned halo_owner_mask;  // workers that own at least one assigned halo slot
     unsigned long long* rows_sent;   // device, per hop: halo rows shipped by the last batch

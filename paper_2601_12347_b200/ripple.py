@@ -96,7 +96,8 @@ class _Stats(ctypes.Structure):
 class _PartExports(ctypes.Structure):
     _fields_ = [("accumulator", ctypes.c_void_p * (MAX_LAYERS + 1)), ("accumulator_ld", ctypes.c_int64 * (MAX_LAYERS + 1)),
                 ("embeddings", ctypes.c_void_p * (MAX_LAYERS + 1)), ("embeddings_ld", ctypes.c_int64 * (MAX_LAYERS + 1)),
-                ("frontier_bitmap", ctypes.c_void_p), ("out_degrees", ctypes.c_void_p)]
+                ("frontier_bitmap", ctypes.c_void_p), ("out_degrees", ctypes.c_void_p),
+                ("num_vertices", ctypes.c_int64)]
 
 
 class _PartIpc(ctypes.Structure):
@@ -104,7 +105,8 @@ class _PartIpc(ctypes.Structure):
                 ("embeddings", (ctypes.c_ubyte * 64) * (MAX_LAYERS + 1)),
                 ("frontier_bitmap", ctypes.c_ubyte * 64), ("out_degrees", ctypes.c_ubyte * 64),
                 ("accumulator_ld", ctypes.c_int64 * (MAX_LAYERS + 1)),
-                ("embeddings_ld", ctypes.c_int64 * (MAX_LAYERS + 1)), ("num_layers", ctypes.c_int32)]
+                ("embeddings_ld", ctypes.c_int64 * (MAX_LAYERS + 1)), ("num_vertices", ctypes.c_int64),
+                ("num_layers", ctypes.c_int32)]
 
 
 _lib = None

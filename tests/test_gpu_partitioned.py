@@ -146,6 +146,13 @@ def test_partitioned_context_refuses_what_it_cannot_do(env):
         lone.bootstrap_layer(1)
     with pytest.raises(ripple.RippleError):
         lone.set_halos(0, np.array([99], dtype=np.int32), np.array([0], dtype=np.int32))
+    # ... and one whose halo slot names a vertex its owner does not have
+    for r, wk in enumerate(cl.workers):
+        lone.set_peer(r, wk.exports())
+    lone.set_halos(0, np.array([0], dtype=np.int32), np.array([cl.workers[0].n + 5], dtype=np.int32))
+    with pytest.raises(ripple.RippleError) as e:
+        lone.bootstrap_layer(1)
+    assert e.value.status == ripple.ERR_VERTEX_RANGE
     lone.close()
     cl.close()
     model = I.graphconv_model([18, 36, 10], I.AGG_MAX)
