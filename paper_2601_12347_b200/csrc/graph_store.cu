@@ -688,7 +688,7 @@ k_apply_small(Ctl* ctl, const int* params, const ripple_update* __restrict__ ups
               int32_t* vdel_seq, Side out, Side in, Rec* rec, uint32_t* bitmap, const float* __restrict__ op_w,
               int32_t* grow_out, int32_t* grow_in, int32_t* shrink_out, int32_t* shrink_in, int64_t* moved_start,
               int32_t* moved_cap, int32_t* deg_out_old, const float* __restrict__ feat, int d0, float* H0, int ld,
-              float* D, int keep_old, int32_t* A0, int32_t* senders, int32_t* posmap, int64_t* coff) {
+              float* D, int keep_old, int32_t* A0, int build_senders, int32_t* senders, int32_t* posmap, int64_t* coff) {
     pdl_enter();
     __shared__ int s_ids[RP_TINY_BATCH];
     __shared__ int s_n;
@@ -732,7 +732,7 @@ k_apply_small(Ctl* ctl, const int* params, const ripple_update* __restrict__ ups
     }
     __syncthreads();
     if (mine >= 0) { s_ids[rank] = mine; A0[rank] = mine; }
-    if (threadIdx.x == 0) { ctl->nA[0] = na; ctl->nC[0] = na; }
+    if (threadIdx.x == 0) { ctl->nA[0] = na; if (build_senders) ctl->nC[0] = na; }
     __syncthreads();
     // feature rows: one warp per vertex of A_0
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -746,8 +746,9 @@ k_apply_small(Ctl* ctl, const int* params, const ripple_update* __restrict__ ups
             H0[(size_t)v * ld + k] = x;
         }
     }
-    // senders of hop 1 = A_0, with the prefix of their out-degrees
-    if (threadIdx.x == 0) {
+    // senders of hop 1 = A_0, with the prefix of their out-degrees (max / min aggregation lists its own: the rows
+    // of A_0 whose values really changed)
+    if (build_senders && threadIdx.x == 0) {
         int64_t sum = 0;
         for (int i = 0; i < na; ++i) {
             const int v = s_ids[i];
@@ -769,8 +770,8 @@ void graph_batch_apply_small(Ctx* c, int n) {
               (const int32_t*)c->op_seq, c->N, c->hkeys, c->hwin, c->hsize - 1, c->op_slot, c->feat_last, c->vdel_seq, o, i,
               c->rec, c->bitmap, (const float*)(c->has_opw ? c->opw_dev : nullptr), c->grow_list[0], c->grow_list[1],
               c->shrink_list[0], c->shrink_list[1], c->moved_start, c->moved_cap, c->deg_out_old,
-              (const float*)c->feat_dev, c->d[0], c->H[0], c->ld[0], c->D[0], (int)c->attention, c->A[0], c->Clist[0],
-              c->posmap, c->coff);
+              (const float*)c->feat_dev, c->d[0], c->H[0], c->ld[0], c->D[0], (int)(c->attention || rp_monotonic(c->agg)),
+              c->A[0], (int)!rp_monotonic(c->agg), c->Clist[0], c->posmap, c->coff);
 }
 
 void graph_batch_mutate(Ctx* c, int n) {

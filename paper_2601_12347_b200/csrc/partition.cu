@@ -65,7 +65,7 @@ k_part_ship(Ctl* ctl, int l, int n_local, int n_words, uint32_t* bitmap, float* 
 // side (src_norm: 1 / sqrt of the out-degree) the gather that follows would scale the row by this worker's
 // partial out-degree of the halo vertex; the copy is pre-scaled so that the product is the owner's coefficient.
 __global__ void __launch_bounds__(256)
-k_part_fetch(int l, int n_local, int n_halo, float* H, int ld, const int32_t* __restrict__ halo_owner,
+k_part_fetch(int n_local, int n_halo, float* H, int ld, const int32_t* __restrict__ halo_owner,
              const int32_t* __restrict__ halo_rid, PeerTab peers, int src_norm, const int32_t* __restrict__ deg_out) {
     pdl_enter();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -85,7 +85,6 @@ k_part_fetch(int l, int n_local, int n_halo, float* H, int ld, const int32_t* __
             dst[q] = make_float4(a * x.x, a * x.y, a * x.z, a * x.w);
         }
     }
-    (void)l;
 }
 
 static PeerTab peer_table(const Ctx* c, int l) {
@@ -109,7 +108,7 @@ void part_ship(Ctx* c, int l) {
 void part_fetch_halo_rows(Ctx* c, int l) {
     const int n_halo = c->N - c->n_local;
     if (n_halo <= 0) return;
-    RP_LAUNCH(c, k_part_fetch, std::min(div_up(n_halo, 8), c->n_sm * 8), 256, 0, l, c->n_local, n_halo, c->H[l], c->ld[l],
+    RP_LAUNCH(c, k_part_fetch, std::min(div_up(n_halo, 8), c->n_sm * 8), 256, 0, c->n_local, n_halo, c->H[l], c->ld[l],
               c->halo_owner, c->halo_rid, peer_table(c, l), (int)c->src_norm, c->side[0].deg);
 }
 

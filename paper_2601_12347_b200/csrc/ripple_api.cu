@@ -438,9 +438,10 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
     // A handful of updates: the whole of Apply and the hop-0 sender list in one block (the chain of a small batch
     // is bound by the number of dependent steps, not by their work); also the merged frontier kernel below.
     const bool tiny = nb >= 1 && nb <= RP_TINY_BATCH && !c->may_expand && !c->src_norm && !rp_monotonic(c->agg);
-    if (tiny && nb <= RP_TINY_APPLY) {
+    if (nb >= 1 && nb <= RP_TINY_APPLY && !c->may_expand && !c->src_norm) {
         STAMP();  // 0
         graph_batch_apply_small(c, nb);
+        if (rp_monotonic(c->agg)) max_senders_build(c, 0);
     } else {
         RP_LAUNCH(c, k_ctl_reset, 1, 1, 0, c->ctl, c->params_dev);
         STAMP();  // 0

@@ -14,7 +14,7 @@ of a hop in the library's kernels.  Two ways to run the workers:
 from __future__ import annotations
 
 import ctypes
-from typing import Dict, List, Optional, Sequence, Tuple
+from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
 
@@ -266,7 +266,7 @@ class Cluster:
         d = self.workers[0].dims[l]
         out = np.zeros((n, d), dtype=np.float32)
         for r, w in enumerate(self.workers):
-            nl = w_n_local(w)
+            nl = w.n_local
             gof = self.router.global_ids(r, w.n)[:nl].astype(np.int64)
             h = w.embeddings(l)[:nl].cpu().numpy()
             out[gof[gof >= 0]] = h[gof >= 0]
@@ -283,10 +283,6 @@ class Cluster:
         for w in self.workers:
             tot += np.array(w.rows_sent())
         return tot.tolist()
-
-
-def w_n_local(w: Worker) -> int:
-    return int(w.n_local)
 
 
 class DistributedWorker:
