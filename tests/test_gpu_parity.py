@@ -801,3 +801,37 @@ def test_bounded_wait_reports_a_timeout_and_the_device_stays_usable(env, monkeyp
     check_graph(rp, orc)
     check_values(rp, orc.full(), 3)
     rp.close()
+
+
+def test_checkpoint_and_resume_through_the_public_calls(env):
+    """A context's durable state is its graph and its feature rows: export them, create a new context from
+    them (the bootstrap recomputes every cached row), and both contexts follow the same stream to the same
+    embeddings and hop sets."""
+    ripple, Oracle = env
+    n, src, dst, X, model, W = _small(seed=23)
+    rp = ripple.Ripple(n, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 23)
+    for _ in range(5):
+        ups, rows = stream.next_batch(40)
+        rp.apply_batch(ups, rows)
+    rowptr, col = rp.export_graph()                      # the checkpoint
+    feats = rp.embeddings(0).cpu().numpy().copy()
+    src2 = np.repeat(np.arange(n, dtype=np.int32), np.diff(rowptr))
+    resumed = ripple.Ripple(n, src2, col, feats, model, W)
+    for l in range(3):
+        a, b = rp.embeddings(l).cpu().numpy(), resumed.embeddings(l).cpu().numpy()
+        assert float(np.max(np.abs(a - b) / (1.0 + np.abs(b)))) <= TOL
+    for _ in range(5):
+        ups, rows = stream.next_batch(40)
+        rp.apply_batch(ups, rows)
+        resumed.apply_batch(ups, rows)
+        for l in range(3):
+            assert np.array_equal(rp.affected(l).cpu().numpy(), resumed.affected(l).cpu().numpy())
+    r1, c1 = rp.export_graph()
+    r2, c2 = resumed.export_graph()
+    assert np.array_equal(r1, r2) and np.array_equal(c1, c2)
+    for l in range(3):
+        a, b = rp.embeddings(l).cpu().numpy(), resumed.embeddings(l).cpu().numpy()
+        assert float(np.max(np.abs(a - b) / (1.0 + np.abs(b)))) <= TOL
+    rp.close()
+    resumed.close()
