@@ -242,3 +242,31 @@ def test_monotonic_aggregation_is_refused_for_attention_layers():
     ups = np.zeros(1, dtype=I.UPDATE_DTYPE)
     ups[0] = (I.OP_ADD_EDGE, 0, 1)
     assert o.apply_incremental(ups, None) == -3
+
+
+def test_worked_example_of_the_attention_section():
+    """Sec. 3.4.1's example: D aggregates over A and C; when C's features change, the only parts of D's
+    numerator and denominator that move are C's terms, by exp(z_new) h_new - exp(z_old) h_old and
+    exp(z_new) - exp(z_old) (the paper writes the message as old minus new; the sink subtracts it)."""
+    A, B, C, D = 0, 1, 2, 3
+    src = np.array([A, C, B], dtype=np.int32)
+    dst = np.array([D, D, A], dtype=np.int32)
+    model = I.gat_model(3, 1, d_att=2, slope=1.0)
+    W = I.make_weights(model, 5)
+    X = I.features(4, 3, 5)
+    o = Oracle(4, src, dst, X, model, W)
+    num0, den0 = o.S(1)[D].copy(), float(o.Den(1)[D])
+    new_row = I.features(1, 3, 6)
+    ups = np.zeros(1, dtype=I.UPDATE_DTYPE)
+    ups[0] = (I.OP_SET_FEATURE, C, 0)
+    assert o.apply_incremental(ups, new_row) == 0
+    Wa, a_s, a_d = (W[0][k].astype(np.float64) for k in ("Wa", "ba", "bb"))
+    t_D = X[D].astype(np.float64) @ Wa @ a_d
+    z_old = X[C].astype(np.float64) @ Wa @ a_s + t_D
+    z_new = new_row[0].astype(np.float64) @ Wa @ a_s + t_D
+    assert np.allclose(o.S(1)[D] - num0, np.exp(z_new) * new_row[0] - np.exp(z_old) * X[C], rtol=1e-12, atol=1e-13)
+    assert np.isclose(o.Den(1)[D] - den0, np.exp(z_new) - np.exp(z_old), rtol=1e-12, atol=1e-13)
+    assert o.affected(1).tolist() == [C, D]      # C was in the tree at hop 0, so it is at hop 1 (it recomputes); D by the message
+    z_A = X[A].astype(np.float64) @ Wa @ a_s + t_D
+    want = (np.exp(z_A) * X[A] + np.exp(z_new) * new_row[0]) / (np.exp(z_A) + np.exp(z_new))
+    assert np.allclose(o.H(1)[D], want, rtol=1e-12, atol=1e-13)
