@@ -53,7 +53,8 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples clocks and throttle reasons while the timed region runs: nvidia-smi every 100 ms, and, because the
+    default region is a few tens of milliseconds long, the same counters read through NVML every 2 ms (reads only)."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -62,6 +63,23 @@ class ClockSampler:
         self.gpu = gpu_index
         self.proc = None
         self.lines = []
+        self.nvml = []          # (sm MHz, max sm MHz, throttle-reason bits)
+        self.running = False
+
+    def _poll_nvml(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            idx = int(visible.split(",")[self.gpu]) if visible and visible.split(",")[self.gpu].isdigit() else self.gpu
+            h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            mx = pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM)
+            while self.running:
+                self.nvml.append((pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM), mx,
+                                  pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h)))
+                time.sleep(0.002)
+        except Exception:
+            pass
 
     def start(self):
         try:
@@ -72,21 +90,35 @@ class ClockSampler:
             self.t.start()
         except Exception:
             self.proc = None
+        self.running = True
+        self.t2 = threading.Thread(target=self._poll_nvml, daemon=True)
+        self.t2.start()
 
     def _read(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
     def stop(self):
-        if self.proc is None:
+        self.running = False
+        if self.proc is None and not self.nvml:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=2)
-        except Exception:
-            pass
+        if self.proc is None:
+            self.lines = []
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                pass
         sm, mx, reasons = [], [], set()
+        # NVML reason bits: 0x8 hw slowdown, 0x40 hw thermal slowdown, 0x20 sw thermal slowdown, 0x4 sw power cap
+        for clk, cmax, bits in self.nvml:
+            sm.append(float(clk)); mx.append(float(cmax))
+            for name, bit in (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20),
+                              ("sw_power_cap", 0x4)):
+                if bits & bit:
+                    reasons.add(name)
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
