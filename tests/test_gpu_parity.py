@@ -835,3 +835,34 @@ def test_checkpoint_and_resume_through_the_public_calls(env):
         assert float(np.max(np.abs(a - b) / (1.0 + np.abs(b)))) <= TOL
     rp.close()
     resumed.close()
+
+
+@pytest.mark.parametrize("name", ["sage_mean", "gcn_wsum_3l", "gin_3l"])
+def test_batch_sizes_around_the_small_batch_thresholds(env, name):
+    """Batches of up to 4 updates run Apply in one block, up to 32 list their frontiers in one block, up to 128
+    carry the few-row form of the row update: sizes on both sides of every threshold, with a hub among the
+    endpoints so that a small batch can still have a large frontier."""
+    ripple, Oracle = env
+    model = small_models()[name]
+    L = len(model.layers)
+    n, m = 900, 7000
+    src, dst = I.er_graph(n, m, 31)
+    have = set(zip(src.tolist(), dst.tolist()))
+    extra = [(0, int(v)) for v in range(1, 600) if (0, int(v)) not in have]
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    X = I.features(n, model.dims[0], 31)
+    W = I.make_weights(model, 31, zero_bias=False)
+    rp = ripple.Ripple(n, src, dst, X, model, W)
+    orc = Oracle(n, src, dst, X, model, W)
+    stream = I.UpdateStream(n, src, dst, model.dims[0], 31)
+    for b, bs in enumerate([3, 4, 5, 4, 31, 32, 33, 32, 127, 128, 129, 4, 1]):
+        ups, rows = stream.next_batch(bs)
+        if b % 4 == 1:      # the hub's features change: hundreds of rows at hop 1 from a batch of a few updates
+            ups[0] = (I.OP_SET_FEATURE, 0, 0) if rows.shape[0] else ups[0]
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, L)
+        check_values(rp, orc.full(), L)
+    rp.close()
