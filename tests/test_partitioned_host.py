@@ -193,3 +193,27 @@ def test_two_processes_run_the_phases_with_real_exchange(PT):
     assert sum(res[r][1] for r in range(world)) == 80
     for r in range(world):
         assert res[r][0] < 1e-10
+
+
+def test_payload_rows_of_a_worker_have_zeros_for_deleted_vertices(PT):
+    rows = np.arange(12, dtype=np.float32).reshape(3, 4)
+    out = PT.payload_rows(rows, np.array([2, -1, 0], dtype=np.int32), 4)
+    assert np.array_equal(out, np.stack([rows[2], np.zeros(4, dtype=np.float32), rows[0]]))
+    assert PT.payload_rows(None, np.array([-1], dtype=np.int32), 4).tolist() == [[0.0] * 4]
+    assert PT.payload_rows(rows, np.zeros(0, dtype=np.int32), 4) is None
+
+
+def test_vertex_deletion_reaches_both_workers_of_every_cut_edge(PT):
+    owner = np.array([0, 0, 1, 1], dtype=np.int32)
+    src = np.array([0, 2, 1, 0], dtype=np.int32)      # 0->1 (local to 0), 2->0 and 0->3 (cut), 1->2 (cut)
+    dst = np.array([1, 0, 2, 3], dtype=np.int32)
+    r = PT.Router(2, owner, src, dst, halo_capacity=4)
+    r.route(ups_array([(I.OP_DEL_VERTEX, 0, 0)]))
+    lu, nc, row_of, _, _, _, op_of = r.batch(0)
+    g = lambda p, x: r.global_id(p, int(x))
+    ops0 = [(int(x["op"]), g(0, x["u"]), g(0, x["v"]) if x["op"] != I.OP_SET_FEATURE else int(row_of[x["v"]]), int(c)) for x, c in zip(lu, nc)]
+    assert ops0 == [(I.OP_DEL_EDGE, 0, 1, 0), (I.OP_DEL_EDGE, 0, 3, 0), (I.OP_DEL_EDGE, 2, 0, 1), (I.OP_SET_FEATURE, 0, -1, 0)]
+    assert op_of.tolist() == [0, 0, 0, 0]
+    lu, nc, _, _, _, _, _ = r.batch(1)
+    ops1 = [(int(x["op"]), g(1, x["u"]), g(1, x["v"]), int(c)) for x, c in zip(lu, nc)]
+    assert ops1 == [(I.OP_DEL_EDGE, 0, 3, 1), (I.OP_DEL_EDGE, 2, 0, 0)]
