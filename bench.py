@@ -636,6 +636,63 @@ def run_partitioned(args):
         torch.cuda.empty_cache()
 
 
+def run_partitioned_dist(args, rank, world, local_rank):
+    """One worker of the partitioned execution (Sec. 4 of the paper) per process: the whole graph is split over
+    the ranks (uniformly random vertex-partition map, the worst cut), every rank routes the same batches with
+    its own replica of the router, peers are reached through CUDA IPC mappings, a barrier separates the phases
+    of a hop.  Strong scaling: the job is one stream of batches.  Times are wall clock between barriers, the
+    maximum over ranks.  With fewer GPUs than ranks (how this mode was exercised: two processes on one GPU) the
+    ranks share devices and the process group runs on gloo."""
+    import torch
+    import torch.distributed as dist
+    from paper_2601_12347_b200 import build as B
+    from paper_2601_12347_b200 import partitioned as PT
+    B.build_library()
+    ndev = torch.cuda.device_count()
+    torch.cuda.set_device(local_rank % ndev)
+    shared = world > ndev
+    if shared:
+        dist.init_process_group("gloo")
+    else:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    w, src, dst, X, W = make_workload(args.workload, args.seed)
+    owner = np.random.default_rng(args.seed).integers(0, world, size=w.n).astype(np.int32)
+    dw = PT.DistributedWorker(owner, src, dst, X, w.model, W, max_batch=max(args.batch, 16) * 2, edge_weights=w.edge_w)
+    stream = I.make_stream(w, src, dst, args.seed)
+    K, Wm = args.steps, args.warmup
+    batches = [draw_batch(stream, w, args.batch) for _ in range(Wm + K)]
+    for b in batches[:Wm]:
+        dw.apply_batch(*b)
+    L = len(w.model.layers)
+    sent = np.zeros(L + 1)
+    dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for b in batches[Wm:]:
+        dw.apply_batch(*b)
+        sent += np.array(dw.worker.rows_sent())
+    torch.cuda.synchronize()
+    dist.barrier()
+    ms = (time.perf_counter() - t0) * 1e3
+    (ms,) = max_over_ranks([ms], world, device="cpu" if shared else "cuda")
+    tot = torch.tensor(sent, dtype=torch.float64, device="cpu" if shared else "cuda")
+    dist.all_reduce(tot)
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": args.batch * K / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": Wm, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{args.workload}, batch {args.batch}", "batch": args.batch,
+                       "parallelism": f"partitioned over {world} workers, uniformly random owners",
+                       "devices": min(world, ndev)},
+            "halo_rows_sent_per_step": (tot[1:] / K).round(1).tolist(),
+            "note": "wall clock between barriers, max over ranks" + ("; ranks share GPUs: not a scaling measurement" if shared else "")}),
+            flush=True)
+    dist.barrier()
+    dw.close()
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--table", default="", help="comma-separated workloads: print one line per batch size")
@@ -655,6 +712,8 @@ def main():
     ap.add_argument("--scatter", type=int, default=0, help="0 auto, 1 push, 2 pull")
     ap.add_argument("--partitioned", type=int, default=0,
                     help="with --table: run the workloads as this many workers of the partitioned execution, all on one GPU")
+    ap.add_argument("--partitioned-dist", action="store_true",
+                    help="under torchrun: one worker of the partitioned execution per rank (strong scaling) instead of replicas")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--verbose-steps", action="store_true", help="per timed step: messages and scatter time (stderr)")
     args = ap.parse_args()
@@ -662,7 +721,9 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.table and args.partitioned > 0:
+    if args.partitioned_dist and args.impl == "ours":
+        run_partitioned_dist(args, rank, world, local_rank)
+    elif args.table and args.partitioned > 0:
         if rank == 0:
             run_partitioned(args)
     elif args.table:
