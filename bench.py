@@ -685,7 +685,7 @@ def run_partitioned_dist(args, rank, world, local_rank):
             "config": {"workload": f"{args.workload}, batch {args.batch}", "batch": args.batch,
                        "parallelism": f"partitioned over {world} workers, uniformly random owners",
                        "devices": min(world, ndev)},
-            "halo_rows_sent_per_step": (tot[1:] / K).round(1).tolist(),
+            "halo_rows_sent_per_step": [round(float(x) / K, 1) for x in tot[1:].tolist()],
             "note": "wall clock between barriers, max over ranks" + ("; ranks share GPUs: not a scaling measurement" if shared else "")}),
             flush=True)
     dist.barrier()
