@@ -223,23 +223,29 @@ __global__ void k_classify(const ripple_update* __restrict__ ups, const int32_t*
 }
 
 // Position of x in row [base, base + deg), or -1; the whole block calls this.  Rows start on
-// 16-byte boundaries, so every thread compares four entries per load; a hub row of 150 K entries
-// costs a block of 256 threads about 150 iterations.
+// 16-byte boundaries, so every thread compares four entries per load, and it keeps eight loads in
+// flight: a hub row of 150 K entries costs a block of 256 threads about 19 round trips to memory.
 __device__ __forceinline__ int block_find(const int32_t* __restrict__ col, int64_t base, int deg, int x,
                                           volatile int* s_found) {
+    constexpr int FIND_UNROLL = 8;
     __syncthreads();
     if (threadIdx.x == 0) *s_found = -1;
     __syncthreads();
     const int4* row4 = reinterpret_cast<const int4*>(col + base);
     const int n4 = deg >> 2;
-    for (int q0 = 0; q0 < n4; q0 += blockDim.x) {
-        int q = q0 + threadIdx.x;
-        if (q < n4) {
-            int4 e = __ldg(row4 + q);
-            int hit = e.x == x ? 0 : e.y == x ? 1 : e.z == x ? 2 : e.w == x ? 3 : -1;
-            if (hit >= 0) *s_found = 4 * q + hit;
+    for (int q0 = 0; q0 < n4; q0 += FIND_UNROLL * blockDim.x) {
+        int4 e[FIND_UNROLL];
+#pragma unroll
+        for (int k = 0; k < FIND_UNROLL; ++k) {
+            int q = q0 + k * blockDim.x + threadIdx.x;
+            e[k] = q < n4 ? __ldg(row4 + q) : make_int4(-1, -1, -1, -1);   // x is a vertex id: never negative
         }
-        if ((q0 & (4 * blockDim.x - 1)) == 0 && *s_found >= 0) break;  // peek now and then
+#pragma unroll
+        for (int k = 0; k < FIND_UNROLL; ++k) {
+            int hit = e[k].x == x ? 0 : e[k].y == x ? 1 : e[k].z == x ? 2 : e[k].w == x ? 3 : -1;
+            if (hit >= 0) *s_found = 4 * (q0 + k * blockDim.x + threadIdx.x) + hit;
+        }
+        if (*s_found >= 0) break;   // a peek per round; a thread that misses it only reads on
     }
     int j = 4 * n4 + threadIdx.x;
     if (j < deg && col[base + j] == x) *s_found = j;
