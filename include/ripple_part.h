@@ -97,9 +97,14 @@ ripple_status ripple_part_ipc_open(ripple_ctx* ctx, int32_t rank, const ripple_p
 ripple_status ripple_part_set_halos(ripple_ctx* ctx, int32_t first, int32_t count, const int32_t* owner,
                                     const int32_t* remote_id);
 
-/* Bootstrap of layer l (Eq. 1-2 on the initial graph): fetches H^{l-1} of every assigned halo slot from
- * its owner (peer loads), then computes the cached aggregates and H^l of all local vertices.  Returns
- * when done.  Every worker must have finished layer l - 1 before any worker starts layer l. */
+/* Layer-wise inference of layer l (Eq. 1-2 on the graph as it stands): fetches H^{l-1} of every assigned
+ * halo slot from its owner (peer loads), then computes the cached aggregates and H^l of all local
+ * vertices.  Returns when done.  Every worker must have finished layer l - 1 before any worker starts
+ * layer l.  Run for l = 1..L after ripple_create, it is the bootstrap; run again for l = 1..L between
+ * two batches (no phase of a batch outstanding on any worker), it recomputes every cached row from the
+ * current graph and features, which also discards the rounding that incremental additions have left
+ * in the cached sums (a partitioned context has no per-row rebuild of its own: the rows of a vertex's
+ * remote in-neighbours are not resident). */
 ripple_status ripple_part_bootstrap_layer(ripple_ctx* ctx, int32_t l);
 
 /* One batch, in phases (Sec. 4.5).  ups / feat_rows / no_compute / edge_weights as in ripple_apply_batch_weighted

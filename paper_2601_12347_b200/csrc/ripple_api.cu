@@ -1112,7 +1112,6 @@ extern "C" ripple_status ripple_part_bootstrap_layer(ripple_ctx* ctx, int32_t l)
     part_fetch_halo_rows(c, l - 1);
     full_layer(c, l);
     c->stats.num_layers = c->L;
-    c->stats.num_edges = c->E0;
     return finish_phase(c);
 }
 

@@ -237,6 +237,12 @@ class Cluster:
             for w in self.workers:
                 w.bootstrap_layer(l)
 
+    def recompute_full(self) -> None:
+        """Layer-wise inference on the current graph on every worker (between two batches): all cached rows anew."""
+        for l in range(1, self.L + 1):
+            for w in self.workers:
+                w.bootstrap_layer(l)
+
     def close(self):
         for w in self.workers:
             w.close()
@@ -306,10 +312,15 @@ class DistributedWorker:
                 self.worker.set_peer(r, self.worker.exports())
             else:
                 self.worker.ipc_open(r, blob)
+        self.recompute_full()
+
+    def recompute_full(self) -> None:
+        """Layer-wise inference on the current graph, in step with the other ranks (the bootstrap; between two
+        batches: every cached row anew).  Collective."""
         for l in range(1, self.L + 1):
-            dist.barrier()
+            self.dist.barrier()
             self.worker.bootstrap_layer(l)
-        dist.barrier()
+        self.dist.barrier()
 
     def apply_batch(self, ups: np.ndarray, rows: Optional[np.ndarray], op_weights: Optional[np.ndarray] = None) -> None:
         self.router.route(ups)
