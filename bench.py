@@ -389,7 +389,7 @@ def run_ours(args, rank, world, local_rank):
                 "traffic": traffic,
                 "frac_hbm": (traffic / 1e9 / (sc_ms / K / 1e3) / hbm_peak) if (traffic and sc_ms > 0) else None,
                 "hbm_peak": hbm_peak, "hbm_peak_source": f"of {peak_kind}",
-                "kernel": f"{'k_scatter_pull' if pulls * 2 > K else 'k_scatter_push'} (hop {L}, row width {ld_last} floats)",
+                "kernel": f"{'k_scatter_gather' if pulls * 2 > K else 'k_scatter_push'} (hop {L}, row width {ld_last} floats)",
                 "pull_steps": int(pulls),
                 "ms_per_launch": sc_ms / K,
                 "messages_per_launch": msgs,
@@ -709,7 +709,7 @@ def main():
     ap.add_argument("--workload", default="dense-2l")
     ap.add_argument("--batch", type=int, default=1000)
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--scatter", type=int, default=0, help="0 auto, 1 push, 2 pull")
+    ap.add_argument("--scatter", type=int, default=0, help="0 auto, 1 push, 2 gather per sink")
     ap.add_argument("--partitioned", type=int, default=0,
                     help="with --table: run the workloads as this many workers of the partitioned execution, all on one GPU")
     ap.add_argument("--partitioned-dist", action="store_true",

@@ -142,7 +142,9 @@ typedef struct {
  * scattered along the senders' out-edges or gathered per affected sink.  REGATHER: the aggregates
  * of the affected vertices are rebuilt from their in-lists (the scoped recomputation of Sec. 3.2,
  * for this hop only).  AUTO: PUSH, except that a hop whose senders own at least
- * regather_threshold of all edges rebuilds. */
+ * regather_threshold of all edges rebuilds, and that a hop of wide messages (128 floats or more)
+ * from few senders gathers per sink (chosen per hop from what the hop carried in the batch before:
+ * at least 2^20 messages, eight or more per affected sink, sender rows of at most 32 MiB in all). */
 typedef enum {
     RIPPLE_SCATTER_AUTO = 0, RIPPLE_SCATTER_PUSH = 1, RIPPLE_SCATTER_PULL = 2, RIPPLE_SCATTER_REGATHER = 3,
     RIPPLE_SCATTER_PUSH_BULK = 4 /* PUSH with one bulk reduction of the copy engine per message (cp.reduce.async.bulk)
@@ -194,7 +196,7 @@ typedef struct {
     int64_t affected[RIPPLE_MAX_LAYERS + 1];      /* |A_l|, l = 0..L                                      */
     int64_t senders[RIPPLE_MAX_LAYERS + 1];       /* |C_l|: vertices whose outgoing message changed       */
     int64_t active_edges[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: edges carrying a message at hop l          */
-    int32_t scatter_pull[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: 0 push, 1 pull, 2 aggregates rebuilt       */
+    int32_t scatter_pull[RIPPLE_MAX_LAYERS + 1];  /* l = 1..L: 0 pushed, 1 gathered per sink, 2 rebuilt  */
     int64_t in_edges[RIPPLE_MAX_LAYERS + 1];      /* l = 1..L: in-edges of A_l (what a gather walks)      */
     int32_t message_width[RIPPLE_MAX_LAYERS + 1]; /* l = 1..L: floats per message / aggregate row (padded) */
     int64_t pool_used, pool_size;                 /* overflow pool, out-direction, in edges: handed out so far
@@ -204,7 +206,7 @@ typedef struct {
     float ms_frontier[RIPPLE_MAX_LAYERS + 1];
     float ms_scatter[RIPPLE_MAX_LAYERS + 1];
     float ms_update[RIPPLE_MAX_LAYERS + 1];
-    float ms_scatter_kernel[RIPPLE_MAX_LAYERS + 1]; /* the push or pull kernel alone, l = 1..L               */
+    float ms_scatter_kernel[RIPPLE_MAX_LAYERS + 1]; /* the push or gather kernels alone, l = 1..L           */
     float ms_regather[RIPPLE_MAX_LAYERS + 1];     /* the gather of a rebuilding hop alone, l = 1..L       */
     float ms_bootstrap;                           /* last ripple_create / ripple_recompute_full           */
     int64_t gpu_launches;                         /* kernels launched by the last call                    */

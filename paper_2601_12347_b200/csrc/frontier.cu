@@ -205,7 +205,7 @@ __global__ void k_mark_frontier(Ctl* ctl, int l, int self_term, int walk, const 
     if (self_term)
         for (int i = gtid; i < ctl->nA[l - 1]; i += gsize) set_bit(bitmap, A_prev[i]);
     // out-neighbours of the senders of the previous hop (the push scatter marks them itself)
-    if (!walk) return;
+    if (!walk || ctl->regather[l]) return;   // (a rebuilding hop marks bottom-up)
     const int nC = ctl->nC[l - 1];
     if (nC == 0) return;
     const int64_t E = coff[nC];

@@ -215,6 +215,13 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             const char* e = getenv("RIPPLE_NO_PDL");
             c->pdl = !(e && e[0] == '1');
         }
+        {
+            // Hops whose messages are at least this wide gather per sink once they carry a million messages
+            // (measured on the dense graph, 256 floats: see scatter.cu); 0 = never.
+            const char* e = getenv("RIPPLE_GATHER_MIN_WIDTH");
+            c->gather_min_width = e ? atoi(e) : 128;
+            c->gather_min_messages = 1 << 20;
+        }
         tc_prepare();
         max_prepare();
         CK(cudaMallocHost(&c->ctl_host, sizeof(Ctl)));
@@ -485,7 +492,7 @@ static int enqueue_batch(Ctx* c, int nb, bool stamps) {
         // The push scatter walks the same out-lists as the frontier and marks the sinks itself; the
         // gathering forms need the list A_l first, so the frontier walk is a pass of its own for them
         // (decided per hop on the device for the rebuilding form).
-        const bool pull = c->scatter_mode == RIPPLE_SCATTER_PULL;
+        const bool pull = c->pull_hop[l] != 0;
         choose_direction(c, l);
         frontier_mark(c, l, pull, nb);
         if (pull) frontier_compact(c, l);
@@ -530,6 +537,16 @@ static void arm_rebuild(Ctx* c, int nb) {
                                        0.5 * (double)c->regather_threshold[l] * (double)c->stats.num_edges) &&
                     c->stats.num_edges + c->max_batch >= c->regather_min_messages;
         c->rebuild_armed[l] = armed;
+        // The gathering form of the delta scatter is chosen here, from what the hop carried in the batch before
+        // (any choice is correct; a hop that turns out small gathers over a small frontier).
+        bool gather = c->scatter_mode == RIPPLE_SCATTER_PULL;
+        if (c->scatter_mode == RIPPLE_SCATTER_AUTO && !rp_monotonic(c->agg) && !c->attention && c->n_local == 0 &&
+            c->gather_min_width > 0 && c->ws[l] >= c->gather_min_width && !no_history)
+            gather = c->stats.active_edges[l] >= c->gather_min_messages && c->stats.scatter_pull[l] != 2 &&
+                     // the senders' delta rows stay in L2 with room to spare, and a sink's one addition replaces many
+                     (double)c->stats.senders[l - 1] * c->ws[l] * sizeof(float) <= 32.0 * (1 << 20) &&
+                     c->stats.active_edges[l] >= 8 * c->stats.affected[l];
+        c->pull_hop[l] = gather;
     }
 }
 
@@ -541,7 +558,7 @@ static bool launch_batch_graph(Ctx* c, int nb) {
     int key = 4 * nb + (c->may_expand ? 1 : 0) + (c->has_opw ? 2 : 0);
     key = 2 * key + (c->tc_armed ? 1 : 0);
     key = 2 * key + (c->packed_now ? 1 : 0);   // (the chain holds the addresses its kernels read the batch from)
-    for (int l = 1; l <= c->L; ++l) key = 2 * key + (c->rebuild_armed[l] ? 1 : 0);
+    for (int l = 1; l <= c->L; ++l) key = 4 * key + (c->rebuild_armed[l] ? 1 : 0) + (c->pull_hop[l] ? 2 : 0);
     int slot = -1;
     for (int i = 0; i < RP_GRAPH_SLOTS; ++i)
         if (c->graph_exec[i] && c->graph_n[i] == key) slot = i;

@@ -7,6 +7,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+
 #include <stdint.h>
 #include <string.h>
 
@@ -62,6 +63,9 @@ struct Ctl {
     int n_rebuilt[RP_MAXL + 1];       // aggregate rows of hop l gathered anew because their rounding budget ran out
     int rebuild_items[RP_MAXL + 1];   // (vertex, chunk) work items of the long rows among them
     int max_items[RP_MAXL + 1];       // max / min: (long row, chunk) work items of hop l's recomputation
+    int regather_ticket[RP_MAXL + 1]; // rebuilding form: next unassigned position of A_l
+    int gather_ticket[RP_MAXL + 1];   // gathering form of the delta scatter: next unassigned position of A_l
+    int gather_items[RP_MAXL + 1];    // gathering form of the delta scatter: (sink, chunk) work items of the long in-lists
     long long num_edges;              // current edge count (kept across batches)
     int work_counter[8];              // dynamic work distribution tickets (reset by the consumer)
 };
@@ -177,6 +181,9 @@ struct Ctx {
     int scatter_mode, gemm_mode, timing;
     int rebuild_armed[RP_MAXL + 1];   // per hop: the rebuilding form is enqueued for this batch (see arm_rebuild)
     int tc_armed;                     // the tensor-core form of the layer update is enqueued for this batch
+    int pull_hop[RP_MAXL + 1];        // per hop: the delta scatter of this batch gathers per sink instead of pushing (see arm_rebuild)
+    int gather_min_width;             // narrowest message row (floats) whose hop may gather (environment RIPPLE_GATHER_MIN_WIDTH)
+    long long gather_min_messages;    // ... if the hop delivered at least this many messages in the batch before
     long long batches_done;
     int last_nb;
     int debug_tc_withhold;   // diagnostic (environment RIPPLE_DEBUG_TC_WITHHOLD=1): see ripple_create

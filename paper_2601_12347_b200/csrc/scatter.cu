@@ -102,12 +102,17 @@ __device__ __forceinline__ void spmm_accumulate(float4 (&acc)[NV], const Side& i
 template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
 k_spmm_pull(int N, Side in, const int32_t* __restrict__ deg_out, int src_norm,
-            const float* __restrict__ M, int ld, float* __restrict__ S, int2* items, int* n_items) {
+            const float* __restrict__ M, int ld, float* __restrict__ S, int2* items, int* n_items, int* ticket) {
     pdl_enter();
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
     const int sub = lane / LPR, ql = lane % LPR;
-    for (int v = warp; v < N; v += nwarps) {
+    // vertices are handed out in runs of eight by ticket: in-lists differ in length
+    for (;;) {
+        int v0 = 0;
+        if (lane == 0) v0 = atomicAdd(ticket, 8);
+        v0 = __shfl_sync(FULL, v0, 0);
+        if (v0 >= N) break;
+    for (int v = v0; v < min(v0 + 8, N); ++v) {
         const int deg = in.deg[v];
         float4 acc[NV];
 #pragma unroll
@@ -129,6 +134,7 @@ k_spmm_pull(int N, Side in, const int32_t* __restrict__ deg_out, int src_norm,
                 if (q < nq) dst[q] = acc[k];
             }
         }
+    }
     }
 }
 
@@ -175,7 +181,7 @@ void spmm_full(Ctx* c, int l) {
 #define SPMM(NV, LPR)                                                                                              \
     do {                                                                                                           \
         RP_LAUNCH(c, (k_spmm_pull<NV, LPR>), grid, T, 0, c->N, c->side[1], c->side[0].deg, (int)c->src_norm, M,   \
-                  ld, c->S[l], items, n_items);                                                                    \
+                  ld, c->S[l], items, n_items, &c->ctl->regather_ticket[l]);                                      \
         RP_LAUNCH(c, (k_spmm_hubs<NV, LPR>), grid, T, 0, c->side[1], c->side[0].deg, (int)c->src_norm, M, ld,     \
                   c->S[l], items, n_items);                                                                        \
     } while (0)
@@ -381,56 +387,175 @@ k_scatter_push_bulk(Ctl* ctl, int l, const int32_t* __restrict__ senders, const 
 }
 
 // ---------------------------------------------------------------------------------------------
-// pull scatter
+// gathering form of the delta scatter: per affected sink, the delta rows of the senders among its
+// in-neighbours are summed in registers and reach the accumulator row as ONE addition.  The sender
+// delta rows are few (they stay in L2, the hubs' rows in L1) and are read with plain loads; no
+// accumulator row is touched more than once.  It pays where a message is wide: 256-float
+// messages cost the push one kilobyte of read-modify-write each in the L2 slices and evict each
+// other's accumulator rows in between.
+//
+// A warp examines GATHER_WINDOW in-list entries at a time (four per lane, their position-map
+// lookups in flight together), compacts the hits into shared memory and then gathers them like
+// the bootstrap gather does: LPR lanes per row, 32 / LPR rows per step, several steps in flight.
 // ---------------------------------------------------------------------------------------------
+constexpr int GATHER_WINDOW = 128;
+constexpr int GATHER_LONG = 1024;    // longer in-lists are cut into work items of this many entries
+constexpr int GATHER_TAKE = 8;       // sinks per ticket
+
+template <int NV, int LPR>
+__device__ __forceinline__ bool gather_accumulate(float4 (&acc)[NV], const Side& in, int v, int j_begin, int j_end,
+                                                  const int32_t* __restrict__ posmap, const float* __restrict__ D,
+                                                  int ld, int2* hits) {
+    const int lane = lane_id(), nq = ld >> 2;
+    constexpr int EPI = 32 / LPR;
+    constexpr int UNR = NV <= 2 ? 4 : 2;
+    constexpr int PER_LANE = GATHER_WINDOW / 32;
+    const int sub = lane / LPR, ql = lane % LPR;
+    const int64_t base = in.start[v];
+    const unsigned lt = (1u << lane) - 1u;
+    bool any = false;
+    for (int j0 = j_begin; j0 < j_end; j0 += GATHER_WINDOW) {
+        int u[PER_LANE], p[PER_LANE];
+        float w[PER_LANE];
+#pragma unroll
+        for (int k = 0; k < PER_LANE; ++k) {
+            const int j = j0 + 32 * k + lane;
+            u[k] = j < j_end ? in.col[base + j] : -1;
+            w[k] = (in.w && j < j_end) ? in.w[base + j] : 1.0f;
+        }
+#pragma unroll
+        for (int k = 0; k < PER_LANE; ++k) p[k] = u[k] >= 0 ? posmap[u[k]] : -1;
+        int cnt = 0;
+        __syncwarp();   // the hits of the window before have all been read
+#pragma unroll
+        for (int k = 0; k < PER_LANE; ++k) {
+            const unsigned m = __ballot_sync(FULL, p[k] >= 0);
+            if (p[k] >= 0) hits[cnt + __popc(m & lt)] = make_int2(p[k], __float_as_int(w[k]));
+            cnt += __popc(m);
+        }
+        __syncwarp();
+        if (cnt == 0) continue;
+        any = true;
+        for (int j = 0; j < cnt; j += UNR * EPI) {
+            int pj[UNR];
+            float a[UNR];
+            float4 x[UNR][NV];
+#pragma unroll
+            for (int t = 0; t < UNR; ++t) {
+                const int jj = j + t * EPI + sub;
+                pj[t] = -1;
+                a[t] = 0.f;
+                if (jj < cnt) {
+                    const int2 h = hits[jj];
+                    pj[t] = h.x;
+                    a[t] = __int_as_float(h.y);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < UNR; ++t) {
+                const float4* row = reinterpret_cast<const float4*>(D + (size_t)max(pj[t], 0) * ld);
+#pragma unroll
+                for (int k = 0; k < NV; ++k) {
+                    const int q = ql + LPR * k;
+                    x[t][k] = (pj[t] >= 0 && q < nq) ? __ldg(row + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < UNR; ++t)
+#pragma unroll
+                for (int k = 0; k < NV; ++k) add4(acc[k], x[t][k], a[t]);
+        }
+    }
+    if (any) {
+#pragma unroll
+        for (int k = 0; k < NV; ++k) {
+#pragma unroll
+            for (int o = LPR; o < 32; o <<= 1) {
+                acc[k].x += __shfl_xor_sync(FULL, acc[k].x, o);
+                acc[k].y += __shfl_xor_sync(FULL, acc[k].y, o);
+                acc[k].z += __shfl_xor_sync(FULL, acc[k].z, o);
+                acc[k].w += __shfl_xor_sync(FULL, acc[k].w, o);
+            }
+        }
+    }
+    return any;
+}
+
+// One warp per affected sink; a sink with a long in-list only queues (sink, chunk) work items.
 template <int NV, int LPR>
 __global__ void __launch_bounds__(256)
-k_scatter_pull(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_t* __restrict__ posmap,
-               const float* __restrict__ D, int ld, float* S) {
+k_scatter_gather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_t* __restrict__ posmap,
+                 const float* __restrict__ D, int ld, float* dS, int2* items) {
     pdl_enter();
+    __shared__ int2 s_hits[8][GATHER_WINDOW];
     if (ctl->abort || !ctl->pull[l] || ctl->regather[l]) return;
     const int nA = ctl->nA[l];
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
-    for (int i = warp; i < nA; i += nwarps) {
+    const int sub = lane / LPR, ql = lane % LPR;
+    int2* hits = s_hits[threadIdx.x >> 5];
+    // sinks are handed out in runs of GATHER_TAKE by ticket: in-lists differ in length by orders of magnitude,
+    // and the grid need not match the number of resident blocks
+    for (;;) {
+        int i0 = 0;
+        if (lane == 0) i0 = atomicAdd(&ctl->gather_ticket[l], GATHER_TAKE);
+        i0 = __shfl_sync(FULL, i0, 0);
+        if (i0 >= nA) break;
+    for (int i = i0; i < min(i0 + GATHER_TAKE, nA); ++i) {
         const int v = A[i];
+        const int deg = in.deg[v];
+        if (deg > GATHER_LONG) {
+            const int nch = (deg + GATHER_LONG - 1) / GATHER_LONG;
+            int first = 0;
+            if (lane == 0) first = atomicAdd(&ctl->gather_items[l], nch);
+            first = __shfl_sync(FULL, first, 0);
+            for (int ch = lane; ch < nch; ch += 32) items[first + ch] = make_int2(v, ch);
+            continue;
+        }
         float4 acc[NV];
 #pragma unroll
         for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        const int64_t base = in.start[v];
-        const int deg = in.deg[v];
-        bool any = false;
-        for (int j0 = 0; j0 < deg; j0 += 32) {
-            int p = -1;
-            float wj = 1.0f;
-            if (j0 + lane < deg) {
-                p = posmap[in.col[base + j0 + lane]];
-                if (in.w) wj = in.w[base + j0 + lane];
-            }
-            unsigned m = __ballot_sync(FULL, p >= 0);
-            any |= m != 0;
-            while (m) {
-                int j = __ffs(m) - 1;
-                m &= m - 1;
-                int pj = __shfl_sync(FULL, p, j);
-                const float a = __shfl_sync(FULL, wj, j);
-                const float4* drow = reinterpret_cast<const float4*>(D + (size_t)pj * ld);
+        if (!gather_accumulate<NV, LPR>(acc, in, v, 0, deg, posmap, D, ld, hits)) continue;
+        if (sub == 0) {
+            // the accumulator is zero outside a batch and this is the hop's first kernel to touch the row
+            // (edge records are added after it): a plain store
+            float4* dst = reinterpret_cast<float4*>(dS + (size_t)v * ld);
 #pragma unroll
-                for (int k = 0; k < NV; ++k) {
-                    int q = lane + 32 * k;
-                    if (q < nq) add4(acc[k], __ldg(drow + q), a);
-                }
+            for (int k = 0; k < NV; ++k) {
+                const int q = ql + LPR * k;
+                if (q < nq) dst[q] = acc[k];
             }
         }
-        if (!any) continue;
-        float4* dst = reinterpret_cast<float4*>(S + (size_t)v * ld);
+    }
+    }
+}
+
+// the chunks of the long in-lists: several warps add into the same accumulator row
+template <int NV, int LPR>
+__global__ void __launch_bounds__(256)
+k_scatter_gather_long(Ctl* ctl, int l, Side in, const int32_t* __restrict__ posmap, const float* __restrict__ D, int ld,
+                      float* dS, const int2* __restrict__ items) {
+    pdl_enter();
+    __shared__ int2 s_hits[8][GATHER_WINDOW];
+    if (ctl->abort || !ctl->pull[l] || ctl->regather[l]) return;
+    const int n = ctl->gather_items[l];
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = lane_id(), nq = ld >> 2;
+    const int sub = lane / LPR, ql = lane % LPR;
+    int2* hits = s_hits[threadIdx.x >> 5];
+    for (int it = warp; it < n; it += nwarps) {
+        const int2 w = items[it];
+        const int deg = in.deg[w.x];
+        float4 acc[NV];
 #pragma unroll
-        for (int k = 0; k < NV; ++k) {
-            int q = lane + 32 * k;
-            if (q < nq) {
-                float4 s = dst[q];
-                s.x += acc[k].x; s.y += acc[k].y; s.z += acc[k].z; s.w += acc[k].w;
-                dst[q] = s;
+        for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (!gather_accumulate<NV, LPR>(acc, in, w.x, w.y * GATHER_LONG, min(deg, (w.y + 1) * GATHER_LONG), posmap, D, ld,
+                                        hits))
+            continue;
+        if (sub == 0) {
+#pragma unroll
+            for (int k = 0; k < NV; ++k) {
+                const int q = ql + LPR * k;
+                if (q < nq) red_add_v4(dS + (size_t)w.x * ld + 4 * q, acc[k]);
             }
         }
     }
@@ -482,10 +607,15 @@ k_regather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_
     pdl_enter();
     if (ctl->abort || !ctl->regather[l]) return;
     const int nA = ctl->nA[l];
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
     const int sub = lane / LPR, ql = lane % LPR;
-    for (int i = warp; i < nA; i += nwarps) {
+    // rows are handed out in runs of eight by ticket (the grid need not match the number of resident blocks)
+    for (;;) {
+        int i0 = 0;
+        if (lane == 0) i0 = atomicAdd(&ctl->regather_ticket[l], 8);
+        i0 = __shfl_sync(FULL, i0, 0);
+        if (i0 >= nA) break;
+    for (int i = i0; i < min(i0 + 8, nA); ++i) {
         const int v = A[i];
         const int deg = in.deg[v];
         float4 acc[NV];
@@ -509,6 +639,7 @@ k_regather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const int32_
             }
         }
         if (budget && lane == 0) budget[v] = 0.f;   // a freshly gathered row has spent nothing
+    }
     }
 }
 
@@ -576,8 +707,8 @@ k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int
 //
 // Delta form: the out-edges of the senders each carry one message, added to the sink's aggregate
 // by a vector reduction (push), or gathered per sink over the senders among its in-neighbours
-// (pull; measured slower at every size because of the per-edge membership lookup, kept
-// selectable for comparison).
+// (k_scatter_gather: chosen on the host, per hop, for wide messages from few senders; slower than
+// the push for narrow rows because of the per-edge membership lookup).
 //
 // Rebuilding form: once the senders' out-edges are most of the graph, reading every in-edge of
 // the affected sinks once and overwriting their aggregates costs less than one reduction per
@@ -587,7 +718,7 @@ k_regather_rows(Ctl* ctl, int l, const Rec* __restrict__ rec, Side in, const int
 // of fewer than min_messages messages pushes regardless: on a graph of a million edges neither
 // form is throughput-bound, and the edge-balanced push is the more parallel of the two (measured
 // on the sparse graph, 256 floats per row: 0.24 ms pushed, 0.26 to 0.47 ms rebuilt).
-__global__ void k_choose_direction(Ctl* ctl, int l, int mode, float threshold, long long min_messages) {
+__global__ void k_choose_direction(Ctl* ctl, int l, int mode, int gather, float threshold, long long min_messages) {
     pdl_enter();
     const int nC = ctl->nC[l - 1];
     int re = 0;
@@ -598,7 +729,7 @@ __global__ void k_choose_direction(Ctl* ctl, int l, int mode, float threshold, l
              msgs >= (unsigned long long)min_messages;
     }
     if (nC == 0 && ctl->n_rec == 0) re = 0;
-    ctl->pull[l] = mode == RIPPLE_SCATTER_PULL;
+    ctl->pull[l] = gather;
     ctl->regather[l] = re;
 }
 
@@ -685,9 +816,10 @@ void fold_deltas(Ctx* c, int l) {
 
 void choose_direction(Ctx* c, int l) {
     // nothing to decide for a pushing hop: the control block's flags are already zero after its reset
-    if (!c->rebuild_armed[l] && (c->scatter_mode == RIPPLE_SCATTER_AUTO || c->scatter_mode == RIPPLE_SCATTER_PUSH ||
-                                 c->scatter_mode == RIPPLE_SCATTER_PUSH_BULK)) return;
-    RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode,
+    if (!c->rebuild_armed[l] && !c->pull_hop[l] &&
+        (c->scatter_mode == RIPPLE_SCATTER_AUTO || c->scatter_mode == RIPPLE_SCATTER_PUSH ||
+         c->scatter_mode == RIPPLE_SCATTER_PUSH_BULK)) return;
+    RP_LAUNCH(c, k_choose_direction, 1, 1, 0, c->ctl, l, c->scatter_mode, (int)c->pull_hop[l],
               c->rebuild_armed[l] ? c->regather_threshold[l] : -1.f, c->regather_min_messages);
 }
 
@@ -710,12 +842,19 @@ void scatter_layer(Ctx* c, int l, int n) {
     }
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l], c->stream);
 #define PUSH(NV, LPR) RP_LAUNCH(c, (k_scatter_push<NV, LPR>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, ld, c->dS[l], c->bitmap)
-#define PULL(NV, LPR) RP_LAUNCH(c, (k_scatter_pull<NV, 32>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->posmap, Dm, ld, c->dS[l])
+    int2* gather_items = reinterpret_cast<int2*>(c->coff);   // (the marking walk was the last reader of the degree prefix)
+#define PULL(NV, LPR)                                                                                                  \
+    do {                                                                                                               \
+        RP_LAUNCH(c, (k_scatter_gather<NV, LPR>), grid, T, 0, c->ctl, l, c->A[l], c->side[1], c->posmap, Dm, ld,      \
+                  c->dS[l], gather_items);                                                                             \
+        RP_LAUNCH(c, (k_scatter_gather_long<NV, LPR>), grid, T, 0, c->ctl, l, c->side[1], c->posmap, Dm, ld, c->dS[l], \
+                  (const int2*)gather_items);                                                                          \
+    } while (0)
     // (rows too wide for two staging buffers per warp in the default shared-memory allowance take the ordinary form)
     if (c->scatter_mode == RIPPLE_SCATTER_PUSH_BULK && !c->weighted && (size_t)8 * 2 * ld * sizeof(float) <= (48u << 10)) {
         RP_LAUNCH(c, k_scatter_push_bulk, grid, T, (size_t)8 * 2 * ld * sizeof(float), c->ctl, l, senders, c->coff,
                   c->side[0], Dm, ld, c->dS[l], c->bitmap);
-    } else if (c->scatter_mode != RIPPLE_SCATTER_PULL && c->scatter_mode != RIPPLE_SCATTER_REGATHER) {
+    } else if (!c->pull_hop[l] && c->scatter_mode != RIPPLE_SCATTER_REGATHER) {
 #define PACKED(NQ, WGT) RP_LAUNCH(c, (k_scatter_push_packed<NQ, WGT>), grid, T, 0, c->ctl, l, senders, c->coff, c->side[0], Dm, c->dS[l], c->bitmap)
         if (ld == 48 && c->weighted) PACKED(12, true);
         else if (ld == 48) PACKED(12, false);
@@ -724,7 +863,7 @@ void scatter_layer(Ctx* c, int l, int n) {
 #undef PACKED
         else RP_WIDTH_DISPATCH(ld, PUSH);
     }
-    if (c->scatter_mode == RIPPLE_SCATTER_PULL) RP_WIDTH_DISPATCH(ld, PULL);
+    if (c->pull_hop[l]) RP_WIDTH_DISPATCH(ld, PULL);
 #undef PUSH
 #undef PULL
     if (c->timing) cudaEventRecord(c->ev_sc[2 * l + 1], c->stream);
@@ -732,7 +871,7 @@ void scatter_layer(Ctx* c, int l, int n) {
         RP_LAUNCH(c, k_scatter_records, std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec,
                   (int)c->src_norm, c->side[0].deg, c->posmap, Mrows, Dm, ld, c->dS[l]);
         const float* rows = c->pre[l] ? c->P[l] : c->H[l - 1];
-#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l], c->Eb[l], senders, c->posmap, (int)(c->scatter_mode != RIPPLE_SCATTER_PULL), (int)c->self_term, c->A[l - 1], c->bitmap, (int)(c->n_local > 0))
+#define ROWS(NV, LPR) RP_LAUNCH(c, (k_regather_rows<NV, LPR>), std::min(div_up(n, T / 32), c->n_sm * 8), T, 0, c->ctl, l, c->rec, c->side[1], c->side[0].deg, (int)c->src_norm, rows, ld, c->S[l], c->dS[l], c->Eb[l], senders, c->posmap, (int)(!c->pull_hop[l]), (int)c->self_term, c->A[l - 1], c->bitmap, (int)(c->n_local > 0))
         RP_WIDTH_DISPATCH(ld, ROWS);
 #undef ROWS
     }

@@ -230,12 +230,13 @@ def test_full_size_gcx_batches_against_the_hybrid_oracle(env):
     orc.close()
 
 
-# workload, batches, the form of each hop in the last batch (0 = delta messages pushed, 2 = aggregates rebuilt)
+# workload, batches, the form of each hop in the last batch (0 = delta messages pushed, 1 = delta messages gathered per
+# sink: wide messages from few senders, chosen from the batch before; 2 = aggregates rebuilt)
 DEEP_CASES = [
-    ("dense-3l", 2, [0, 0, 2]),
+    ("dense-3l", 3, [0, 1, 2]),
     ("dense-3l-hub-feature", 5, [0, 2, 2]),
     ("dense-3l-hub-delete", 5, [0, 2, 2]),
-    ("dense-4l", 2, [0, 0, 2, 2]),
+    ("dense-4l", 2, [0, 1, 2, 2]),
     ("dense-gat-2l", 3, [0, 0]),        # attention layers never take the rebuilding form: recomputation is per vertex
     ("dense-gat-3l", 2, [0, 0, 0]),
     ("reddit-2l", 2, [0, 2]),
