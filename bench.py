@@ -487,7 +487,7 @@ def run_table(args):
             lat, sc_ms, sc_bytes = [], 0.0, 0
             stage = {"graph": 0.0, "frontier": 0.0, "scatter": 0.0, "update": 0.0}
             aff, act = np.zeros(L + 1), np.zeros(L + 1)
-            hop = {k: np.zeros(L + 1) for k in ("scatter", "update", "regather", "rebuilt", "in_edges", "rows_rebuilt")}
+            hop = {k: np.zeros(L + 1) for k in ("scatter", "update", "regather", "rebuilt", "gathered", "in_edges", "rows_rebuilt")}
             rp.set_timing(False)
             for i, (u, r, ow) in enumerate(pinned):
                 if i == 5 + nb:
@@ -511,6 +511,7 @@ def run_table(args):
                 hop["update"] += np.array(s["ms_update"][: L + 1])
                 hop["regather"] += np.array(s["ms_regather"][: L + 1])
                 hop["rebuilt"] += np.array(s["scatter_pull"][: L + 1]) == 2
+                hop["gathered"] += np.array(s["scatter_pull"][: L + 1]) == 1
                 hop["in_edges"] += np.array(s["in_edges"][: L + 1]) * (np.array(s["scatter_pull"][: L + 1]) == 2)
                 hop["rows_rebuilt"] += np.array(s["rows_rebuilt"][: L + 1])
                 sc_bytes += scatter_bytes(s, L, s["message_width"][L])
