@@ -313,7 +313,8 @@ def run_ours(args, rank, world, local_rank):
     sc_ms, sc_bytes, stage = 0.0, 0, {"graph": 0.0, "frontier": 0.0, "scatter": 0.0, "update": 0.0}
     sizes = {"affected": np.zeros(L + 1), "active_edges": np.zeros(L + 1)}
     ld_last = (w.model.dims[L - 1] + 3) // 4 * 4
-    pulls = 0
+    pulls = rebuilt = 0
+    rg_ms, rg_edges = 0.0, 0
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     sampler.start()
@@ -327,7 +328,10 @@ def run_ours(args, rank, world, local_rank):
             stage["frontier"] += s["ms_frontier"][l]
             stage["scatter"] += s["ms_scatter"][l]
             stage["update"] += s["ms_update"][l]
-        pulls += s["scatter_pull"][L]
+        pulls += s["scatter_pull"][L] == 1
+        rebuilt += s["scatter_pull"][L] == 2
+        rg_ms += s["ms_regather"][L]
+        rg_edges += s["in_edges"][L] if s["scatter_pull"][L] == 2 else 0
         sc_ms += s["ms_scatter_kernel"][L]
         ld_last = s["message_width"][L]
         sc_bytes += scatter_bytes(s, L, ld_last)
@@ -379,7 +383,7 @@ def run_ours(args, rank, world, local_rank):
     # window, the fastest pattern of that path, timed live by the library's probe.
     msgs = float(sizes["active_edges"][L]) / K
     graph_kind = args.workload.split("-")[0]
-    per_msg = NCU_DRAM_BYTES_PER_MESSAGE.get((graph_kind, ld_last)) if pulls == 0 else None
+    per_msg = NCU_DRAM_BYTES_PER_MESSAGE.get((graph_kind, ld_last)) if pulls == 0 and rebuilt == 0 else None
     traffic = per_msg * msgs if per_msg else None
     payload = msgs * ld_last * 4
     achieved = payload / 1e9 / (sc_ms / K / 1e3) if sc_ms > 0 else None
@@ -427,7 +431,25 @@ def run_ours(args, rank, world, local_rank):
     rp.close()
     del rp
     torch.cuda.empty_cache()
-    if pulls == 0 and sc_ms > 0 and msgs >= 1:
+    if rebuilt * 2 > K and rg_ms > 0:
+        # The last hop rebuilt its aggregates in most steps: the dominant kernels are the gather over the in-lists of
+        # the affected sinks, bounded by the rate at which L2 serves whole-row gathers.  achieved = in-edges x row
+        # bytes per second; peak = the library's gather probe (same lane layout, no index traffic) on a 64 MB window.
+        edges = rg_edges / rebuilt
+        ms = rg_ms / rebuilt
+        got = edges * ld_last * 4 / 1e9 / (ms / 1e3)
+        pk = edges * ld_last * 4 / 1e9 / (ripple.probe_gather_rate(max(1, (64 << 20) // (ld_last * 4)), ld_last, int(edges)) / 1e3)
+        per_edge = NCU_DRAM_BYTES_PER_IN_EDGE.get((graph_kind, ld_last))
+        traffic = per_edge * edges if per_edge else None
+        line["roofline"] = {
+            "bound": "l2-gather", "achieved": got, "peak": pk, "unit": "GB/s", "frac": got / pk, "traffic": traffic,
+            "frac_hbm": (traffic / 1e9 / (ms / 1e3) / hbm_peak) if traffic else None,
+            "hbm_peak": hbm_peak, "hbm_peak_source": f"of {peak_kind}",
+            "kernel": f"k_regather + k_spmm_hubs (hop {L}, row width {ld_last} floats)",
+            "ms_per_launch": ms, "in_edges_per_launch": edges, "rebuilt_steps": int(rebuilt),
+            "note": "the last hop rebuilds the affected aggregates from their in-lists; achieved = in-edges x row bytes / "
+                    "time of the two gather kernels; peak = probe of L2 row gathers on a 64 MB window"}
+    elif pulls == 0 and sc_ms > 0 and msgs >= 1:
         # The push scatter is made of 16-byte vector reductions that mostly land in L2.  The same
         # number of reductions of the same row width into pseudo-random rows, timed alone, gives the
         # ceiling of that path on this GPU: with a window that fits L2, and with a window of the

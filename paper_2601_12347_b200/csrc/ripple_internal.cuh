@@ -65,6 +65,7 @@ struct Ctl {
     int max_items[RP_MAXL + 1];       // max / min: (long row, chunk) work items of hop l's recomputation
     int regather_ticket[RP_MAXL + 1]; // rebuilding form: next unassigned position of A_l
     int gather_ticket[RP_MAXL + 1];   // gathering form of the delta scatter: next unassigned position of A_l
+    int gather_long_ticket[RP_MAXL + 1];  // ... and next unassigned work item of the long in-lists
     int gather_items[RP_MAXL + 1];    // gathering form of the delta scatter: (sink, chunk) work items of the long in-lists
     long long num_edges;              // current edge count (kept across batches)
     int work_counter[8];              // dynamic work distribution tickets (reset by the consumer)

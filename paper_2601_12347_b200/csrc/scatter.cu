@@ -399,7 +399,8 @@ k_scatter_push_bulk(Ctl* ctl, int l, const int32_t* __restrict__ senders, const 
 // the bootstrap gather does: LPR lanes per row, 32 / LPR rows per step, several steps in flight.
 // ---------------------------------------------------------------------------------------------
 constexpr int GATHER_WINDOW = 128;
-constexpr int GATHER_LONG = 1024;    // longer in-lists are cut into work items of this many entries
+constexpr int GATHER_LONG = 512;     // longer in-lists are cut into work items of GATHER_ITEM entries
+constexpr int GATHER_ITEM = 256;
 constexpr int GATHER_TAKE = 8;       // sinks per ticket
 
 template <int NV, int LPR>
@@ -504,7 +505,7 @@ k_scatter_gather(Ctl* ctl, int l, const int32_t* __restrict__ A, Side in, const 
         const int v = A[i];
         const int deg = in.deg[v];
         if (deg > GATHER_LONG) {
-            const int nch = (deg + GATHER_LONG - 1) / GATHER_LONG;
+            const int nch = (deg + GATHER_ITEM - 1) / GATHER_ITEM;
             int first = 0;
             if (lane == 0) first = atomicAdd(&ctl->gather_items[l], nch);
             first = __shfl_sync(FULL, first, 0);
@@ -538,17 +539,21 @@ k_scatter_gather_long(Ctl* ctl, int l, Side in, const int32_t* __restrict__ posm
     __shared__ int2 s_hits[8][GATHER_WINDOW];
     if (ctl->abort || !ctl->pull[l] || ctl->regather[l]) return;
     const int n = ctl->gather_items[l];
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     const int lane = lane_id(), nq = ld >> 2;
     const int sub = lane / LPR, ql = lane % LPR;
     int2* hits = s_hits[threadIdx.x >> 5];
-    for (int it = warp; it < n; it += nwarps) {
+    // items by ticket: they are equally long, but the senders among their entries are not equally many
+    for (;;) {
+        int it = 0;
+        if (lane == 0) it = atomicAdd(&ctl->gather_long_ticket[l], 1);
+        it = __shfl_sync(FULL, it, 0);
+        if (it >= n) break;
         const int2 w = items[it];
         const int deg = in.deg[w.x];
         float4 acc[NV];
 #pragma unroll
         for (int k = 0; k < NV; ++k) acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (!gather_accumulate<NV, LPR>(acc, in, w.x, w.y * GATHER_LONG, min(deg, (w.y + 1) * GATHER_LONG), posmap, D, ld,
+        if (!gather_accumulate<NV, LPR>(acc, in, w.x, w.y * GATHER_ITEM, min(deg, (w.y + 1) * GATHER_ITEM), posmap, D, ld,
                                         hits))
             continue;
         if (sub == 0) {

@@ -628,6 +628,53 @@ def test_rebuilding_hops_with_long_in_lists(env):
     rp.close()
 
 
+@pytest.mark.parametrize("kind", ["sage_mean", "gcn_wsum", "gcw"])
+def test_gathered_delta_scatter_with_long_in_lists(env, kind):
+    """The gathering form of the delta scatter on every hop: sinks whose in-lists are cut into work items of 1024
+    entries (5000 and 2300 in-neighbours, a ragged last item and a ragged last window of 128), few and many senders
+    among them, widths on both sides of a warp per row, stored edge weights."""
+    ripple, Oracle = env
+    if kind == "sage_mean":
+        model = I.sage_model([20, 128, 160, 12], I.AGG_MEAN)
+    elif kind == "gcn_wsum":
+        model = I.graphconv_model([20, 36, 260, 12], I.AGG_WSUM_GCN)
+    else:
+        model = I.graphconv_model([20, 132, 40, 12], I.AGG_WSUM_EDGE)
+    L = 3
+    n = 6000
+    src, dst = I.er_graph(n, 30000, 12)
+    have = set(zip(src.tolist(), dst.tolist()))
+    extra = [(u, 7) for u in range(100, 5100) if (u, 7) not in have]
+    extra += [(u, 9) for u in range(0, 2300) if (u, 9) not in have and u != 9]
+    extra += [(7, v) for v in range(200, 3200) if (7, v) not in have]
+    src = np.concatenate([src, np.array([a for a, _ in extra], dtype=np.int32)])
+    dst = np.concatenate([dst, np.array([b for _, b in extra], dtype=np.int32)])
+    X = I.features(n, 20, 12)
+    W = I.make_weights(model, 12, zero_bias=False)
+    kw = {"edge_weights": I.edge_weights(src.size, 12)} if kind == "gcw" else {}
+    rp = ripple.Ripple(n, src, dst, X, model, W, scatter_mode=ripple.SCATTER_PULL, **kw)
+    orc = Oracle(n, src, dst, X, model, W, **kw)
+    stream = I.UpdateStream(n, src, dst, 20, 12)
+    for b, bs in enumerate([1, 20, 300, 5, 1000, 50, 2, 400]):
+        if kind == "gcw":
+            ups, rows, ow = stream.next_batch_weighted(bs)
+        else:
+            (ups, rows), ow = stream.next_batch(bs), None
+        if b == 3:   # the hub's 3000 out-edges carry a message, then most of the graph sends
+            if rows.shape[0] == 0:
+                rows = I.features(1, 20, 99)
+            ups = np.concatenate([ups, ups_array([(I.OP_SET_FEATURE, 7, 0)])])
+            if ow is not None:
+                ow = np.concatenate([ow, np.ones(1, dtype=np.float32)])
+        rp.apply_batch(ups, rows, ow) if ow is not None else rp.apply_batch(ups, rows)
+        assert (orc.apply_incremental(ups, rows, op_weights=ow) if ow is not None else orc.apply_incremental(ups, rows)) == 0
+        check_graph(rp, orc)
+        check_frontiers(rp, orc, L)
+        assert all(f == 1 for f in rp.stats()["scatter_pull"][1:L + 1])
+        check_values(rp, orc.full(), L, [None] + [orc.full_S(l) for l in range(1, L + 1)])
+    rp.close()
+
+
 def test_rounding_budget_gathers_rows_anew(env):
     """Every fold of a batch's messages into a cached aggregate rounds at the row's magnitude of the
     moment.  A sink that loses the edge from a vertex with a huge row keeps that rounding on its now
