@@ -47,6 +47,7 @@ struct UpdParams {
     int tc_mode;                    // TC_OFF: SIMT only
     int tc_min_rows;
     int tc_withhold;                // diagnostic: the tensor-core kernel never signals its first finished tile
+    int narrow_min_rows;            // > 0: launches of at least this many rows belong to the form for narrow outputs
 };
 
 __device__ __forceinline__ float coef_deg(int deg) { return deg > 0 ? 1.0f / sqrtf((float)deg) : 0.0f; }
@@ -56,6 +57,11 @@ __device__ __forceinline__ int upd_rows(const UpdParams& p) { return p.n_dev ? *
 // true if this launch's row count belongs to the tensor-core kernel
 __device__ __forceinline__ bool upd_use_tc(const UpdParams& p, int n) {
     return p.tc_mode != TC_OFF && n >= p.tc_min_rows;
+}
+
+// true if this launch's row count belongs to the SIMT form for narrow outputs (k_update_rows_narrow)
+__device__ __forceinline__ bool upd_use_narrow(const UpdParams& p, int n) {
+    return p.narrow_min_rows > 0 && n >= p.narrow_min_rows;
 }
 
 __device__ __forceinline__ float upd_row_scale(const UpdParams& p, int v) {
