@@ -173,27 +173,37 @@ k_update_rows(const Ctl* ctl, UpdParams p) {
 // Outputs of at most 48 columns over many rows (the last layers of the configurations: 47 and 40 classes, as the
 // neighbour and the self projection of a million senders): the 64 x 64 tile above leaves a quarter of its threads
 // multiplying zero columns, and it waits for every chunk of K before it multiplies it.  Here a tile is 256 rows x 48
-// columns; a warp owns six columns (its loads of the weights are uniform: one broadcast), a lane eight rows, four
-// consecutive ones in each half of the tile (its 16-byte loads of A are consecutive across the lanes); K is walked in
-// chunks of 16 that are requested one chunk ahead, raw, so that they travel while the chunk before is multiplied
-// (the factor on the A operand is applied when the chunk is put into shared memory); the finished tile goes through
-// shared memory once more so that the epilogue sees 16-byte pieces of rows.  One source per A entry: the operand
-// alpha h + scale S of GIN layers stays with the tiled form.
-constexpr int NBM = 256, NBN = 48, NBK = 16, NTM = 8, NTN = 6, NARROW_MIN_ROWS = 4096;
+// columns.  The gathered rows arrive through a ring of NST stages filled by cp.async, 16 entries of K per stage and
+// row, NST - 1 chunks ahead of the one being multiplied and without passing through registers.  A warp owns six
+// columns (its loads of the weights are uniform: one broadcast), a lane the eight rows ty, ty + 32, ...; it reads
+// four entries of K per row with one 16-byte load (rows are 20 floats apart in a stage, so the loads of eight
+// consecutive lanes fall into eight different 16-byte bank groups).  The factor on the A operand is per row: it is
+// applied to the finished sums.  The finished tile goes through shared memory once more so that the epilogue sees
+// 16-byte pieces of rows.  One source per A entry: the operand alpha h + scale S of GIN layers stays with the tiled form.
+constexpr int NBM = 256, NBN = 48, NBK = 16, NTM = 8, NTN = 6, NST = 4, NARROW_MIN_ROWS = 65536;
+constexpr int NAS_LD = NBK + 4, NCS_LD = NBN + 4;
+constexpr size_t NARROW_SMEM = sizeof(float) * ((size_t)NST * NBM * NAS_LD + 2 * NBK * NBN + 2 * NBM) + sizeof(int) * NBM;
+static_assert(NST * NBM * NAS_LD >= (NBM / 2) * NCS_LD, "the finished half tile is staged in the ring");
+
+__device__ __forceinline__ void cp_async16_zfill(float* smem_dst, const float* gptr, bool valid) {
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    const int bytes = valid ? 16 : 0;      // (0: sixteen zero bytes are written, nothing is read)
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gptr), "r"(bytes) : "memory");
+}
 
 __global__ void __launch_bounds__(256, 2)
 k_update_rows_narrow(const Ctl* ctl, UpdParams p) {
     pdl_enter();
     if (ctl->abort) return;
-    constexpr int AS_LD = NBM + 4, CS_LD = NBN + 4;
-    constexpr int BUF = NBK * AS_LD > (NBM / 2) * CS_LD ? NBK * AS_LD : (NBM / 2) * CS_LD;
-    __shared__ __align__(16) float buf[BUF];             // As[NBK][AS_LD], later the finished tile, half at a time
-    __shared__ __align__(16) float Bs[NBK][64];          // a warp's six columns start at a multiple of eight
-    __shared__ int row_id[NBM];
-    __shared__ float row_scale[NBM];
+    extern __shared__ __align__(16) float nsm[];
+    float* ring = nsm;                                   // [NST][NBM][NAS_LD], later the finished tile, half at a time
+    float* Bs = ring + (size_t)NST * NBM * NAS_LD;       // [2][NBK][NBN]
+    float* row_scale = Bs + 2 * NBK * NBN;               // [NBM]
+    float* row_fac = row_scale + NBM;                    // [NBM]
+    int* row_id = reinterpret_cast<int*>(row_fac + NBM); // [NBM]
     const int n = upd_rows(p);
     if (!upd_use_narrow(p, n)) return;
-    const int row_tiles = (n + NBM - 1) / NBM;
+    const int row_tiles = (n + NBM - 1) / NBM, chunks = (p.K + NBK - 1) / NBK;
     const int tid = threadIdx.x, tx = tid >> 5, ty = tid & 31;
     for (int rt = blockIdx.x; rt < row_tiles; rt += gridDim.x) {
         const int r0 = rt * NBM;
@@ -208,6 +218,7 @@ k_update_rows_narrow(const Ctl* ctl, UpdParams p) {
             }
             row_id[tid] = v;
             row_scale[tid] = sc;
+            row_fac[tid] = p.a_mode == A_DENSE ? 1.0f : p.a_mode == A_SELF ? p.alpha : sc;
         }
         __syncthreads();
         float acc[NTM][NTN];
@@ -215,85 +226,98 @@ k_update_rows_narrow(const Ctl* ctl, UpdParams p) {
         for (int a2 = 0; a2 < NTM; ++a2)
 #pragma unroll
             for (int b2 = 0; b2 < NTN; ++b2) acc[a2][b2] = 0.f;
-        const int ar = tid >> 2, ak = (tid & 3) * 4;   // A tile: rows ar + 64 s, k offset ak .. ak + 3
-        const int bk = tid / (NBN / 4), bq = tid - bk * (NBN / 4);   // B tile: NBK rows of NBN / 4 pieces (192 threads)
+        // this thread's part of a chunk of A: rows ar + 64 s, entries ak .. ak + 3 of the chunk
+        const int ar = tid >> 2, ak = (tid & 3) * 4;
         const float* src[4];
-        float fac[4];
 #pragma unroll
         for (int s2 = 0; s2 < 4; ++s2) {
             const int r = ar + 64 * s2, v = row_id[r];
             src[s2] = nullptr;
-            fac[s2] = 1.0f;
             if (v >= 0) {
                 if (p.a_mode == A_DENSE) src[s2] = p.Hprev + (size_t)(r0 + r) * p.ld_h;
-                else if (p.a_mode == A_SELF) { src[s2] = p.Hprev + (size_t)v * p.ld_h; fac[s2] = p.alpha; }
-                else { src[s2] = p.S + (size_t)v * p.ld_s; fac[s2] = row_scale[r]; }
+                else if (p.a_mode == A_SELF) src[s2] = p.Hprev + (size_t)v * p.ld_h;
+                else src[s2] = p.S + (size_t)v * p.ld_s;
             }
         }
-        float4 a[4], b;
-        auto request = [&](int k0) {
+        auto request = [&](int c) {      // chunk c of A into its stage (beyond K: an empty group keeps the count)
+            if (c < chunks) {
+                float* stage = ring + (size_t)(c % NST) * NBM * NAS_LD;
+                const int k = c * NBK + ak;
 #pragma unroll
-            for (int s2 = 0; s2 < 4; ++s2)
-                a[s2] = (src[s2] && k0 + ak < p.K) ? *reinterpret_cast<const float4*>(src[s2] + k0 + ak)
-                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
-            b = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (bk < NBK && k0 + bk < p.K && 4 * bq < p.n_cols)
-                b = __ldg(reinterpret_cast<const float4*>(p.W + (size_t)(k0 + bk) * p.ldw + 4 * bq));
-        };
-        request(0);
-        for (int k0 = 0; k0 < p.K; k0 += NBK) {
-            __syncthreads();
-#pragma unroll
-            for (int s2 = 0; s2 < 4; ++s2) {
-                const int r = ar + 64 * s2;
-                buf[(ak + 0) * AS_LD + r] = fac[s2] * a[s2].x; buf[(ak + 1) * AS_LD + r] = fac[s2] * a[s2].y;
-                buf[(ak + 2) * AS_LD + r] = fac[s2] * a[s2].z; buf[(ak + 3) * AS_LD + r] = fac[s2] * a[s2].w;
-            }
-            if (bk < NBK) {
-                // column c of the tile lives at Bs[k][8 * (c / 6) + c % 6]
-                const float e[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const int c = 4 * bq + t;
-                    Bs[bk][8 * (c / NTN) + c % NTN] = e[t];
+                for (int s2 = 0; s2 < 4; ++s2) {
+                    const bool ok = src[s2] && k < p.K;
+                    cp_async16_zfill(stage + (ar + 64 * s2) * NAS_LD + ak, ok ? src[s2] + k : p.W, ok);
                 }
             }
-            __syncthreads();
-            if (k0 + NBK < p.K) request(k0 + NBK);
-            const int kmax = min(NBK, p.K - k0);
-#pragma unroll 8
-            for (int k = 0; k < kmax; ++k) {
-                const float4 a0 = *reinterpret_cast<const float4*>(&buf[k * AS_LD + ty * 4]);
-                const float4 a1 = *reinterpret_cast<const float4*>(&buf[k * AS_LD + NBM / 2 + ty * 4]);
-                const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 8]);
-                const float2 b1 = *reinterpret_cast<const float2*>(&Bs[k][tx * 8 + 4]);
-                const float av[NTM] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-                const float bv[NTN] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y};
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        // this thread's piece of a chunk of the weights (192 threads): row bk of the chunk, columns 4 bq .. 4 bq + 3
+        const int bk = tid / (NBN / 4), bq = tid - bk * (NBN / 4);
+        auto load_b = [&](int c) {
+            float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (bk < NBK && c * NBK + bk < p.K && 4 * bq < p.n_cols)
+                b = __ldg(reinterpret_cast<const float4*>(p.W + (size_t)(c * NBK + bk) * p.ldw + 4 * bq));
+            return b;
+        };
+#pragma unroll
+        for (int c = 0; c < NST - 1; ++c) request(c);
+        float4 b = load_b(0);
+        for (int c = 0; c < chunks; ++c) {
+            float* Bc = Bs + (c & 1) * NBK * NBN;
+            if (bk < NBK) *reinterpret_cast<float4*>(Bc + bk * NBN + 4 * bq) = b;
+            asm volatile("cp.async.wait_group %0;" ::"n"(NST - 2) : "memory");   // this thread's pieces of chunk c are in
+            __syncthreads();                  // everyone's are, the weights too; and chunk c - 1 has been multiplied
+            request(c + NST - 1);             // into the stage that chunk c - 1 has left
+            b = load_b(c + 1);
+            const float* stage = ring + (size_t)(c % NST) * NBM * NAS_LD;
+            const int kmax = min(NBK, p.K - c * NBK);      // a multiple of four
+            for (int k = 0; k < kmax; k += 4) {
+                float4 av[NTM];
 #pragma unroll
                 for (int a2 = 0; a2 < NTM; ++a2)
+                    av[a2] = *reinterpret_cast<const float4*>(stage + (a2 * 32 + ty) * NAS_LD + k);
 #pragma unroll
-                    for (int b2 = 0; b2 < NTN; ++b2) acc[a2][b2] = fmaf(av[a2], bv[b2], acc[a2][b2]);
+                for (int kk = 0; kk < 4; ++kk) {
+                    const float2 w0 = *reinterpret_cast<const float2*>(Bc + (k + kk) * NBN + tx * NTN);
+                    const float2 w1 = *reinterpret_cast<const float2*>(Bc + (k + kk) * NBN + tx * NTN + 2);
+                    const float2 w2 = *reinterpret_cast<const float2*>(Bc + (k + kk) * NBN + tx * NTN + 4);
+                    const float bv[NTN] = {w0.x, w0.y, w1.x, w1.y, w2.x, w2.y};
+#pragma unroll
+                    for (int a2 = 0; a2 < NTM; ++a2) {
+                        const float x = kk == 0 ? av[a2].x : kk == 1 ? av[a2].y : kk == 2 ? av[a2].z : av[a2].w;
+#pragma unroll
+                        for (int b2 = 0; b2 < NTN; ++b2) acc[a2][b2] = fmaf(x, bv[b2], acc[a2][b2]);
+                    }
+                }
             }
         }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
         // the finished tile, 128 rows at a time, through shared memory to the epilogue
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             __syncthreads();
 #pragma unroll
-            for (int a2 = 0; a2 < NTM / 2; ++a2)
+            for (int a2 = 0; a2 < NTM / 2; ++a2) {
+                const int r = (half * (NTM / 2) + a2) * 32 + ty;
+                const float f = row_fac[r];
 #pragma unroll
                 for (int b2 = 0; b2 < NTN; ++b2)
-                    buf[(ty * 4 + a2) * CS_LD + tx * NTN + b2] = acc[half * (NTM / 2) + a2][b2];
+                    ring[(a2 * 32 + ty) * NCS_LD + tx * NTN + b2] = f * acc[half * (NTM / 2) + a2][b2];
+            }
             __syncthreads();
             for (int it = tid; it < (NBM / 2) * (NBN / 4); it += 256) {
                 const int lr = it / (NBN / 4), q = it - lr * (NBN / 4);
                 const int r = half * (NBM / 2) + lr, v = row_id[r];
                 if (v < 0 || 4 * q >= p.n_cols) continue;
-                const float4 h = *reinterpret_cast<const float4*>(&buf[lr * CS_LD + 4 * q]);
+                const float4 h = *reinterpret_cast<const float4*>(&ring[lr * NCS_LD + 4 * q]);
                 upd_epilogue4(p, v, r0 + r, 4 * q, h, row_scale[r]);
             }
         }
     }
+}
+
+void narrow_prepare() {
+    cudaFuncSetAttribute(k_update_rows_narrow, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)NARROW_SMEM);
 }
 
 // K = 0: the layer's self projection and transformed aggregate are both cached, so the update is
@@ -334,7 +358,7 @@ static void launch_update(Ctx* c, UpdParams& p, const TcW& tw) {
     p.narrow_min_rows = (p.n_cols <= NBN && p.a_mode != A_SUM && p.tc_mode == TC_OFF && (c->tc_armed || !p.list)) ? NARROW_MIN_ROWS : 0;
     if (c->few_rows_form && p.list) RP_LAUNCH(c, k_update_rows<true>, c->n_sm * 4, 256, 0, c->ctl, p);
     else RP_LAUNCH(c, k_update_rows<false>, c->n_sm * 4, 256, 0, c->ctl, p);
-    if (p.narrow_min_rows) RP_LAUNCH(c, k_update_rows_narrow, c->n_sm * 4, 256, 0, c->ctl, p);
+    if (p.narrow_min_rows) RP_LAUNCH(c, k_update_rows_narrow, c->n_sm * 2, 256, NARROW_SMEM, c->ctl, p);
     if (p.tc_mode != TC_OFF) launch_update_tc(c, p);
 }
 

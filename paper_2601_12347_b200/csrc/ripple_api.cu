@@ -223,6 +223,7 @@ extern "C" ripple_status ripple_create(const ripple_graph* g, const float* featu
             c->gather_min_messages = 1 << 20;
         }
         tc_prepare();
+        narrow_prepare();
         max_prepare();
         CK(cudaMallocHost(&c->ctl_host, sizeof(Ctl)));
         memset(c->ctl_host, 0, sizeof(Ctl));

@@ -358,5 +358,6 @@ void extra_sender_rows(Ctx* c, int l, int n);           // deltas of senders who
 // layer_update_tc.cu
 cudaError_t tc_weights_build(TcW* out, const float* W_host, int K, int ldw);
 void tc_prepare();   // one-time kernel attributes (not allowed inside a stream capture)
+void narrow_prepare();   // likewise, for the update form for narrow outputs
 
 }  // namespace rp

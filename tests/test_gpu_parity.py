@@ -434,6 +434,34 @@ def test_recompute_full_matches_incremental_state(env):
     rp.close()
 
 
+@pytest.mark.parametrize("pre", [True, False], ids=["transform-first", "aggregate-first"])
+@pytest.mark.parametrize("kind", ["sage", "graphconv"])
+def test_narrow_output_layers_over_many_rows(env, kind, pre):
+    """Layers of at most 48 output columns over more than 65 536 rows take an update kernel of their own (here: the
+    whole-graph passes of the sparse graph, and a batch whose last frontier is most of the graph); its operand is a
+    compact row, the vertex's previous row or its scaled aggregate depending on the layer kind and on whether the
+    layer transforms before the scatter.  Widths of 40 and 47 columns."""
+    ripple, Oracle = env
+    w = I.workloads()["sparse"]
+    src, dst = I.make_graph(w)
+    model = I.sage_model([128, 64, 40], I.AGG_MEAN) if kind == "sage" else I.graphconv_model([128, 96, 47], I.AGG_WSUM_GCN)
+    X = I.features(w.n, 128, 5)
+    W = I.make_weights(model, 5, zero_bias=False)
+    rp = ripple.Ripple(w.n, src, dst, X, model, W, pre_transform=pre, max_batch=4096)
+    orc = Oracle(w.n, src, dst, X, model, W)
+    check_values(rp, orc.full(), 2, [None] + [orc.full_S(l) for l in range(1, 3)])
+    stream = I.UpdateStream(w.n, src, dst, 128, 5)
+    for bs in (2000, 2000, 50):
+        ups, rows = stream.next_batch(bs)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows, pull=True) == 0
+        check_frontiers(rp, orc, 2)
+    check_values(rp, orc.full(), 2, [None] + [orc.full_S(l) for l in range(1, 3)])
+    rp.recompute_full()
+    check_values(rp, orc.full(), 2, [None] + [orc.full_S(l) for l in range(1, 3)])
+    rp.close()
+
+
 # ---------------------------------------------------------------------------------------------
 # the named workloads
 # ---------------------------------------------------------------------------------------------
