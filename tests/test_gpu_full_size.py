@@ -309,3 +309,32 @@ def test_full_size_two_workers_of_the_partitioned_execution(env):
           f"halo rows sent in the last batch {sent[1:]}")
     cl.close()
     orc.close()
+
+
+def test_mid_size_every_row_of_every_layer_through_pushed_gathered_and_rebuilt_hops(env):
+    """The 3-layer configuration on the graph of a million vertices, where the oracle's incremental route still
+    follows batches of 1000: after every batch ALL rows of all layers against it (not a sample), hop sets and counters
+    exact.  From the second batch on hop 1 pushes its messages, hop 2 gathers them per sink (wide messages from few
+    senders) and hop 3 rebuilds; the last layer's products run on the update kernel for narrow outputs."""
+    import test_gpu_parity as G
+    ripple, Oracle = env
+    w, (src, dst) = graph_of("mid-3l")
+    X = I.features(w.n, w.model.dims[0], w.seed)
+    W = I.make_weights(w.model, w.seed)
+    L = len(w.model.layers)
+    rp = ripple.Ripple(w.n, src, dst, X, w.model, W, max_batch=1000)
+    orc = Oracle(w.n, src, dst, X, w.model, W)
+    stream = I.make_stream(w, src, dst, 77)
+    worst = 0.0
+    for b, bsz in enumerate([1000, 1000, 300]):
+        ups, rows = stream.next_batch(bsz)
+        rp.apply_batch(ups, rows)
+        assert orc.apply_incremental(ups, rows, pull=True) == 0
+        G.check_frontiers(rp, orc, L)
+        worst = max(worst, G.check_values(rp, [orc.H(l) for l in range(L + 1)], L))
+        if b >= 1:
+            assert list(rp.stats()["scatter_pull"][1:L + 1]) == [0, 1, 2]
+    G.check_graph(rp, orc)
+    print(f"mid-3l, 3 batches, every row of {L + 1} layers: worst err {worst:.2e}")
+    rp.close()
+    orc.close()
