@@ -144,7 +144,8 @@ typedef struct {
  * for this hop only).  AUTO: PUSH, except that a hop whose senders own at least
  * regather_threshold of all edges rebuilds, and that a hop of wide messages (128 floats or more)
  * from few senders gathers per sink (chosen per hop from what the hop carried in the batch before:
- * at least 2^20 messages, eight or more per affected sink, sender rows of at most 32 MiB in all). */
+ * at least 2^20 messages, eight or more per affected sink, sender rows of at most 32 MiB in all;
+ * the environment variable RIPPLE_GATHER_MIN_WIDTH, read by ripple_create, replaces the 128: 0 = never). */
 typedef enum {
     RIPPLE_SCATTER_AUTO = 0, RIPPLE_SCATTER_PUSH = 1, RIPPLE_SCATTER_PULL = 2, RIPPLE_SCATTER_REGATHER = 3,
     RIPPLE_SCATTER_PUSH_BULK = 4 /* PUSH with one bulk reduction of the copy engine per message (cp.reduce.async.bulk)
