@@ -183,8 +183,64 @@ k_att_fold(Ctl* ctl, int l, const int32_t* __restrict__ A, const int* n_dev, int
         const size_t off = (size_t)v * ld;
         float4* s = reinterpret_cast<float4*>(S + off);
         float4* dd = reinterpret_cast<float4*>(dS + off);
+        const bool fast = !all && nq <= 32 && (ld_h & 3) == 0;
+        // (the fast form asks for the row together with the two words that decide whether it is used)
+        float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), y0 = x0, hold0 = x0;
+        float spent0 = 0.f;
+        if (fast) {
+            if (lane < nq) { x0 = s[lane]; y0 = dd[lane]; }
+            if (lane < (ld_h >> 2)) hold0 = reinterpret_cast<const float4*>(H + (size_t)v * ld_h)[lane];
+            if (budget) spent0 = budget[v];
+        }
         bool anew = all || posmap[v] >= 0 || deg_in[v] == 0;   // (no in-neighbour left: exact zeros)
         bool on_budget = false;
+        if (!anew && fast) {
+            // Rows of up to 128 floats: one 16-byte piece per lane, so the row, its accumulator, its budget and the
+            // old embedding are requested together and the new embedding is made from registers.  (A warp works
+            // through its rows one after the other: the loop form below pays five dependent trips to memory per
+            // row, this one two.)
+            const int nqh = ld_h >> 2;
+            float4 x = x0;
+            const float4 y = y0, hold = hold0;
+            float4* hrow4 = reinterpret_cast<float4*>(H + (size_t)v * ld_h);
+            const float spent_before = spent0;
+            float m_old = fmaxf(fmaxf(fabsf(x.x), fabsf(x.y)), fmaxf(fabsf(x.z), fabsf(x.w)));
+            x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
+            float m_new = fmaxf(fmaxf(fabsf(x.x), fabsf(x.y)), fmaxf(fabsf(x.z), fabsf(x.w)));
+            if (lane < nq) { s[lane] = x; dd[lane] = make_float4(0.f, 0.f, 0.f, 0.f); }
+            bool keep = true;
+            if (budget) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    m_old = fmaxf(m_old, __shfl_xor_sync(FULL, m_old, o));
+                    m_new = fmaxf(m_new, __shfl_xor_sync(FULL, m_new, o));
+                }
+                const float m = fmaxf(m_old, m_new);
+                const float spent = spent_before + m * m;
+                const float limit = tau2 * (0.5f + (float)(mix64((uint64_t)v) & 255u) * (1.0f / 512.0f)) * m_new * m_new;
+                keep = !(spent > limit);
+                if (keep && lane == 0) budget[v] = spent;
+            }
+            if (keep) {
+                const int c = d & 3;
+                const float mine = c == 0 ? x.x : c == 1 ? x.y : c == 2 ? x.z : x.w;
+                const float den = __shfl_sync(FULL, mine, d >> 2);
+                if (lane < nqh) {
+                    const float e[4] = {x.x, x.y, x.z, x.w};
+                    float h[4];
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        h[t] = (den > 0.f && 4 * lane + t < d) ? e[t] / den : 0.f;
+                        if (act == RIPPLE_ACT_RELU) h[t] = fmaxf(h[t], 0.f);
+                    }
+                    if (Old) *reinterpret_cast<float4*>(Old + (size_t)i * ld_h + 4 * lane) = hold;
+                    hrow4[lane] = make_float4(h[0], h[1], h[2], h[3]);
+                }
+                continue;
+            }
+            __syncwarp();
+            anew = on_budget = true;
+        }
         if (!anew) {
             float m_old = 0.f, m_new = 0.f;
             for (int q = lane; q < nq; q += 32) {
