@@ -389,7 +389,7 @@ k_scatter_push_bulk(Ctl* ctl, int l, const int32_t* __restrict__ senders, const 
 // ---------------------------------------------------------------------------------------------
 // gathering form of the delta scatter: per affected sink, the delta rows of the senders among its
 // in-neighbours are summed in registers and reach the accumulator row as ONE addition.  The sender
-// delta rows are few (they stay in L2, the hubs' rows in L1) and are read with plain loads; no
+// delta rows are few (they stay in L2) and are read with plain loads; no
 // accumulator row is touched more than once.  It pays where a message is wide: 256-float
 // messages cost the push one kilobyte of read-modify-write each in the L2 slices and evict each
 // other's accumulator rows in between.
